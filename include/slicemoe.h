@@ -1,0 +1,219 @@
+/*
+ * slicemoe.h - C ABI of the B200 (sm_100a) SliceMoE hot path: the MoE expert FFN computed
+ * directly from bit-sliced AMAT weights (arxiv 2512.12990).
+ *
+ * Conventions for every entry point
+ *   - Return value: 0 (SLICEMOE_OK) or a negative SLICEMOE_E_* code; slicemoe_strerror() names it.
+ *     Nothing throws, aborts or prints.  Invalid arguments are rejected on the host before any
+ *     launch; conditions only visible on the device (an out-of-range expert id in a device list, a
+ *     wait that ran out) set bits in the status word of the workspace, see slicemoe_get_status().
+ *   - "device" pointers are CUDA device memory of the current device, owned by the caller, and must
+ *     stay valid until the work enqueued on `stream` has finished.  "host" pointers are ordinary
+ *     host memory.  `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Unless
+ *     stated, calls only enqueue work and do not synchronise.
+ *   - The library allocates no device memory.
+ *   - Weight matrices are row-major [N, K] (N outputs, K inputs = contraction axis); quantisation
+ *     groups run along K.
+ *
+ * Weight format (Section 4.2 of the paper; Table 1 footnote 1: grouped asymmetric integer codes).
+ *   Every weight has an 8-bit code q; every (row, K-group) has an fp16 scale s and a u8 zero-point
+ *   zp.  The code is stored as two 4-bit slice planes: MSB = q >> 4 and LSB = q & 15 (Section 4.1:
+ *   MSB and LSB slices are cached separately).  With both slices the weight is s*(q - zp); from the
+ *   MSB slice alone it is 16*s*((q >> 4) - (zp >> 4)), i.e. the paper's joint truncation of code
+ *   and zero-point with shift = 4.
+ *
+ *   Physical layout of a plane (N % 16 == 0, K % 128 == 0), N*K/2 bytes: rows are grouped in blocks
+ *   of 16 and K in tiles of 64; block (rb, st) is 512 contiguous bytes at ((rb*(K/64) + st)*512),
+ *   made of 32 lanes x 4 little-endian 32-bit words.  Word w of lane L = 4*g + c holds, in nibble
+ *   position p = i + 4*hf (bits 4p..4p+3), the element
+ *        row = 16*rb + g + 8*(i & 1),   k = 64*st + 16*w + 4*c + 2*(i >> 1) + hf
+ *   (i in 0..3, hf in 0..1).  Scales and zero-points are stored as [N/16][K/group][16] (row within
+ *   the block fastest).  slicemoe_unpack_plane / slicemoe_unpack_meta return the canonical
+ *   row-major arrays.
+ */
+#ifndef SLICEMOE_H
+#define SLICEMOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SLICEMOE_OK 0
+#define SLICEMOE_E_INVALID_ARG (-1) /* null pointer, bad size, K % group != 0, k > E, workspace too small ... */
+#define SLICEMOE_E_UNSUPPORTED (-2) /* a format or size this build does not implement */
+#define SLICEMOE_E_CUDA (-3)        /* a CUDA runtime call failed */
+#define SLICEMOE_E_NOMEM (-4)       /* host allocation failed (host-side objects only) */
+
+/* Bits of the device status word (slicemoe_get_status). */
+#define SLICEMOE_STATUS_BAD_EXPERT_ID 1 /* an id in a device list was outside [0, n_experts): skipped */
+#define SLICEMOE_STATUS_WAIT_TIMEOUT 2  /* a bounded device-side wait ran out; the output is invalid */
+
+#define SLICEMOE_MAX_TOP_K 16
+#define SLICEMOE_MAX_SHARED 4
+
+/* One MoE layer's shape. */
+typedef struct slicemoe_shape {
+  int32_t hidden;              /* model width; multiple of 128, <= 4096 */
+  int32_t inter;               /* routed experts' SwiGLU intermediate width; multiple of 128 */
+  int32_t n_experts;           /* routed experts E */
+  int32_t top_k;               /* experts per token k <= SLICEMOE_MAX_TOP_K */
+  int32_t group;               /* quantisation group along K: 32, 64 or 128 */
+  int32_t b_high, b_low;       /* slice configuration; this build implements (8, 4) */
+  int32_t n_shared;            /* always-on shared experts (<= SLICEMOE_MAX_SHARED), run at 8 bits */
+  int32_t shared_inter;        /* their intermediate width; multiple of 128 */
+  int32_t shared_sigmoid_gate; /* 1: shared output is scaled by sigmoid(v . x) */
+} slicemoe_shape;
+
+/* One packed weight matrix; all pointers are device pointers in the physical layout above. */
+typedef struct slicemoe_mat {
+  const void *msb;       /* N*K/2 bytes */
+  const void *lsb;       /* N*K/2 bytes; may be NULL for a matrix that is never run at 8 bits */
+  const uint16_t *scale; /* fp16 bit patterns, N*K/group entries */
+  const uint8_t *zp;     /* N*K/group entries */
+  int32_t N, K;
+} slicemoe_mat;
+
+/* One SwiGLU expert: gate, up [inter, hidden]; down [hidden, inter]. */
+typedef struct slicemoe_expert {
+  slicemoe_mat gate, up, down;
+} slicemoe_expert;
+
+const char *slicemoe_strerror(int code);
+int slicemoe_version(void);
+
+/* ---- sizes ------------------------------------------------------------------------------- */
+size_t slicemoe_plane_bytes(int N, int K);           /* bytes of one slice plane: N*K/2 */
+size_t slicemoe_meta_count(int N, int K, int group); /* number of (scale, zp) entries: N*K/group */
+
+/*
+ * slicemoe_pack - offline preparation of one weight matrix: quantise (Table 1 fn. 1, Section 5.1:
+ * grouped asymmetric codes) and split into MSB / LSB slice planes (Sections 4.1, 4.2).
+ *   W      device, float32 [N, K] row-major (read only)
+ *   msb, lsb, scale, zp   device outputs in the physical layout; sizes from the functions above
+ * Per (row, group), in float32: lo = min(min w, 0), hi = max(max w, 0), s = fp16((hi - lo)/255)
+ * (round to nearest even; a group with hi == lo or s in {0, inf} gets s = 1, zp = 0),
+ * zp = clamp(rint(-lo/s), 0, 255), q = clamp(rint(w/s) + zp, 0, 255) with IEEE division and
+ * round-half-even.  Bit-exact and deterministic.
+ * Errors: INVALID_ARG (null, N % 16, K % 128, K % group), UNSUPPORTED ((b_high,b_low) != (8,4),
+ * group not in {32,64,128}), CUDA.
+ */
+int slicemoe_pack(const float *W, int N, int K, int group, int b_high, int b_low, void *msb,
+                  void *lsb, uint16_t *scale, uint8_t *zp, void *stream);
+
+/* Inverse of the physical layout (test hook and dump helper): nibbles[n*K + k] in 0..15. */
+int slicemoe_unpack_plane(const void *plane, int N, int K, uint8_t *nibbles, void *stream);
+/* scale_rm / zp_rm: row-major [N, K/group]. */
+int slicemoe_unpack_meta(const uint16_t *scale, const uint8_t *zp, int N, int K, int group,
+                         uint16_t *scale_rm, uint8_t *zp_rm, void *stream);
+
+/*
+ * slicemoe_route_topk - top-k gating (Section 1) with an optional cache-priority bias (Section 2.1:
+ * cache-aware routing boosts the gating scores of cached experts) and the precision request of
+ * Section 4.1 (critical experts ask for both slices).
+ *   logits   device float32 [T, E]
+ *   bias     device float32 [E] or NULL; added to the logit in float32 for SELECTION only
+ *   renorm   1: divide the k weights by their sum
+ *   tau, rank_high   precision request: flag 1 (MSB+LSB) iff the expert's softmax probability
+ *            (unbiased, before renormalisation) >= tau or its position in the selection < rank_high;
+ *            pass tau > 1 and rank_high = 0 for "never"
+ *   ids      device int32 [T, k]: experts by descending key; ties -> lower index; NaN logit = -inf
+ *   weights  device float32 [T, k]: softmax(logits)[id]
+ *   prec_req device uint8 [T, k] or NULL
+ * Errors: INVALID_ARG (null, T <= 0, k < 1, k > E, k > SLICEMOE_MAX_TOP_K), UNSUPPORTED (E > 512).
+ */
+int slicemoe_route_topk(const float *logits, int T, int E, int k, const float *bias, int renorm,
+                        float tau, int rank_high, int32_t *ids, float *weights, uint8_t *prec_req,
+                        void *stream);
+
+/*
+ * Workspace.  The FFN kernels need caller-owned device scratch: a header (grid barrier, tickets,
+ * status word), the fp32 intermediate h and per-expert partial outputs.  Allocate
+ * slicemoe_workspace_bytes() bytes (256-byte aligned) and call slicemoe_workspace_init() once
+ * before first use (it zeroes the header; the kernels leave it zeroed again when they finish).
+ * One workspace serves one stream at a time.
+ */
+size_t slicemoe_workspace_bytes(const slicemoe_shape *shape);
+int slicemoe_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
+/* Copies the status word to *status_out (host) and clears it.  Synchronises `stream`. */
+int slicemoe_get_status(void *workspace, int *status_out, void *stream);
+
+/*
+ * slicemoe_expert_ffn - the mixed-precision expert FFN of Section 4.1 over an expert-id/precision
+ * list:   y[t] = sum_j weights[t,j] * Wd_e ( silu(Wg_e x[t]) * (Wu_e x[t]) ),  e = ids[t,j],
+ * each W dequantised from both slices when prec[t,j] = 1 and from the MSB slice alone when 0.
+ *   experts  device array [shape->n_experts] of slicemoe_expert
+ *   x        device bf16 [T, hidden]
+ *   ids, prec, weights   device [T, k] (int32, uint8, float32), k = shape->top_k
+ *   y        device float32 [T, hidden], overwritten
+ * Tokens are processed one after another by the batch-1 decode kernel (weights are streamed once
+ * per token); accumulation is fp32, h stays fp32 between the two projections, the summation
+ * order is fixed (results are bit-reproducible run to run).
+ * Errors: INVALID_ARG, UNSUPPORTED (shape limits above; sum of intermediate widths over the k + n_shared
+ * slots must be <= 12288), CUDA.
+ */
+int slicemoe_expert_ffn(const slicemoe_shape *shape, const slicemoe_expert *experts, const void *x,
+                        int T, const int32_t *ids, const uint8_t *prec, const float *weights,
+                        float *y, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * slicemoe_layer - routed experts as above plus the always-on shared experts of the two evaluated
+ * model architectures (not part of the paper's method): each shared expert runs at 8 bits and is
+ * added with weight 1, or with weight sigmoid(shared_gate_vec . x[t]) when shape->shared_sigmoid_gate.
+ *   shared           device array [shape->n_shared] of slicemoe_expert (inter = shape->shared_inter)
+ *   shared_gate_vec  device float32 [hidden] or NULL (required iff shared_sigmoid_gate)
+ */
+int slicemoe_layer(const slicemoe_shape *shape, const slicemoe_expert *experts,
+                   const slicemoe_expert *shared, const float *shared_gate_vec, const void *x, int T,
+                   const int32_t *ids, const uint8_t *prec, const float *weights, float *y,
+                   void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * slicemoe_decode_step_host - one batch-1 decode step of a layer with HOST inputs and outputs:
+ * copies x (bf16 [hidden]) and logits (float32 [E]) to the device, runs slicemoe_route_topk
+ * (bias/tau/rank_high as there; the precision request is used as the precision list) and
+ * slicemoe_layer, copies y (float32 [hidden]) back and synchronises `stream`.  x_host, logits_host
+ * and y_host should be pinned for the copies to be asynchronous.  Weights stay resident on the
+ * device.  Staging buffers live in the workspace.
+ */
+int slicemoe_decode_step_host(const slicemoe_shape *shape, const slicemoe_expert *experts,
+                              const slicemoe_expert *shared, const float *shared_gate_vec,
+                              const void *x_host, const float *logits_host, const float *bias,
+                              int renorm, float tau, int rank_high, float *y_host, void *workspace,
+                              size_t workspace_bytes, void *stream);
+
+/*
+ * Host-side Dynamic Bit-Sliced Caching bookkeeping (Section 4.1; cache implementation of Section
+ * 5.1).  Pure host code: it only turns (expert id, precision request) lists into the precision
+ * list the FFN runs with, plus hit/miss accounting.  MSB slices: LRU.  LSB slices: lowest priority,
+ * evicted (oldest first) before any MSB slice.  One cache for all layers.  Optional miss budget:
+ * once step >= warmup_steps, while bytes fetched / full-precision bytes of the same requests
+ * exceeds miss_budget, an LSB miss is not fetched and the expert runs MSB-only.
+ */
+typedef struct slicemoe_dbsc slicemoe_dbsc;
+/* miss_budget < 0 disables the budget.  Returns NULL on allocation failure or bad arguments. */
+slicemoe_dbsc *slicemoe_dbsc_create(int64_t capacity_bytes, int64_t msb_bytes, int64_t lsb_bytes,
+                                    double miss_budget, int warmup_steps);
+void slicemoe_dbsc_destroy(slicemoe_dbsc *c);
+/* Serves one selected expert.  Returns the execution precision (1 = MSB+LSB, 0 = MSB only) or a
+ * negative error.  msb_hit / lsb_hit (nullable): 1 hit, 0 miss, -1 (lsb only) not requested.
+ * fetched_bytes (nullable): bytes this request had to fetch. */
+int slicemoe_dbsc_request(slicemoe_dbsc *c, int step, int layer, int expert, int need_lsb,
+                          int *msb_hit, int *lsb_hit, int64_t *fetched_bytes);
+/* Serves n selected experts of one (step, layer) in list order: prec_out[i] for ids[i] with request
+ * prec_req[i].  All host pointers. */
+int slicemoe_dbsc_assign(slicemoe_dbsc *c, int step, int layer, const int32_t *ids,
+                         const uint8_t *prec_req, int n, uint8_t *prec_out);
+#define SLICEMOE_DBSC_NSTATS 12
+/* out[0..11] = requests, msb_hit, msb_miss, lsb_hit, lsb_miss, lsb_skipped, bytes_fetched,
+ * high_exec, low_exec, win_bytes_fetched, win_bytes_full, bytes_used. */
+int slicemoe_dbsc_stats(const slicemoe_dbsc *c, int64_t *out);
+/* 1/0 presence of the two slices of (layer, expert). */
+int slicemoe_dbsc_contains(const slicemoe_dbsc *c, int layer, int expert, int *has_msb, int *has_lsb);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLICEMOE_H */

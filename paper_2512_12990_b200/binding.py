@@ -1,0 +1,326 @@
+"""Thin ctypes binding over libslicemoe.so: argument marshalling only.
+
+Function names and argument order follow include/slicemoe.h.  Device buffers are torch CUDA
+tensors (torch is used for device memory and streams, nothing else); every step of the path
+runs in the library's kernels.  There is no fallback: if the library is missing or a call
+fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import (POINTER, Structure, c_char_p, c_double, c_float, c_int, c_int32, c_int64, c_size_t,
+                    c_uint8, c_uint16, c_void_p)
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libslicemoe.so")
+_lib = None
+
+OK = 0
+E_INVALID_ARG, E_UNSUPPORTED, E_CUDA, E_NOMEM = -1, -2, -3, -4
+STATUS_BAD_EXPERT_ID, STATUS_WAIT_TIMEOUT = 1, 2
+MAX_TOP_K, MAX_SHARED = 16, 4
+DBSC_NSTATS = 12
+DBSC_STAT_NAMES = ("requests", "msb_hit", "msb_miss", "lsb_hit", "lsb_miss", "lsb_skipped", "bytes_fetched",
+                   "high_exec", "low_exec", "win_bytes_fetched", "win_bytes_full", "bytes_used")
+
+# every symbol include/slicemoe.h declares
+EXPORTS = (
+    "slicemoe_strerror", "slicemoe_version", "slicemoe_plane_bytes", "slicemoe_meta_count", "slicemoe_pack",
+    "slicemoe_unpack_plane", "slicemoe_unpack_meta", "slicemoe_route_topk", "slicemoe_workspace_bytes",
+    "slicemoe_workspace_init", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer",
+    "slicemoe_decode_step_host", "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
+    "slicemoe_dbsc_assign", "slicemoe_dbsc_stats", "slicemoe_dbsc_contains",
+)
+
+
+class SliceMoEError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+class Shape(Structure):
+    _fields_ = [("hidden", c_int32), ("inter", c_int32), ("n_experts", c_int32), ("top_k", c_int32),
+                ("group", c_int32), ("b_high", c_int32), ("b_low", c_int32), ("n_shared", c_int32),
+                ("shared_inter", c_int32), ("shared_sigmoid_gate", c_int32)]
+
+
+class Mat(Structure):
+    _fields_ = [("msb", c_void_p), ("lsb", c_void_p), ("scale", c_void_p), ("zp", c_void_p),
+                ("N", c_int32), ("K", c_int32)]
+
+
+class Expert(Structure):
+    _fields_ = [("gate", Mat), ("up", Mat), ("down", Mat)]
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the C-ABI library on first use; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} not found: build it with `python -m paper_2512_12990_b200.build` "
+                          "(there is no fallback path)")
+    L = ctypes.CDLL(_LIB_PATH)
+    L.slicemoe_strerror.restype = c_char_p
+    L.slicemoe_strerror.argtypes = [c_int]
+    L.slicemoe_version.restype = c_int
+    L.slicemoe_plane_bytes.restype = c_size_t
+    L.slicemoe_plane_bytes.argtypes = [c_int, c_int]
+    L.slicemoe_meta_count.restype = c_size_t
+    L.slicemoe_meta_count.argtypes = [c_int, c_int, c_int]
+    L.slicemoe_pack.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p,
+                                c_void_p, c_void_p]
+    L.slicemoe_unpack_plane.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p]
+    L.slicemoe_unpack_meta.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p]
+    L.slicemoe_route_topk.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_int, c_float, c_int, c_void_p,
+                                      c_void_p, c_void_p, c_void_p]
+    L.slicemoe_workspace_bytes.restype = c_size_t
+    L.slicemoe_workspace_bytes.argtypes = [POINTER(Shape)]
+    L.slicemoe_workspace_init.argtypes = [c_void_p, c_size_t, c_void_p]
+    L.slicemoe_get_status.argtypes = [c_void_p, POINTER(c_int), c_void_p]
+    L.slicemoe_expert_ffn.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
+                                      c_void_p, c_void_p, c_size_t, c_void_p]
+    L.slicemoe_layer.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
+                                 c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.slicemoe_decode_step_host.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                            c_void_p, c_int, c_float, c_int, c_void_p, c_void_p, c_size_t,
+                                            c_void_p]
+    L.slicemoe_dbsc_create.restype = c_void_p
+    L.slicemoe_dbsc_create.argtypes = [c_int64, c_int64, c_int64, c_double, c_int]
+    L.slicemoe_dbsc_destroy.restype = None
+    L.slicemoe_dbsc_destroy.argtypes = [c_void_p]
+    L.slicemoe_dbsc_request.argtypes = [c_void_p, c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int),
+                                        POINTER(c_int64)]
+    L.slicemoe_dbsc_assign.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_void_p]
+    L.slicemoe_dbsc_stats.argtypes = [c_void_p, POINTER(c_int64)]
+    L.slicemoe_dbsc_contains.argtypes = [c_void_p, c_int, c_int, POINTER(c_int), POINTER(c_int)]
+    _lib = L
+    return L
+
+
+def strerror(code: int) -> str:
+    return lib().slicemoe_strerror(code).decode()
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != OK:
+        raise SliceMoEError(rc, where)
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return c_void_p(s.cuda_stream)
+
+
+def make_shape(hidden, inter, n_experts, top_k, group, n_shared=0, shared_inter=0, shared_sigmoid_gate=False,
+               b_high=8, b_low=4) -> Shape:
+    return Shape(hidden, inter, n_experts, top_k, group, b_high, b_low, n_shared, shared_inter,
+                 1 if shared_sigmoid_gate else 0)
+
+
+# ---- sizes ---------------------------------------------------------------------------------------
+def slicemoe_plane_bytes(N: int, K: int) -> int:
+    return lib().slicemoe_plane_bytes(N, K)
+
+
+def slicemoe_meta_count(N: int, K: int, group: int) -> int:
+    return lib().slicemoe_meta_count(N, K, group)
+
+
+# ---- pack ----------------------------------------------------------------------------------------
+class PackedMat:
+    """Device buffers of one packed matrix (physical layout) and its Mat descriptor."""
+
+    def __init__(self, N, K, group, msb, lsb, scale, zp):
+        self.N, self.K, self.group = N, K, group
+        self.msb, self.lsb, self.scale, self.zp = msb, lsb, scale, zp
+
+    def desc(self) -> Mat:
+        return Mat(self.msb.data_ptr(), self.lsb.data_ptr() if self.lsb is not None else None,
+                   self.scale.data_ptr(), self.zp.data_ptr(), self.N, self.K)
+
+
+def slicemoe_pack(W, group: int, b_high: int = 8, b_low: int = 4, stream=None, out: PackedMat | None = None) -> PackedMat:
+    """W: CUDA float32 [N, K] contiguous.  Allocates the outputs with torch unless `out` is given."""
+    import torch
+    assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous() and W.dim() == 2
+    N, K = W.shape
+    if out is None:
+        nb = max(int(slicemoe_plane_bytes(N, K)), 1)
+        nm = max(int(slicemoe_meta_count(N, K, group)) if group > 0 else 1, 1)
+        out = PackedMat(N, K, group,
+                        torch.empty(nb, dtype=torch.uint8, device=W.device),
+                        torch.empty(nb, dtype=torch.uint8, device=W.device),
+                        torch.empty(nm, dtype=torch.int16, device=W.device),
+                        torch.empty(nm, dtype=torch.uint8, device=W.device))
+    rc = lib().slicemoe_pack(_ptr(W), N, K, group, b_high, b_low, _ptr(out.msb), _ptr(out.lsb), _ptr(out.scale),
+                             _ptr(out.zp), _stream(stream))
+    _check(rc, "slicemoe_pack")
+    return out
+
+
+def slicemoe_unpack_plane(plane, N: int, K: int, stream=None):
+    import torch
+    out = torch.empty((N, K), dtype=torch.uint8, device=plane.device)
+    _check(lib().slicemoe_unpack_plane(_ptr(plane), N, K, _ptr(out), _stream(stream)), "slicemoe_unpack_plane")
+    return out
+
+
+def slicemoe_unpack_meta(scale, zp, N: int, K: int, group: int, stream=None):
+    """Returns (scale fp16 [N, K/group], zp uint8 [N, K/group]) row-major."""
+    import torch
+    ng = K // group
+    s = torch.empty((N, ng), dtype=torch.float16, device=scale.device)
+    z = torch.empty((N, ng), dtype=torch.uint8, device=scale.device)
+    _check(lib().slicemoe_unpack_meta(_ptr(scale), _ptr(zp), N, K, group, _ptr(s), _ptr(z), _stream(stream)),
+           "slicemoe_unpack_meta")
+    return s, z
+
+
+# ---- route ---------------------------------------------------------------------------------------
+def slicemoe_route_topk(logits, k: int, bias=None, renorm: bool = False, tau: float = 2.0, rank_high: int = 0,
+                        want_prec: bool = True, stream=None):
+    """logits CUDA float32 [T, E].  Returns (ids int32 [T,k], weights float32 [T,k], prec_req uint8 [T,k] | None)."""
+    import torch
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous() and logits.dim() == 2
+    T, E = logits.shape
+    kk = max(k, 1)
+    ids = torch.empty((T, kk), dtype=torch.int32, device=logits.device)
+    w = torch.empty((T, kk), dtype=torch.float32, device=logits.device)
+    pr = torch.empty((T, kk), dtype=torch.uint8, device=logits.device) if want_prec else None
+    rc = lib().slicemoe_route_topk(_ptr(logits), T, E, k, _ptr(bias), 1 if renorm else 0, tau, rank_high,
+                                   _ptr(ids), _ptr(w), _ptr(pr), _stream(stream))
+    _check(rc, "slicemoe_route_topk")
+    return ids, w, pr
+
+
+# ---- workspace -----------------------------------------------------------------------------------
+def slicemoe_workspace_bytes(shape: Shape) -> int:
+    return lib().slicemoe_workspace_bytes(ctypes.byref(shape))
+
+
+def new_workspace(shape: Shape, device="cuda", stream=None):
+    import torch
+    nbytes = slicemoe_workspace_bytes(shape)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    assert ws.data_ptr() % 256 == 0
+    _check(lib().slicemoe_workspace_init(_ptr(ws), nbytes, _stream(stream)), "slicemoe_workspace_init")
+    return ws
+
+
+def slicemoe_get_status(ws, stream=None) -> int:
+    out = c_int(0)
+    _check(lib().slicemoe_get_status(_ptr(ws), ctypes.byref(out), _stream(stream)), "slicemoe_get_status")
+    return out.value
+
+
+# ---- expert tables ---------------------------------------------------------------------------------
+def expert_table(experts, device="cuda"):
+    """experts: list of dict(gate=PackedMat, up=PackedMat, down=PackedMat) -> CUDA uint8 tensor holding the
+    slicemoe_expert array (keep the PackedMats alive as long as the table is used)."""
+    import torch
+    arr = (Expert * len(experts))()
+    for i, e in enumerate(experts):
+        arr[i] = Expert(e["gate"].desc(), e["up"].desc(), e["down"].desc())
+    raw = bytes(arr)
+    host = torch.frombuffer(bytearray(raw), dtype=torch.uint8)
+    return host.to(device)
+
+
+# ---- FFN -----------------------------------------------------------------------------------------
+def slicemoe_expert_ffn(shape: Shape, experts_tbl, x, ids, prec, weights, ws, y=None, stream=None):
+    """x CUDA bf16 [T, hidden]; ids int32, prec uint8, weights float32 [T, k].  Returns y float32 [T, hidden]."""
+    import torch
+    T = x.shape[0]
+    if y is None:
+        y = torch.empty((T, shape.hidden), dtype=torch.float32, device=x.device)
+    rc = lib().slicemoe_expert_ffn(ctypes.byref(shape), _ptr(experts_tbl), _ptr(x), T, _ptr(ids), _ptr(prec),
+                                   _ptr(weights), _ptr(y), _ptr(ws), ws.numel(), _stream(stream))
+    _check(rc, "slicemoe_expert_ffn")
+    return y
+
+
+def slicemoe_layer(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x, ids, prec, weights, ws, y=None,
+                   stream=None):
+    import torch
+    T = x.shape[0]
+    if y is None:
+        y = torch.empty((T, shape.hidden), dtype=torch.float32, device=x.device)
+    rc = lib().slicemoe_layer(ctypes.byref(shape), _ptr(experts_tbl), _ptr(shared_tbl), _ptr(shared_gate_vec),
+                              _ptr(x), T, _ptr(ids), _ptr(prec), _ptr(weights), _ptr(y), _ptr(ws), ws.numel(),
+                              _stream(stream))
+    _check(rc, "slicemoe_layer")
+    return y
+
+
+def slicemoe_decode_step_host(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x_host, logits_host, y_host,
+                              ws, bias=None, renorm=False, tau=2.0, rank_high=0, stream=None):
+    """x_host: pinned CPU bf16 [hidden]; logits_host: pinned CPU float32 [E]; y_host: pinned CPU float32
+    [hidden] (written).  Synchronises the stream."""
+    rc = lib().slicemoe_decode_step_host(ctypes.byref(shape), _ptr(experts_tbl), _ptr(shared_tbl),
+                                         _ptr(shared_gate_vec), c_void_p(x_host.data_ptr()),
+                                         c_void_p(logits_host.data_ptr()), _ptr(bias), 1 if renorm else 0, tau,
+                                         rank_high, c_void_p(y_host.data_ptr()), _ptr(ws), ws.numel(),
+                                         _stream(stream))
+    _check(rc, "slicemoe_decode_step_host")
+    return y_host
+
+
+# ---- host DBSC -------------------------------------------------------------------------------------
+class Dbsc:
+    """Host slice cache (slicemoe_dbsc_*).  No GPU needed."""
+
+    def __init__(self, capacity_bytes: int, msb_bytes: int, lsb_bytes: int, miss_budget: float | None = None,
+                 warmup_steps: int = 10):
+        self._h = lib().slicemoe_dbsc_create(capacity_bytes, msb_bytes, lsb_bytes,
+                                             -1.0 if miss_budget is None else float(miss_budget), warmup_steps)
+        if not self._h:
+            raise SliceMoEError(E_INVALID_ARG, "slicemoe_dbsc_create")
+
+    def close(self):
+        if self._h:
+            lib().slicemoe_dbsc_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def request(self, step: int, layer: int, expert: int, need_lsb: bool):
+        mh, lh, fb = c_int(0), c_int(0), c_int64(0)
+        prec = lib().slicemoe_dbsc_request(self._h, step, layer, expert, 1 if need_lsb else 0, ctypes.byref(mh),
+                                           ctypes.byref(lh), ctypes.byref(fb))
+        if prec < 0:
+            raise SliceMoEError(prec, "slicemoe_dbsc_request")
+        return prec, bool(mh.value), (None if lh.value < 0 else bool(lh.value)), fb.value
+
+    def assign(self, step: int, layer: int, ids, prec_req):
+        """ids: numpy int32 [n]; prec_req: numpy uint8 [n] -> numpy uint8 [n]."""
+        import numpy as np
+        ids = np.ascontiguousarray(ids, dtype=np.int32)
+        prec_req = np.ascontiguousarray(prec_req, dtype=np.uint8)
+        out = np.empty(ids.shape, dtype=np.uint8)
+        rc = lib().slicemoe_dbsc_assign(self._h, step, layer, ids.ctypes.data_as(c_void_p),
+                                        prec_req.ctypes.data_as(c_void_p), ids.size, out.ctypes.data_as(c_void_p))
+        _check(rc, "slicemoe_dbsc_assign")
+        return out
+
+    def stats(self) -> dict:
+        buf = (c_int64 * DBSC_NSTATS)()
+        _check(lib().slicemoe_dbsc_stats(self._h, buf), "slicemoe_dbsc_stats")
+        return dict(zip(DBSC_STAT_NAMES, list(buf)))
+
+    def contains(self, layer: int, expert: int):
+        a, b = c_int(0), c_int(0)
+        _check(lib().slicemoe_dbsc_contains(self._h, layer, expert, ctypes.byref(a), ctypes.byref(b)),
+               "slicemoe_dbsc_contains")
+        return bool(a.value), bool(b.value)

@@ -1,0 +1,183 @@
+// Host-side Dynamic Bit-Sliced Caching bookkeeping (Section 4.1 of the paper).  Plain C++; no CUDA.
+//
+// Two intrusive orderings over cached slices: MSB slices in LRU order, LSB slices in insertion
+// order.  Eviction always drains the LSB queue (oldest first) before touching the MSB list (least
+// recently used first).  Keys are (layer, expert); one cache serves all layers.
+#include <cstdint>
+#include <list>
+#include <new>
+#include <unordered_map>
+
+#include "slicemoe.h"
+
+namespace {
+
+inline uint64_t make_key(int layer, int expert) {
+  return (static_cast<uint64_t>(static_cast<uint32_t>(layer)) << 32) | static_cast<uint32_t>(expert);
+}
+
+struct Queue {
+  std::list<uint64_t> order;  // front = next victim
+  std::unordered_map<uint64_t, std::list<uint64_t>::iterator> where;
+
+  bool has(uint64_t k) const { return where.find(k) != where.end(); }
+  void push_back(uint64_t k) {
+    order.push_back(k);
+    where[k] = std::prev(order.end());
+  }
+  void touch(uint64_t k) {  // move to the most-recently-used end
+    auto it = where.find(k);
+    order.splice(order.end(), order, it->second);
+  }
+  // Removes the first entry that is not `protect`; false if there is none.
+  bool evict_one(uint64_t protect) {
+    for (auto it = order.begin(); it != order.end(); ++it) {
+      if (*it != protect) {
+        where.erase(*it);
+        order.erase(it);
+        return true;
+      }
+    }
+    return false;
+  }
+};
+
+}  // namespace
+
+struct slicemoe_dbsc {
+  int64_t capacity, msb_bytes, lsb_bytes, used;
+  double miss_budget;
+  int warmup_steps;
+  Queue msb, lsb;
+  int64_t requests, msb_hit, msb_miss, lsb_hit, lsb_miss, lsb_skipped, bytes_fetched, high_exec, low_exec,
+      win_fetched, win_full;
+
+  bool make_room(int64_t need, uint64_t protect) {
+    if (need > capacity) return false;
+    while (capacity - used < need) {
+      if (lsb.evict_one(protect)) {
+        used -= lsb_bytes;
+      } else if (msb.evict_one(protect)) {
+        used -= msb_bytes;
+      } else {
+        return false;
+      }
+    }
+    return true;
+  }
+
+  bool over_budget(int step) const {
+    if (miss_budget < 0.0 || step < warmup_steps || win_full <= 0) return false;
+    return static_cast<double>(win_fetched) / static_cast<double>(win_full) > miss_budget;
+  }
+
+  int request(int step, int layer, int expert, bool need_lsb, int* msb_hit_out, int* lsb_hit_out,
+              int64_t* fetched_out) {
+    const uint64_t key = make_key(layer, expert);
+    ++requests;
+    int64_t fetched = 0;
+    int mh, lh = -1, prec = 0;
+    if (msb.has(key)) {
+      msb.touch(key);
+      mh = 1;
+      ++msb_hit;
+    } else {
+      mh = 0;
+      ++msb_miss;
+      fetched += msb_bytes;
+      if (make_room(msb_bytes, key)) {
+        msb.push_back(key);
+        used += msb_bytes;
+      }
+    }
+    if (need_lsb) {
+      if (lsb.has(key)) {
+        lh = 1;
+        ++lsb_hit;
+        prec = 1;
+      } else {
+        lh = 0;
+        if (over_budget(step)) {
+          ++lsb_skipped;
+        } else {
+          ++lsb_miss;
+          fetched += lsb_bytes;
+          prec = 1;
+          if (make_room(lsb_bytes, key)) {
+            lsb.push_back(key);
+            used += lsb_bytes;
+          }
+        }
+      }
+    }
+    bytes_fetched += fetched;
+    if (prec) ++high_exec; else ++low_exec;
+    if (step >= warmup_steps) {
+      win_fetched += fetched;
+      win_full += msb_bytes + lsb_bytes;
+    }
+    if (msb_hit_out) *msb_hit_out = mh;
+    if (lsb_hit_out) *lsb_hit_out = lh;
+    if (fetched_out) *fetched_out = fetched;
+    return prec;
+  }
+};
+
+extern "C" slicemoe_dbsc* slicemoe_dbsc_create(int64_t capacity_bytes, int64_t msb_bytes, int64_t lsb_bytes,
+                                               double miss_budget, int warmup_steps) {
+  if (capacity_bytes < 0 || msb_bytes <= 0 || lsb_bytes <= 0 || warmup_steps < 0) return nullptr;
+  slicemoe_dbsc* c = new (std::nothrow) slicemoe_dbsc();
+  if (!c) return nullptr;
+  c->capacity = capacity_bytes;
+  c->msb_bytes = msb_bytes;
+  c->lsb_bytes = lsb_bytes;
+  c->used = 0;
+  c->miss_budget = miss_budget;
+  c->warmup_steps = warmup_steps;
+  c->requests = c->msb_hit = c->msb_miss = c->lsb_hit = c->lsb_miss = c->lsb_skipped = 0;
+  c->bytes_fetched = c->high_exec = c->low_exec = c->win_fetched = c->win_full = 0;
+  return c;
+}
+
+extern "C" void slicemoe_dbsc_destroy(slicemoe_dbsc* c) { delete c; }
+
+extern "C" int slicemoe_dbsc_request(slicemoe_dbsc* c, int step, int layer, int expert, int need_lsb,
+                                     int* msb_hit, int* lsb_hit, int64_t* fetched_bytes) {
+  if (!c || layer < 0 || expert < 0 || step < 0) return SLICEMOE_E_INVALID_ARG;
+  try {
+    return c->request(step, layer, expert, need_lsb != 0, msb_hit, lsb_hit, fetched_bytes);
+  } catch (...) {
+    return SLICEMOE_E_NOMEM;
+  }
+}
+
+extern "C" int slicemoe_dbsc_assign(slicemoe_dbsc* c, int step, int layer, const int32_t* ids,
+                                    const uint8_t* prec_req, int n, uint8_t* prec_out) {
+  if (!c || !ids || !prec_req || !prec_out || n < 0 || layer < 0 || step < 0) return SLICEMOE_E_INVALID_ARG;
+  for (int i = 0; i < n; ++i)
+    if (ids[i] < 0) return SLICEMOE_E_INVALID_ARG;
+  try {
+    for (int i = 0; i < n; ++i)
+      prec_out[i] = static_cast<uint8_t>(c->request(step, layer, ids[i], prec_req[i] != 0, nullptr, nullptr, nullptr));
+  } catch (...) {
+    return SLICEMOE_E_NOMEM;
+  }
+  return SLICEMOE_OK;
+}
+
+extern "C" int slicemoe_dbsc_stats(const slicemoe_dbsc* c, int64_t* out) {
+  if (!c || !out) return SLICEMOE_E_INVALID_ARG;
+  const int64_t v[SLICEMOE_DBSC_NSTATS] = {c->requests,   c->msb_hit,       c->msb_miss,  c->lsb_hit,
+                                           c->lsb_miss,   c->lsb_skipped,   c->bytes_fetched, c->high_exec,
+                                           c->low_exec,   c->win_fetched,   c->win_full,  c->used};
+  for (int i = 0; i < SLICEMOE_DBSC_NSTATS; ++i) out[i] = v[i];
+  return SLICEMOE_OK;
+}
+
+extern "C" int slicemoe_dbsc_contains(const slicemoe_dbsc* c, int layer, int expert, int* has_msb, int* has_lsb) {
+  if (!c || layer < 0 || expert < 0) return SLICEMOE_E_INVALID_ARG;
+  const uint64_t key = make_key(layer, expert);
+  if (has_msb) *has_msb = c->msb.has(key) ? 1 : 0;
+  if (has_lsb) *has_lsb = c->lsb.has(key) ? 1 : 0;
+  return SLICEMOE_OK;
+}
