@@ -24,12 +24,11 @@
  *
  *   Physical layout of a plane (N % 16 == 0, K % 128 == 0), N*K/2 bytes: rows are grouped in blocks
  *   of 16 and K in tiles of 64; block (rb, st) is 512 contiguous bytes at ((rb*(K/64) + st)*512),
- *   made of 32 lanes x 4 little-endian 32-bit words.  Word w of lane L = 4*g + c holds, in nibble
- *   position p = i + 4*hf (bits 4p..4p+3), the element
- *        row = 16*rb + g + 8*(i & 1),   k = 64*st + 16*w + 4*c + 2*(i >> 1) + hf
- *   (i in 0..3, hf in 0..1).  Scales and zero-points are stored as [N/16][K/group][16] (row within
- *   the block fastest).  slicemoe_unpack_plane / slicemoe_unpack_meta return the canonical
- *   row-major arrays.
+ *   made of 32 lanes x 4 little-endian 32-bit words.  Byte j (bits 8j..8j+7) of word w of lane
+ *   L = 4*g + c holds, for k = 64*st + 16*w + 4*c + j, the element (row 16*rb + g, k) in its low
+ *   nibble and the element (row 16*rb + g + 8, k) in its high nibble.  Scales and zero-points are
+ *   stored as [N/16][K/group][16] (row within the block fastest).  slicemoe_unpack_plane /
+ *   slicemoe_unpack_meta return the canonical row-major arrays.
  */
 #ifndef SLICEMOE_H
 #define SLICEMOE_H

@@ -21,20 +21,23 @@
 namespace slicemoe {
 
 // ---- physical layout of a slice plane (see slicemoe.h) --------------------------------------
-// 32-bit word index of (row-block rb, k-step t = k/16, lane L) in a plane of a matrix with K columns.
-__host__ __device__ inline size_t plane_word_index(int K, int rb, int t, int lane) {
-  return ((size_t)rb * (K >> 6) + (t >> 2)) * 128 + (size_t)lane * 4 + (t & 3);
+// A plane is a sequence of 512-byte blocks, one per (16-row block rb, 64-column tile st), at block index
+// rb * (K / 64) + st.  A block is 32 lanes x 4 little-endian 32-bit words; lane L = 4 * g + c.  Byte j of
+// word w holds the element (row 16 rb + g, k) in its low nibble and (row 16 rb + g + 8, k) in its high
+// nibble, with k = 64 st + 16 w + 4 c + j.  So `word & 0x0f0f0f0f` and `(word >> 4) & 0x0f0f0f0f` are the
+// two row halves of an m16n8k32 integer mma A fragment.
+__host__ __device__ inline size_t plane_word_index(int K, int rb, int st, int lane, int w) {
+  return ((size_t)rb * (K >> 6) + st) * 128 + (size_t)lane * 4 + w;
 }
 
 // Where element (n, k) lives: word index and nibble position within the word.
 __host__ __device__ inline void plane_locate(int K, int n, int k, size_t* word, int* pos) {
   const int rb = n >> 4, r = n & 15;
-  const int g = r & 7, i0 = r >> 3;
-  const int t = k >> 4, kk = k & 15;
-  const int c = kk >> 2, rem = kk & 3;
-  const int i = i0 + 2 * (rem >> 1), hf = rem & 1;
-  *word = plane_word_index(K, rb, t, g * 4 + c);
-  *pos = i + 4 * hf;
+  const int g = r & 7, hi = r >> 3;
+  const int st = k >> 6, kk = k & 63;
+  const int w = kk >> 4, c = (kk & 15) >> 2, j = kk & 3;
+  *word = plane_word_index(K, rb, st, g * 4 + c, w);
+  *pos = 2 * j + hi;
 }
 
 // Index of the (scale, zp) entry of (row n, group g): [N/16][K/group][16].

@@ -1,24 +1,28 @@
 // Batch-1 decode of one MoE layer from bit-sliced AMAT weights (Section 4.1 of the paper: an expert
 // runs from MSB+LSB slices at full precision or from the MSB slice alone), as ONE persistent kernel.
 //
-// The work is a pure weight stream: every plane byte is used once, so the bound is HBM bandwidth.
-// Design:
+// The work is a pure weight stream: every plane byte is used once, so the bound is HBM bandwidth and
+// everything else is arranged so that the stream never stops.
 //   * One CTA per SM.  A producer thread streams 16-row x <=2048-column plane tiles (<=16 KB, one
-//     contiguous run each thanks to the tiled layout) plus their scales / zero-points into an
-//     8-stage shared-memory ring with cp.async.bulk + mbarriers.  The producer never waits for the
-//     gate/up -> down dependency, so down-projection tiles are already in flight while the grid
-//     finishes the first phase.
-//   * 8 consumer warps split the K range of a tile.  Nibbles are turned into bf16 (128 + n) pairs with
-//     one lop3 per two weights (the plane layout stores them in mma fragment order) and multiplied
-//     with the activation vector by mma.sync m16n8k16 (bf16 x bf16 -> fp32): the tensor pipe is used
-//     as a wide FMA unit because the plain ALUs cannot unpack + convert + FMA 2 nibbles per byte at
-//     HBM rate.  The zero-point and the +128 bias are folded out:
-//        sum_k x_k s (q_k - zp) = s (sum_k x_k (q_k + bias) - (bias + zp) sum_{k in group} x_k).
-//     h is split into bf16 hi + lo parts for the down projection, so no activation precision is lost.
-//   * An epilogue warp reduces the 8 per-warp partial rows, applies SwiGLU, writes h (fp32) to the
-//     workspace, takes part in the single grid barrier (bounded spin) and, in the second phase,
-//     performs the weighted top-k combine in a fixed order through a last-arriver ticket per
-//     16-row output block (deterministic; no float atomics).
+//     contiguous run each thanks to the tiled layout) plus their scales / zero-points into a
+//     shared-memory ring with cp.async.bulk + mbarriers.  The producer never waits for the gate/up ->
+//     down dependency, so down-projection tiles are already in flight (up to the whole ring) while
+//     the grid exchanges h.
+//   * Integer arithmetic on the tensor pipe.  The activation vector (x, later h) is converted once to
+//     23-bit fixed point relative to its largest magnitude and split into three balanced base-256
+//     digits (int8).  The digits sit in separate columns of the B operand of mma.sync m16n8k32
+//     (u8 x s8 -> s32); the A operand is the raw nibble plane: the layout stores the two row halves of
+//     a fragment in the low and high nibbles of each byte, so `w & 0x0f0f0f0f` and `(w >> 4) & 0x0f0f0f0f`
+//     are the whole unpack (2 ALU operations per 8 weights).  Sums are exact in int32; MSB and LSB
+//     planes combine as 16 * Cm + Cl.  Scale and zero-point are applied once per (row, group):
+//        sum_k x_k s (q_k - zp) = s (sum_k q_k x_k - zp sum_{k in group} x_k).
+//     The plain ALUs could not unpack + convert + FMA two weights per byte at HBM rate; this costs
+//     about nine instructions per 512 weights.
+//   * Phase 1 (gate/up + SwiGLU): tasks are (expert slot, 16-row block), split over the CTAs by
+//     bytes.  h goes to the workspace in fp32; one bounded grid barrier publishes it.
+//   * Phase 2 (down + weighted combine): a task is a 16-row block of the OUTPUT over ALL slots, so
+//     the top-k combine stays inside the CTA: no atomics, no cross-CTA reduction, fixed summation
+//     order (results are bit-reproducible).
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -27,10 +31,9 @@
 namespace slicemoe {
 
 constexpr int kConsumerWarps = 8;
-constexpr int kProducerWarp = 8;
-constexpr int kEpilogueWarp = 9;
-constexpr int kThreads = 320;
-constexpr int kStages = 8;
+constexpr int kProducerWarp = kConsumerWarps;
+constexpr int kThreads = 32 * (kConsumerWarps + 1);
+constexpr int kStages = 7;
 constexpr int kChunkK = 2048;                              // K columns per ring stage
 constexpr int kPlaneStageBytes = 16 * kChunkK / 2;         // 16384
 constexpr int kScaleStageBytes = 16 * (kChunkK / 32) * 2;  // 2048 (group 32 is the worst case)
@@ -43,16 +46,14 @@ constexpr unsigned long long kWaitCycles = 4000000000ull;  // ~2 s: every device
 
 // ---- workspace --------------------------------------------------------------------------------
 struct WsHeader {
-  unsigned bar_arrive;  // grid barrier: CTAs that finished the gate/up phase
-  unsigned depart;      // CTAs that finished the kernel (the last one re-zeroes the header)
-  unsigned status;      // SLICEMOE_STATUS_* bits
-  unsigned pad[61];
-  unsigned ticket[kMaxHidden / 16];  // per 16-row output block: finished (block, slot) tasks
+  unsigned bar_arrive;        // grid barrier: CTAs that finished the gate/up phase
+  unsigned depart;            // CTAs that finished the kernel (the last one re-zeroes the header)
+  unsigned status;            // SLICEMOE_STATUS_* bits
+  unsigned pad;
+  unsigned hmax[kMaxSlots];   // per slot: bit pattern of max |h| (non-negative floats order as integers)
 };
-constexpr size_t kWsHeaderBytes = sizeof(WsHeader);                     // 1280
-constexpr size_t kWsHOff = 2048;                                        // float h[kHCap]
-constexpr size_t kWsPOff = kWsHOff + sizeof(float) * kHCap;             // float P[kMaxSlots][hidden]
-constexpr size_t kWsStageOff = kWsPOff + sizeof(float) * kMaxSlots * kMaxHidden;
+constexpr size_t kWsHOff = 2048;                              // float h[kHCap]
+constexpr size_t kWsStageOff = kWsHOff + sizeof(float) * kHCap;
 // host-step staging: x bf16[kMaxHidden] | logits f32[512] | ids i32[16] | w f32[16] | prec u8[16] | y f32[kMaxHidden]
 constexpr size_t kWsStX = kWsStageOff;
 constexpr size_t kWsStLogits = kWsStX + 2 * kMaxHidden;
@@ -61,6 +62,7 @@ constexpr size_t kWsStW = kWsStIds + 64;
 constexpr size_t kWsStPrec = kWsStW + 64;
 constexpr size_t kWsStY = kWsStPrec + 64;
 constexpr size_t kWsBytes = kWsStY + 4 * kMaxHidden;
+static_assert(sizeof(WsHeader) <= kWsHOff, "workspace header");
 
 // ---- kernel parameters -------------------------------------------------------------------------
 struct DecodeParams {
@@ -74,7 +76,6 @@ struct DecodeParams {
   float* y;
   WsHeader* ws;
   float* ws_h;
-  float* ws_p;
   int n_experts, n_shared, k;
   int hidden, inter, shared_inter, group;
   int sigmoid_gate;
@@ -85,55 +86,64 @@ struct Slot {
   const uint8_t* lsb[3];
   const uint16_t* sc[3];
   const uint8_t* zp[3];
+  const slicemoe_expert* src;  // where the pointers above come from
   int inter;
   int prec;
   float coef;
-  int hoff;   // offset of this slot's h in the workspace / shared-memory h vector
-  int gated;  // 1: coef is replaced by sigmoid(gate_vec . x)
-  int pad_;
+  int hoff;     // offset of this slot's h in the workspace / in the digit buffer
+  int gated;    // 1: coef is sigmoid(gate_vec . x)
+  float hinv;   // 2^-e of this slot's fixed-point h
 };
 
 struct StageDesc {
   uint32_t flags;
   uint16_t slot, rot;
   uint32_t rb;
-  uint16_t kstep0, nblocks;
+  uint16_t kstep0, nblocks;  // first 32-column step of the chunk within the matrix; 128-column blocks in it
 };
 enum : uint32_t {
   kFlagLsb = 1,           // this stage carries the LSB plane of the chunk (accumulate onto 16 x MSB sums)
   kFlagMeta = 2,          // last plane of the chunk: scales / zero-points are in the stage; fold the chunk
   kFlagLastOfMatrix = 4,  // last chunk of the matrix row block
-  kFlagLastOfTask = 8,    // last matrix of the task: publish partial rows
+  kFlagLastOfTask = 8,    // last matrix of the task: reduce over the warps and write out
   kFlagEnd = 16,          // sentinel, no data
   kFlagPrec8 = 32,
   kFlagPhase2 = 64,
 };
 
 struct Plan {
-  int first_slot[2], first_idx[2], count[2];
+  int first_slot, first_idx, count1;  // phase 1: contiguous run of (slot, row block) tasks
+  int count2;                         // phase 2: output row blocks blockIdx.x, + gridDim.x, ...
   int nslots;
-  int last_slot2;  // last slot this CTA touches in the down phase
+  int htotal;  // sum of the slots' intermediate widths
+  float xinv;  // 2^-e of the fixed-point x
 };
 
 struct SmemLayout {
   // offsets into dynamic shared memory
   static constexpr int ring = 0;
-  static constexpr int hs = ring + kStages * kStageBytes;  // uint4[kHCap/4]
-  static constexpr int xs = hs + kHCap * 4;                // bf16[kMaxHidden]
-  static constexpr int xsum = xs + kMaxHidden * 2;         // float[kMaxHidden/32]
-  static constexpr int hsum = xsum + (kMaxHidden / 32) * 4;  // float[kHCap/32]
-  static constexpr int partial = hsum + (kHCap / 32) * 4;    // float[2][8][16][2]
+  static constexpr int hdig = ring + kStages * kStageBytes;  // int8 [kHCap/32][4 digits][32]
+  static constexpr int xdig = hdig + kHCap * 4;              // int8 [kMaxHidden/32][4][32]
+  static constexpr int xsumw = xdig + kMaxHidden * 4;        // float [kMaxHidden/32][2]: weighted digit sums per group
+  static constexpr int hsumw = xsumw + (kMaxHidden / 32) * 8;  // float [kHCap/32][2]
+  static constexpr int partial = hsumw + (kHCap / 32) * 8;     // float [2][warps][16][2]
   static constexpr int slots = partial + 2 * kConsumerWarps * 16 * 2 * 4;
   static constexpr int desc = slots + kMaxSlots * (int)sizeof(Slot);
-  static constexpr int pinfo = desc + kStages * (int)sizeof(StageDesc);  // uint32[2][4]
-  static constexpr int plan = pinfo + 32;
+  static constexpr int stage_in = desc + kStages * (int)sizeof(StageDesc);  // ids i32[16] | w f32[16] | prec i32[16] | gate f32 | xmax u32
+  static constexpr int plan = stage_in + 4 * (3 * SLICEMOE_MAX_TOP_K + 4);
   static constexpr int bars = (plan + (int)sizeof(Plan) + 15) & ~15;  // uint64 barriers
-  static constexpr int nbars = 2 * kStages + 5;
+  static constexpr int nbars = 2 * kStages + 7;
   static constexpr int dead = bars + nbars * 8;
   static constexpr int total = dead + 16;
 };
 static_assert(SmemLayout::total <= 227 * 1024, "shared memory budget");
 static_assert(sizeof(Slot) % 8 == 0, "slot alignment");
+static_assert(SmemLayout::slots % 8 == 0 && SmemLayout::hdig % 16 == 0 && SmemLayout::xdig % 16 == 0 &&
+                  SmemLayout::desc % 16 == 0,
+              "alignment");
+
+// barrier indices after the 2*kStages ring barriers
+enum { kBarPFull0 = 0, kBarPFull1, kBarPEmpty0, kBarPEmpty1, kBarHxArrive, kBarHxGo, kBarHsReady };
 
 // ---- PTX helpers -------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -182,11 +192,11 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
-__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
   asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
@@ -195,94 +205,164 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
   return v;
 }
 
+// ---- fixed-point activations ---------------------------------------------------------------------
+// 2^e with 2^e * vmax < 2^22 (vmax given as the bit pattern of a non-negative float), and 2^-e: every
+// value then rounds to an integer |X| <= 2^22 whose third balanced base-256 digit fits int8 with room.
+__device__ __forceinline__ void fixed_scale(unsigned vmax_bits, float* scale, float* inv) {
+  int ex = (int)((vmax_bits >> 23) & 0xffu) - 127;  // floor(log2 vmax) for normal numbers
+  int e = 21 - ex;
+  e = max(-100, min(100, e));
+  *scale = __uint_as_float((unsigned)(127 + e) << 23);
+  *inv = __uint_as_float((unsigned)(127 - e) << 23);
+}
+// Four values -> three words of balanced base-256 digits (byte j of word t = digit t of value j).
+__device__ __forceinline__ void to_digits4(const float (&v)[4], float scale, uint32_t (&dw)[3], int (&dsum)[3]) {
+  dw[0] = dw[1] = dw[2] = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    int X = __float2int_rn(v[j] * scale);
+    X = max(-4194304, min(4194304, X));
+    const int d0 = ((X + 128) & 255) - 128;
+    X = (X - d0) >> 8;
+    const int d1 = ((X + 128) & 255) - 128;
+    const int d2 = (X - d1) >> 8;
+    dw[0] |= (uint32_t)(d0 & 255) << (8 * j);
+    dw[1] |= (uint32_t)(d1 & 255) << (8 * j);
+    dw[2] |= (uint32_t)(d2 & 255) << (8 * j);
+    dsum[0] += d0;
+    dsum[1] += d1;
+    dsum[2] += d2;
+  }
+}
+// Byte offset, inside the digit buffer, of digit t of the four values k..k+3 (k % 4 == 0): steps of 32
+// columns, 4 digit rows of 32 bytes (the fourth stays zero), and inside a row the order in which the B
+// fragment of m16n8k32 wants them: (k % 16) / 4 selects the lane quad position, (k % 32) / 16 the register.
+__device__ __forceinline__ int digit_offset(int k, int t) {
+  return (k >> 5) * 128 + t * 32 + ((k >> 2) & 3) * 8 + ((k >> 4) & 1) * 4;
+}
+
 // ---- task enumeration (identical in every role) ---------------------------------------------------
 __device__ __forceinline__ int nchunks_of(int K) { return (K + kChunkK - 1) / kChunkK; }
-// tasks / stages-per-task of a slot in a phase
-__device__ __forceinline__ int slot_ntasks(const Slot& s, int phase, int hidden) {
-  return phase == 0 ? s.inter / 16 : hidden / 16;
-}
-__device__ __forceinline__ int slot_spt(const Slot& s, int phase, int hidden) {
-  const int planes = s.prec ? 2 : 1;
-  return phase == 0 ? 2 * planes * nchunks_of(hidden) : planes * nchunks_of(s.inter);
-}
+// ring stages of one phase-1 task (gate + up of a 16-row block) of a slot
+__device__ __forceinline__ int slot_spt1(const Slot& s, int hidden) { return 2 * (s.prec ? 2 : 1) * nchunks_of(hidden); }
 
-// First task whose cumulative stage offset is >= bound; returns its ordinal, slot and index.
-__device__ void locate_task(const Slot* slots, int nslots, int phase, int hidden, long long bound, int* ord,
-                            int* slot, int* idx) {
-  long long off = 0;
-  int o = 0;
-  for (int j = 0; j < nslots; ++j) {
-    const int nt = slot_ntasks(slots[j], phase, hidden), sp = slot_spt(slots[j], phase, hidden);
-    const long long end = off + (long long)nt * sp;
-    if (bound < end) {
-      long long i = bound <= off ? 0 : (bound - off + sp - 1) / sp;
-      if (i < nt) {
-        *ord = o + (int)i;
-        *slot = j;
-        *idx = (int)i;
-        return;
-      }
-    }
-    off = end;
-    o += nt;
-  }
-  *ord = o;
-  *slot = nslots;
-  *idx = 0;
-}
-
-__device__ __forceinline__ void next_task(const Slot* slots, int phase, int hidden, int& slot, int& idx) {
-  if (++idx >= slot_ntasks(slots[slot], phase, hidden)) {
-    idx = 0;
-    ++slot;
-  }
-}
-
-// ---- consumer: one ring stage ----------------------------------------------------------------------
+// ---- consumer ------------------------------------------------------------------------------------
+// One plane stage: this warp's (up to two) 128-column blocks.  `dig` points at the digit buffer entry
+// of the matrix' first column (x digits in phase 1, the slot's h digits in phase 2).
 template <int G>
-struct Acc {
-  static constexpr int SG = 128 / G;
-  float c[2][SG][4];
-};
-
-template <int G, bool PHASE2>
-__device__ __forceinline__ void consume_blocks(Acc<G>& acc, const uint8_t* stage, int b0, bool v0, int b1, bool v1,
-                                               const uint8_t* bvec /* xs or hs + slot offset, byte pointer */,
-                                               int kstep0, int lane) {
-  constexpr int KS_PER_SG = G / 16;
-  const int c = lane & 3;
+__device__ __forceinline__ void consume_blocks(int (&acc)[2][128 / G][4], const uint8_t* stage, int b0, bool v0, int b1,
+                                               bool v1, const uint8_t* dig, int kstep0, int lane) {
+  const int boff = ((lane >> 2) & 3) * 32 + (lane & 3) * 8;  // digit row = column of B this lane feeds
 #pragma unroll
   for (int u = 0; u < 2; ++u) {
     uint4 w0 = make_uint4(0, 0, 0, 0), w1 = make_uint4(0, 0, 0, 0);
     if (v0) w0 = *reinterpret_cast<const uint4*>(stage + (2 * b0 + u) * 512 + lane * 16);
     if (v1) w1 = *reinterpret_cast<const uint4*>(stage + (2 * b1 + u) * 512 + lane * 16);
-    const uint32_t ww0[4] = {w0.x, w0.y, w0.z, w0.w};
-    const uint32_t ww1[4] = {w1.x, w1.y, w1.z, w1.w};
 #pragma unroll
-    for (int tw = 0; tw < 4; ++tw) {
-      const int sg = (4 * u + tw) / KS_PER_SG;
+    for (int h = 0; h < 2; ++h) {
+      const int s4 = 2 * u + h;         // 32-column step within the 128-column block
+      const int sg = (32 * s4) / G;     // group within the block
 #pragma unroll
       for (int bi = 0; bi < 2; ++bi) {
         const bool valid = bi ? v1 : v0;
         if (!valid) continue;
-        const uint32_t w = bi ? ww1[tw] : ww0[tw];
+        const uint4 w = bi ? w1 : w0;
+        const uint32_t wa = h ? w.z : w.x, wb = h ? w.w : w.y;
         const int b = bi ? b1 : b0;
-        const int kstep = kstep0 + 8 * b + 4 * u + tw;
-        const uint32_t a0 = (w & 0x000f000fu) | 0x43004300u;
-        const uint32_t a1 = ((w >> 4) & 0x000f000fu) | 0x43004300u;
-        const uint32_t a2 = ((w >> 8) & 0x000f000fu) | 0x43004300u;
-        const uint32_t a3 = ((w >> 12) & 0x000f000fu) | 0x43004300u;
-        if (!PHASE2) {
-          const uint2 bv = *reinterpret_cast<const uint2*>(bvec + (kstep * 16 + 4 * c) * 2);
-          mma_bf16(acc.c[bi][sg], a0, a1, a2, a3, bv.x, bv.y);
-        } else {
-          const uint4 hv = *reinterpret_cast<const uint4*>(bvec + (kstep * 16 + 4 * c) * 4);
-          mma_bf16(acc.c[bi][sg], a0, a1, a2, a3, hv.x, hv.y);
-          mma_bf16(acc.c[bi][sg], a0, a1, a2, a3, hv.z, hv.w);
-        }
+        const uint2 bv = *reinterpret_cast<const uint2*>(dig + (kstep0 + 4 * b + s4) * 128 + boff);
+        mma_u8s8(acc[bi][sg], wa & 0x0f0f0f0fu, (wa >> 4) & 0x0f0f0f0fu, wb & 0x0f0f0f0fu, (wb >> 4) & 0x0f0f0f0fu, bv.x,
+                 bv.y);
       }
     }
   }
+}
+
+// All consumer warps: fp32 h (workspace, L2) -> fixed-point digits and weighted digit sums in shared memory.
+template <int G>
+__device__ void load_h_to_smem(const DecodeParams& p, uint8_t* smem, int warp, int lane, int htotal) {
+  Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
+  const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
+  uint8_t* hdig = smem + SmemLayout::hdig;
+  float* hsumw = reinterpret_cast<float*>(smem + SmemLayout::hsumw);
+  constexpr int lanes_per_group = G / 4;    // 8, 16 or 32 consecutive lanes cover one group
+  const int n4 = htotal / 4;                // multiple of 32: every slot width is a multiple of 128
+  constexpr int kMaxIt = (kHCap / 4 + kConsumerWarps * 32 - 1) / (kConsumerWarps * 32);
+  float4 v[kMaxIt];
+#pragma unroll
+  for (int it = 0; it < kMaxIt; ++it) {
+    const int i = (it * kConsumerWarps + warp) * 32 + lane;
+    if (i < n4) v[it] = __ldcg(reinterpret_cast<const float4*>(p.ws_h) + i);
+  }
+  // per-slot scale from the published maxima (every warp computes the few it needs)
+  int slot = 0;
+#pragma unroll
+  for (int it = 0; it < kMaxIt; ++it) {
+    const int i = (it * kConsumerWarps + warp) * 32 + lane;
+    if (i < n4) {  // uniform per warp; a warp's 128 values lie in one slot
+      const int k = 4 * i;
+      while (slot + 1 < plan.nslots && k >= slots[slot + 1].hoff) ++slot;
+      float scale, inv;
+      fixed_scale(__ldcg(&p.ws->hmax[slot]), &scale, &inv);
+      if (k == slots[slot].hoff) slots[slot].hinv = inv;  // first lane of the slot's first warp row
+      const float q[4] = {v[it].x, v[it].y, v[it].z, v[it].w};
+      uint32_t dw[3];
+      int ds[3] = {0, 0, 0};
+      to_digits4(q, scale, dw, ds);
+#pragma unroll
+      for (int t = 0; t < 3; ++t) *reinterpret_cast<uint32_t*>(hdig + digit_offset(k, t)) = dw[t];
+      *reinterpret_cast<uint32_t*>(hdig + digit_offset(k, 3)) = 0u;
+#pragma unroll
+      for (int off = 1; off < lanes_per_group; off <<= 1) {
+        ds[0] += __shfl_xor_sync(0xffffffffu, ds[0], off);
+        ds[1] += __shfl_xor_sync(0xffffffffu, ds[1], off);
+        ds[2] += __shfl_xor_sync(0xffffffffu, ds[2], off);
+      }
+      if ((lane & (lanes_per_group - 1)) == 0) {
+        hsumw[(k / G) * 2 + 0] = (float)ds[0] + 256.f * (float)ds[1];
+        hsumw[(k / G) * 2 + 1] = 65536.f * (float)ds[2];
+      }
+    }
+  }
+}
+
+// The single grid-wide dependency: every CTA has written its rows of h.  Executed by all consumer
+// warps; returns false if a wait ran out.
+template <int G>
+__device__ bool exchange_h(const DecodeParams& p, uint8_t* smem, int warp, int lane, bool need_h, int htotal,
+                           volatile int* dead, unsigned* status, uint32_t xbars) {
+  const uint32_t hx_arrive = xbars + 8 * kBarHxArrive, hx_go = xbars + 8 * kBarHxGo, hs_ready = xbars + 8 * kBarHsReady;
+  __syncwarp();
+  if (lane == 0) mbar_arrive(hx_arrive);  // this warp's h rows are written
+  if (warp == 0) {
+    // the whole warp stays converged while it waits: no lane spins on something another lane must provide
+    if (!mbar_wait(hx_arrive, 0, dead, status)) return false;
+    if (lane == 0) {
+      __threadfence();
+      atomicAdd(&p.ws->bar_arrive, 1u);
+    }
+    __syncwarp();
+    if (need_h) {
+      const long long t0 = clock64();
+      while (ld_acquire_u32(&p.ws->bar_arrive) < gridDim.x) {
+        if (*dead) break;
+        if ((unsigned long long)(clock64() - t0) > kWaitCycles) {
+          *dead = 1;
+          atomicOr(status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
+          break;
+        }
+      }
+      __threadfence();
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(hx_go);
+  }
+  if (!need_h) return true;
+  if (!mbar_wait(hx_go, 0, dead, status)) return false;
+  if (*dead) return false;
+  load_h_to_smem<G>(p, smem, warp, lane, htotal);
+  __syncwarp();
+  if (lane == 0) mbar_arrive(hs_ready);
+  return mbar_wait(hs_ready, 0, dead, status);
 }
 
 template <int G>
@@ -290,37 +370,51 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
   constexpr int SG = 128 / G;
   const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
   const StageDesc* descs = reinterpret_cast<const StageDesc*>(smem + SmemLayout::desc);
-  const float* xsum = reinterpret_cast<const float*>(smem + SmemLayout::xsum);
-  const float* hsum = reinterpret_cast<const float*>(smem + SmemLayout::hsum);
+  const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
+  const float* xsumw = reinterpret_cast<const float*>(smem + SmemLayout::xsumw);
+  const float* hsumw = reinterpret_cast<const float*>(smem + SmemLayout::hsumw);
   float* partial = reinterpret_cast<float*>(smem + SmemLayout::partial);
-  uint32_t* pinfo = reinterpret_cast<uint32_t*>(smem + SmemLayout::pinfo);
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t full0 = bars, empty0 = bars + 8 * kStages, pfull0 = bars + 16 * kStages,
-                 pempty0 = pfull0 + 16, hready = pempty0 + 16;
+  const uint32_t full0 = bars, empty0 = bars + 8 * kStages, xbars = bars + 16 * kStages;
+  const uint32_t pfull0 = xbars + 8 * kBarPFull0, pempty0 = xbars + 8 * kBarPEmpty0;
   unsigned* status = &p.ws->status;
 
+  // The lane folds row r of the 16-row block for the digit columns it holds: lanes with c in {0, 1} take
+  // the accumulators of row g, lanes with c in {2, 3} those of row g + 8; even c holds digits 0 and 1, odd c
+  // digit 2 (and the unused fourth column).
   const int c = lane & 3, g8 = lane >> 2;
-  const int r = g8 + 8 * (c & 1);  // the row of the 16-row block this lane folds in the epilogue
-  Acc<G> acc;
+  const int r = g8 + 8 * (c >> 1);
+  const int cq = c & 1;
+  const float w0 = cq ? 65536.f : 1.f, w1 = cq ? 0.f : 256.f;
+  int acc[2][SG][4];
   float rowacc = 0.f, part0 = 0.f, part1 = 0.f;
-  bool h_ready_seen = false;
+  bool exchanged = false;
   int taskcount = 0;
 
   for (int it = 0;; ++it) {
     const int stage = it % kStages;
     if (!mbar_wait(full0 + 8 * stage, (it / kStages) & 1, dead, status)) return;
-    const StageDesc d = descs[stage];
-    if (d.flags & kFlagEnd) break;
+    const uint4 draw = *reinterpret_cast<const uint4*>(descs + stage);
+    StageDesc d;
+    d.flags = draw.x;
+    d.slot = (uint16_t)(draw.y & 0xffffu);
+    d.rot = (uint16_t)(draw.y >> 16);
+    d.rb = draw.z;
+    d.kstep0 = (uint16_t)(draw.w & 0xffffu);
+    d.nblocks = (uint16_t)(draw.w >> 16);
     const bool phase2 = (d.flags & kFlagPhase2) != 0;
-    if (phase2 && !h_ready_seen) {
-      if (!mbar_wait(hready, 0, dead, status)) return;
-      h_ready_seen = true;
+    if (((d.flags & kFlagEnd) || phase2) && !exchanged) {
+      if (!exchange_h<G>(p, smem, warp, lane, phase2, plan.htotal, dead, status, xbars)) return;
+      exchanged = true;
     }
+    if (d.flags & kFlagEnd) break;
     const Slot& sl = slots[d.slot];
     const uint8_t* stg = smem + SmemLayout::ring + stage * kStageBytes;
-    // blocks (128 columns) of this chunk handled by this warp: b0 and b0 + 8
-    const int b0 = (warp - d.rot) & 7, b1 = b0 + 8;
+    // blocks (128 columns) of this chunk handled by this warp: b0 and b0 + warps
+    int b0 = warp - (int)d.rot;
+    if (b0 < 0) b0 += kConsumerWarps;
+    const int b1 = b0 + kConsumerWarps;
     const bool v0 = b0 < d.nblocks, v1 = b1 < d.nblocks;
     if (!(d.flags & kFlagLsb)) {
 #pragma unroll
@@ -328,24 +422,21 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
 #pragma unroll
         for (int sg = 0; sg < SG; ++sg)
 #pragma unroll
-          for (int q = 0; q < 4; ++q) acc.c[bi][sg][q] = 0.f;
+          for (int q = 0; q < 4; ++q) acc[bi][sg][q] = 0;
     } else {
 #pragma unroll
       for (int bi = 0; bi < 2; ++bi)
 #pragma unroll
         for (int sg = 0; sg < SG; ++sg)
 #pragma unroll
-          for (int q = 0; q < 4; ++q) acc.c[bi][sg][q] *= 16.f;
+          for (int q = 0; q < 4; ++q) acc[bi][sg][q] <<= 4;
     }
-    if (!phase2) {
-      consume_blocks<G, false>(acc, stg, b0, v0, b1, v1, smem + SmemLayout::xs, d.kstep0, lane);
-    } else {
-      consume_blocks<G, true>(acc, stg, b0, v0, b1, v1, smem + SmemLayout::hs + sl.hoff * 4, d.kstep0, lane);
-    }
+    const uint8_t* dig = phase2 ? smem + SmemLayout::hdig + sl.hoff * 4 : smem + SmemLayout::xdig;
+    consume_blocks<G>(acc, stg, b0, v0, b1, v1, dig, d.kstep0, lane);
     if (d.flags & kFlagMeta) {
       const uint16_t* ms = reinterpret_cast<const uint16_t*>(stg + kPlaneStageBytes);
       const uint8_t* mz = stg + kPlaneStageBytes + kScaleStageBytes;
-      const float* xs_sum = phase2 ? hsum + (sl.hoff + d.kstep0 * 16) / G : xsum + (d.kstep0 * 16) / G;
+      const float* sumw = phase2 ? hsumw + ((sl.hoff + d.kstep0 * 32) / G) * 2 : xsumw + ((d.kstep0 * 32) / G) * 2;
       const bool p8 = (d.flags & kFlagPrec8) != 0;
 #pragma unroll
       for (int bi = 0; bi < 2; ++bi) {
@@ -355,38 +446,66 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
 #pragma unroll
         for (int sg = 0; sg < SG; ++sg) {
           const int gl = b * SG + sg;
-          const float cv = (c & 1) ? acc.c[bi][sg][2] : acc.c[bi][sg][0];
+          const int ca = (c >> 1) ? acc[bi][sg][2] : acc[bi][sg][0];
+          const int cb = (c >> 1) ? acc[bi][sg][3] : acc[bi][sg][1];
+          const float t = fmaf((float)cb, w1, (float)ca * w0);
           const float s = __half2float(__ushort_as_half(ms[gl * 16 + r]));
           const int z = mz[gl * 16 + r];
-          const float X = xs_sum[gl];
-          // both slices: s (16 Cm + Cl - (16*128 + 128 + zp) X); MSB only: 16 s (Cm - (128 + (zp >> 4)) X)
-          if (p8) rowacc = fmaf(s, fmaf(-(2176.f + (float)z), X, cv), rowacc);
-          else rowacc = fmaf(16.f * s, fmaf(-(128.f + (float)(z >> 4)), X, cv), rowacc);
+          const float X = sumw[gl * 2 + cq];
+          // both slices: s (16 Cm + Cl - zp X); MSB only: 16 s (Cm - (zp >> 4) X)
+          if (p8) rowacc = fmaf(s, fmaf(-(float)z, X, t), rowacc);
+          else rowacc = fmaf(16.f * s, fmaf(-(float)(z >> 4), X, t), rowacc);
         }
       }
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(empty0 + 8 * stage);
     if (d.flags & kFlagLastOfMatrix) {
-      if (!phase2 && !(d.flags & kFlagLastOfTask)) part0 = rowacc;  // gate
-      else part1 = rowacc;                                            // up, or down
+      rowacc += __shfl_xor_sync(0xffffffffu, rowacc, 1);  // digits 0,1 (even c) + digit 2 (odd c)
+      if (!phase2) {
+        rowacc *= plan.xinv;
+        if (!(d.flags & kFlagLastOfTask)) part0 = rowacc;  // gate
+        else part1 = rowacc;                               // up
+      } else {
+        part1 = fmaf(sl.coef * sl.hinv, rowacc, part1);  // weighted combine over the slots, in slot order
+      }
       rowacc = 0.f;
     }
     if (d.flags & kFlagLastOfTask) {
+      // cross-warp reduction of the K split: warp 0 adds the partial rows in warp order
       const int buf = taskcount & 1;
       if (!mbar_wait(pempty0 + 8 * buf, ((taskcount >> 1) & 1) ^ 1, dead, status)) return;
-      if (c < 2) {
+      if (cq == 0) {
         float* dst = partial + ((buf * kConsumerWarps + warp) * 16 + r) * 2;
         dst[0] = part0;
         dst[1] = part1;
       }
-      if (warp == 0 && lane == 0) {
-        pinfo[buf * 4 + 0] = phase2 ? 1u : 0u;
-        pinfo[buf * 4 + 1] = d.slot;
-        pinfo[buf * 4 + 2] = d.rb;
-      }
       __syncwarp();
       if (lane == 0) mbar_arrive(pfull0 + 8 * buf);
+      if (warp == 0) {
+        if (!mbar_wait(pfull0 + 8 * buf, (taskcount >> 1) & 1, dead, status)) return;
+        float a = 0.f, b = 0.f;
+        if (lane < 16) {
+#pragma unroll
+          for (int w = 0; w < kConsumerWarps; ++w) {
+            const float* src = partial + ((buf * kConsumerWarps + w) * 16 + lane) * 2;
+            a += src[0];
+            b += src[1];
+          }
+        }
+        if (!phase2) {
+          const float h = a / (1.f + expf(-a)) * b;  // silu(gate) * up
+          if (lane < 16) p.ws_h[sl.hoff + d.rb * 16 + lane] = h;
+          float m = lane < 16 ? fabsf(h) : 0.f;
+#pragma unroll
+          for (int off = 8; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+          if (lane == 0 && m == m) atomicMax(&p.ws->hmax[d.slot], __float_as_uint(m));
+        } else if (lane < 16) {
+          p.y[d.rb * 16 + lane] = b;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pempty0 + 8 * buf);
+      }
       ++taskcount;
       part0 = part1 = 0.f;
     }
@@ -394,219 +513,105 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
 }
 
 // ---- producer --------------------------------------------------------------------------------------
+struct ProducerState {
+  int it;
+  int chunk;  // running chunk counter: rotates the warp -> block assignment
+};
+
+// Streams the planes of one (slot, matrix, row block) into the ring.  Returns false if a wait ran out.
+template <int G>
+__device__ __forceinline__ bool produce_matrix(uint8_t* smem, ProducerState& ps, const Slot& s, int slot, int mat, int K,
+                                               int rb, uint32_t base_flags, bool last_matrix, volatile int* dead,
+                                               unsigned* status) {
+  constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
+  uint4* descs = reinterpret_cast<uint4*>(smem + SmemLayout::desc);
+  const uint32_t bars = smem_u32(smem + SmemLayout::bars);
+  const uint32_t full0 = bars, empty0 = bars + 8 * kStages;
+  const uint32_t ring = smem_u32(smem + SmemLayout::ring);
+  const int nplanes = s.prec ? 2 : 1;
+  const uint8_t* pm = s.msb[mat] + (size_t)((unsigned)rb * (unsigned)(K >> 6)) * 512u;
+  const uint8_t* pl_ = s.lsb[mat] + (size_t)((unsigned)rb * (unsigned)(K >> 6)) * 512u;
+  const unsigned mo0 = (unsigned)rb * (unsigned)(K >> LG) * 16u;
+  const uint16_t* psc = s.sc[mat] + mo0;
+  const uint8_t* pzp = s.zp[mat] + mo0;
+  const uint32_t flags0 = base_flags | (s.prec ? kFlagPrec8 : 0u);
+  for (int k0 = 0; k0 < K; k0 += kChunkK) {
+    const int kc = min(kChunkK, K - k0);
+    const bool last_chunk = k0 + kChunkK >= K;
+    for (int pl = 0; pl < nplanes; ++pl) {
+      int stage = ps.it % kStages;
+      if (!mbar_wait(empty0 + 8 * stage, ((ps.it / kStages) & 1) ^ 1, dead, status)) return false;
+      const bool has_meta = (pl == nplanes - 1);
+      uint32_t flags = flags0 | (pl ? kFlagLsb : 0u) | (has_meta ? kFlagMeta : 0u);
+      if (has_meta && last_chunk) flags |= kFlagLastOfMatrix | (last_matrix ? kFlagLastOfTask : 0u);
+      descs[stage] = make_uint4(flags, (uint32_t)slot | ((uint32_t)(ps.chunk % kConsumerWarps) << 16), (uint32_t)rb,
+                                (uint32_t)(k0 >> 5) | ((uint32_t)(kc >> 7) << 16));
+      const uint32_t plane_bytes = (uint32_t)kc * 8u;
+      const uint32_t ngc = (uint32_t)(kc >> LG);
+      const uint32_t bar = full0 + 8 * stage;
+      const uint32_t dst = ring + stage * kStageBytes;
+      mbar_arrive_expect_tx(bar, plane_bytes + (has_meta ? ngc * 48u : 0u));
+      bulk_g2s(dst, (pl ? pl_ : pm) + (size_t)k0 * 8u, plane_bytes, bar);
+      if (has_meta) {
+        const unsigned mo = (unsigned)(k0 >> LG) * 16u;
+        bulk_g2s(dst + kPlaneStageBytes, psc + mo, ngc * 32u, bar);
+        bulk_g2s(dst + kPlaneStageBytes + kScaleStageBytes, pzp + mo, ngc * 16u, bar);
+      }
+      ++ps.it;
+    }
+    ++ps.chunk;
+  }
+  return true;
+}
+
+template <int G>
 __device__ void producer_loop(const DecodeParams& p, uint8_t* smem) {
   const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
-  StageDesc* descs = reinterpret_cast<StageDesc*>(smem + SmemLayout::desc);
+  uint4* descs = reinterpret_cast<uint4*>(smem + SmemLayout::desc);
   const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
   const uint32_t full0 = bars, empty0 = bars + 8 * kStages;
-  const uint32_t ring = smem_u32(smem + SmemLayout::ring);
   unsigned* status = &p.ws->status;
-  const int G = p.group;
-  int it = 0;
+  ProducerState ps;
+  ps.it = 0;
+  ps.chunk = 0;
   bool ok = true;
-  for (int phase = 0; phase < 2 && ok; ++phase) {
-    int slot = plan.first_slot[phase], idx = plan.first_idx[phase];
-    for (int n = 0; n < plan.count[phase] && ok; ++n) {
+  // phase 1: gate and up of (slot, row block) tasks
+  {
+    int slot = plan.first_slot, idx = plan.first_idx;
+    for (int n = 0; n < plan.count1 && ok; ++n) {
       const Slot& s = slots[slot];
-      const int K = phase == 0 ? p.hidden : s.inter;
-      const int nch = nchunks_of(K);
-      const int nmat = phase == 0 ? 2 : 1;
-      const int nplanes = s.prec ? 2 : 1;
-      for (int m = 0; m < nmat && ok; ++m) {
-        const int mat = phase == 0 ? m : 2;
-        for (int ch = 0; ch < nch && ok; ++ch) {
-          const int k0 = ch * kChunkK;
-          const int kc = min(kChunkK, K - k0);
-          for (int pl = 0; pl < nplanes; ++pl) {
-            const int stage = it % kStages;
-            if (!mbar_wait(empty0 + 8 * stage, ((it / kStages) & 1) ^ 1, dead, status)) {
-              ok = false;
-              break;
-            }
-            const bool has_meta = (pl == nplanes - 1);
-            StageDesc d;
-            d.flags = (pl ? kFlagLsb : 0u) | (has_meta ? kFlagMeta : 0u) | (s.prec ? kFlagPrec8 : 0u) |
-                      (phase ? kFlagPhase2 : 0u);
-            if (has_meta && ch == nch - 1) {
-              d.flags |= kFlagLastOfMatrix;
-              if (m == nmat - 1) d.flags |= kFlagLastOfTask;
-            }
-            d.slot = (uint16_t)slot;
-            d.rot = (uint16_t)(n & 7);
-            d.rb = (uint32_t)idx;
-            d.kstep0 = (uint16_t)(k0 / 16);
-            d.nblocks = (uint16_t)(kc / 128);
-            descs[stage] = d;
-            const uint32_t plane_bytes = (uint32_t)kc * 8u;
-            const uint32_t ngc = (uint32_t)(kc / G);
-            const uint32_t bytes = plane_bytes + (has_meta ? ngc * 48u : 0u);
-            const uint32_t bar = full0 + 8 * stage;
-            const uint32_t dst = ring + stage * kStageBytes;
-            mbar_arrive_expect_tx(bar, bytes);
-            const uint8_t* plane = pl ? s.lsb[mat] : s.msb[mat];
-            bulk_g2s(dst, plane + ((size_t)idx * (K >> 6) + (k0 >> 6)) * 512, plane_bytes, bar);
-            if (has_meta) {
-              const size_t mo = ((size_t)idx * (K / G) + (k0 / G)) * 16;
-              bulk_g2s(dst + kPlaneStageBytes, s.sc[mat] + mo, ngc * 32u, bar);
-              bulk_g2s(dst + kPlaneStageBytes + kScaleStageBytes, s.zp[mat] + mo, ngc * 16u, bar);
-            }
-            ++it;
-          }
-        }
+      ok = produce_matrix<G>(smem, ps, s, slot, 0, p.hidden, idx, 0u, false, dead, status) &&
+           produce_matrix<G>(smem, ps, s, slot, 1, p.hidden, idx, 0u, true, dead, status);
+      if (++idx >= s.inter / 16) {
+        idx = 0;
+        ++slot;
       }
-      next_task(slots, phase, p.hidden, slot, idx);
     }
   }
+  // phase 2: down rows of every slot for the output row blocks of this CTA
+  for (int n = 0; n < plan.count2 && ok; ++n) {
+    const int rb = blockIdx.x + n * gridDim.x;
+    for (int slot = 0; slot < plan.nslots && ok; ++slot)
+      ok = produce_matrix<G>(smem, ps, slots[slot], slot, 2, slots[slot].inter, rb, kFlagPhase2, slot == plan.nslots - 1,
+                             dead, status);
+  }
   if (ok) {
-    const int stage = it % kStages;
-    if (mbar_wait(empty0 + 8 * stage, ((it / kStages) & 1) ^ 1, dead, status)) {
-      StageDesc d;
-      d.flags = kFlagEnd;
-      d.slot = d.rot = 0;
-      d.rb = 0;
-      d.kstep0 = d.nblocks = 0;
-      descs[stage] = d;
+    const int stage = ps.it % kStages;
+    if (mbar_wait(empty0 + 8 * stage, ((ps.it / kStages) & 1) ^ 1, dead, status)) {
+      descs[stage] = make_uint4(kFlagEnd, 0u, 0u, 0u);
       mbar_arrive(full0 + 8 * stage);
-      ++it;
+      ++ps.it;
     }
   }
   // Never leave the CTA with bulk copies still landing in its shared memory: wait (bounded) for the
   // last kStages armed barriers.  In the normal path they have all completed long ago.
-  for (int j = max(0, it - kStages); j < it; ++j) {
+  for (int j = max(0, ps.it - kStages); j < ps.it; ++j) {
     const uint32_t bar = full0 + 8 * (j % kStages);
     const long long t0 = clock64();
     while (!mbar_try(bar, (j / kStages) & 1)) {
       if ((unsigned long long)(clock64() - t0) > kWaitCycles) break;
-    }
-  }
-}
-
-// ---- epilogue warp ---------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-  return *reinterpret_cast<const uint32_t*>(&v);
-}
-
-__device__ void load_h_to_smem(const DecodeParams& p, uint8_t* smem, int lane, int slot_lo, int slot_hi) {
-  const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
-  uint4* hs = reinterpret_cast<uint4*>(smem + SmemLayout::hs);
-  float* hsum = reinterpret_cast<float*>(smem + SmemLayout::hsum);
-  const int lanes_per_group = p.group / 4;  // 8, 16 or 32 consecutive lanes cover one group
-  for (int j = slot_lo; j <= slot_hi; ++j) {
-    const int hoff = slots[j].hoff, n4 = slots[j].inter / 4;
-    for (int i = lane; i < n4; i += 32) {
-      const float4 v = __ldcg(reinterpret_cast<const float4*>(p.ws_h + hoff) + i);
-      const __nv_bfloat16 h0 = __float2bfloat16_rn(v.x), h1 = __float2bfloat16_rn(v.y),
-                          h2 = __float2bfloat16_rn(v.z), h3 = __float2bfloat16_rn(v.w);
-      const float f0 = __bfloat162float(h0), f1 = __bfloat162float(h1), f2 = __bfloat162float(h2),
-                  f3 = __bfloat162float(h3);
-      const float l0 = v.x - f0, l1 = v.y - f1, l2 = v.z - f2, l3 = v.w - f3;
-      const __nv_bfloat16 g0 = __float2bfloat16_rn(l0), g1 = __float2bfloat16_rn(l1),
-                          g2 = __float2bfloat16_rn(l2), g3 = __float2bfloat16_rn(l3);
-      uint4 o;
-      o.x = pack_bf16x2(f0, f1);
-      o.y = pack_bf16x2(f2, f3);
-      o.z = pack_bf16x2(l0, l1);
-      o.w = pack_bf16x2(l2, l3);
-      hs[hoff / 4 + i] = o;
-      // group sum of what the tensor cores will actually multiply: hi + lo
-      float ssum = (f0 + __bfloat162float(g0)) + (f1 + __bfloat162float(g1)) + (f2 + __bfloat162float(g2)) +
-                   (f3 + __bfloat162float(g3));
-      for (int off = 1; off < lanes_per_group; off <<= 1) ssum += __shfl_xor_sync(0xffffffffu, ssum, off);
-      if ((lane & (lanes_per_group - 1)) == 0) hsum[(hoff + 4 * i) / p.group] = ssum;
-    }
-  }
-}
-
-__device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
-  Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
-  const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
-  const float* partial = reinterpret_cast<const float*>(smem + SmemLayout::partial);
-  const uint32_t* pinfo = reinterpret_cast<const uint32_t*>(smem + SmemLayout::pinfo);
-  volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
-  const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t pfull0 = bars + 16 * kStages, pempty0 = pfull0 + 16, hready = pempty0 + 16;
-  unsigned* status = &p.ws->status;
-  const int nslots = plan.nslots;
-
-  // Qwen-style shared-expert gate: sigmoid(v . x), needed only for the final combine.
-  if (p.sigmoid_gate && p.n_shared > 0) {
-    const __nv_bfloat16* xs = reinterpret_cast<const __nv_bfloat16*>(smem + SmemLayout::xs);
-    float dot = 0.f;
-    for (int i = lane; i < p.hidden; i += 32) dot = fmaf(p.gate_vec[i], __bfloat162float(xs[i]), dot);
-    for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
-    const float cgate = 1.f / (1.f + expf(-dot));
-    if (lane == 0)
-      for (int j = 0; j < nslots; ++j)
-        if (slots[j].gated) slots[j].coef = cgate;
-    __syncwarp();
-  }
-
-  const int total = plan.count[0] + plan.count[1];
-  for (int tc = 0;; ++tc) {
-    if (tc == plan.count[0]) {
-      // ---- grid barrier: every CTA has written its part of h ----
-      __threadfence();
-      __syncwarp();
-      if (lane == 0) {
-        atomicAdd(&p.ws->bar_arrive, 1u);
-        const long long t0 = clock64();
-        while (ld_acquire_u32(&p.ws->bar_arrive) < gridDim.x) {
-          __nanosleep(64);
-          if (*dead) break;
-          if ((unsigned long long)(clock64() - t0) > kWaitCycles) {
-            *dead = 1;
-            atomicOr(status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
-            break;
-          }
-        }
-      }
-      __syncwarp();
-      if (*dead) return;
-      if (plan.count[1] > 0) load_h_to_smem(p, smem, lane, plan.first_slot[1], plan.last_slot2);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(hready);
-    }
-    if (tc == total) break;
-    const int buf = tc & 1;
-    if (!mbar_wait(pfull0 + 8 * buf, (tc >> 1) & 1, dead, status)) return;
-    const uint32_t phase2 = pinfo[buf * 4 + 0], slot = pinfo[buf * 4 + 1], rb = pinfo[buf * 4 + 2];
-    float a = 0.f, b = 0.f;
-    if (lane < 16) {
-#pragma unroll
-      for (int w = 0; w < kConsumerWarps; ++w) {
-        const float* src = partial + ((buf * kConsumerWarps + w) * 16 + lane) * 2;
-        a += src[0];
-        b += src[1];
-      }
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(pempty0 + 8 * buf);
-    if (!phase2) {
-      if (lane < 16) {
-        const float h = a / (1.f + expf(-a)) * b;  // silu(gate) * up
-        p.ws_h[slots[slot].hoff + rb * 16 + lane] = h;
-      }
-    } else {
-      if (lane < 16) p.ws_p[(size_t)slot * p.hidden + rb * 16 + lane] = b;
-      __threadfence();
-      __syncwarp();
-      unsigned ticket = 0;
-      if (lane == 0) ticket = atomicAdd(&p.ws->ticket[rb], 1u);
-      ticket = __shfl_sync(0xffffffffu, ticket, 0);
-      if (ticket == (unsigned)(nslots - 1)) {
-        // last (block, slot) task of this output block: weighted combine in slot order
-        __threadfence();
-        if (lane < 16) {
-          float yv = 0.f;
-          for (int j = 0; j < nslots; ++j)
-            yv = fmaf(slots[j].coef, __ldcg(p.ws_p + (size_t)j * p.hidden + rb * 16 + lane), yv);
-          p.y[rb * 16 + lane] = yv;
-        }
-        if (lane == 0) p.ws->ticket[rb] = 0;
-      }
     }
   }
 }
@@ -619,109 +624,228 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
   Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
   Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
   int* dead = reinterpret_cast<int*>(smem + SmemLayout::dead);
+  int32_t* in_ids = reinterpret_cast<int32_t*>(smem + SmemLayout::stage_in);
+  float* in_w = reinterpret_cast<float*>(in_ids + SLICEMOE_MAX_TOP_K);
+  int32_t* in_prec = reinterpret_cast<int32_t*>(in_w + SLICEMOE_MAX_TOP_K);
+  float* in_gate = reinterpret_cast<float*>(in_prec + SLICEMOE_MAX_TOP_K);
+  unsigned* in_xmax = reinterpret_cast<unsigned*>(in_gate + 1);
 
-  // x -> shared memory (bf16, as is)
-  {
-    const uint32_t* src = reinterpret_cast<const uint32_t*>(p.x);
-    uint32_t* dst = reinterpret_cast<uint32_t*>(smem + SmemLayout::xs);
-    for (int i = tid; i < p.hidden / 2; i += kThreads) dst[i] = src[i];
+  // ---- step 1: every independent global read at once: x (kept in registers), the routing list ----
+  // thread t owns x[4t .. 4t+3] (and 4(t + kThreads) ...): hidden <= kMaxHidden = 4 * 4 * kThreads is checked on the host
+  constexpr int kXIt = (kMaxHidden / 4 + kThreads - 1) / kThreads;
+  float xv[kXIt][4];
+  float xmax = 0.f;
+#pragma unroll
+  for (int it = 0; it < kXIt; ++it) {
+    const int i = it * kThreads + tid;
+    if (4 * i < p.hidden) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(p.x + 4 * i);
+      xv[it][0] = __uint_as_float(raw.x << 16);
+      xv[it][1] = __uint_as_float(raw.x & 0xffff0000u);
+      xv[it][2] = __uint_as_float(raw.y << 16);
+      xv[it][3] = __uint_as_float(raw.y & 0xffff0000u);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float a = fabsf(xv[it][j]);
+        if (a == a) xmax = fmaxf(xmax, a);
+      }
+    }
   }
-  if (tid == 0) {
+  if (tid < p.k) {
+    in_ids[tid] = p.ids[tid];
+    in_w[tid] = p.weights[tid];
+    in_prec[tid] = p.prec[tid];
+  }
+  if (tid == kThreads - 1) {
     *dead = 0;
-    // slot table: routed experts in list order, then the shared experts
+    *in_xmax = 0u;
+    const uint32_t bars = smem_u32(smem + SmemLayout::bars);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bars + 8 * s, 1);                             // full: producer's expect_tx arrive
+      mbar_init(bars + 8 * kStages + 8 * s, kConsumerWarps);  // empty: one arrive per consumer warp
+    }
+    const uint32_t xbars = bars + 16 * kStages;
+    mbar_init(xbars + 8 * kBarPFull0, kConsumerWarps);
+    mbar_init(xbars + 8 * kBarPFull1, kConsumerWarps);
+    mbar_init(xbars + 8 * kBarPEmpty0, 1);
+    mbar_init(xbars + 8 * kBarPEmpty1, 1);
+    mbar_init(xbars + 8 * kBarHxArrive, kConsumerWarps);
+    mbar_init(xbars + 8 * kBarHxGo, 1);
+    mbar_init(xbars + 8 * kBarHsReady, kConsumerWarps);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) xmax = fmaxf(xmax, __shfl_xor_sync(0xffffffffu, xmax, off));
+  if (lane == 0) atomicMax(in_xmax, __float_as_uint(xmax));
+
+  // ---- step 2: slot list (thread 0); the shared-expert gate (last warp) ----
+  if (tid == 0) {
     int n = 0, hoff = 0;
     for (int j = 0; j < p.k; ++j) {
-      const int e = p.ids[j];
+      const int e = in_ids[j];
       if (e < 0 || e >= p.n_experts) {
         atomicOr(&p.ws->status, (unsigned)SLICEMOE_STATUS_BAD_EXPERT_ID);
         continue;
       }
-      const slicemoe_expert& ex = p.experts[e];
       Slot& s = slots[n];
-      const slicemoe_mat* m[3] = {&ex.gate, &ex.up, &ex.down};
-      for (int q = 0; q < 3; ++q) {
-        s.msb[q] = reinterpret_cast<const uint8_t*>(m[q]->msb);
-        s.lsb[q] = reinterpret_cast<const uint8_t*>(m[q]->lsb);
-        s.sc[q] = m[q]->scale;
-        s.zp[q] = m[q]->zp;
-      }
+      s.src = p.experts + e;
       s.inter = p.inter;
-      s.prec = (p.prec[j] != 0 && s.lsb[0] && s.lsb[1] && s.lsb[2]) ? 1 : 0;
-      s.coef = p.weights[j];
+      s.prec = in_prec[j] != 0;
+      s.coef = in_w[j];
       s.gated = 0;
       s.hoff = hoff;
+      s.hinv = 0.f;
       hoff += p.inter;
       ++n;
     }
     for (int j = 0; j < p.n_shared; ++j) {
-      const slicemoe_expert& ex = p.shared[j];
       Slot& s = slots[n];
-      const slicemoe_mat* m[3] = {&ex.gate, &ex.up, &ex.down};
-      for (int q = 0; q < 3; ++q) {
-        s.msb[q] = reinterpret_cast<const uint8_t*>(m[q]->msb);
-        s.lsb[q] = reinterpret_cast<const uint8_t*>(m[q]->lsb);
-        s.sc[q] = m[q]->scale;
-        s.zp[q] = m[q]->zp;
-      }
+      s.src = p.shared + j;
       s.inter = p.shared_inter;
       s.prec = 1;
       s.coef = 1.f;
       s.gated = p.sigmoid_gate;
       s.hoff = hoff;
+      s.hinv = 0.f;
       hoff += p.shared_inter;
       ++n;
     }
     plan->nslots = n;
-    // static partition: equal shares of ring stages per phase, at task granularity
-    for (int phase = 0; phase < 2; ++phase) {
-      long long S = 0;
-      for (int j = 0; j < n; ++j) S += (long long)slot_ntasks(slots[j], phase, p.hidden) * slot_spt(slots[j], phase, p.hidden);
-      const long long lo = ((long long)blockIdx.x * S + gridDim.x - 1) / gridDim.x;
-      const long long hi = ((long long)(blockIdx.x + 1) * S + gridDim.x - 1) / gridDim.x;
-      int o0, s0, i0, o1, s1, i1;
-      locate_task(slots, n, phase, p.hidden, lo, &o0, &s0, &i0);
-      locate_task(slots, n, phase, p.hidden, hi, &o1, &s1, &i1);
-      plan->first_slot[phase] = s0;
-      plan->first_idx[phase] = i0;
-      plan->count[phase] = o1 - o0;
-      if (phase == 1) plan->last_slot2 = (i1 == 0) ? s1 - 1 : s1;
+    plan->htotal = hoff;
+  } else if (warp == kProducerWarp && p.sigmoid_gate && p.n_shared > 0) {
+    // Qwen-style shared-expert gate: sigmoid(v . x)
+    float dot = 0.f;
+    for (int i = lane; i < p.hidden / 2; i += 32) {
+      const uint32_t raw = *reinterpret_cast<const uint32_t*>(p.x + 2 * i);
+      const float2 gv = __ldg(reinterpret_cast<const float2*>(p.gate_vec) + i);
+      dot = fmaf(gv.x, __uint_as_float(raw << 16), dot);
+      dot = fmaf(gv.y, __uint_as_float(raw & 0xffff0000u), dot);
     }
-    if (plan->last_slot2 >= n) plan->last_slot2 = n - 1;
-    // barriers
-    const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(bars + 8 * s, 1);                              // full: producer's expect_tx arrive
-      mbar_init(bars + 8 * kStages + 8 * s, kConsumerWarps);   // empty: one arrive per consumer warp
-    }
-    mbar_init(bars + 16 * kStages + 0, kConsumerWarps);  // pfull[0]
-    mbar_init(bars + 16 * kStages + 8, kConsumerWarps);  // pfull[1]
-    mbar_init(bars + 16 * kStages + 16, 1);              // pempty[0]
-    mbar_init(bars + 16 * kStages + 24, 1);              // pempty[1]
-    mbar_init(bars + 16 * kStages + 32, 1);              // hready
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    if (lane == 0) *in_gate = 1.f / (1.f + expf(-dot));
   }
   __syncthreads();
-  // group sums of x
+
+  // ---- step 3: the slots' plane pointers, one 8-byte load per thread; x -> fixed-point digits ----
+  const int nslots = plan->nslots;
+  for (int i = tid; i < nslots * 12; i += kThreads) {
+    const int s = i / 12, q = i % 12, m = q >> 2, f = q & 3;
+    const slicemoe_mat* mat = reinterpret_cast<const slicemoe_mat*>(slots[s].src) + m;
+    const void* ptr = *(reinterpret_cast<const void* const*>(mat) + f);
+    if (f == 0) slots[s].msb[m] = reinterpret_cast<const uint8_t*>(ptr);
+    else if (f == 1) slots[s].lsb[m] = reinterpret_cast<const uint8_t*>(ptr);
+    else if (f == 2) slots[s].sc[m] = reinterpret_cast<const uint16_t*>(ptr);
+    else slots[s].zp[m] = reinterpret_cast<const uint8_t*>(ptr);
+  }
   {
-    const __nv_bfloat16* xs = reinterpret_cast<const __nv_bfloat16*>(smem + SmemLayout::xs);
-    float* xsum = reinterpret_cast<float*>(smem + SmemLayout::xsum);
-    for (int g = tid; g < p.hidden / G; g += kThreads) {
-      float s = 0.f;
-      for (int i = 0; i < G; ++i) s += __bfloat162float(xs[g * G + i]);
-      xsum[g] = s;
+    float xscale, xinv;
+    fixed_scale(*in_xmax, &xscale, &xinv);
+    if (tid == 0) plan->xinv = xinv;
+    uint8_t* xdig = smem + SmemLayout::xdig;
+    float* xsumw = reinterpret_cast<float*>(smem + SmemLayout::xsumw);
+    constexpr int lanes_per_group = G / 4;
+#pragma unroll
+    for (int it = 0; it < kXIt; ++it) {
+      const int i = it * kThreads + tid;
+      if (4 * (it * kThreads + (tid & ~31)) < p.hidden) {  // uniform per warp (hidden % 128 == 0)
+        const int k = 4 * i;
+        uint32_t dw[3];
+        int ds[3] = {0, 0, 0};
+        to_digits4(xv[it], xscale, dw, ds);
+#pragma unroll
+        for (int t = 0; t < 3; ++t) *reinterpret_cast<uint32_t*>(xdig + digit_offset(k, t)) = dw[t];
+        *reinterpret_cast<uint32_t*>(xdig + digit_offset(k, 3)) = 0u;
+#pragma unroll
+        for (int off = 1; off < lanes_per_group; off <<= 1) {
+          ds[0] += __shfl_xor_sync(0xffffffffu, ds[0], off);
+          ds[1] += __shfl_xor_sync(0xffffffffu, ds[1], off);
+          ds[2] += __shfl_xor_sync(0xffffffffu, ds[2], off);
+        }
+        if ((lane & (lanes_per_group - 1)) == 0) {
+          xsumw[(k / G) * 2 + 0] = (float)ds[0] + 256.f * (float)ds[1];
+          xsumw[(k / G) * 2 + 1] = 65536.f * (float)ds[2];
+        }
+      }
     }
   }
-  if (plan->nslots == 0 && blockIdx.x == 0)
+  __syncthreads();
+
+  // ---- step 4: precision fix-up and the static partition (warp 0: lane j owns slot j) ----
+  if (warp == 0) {
+    int nt = 0, sp = 0;
+    if (lane < nslots) {
+      Slot& s = slots[lane];
+      if (!(s.lsb[0] && s.lsb[1] && s.lsb[2])) s.prec = 0;
+      if (s.gated) s.coef = *in_gate;
+      nt = s.inter / 16;
+      sp = slot_spt1(s, p.hidden);
+    }
+    // inclusive scans of stages and tasks over the slots
+    unsigned cs = (unsigned)(nt * sp), ct = (unsigned)nt;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const unsigned a = __shfl_up_sync(0xffffffffu, cs, off), b = __shfl_up_sync(0xffffffffu, ct, off);
+      if (lane >= off) {
+        cs += a;
+        ct += b;
+      }
+    }
+    const unsigned S = __shfl_sync(0xffffffffu, cs, 31);
+    const unsigned NT = __shfl_sync(0xffffffffu, ct, 31);
+    // phase 1: equal shares of ring stages, at task granularity: the tasks whose first stage lies in [lo, hi)
+    const unsigned lo = (blockIdx.x * S + gridDim.x - 1) / gridDim.x;
+    const unsigned hi = ((blockIdx.x + 1) * S + gridDim.x - 1) / gridDim.x;
+    const unsigned off_s = cs - (unsigned)(nt * sp), off_t = ct - (unsigned)nt;  // exclusive
+    // ordinal of the first task at or after a bound, seen from the slot that contains it
+    unsigned ord_lo = NT, ord_hi = NT;
+    int slot_lo = nslots, idx_lo = 0;
+    if (lane < nslots && nt > 0) {
+      if (lo < cs && (lo >= off_s || lane == 0)) {
+        const unsigned i = lo <= off_s ? 0u : (lo - off_s + sp - 1) / sp;
+        ord_lo = off_t + i;  // i may equal nt: then it is the first task of the next slot
+        slot_lo = lane;
+        idx_lo = (int)i;
+      }
+      if (hi < cs && (hi >= off_s || lane == 0)) {
+        const unsigned i = hi <= off_s ? 0u : (hi - off_s + sp - 1) / sp;
+        ord_hi = off_t + i;
+      }
+    }
+    // exactly one lane (or none, when the bound is past the end) holds each answer
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const unsigned o = __shfl_xor_sync(0xffffffffu, ord_lo, off);
+      const int sl2 = __shfl_xor_sync(0xffffffffu, slot_lo, off), ix2 = __shfl_xor_sync(0xffffffffu, idx_lo, off);
+      if (sl2 < slot_lo) {
+        ord_lo = o;
+        slot_lo = sl2;
+        idx_lo = ix2;
+      }
+      ord_hi = min(ord_hi, __shfl_xor_sync(0xffffffffu, ord_hi, off));
+    }
+    if (lane == 0) {
+      if (slot_lo < nslots && idx_lo >= slots[slot_lo].inter / 16) {  // bound fell on the slot's end
+        idx_lo = 0;
+        ++slot_lo;
+      }
+      plan->first_slot = slot_lo;
+      plan->first_idx = idx_lo;
+      plan->count1 = (int)(ord_hi - ord_lo);
+      const int nrb = p.hidden / 16;
+      plan->count2 = (nslots > 0 && (int)blockIdx.x < nrb) ? (nrb - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    }
+  }
+  if (nslots == 0 && blockIdx.x == 0)
     for (int i = tid; i < p.hidden; i += kThreads) p.y[i] = 0.f;
   __syncthreads();
 
   if (warp < kConsumerWarps) {
     consumer_loop<G>(p, smem, warp, lane);
-  } else if (warp == kProducerWarp) {
-    if (lane == 0) producer_loop(p, smem);
-  } else {
-    epilogue_loop(p, smem, lane);
+  } else if (lane == 0) {
+    producer_loop<G>(p, smem);
   }
   __syncthreads();
   if (tid == 0) {
@@ -729,6 +853,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
     if (old == gridDim.x - 1) {  // everyone is past the barrier: make the header reusable
       p.ws->bar_arrive = 0;
       p.ws->depart = 0;
+      for (int j = 0; j < kMaxSlots; ++j) p.ws->hmax[j] = 0u;
       __threadfence();
     }
   }
@@ -787,6 +912,7 @@ static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts
   if (n_shared > 0 && !shared) return SLICEMOE_E_INVALID_ARG;
   if (n_shared > 0 && shape->shared_sigmoid_gate && !gate_vec) return SLICEMOE_E_INVALID_ARG;
   if (workspace_bytes < kWsBytes || (reinterpret_cast<uintptr_t>(workspace) & 255)) return SLICEMOE_E_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(x) & 15) return SLICEMOE_E_INVALID_ARG;
   const long long hsum = (long long)shape->top_k * shape->inter + (long long)n_shared * shape->shared_inter;
   if (hsum > kHCap) return SLICEMOE_E_UNSUPPORTED;
   int dev, sms;
@@ -799,7 +925,6 @@ static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts
   p.gate_vec = gate_vec;
   p.ws = reinterpret_cast<WsHeader*>(workspace);
   p.ws_h = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + kWsHOff);
-  p.ws_p = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + kWsPOff);
   p.n_experts = shape->n_experts;
   p.n_shared = n_shared;
   p.k = shape->top_k;

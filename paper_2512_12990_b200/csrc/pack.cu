@@ -59,38 +59,37 @@ __global__ void pack_planes_kernel(const float* __restrict__ W, int N, int K, in
                                    const uint16_t* __restrict__ scale, const uint8_t* __restrict__ zp,
                                    uint32_t* __restrict__ msb, uint32_t* __restrict__ lsb) {
   const size_t nwords = (size_t)N * K / 8;
-  const size_t w = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (w >= nwords) return;
-  // invert plane_word_index: w = ((rb*(K/64) + st)*32 + lane)*4 + tw
-  const int tw = (int)(w & 3);
-  const int lane = (int)((w >> 2) & 31);
-  const size_t blk = w >> 7;
+  const size_t widx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (widx >= nwords) return;
+  // invert plane_word_index: widx = ((rb*(K/64) + st)*32 + lane)*4 + w
+  const int w = (int)(widx & 3);
+  const int lane = (int)((widx >> 2) & 31);
+  const size_t blk = widx >> 7;
   const int st = (int)(blk % (size_t)(K >> 6));
   const int rb = (int)(blk / (size_t)(K >> 6));
   const int g8 = lane >> 2, c = lane & 3;
-  const int k0 = st * 64 + tw * 16 + c * 4;
+  const int k0 = st * 64 + w * 16 + c * 4;
   const int ngroups = K / group;
   const int grp = k0 / group;  // the 4 consecutive k share a group (group % 16 == 0)
   uint32_t mw = 0, lw = 0;
 #pragma unroll
-  for (int half_rows = 0; half_rows < 2; ++half_rows) {
-    const int n = rb * 16 + g8 + 8 * half_rows;
+  for (int hi = 0; hi < 2; ++hi) {
+    const int n = rb * 16 + g8 + 8 * hi;
     const float4 v = *reinterpret_cast<const float4*>(W + (size_t)n * K + k0);
     const size_t mi = meta_index(ngroups, n, grp);
     const float s = __half2float(__ushort_as_half(scale[mi]));
     const int z = zp[mi];
     const float vals[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-    for (int rem = 0; rem < 4; ++rem) {
-      const int q = quantise_one(vals[rem], s, z);
-      const int i = half_rows + 2 * (rem >> 1), hf = rem & 1;
-      const int pos = i + 4 * hf;
+    for (int j = 0; j < 4; ++j) {
+      const int q = quantise_one(vals[j], s, z);
+      const int pos = 2 * j + hi;
       mw |= (uint32_t)(q >> 4) << (4 * pos);
       lw |= (uint32_t)(q & 15) << (4 * pos);
     }
   }
-  msb[w] = mw;
-  lsb[w] = lw;
+  msb[widx] = mw;
+  lsb[widx] = lw;
 }
 
 __global__ void unpack_plane_kernel(const uint32_t* __restrict__ plane, int N, int K,

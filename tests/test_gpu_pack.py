@@ -94,11 +94,10 @@ def test_physical_layout_matches_header():
                 g, c = L // 4, L % 4
                 for w in range(4):
                     word = 0
-                    for i in range(4):
-                        for hf in range(2):
-                            row = 16 * rb + g + 8 * (i & 1)
-                            k = 64 * st + 16 * w + 4 * c + 2 * (i >> 1) + hf
-                            word |= int(o["msb"][row, k]) << (4 * (i + 4 * hf))
+                    for j in range(4):
+                        k = 64 * st + 16 * w + 4 * c + j
+                        word |= int(o["msb"][16 * rb + g, k]) << (8 * j)
+                        word |= int(o["msb"][16 * rb + g + 8, k]) << (8 * j + 4)
                     expect[((rb * (K // 64) + st) * 32 + L) * 4 + w] = word
     assert np.array_equal(raw, expect)
     ng = K // group
