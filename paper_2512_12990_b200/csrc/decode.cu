@@ -3,23 +3,25 @@
 //
 // The work is a pure weight stream: every plane byte is used once, so the bound is HBM bandwidth and
 // everything else is arranged so that the stream never stops.
-//   * One CTA per SM.  A producer thread streams 16-row x <=2048-column plane tiles (<=16 KB, one
-//     contiguous run each thanks to the tiled layout) plus their scales / zero-points into a
-//     shared-memory ring with cp.async.bulk + mbarriers.  The producer never waits for the gate/up ->
-//     down dependency, so down-projection tiles are already in flight (up to the whole ring) while
-//     the grid exchanges h.
-//   * Integer arithmetic on the tensor pipe.  The activation vector (x, later h) is converted once to
-//     23-bit fixed point relative to its largest magnitude and split into three balanced base-256
-//     digits (int8).  The digits sit in separate columns of the B operand of mma.sync m16n8k32
-//     (u8 x s8 -> s32); the A operand is the raw nibble plane: the layout stores the two row halves of
-//     a fragment in the low and high nibbles of each byte, so `w & 0x0f0f0f0f` and `(w >> 4) & 0x0f0f0f0f`
-//     are the whole unpack (2 ALU operations per 8 weights).  Sums are exact in int32; MSB and LSB
-//     planes combine as 16 * Cm + Cl.  Scale and zero-point are applied once per (row, group):
+//   * One CTA per SM: 16 consumer warps, one epilogue warp, one producer thread.  The producer streams
+//     16-row x <=2048-column plane tiles (<=16 KB, one contiguous run each thanks to the tiled layout)
+//     plus their scales / zero-points into a shared-memory ring with cp.async.bulk + mbarriers.  It
+//     never waits for the gate/up -> down dependency, so down-projection tiles are already in flight
+//     (up to the whole ring) while the grid exchanges h.
+//   * Integer arithmetic on the tensor pipe.  The activation vector (x, later h) is converted once,
+//     per 128-element block, to fixed point relative to the block's largest magnitude and split into
+//     three balanced base-256 digits (int8).  The digits sit in separate columns of the B operand of
+//     mma.sync m16n8k32 (u8 x s8 -> s32); the A operand is the raw nibble plane: the layout stores
+//     the two row halves of a fragment in the low and high nibbles of each byte, so `w & 0x0f0f0f0f`
+//     and `w & 0xf0f0f0f0` are the whole unpack (the second half comes out 16 times too large, which
+//     the per-row fold divides away).  Sums are exact in int32; MSB and LSB planes combine as
+//     16 * Cm + Cl.  Scale and zero-point are applied once per (row, group):
 //        sum_k x_k s (q_k - zp) = s (sum_k q_k x_k - zp sum_{k in group} x_k).
 //     The plain ALUs could not unpack + convert + FMA two weights per byte at HBM rate; this costs
-//     about nine instructions per 512 weights.
+//     about seven instructions per 512 weights.
 //   * Phase 1 (gate/up + SwiGLU): tasks are (expert slot, 16-row block), split over the CTAs by
-//     bytes.  h goes to the workspace in fp32; one bounded grid barrier publishes it.
+//     bytes.  The epilogue warp adds the warps' partial rows, applies SwiGLU and writes h (fp32) to
+//     the workspace; one bounded grid barrier publishes it.
 //   * Phase 2 (down + weighted combine): a task is a 16-row block of the OUTPUT over ALL slots, so
 //     the top-k combine stays inside the CTA: no atomics, no cross-CTA reduction, fixed summation
 //     order (results are bit-reproducible).
@@ -30,11 +32,12 @@
 
 namespace slicemoe {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kProducerWarp = kConsumerWarps;
-constexpr int kThreads = 32 * (kConsumerWarps + 1);
+constexpr int kConsumerWarps = 16;
+constexpr int kEpilogueWarp = kConsumerWarps;
+constexpr int kProducerWarp = kConsumerWarps + 1;
+constexpr int kThreads = 32 * (kConsumerWarps + 2);
 constexpr int kStages = 7;
-constexpr int kChunkK = 2048;                              // K columns per ring stage
+constexpr int kChunkK = 128 * kConsumerWarps;              // K columns per ring stage: one 128-column block per warp
 constexpr int kPlaneStageBytes = 16 * kChunkK / 2;         // 16384
 constexpr int kScaleStageBytes = 16 * (kChunkK / 32) * 2;  // 2048 (group 32 is the worst case)
 constexpr int kZpStageBytes = 16 * (kChunkK / 32);         // 1024
@@ -46,11 +49,10 @@ constexpr unsigned long long kWaitCycles = 4000000000ull;  // ~2 s: every device
 
 // ---- workspace --------------------------------------------------------------------------------
 struct WsHeader {
-  unsigned bar_arrive;        // grid barrier: CTAs that finished the gate/up phase
-  unsigned depart;            // CTAs that finished the kernel (the last one re-zeroes the header)
-  unsigned status;            // SLICEMOE_STATUS_* bits
+  unsigned bar_arrive;  // grid barrier: CTAs that finished the gate/up phase
+  unsigned depart;      // CTAs that finished the kernel (the last one re-zeroes the header)
+  unsigned status;      // SLICEMOE_STATUS_* bits
   unsigned pad;
-  unsigned hmax[kMaxSlots];   // per slot: bit pattern of max |h| (non-negative floats order as integers)
 };
 constexpr size_t kWsHOff = 2048;                              // float h[kHCap]
 constexpr size_t kWsStageOff = kWsHOff + sizeof(float) * kHCap;
@@ -90,22 +92,21 @@ struct Slot {
   int inter;
   int prec;
   float coef;
-  int hoff;     // offset of this slot's h in the workspace / in the digit buffer
-  int gated;    // 1: coef is sigmoid(gate_vec . x)
-  float hinv;   // 2^-e of this slot's fixed-point h
+  int hoff;   // offset of this slot's h in the workspace / in the digit buffer
+  int gated;  // 1: the combine weight is sigmoid(gate_vec . x)
+  int pad_;
 };
 
-struct StageDesc {
-  uint32_t flags;
-  uint16_t slot, rot;
-  uint32_t rb;
-  uint16_t kstep0, nblocks;  // first 32-column step of the chunk within the matrix; 128-column blocks in it
-};
+// One ring stage as the consumers see it (16 bytes, written by the producer):
+//   x: flags | nblocks << 8 | rot << 16 | slot << 24
+//   y: byte offset in shared memory of the activation digits of the chunk's first column
+//   z: byte offset in shared memory of the chunk's first (group, digit-pair) weighted digit sum
+//   w: byte offset in shared memory of the chunk's first per-128-block inverse scale
 enum : uint32_t {
   kFlagLsb = 1,           // this stage carries the LSB plane of the chunk (accumulate onto 16 x MSB sums)
   kFlagMeta = 2,          // last plane of the chunk: scales / zero-points are in the stage; fold the chunk
   kFlagLastOfMatrix = 4,  // last chunk of the matrix row block
-  kFlagLastOfTask = 8,    // last matrix of the task: reduce over the warps and write out
+  kFlagLastOfTask = 8,    // last matrix of the task: hand the partial rows to the epilogue warp
   kFlagEnd = 16,          // sentinel, no data
   kFlagPrec8 = 32,
   kFlagPhase2 = 64,
@@ -116,7 +117,8 @@ struct Plan {
   int count2;                         // phase 2: output row blocks blockIdx.x, + gridDim.x, ...
   int nslots;
   int htotal;  // sum of the slots' intermediate widths
-  float xinv;  // 2^-e of the fixed-point x
+  float gate;  // sigmoid(gate_vec . x) when the shared experts are gated
+  int pad_;
 };
 
 struct SmemLayout {
@@ -124,26 +126,27 @@ struct SmemLayout {
   static constexpr int ring = 0;
   static constexpr int hdig = ring + kStages * kStageBytes;  // int8 [kHCap/32][4 digits][32]
   static constexpr int xdig = hdig + kHCap * 4;              // int8 [kMaxHidden/32][4][32]
-  static constexpr int xsumw = xdig + kMaxHidden * 4;        // float [kMaxHidden/32][2]: weighted digit sums per group
-  static constexpr int hsumw = xsumw + (kMaxHidden / 32) * 8;  // float [kHCap/32][2]
-  static constexpr int partial = hsumw + (kHCap / 32) * 8;     // float [2][warps][16][2]
+  static constexpr int hsumw = xdig + kMaxHidden * 4;        // float [kHCap/32][2]: weighted digit sums per group
+  static constexpr int xsumw = hsumw + (kHCap / 32) * 8;     // float [kMaxHidden/32][2]
+  static constexpr int hinv = xsumw + (kMaxHidden / 32) * 8;  // float [kHCap/128]: 2^-e of each 128-block of h
+  static constexpr int xinv = hinv + (kHCap / 128) * 4;       // float [kMaxHidden/128]
+  static constexpr int partial = xinv + (kMaxHidden / 128) * 4;  // float [2][warps][16][2]
   static constexpr int slots = partial + 2 * kConsumerWarps * 16 * 2 * 4;
-  static constexpr int desc = slots + kMaxSlots * (int)sizeof(Slot);
-  static constexpr int stage_in = desc + kStages * (int)sizeof(StageDesc);  // ids i32[16] | w f32[16] | prec i32[16] | gate f32 | xmax u32
-  static constexpr int plan = stage_in + 4 * (3 * SLICEMOE_MAX_TOP_K + 4);
+  static constexpr int desc = slots + kMaxSlots * (int)sizeof(Slot);  // uint4 [kStages]
+  static constexpr int plan = desc + kStages * 16;
   static constexpr int bars = (plan + (int)sizeof(Plan) + 15) & ~15;  // uint64 barriers
-  static constexpr int nbars = 2 * kStages + 7;
+  static constexpr int nbars = 2 * kStages + 6;
   static constexpr int dead = bars + nbars * 8;
   static constexpr int total = dead + 16;
 };
 static_assert(SmemLayout::total <= 227 * 1024, "shared memory budget");
 static_assert(sizeof(Slot) % 8 == 0, "slot alignment");
 static_assert(SmemLayout::slots % 8 == 0 && SmemLayout::hdig % 16 == 0 && SmemLayout::xdig % 16 == 0 &&
-                  SmemLayout::desc % 16 == 0,
+                  SmemLayout::desc % 16 == 0 && SmemLayout::plan % 8 == 0,
               "alignment");
 
 // barrier indices after the 2*kStages ring barriers
-enum { kBarPFull0 = 0, kBarPFull1, kBarPEmpty0, kBarPEmpty1, kBarHxArrive, kBarHxGo, kBarHsReady };
+enum { kBarPFull0 = 0, kBarPFull1, kBarPEmpty0, kBarPEmpty1, kBarHxGo, kBarHsReady };
 
 // ---- PTX helpers -------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -194,8 +197,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 }
 __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -206,18 +208,33 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
 }
 
 // ---- fixed-point activations ---------------------------------------------------------------------
-// 2^e with 2^e * vmax < 2^22 (vmax given as the bit pattern of a non-negative float), and 2^-e: every
-// value then rounds to an integer |X| <= 2^22 whose third balanced base-256 digit fits int8 with room.
-__device__ __forceinline__ void fixed_scale(unsigned vmax_bits, float* scale, float* inv) {
-  int ex = (int)((vmax_bits >> 23) & 0xffu) - 127;  // floor(log2 vmax) for normal numbers
-  int e = 21 - ex;
-  e = max(-100, min(100, e));
-  *scale = __uint_as_float((unsigned)(127 + e) << 23);
-  *inv = __uint_as_float((unsigned)(127 - e) << 23);
+// Byte offset, inside a digit buffer, of digit t of the four values k..k+3 (k % 4 == 0): steps of 32
+// columns, 4 digit rows of 32 bytes (the fourth stays zero), and inside a row the order in which the B
+// fragment of m16n8k32 wants them: (k % 16) / 4 selects the lane quad position, (k % 32) / 16 the register.
+__device__ __forceinline__ int digit_offset(int k, int t) {
+  return (k >> 5) * 128 + t * 32 + ((k >> 2) & 3) * 8 + ((k >> 4) & 1) * 4;
 }
-// Four values -> three words of balanced base-256 digits (byte j of word t = digit t of value j).
-__device__ __forceinline__ void to_digits4(const float (&v)[4], float scale, uint32_t (&dw)[3], int (&dsum)[3]) {
-  dw[0] = dw[1] = dw[2] = 0;
+
+// One warp converts one 128-element block (lane L holds elements 4L..4L+3 of the block, whose first
+// element has index k0 in its vector): fixed point X = rint(v * 2^e) with 2^e * max|v| < 2^22, split into
+// balanced base-256 digits d0 + 256 d1 + 65536 d2 (each in int8 range), stored in B-fragment order; the
+// weighted digit sums of every group of G elements (the zero-point term of the fold) and the block's 2^-e.
+template <int G>
+__device__ __forceinline__ void block_to_digits(const float (&v)[4], int k0, int lane, uint8_t* dig, float* sumw,
+                                                float* inv) {
+  float m = 0.f;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float a = fabsf(v[j]);
+    if (a == a) m = fmaxf(m, a);  // a NaN input gives an undefined result, never a fault
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+  const int ex = (int)((__float_as_uint(m) >> 23) & 0xffu) - 127;  // floor(log2 m) for normal numbers
+  const int e = max(-100, min(100, 21 - ex));
+  const float scale = __uint_as_float((unsigned)(127 + e) << 23);
+  uint32_t dw[3] = {0u, 0u, 0u};
+  int ds[3] = {0, 0, 0};
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     int X = __float2int_rn(v[j] * scale);
@@ -229,16 +246,26 @@ __device__ __forceinline__ void to_digits4(const float (&v)[4], float scale, uin
     dw[0] |= (uint32_t)(d0 & 255) << (8 * j);
     dw[1] |= (uint32_t)(d1 & 255) << (8 * j);
     dw[2] |= (uint32_t)(d2 & 255) << (8 * j);
-    dsum[0] += d0;
-    dsum[1] += d1;
-    dsum[2] += d2;
+    ds[0] += d0;
+    ds[1] += d1;
+    ds[2] += d2;
   }
-}
-// Byte offset, inside the digit buffer, of digit t of the four values k..k+3 (k % 4 == 0): steps of 32
-// columns, 4 digit rows of 32 bytes (the fourth stays zero), and inside a row the order in which the B
-// fragment of m16n8k32 wants them: (k % 16) / 4 selects the lane quad position, (k % 32) / 16 the register.
-__device__ __forceinline__ int digit_offset(int k, int t) {
-  return (k >> 5) * 128 + t * 32 + ((k >> 2) & 3) * 8 + ((k >> 4) & 1) * 4;
+  const int k = k0 + 4 * lane;
+#pragma unroll
+  for (int t = 0; t < 3; ++t) *reinterpret_cast<uint32_t*>(dig + digit_offset(k, t)) = dw[t];
+  *reinterpret_cast<uint32_t*>(dig + digit_offset(k, 3)) = 0u;
+  constexpr int lanes_per_group = G / 4;  // 8, 16 or 32 consecutive lanes cover one group
+#pragma unroll
+  for (int off = 1; off < lanes_per_group; off <<= 1) {
+    ds[0] += __shfl_xor_sync(0xffffffffu, ds[0], off);
+    ds[1] += __shfl_xor_sync(0xffffffffu, ds[1], off);
+    ds[2] += __shfl_xor_sync(0xffffffffu, ds[2], off);
+  }
+  if ((lane & (lanes_per_group - 1)) == 0) {
+    sumw[(k / G) * 2 + 0] = (float)ds[0] + 256.f * (float)ds[1];
+    sumw[(k / G) * 2 + 1] = 65536.f * (float)ds[2];
+  }
+  if (lane == 0) inv[k0 >> 7] = __uint_as_float((unsigned)(127 - e) << 23);
 }
 
 // ---- task enumeration (identical in every role) ---------------------------------------------------
@@ -246,120 +273,32 @@ __device__ __forceinline__ int nchunks_of(int K) { return (K + kChunkK - 1) / kC
 // ring stages of one phase-1 task (gate + up of a 16-row block) of a slot
 __device__ __forceinline__ int slot_spt1(const Slot& s, int hidden) { return 2 * (s.prec ? 2 : 1) * nchunks_of(hidden); }
 
-// ---- consumer ------------------------------------------------------------------------------------
-// One plane stage: this warp's (up to two) 128-column blocks.  `dig` points at the digit buffer entry
-// of the matrix' first column (x digits in phase 1, the slot's h digits in phase 2).
+// ---- consumers -----------------------------------------------------------------------------------
+// Phase change: wait until the epilogue warp has seen the whole grid's h in the workspace, then turn it
+// into digits (all consumer warps, one 128-block at a time).  Returns false if a wait ran out.
 template <int G>
-__device__ __forceinline__ void consume_blocks(int (&acc)[2][128 / G][4], const uint8_t* stage, int b0, bool v0, int b1,
-                                               bool v1, const uint8_t* dig, int kstep0, int lane) {
-  const int boff = ((lane >> 2) & 3) * 32 + (lane & 3) * 8;  // digit row = column of B this lane feeds
-#pragma unroll
-  for (int u = 0; u < 2; ++u) {
-    uint4 w0 = make_uint4(0, 0, 0, 0), w1 = make_uint4(0, 0, 0, 0);
-    if (v0) w0 = *reinterpret_cast<const uint4*>(stage + (2 * b0 + u) * 512 + lane * 16);
-    if (v1) w1 = *reinterpret_cast<const uint4*>(stage + (2 * b1 + u) * 512 + lane * 16);
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int s4 = 2 * u + h;         // 32-column step within the 128-column block
-      const int sg = (32 * s4) / G;     // group within the block
-#pragma unroll
-      for (int bi = 0; bi < 2; ++bi) {
-        const bool valid = bi ? v1 : v0;
-        if (!valid) continue;
-        const uint4 w = bi ? w1 : w0;
-        const uint32_t wa = h ? w.z : w.x, wb = h ? w.w : w.y;
-        const int b = bi ? b1 : b0;
-        const uint2 bv = *reinterpret_cast<const uint2*>(dig + (kstep0 + 4 * b + s4) * 128 + boff);
-        mma_u8s8(acc[bi][sg], wa & 0x0f0f0f0fu, (wa >> 4) & 0x0f0f0f0fu, wb & 0x0f0f0f0fu, (wb >> 4) & 0x0f0f0f0fu, bv.x,
-                 bv.y);
-      }
-    }
-  }
-}
-
-// All consumer warps: fp32 h (workspace, L2) -> fixed-point digits and weighted digit sums in shared memory.
-template <int G>
-__device__ void load_h_to_smem(const DecodeParams& p, uint8_t* smem, int warp, int lane, int htotal) {
-  Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
-  const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
-  uint8_t* hdig = smem + SmemLayout::hdig;
-  float* hsumw = reinterpret_cast<float*>(smem + SmemLayout::hsumw);
-  constexpr int lanes_per_group = G / 4;    // 8, 16 or 32 consecutive lanes cover one group
-  const int n4 = htotal / 4;                // multiple of 32: every slot width is a multiple of 128
-  constexpr int kMaxIt = (kHCap / 4 + kConsumerWarps * 32 - 1) / (kConsumerWarps * 32);
+__device__ bool fetch_h(const DecodeParams& p, uint8_t* smem, int warp, int lane, int htotal, volatile int* dead,
+                        unsigned* status, uint32_t xbars) {
+  const uint32_t hx_go = xbars + 8 * kBarHxGo, hs_ready = xbars + 8 * kBarHsReady;
+  if (!mbar_wait(hx_go, 0, dead, status)) return false;
+  if (*dead) return false;
+  const int nblk = htotal >> 7;
+  constexpr int kMaxIt = (kHCap / 128 + kConsumerWarps - 1) / kConsumerWarps;
   float4 v[kMaxIt];
 #pragma unroll
   for (int it = 0; it < kMaxIt; ++it) {
-    const int i = (it * kConsumerWarps + warp) * 32 + lane;
-    if (i < n4) v[it] = __ldcg(reinterpret_cast<const float4*>(p.ws_h) + i);
+    const int blk = it * kConsumerWarps + warp;
+    if (blk < nblk) v[it] = __ldcg(reinterpret_cast<const float4*>(p.ws_h) + blk * 32 + lane);
   }
-  // per-slot scale from the published maxima (every warp computes the few it needs)
-  int slot = 0;
 #pragma unroll
   for (int it = 0; it < kMaxIt; ++it) {
-    const int i = (it * kConsumerWarps + warp) * 32 + lane;
-    if (i < n4) {  // uniform per warp; a warp's 128 values lie in one slot
-      const int k = 4 * i;
-      while (slot + 1 < plan.nslots && k >= slots[slot + 1].hoff) ++slot;
-      float scale, inv;
-      fixed_scale(__ldcg(&p.ws->hmax[slot]), &scale, &inv);
-      if (k == slots[slot].hoff) slots[slot].hinv = inv;  // first lane of the slot's first warp row
+    const int blk = it * kConsumerWarps + warp;
+    if (blk < nblk) {
       const float q[4] = {v[it].x, v[it].y, v[it].z, v[it].w};
-      uint32_t dw[3];
-      int ds[3] = {0, 0, 0};
-      to_digits4(q, scale, dw, ds);
-#pragma unroll
-      for (int t = 0; t < 3; ++t) *reinterpret_cast<uint32_t*>(hdig + digit_offset(k, t)) = dw[t];
-      *reinterpret_cast<uint32_t*>(hdig + digit_offset(k, 3)) = 0u;
-#pragma unroll
-      for (int off = 1; off < lanes_per_group; off <<= 1) {
-        ds[0] += __shfl_xor_sync(0xffffffffu, ds[0], off);
-        ds[1] += __shfl_xor_sync(0xffffffffu, ds[1], off);
-        ds[2] += __shfl_xor_sync(0xffffffffu, ds[2], off);
-      }
-      if ((lane & (lanes_per_group - 1)) == 0) {
-        hsumw[(k / G) * 2 + 0] = (float)ds[0] + 256.f * (float)ds[1];
-        hsumw[(k / G) * 2 + 1] = 65536.f * (float)ds[2];
-      }
+      block_to_digits<G>(q, blk * 128, lane, smem + SmemLayout::hdig, reinterpret_cast<float*>(smem + SmemLayout::hsumw),
+                         reinterpret_cast<float*>(smem + SmemLayout::hinv));
     }
   }
-}
-
-// The single grid-wide dependency: every CTA has written its rows of h.  Executed by all consumer
-// warps; returns false if a wait ran out.
-template <int G>
-__device__ bool exchange_h(const DecodeParams& p, uint8_t* smem, int warp, int lane, bool need_h, int htotal,
-                           volatile int* dead, unsigned* status, uint32_t xbars) {
-  const uint32_t hx_arrive = xbars + 8 * kBarHxArrive, hx_go = xbars + 8 * kBarHxGo, hs_ready = xbars + 8 * kBarHsReady;
-  __syncwarp();
-  if (lane == 0) mbar_arrive(hx_arrive);  // this warp's h rows are written
-  if (warp == 0) {
-    // the whole warp stays converged while it waits: no lane spins on something another lane must provide
-    if (!mbar_wait(hx_arrive, 0, dead, status)) return false;
-    if (lane == 0) {
-      __threadfence();
-      atomicAdd(&p.ws->bar_arrive, 1u);
-    }
-    __syncwarp();
-    if (need_h) {
-      const long long t0 = clock64();
-      while (ld_acquire_u32(&p.ws->bar_arrive) < gridDim.x) {
-        if (*dead) break;
-        if ((unsigned long long)(clock64() - t0) > kWaitCycles) {
-          *dead = 1;
-          atomicOr(status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
-          break;
-        }
-      }
-      __threadfence();
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(hx_go);
-  }
-  if (!need_h) return true;
-  if (!mbar_wait(hx_go, 0, dead, status)) return false;
-  if (*dead) return false;
-  load_h_to_smem<G>(p, smem, warp, lane, htotal);
   __syncwarp();
   if (lane == 0) mbar_arrive(hs_ready);
   return mbar_wait(hs_ready, 0, dead, status);
@@ -369,10 +308,8 @@ template <int G>
 __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, int lane) {
   constexpr int SG = 128 / G;
   const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
-  const StageDesc* descs = reinterpret_cast<const StageDesc*>(smem + SmemLayout::desc);
+  const uint4* descs = reinterpret_cast<const uint4*>(smem + SmemLayout::desc);
   const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
-  const float* xsumw = reinterpret_cast<const float*>(smem + SmemLayout::xsumw);
-  const float* hsumw = reinterpret_cast<const float*>(smem + SmemLayout::hsumw);
   float* partial = reinterpret_cast<float*>(smem + SmemLayout::partial);
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
@@ -381,133 +318,168 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
   unsigned* status = &p.ws->status;
 
   // The lane folds row r of the 16-row block for the digit columns it holds: lanes with c in {0, 1} take
-  // the accumulators of row g, lanes with c in {2, 3} those of row g + 8; even c holds digits 0 and 1, odd c
+  // the accumulators of row g, lanes with c in {2, 3} those of row g + 8 (which are 16 times too large
+  // because their nibbles were left in the high half of the byte); even c holds digits 0 and 1, odd c
   // digit 2 (and the unused fourth column).
   const int c = lane & 3, g8 = lane >> 2;
   const int r = g8 + 8 * (c >> 1);
   const int cq = c & 1;
-  const float w0 = cq ? 65536.f : 1.f, w1 = cq ? 0.f : 256.f;
-  int acc[2][SG][4];
+  const float rowfix = (c >> 1) ? 0.0625f : 1.f;
+  const float w0 = (cq ? 65536.f : 1.f) * rowfix, w1 = (cq ? 0.f : 256.f) * rowfix;
+  const int boff = (g8 & 3) * 32 + c * 8;  // digit row = column of B this lane feeds
+  int acc[SG][4];
   float rowacc = 0.f, part0 = 0.f, part1 = 0.f;
-  bool exchanged = false;
+  bool fetched = false;
   int taskcount = 0;
 
   for (int it = 0;; ++it) {
     const int stage = it % kStages;
     if (!mbar_wait(full0 + 8 * stage, (it / kStages) & 1, dead, status)) return;
-    const uint4 draw = *reinterpret_cast<const uint4*>(descs + stage);
-    StageDesc d;
-    d.flags = draw.x;
-    d.slot = (uint16_t)(draw.y & 0xffffu);
-    d.rot = (uint16_t)(draw.y >> 16);
-    d.rb = draw.z;
-    d.kstep0 = (uint16_t)(draw.w & 0xffffu);
-    d.nblocks = (uint16_t)(draw.w >> 16);
-    const bool phase2 = (d.flags & kFlagPhase2) != 0;
-    if (((d.flags & kFlagEnd) || phase2) && !exchanged) {
-      if (!exchange_h<G>(p, smem, warp, lane, phase2, plan.htotal, dead, status, xbars)) return;
-      exchanged = true;
+    const uint4 d = descs[stage];
+    const uint32_t flags = d.x & 0xffu;
+    if (flags & kFlagEnd) break;
+    if ((flags & kFlagPhase2) && !fetched) {
+      if (!fetch_h<G>(p, smem, warp, lane, plan.htotal, dead, status, xbars)) return;
+      fetched = true;
     }
-    if (d.flags & kFlagEnd) break;
-    const Slot& sl = slots[d.slot];
-    const uint8_t* stg = smem + SmemLayout::ring + stage * kStageBytes;
-    // blocks (128 columns) of this chunk handled by this warp: b0 and b0 + warps
-    int b0 = warp - (int)d.rot;
-    if (b0 < 0) b0 += kConsumerWarps;
-    const int b1 = b0 + kConsumerWarps;
-    const bool v0 = b0 < d.nblocks, v1 = b1 < d.nblocks;
-    if (!(d.flags & kFlagLsb)) {
-#pragma unroll
-      for (int bi = 0; bi < 2; ++bi)
+    // the 128-column block of this chunk handled by this warp
+    int b = warp - (int)((d.x >> 16) & 0xffu);
+    if (b < 0) b += kConsumerWarps;
+    const bool valid = b < (int)((d.x >> 8) & 0xffu);
+    if (valid) {
+      if (!(flags & kFlagLsb)) {
 #pragma unroll
         for (int sg = 0; sg < SG; ++sg)
 #pragma unroll
-          for (int q = 0; q < 4; ++q) acc[bi][sg][q] = 0;
-    } else {
-#pragma unroll
-      for (int bi = 0; bi < 2; ++bi)
+          for (int q = 0; q < 4; ++q) acc[sg][q] = 0;
+      } else {
 #pragma unroll
         for (int sg = 0; sg < SG; ++sg)
 #pragma unroll
-          for (int q = 0; q < 4; ++q) acc[bi][sg][q] <<= 4;
-    }
-    const uint8_t* dig = phase2 ? smem + SmemLayout::hdig + sl.hoff * 4 : smem + SmemLayout::xdig;
-    consume_blocks<G>(acc, stg, b0, v0, b1, v1, dig, d.kstep0, lane);
-    if (d.flags & kFlagMeta) {
-      const uint16_t* ms = reinterpret_cast<const uint16_t*>(stg + kPlaneStageBytes);
-      const uint8_t* mz = stg + kPlaneStageBytes + kScaleStageBytes;
-      const float* sumw = phase2 ? hsumw + ((sl.hoff + d.kstep0 * 32) / G) * 2 : xsumw + ((d.kstep0 * 32) / G) * 2;
-      const bool p8 = (d.flags & kFlagPrec8) != 0;
-#pragma unroll
-      for (int bi = 0; bi < 2; ++bi) {
-        const bool valid = bi ? v1 : v0;
-        if (!valid) continue;
-        const int b = bi ? b1 : b0;
+          for (int q = 0; q < 4; ++q) acc[sg][q] <<= 4;
+      }
+      const uint8_t* ap = smem + SmemLayout::ring + stage * kStageBytes + b * 1024 + lane * 16;
+      const uint8_t* bp = smem + d.y + b * 512 + boff;
+      const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
+      const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
+      const uint2 bv0 = *reinterpret_cast<const uint2*>(bp);
+      const uint2 bv1 = *reinterpret_cast<const uint2*>(bp + 128);
+      const uint2 bv2 = *reinterpret_cast<const uint2*>(bp + 256);
+      const uint2 bv3 = *reinterpret_cast<const uint2*>(bp + 384);
+      mma_u8s8(acc[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
+      mma_u8s8(acc[32 / G], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x,
+               bv1.y);
+      mma_u8s8(acc[64 / G], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x,
+               bv2.y);
+      mma_u8s8(acc[96 / G], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x,
+               bv3.y);
+      if (flags & kFlagMeta) {
+        const uint8_t* stg = smem + SmemLayout::ring + stage * kStageBytes;
+        const uint16_t* ms = reinterpret_cast<const uint16_t*>(stg + kPlaneStageBytes) + (b * SG) * 16 + r;
+        const uint8_t* mz = stg + kPlaneStageBytes + kScaleStageBytes + (b * SG) * 16 + r;
+        const float* sumw = reinterpret_cast<const float*>(smem + d.z) + (b * SG) * 2 + cq;
+        const float binv = *(reinterpret_cast<const float*>(smem + d.w) + b);
+        const bool p8 = (flags & kFlagPrec8) != 0;
+        const float sfix = p8 ? binv : 16.f * binv;
+        const int zsh = p8 ? 0 : 4;
 #pragma unroll
         for (int sg = 0; sg < SG; ++sg) {
-          const int gl = b * SG + sg;
-          const int ca = (c >> 1) ? acc[bi][sg][2] : acc[bi][sg][0];
-          const int cb = (c >> 1) ? acc[bi][sg][3] : acc[bi][sg][1];
+          const int ca = (c >> 1) ? acc[sg][2] : acc[sg][0];
+          const int cb = (c >> 1) ? acc[sg][3] : acc[sg][1];
           const float t = fmaf((float)cb, w1, (float)ca * w0);
-          const float s = __half2float(__ushort_as_half(ms[gl * 16 + r]));
-          const int z = mz[gl * 16 + r];
-          const float X = sumw[gl * 2 + cq];
+          const float s = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
+          const float z = (float)((int)mz[sg * 16] >> zsh);
           // both slices: s (16 Cm + Cl - zp X); MSB only: 16 s (Cm - (zp >> 4) X)
-          if (p8) rowacc = fmaf(s, fmaf(-(float)z, X, t), rowacc);
-          else rowacc = fmaf(16.f * s, fmaf(-(float)(z >> 4), X, t), rowacc);
+          rowacc = fmaf(s, fmaf(-z, sumw[sg * 2], t), rowacc);
         }
       }
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(empty0 + 8 * stage);
-    if (d.flags & kFlagLastOfMatrix) {
+    if (flags & kFlagLastOfMatrix) {
       rowacc += __shfl_xor_sync(0xffffffffu, rowacc, 1);  // digits 0,1 (even c) + digit 2 (odd c)
-      if (!phase2) {
-        rowacc *= plan.xinv;
-        if (!(d.flags & kFlagLastOfTask)) part0 = rowacc;  // gate
-        else part1 = rowacc;                               // up
+      if (!(flags & kFlagPhase2)) {
+        if (!(flags & kFlagLastOfTask)) part0 = rowacc;  // gate
+        else part1 = rowacc;                             // up
       } else {
-        part1 = fmaf(sl.coef * sl.hinv, rowacc, part1);  // weighted combine over the slots, in slot order
+        const Slot& sl = slots[d.x >> 24];
+        part1 = fmaf(sl.gated ? plan.gate : sl.coef, rowacc, part1);  // weighted combine, in slot order
       }
       rowacc = 0.f;
+      if (flags & kFlagLastOfTask) {
+        // hand this warp's share of the K split to the epilogue warp
+        const int buf = taskcount & 1;
+        if (!mbar_wait(pempty0 + 8 * buf, ((taskcount >> 1) & 1) ^ 1, dead, status)) return;
+        if (cq == 0) *reinterpret_cast<float2*>(partial + ((buf * kConsumerWarps + warp) * 16 + r) * 2) = make_float2(part0, part1);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pfull0 + 8 * buf);
+        ++taskcount;
+        part0 = part1 = 0.f;
+      }
     }
-    if (d.flags & kFlagLastOfTask) {
-      // cross-warp reduction of the K split: warp 0 adds the partial rows in warp order
-      const int buf = taskcount & 1;
-      if (!mbar_wait(pempty0 + 8 * buf, ((taskcount >> 1) & 1) ^ 1, dead, status)) return;
-      if (cq == 0) {
-        float* dst = partial + ((buf * kConsumerWarps + warp) * 16 + r) * 2;
-        dst[0] = part0;
-        dst[1] = part1;
+  }
+}
+
+// ---- epilogue warp ---------------------------------------------------------------------------------
+__device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
+  const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
+  const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
+  const float* partial = reinterpret_cast<const float*>(smem + SmemLayout::partial);
+  volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
+  const uint32_t bars = smem_u32(smem + SmemLayout::bars);
+  const uint32_t xbars = bars + 16 * kStages;
+  const uint32_t pfull0 = xbars + 8 * kBarPFull0, pempty0 = xbars + 8 * kBarPEmpty0, hx_go = xbars + 8 * kBarHxGo;
+  unsigned* status = &p.ws->status;
+  const int total = plan.count1 + plan.count2;
+  int slot = plan.first_slot, idx = plan.first_idx;
+  for (int tc = 0;; ++tc) {
+    if (tc == plan.count1) {
+      // ---- the single grid-wide dependency: every CTA has written its rows of h ----
+      __syncwarp();
+      if (lane == 0) {
+        __threadfence();
+        atomicAdd(&p.ws->bar_arrive, 1u);
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(pfull0 + 8 * buf);
-      if (warp == 0) {
-        if (!mbar_wait(pfull0 + 8 * buf, (taskcount >> 1) & 1, dead, status)) return;
-        float a = 0.f, b = 0.f;
-        if (lane < 16) {
-#pragma unroll
-          for (int w = 0; w < kConsumerWarps; ++w) {
-            const float* src = partial + ((buf * kConsumerWarps + w) * 16 + lane) * 2;
-            a += src[0];
-            b += src[1];
+      if (plan.count2 > 0) {
+        // the whole warp polls, converged: no lane spins on something another lane must provide
+        const long long t0 = clock64();
+        while (ld_acquire_u32(&p.ws->bar_arrive) < gridDim.x) {
+          if (*dead) break;
+          if ((unsigned long long)(clock64() - t0) > kWaitCycles) {
+            *dead = 1;
+            atomicOr(status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
+            break;
           }
         }
-        if (!phase2) {
-          const float h = a / (1.f + expf(-a)) * b;  // silu(gate) * up
-          if (lane < 16) p.ws_h[sl.hoff + d.rb * 16 + lane] = h;
-          float m = lane < 16 ? fabsf(h) : 0.f;
-#pragma unroll
-          for (int off = 8; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-          if (lane == 0 && m == m) atomicMax(&p.ws->hmax[d.slot], __float_as_uint(m));
-        } else if (lane < 16) {
-          p.y[d.rb * 16 + lane] = b;
-        }
+        __threadfence();
         __syncwarp();
-        if (lane == 0) mbar_arrive(pempty0 + 8 * buf);
+        if (*dead) return;
+        if (lane == 0) mbar_arrive(hx_go);
       }
-      ++taskcount;
-      part0 = part1 = 0.f;
+    }
+    if (tc == total) break;
+    const int buf = tc & 1;
+    if (!mbar_wait(pfull0 + 8 * buf, (tc >> 1) & 1, dead, status)) return;
+    float a = 0.f, b = 0.f;
+    if (lane < 16) {
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) {
+        const float2 v = *reinterpret_cast<const float2*>(partial + ((buf * kConsumerWarps + w) * 16 + lane) * 2);
+        a += v.x;
+        b += v.y;
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(pempty0 + 8 * buf);
+    if (tc < plan.count1) {
+      if (lane < 16) p.ws_h[slots[slot].hoff + idx * 16 + lane] = a / (1.f + expf(-a)) * b;  // silu(gate) * up
+      if (++idx >= slots[slot].inter / 16) {
+        idx = 0;
+        ++slot;
+      }
+    } else if (lane < 16) {
+      p.y[(blockIdx.x + (tc - plan.count1) * gridDim.x) * 16 + lane] = b;
     }
   }
 }
@@ -519,10 +491,12 @@ struct ProducerState {
 };
 
 // Streams the planes of one (slot, matrix, row block) into the ring.  Returns false if a wait ran out.
+// act_* are the shared-memory byte offsets of the activation digits / digit sums / block scales that go
+// with the matrix' first column.
 template <int G>
 __device__ __forceinline__ bool produce_matrix(uint8_t* smem, ProducerState& ps, const Slot& s, int slot, int mat, int K,
-                                               int rb, uint32_t base_flags, bool last_matrix, volatile int* dead,
-                                               unsigned* status) {
+                                               int rb, uint32_t base_flags, bool last_matrix, uint32_t act_dig,
+                                               uint32_t act_sum, uint32_t act_inv, volatile int* dead, unsigned* status) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
   uint4* descs = reinterpret_cast<uint4*>(smem + SmemLayout::desc);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
@@ -539,13 +513,15 @@ __device__ __forceinline__ bool produce_matrix(uint8_t* smem, ProducerState& ps,
     const int kc = min(kChunkK, K - k0);
     const bool last_chunk = k0 + kChunkK >= K;
     for (int pl = 0; pl < nplanes; ++pl) {
-      int stage = ps.it % kStages;
+      const int stage = ps.it % kStages;
       if (!mbar_wait(empty0 + 8 * stage, ((ps.it / kStages) & 1) ^ 1, dead, status)) return false;
       const bool has_meta = (pl == nplanes - 1);
       uint32_t flags = flags0 | (pl ? kFlagLsb : 0u) | (has_meta ? kFlagMeta : 0u);
       if (has_meta && last_chunk) flags |= kFlagLastOfMatrix | (last_matrix ? kFlagLastOfTask : 0u);
-      descs[stage] = make_uint4(flags, (uint32_t)slot | ((uint32_t)(ps.chunk % kConsumerWarps) << 16), (uint32_t)rb,
-                                (uint32_t)(k0 >> 5) | ((uint32_t)(kc >> 7) << 16));
+      descs[stage] = make_uint4(flags | ((uint32_t)(kc >> 7) << 8) | ((uint32_t)(ps.chunk % kConsumerWarps) << 16) |
+                                    ((uint32_t)slot << 24),
+                                act_dig + (uint32_t)k0 * 4u, act_sum + (uint32_t)(k0 >> LG) * 8u,
+                                act_inv + (uint32_t)(k0 >> 7) * 4u);
       const uint32_t plane_bytes = (uint32_t)kc * 8u;
       const uint32_t ngc = (uint32_t)(kc >> LG);
       const uint32_t bar = full0 + 8 * stage;
@@ -566,6 +542,7 @@ __device__ __forceinline__ bool produce_matrix(uint8_t* smem, ProducerState& ps,
 
 template <int G>
 __device__ void producer_loop(const DecodeParams& p, uint8_t* smem) {
+  constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
   const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
   uint4* descs = reinterpret_cast<uint4*>(smem + SmemLayout::desc);
   const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
@@ -582,8 +559,10 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem) {
     int slot = plan.first_slot, idx = plan.first_idx;
     for (int n = 0; n < plan.count1 && ok; ++n) {
       const Slot& s = slots[slot];
-      ok = produce_matrix<G>(smem, ps, s, slot, 0, p.hidden, idx, 0u, false, dead, status) &&
-           produce_matrix<G>(smem, ps, s, slot, 1, p.hidden, idx, 0u, true, dead, status);
+      ok = produce_matrix<G>(smem, ps, s, slot, 0, p.hidden, idx, 0u, false, SmemLayout::xdig, SmemLayout::xsumw,
+                             SmemLayout::xinv, dead, status) &&
+           produce_matrix<G>(smem, ps, s, slot, 1, p.hidden, idx, 0u, true, SmemLayout::xdig, SmemLayout::xsumw,
+                             SmemLayout::xinv, dead, status);
       if (++idx >= s.inter / 16) {
         idx = 0;
         ++slot;
@@ -593,9 +572,12 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem) {
   // phase 2: down rows of every slot for the output row blocks of this CTA
   for (int n = 0; n < plan.count2 && ok; ++n) {
     const int rb = blockIdx.x + n * gridDim.x;
-    for (int slot = 0; slot < plan.nslots && ok; ++slot)
-      ok = produce_matrix<G>(smem, ps, slots[slot], slot, 2, slots[slot].inter, rb, kFlagPhase2, slot == plan.nslots - 1,
-                             dead, status);
+    for (int slot = 0; slot < plan.nslots && ok; ++slot) {
+      const Slot& s = slots[slot];
+      ok = produce_matrix<G>(smem, ps, s, slot, 2, s.inter, rb, kFlagPhase2, slot == plan.nslots - 1,
+                             SmemLayout::hdig + (uint32_t)s.hoff * 4u, SmemLayout::hsumw + (uint32_t)(s.hoff >> LG) * 8u,
+                             SmemLayout::hinv + (uint32_t)(s.hoff >> 7) * 4u, dead, status);
+    }
   }
   if (ok) {
     const int stage = ps.it % kStages;
@@ -616,122 +598,45 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem) {
   }
 }
 
-// ---- the kernel ------------------------------------------------------------------------------------
-template <int G>
-__global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_constant__ DecodeParams p) {
-  extern __shared__ __align__(128) uint8_t smem[];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+// ---- prologue pieces ---------------------------------------------------------------------------------
+// Warp 0: the routing list -> slot table -> plane pointers -> the static partition.
+__device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
   Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
   Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
-  int* dead = reinterpret_cast<int*>(smem + SmemLayout::dead);
-  int32_t* in_ids = reinterpret_cast<int32_t*>(smem + SmemLayout::stage_in);
-  float* in_w = reinterpret_cast<float*>(in_ids + SLICEMOE_MAX_TOP_K);
-  int32_t* in_prec = reinterpret_cast<int32_t*>(in_w + SLICEMOE_MAX_TOP_K);
-  float* in_gate = reinterpret_cast<float*>(in_prec + SLICEMOE_MAX_TOP_K);
-  unsigned* in_xmax = reinterpret_cast<unsigned*>(in_gate + 1);
-
-  // ---- step 1: every independent global read at once: x (kept in registers), the routing list ----
-  // thread t owns x[4t .. 4t+3] (and 4(t + kThreads) ...): hidden <= kMaxHidden = 4 * 4 * kThreads is checked on the host
-  constexpr int kXIt = (kMaxHidden / 4 + kThreads - 1) / kThreads;
-  float xv[kXIt][4];
-  float xmax = 0.f;
-#pragma unroll
-  for (int it = 0; it < kXIt; ++it) {
-    const int i = it * kThreads + tid;
-    if (4 * i < p.hidden) {
-      const uint2 raw = *reinterpret_cast<const uint2*>(p.x + 4 * i);
-      xv[it][0] = __uint_as_float(raw.x << 16);
-      xv[it][1] = __uint_as_float(raw.x & 0xffff0000u);
-      xv[it][2] = __uint_as_float(raw.y << 16);
-      xv[it][3] = __uint_as_float(raw.y & 0xffff0000u);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float a = fabsf(xv[it][j]);
-        if (a == a) xmax = fmaxf(xmax, a);
-      }
-    }
+  // routed experts: lane j reads entry j of the list; out-of-range ids are dropped and reported
+  int e = -1, pr = 0;
+  float w = 0.f;
+  if (lane < p.k) {
+    e = p.ids[lane];
+    pr = p.prec[lane];
+    w = p.weights[lane];
   }
-  if (tid < p.k) {
-    in_ids[tid] = p.ids[tid];
-    in_w[tid] = p.weights[tid];
-    in_prec[tid] = p.prec[tid];
+  const bool valid = lane < p.k && e >= 0 && e < p.n_experts;
+  const unsigned vmask = __ballot_sync(0xffffffffu, valid);
+  if (lane < p.k && !valid) atomicOr(&p.ws->status, (unsigned)SLICEMOE_STATUS_BAD_EXPERT_ID);
+  const int nrouted = __popc(vmask);
+  const int nslots = nrouted + p.n_shared;
+  if (valid) {
+    Slot& s = slots[__popc(vmask & ((1u << lane) - 1u))];
+    s.src = p.experts + e;
+    s.inter = p.inter;
+    s.prec = pr != 0;
+    s.coef = w;
+    s.gated = 0;
+    s.hoff = __popc(vmask & ((1u << lane) - 1u)) * p.inter;
   }
-  if (tid == kThreads - 1) {
-    *dead = 0;
-    *in_xmax = 0u;
-    const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(bars + 8 * s, 1);                             // full: producer's expect_tx arrive
-      mbar_init(bars + 8 * kStages + 8 * s, kConsumerWarps);  // empty: one arrive per consumer warp
-    }
-    const uint32_t xbars = bars + 16 * kStages;
-    mbar_init(xbars + 8 * kBarPFull0, kConsumerWarps);
-    mbar_init(xbars + 8 * kBarPFull1, kConsumerWarps);
-    mbar_init(xbars + 8 * kBarPEmpty0, 1);
-    mbar_init(xbars + 8 * kBarPEmpty1, 1);
-    mbar_init(xbars + 8 * kBarHxArrive, kConsumerWarps);
-    mbar_init(xbars + 8 * kBarHxGo, 1);
-    mbar_init(xbars + 8 * kBarHsReady, kConsumerWarps);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (lane < p.n_shared) {
+    Slot& s = slots[nrouted + lane];
+    s.src = p.shared + lane;
+    s.inter = p.shared_inter;
+    s.prec = 1;
+    s.coef = 1.f;
+    s.gated = p.sigmoid_gate;
+    s.hoff = nrouted * p.inter + lane * p.shared_inter;
   }
-  __syncthreads();
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) xmax = fmaxf(xmax, __shfl_xor_sync(0xffffffffu, xmax, off));
-  if (lane == 0) atomicMax(in_xmax, __float_as_uint(xmax));
-
-  // ---- step 2: slot list (thread 0); the shared-expert gate (last warp) ----
-  if (tid == 0) {
-    int n = 0, hoff = 0;
-    for (int j = 0; j < p.k; ++j) {
-      const int e = in_ids[j];
-      if (e < 0 || e >= p.n_experts) {
-        atomicOr(&p.ws->status, (unsigned)SLICEMOE_STATUS_BAD_EXPERT_ID);
-        continue;
-      }
-      Slot& s = slots[n];
-      s.src = p.experts + e;
-      s.inter = p.inter;
-      s.prec = in_prec[j] != 0;
-      s.coef = in_w[j];
-      s.gated = 0;
-      s.hoff = hoff;
-      s.hinv = 0.f;
-      hoff += p.inter;
-      ++n;
-    }
-    for (int j = 0; j < p.n_shared; ++j) {
-      Slot& s = slots[n];
-      s.src = p.shared + j;
-      s.inter = p.shared_inter;
-      s.prec = 1;
-      s.coef = 1.f;
-      s.gated = p.sigmoid_gate;
-      s.hoff = hoff;
-      s.hinv = 0.f;
-      hoff += p.shared_inter;
-      ++n;
-    }
-    plan->nslots = n;
-    plan->htotal = hoff;
-  } else if (warp == kProducerWarp && p.sigmoid_gate && p.n_shared > 0) {
-    // Qwen-style shared-expert gate: sigmoid(v . x)
-    float dot = 0.f;
-    for (int i = lane; i < p.hidden / 2; i += 32) {
-      const uint32_t raw = *reinterpret_cast<const uint32_t*>(p.x + 2 * i);
-      const float2 gv = __ldg(reinterpret_cast<const float2*>(p.gate_vec) + i);
-      dot = fmaf(gv.x, __uint_as_float(raw << 16), dot);
-      dot = fmaf(gv.y, __uint_as_float(raw & 0xffff0000u), dot);
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
-    if (lane == 0) *in_gate = 1.f / (1.f + expf(-dot));
-  }
-  __syncthreads();
-
-  // ---- step 3: the slots' plane pointers, one 8-byte load per thread; x -> fixed-point digits ----
-  const int nslots = plan->nslots;
-  for (int i = tid; i < nslots * 12; i += kThreads) {
+  __syncwarp();
+  // plane pointers: one 8-byte load per (slot, matrix, field)
+  for (int i = lane; i < nslots * 12; i += 32) {
     const int s = i / 12, q = i % 12, m = q >> 2, f = q & 3;
     const slicemoe_mat* mat = reinterpret_cast<const slicemoe_mat*>(slots[s].src) + m;
     const void* ptr = *(reinterpret_cast<const void* const*>(mat) + f);
@@ -740,110 +645,128 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
     else if (f == 2) slots[s].sc[m] = reinterpret_cast<const uint16_t*>(ptr);
     else slots[s].zp[m] = reinterpret_cast<const uint8_t*>(ptr);
   }
-  {
-    float xscale, xinv;
-    fixed_scale(*in_xmax, &xscale, &xinv);
-    if (tid == 0) plan->xinv = xinv;
-    uint8_t* xdig = smem + SmemLayout::xdig;
-    float* xsumw = reinterpret_cast<float*>(smem + SmemLayout::xsumw);
-    constexpr int lanes_per_group = G / 4;
+  __syncwarp();
+  // lane j owns slot j: a slot without LSB planes runs MSB-only; stages and tasks per slot
+  int nt = 0, sp = 0;
+  if (lane < nslots) {
+    Slot& s = slots[lane];
+    if (!(s.lsb[0] && s.lsb[1] && s.lsb[2])) s.prec = 0;
+    nt = s.inter / 16;
+    sp = slot_spt1(s, p.hidden);
+  }
+  unsigned cs = (unsigned)(nt * sp), ct = (unsigned)nt;  // inclusive scans over the slots
 #pragma unroll
-    for (int it = 0; it < kXIt; ++it) {
-      const int i = it * kThreads + tid;
-      if (4 * (it * kThreads + (tid & ~31)) < p.hidden) {  // uniform per warp (hidden % 128 == 0)
-        const int k = 4 * i;
-        uint32_t dw[3];
-        int ds[3] = {0, 0, 0};
-        to_digits4(xv[it], xscale, dw, ds);
-#pragma unroll
-        for (int t = 0; t < 3; ++t) *reinterpret_cast<uint32_t*>(xdig + digit_offset(k, t)) = dw[t];
-        *reinterpret_cast<uint32_t*>(xdig + digit_offset(k, 3)) = 0u;
-#pragma unroll
-        for (int off = 1; off < lanes_per_group; off <<= 1) {
-          ds[0] += __shfl_xor_sync(0xffffffffu, ds[0], off);
-          ds[1] += __shfl_xor_sync(0xffffffffu, ds[1], off);
-          ds[2] += __shfl_xor_sync(0xffffffffu, ds[2], off);
-        }
-        if ((lane & (lanes_per_group - 1)) == 0) {
-          xsumw[(k / G) * 2 + 0] = (float)ds[0] + 256.f * (float)ds[1];
-          xsumw[(k / G) * 2 + 1] = 65536.f * (float)ds[2];
-        }
-      }
+  for (int off = 1; off < 32; off <<= 1) {
+    const unsigned a = __shfl_up_sync(0xffffffffu, cs, off), b = __shfl_up_sync(0xffffffffu, ct, off);
+    if (lane >= off) {
+      cs += a;
+      ct += b;
     }
   }
-  __syncthreads();
+  const unsigned S = __shfl_sync(0xffffffffu, cs, 31);
+  const unsigned NT = __shfl_sync(0xffffffffu, ct, 31);
+  // phase 1: equal shares of ring stages, at task granularity: the tasks whose first stage lies in [lo, hi)
+  const unsigned lo = (blockIdx.x * S + gridDim.x - 1) / gridDim.x;
+  const unsigned hi = ((blockIdx.x + 1) * S + gridDim.x - 1) / gridDim.x;
+  const unsigned off_s = cs - (unsigned)(nt * sp), off_t = ct - (unsigned)nt;  // exclusive
+  unsigned ord_lo = NT, ord_hi = NT;
+  int slot_lo = nslots, idx_lo = 0;
+  if (lane < nslots && nt > 0) {
+    if (lo >= off_s && lo < cs) {
+      const unsigned i = (lo - off_s + sp - 1) / sp;  // may equal nt: then it is the next slot's first task
+      ord_lo = off_t + i;
+      slot_lo = lane;
+      idx_lo = (int)i;
+    }
+    if (hi >= off_s && hi < cs) ord_hi = off_t + (hi - off_s + sp - 1) / sp;
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {  // at most one lane holds each answer
+    const unsigned o = __shfl_xor_sync(0xffffffffu, ord_lo, off);
+    const int sl2 = __shfl_xor_sync(0xffffffffu, slot_lo, off), ix2 = __shfl_xor_sync(0xffffffffu, idx_lo, off);
+    if (sl2 < slot_lo) {
+      ord_lo = o;
+      slot_lo = sl2;
+      idx_lo = ix2;
+    }
+    ord_hi = min(ord_hi, __shfl_xor_sync(0xffffffffu, ord_hi, off));
+  }
+  if (lane == 0) {
+    if (slot_lo < nslots && idx_lo >= slots[slot_lo].inter / 16) {  // the bound fell on the slot's end
+      idx_lo = 0;
+      ++slot_lo;
+    }
+    plan->first_slot = slot_lo;
+    plan->first_idx = idx_lo;
+    plan->count1 = (int)(ord_hi - ord_lo);
+    const int nrb = p.hidden / 16;
+    plan->count2 = (nslots > 0 && (int)blockIdx.x < nrb) ? (nrb - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    plan->nslots = nslots;
+    plan->htotal = nrouted * p.inter + p.n_shared * p.shared_inter;
+  }
+}
 
-  // ---- step 4: precision fix-up and the static partition (warp 0: lane j owns slot j) ----
+// ---- the kernel ------------------------------------------------------------------------------------
+template <int G>
+__global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_constant__ DecodeParams p) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
+
+  // Prologue, all roles in parallel and one barrier at the end: warp 0 builds the slot table and the
+  // partition (two dependent global reads: the routing list, then the experts' plane pointers); the other
+  // warps turn x into digits, one 128-element block per warp; the last warp sets up the barriers and the
+  // shared-expert gate.
   if (warp == 0) {
-    int nt = 0, sp = 0;
-    if (lane < nslots) {
-      Slot& s = slots[lane];
-      if (!(s.lsb[0] && s.lsb[1] && s.lsb[2])) s.prec = 0;
-      if (s.gated) s.coef = *in_gate;
-      nt = s.inter / 16;
-      sp = slot_spt1(s, p.hidden);
-    }
-    // inclusive scans of stages and tasks over the slots
-    unsigned cs = (unsigned)(nt * sp), ct = (unsigned)nt;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const unsigned a = __shfl_up_sync(0xffffffffu, cs, off), b = __shfl_up_sync(0xffffffffu, ct, off);
-      if (lane >= off) {
-        cs += a;
-        ct += b;
-      }
-    }
-    const unsigned S = __shfl_sync(0xffffffffu, cs, 31);
-    const unsigned NT = __shfl_sync(0xffffffffu, ct, 31);
-    // phase 1: equal shares of ring stages, at task granularity: the tasks whose first stage lies in [lo, hi)
-    const unsigned lo = (blockIdx.x * S + gridDim.x - 1) / gridDim.x;
-    const unsigned hi = ((blockIdx.x + 1) * S + gridDim.x - 1) / gridDim.x;
-    const unsigned off_s = cs - (unsigned)(nt * sp), off_t = ct - (unsigned)nt;  // exclusive
-    // ordinal of the first task at or after a bound, seen from the slot that contains it
-    unsigned ord_lo = NT, ord_hi = NT;
-    int slot_lo = nslots, idx_lo = 0;
-    if (lane < nslots && nt > 0) {
-      if (lo < cs && (lo >= off_s || lane == 0)) {
-        const unsigned i = lo <= off_s ? 0u : (lo - off_s + sp - 1) / sp;
-        ord_lo = off_t + i;  // i may equal nt: then it is the first task of the next slot
-        slot_lo = lane;
-        idx_lo = (int)i;
-      }
-      if (hi < cs && (hi >= off_s || lane == 0)) {
-        const unsigned i = hi <= off_s ? 0u : (hi - off_s + sp - 1) / sp;
-        ord_hi = off_t + i;
-      }
-    }
-    // exactly one lane (or none, when the bound is past the end) holds each answer
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-      const unsigned o = __shfl_xor_sync(0xffffffffu, ord_lo, off);
-      const int sl2 = __shfl_xor_sync(0xffffffffu, slot_lo, off), ix2 = __shfl_xor_sync(0xffffffffu, idx_lo, off);
-      if (sl2 < slot_lo) {
-        ord_lo = o;
-        slot_lo = sl2;
-        idx_lo = ix2;
-      }
-      ord_hi = min(ord_hi, __shfl_xor_sync(0xffffffffu, ord_hi, off));
-    }
+    build_plan(p, smem, lane);
+  } else if (warp == kProducerWarp) {
     if (lane == 0) {
-      if (slot_lo < nslots && idx_lo >= slots[slot_lo].inter / 16) {  // bound fell on the slot's end
-        idx_lo = 0;
-        ++slot_lo;
+      *reinterpret_cast<int*>(smem + SmemLayout::dead) = 0;
+      const uint32_t bars = smem_u32(smem + SmemLayout::bars);
+      for (int s = 0; s < kStages; ++s) {
+        mbar_init(bars + 8 * s, 1);                             // full: producer's expect_tx arrive
+        mbar_init(bars + 8 * kStages + 8 * s, kConsumerWarps);  // empty: one arrive per consumer warp
       }
-      plan->first_slot = slot_lo;
-      plan->first_idx = idx_lo;
-      plan->count1 = (int)(ord_hi - ord_lo);
-      const int nrb = p.hidden / 16;
-      plan->count2 = (nslots > 0 && (int)blockIdx.x < nrb) ? (nrb - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+      const uint32_t xbars = bars + 16 * kStages;
+      mbar_init(xbars + 8 * kBarPFull0, kConsumerWarps);
+      mbar_init(xbars + 8 * kBarPFull1, kConsumerWarps);
+      mbar_init(xbars + 8 * kBarPEmpty0, 1);
+      mbar_init(xbars + 8 * kBarPEmpty1, 1);
+      mbar_init(xbars + 8 * kBarHxGo, 1);
+      mbar_init(xbars + 8 * kBarHsReady, kConsumerWarps);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (p.sigmoid_gate && p.n_shared > 0) {
+      // Qwen-style shared-expert gate: sigmoid(v . x)
+      float dot = 0.f;
+      for (int i = lane; i < p.hidden / 2; i += 32) {
+        const uint32_t raw = *reinterpret_cast<const uint32_t*>(p.x + 2 * i);
+        const float2 gv = __ldg(reinterpret_cast<const float2*>(p.gate_vec) + i);
+        dot = fmaf(gv.x, __uint_as_float(raw << 16), dot);
+        dot = fmaf(gv.y, __uint_as_float(raw & 0xffff0000u), dot);
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+      if (lane == 0) plan->gate = 1.f / (1.f + expf(-dot));
+    }
+  } else {
+    for (int blk = warp - 1; blk < p.hidden / 128; blk += kConsumerWarps) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(p.x + blk * 128 + 4 * lane);
+      const float v[4] = {__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u),
+                          __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u)};
+      block_to_digits<G>(v, blk * 128, lane, smem + SmemLayout::xdig, reinterpret_cast<float*>(smem + SmemLayout::xsumw),
+                         reinterpret_cast<float*>(smem + SmemLayout::xinv));
     }
   }
-  if (nslots == 0 && blockIdx.x == 0)
-    for (int i = tid; i < p.hidden; i += kThreads) p.y[i] = 0.f;
   __syncthreads();
+  if (plan->nslots == 0 && blockIdx.x == 0)
+    for (int i = tid; i < p.hidden; i += kThreads) p.y[i] = 0.f;
 
   if (warp < kConsumerWarps) {
     consumer_loop<G>(p, smem, warp, lane);
+  } else if (warp == kEpilogueWarp) {
+    epilogue_loop(p, smem, lane);
   } else if (lane == 0) {
     producer_loop<G>(p, smem);
   }
@@ -853,7 +776,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
     if (old == gridDim.x - 1) {  // everyone is past the barrier: make the header reusable
       p.ws->bar_arrive = 0;
       p.ws->depart = 0;
-      for (int j = 0; j < kMaxSlots; ++j) p.ws->hmax[j] = 0u;
       __threadfence();
     }
   }
