@@ -3,11 +3,12 @@
 //
 // The work is a pure weight stream: every plane byte is used once, so the bound is HBM bandwidth and
 // everything else is arranged so that the stream never stops.
-//   * One CTA per SM: 16 consumer warps, one epilogue warp, one producer thread.  The producer streams
-//     16-row x <=2048-column plane tiles (<=16 KB, one contiguous run each thanks to the tiled layout)
-//     plus their scales / zero-points into a shared-memory ring with cp.async.bulk + mbarriers.  It
-//     never waits for the gate/up -> down dependency, so down-projection tiles are already in flight
-//     (up to the whole ring) while the grid exchanges h.
+//   * One CTA per SM: 16 consumer warps, one epilogue warp, one producer warp (4 lanes, one per bulk
+//     copy of a chunk).  The producer streams chunks - 16 rows x <=2048 columns: the MSB plane tile,
+//     the LSB plane tile when the expert runs at 8 bits (<=16 KB each, one contiguous run thanks to the
+//     tiled layout), scales and zero-points - into a ring of eight 16 KB units with cp.async.bulk +
+//     mbarriers.  It never waits for the gate/up -> down dependency, so down-projection tiles are
+//     already in flight (up to the whole ring) while the grid exchanges h.
 //   * Integer arithmetic on the tensor pipe.  The activation vector (x, later h) is converted once,
 //     per 128-element block, to fixed point relative to the block's largest magnitude and split into
 //     three balanced base-256 digits (int8).  The digits sit in separate columns of the B operand of
@@ -36,12 +37,12 @@ constexpr int kConsumerWarps = 16;
 constexpr int kEpilogueWarp = kConsumerWarps;
 constexpr int kProducerWarp = kConsumerWarps + 1;
 constexpr int kThreads = 32 * (kConsumerWarps + 2);
-constexpr int kStages = 7;
-constexpr int kChunkK = 128 * kConsumerWarps;              // K columns per ring stage: one 128-column block per warp
-constexpr int kPlaneStageBytes = 16 * kChunkK / 2;         // 16384
-constexpr int kScaleStageBytes = 16 * (kChunkK / 32) * 2;  // 2048 (group 32 is the worst case)
-constexpr int kZpStageBytes = 16 * (kChunkK / 32);         // 1024
-constexpr int kStageBytes = kPlaneStageBytes + kScaleStageBytes + kZpStageBytes;  // 19456
+constexpr int kUnits = 8;                                 // ring units; a chunk takes one per plane
+constexpr int kChunkK = 128 * kConsumerWarps;             // K columns per chunk: one 128-column block per warp
+constexpr int kPlaneUnitBytes = 16 * kChunkK / 2;         // 16384
+constexpr int kScaleUnitBytes = 16 * (kChunkK / 32) * 2;  // 2048 (group 32 is the worst case)
+constexpr int kZpUnitBytes = 16 * (kChunkK / 32);         // 1024
+constexpr int kUnitBytes = kPlaneUnitBytes + kScaleUnitBytes + kZpUnitBytes;  // 19456
 constexpr int kMaxSlots = SLICEMOE_MAX_TOP_K + SLICEMOE_MAX_SHARED;
 constexpr int kMaxHidden = 4096;
 constexpr int kHCap = 12288;  // sum of intermediate widths over all slots of a layer
@@ -97,18 +98,16 @@ struct Slot {
   int pad_;
 };
 
-// One ring stage as the consumers see it (16 bytes, written by the producer):
+// One chunk as the consumers see it (16 bytes, written by the producer):
 //   x: flags | nblocks << 8 | rot << 16 | slot << 24
 //   y: byte offset in shared memory of the activation digits of the chunk's first column
 //   z: byte offset in shared memory of the chunk's first (group, digit-pair) weighted digit sum
 //   w: byte offset in shared memory of the chunk's first per-128-block inverse scale
 enum : uint32_t {
-  kFlagLsb = 1,           // this stage carries the LSB plane of the chunk (accumulate onto 16 x MSB sums)
-  kFlagMeta = 2,          // last plane of the chunk: scales / zero-points are in the stage; fold the chunk
   kFlagLastOfMatrix = 4,  // last chunk of the matrix row block
   kFlagLastOfTask = 8,    // last matrix of the task: hand the partial rows to the epilogue warp
   kFlagEnd = 16,          // sentinel, no data
-  kFlagPrec8 = 32,
+  kFlagPrec8 = 32,        // two units: MSB plane, then LSB plane (sums combine as 16 Cm + Cl)
   kFlagPhase2 = 64,
 };
 
@@ -124,18 +123,18 @@ struct Plan {
 struct SmemLayout {
   // offsets into dynamic shared memory
   static constexpr int ring = 0;
-  static constexpr int hdig = ring + kStages * kStageBytes;  // int8 [kHCap/32][4 digits][32]
-  static constexpr int xdig = hdig + kHCap * 4;              // int8 [kMaxHidden/32][4][32]
-  static constexpr int hsumw = xdig + kMaxHidden * 4;        // float [kHCap/32][2]: weighted digit sums per group
+  static constexpr int hdig = ring + kUnits * kUnitBytes;    // int8 [kHCap/32][3 digits][32]
+  static constexpr int xdig = hdig + kHCap * 3;              // int8 [kMaxHidden/32][3][32]
+  static constexpr int hsumw = xdig + kMaxHidden * 3;        // float [kHCap/32][2]: weighted digit sums per group
   static constexpr int xsumw = hsumw + (kHCap / 32) * 8;     // float [kMaxHidden/32][2]
   static constexpr int hinv = xsumw + (kMaxHidden / 32) * 8;  // float [kHCap/128]: 2^-e of each 128-block of h
   static constexpr int xinv = hinv + (kHCap / 128) * 4;       // float [kMaxHidden/128]
   static constexpr int partial = xinv + (kMaxHidden / 128) * 4;  // float [2][warps][16][2]
   static constexpr int slots = partial + 2 * kConsumerWarps * 16 * 2 * 4;
-  static constexpr int desc = slots + kMaxSlots * (int)sizeof(Slot);  // uint4 [kStages]
-  static constexpr int plan = desc + kStages * 16;
+  static constexpr int desc = slots + kMaxSlots * (int)sizeof(Slot);  // uint4 [kUnits]
+  static constexpr int plan = desc + kUnits * 16;
   static constexpr int bars = (plan + (int)sizeof(Plan) + 15) & ~15;  // uint64 barriers
-  static constexpr int nbars = 2 * kStages + 6;
+  static constexpr int nbars = 2 * kUnits + 6;
   static constexpr int dead = bars + nbars * 8;
   static constexpr int total = dead + 16;
 };
@@ -145,7 +144,8 @@ static_assert(SmemLayout::slots % 8 == 0 && SmemLayout::hdig % 16 == 0 && SmemLa
                   SmemLayout::desc % 16 == 0 && SmemLayout::plan % 8 == 0,
               "alignment");
 
-// barrier indices after the 2*kStages ring barriers
+// Ring barriers: full[c % kUnits] for chunk number c (armed with the chunk's bytes), empty[u] for unit u
+// (one arrive per consumer warp).  Barrier indices after the 2 * kUnits ring barriers:
 enum { kBarPFull0 = 0, kBarPFull1, kBarPEmpty0, kBarPEmpty1, kBarHxGo, kBarHsReady };
 
 // ---- PTX helpers -------------------------------------------------------------------------------
@@ -209,10 +209,10 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
 
 // ---- fixed-point activations ---------------------------------------------------------------------
 // Byte offset, inside a digit buffer, of digit t of the four values k..k+3 (k % 4 == 0): steps of 32
-// columns, 4 digit rows of 32 bytes (the fourth stays zero), and inside a row the order in which the B
-// fragment of m16n8k32 wants them: (k % 16) / 4 selects the lane quad position, (k % 32) / 16 the register.
+// columns, 3 digit rows of 32 bytes, and inside a row the order in which the B fragment of m16n8k32 wants
+// them: (k % 16) / 4 selects the lane quad position, (k % 32) / 16 the register.
 __device__ __forceinline__ int digit_offset(int k, int t) {
-  return (k >> 5) * 128 + t * 32 + ((k >> 2) & 3) * 8 + ((k >> 4) & 1) * 4;
+  return (k >> 5) * 96 + t * 32 + ((k >> 2) & 3) * 8 + ((k >> 4) & 1) * 4;
 }
 
 // One warp converts one 128-element block (lane L holds elements 4L..4L+3 of the block, whose first
@@ -222,15 +222,14 @@ __device__ __forceinline__ int digit_offset(int k, int t) {
 template <int G>
 __device__ __forceinline__ void block_to_digits(const float (&v)[4], int k0, int lane, uint8_t* dig, float* sumw,
                                                 float* inv) {
-  float m = 0.f;
+  unsigned mb = 0u;  // bit pattern of max |v|: non-negative floats order like their bit patterns
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    const float a = fabsf(v[j]);
-    if (a == a) m = fmaxf(m, a);  // a NaN input gives an undefined result, never a fault
+    const unsigned a = __float_as_uint(v[j]) & 0x7fffffffu;
+    if (a <= 0x7f800000u) mb = max(mb, a);  // a NaN input gives an undefined result, never a fault
   }
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-  const int ex = (int)((__float_as_uint(m) >> 23) & 0xffu) - 127;  // floor(log2 m) for normal numbers
+  mb = __reduce_max_sync(0xffffffffu, mb);
+  const int ex = (int)(mb >> 23) - 127;  // floor(log2 max) for normal numbers
   const int e = max(-100, min(100, 21 - ex));
   const float scale = __uint_as_float((unsigned)(127 + e) << 23);
   uint32_t dw[3] = {0u, 0u, 0u};
@@ -253,14 +252,12 @@ __device__ __forceinline__ void block_to_digits(const float (&v)[4], int k0, int
   const int k = k0 + 4 * lane;
 #pragma unroll
   for (int t = 0; t < 3; ++t) *reinterpret_cast<uint32_t*>(dig + digit_offset(k, t)) = dw[t];
-  *reinterpret_cast<uint32_t*>(dig + digit_offset(k, 3)) = 0u;
   constexpr int lanes_per_group = G / 4;  // 8, 16 or 32 consecutive lanes cover one group
-#pragma unroll
-  for (int off = 1; off < lanes_per_group; off <<= 1) {
-    ds[0] += __shfl_xor_sync(0xffffffffu, ds[0], off);
-    ds[1] += __shfl_xor_sync(0xffffffffu, ds[1], off);
-    ds[2] += __shfl_xor_sync(0xffffffffu, ds[2], off);
-  }
+  const unsigned gmask = lanes_per_group == 32 ? 0xffffffffu
+                                               : ((1u << lanes_per_group) - 1u) << (lane & ~(lanes_per_group - 1));
+  ds[0] = __reduce_add_sync(gmask, ds[0]);
+  ds[1] = __reduce_add_sync(gmask, ds[1]);
+  ds[2] = __reduce_add_sync(gmask, ds[2]);
   if ((lane & (lanes_per_group - 1)) == 0) {
     sumw[(k / G) * 2 + 0] = (float)ds[0] + 256.f * (float)ds[1];
     sumw[(k / G) * 2 + 1] = 65536.f * (float)ds[2];
@@ -270,7 +267,7 @@ __device__ __forceinline__ void block_to_digits(const float (&v)[4], int k0, int
 
 // ---- task enumeration (identical in every role) ---------------------------------------------------
 __device__ __forceinline__ int nchunks_of(int K) { return (K + kChunkK - 1) / kChunkK; }
-// ring stages of one phase-1 task (gate + up of a 16-row block) of a slot
+// ring units of one phase-1 task (gate + up of a 16-row block) of a slot
 __device__ __forceinline__ int slot_spt1(const Slot& s, int hidden) { return 2 * (s.prec ? 2 : 1) * nchunks_of(hidden); }
 
 // ---- consumers -----------------------------------------------------------------------------------
@@ -313,7 +310,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
   float* partial = reinterpret_cast<float*>(smem + SmemLayout::partial);
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t full0 = bars, empty0 = bars + 8 * kStages, xbars = bars + 16 * kStages;
+  const uint32_t full0 = bars, empty0 = bars + 8 * kUnits, xbars = bars + 16 * kUnits;
   const uint32_t pfull0 = xbars + 8 * kBarPFull0, pempty0 = xbars + 8 * kBarPEmpty0;
   unsigned* status = &p.ws->status;
 
@@ -326,60 +323,73 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
   const int cq = c & 1;
   const float rowfix = (c >> 1) ? 0.0625f : 1.f;
   const float w0 = (cq ? 65536.f : 1.f) * rowfix, w1 = (cq ? 0.f : 256.f) * rowfix;
-  const int boff = (g8 & 3) * 32 + c * 8;  // digit row = column of B this lane feeds
+  // B column n = g8 takes digit n % 4; the fourth is unused, so those lanes re-read digit 0 and are ignored
+  const int boff = ((g8 & 3) == 3 ? 0 : (g8 & 3)) * 32 + c * 8;
   int acc[SG][4];
   float rowacc = 0.f, part0 = 0.f, part1 = 0.f;
   bool fetched = false;
   int taskcount = 0;
+  int unit = 0;  // running unit counter
 
-  for (int it = 0;; ++it) {
-    const int stage = it % kStages;
-    if (!mbar_wait(full0 + 8 * stage, (it / kStages) & 1, dead, status)) return;
-    const uint4 d = descs[stage];
+  for (int cn = 0;; ++cn) {  // chunk number
+    if (!mbar_wait(full0 + 8 * (cn % kUnits), (cn / kUnits) & 1, dead, status)) return;
+    const uint4 d = descs[cn % kUnits];
     const uint32_t flags = d.x & 0xffu;
     if (flags & kFlagEnd) break;
     if ((flags & kFlagPhase2) && !fetched) {
       if (!fetch_h<G>(p, smem, warp, lane, plan.htotal, dead, status, xbars)) return;
       fetched = true;
     }
+    const bool p8 = (flags & kFlagPrec8) != 0;
+    const int u0 = unit % kUnits, u1 = (unit + 1) % kUnits;
     // the 128-column block of this chunk handled by this warp
     int b = warp - (int)((d.x >> 16) & 0xffu);
     if (b < 0) b += kConsumerWarps;
-    const bool valid = b < (int)((d.x >> 8) & 0xffu);
-    if (valid) {
-      if (!(flags & kFlagLsb)) {
+    if (b < (int)((d.x >> 8) & 0xffu)) {
 #pragma unroll
-        for (int sg = 0; sg < SG; ++sg)
+      for (int sg = 0; sg < SG; ++sg)
 #pragma unroll
-          for (int q = 0; q < 4; ++q) acc[sg][q] = 0;
-      } else {
+        for (int q = 0; q < 4; ++q) acc[sg][q] = 0;
+      const uint8_t* bp = smem + d.y + b * 384 + boff;
+      const uint2 bv0 = *reinterpret_cast<const uint2*>(bp);
+      const uint2 bv1 = *reinterpret_cast<const uint2*>(bp + 96);
+      const uint2 bv2 = *reinterpret_cast<const uint2*>(bp + 192);
+      const uint2 bv3 = *reinterpret_cast<const uint2*>(bp + 288);
+      const uint8_t* ap = smem + SmemLayout::ring + u0 * kUnitBytes + b * 1024 + lane * 16;
+      {
+        const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
+        const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
+        mma_u8s8(acc[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
+        mma_u8s8(acc[32 / G], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x,
+                 bv1.y);
+        mma_u8s8(acc[64 / G], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x,
+                 bv2.y);
+        mma_u8s8(acc[96 / G], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x,
+                 bv3.y);
+      }
+      if (p8) {
+        const uint8_t* ap2 = smem + SmemLayout::ring + u1 * kUnitBytes + b * 1024 + lane * 16;
+        const uint4 wlo = *reinterpret_cast<const uint4*>(ap2);
+        const uint4 whi = *reinterpret_cast<const uint4*>(ap2 + 512);
 #pragma unroll
         for (int sg = 0; sg < SG; ++sg)
 #pragma unroll
           for (int q = 0; q < 4; ++q) acc[sg][q] <<= 4;
+        mma_u8s8(acc[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
+        mma_u8s8(acc[32 / G], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x,
+                 bv1.y);
+        mma_u8s8(acc[64 / G], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x,
+                 bv2.y);
+        mma_u8s8(acc[96 / G], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x,
+                 bv3.y);
       }
-      const uint8_t* ap = smem + SmemLayout::ring + stage * kStageBytes + b * 1024 + lane * 16;
-      const uint8_t* bp = smem + d.y + b * 512 + boff;
-      const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
-      const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
-      const uint2 bv0 = *reinterpret_cast<const uint2*>(bp);
-      const uint2 bv1 = *reinterpret_cast<const uint2*>(bp + 128);
-      const uint2 bv2 = *reinterpret_cast<const uint2*>(bp + 256);
-      const uint2 bv3 = *reinterpret_cast<const uint2*>(bp + 384);
-      mma_u8s8(acc[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
-      mma_u8s8(acc[32 / G], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x,
-               bv1.y);
-      mma_u8s8(acc[64 / G], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x,
-               bv2.y);
-      mma_u8s8(acc[96 / G], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x,
-               bv3.y);
-      if (flags & kFlagMeta) {
-        const uint8_t* stg = smem + SmemLayout::ring + stage * kStageBytes;
-        const uint16_t* ms = reinterpret_cast<const uint16_t*>(stg + kPlaneStageBytes) + (b * SG) * 16 + r;
-        const uint8_t* mz = stg + kPlaneStageBytes + kScaleStageBytes + (b * SG) * 16 + r;
+      // fold: scales / zero-points travel in the first unit of the chunk
+      {
+        const uint8_t* meta = smem + SmemLayout::ring + u0 * kUnitBytes + kPlaneUnitBytes;
+        const uint16_t* ms = reinterpret_cast<const uint16_t*>(meta) + (b * SG) * 16 + r;
+        const uint8_t* mz = meta + kScaleUnitBytes + (b * SG) * 16 + r;
         const float* sumw = reinterpret_cast<const float*>(smem + d.z) + (b * SG) * 2 + cq;
         const float binv = *(reinterpret_cast<const float*>(smem + d.w) + b);
-        const bool p8 = (flags & kFlagPrec8) != 0;
         const float sfix = p8 ? binv : 16.f * binv;
         const int zsh = p8 ? 0 : 4;
 #pragma unroll
@@ -387,15 +397,19 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
           const int ca = (c >> 1) ? acc[sg][2] : acc[sg][0];
           const int cb = (c >> 1) ? acc[sg][3] : acc[sg][1];
           const float t = fmaf((float)cb, w1, (float)ca * w0);
-          const float s = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
+          const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
           const float z = (float)((int)mz[sg * 16] >> zsh);
           // both slices: s (16 Cm + Cl - zp X); MSB only: 16 s (Cm - (zp >> 4) X)
-          rowacc = fmaf(s, fmaf(-z, sumw[sg * 2], t), rowacc);
+          rowacc = fmaf(sc, fmaf(-z, sumw[sg * 2], t), rowacc);
         }
       }
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(empty0 + 8 * stage);
+    if (lane == 0) {
+      mbar_arrive(empty0 + 8 * u0);
+      if (p8) mbar_arrive(empty0 + 8 * u1);
+    }
+    unit += p8 ? 2 : 1;
     if (flags & kFlagLastOfMatrix) {
       rowacc += __shfl_xor_sync(0xffffffffu, rowacc, 1);  // digits 0,1 (even c) + digit 2 (odd c)
       if (!(flags & kFlagPhase2)) {
@@ -427,7 +441,7 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
   const float* partial = reinterpret_cast<const float*>(smem + SmemLayout::partial);
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t xbars = bars + 16 * kStages;
+  const uint32_t xbars = bars + 16 * kUnits;
   const uint32_t pfull0 = xbars + 8 * kBarPFull0, pempty0 = xbars + 8 * kBarPEmpty0, hx_go = xbars + 8 * kBarHxGo;
   unsigned* status = &p.ws->status;
   const int total = plan.count1 + plan.count2;
@@ -486,82 +500,100 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
 
 // ---- producer --------------------------------------------------------------------------------------
 struct ProducerState {
-  int it;
-  int chunk;  // running chunk counter: rotates the warp -> block assignment
+  int cn;    // chunk number: selects the full barrier and the descriptor slot
+  int unit;  // running unit counter: a chunk takes one unit per plane
 };
 
-// Streams the planes of one (slot, matrix, row block) into the ring.  Returns false if a wait ran out.
-// act_* are the shared-memory byte offsets of the activation digits / digit sums / block scales that go
-// with the matrix' first column.
+// Streams the chunks of one (slot, matrix, row block) into the ring.  Run by lanes 0..3 of the producer
+// warp together: lane 0 copies the MSB plane tile, lane 1 the LSB tile (8-bit slots), lane 2 the scales,
+// lane 3 the zero-points.  Returns false if a wait ran out.  act_* are the shared-memory byte offsets of
+// the activation digits / digit sums / block scales that go with the matrix' first column.
 template <int G>
-__device__ __forceinline__ bool produce_matrix(uint8_t* smem, ProducerState& ps, const Slot& s, int slot, int mat, int K,
-                                               int rb, uint32_t base_flags, bool last_matrix, uint32_t act_dig,
-                                               uint32_t act_sum, uint32_t act_inv, volatile int* dead, unsigned* status) {
+__device__ __forceinline__ bool produce_matrix(uint8_t* smem, ProducerState& ps, int lane, const Slot& s, int slot,
+                                               int mat, int K, int rb, uint32_t base_flags, bool last_matrix,
+                                               uint32_t act_dig, uint32_t act_sum, uint32_t act_inv, volatile int* dead,
+                                               unsigned* status) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
   uint4* descs = reinterpret_cast<uint4*>(smem + SmemLayout::desc);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t full0 = bars, empty0 = bars + 8 * kStages;
+  const uint32_t full0 = bars, empty0 = bars + 8 * kUnits;
   const uint32_t ring = smem_u32(smem + SmemLayout::ring);
-  const int nplanes = s.prec ? 2 : 1;
-  const uint8_t* pm = s.msb[mat] + (size_t)((unsigned)rb * (unsigned)(K >> 6)) * 512u;
-  const uint8_t* pl_ = s.lsb[mat] + (size_t)((unsigned)rb * (unsigned)(K >> 6)) * 512u;
-  const unsigned mo0 = (unsigned)rb * (unsigned)(K >> LG) * 16u;
-  const uint16_t* psc = s.sc[mat] + mo0;
-  const uint8_t* pzp = s.zp[mat] + mo0;
-  const uint32_t flags0 = base_flags | (s.prec ? kFlagPrec8 : 0u);
+  const bool p8 = s.prec != 0;
+  // this lane's source: base for the row block, bytes per column block of kChunkK, destination inside the unit
+  const unsigned plane_off = (unsigned)rb * (unsigned)(K >> 6) * 512u;
+  const unsigned meta_off = (unsigned)rb * (unsigned)(K >> LG) * 16u;  // entries
+  const uint8_t* src;
+  uint32_t per_k_shift_bytes;  // bytes per 128 columns
+  uint32_t dst_in_unit;
+  if (lane == 0) {
+    src = s.msb[mat] + plane_off;
+    per_k_shift_bytes = 1024u;
+    dst_in_unit = 0u;
+  } else if (lane == 1) {
+    src = s.lsb[mat] + plane_off;
+    per_k_shift_bytes = 1024u;
+    dst_in_unit = (uint32_t)kUnitBytes;  // the chunk's second unit
+  } else if (lane == 2) {
+    src = reinterpret_cast<const uint8_t*>(s.sc[mat] + meta_off);
+    per_k_shift_bytes = (128u >> LG) * 32u;
+    dst_in_unit = (uint32_t)kPlaneUnitBytes;
+  } else {
+    src = s.zp[mat] + meta_off;
+    per_k_shift_bytes = (128u >> LG) * 16u;
+    dst_in_unit = (uint32_t)(kPlaneUnitBytes + kScaleUnitBytes);
+  }
+  const bool active = lane != 1 || p8;
+  const uint32_t flags0 = base_flags | (p8 ? kFlagPrec8 : 0u);
   for (int k0 = 0; k0 < K; k0 += kChunkK) {
     const int kc = min(kChunkK, K - k0);
-    const bool last_chunk = k0 + kChunkK >= K;
-    for (int pl = 0; pl < nplanes; ++pl) {
-      const int stage = ps.it % kStages;
-      if (!mbar_wait(empty0 + 8 * stage, ((ps.it / kStages) & 1) ^ 1, dead, status)) return false;
-      const bool has_meta = (pl == nplanes - 1);
-      uint32_t flags = flags0 | (pl ? kFlagLsb : 0u) | (has_meta ? kFlagMeta : 0u);
-      if (has_meta && last_chunk) flags |= kFlagLastOfMatrix | (last_matrix ? kFlagLastOfTask : 0u);
-      descs[stage] = make_uint4(flags | ((uint32_t)(kc >> 7) << 8) | ((uint32_t)(ps.chunk % kConsumerWarps) << 16) |
-                                    ((uint32_t)slot << 24),
-                                act_dig + (uint32_t)k0 * 4u, act_sum + (uint32_t)(k0 >> LG) * 8u,
-                                act_inv + (uint32_t)(k0 >> 7) * 4u);
-      const uint32_t plane_bytes = (uint32_t)kc * 8u;
-      const uint32_t ngc = (uint32_t)(kc >> LG);
-      const uint32_t bar = full0 + 8 * stage;
-      const uint32_t dst = ring + stage * kStageBytes;
-      mbar_arrive_expect_tx(bar, plane_bytes + (has_meta ? ngc * 48u : 0u));
-      bulk_g2s(dst, (pl ? pl_ : pm) + (size_t)k0 * 8u, plane_bytes, bar);
-      if (has_meta) {
-        const unsigned mo = (unsigned)(k0 >> LG) * 16u;
-        bulk_g2s(dst + kPlaneStageBytes, psc + mo, ngc * 32u, bar);
-        bulk_g2s(dst + kPlaneStageBytes + kScaleStageBytes, pzp + mo, ngc * 16u, bar);
-      }
-      ++ps.it;
+    const int u0 = ps.unit % kUnits, u1 = (ps.unit + 1) % kUnits;
+    if (!mbar_wait(empty0 + 8 * u0, ((ps.unit / kUnits) & 1) ^ 1, dead, status)) return false;
+    if (p8 && !mbar_wait(empty0 + 8 * u1, (((ps.unit + 1) / kUnits) & 1) ^ 1, dead, status)) return false;
+    const uint32_t bar = full0 + 8 * (ps.cn % kUnits);
+    if (lane == 0) {
+      uint32_t flags = flags0;
+      if (k0 + kChunkK >= K) flags |= kFlagLastOfMatrix | (last_matrix ? kFlagLastOfTask : 0u);
+      descs[ps.cn % kUnits] = make_uint4(flags | ((uint32_t)(kc >> 7) << 8) |
+                                             ((uint32_t)(ps.cn % kConsumerWarps) << 16) | ((uint32_t)slot << 24),
+                                         act_dig + (uint32_t)k0 * 3u, act_sum + (uint32_t)(k0 >> LG) * 8u,
+                                         act_inv + (uint32_t)(k0 >> 7) * 4u);
+      const uint32_t nblk = (uint32_t)(kc >> 7);
+      mbar_arrive_expect_tx(bar, nblk * ((p8 ? 2048u : 1024u) + (128u >> LG) * 48u));
     }
-    ++ps.chunk;
+    __syncwarp(0xfu);
+    if (active) {
+      // a second-unit destination wraps around the ring with the unit index
+      const uint32_t dst = ring + (lane == 1 ? (uint32_t)u1 * kUnitBytes : (uint32_t)u0 * kUnitBytes + dst_in_unit);
+      bulk_g2s(dst, src + (size_t)(k0 >> 7) * per_k_shift_bytes, (uint32_t)(kc >> 7) * per_k_shift_bytes, bar);
+    }
+    ps.unit += p8 ? 2 : 1;
+    ++ps.cn;
   }
   return true;
 }
 
 template <int G>
-__device__ void producer_loop(const DecodeParams& p, uint8_t* smem) {
+__device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
   const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
   uint4* descs = reinterpret_cast<uint4*>(smem + SmemLayout::desc);
   const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t full0 = bars, empty0 = bars + 8 * kStages;
+  const uint32_t full0 = bars;
   unsigned* status = &p.ws->status;
   ProducerState ps;
-  ps.it = 0;
-  ps.chunk = 0;
+  ps.cn = 0;
+  ps.unit = 0;
   bool ok = true;
   // phase 1: gate and up of (slot, row block) tasks
   {
     int slot = plan.first_slot, idx = plan.first_idx;
     for (int n = 0; n < plan.count1 && ok; ++n) {
       const Slot& s = slots[slot];
-      ok = produce_matrix<G>(smem, ps, s, slot, 0, p.hidden, idx, 0u, false, SmemLayout::xdig, SmemLayout::xsumw,
+      ok = produce_matrix<G>(smem, ps, lane, s, slot, 0, p.hidden, idx, 0u, false, SmemLayout::xdig, SmemLayout::xsumw,
                              SmemLayout::xinv, dead, status) &&
-           produce_matrix<G>(smem, ps, s, slot, 1, p.hidden, idx, 0u, true, SmemLayout::xdig, SmemLayout::xsumw,
+           produce_matrix<G>(smem, ps, lane, s, slot, 1, p.hidden, idx, 0u, true, SmemLayout::xdig, SmemLayout::xsumw,
                              SmemLayout::xinv, dead, status);
       if (++idx >= s.inter / 16) {
         idx = 0;
@@ -574,32 +606,36 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem) {
     const int rb = blockIdx.x + n * gridDim.x;
     for (int slot = 0; slot < plan.nslots && ok; ++slot) {
       const Slot& s = slots[slot];
-      ok = produce_matrix<G>(smem, ps, s, slot, 2, s.inter, rb, kFlagPhase2, slot == plan.nslots - 1,
-                             SmemLayout::hdig + (uint32_t)s.hoff * 4u, SmemLayout::hsumw + (uint32_t)(s.hoff >> LG) * 8u,
+      ok = produce_matrix<G>(smem, ps, lane, s, slot, 2, s.inter, rb, kFlagPhase2, slot == plan.nslots - 1,
+                             SmemLayout::hdig + (uint32_t)s.hoff * 3u, SmemLayout::hsumw + (uint32_t)(s.hoff >> LG) * 8u,
                              SmemLayout::hinv + (uint32_t)(s.hoff >> 7) * 4u, dead, status);
     }
   }
-  if (ok) {
-    const int stage = ps.it % kStages;
-    if (mbar_wait(empty0 + 8 * stage, ((ps.it / kStages) & 1) ^ 1, dead, status)) {
-      descs[stage] = make_uint4(kFlagEnd, 0u, 0u, 0u);
-      mbar_arrive(full0 + 8 * stage);
-      ++ps.it;
+  // The sentinel takes a descriptor slot but no unit.  Waiting for the next unit to be free, as a real
+  // chunk would, is what guarantees that chunk cn - kUnits (the slot's previous user) has been consumed.
+  if (ok && mbar_wait(bars + 8 * kUnits + 8 * (ps.unit % kUnits), ((ps.unit / kUnits) & 1) ^ 1, dead, status)) {
+    if (lane == 0) {
+      descs[ps.cn % kUnits] = make_uint4(kFlagEnd, 0u, 0u, 0u);
+      mbar_arrive(full0 + 8 * (ps.cn % kUnits));
     }
+    ++ps.cn;
   }
   // Never leave the CTA with bulk copies still landing in its shared memory: wait (bounded) for the
-  // last kStages armed barriers.  In the normal path they have all completed long ago.
-  for (int j = max(0, ps.it - kStages); j < ps.it; ++j) {
-    const uint32_t bar = full0 + 8 * (j % kStages);
+  // last kUnits armed barriers.  In the normal path they have all completed long ago.
+  for (int j = max(0, ps.cn - kUnits); j < ps.cn; ++j) {
+    const uint32_t bar = full0 + 8 * (j % kUnits);
     const long long t0 = clock64();
-    while (!mbar_try(bar, (j / kStages) & 1)) {
-      if ((unsigned long long)(clock64() - t0) > kWaitCycles) break;
+    while (!mbar_try(bar, (j / kUnits) & 1)) {
+      if (*dead || (unsigned long long)(clock64() - t0) > kWaitCycles) break;
     }
   }
 }
 
 // ---- prologue pieces ---------------------------------------------------------------------------------
 // Warp 0: the routing list -> slot table -> plane pointers -> the static partition.
+// Slot order: shared experts, then the routed experts that run at 8 bits, then those that run at 4 bits,
+// each group in list order.  With the larger tasks first, windows of a multiple of the larger task size cut
+// the phase-1 unit sequence at task boundaries, so every CTA gets the same number of units.
 __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
   Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
   Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
@@ -613,26 +649,29 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
   }
   const bool valid = lane < p.k && e >= 0 && e < p.n_experts;
   const unsigned vmask = __ballot_sync(0xffffffffu, valid);
+  const unsigned bigmask = __ballot_sync(0xffffffffu, valid && pr != 0);
   if (lane < p.k && !valid) atomicOr(&p.ws->status, (unsigned)SLICEMOE_STATUS_BAD_EXPERT_ID);
-  const int nrouted = __popc(vmask);
+  const int nrouted = __popc(vmask), nbig = __popc(bigmask);
   const int nslots = nrouted + p.n_shared;
+  const unsigned below = (1u << lane) - 1u;
   if (valid) {
-    Slot& s = slots[__popc(vmask & ((1u << lane) - 1u))];
+    const int pos = pr != 0 ? __popc(bigmask & below) : nbig + __popc(vmask & ~bigmask & below);
+    Slot& s = slots[p.n_shared + pos];
     s.src = p.experts + e;
     s.inter = p.inter;
     s.prec = pr != 0;
     s.coef = w;
     s.gated = 0;
-    s.hoff = __popc(vmask & ((1u << lane) - 1u)) * p.inter;
+    s.hoff = p.n_shared * p.shared_inter + pos * p.inter;
   }
   if (lane < p.n_shared) {
-    Slot& s = slots[nrouted + lane];
+    Slot& s = slots[lane];
     s.src = p.shared + lane;
     s.inter = p.shared_inter;
     s.prec = 1;
     s.coef = 1.f;
     s.gated = p.sigmoid_gate;
-    s.hoff = nrouted * p.inter + lane * p.shared_inter;
+    s.hoff = lane * p.shared_inter;
   }
   __syncwarp();
   // plane pointers: one 8-byte load per (slot, matrix, field)
@@ -646,7 +685,7 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
     else slots[s].zp[m] = reinterpret_cast<const uint8_t*>(ptr);
   }
   __syncwarp();
-  // lane j owns slot j: a slot without LSB planes runs MSB-only; stages and tasks per slot
+  // lane j owns slot j: a slot without LSB planes runs MSB-only; units and tasks per slot
   int nt = 0, sp = 0;
   if (lane < nslots) {
     Slot& s = slots[lane];
@@ -665,9 +704,11 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
   }
   const unsigned S = __shfl_sync(0xffffffffu, cs, 31);
   const unsigned NT = __shfl_sync(0xffffffffu, ct, 31);
-  // phase 1: equal shares of ring stages, at task granularity: the tasks whose first stage lies in [lo, hi)
-  const unsigned lo = (blockIdx.x * S + gridDim.x - 1) / gridDim.x;
-  const unsigned hi = ((blockIdx.x + 1) * S + gridDim.x - 1) / gridDim.x;
+  const unsigned spmax = max(1u, __reduce_max_sync(0xffffffffu, (unsigned)sp));
+  // phase 1: CTA c takes the tasks whose first unit lies in [c T, (c + 1) T), T = the equal share rounded
+  // up to a multiple of the larger task size
+  const unsigned T = ((S + gridDim.x - 1) / gridDim.x + spmax - 1) / spmax * spmax;
+  const unsigned lo = blockIdx.x * T, hi = lo + T;
   const unsigned off_s = cs - (unsigned)(nt * sp), off_t = ct - (unsigned)nt;  // exclusive
   unsigned ord_lo = NT, ord_hi = NT;
   int slot_lo = nslots, idx_lo = 0;
@@ -723,11 +764,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
     if (lane == 0) {
       *reinterpret_cast<int*>(smem + SmemLayout::dead) = 0;
       const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-      for (int s = 0; s < kStages; ++s) {
-        mbar_init(bars + 8 * s, 1);                             // full: producer's expect_tx arrive
-        mbar_init(bars + 8 * kStages + 8 * s, kConsumerWarps);  // empty: one arrive per consumer warp
+      for (int s = 0; s < kUnits; ++s) {
+        mbar_init(bars + 8 * s, 1);                           // full: lane 0's expect_tx arrive
+        mbar_init(bars + 8 * kUnits + 8 * s, kConsumerWarps);  // empty: one arrive per consumer warp
       }
-      const uint32_t xbars = bars + 16 * kStages;
+      const uint32_t xbars = bars + 16 * kUnits;
       mbar_init(xbars + 8 * kBarPFull0, kConsumerWarps);
       mbar_init(xbars + 8 * kBarPFull1, kConsumerWarps);
       mbar_init(xbars + 8 * kBarPEmpty0, 1);
@@ -767,8 +808,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
     consumer_loop<G>(p, smem, warp, lane);
   } else if (warp == kEpilogueWarp) {
     epilogue_loop(p, smem, lane);
-  } else if (lane == 0) {
-    producer_loop<G>(p, smem);
+  } else if (lane < 4) {
+    producer_loop<G>(p, smem, lane);
   }
   __syncthreads();
   if (tid == 0) {
