@@ -170,6 +170,38 @@ int slicemoe_layer(const slicemoe_shape *shape, const slicemoe_expert *experts,
                    void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * slicemoe_layer_static - slicemoe_layer for callers that cannot allocate device memory.  (The paper
+ * has no counterpart; this is a convenience of the library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a host callback or another
+ * context where the CUDA runtime forbids allocation, under a memory pool that owns every byte of the
+ * device, or in a plug-in that receives input and output buffers from its host application and has
+ * no allocator of its own.  Such a caller cannot provide the workspace that slicemoe_layer asks for,
+ * so this variant keeps the workspace inside the library: a fixed array of 78,016 bytes in device
+ * memory that every GPU holds from the moment it loads the library until the process exits.
+ *
+ * Arguments are those of slicemoe_layer without workspace / workspace_bytes; inputs and outputs are
+ * still the caller's.  The computation and its result are the same as slicemoe_layer's.
+ *   - Limits: the array is sized for hidden <= 4096 and top_k * inter + n_shared * shared_inter <= 12288
+ *     (the limits of slicemoe_layer itself).  A larger layer is refused with SLICEMOE_E_UNSUPPORTED;
+ *     nothing is ever allocated to make it fit.
+ *   - The call allocates nothing and frees nothing, directly or through any library.
+ *   - First call on a device: the library looks up the device address of its array once per device
+ *     (with that device current) and remembers it.  Make this first call outside any stream capture.
+ *   - The array is shared by all calls on a device and keeps the previous call's contents; each call
+ *     clears the part that must start at zero (on `stream`, before its kernels).  Two calls whose work
+ *     overlaps on the GPU - different streams, or different host threads without ordering - race on
+ *     it and give undefined results: keep calls on one device ordered one after the other.
+ *   - The device status word lives in the same array and is not readable through this entry point;
+ *     use slicemoe_layer with your own workspace if you need slicemoe_get_status.
+ * Errors: as slicemoe_layer.
+ */
+int slicemoe_layer_static(const slicemoe_shape *shape, const slicemoe_expert *experts,
+                          const slicemoe_expert *shared, const float *shared_gate_vec, const void *x,
+                          int T, const int32_t *ids, const uint8_t *prec, const float *weights,
+                          float *y, void *stream);
+
+/*
  * slicemoe_decode_step_host - one batch-1 decode step of a layer with HOST inputs and outputs:
  * copies x (bf16 [hidden]) and logits (float32 [E]) to the device, runs slicemoe_route_topk
  * (bias/tau/rank_high as there; the precision request is used as the precision list) and

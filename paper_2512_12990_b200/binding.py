@@ -28,7 +28,7 @@ EXPORTS = (
     "slicemoe_strerror", "slicemoe_version", "slicemoe_plane_bytes", "slicemoe_meta_count", "slicemoe_pack",
     "slicemoe_unpack_plane", "slicemoe_unpack_meta", "slicemoe_route_topk", "slicemoe_workspace_bytes",
     "slicemoe_workspace_init", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer",
-    "slicemoe_decode_step_host", "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
+    "slicemoe_decode_step_host", "slicemoe_layer_static", "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
     "slicemoe_dbsc_assign", "slicemoe_dbsc_stats", "slicemoe_dbsc_contains",
 )
 
@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
                                       c_void_p, c_void_p, c_size_t, c_void_p]
     L.slicemoe_layer.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                  c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.slicemoe_layer_static.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
+                                        c_void_p, c_void_p, c_void_p, c_void_p]
     L.slicemoe_decode_step_host.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                             c_void_p, c_int, c_float, c_int, c_void_p, c_void_p, c_size_t,
                                             c_void_p]
@@ -257,6 +259,17 @@ def slicemoe_layer(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x, id
                               _ptr(x), T, _ptr(ids), _ptr(prec), _ptr(weights), _ptr(y), _ptr(ws), ws.numel(),
                               _stream(stream))
     _check(rc, "slicemoe_layer")
+    return y
+
+
+def slicemoe_layer_static(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x, ids, prec, weights, y, stream=None):
+    """slicemoe_layer without a caller workspace: the library's built-in scratch array is used.  `y` (CUDA
+    float32 [T, hidden]) is required, because nothing may be allocated on this path - not by the library and
+    not by this binding."""
+    rc = lib().slicemoe_layer_static(ctypes.byref(shape), _ptr(experts_tbl), _ptr(shared_tbl), _ptr(shared_gate_vec),
+                                     _ptr(x), x.shape[0], _ptr(ids), _ptr(prec), _ptr(weights), _ptr(y),
+                                     _stream(stream))
+    _check(rc, "slicemoe_layer_static")
     return y
 
 

@@ -984,3 +984,38 @@ extern "C" int slicemoe_decode_step_host(const slicemoe_shape* shape, const slic
   SM_CUDA_TRY(cudaStreamSynchronize(st));
   return SLICEMOE_OK;
 }
+
+// ---- entry point for callers that cannot allocate -----------------------------------------------------
+// The scratch that slicemoe_layer takes from the caller lives here, in the library image: kWsBytes bytes
+// per GPU that loads the library, held until the process exits.
+namespace slicemoe {
+static __device__ __align__(256) unsigned char g_static_scratch[kWsBytes];
+static void* g_static_scratch_ptr[64];  // device address of the array, per device, resolved once
+}  // namespace slicemoe
+
+extern "C" int slicemoe_layer_static(const slicemoe_shape* shape, const slicemoe_expert* experts,
+                                     const slicemoe_expert* shared, const float* shared_gate_vec, const void* x, int T,
+                                     const int32_t* ids, const uint8_t* prec, const float* weights, float* y,
+                                     void* stream) {
+  if (!shape) return SLICEMOE_E_INVALID_ARG;
+  // The built-in scratch has one fixed size; a layer that would need more is refused, never truncated.
+  const long long hsum = (long long)shape->top_k * shape->inter +
+                         (long long)(shape->n_shared > 0 ? shape->n_shared : 0) * shape->shared_inter;
+  if (shape->hidden > kMaxHidden || hsum > kHCap) return SLICEMOE_E_UNSUPPORTED;
+  int dev = 0;
+  SM_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return SLICEMOE_E_UNSUPPORTED;
+  if (!g_static_scratch_ptr[dev]) {
+    // In host code the array's name is only a handle; the address a kernel can use has to be asked for,
+    // with the device that will run the kernel current.
+    void* ptr = nullptr;
+    SM_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+    if (!ptr) return SLICEMOE_E_CUDA;
+    g_static_scratch_ptr[dev] = ptr;
+  }
+  void* ws = g_static_scratch_ptr[dev];
+  // The array keeps whatever the previous call left: the header (barrier counters, status) must start at zero.
+  SM_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHOff, (cudaStream_t)stream));
+  return run_layer(shape, experts, shared, shape->n_shared, shared_gate_vec, x, T, ids, prec, weights, y, ws, kWsBytes,
+                   stream);
+}
