@@ -49,6 +49,7 @@ extern "C" {
 /* Bits of the device status word (slicemoe_get_status). */
 #define SLICEMOE_STATUS_BAD_EXPERT_ID 1 /* an id in a device list was outside [0, n_experts): skipped */
 #define SLICEMOE_STATUS_WAIT_TIMEOUT 2  /* a bounded device-side wait ran out; the output is invalid */
+#define SLICEMOE_STATUS_MISSING_LSB 4   /* prec = 1 for an expert whose lsb planes are NULL: the output is invalid */
 
 #define SLICEMOE_MAX_TOP_K 16
 #define SLICEMOE_MAX_SHARED 4
@@ -69,7 +70,8 @@ typedef struct slicemoe_shape {
 /* One packed weight matrix; all pointers are device pointers in the physical layout above. */
 typedef struct slicemoe_mat {
   const void *msb;       /* N*K/2 bytes */
-  const void *lsb;       /* N*K/2 bytes; may be NULL for a matrix that is never run at 8 bits */
+  const void *lsb;       /* N*K/2 bytes; may be NULL for a matrix that is never run at 8 bits (prec 1 for
+                            such an expert is a caller error: no fault, SLICEMOE_STATUS_MISSING_LSB is set) */
   const uint16_t *scale; /* fp16 bit patterns, N*K/group entries */
   const uint8_t *zp;     /* N*K/group entries */
   int32_t N, K;

@@ -17,7 +17,7 @@ _lib = None
 
 OK = 0
 E_INVALID_ARG, E_UNSUPPORTED, E_CUDA, E_NOMEM = -1, -2, -3, -4
-STATUS_BAD_EXPERT_ID, STATUS_WAIT_TIMEOUT = 1, 2
+STATUS_BAD_EXPERT_ID, STATUS_WAIT_TIMEOUT, STATUS_MISSING_LSB = 1, 2, 4
 MAX_TOP_K, MAX_SHARED = 16, 4
 DBSC_NSTATS = 12
 DBSC_STAT_NAMES = ("requests", "msb_hit", "msb_miss", "lsb_hit", "lsb_miss", "lsb_skipped", "bytes_fetched",

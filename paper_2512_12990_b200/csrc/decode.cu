@@ -3,8 +3,10 @@
 //
 // The work is a pure weight stream: every plane byte is used once, so the bound is HBM bandwidth and
 // everything else is arranged so that the stream never stops.
-//   * One CTA per SM: 16 consumer warps, one epilogue warp, one producer warp (4 lanes, one per bulk
-//     copy of a chunk).  The producer streams chunks - 16 rows x <=2048 columns: the MSB plane tile,
+//   * One CTA per SM: 16 consumer warps in 4 groups, one epilogue warp, one producer warp (4 lanes, one
+//     per bulk copy of a chunk).  Chunks go to the groups round-robin and the 4 warps of a group split a
+//     chunk's 128-column blocks, so the per-chunk bookkeeping is paid by 4 warps, not 16, while 4 chunks
+//     are in work at any time.  The producer streams chunks - 16 rows x <=2048 columns: the MSB plane tile,
 //     the LSB plane tile when the expert runs at 8 bits (<=16 KB each, one contiguous run thanks to the
 //     tiled layout), scales and zero-points - into a ring of eight 16 KB units with cp.async.bulk +
 //     mbarriers.  It never waits for the gate/up -> down dependency, so down-projection tiles are
@@ -34,11 +36,15 @@
 namespace slicemoe {
 
 constexpr int kConsumerWarps = 16;
+constexpr int kGroups = 4;       // consumer groups; chunk number c is handled by group c % kGroups
+constexpr int kGroupWarps = 4;   // warps of a group; they split the 128-column blocks of the chunk
+static_assert(kGroups * kGroupWarps == kConsumerWarps, "groups");
 constexpr int kEpilogueWarp = kConsumerWarps;
 constexpr int kProducerWarp = kConsumerWarps + 1;
 constexpr int kThreads = 32 * (kConsumerWarps + 2);
 constexpr int kUnits = 8;                                 // ring units; a chunk takes one per plane
-constexpr int kChunkK = 128 * kConsumerWarps;             // K columns per chunk: one 128-column block per warp
+constexpr int kChunkK = 2048;                             // K columns per chunk (16 blocks of 128)
+constexpr int kBlocksPerWarp = kChunkK / 128 / kGroupWarps;
 constexpr int kPlaneUnitBytes = 16 * kChunkK / 2;         // 16384
 constexpr int kScaleUnitBytes = 16 * (kChunkK / 32) * 2;  // 2048 (group 32 is the worst case)
 constexpr int kZpUnitBytes = 16 * (kChunkK / 32);         // 1024
@@ -85,11 +91,7 @@ struct DecodeParams {
 };
 
 struct Slot {
-  const uint8_t* msb[3];  // gate, up, down
-  const uint8_t* lsb[3];
-  const uint16_t* sc[3];
-  const uint8_t* zp[3];
-  const slicemoe_expert* src;  // where the pointers above come from
+  const uint8_t* ptr[3][4];  // [gate, up, down][MSB plane, LSB plane, scales, zero-points]: slicemoe_expert's pointers
   int inter;
   int prec;
   float coef;
@@ -99,14 +101,13 @@ struct Slot {
 };
 
 // One chunk as the consumers see it (16 bytes, written by the producer):
-//   x: flags | nblocks << 8 | rot << 16 | slot << 24
+//   x: flags | nblocks << 8 | first unit << 13 | task number << 16 | slot << 24   (nblocks <= 16, unit < 8)
 //   y: byte offset in shared memory of the activation digits of the chunk's first column
 //   z: byte offset in shared memory of the chunk's first (group, digit-pair) weighted digit sum
 //   w: byte offset in shared memory of the chunk's first per-128-block inverse scale
 enum : uint32_t {
-  kFlagLastOfMatrix = 4,  // last chunk of the matrix row block
-  kFlagLastOfTask = 8,    // last matrix of the task: hand the partial rows to the epilogue warp
-  kFlagEnd = 16,          // sentinel, no data
+  kFlagUp = 4,            // phase 1: the chunk belongs to the up projection (else gate)
+  kFlagEnd = 16,          // sentinel, no data (one per group)
   kFlagPrec8 = 32,        // two units: MSB plane, then LSB plane (sums combine as 16 Cm + Cl)
   kFlagPhase2 = 64,
 };
@@ -313,6 +314,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
   const uint32_t full0 = bars, empty0 = bars + 8 * kUnits, xbars = bars + 16 * kUnits;
   const uint32_t pfull0 = xbars + 8 * kBarPFull0, pempty0 = xbars + 8 * kBarPEmpty0;
   unsigned* status = &p.ws->status;
+  const int group = warp / kGroupWarps, gw = warp % kGroupWarps;
 
   // The lane folds row r of the 16-row block for the digit columns it holds: lanes with c in {0, 1} take
   // the accumulators of row g, lanes with c in {2, 3} those of row g + 8 (which are 16 times too large
@@ -325,73 +327,90 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
   const float w0 = (cq ? 65536.f : 1.f) * rowfix, w1 = (cq ? 0.f : 256.f) * rowfix;
   // B column n = g8 takes digit n % 4; the fourth is unused, so those lanes re-read digit 0 and are ignored
   const int boff = ((g8 & 3) == 3 ? 0 : (g8 & 3)) * 32 + c * 8;
-  int acc[SG][4];
-  float rowacc = 0.f, part0 = 0.f, part1 = 0.f;
+  float part0 = 0.f, part1 = 0.f;  // this warp's share of the current task: (gate, up) or (-, weighted down)
   bool fetched = false;
-  int taskcount = 0;
-  int unit = 0;  // running unit counter
+  int task = 0;  // the task part0 / part1 belong to
 
-  for (int cn = 0;; ++cn) {  // chunk number
+  for (int cn = group;; cn += kGroups) {  // chunk numbers of this group
     if (!mbar_wait(full0 + 8 * (cn % kUnits), (cn / kUnits) & 1, dead, status)) return;
     const uint4 d = descs[cn % kUnits];
     const uint32_t flags = d.x & 0xffu;
-    if (flags & kFlagEnd) break;
-    if ((flags & kFlagPhase2) && !fetched) {
+    const int dtask = (int)((d.x >> 16) & 0xffu);
+    // tasks this warp has finished (or never touched) go to the epilogue warp, in order
+    while ((task & 0xff) != dtask) {
+      const int buf = task & 1;
+      if (!mbar_wait(pempty0 + 8 * buf, ((task >> 1) & 1) ^ 1, dead, status)) return;
+      if (cq == 0) *reinterpret_cast<float2*>(partial + ((buf * kConsumerWarps + warp) * 16 + r) * 2) = make_float2(part0, part1);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pfull0 + 8 * buf);
+      ++task;
+      part0 = part1 = 0.f;
+    }
+    if (plan.count2 > 0 && !fetched && (flags & (kFlagPhase2 | kFlagEnd))) {
       if (!fetch_h<G>(p, smem, warp, lane, plan.htotal, dead, status, xbars)) return;
       fetched = true;
     }
+    if (flags & kFlagEnd) break;
     const bool p8 = (flags & kFlagPrec8) != 0;
-    const int u0 = unit % kUnits, u1 = (unit + 1) % kUnits;
-    // the 128-column block of this chunk handled by this warp
-    int b = warp - (int)((d.x >> 16) & 0xffu);
-    if (b < 0) b += kConsumerWarps;
-    if (b < (int)((d.x >> 8) & 0xffu)) {
+    const int u0 = (int)((d.x >> 13) & 7u), u1 = (u0 + 1) % kUnits;
+    const int nblocks = (int)((d.x >> 8) & 31u);
+    const uint8_t* unit0 = smem + SmemLayout::ring + u0 * kUnitBytes;
+    const uint8_t* unit1 = smem + SmemLayout::ring + u1 * kUnitBytes;
+    const uint8_t* dig = smem + d.y + boff;
+    const float* sumw = reinterpret_cast<const float*>(smem + d.z) + cq;
+    const float* binv = reinterpret_cast<const float*>(smem + d.w);
+    const float pfix = p8 ? 1.f : 16.f;
+    const int zsh = p8 ? 0 : 4;
+    const int rot = (cn / kGroups) % kGroupWarps;  // rotates which warp gets the short share of a ragged chunk
+    float rowacc = 0.f;
 #pragma unroll
-      for (int sg = 0; sg < SG; ++sg)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) acc[sg][q] = 0;
-      const uint8_t* bp = smem + d.y + b * 384 + boff;
-      const uint2 bv0 = *reinterpret_cast<const uint2*>(bp);
-      const uint2 bv1 = *reinterpret_cast<const uint2*>(bp + 96);
-      const uint2 bv2 = *reinterpret_cast<const uint2*>(bp + 192);
-      const uint2 bv3 = *reinterpret_cast<const uint2*>(bp + 288);
-      const uint8_t* ap = smem + SmemLayout::ring + u0 * kUnitBytes + b * 1024 + lane * 16;
-      {
-        const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
-        const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
-        mma_u8s8(acc[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
-        mma_u8s8(acc[32 / G], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x,
-                 bv1.y);
-        mma_u8s8(acc[64 / G], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x,
-                 bv2.y);
-        mma_u8s8(acc[96 / G], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x,
-                 bv3.y);
-      }
-      if (p8) {
-        const uint8_t* ap2 = smem + SmemLayout::ring + u1 * kUnitBytes + b * 1024 + lane * 16;
-        const uint4 wlo = *reinterpret_cast<const uint4*>(ap2);
-        const uint4 whi = *reinterpret_cast<const uint4*>(ap2 + 512);
+    for (int j = 0; j < kBlocksPerWarp; ++j) {
+      const int b = (gw + kGroupWarps - rot) % kGroupWarps + kGroupWarps * j;  // 128-column block of the chunk
+      if (b < nblocks) {
+        int acc[SG][4];
 #pragma unroll
         for (int sg = 0; sg < SG; ++sg)
 #pragma unroll
-          for (int q = 0; q < 4; ++q) acc[sg][q] <<= 4;
-        mma_u8s8(acc[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
-        mma_u8s8(acc[32 / G], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x,
-                 bv1.y);
-        mma_u8s8(acc[64 / G], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x,
-                 bv2.y);
-        mma_u8s8(acc[96 / G], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x,
-                 bv3.y);
-      }
-      // fold: scales / zero-points travel in the first unit of the chunk
-      {
-        const uint8_t* meta = smem + SmemLayout::ring + u0 * kUnitBytes + kPlaneUnitBytes;
-        const uint16_t* ms = reinterpret_cast<const uint16_t*>(meta) + (b * SG) * 16 + r;
-        const uint8_t* mz = meta + kScaleUnitBytes + (b * SG) * 16 + r;
-        const float* sumw = reinterpret_cast<const float*>(smem + d.z) + (b * SG) * 2 + cq;
-        const float binv = *(reinterpret_cast<const float*>(smem + d.w) + b);
-        const float sfix = p8 ? binv : 16.f * binv;
-        const int zsh = p8 ? 0 : 4;
+          for (int q = 0; q < 4; ++q) acc[sg][q] = 0;
+        const uint8_t* bp = dig + b * 384;
+        const uint2 bv0 = *reinterpret_cast<const uint2*>(bp);
+        const uint2 bv1 = *reinterpret_cast<const uint2*>(bp + 96);
+        const uint2 bv2 = *reinterpret_cast<const uint2*>(bp + 192);
+        const uint2 bv3 = *reinterpret_cast<const uint2*>(bp + 288);
+        {
+          const uint8_t* ap = unit0 + b * 1024 + lane * 16;
+          const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
+          const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
+          mma_u8s8(acc[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x,
+                   bv0.y);
+          mma_u8s8(acc[32 / G], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u,
+                   bv1.x, bv1.y);
+          mma_u8s8(acc[64 / G], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u,
+                   bv2.x, bv2.y);
+          mma_u8s8(acc[96 / G], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u,
+                   bv3.x, bv3.y);
+        }
+        if (p8) {
+          const uint8_t* ap = unit1 + b * 1024 + lane * 16;
+          const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
+          const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
+#pragma unroll
+          for (int sg = 0; sg < SG; ++sg)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[sg][q] <<= 4;
+          mma_u8s8(acc[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x,
+                   bv0.y);
+          mma_u8s8(acc[32 / G], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u,
+                   bv1.x, bv1.y);
+          mma_u8s8(acc[64 / G], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u,
+                   bv2.x, bv2.y);
+          mma_u8s8(acc[96 / G], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u,
+                   bv3.x, bv3.y);
+        }
+        // fold: scales / zero-points travel in the first unit of the chunk
+        const uint16_t* ms = reinterpret_cast<const uint16_t*>(unit0 + kPlaneUnitBytes) + (b * SG) * 16 + r;
+        const uint8_t* mz = unit0 + kPlaneUnitBytes + kScaleUnitBytes + (b * SG) * 16 + r;
+        const float sfix = pfix * binv[b];
 #pragma unroll
         for (int sg = 0; sg < SG; ++sg) {
           const int ca = (c >> 1) ? acc[sg][2] : acc[sg][0];
@@ -400,7 +419,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
           const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
           const float z = (float)((int)mz[sg * 16] >> zsh);
           // both slices: s (16 Cm + Cl - zp X); MSB only: 16 s (Cm - (zp >> 4) X)
-          rowacc = fmaf(sc, fmaf(-z, sumw[sg * 2], t), rowacc);
+          rowacc = fmaf(sc, fmaf(-z, sumw[(b * SG + sg) * 2], t), rowacc);
         }
       }
     }
@@ -409,27 +428,14 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
       mbar_arrive(empty0 + 8 * u0);
       if (p8) mbar_arrive(empty0 + 8 * u1);
     }
-    unit += p8 ? 2 : 1;
-    if (flags & kFlagLastOfMatrix) {
-      rowacc += __shfl_xor_sync(0xffffffffu, rowacc, 1);  // digits 0,1 (even c) + digit 2 (odd c)
-      if (!(flags & kFlagPhase2)) {
-        if (!(flags & kFlagLastOfTask)) part0 = rowacc;  // gate
-        else part1 = rowacc;                             // up
-      } else {
-        const Slot& sl = slots[d.x >> 24];
-        part1 = fmaf(sl.gated ? plan.gate : sl.coef, rowacc, part1);  // weighted combine, in slot order
-      }
-      rowacc = 0.f;
-      if (flags & kFlagLastOfTask) {
-        // hand this warp's share of the K split to the epilogue warp
-        const int buf = taskcount & 1;
-        if (!mbar_wait(pempty0 + 8 * buf, ((taskcount >> 1) & 1) ^ 1, dead, status)) return;
-        if (cq == 0) *reinterpret_cast<float2*>(partial + ((buf * kConsumerWarps + warp) * 16 + r) * 2) = make_float2(part0, part1);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(pfull0 + 8 * buf);
-        ++taskcount;
-        part0 = part1 = 0.f;
-      }
+    rowacc += __shfl_xor_sync(0xffffffffu, rowacc, 1);  // digits 0,1 (even c) + digit 2 (odd c)
+    if (flags & kFlagPhase2) {
+      const Slot& sl = slots[d.x >> 24];
+      part1 = fmaf(sl.gated ? plan.gate : sl.coef, rowacc, part1);  // weighted combine over the slots
+    } else if (flags & kFlagUp) {
+      part1 += rowacc;
+    } else {
+      part0 += rowacc;
     }
   }
 }
@@ -500,17 +506,26 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
 
 // ---- producer --------------------------------------------------------------------------------------
 struct ProducerState {
-  int cn;    // chunk number: selects the full barrier and the descriptor slot
+  int cn;    // chunk number: selects the full barrier, the descriptor slot and the consumer group
   int unit;  // running unit counter: a chunk takes one unit per plane
+  int task;  // running task number (phase-1 tasks, then phase-2 tasks)
+};
+
+// What a producer lane copies: lane 0 the MSB plane tile, lane 1 the LSB tile (8-bit slots), lane 2 the
+// scales, lane 3 the zero-points.  For all four the source of (row block rb, column block kb of 128) is
+// base + (rb * (K / 128) + kb) * bytes_per_block, because planes and scale / zero-point arrays are all
+// stored [row block][column][16 rows].
+struct ProducerLane {
+  uint32_t bytes_per_block;  // bytes per (16 rows x 128 columns)
+  uint32_t dst_in_unit;      // byte offset of the destination inside the chunk's first unit
 };
 
 // Streams the chunks of one (slot, matrix, row block) into the ring.  Run by lanes 0..3 of the producer
-// warp together: lane 0 copies the MSB plane tile, lane 1 the LSB tile (8-bit slots), lane 2 the scales,
-// lane 3 the zero-points.  Returns false if a wait ran out.  act_* are the shared-memory byte offsets of
-// the activation digits / digit sums / block scales that go with the matrix' first column.
+// warp together.  Returns false if a wait ran out.  act_* are the shared-memory byte offsets of the
+// activation digits / digit sums / block scales that go with the matrix' first column.
 template <int G>
-__device__ __forceinline__ bool produce_matrix(uint8_t* smem, ProducerState& ps, int lane, const Slot& s, int slot,
-                                               int mat, int K, int rb, uint32_t base_flags, bool last_matrix,
+__device__ __forceinline__ bool produce_matrix(uint8_t* smem, ProducerState& ps, int lane, const ProducerLane& pl,
+                                               const Slot& s, int slot, int mat, int K, int rb, uint32_t base_flags,
                                                uint32_t act_dig, uint32_t act_sum, uint32_t act_inv, volatile int* dead,
                                                unsigned* status) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
@@ -519,52 +534,30 @@ __device__ __forceinline__ bool produce_matrix(uint8_t* smem, ProducerState& ps,
   const uint32_t full0 = bars, empty0 = bars + 8 * kUnits;
   const uint32_t ring = smem_u32(smem + SmemLayout::ring);
   const bool p8 = s.prec != 0;
-  // this lane's source: base for the row block, bytes per column block of kChunkK, destination inside the unit
-  const unsigned plane_off = (unsigned)rb * (unsigned)(K >> 6) * 512u;
-  const unsigned meta_off = (unsigned)rb * (unsigned)(K >> LG) * 16u;  // entries
-  const uint8_t* src;
-  uint32_t per_k_shift_bytes;  // bytes per 128 columns
-  uint32_t dst_in_unit;
-  if (lane == 0) {
-    src = s.msb[mat] + plane_off;
-    per_k_shift_bytes = 1024u;
-    dst_in_unit = 0u;
-  } else if (lane == 1) {
-    src = s.lsb[mat] + plane_off;
-    per_k_shift_bytes = 1024u;
-    dst_in_unit = (uint32_t)kUnitBytes;  // the chunk's second unit
-  } else if (lane == 2) {
-    src = reinterpret_cast<const uint8_t*>(s.sc[mat] + meta_off);
-    per_k_shift_bytes = (128u >> LG) * 32u;
-    dst_in_unit = (uint32_t)kPlaneUnitBytes;
-  } else {
-    src = s.zp[mat] + meta_off;
-    per_k_shift_bytes = (128u >> LG) * 16u;
-    dst_in_unit = (uint32_t)(kPlaneUnitBytes + kScaleUnitBytes);
+  const uint8_t* src = s.ptr[mat][lane];
+  if (lane == 1 && src == nullptr) {  // 8 bits asked of an expert without LSB planes: defined garbage, reported
+    src = s.ptr[mat][0];
+    if (p8) atomicOr(status, (unsigned)SLICEMOE_STATUS_MISSING_LSB);
   }
+  src += (size_t)((unsigned)rb * (unsigned)(K >> 7)) * pl.bytes_per_block;
   const bool active = lane != 1 || p8;
-  const uint32_t flags0 = base_flags | (p8 ? kFlagPrec8 : 0u);
+  const uint32_t flags0 = base_flags | (p8 ? kFlagPrec8 : 0u) | ((uint32_t)(ps.task & 0xff) << 16) | ((uint32_t)slot << 24);
   for (int k0 = 0; k0 < K; k0 += kChunkK) {
-    const int kc = min(kChunkK, K - k0);
+    const uint32_t nblk = (uint32_t)(min(kChunkK, K - k0) >> 7);
     const int u0 = ps.unit % kUnits, u1 = (ps.unit + 1) % kUnits;
     if (!mbar_wait(empty0 + 8 * u0, ((ps.unit / kUnits) & 1) ^ 1, dead, status)) return false;
     if (p8 && !mbar_wait(empty0 + 8 * u1, (((ps.unit + 1) / kUnits) & 1) ^ 1, dead, status)) return false;
     const uint32_t bar = full0 + 8 * (ps.cn % kUnits);
     if (lane == 0) {
-      uint32_t flags = flags0;
-      if (k0 + kChunkK >= K) flags |= kFlagLastOfMatrix | (last_matrix ? kFlagLastOfTask : 0u);
-      descs[ps.cn % kUnits] = make_uint4(flags | ((uint32_t)(kc >> 7) << 8) |
-                                             ((uint32_t)(ps.cn % kConsumerWarps) << 16) | ((uint32_t)slot << 24),
-                                         act_dig + (uint32_t)k0 * 3u, act_sum + (uint32_t)(k0 >> LG) * 8u,
-                                         act_inv + (uint32_t)(k0 >> 7) * 4u);
-      const uint32_t nblk = (uint32_t)(kc >> 7);
+      descs[ps.cn % kUnits] = make_uint4(flags0 | (nblk << 8) | ((uint32_t)u0 << 13), act_dig + (uint32_t)k0 * 3u,
+                                         act_sum + (uint32_t)(k0 >> LG) * 8u, act_inv + (uint32_t)(k0 >> 7) * 4u);
       mbar_arrive_expect_tx(bar, nblk * ((p8 ? 2048u : 1024u) + (128u >> LG) * 48u));
     }
     __syncwarp(0xfu);
     if (active) {
-      // a second-unit destination wraps around the ring with the unit index
-      const uint32_t dst = ring + (lane == 1 ? (uint32_t)u1 * kUnitBytes : (uint32_t)u0 * kUnitBytes + dst_in_unit);
-      bulk_g2s(dst, src + (size_t)(k0 >> 7) * per_k_shift_bytes, (uint32_t)(kc >> 7) * per_k_shift_bytes, bar);
+      // the LSB tile goes to the chunk's second unit, which wraps around the ring with the unit index
+      const uint32_t dst = ring + (lane == 1 ? (uint32_t)u1 * kUnitBytes : (uint32_t)u0 * kUnitBytes + pl.dst_in_unit);
+      bulk_g2s(dst, src + (size_t)(k0 >> 7) * pl.bytes_per_block, nblk * pl.bytes_per_block, bar);
     }
     ps.unit += p8 ? 2 : 1;
     ++ps.cn;
@@ -585,16 +578,21 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane) {
   ProducerState ps;
   ps.cn = 0;
   ps.unit = 0;
+  ps.task = 0;
+  ProducerLane pl;
+  pl.bytes_per_block = lane < 2 ? 1024u : (lane == 2 ? (128u >> LG) * 32u : (128u >> LG) * 16u);
+  pl.dst_in_unit = lane < 2 ? 0u : (lane == 2 ? (uint32_t)kPlaneUnitBytes : (uint32_t)(kPlaneUnitBytes + kScaleUnitBytes));
   bool ok = true;
   // phase 1: gate and up of (slot, row block) tasks
   {
     int slot = plan.first_slot, idx = plan.first_idx;
     for (int n = 0; n < plan.count1 && ok; ++n) {
       const Slot& s = slots[slot];
-      ok = produce_matrix<G>(smem, ps, lane, s, slot, 0, p.hidden, idx, 0u, false, SmemLayout::xdig, SmemLayout::xsumw,
+      ok = produce_matrix<G>(smem, ps, lane, pl, s, slot, 0, p.hidden, idx, 0u, SmemLayout::xdig, SmemLayout::xsumw,
                              SmemLayout::xinv, dead, status) &&
-           produce_matrix<G>(smem, ps, lane, s, slot, 1, p.hidden, idx, 0u, true, SmemLayout::xdig, SmemLayout::xsumw,
+           produce_matrix<G>(smem, ps, lane, pl, s, slot, 1, p.hidden, idx, kFlagUp, SmemLayout::xdig, SmemLayout::xsumw,
                              SmemLayout::xinv, dead, status);
+      ++ps.task;
       if (++idx >= s.inter / 16) {
         idx = 0;
         ++slot;
@@ -606,19 +604,23 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane) {
     const int rb = blockIdx.x + n * gridDim.x;
     for (int slot = 0; slot < plan.nslots && ok; ++slot) {
       const Slot& s = slots[slot];
-      ok = produce_matrix<G>(smem, ps, lane, s, slot, 2, s.inter, rb, kFlagPhase2, slot == plan.nslots - 1,
-                             SmemLayout::hdig + (uint32_t)s.hoff * 3u, SmemLayout::hsumw + (uint32_t)(s.hoff >> LG) * 8u,
+      ok = produce_matrix<G>(smem, ps, lane, pl, s, slot, 2, s.inter, rb, kFlagPhase2, SmemLayout::hdig + (uint32_t)s.hoff * 3u,
+                             SmemLayout::hsumw + (uint32_t)(s.hoff >> LG) * 8u,
                              SmemLayout::hinv + (uint32_t)(s.hoff >> 7) * 4u, dead, status);
     }
+    ++ps.task;
   }
-  // The sentinel takes a descriptor slot but no unit.  Waiting for the next unit to be free, as a real
-  // chunk would, is what guarantees that chunk cn - kUnits (the slot's previous user) has been consumed.
-  if (ok && mbar_wait(bars + 8 * kUnits + 8 * (ps.unit % kUnits), ((ps.unit / kUnits) & 1) ^ 1, dead, status)) {
-    if (lane == 0) {
-      descs[ps.cn % kUnits] = make_uint4(kFlagEnd, 0u, 0u, 0u);
-      mbar_arrive(full0 + 8 * (ps.cn % kUnits));
+  // One sentinel per consumer group: a descriptor slot each, no unit.  Waiting for the units that real
+  // one-unit chunks would take is what guarantees that the slots' previous users have been consumed.
+  for (int i = 0; i < kGroups && ok; ++i) {
+    ok = mbar_wait(bars + 8 * kUnits + 8 * ((ps.unit + i) % kUnits), (((ps.unit + i) / kUnits) & 1) ^ 1, dead, status);
+    if (ok) {
+      if (lane == 0) {
+        descs[ps.cn % kUnits] = make_uint4(kFlagEnd | ((uint32_t)(ps.task & 0xff) << 16), 0u, 0u, 0u);
+        mbar_arrive(full0 + 8 * (ps.cn % kUnits));
+      }
+      ++ps.cn;
     }
-    ++ps.cn;
   }
   // Never leave the CTA with bulk copies still landing in its shared memory: wait (bounded) for the
   // last kUnits armed barriers.  In the normal path they have all completed long ago.
@@ -632,118 +634,131 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane) {
 }
 
 // ---- prologue pieces ---------------------------------------------------------------------------------
-// Warp 0: the routing list -> slot table -> plane pointers -> the static partition.
 // Slot order: shared experts, then the routed experts that run at 8 bits, then those that run at 4 bits,
 // each group in list order.  With the larger tasks first, windows of a multiple of the larger task size cut
 // the phase-1 unit sequence at task boundaries, so every CTA gets the same number of units.
+//
+// The routing list as one warp sees it: lane j < k holds entry j; out-of-range ids are dropped.
+struct Routed {
+  int e, pr;
+  float w;
+  bool valid;
+  int pos;  // slot index of this lane's entry
+  int nbig, nsmall;
+};
+__device__ __forceinline__ Routed read_routing(const DecodeParams& p, int lane) {
+  Routed rt;
+  rt.e = -1;
+  rt.pr = 0;
+  rt.w = 0.f;
+  if (lane < p.k) {
+    rt.e = p.ids[lane];
+    rt.pr = p.prec[lane];
+    rt.w = p.weights[lane];
+  }
+  rt.valid = lane < p.k && rt.e >= 0 && rt.e < p.n_experts;
+  const unsigned vmask = __ballot_sync(0xffffffffu, rt.valid);
+  const unsigned bigmask = __ballot_sync(0xffffffffu, rt.valid && rt.pr != 0);
+  const unsigned below = (1u << lane) - 1u;
+  rt.nbig = __popc(bigmask);
+  rt.nsmall = __popc(vmask) - rt.nbig;
+  rt.pos = p.n_shared + (rt.pr != 0 ? __popc(bigmask & below) : rt.nbig + __popc(vmask & ~bigmask & below));
+  return rt;
+}
+
+// Warp 0: slot table (all but the pointers) and the static partition, in closed form: the phase-1 unit
+// sequence is three runs of equal tasks (shared, routed 8-bit, routed 4-bit).
 __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
   Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
   Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
-  // routed experts: lane j reads entry j of the list; out-of-range ids are dropped and reported
-  int e = -1, pr = 0;
-  float w = 0.f;
-  if (lane < p.k) {
-    e = p.ids[lane];
-    pr = p.prec[lane];
-    w = p.weights[lane];
-  }
-  const bool valid = lane < p.k && e >= 0 && e < p.n_experts;
-  const unsigned vmask = __ballot_sync(0xffffffffu, valid);
-  const unsigned bigmask = __ballot_sync(0xffffffffu, valid && pr != 0);
-  if (lane < p.k && !valid) atomicOr(&p.ws->status, (unsigned)SLICEMOE_STATUS_BAD_EXPERT_ID);
-  const int nrouted = __popc(vmask), nbig = __popc(bigmask);
-  const int nslots = nrouted + p.n_shared;
-  const unsigned below = (1u << lane) - 1u;
-  if (valid) {
-    const int pos = pr != 0 ? __popc(bigmask & below) : nbig + __popc(vmask & ~bigmask & below);
-    Slot& s = slots[p.n_shared + pos];
-    s.src = p.experts + e;
+  const Routed rt = read_routing(p, lane);
+  if (lane < p.k && !rt.valid) atomicOr(&p.ws->status, (unsigned)SLICEMOE_STATUS_BAD_EXPERT_ID);
+  if (rt.valid) {
+    Slot& s = slots[rt.pos];
     s.inter = p.inter;
-    s.prec = pr != 0;
-    s.coef = w;
+    s.prec = rt.pr != 0;
+    s.coef = rt.w;
     s.gated = 0;
-    s.hoff = p.n_shared * p.shared_inter + pos * p.inter;
+    s.hoff = p.n_shared * p.shared_inter + (rt.pos - p.n_shared) * p.inter;
   }
-  if (lane < p.n_shared) {
-    Slot& s = slots[lane];
-    s.src = p.shared + lane;
+  if (lane >= 16 && lane - 16 < p.n_shared) {
+    Slot& s = slots[lane - 16];
     s.inter = p.shared_inter;
     s.prec = 1;
     s.coef = 1.f;
     s.gated = p.sigmoid_gate;
-    s.hoff = lane * p.shared_inter;
-  }
-  __syncwarp();
-  // plane pointers: one 8-byte load per (slot, matrix, field)
-  for (int i = lane; i < nslots * 12; i += 32) {
-    const int s = i / 12, q = i % 12, m = q >> 2, f = q & 3;
-    const slicemoe_mat* mat = reinterpret_cast<const slicemoe_mat*>(slots[s].src) + m;
-    const void* ptr = *(reinterpret_cast<const void* const*>(mat) + f);
-    if (f == 0) slots[s].msb[m] = reinterpret_cast<const uint8_t*>(ptr);
-    else if (f == 1) slots[s].lsb[m] = reinterpret_cast<const uint8_t*>(ptr);
-    else if (f == 2) slots[s].sc[m] = reinterpret_cast<const uint16_t*>(ptr);
-    else slots[s].zp[m] = reinterpret_cast<const uint8_t*>(ptr);
-  }
-  __syncwarp();
-  // lane j owns slot j: a slot without LSB planes runs MSB-only; units and tasks per slot
-  int nt = 0, sp = 0;
-  if (lane < nslots) {
-    Slot& s = slots[lane];
-    if (!(s.lsb[0] && s.lsb[1] && s.lsb[2])) s.prec = 0;
-    nt = s.inter / 16;
-    sp = slot_spt1(s, p.hidden);
-  }
-  unsigned cs = (unsigned)(nt * sp), ct = (unsigned)nt;  // inclusive scans over the slots
-#pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    const unsigned a = __shfl_up_sync(0xffffffffu, cs, off), b = __shfl_up_sync(0xffffffffu, ct, off);
-    if (lane >= off) {
-      cs += a;
-      ct += b;
-    }
-  }
-  const unsigned S = __shfl_sync(0xffffffffu, cs, 31);
-  const unsigned NT = __shfl_sync(0xffffffffu, ct, 31);
-  const unsigned spmax = max(1u, __reduce_max_sync(0xffffffffu, (unsigned)sp));
-  // phase 1: CTA c takes the tasks whose first unit lies in [c T, (c + 1) T), T = the equal share rounded
-  // up to a multiple of the larger task size
-  const unsigned T = ((S + gridDim.x - 1) / gridDim.x + spmax - 1) / spmax * spmax;
-  const unsigned lo = blockIdx.x * T, hi = lo + T;
-  const unsigned off_s = cs - (unsigned)(nt * sp), off_t = ct - (unsigned)nt;  // exclusive
-  unsigned ord_lo = NT, ord_hi = NT;
-  int slot_lo = nslots, idx_lo = 0;
-  if (lane < nslots && nt > 0) {
-    if (lo >= off_s && lo < cs) {
-      const unsigned i = (lo - off_s + sp - 1) / sp;  // may equal nt: then it is the next slot's first task
-      ord_lo = off_t + i;
-      slot_lo = lane;
-      idx_lo = (int)i;
-    }
-    if (hi >= off_s && hi < cs) ord_hi = off_t + (hi - off_s + sp - 1) / sp;
-  }
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {  // at most one lane holds each answer
-    const unsigned o = __shfl_xor_sync(0xffffffffu, ord_lo, off);
-    const int sl2 = __shfl_xor_sync(0xffffffffu, slot_lo, off), ix2 = __shfl_xor_sync(0xffffffffu, idx_lo, off);
-    if (sl2 < slot_lo) {
-      ord_lo = o;
-      slot_lo = sl2;
-      idx_lo = ix2;
-    }
-    ord_hi = min(ord_hi, __shfl_xor_sync(0xffffffffu, ord_hi, off));
+    s.hoff = (lane - 16) * p.shared_inter;
   }
   if (lane == 0) {
-    if (slot_lo < nslots && idx_lo >= slots[slot_lo].inter / 16) {  // the bound fell on the slot's end
-      idx_lo = 0;
-      ++slot_lo;
+    const unsigned nsh = (unsigned)p.n_shared, nbig = (unsigned)rt.nbig, nsmall = (unsigned)rt.nsmall;
+    const unsigned nts = nsh ? (unsigned)p.shared_inter / 16u : 0u, ntr = (unsigned)p.inter / 16u;
+    const unsigned nch = (unsigned)nchunks_of(p.hidden);
+    const unsigned spb = 4u * nch, sps = 2u * nch;  // units per 8-bit / 4-bit task
+    const unsigned T1 = nsh * nts, T2 = nbig * ntr, T3 = nsmall * ntr;  // tasks per run
+    const unsigned U1 = T1 * spb, U2 = T2 * spb, S = U1 + U2 + T3 * sps;
+    const unsigned spmax = (nsh + nbig) ? spb : sps;
+    const unsigned T = ((S + gridDim.x - 1) / gridDim.x + spmax - 1) / spmax * spmax;
+    // ordinal of the first task that starts at or after a unit offset
+    auto ord_of = [&](unsigned bound) -> unsigned {
+      if (bound >= S) return T1 + T2 + T3;
+      if (bound < U1) return (bound + spb - 1) / spb;
+      if (bound < U1 + U2) return T1 + (bound - U1 + spb - 1) / spb;
+      return T1 + T2 + (bound - U1 - U2 + sps - 1) / sps;
+    };
+    const unsigned lo = blockIdx.x * T;
+    const unsigned o0 = ord_of(lo), o1 = ord_of(lo + T);
+    int slot, idx;
+    if (o0 < T1) {
+      slot = (int)(o0 / nts);
+      idx = (int)(o0 % nts);
+    } else {
+      slot = (int)(nsh + (o0 - T1) / ntr);
+      idx = (int)((o0 - T1) % ntr);
     }
-    plan->first_slot = slot_lo;
-    plan->first_idx = idx_lo;
-    plan->count1 = (int)(ord_hi - ord_lo);
+    const int nslots = (int)(nsh + nbig + nsmall);
+    plan->first_slot = slot;
+    plan->first_idx = idx;
+    plan->count1 = (int)(o1 - o0);
     const int nrb = p.hidden / 16;
     plan->count2 = (nslots > 0 && (int)blockIdx.x < nrb) ? (nrb - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     plan->nslots = nslots;
-    plan->htotal = nrouted * p.inter + p.n_shared * p.shared_inter;
+    plan->htotal = (int)(nsh * (unsigned)p.shared_inter + (nbig + nsmall) * (unsigned)p.inter);
+  }
+}
+
+// Warp 1: the routed slots' plane pointers.  Warp 2: the shared slots' (they do not depend on the list).
+// Each slot's twelve pointers sit in slicemoe_expert in the order the slot table keeps them.
+__device__ void load_slot_pointers(const DecodeParams& p, uint8_t* smem, int lane, bool routed) {
+  Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
+  constexpr int kRounds = (kMaxSlots * 12 + 31) / 32;
+  const uint8_t* const* src[kRounds];
+  int first = 0, count = p.n_shared;
+  if (routed) {
+    const Routed rt = read_routing(p, lane);
+    first = p.n_shared;
+    count = rt.nbig + rt.nsmall;
+    // lane j knows its entry's slot; every lane needs every slot's expert: pass them through the slot table
+    if (rt.valid) slots[rt.pos].ptr[0][0] = reinterpret_cast<const uint8_t*>(p.experts + rt.e);
+    __syncwarp();
+  }
+#pragma unroll
+  for (int rd = 0; rd < kRounds; ++rd) {
+    const int i = rd * 32 + lane;
+    src[rd] = nullptr;
+    if (i < count * 12) {
+      const int sl = first + i / 12, q = i % 12;
+      const slicemoe_expert* ex = routed ? reinterpret_cast<const slicemoe_expert*>(slots[sl].ptr[0][0]) : p.shared + sl;
+      src[rd] = reinterpret_cast<const uint8_t* const*>(reinterpret_cast<const slicemoe_mat*>(ex) + (q >> 2)) + (q & 3);
+    }
+  }
+  __syncwarp();  // every lane has read the experts' addresses before the first slot pointer overwrites one
+  const uint8_t* val[kRounds];
+#pragma unroll
+  for (int rd = 0; rd < kRounds; ++rd) val[rd] = src[rd] ? *src[rd] : nullptr;  // all loads in flight together
+#pragma unroll
+  for (int rd = 0; rd < kRounds; ++rd) {
+    const int i = rd * 32 + lane;
+    if (i < count * 12) slots[first + i / 12].ptr[(i % 12) >> 2][(i % 12) & 3] = val[rd];
   }
 }
 
@@ -754,19 +769,23 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
 
-  // Prologue, all roles in parallel and one barrier at the end: warp 0 builds the slot table and the
-  // partition (two dependent global reads: the routing list, then the experts' plane pointers); the other
-  // warps turn x into digits, one 128-element block per warp; the last warp sets up the barriers and the
-  // shared-expert gate.
+  // Prologue, all roles in parallel and one barrier at the end: warp 0 reads the routing list and builds
+  // the slot table and the partition; warps 1 and 2 fetch the routed and the shared experts' plane
+  // pointers; the next 14 warps turn x into digits, one 128-element block at a time; the last warp sets
+  // up the barriers and the shared-expert gate.
   if (warp == 0) {
     build_plan(p, smem, lane);
+  } else if (warp == 1) {
+    load_slot_pointers(p, smem, lane, true);
+  } else if (warp == 2) {
+    if (p.n_shared > 0) load_slot_pointers(p, smem, lane, false);
   } else if (warp == kProducerWarp) {
     if (lane == 0) {
       *reinterpret_cast<int*>(smem + SmemLayout::dead) = 0;
       const uint32_t bars = smem_u32(smem + SmemLayout::bars);
       for (int s = 0; s < kUnits; ++s) {
         mbar_init(bars + 8 * s, 1);                           // full: lane 0's expect_tx arrive
-        mbar_init(bars + 8 * kUnits + 8 * s, kConsumerWarps);  // empty: one arrive per consumer warp
+        mbar_init(bars + 8 * kUnits + 8 * s, kGroupWarps);  // empty: one arrive per warp of the group
       }
       const uint32_t xbars = bars + 16 * kUnits;
       mbar_init(xbars + 8 * kBarPFull0, kConsumerWarps);
@@ -792,7 +811,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
       if (lane == 0) plan->gate = 1.f / (1.f + expf(-dot));
     }
   } else {
-    for (int blk = warp - 1; blk < p.hidden / 128; blk += kConsumerWarps) {
+    for (int blk = warp - 3; blk < p.hidden / 128; blk += kConsumerWarps - 2) {
       const uint2 raw = *reinterpret_cast<const uint2*>(p.x + blk * 128 + 4 * lane);
       const float v[4] = {__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u),
                           __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u)};
