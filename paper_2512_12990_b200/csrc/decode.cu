@@ -3,7 +3,7 @@
 //
 // The work is a pure weight stream: every plane byte is used once, so the bound is HBM bandwidth and
 // everything else is arranged so that the stream never stops.
-//   * One CTA per SM: 16 consumer warps in 4 groups, one epilogue warp, one producer warp (4 lanes, one
+//   * One CTA per SM: 16 consumer warps in 4 groups, one epilogue warp, one producer warp (6 lanes, one
 //     per bulk copy of a chunk).  Chunks go to the groups round-robin and the 4 warps of a group split a
 //     chunk's 128-column blocks, so the per-chunk bookkeeping is paid by 4 warps, not 16, while 4 chunks
 //     are in work at any time.  The producer streams chunks - 16 rows x <=2048 columns: the MSB plane tile,
@@ -107,6 +107,7 @@ struct Slot {
 //   w: byte offset in shared memory of the chunk's first per-128-block inverse scale
 enum : uint32_t {
   kFlagUp = 4,            // phase 1: the chunk belongs to the up projection (else gate)
+  kFlagPair = 8,          // phase 1, 4-bit slot: two units, the gate's MSB tile and the up's, each with its scales
   kFlagEnd = 16,          // sentinel, no data (one per group)
   kFlagPrec8 = 32,        // two units: MSB plane, then LSB plane (sums combine as 16 Cm + Cl)
   kFlagPhase2 = 64,
@@ -305,6 +306,8 @@ __device__ bool fetch_h(const DecodeParams& p, uint8_t* smem, int warp, int lane
 template <int G>
 __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, int lane) {
   constexpr int SG = 128 / G;
+  constexpr int NACC = G == 32 ? 4 : 2;  // accumulators per plane pass
+  constexpr int kA1 = G == 32 ? 1 : 0, kA2 = G == 32 ? 2 : 1, kA3 = G == 32 ? 3 : 1;  // accumulator of each 32-column step
   const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
   const uint4* descs = reinterpret_cast<const uint4*>(smem + SmemLayout::desc);
   const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
@@ -359,19 +362,22 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
     const uint8_t* dig = smem + d.y + boff;
     const float* sumw = reinterpret_cast<const float*>(smem + d.z) + cq;
     const float* binv = reinterpret_cast<const float*>(smem + d.w);
+    const bool pair = (flags & kFlagPair) != 0;
     const float pfix = p8 ? 1.f : 16.f;
     const int zsh = p8 ? 0 : 4;
     const int rot = (cn / kGroups) % kGroupWarps;  // rotates which warp gets the short share of a ragged chunk
-    float rowacc = 0.f;
+    float rowacc0 = 0.f, rowacc1 = 0.f;
 #pragma unroll
     for (int j = 0; j < kBlocksPerWarp; ++j) {
       const int b = (gw + kGroupWarps - rot) % kGroupWarps + kGroupWarps * j;  // 128-column block of the chunk
       if (b < nblocks) {
-        int acc[SG][4];
+        // Two plane passes with their own accumulators, two (G >= 64) or four (G = 32) per pass, so that the
+        // eight MMAs of a block form four independent chains instead of one.
+        int m[NACC][4], l[NACC][4];
 #pragma unroll
-        for (int sg = 0; sg < SG; ++sg)
+        for (int a2 = 0; a2 < NACC; ++a2)
 #pragma unroll
-          for (int q = 0; q < 4; ++q) acc[sg][q] = 0;
+          for (int q = 0; q < 4; ++q) m[a2][q] = l[a2][q] = 0;
         const uint8_t* bp = dig + b * 384;
         const uint2 bv0 = *reinterpret_cast<const uint2*>(bp);
         const uint2 bv1 = *reinterpret_cast<const uint2*>(bp + 96);
@@ -381,61 +387,84 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
           const uint8_t* ap = unit0 + b * 1024 + lane * 16;
           const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
           const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
-          mma_u8s8(acc[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x,
-                   bv0.y);
-          mma_u8s8(acc[32 / G], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u,
-                   bv1.x, bv1.y);
-          mma_u8s8(acc[64 / G], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u,
-                   bv2.x, bv2.y);
-          mma_u8s8(acc[96 / G], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u,
-                   bv3.x, bv3.y);
+          mma_u8s8(m[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
+          mma_u8s8(m[kA1], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x, bv1.y);
+          mma_u8s8(m[kA2], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x, bv2.y);
+          mma_u8s8(m[kA3], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x, bv3.y);
         }
-        if (p8) {
+        if (p8 || pair) {
           const uint8_t* ap = unit1 + b * 1024 + lane * 16;
           const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
           const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
-#pragma unroll
-          for (int sg = 0; sg < SG; ++sg)
-#pragma unroll
-            for (int q = 0; q < 4; ++q) acc[sg][q] <<= 4;
-          mma_u8s8(acc[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x,
-                   bv0.y);
-          mma_u8s8(acc[32 / G], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u,
-                   bv1.x, bv1.y);
-          mma_u8s8(acc[64 / G], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u,
-                   bv2.x, bv2.y);
-          mma_u8s8(acc[96 / G], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u,
-                   bv3.x, bv3.y);
+          mma_u8s8(l[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
+          mma_u8s8(l[kA1], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x, bv1.y);
+          mma_u8s8(l[kA2], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x, bv2.y);
+          mma_u8s8(l[kA3], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x, bv3.y);
         }
-        // fold: scales / zero-points travel in the first unit of the chunk
-        const uint16_t* ms = reinterpret_cast<const uint16_t*>(unit0 + kPlaneUnitBytes) + (b * SG) * 16 + r;
-        const uint8_t* mz = unit0 + kPlaneUnitBytes + kScaleUnitBytes + (b * SG) * 16 + r;
-        const float sfix = pfix * binv[b];
+        // this lane's row and digit columns of every group's sums (see above)
+        int ca0[SG], cb0[SG], ca1[SG], cb1[SG];
 #pragma unroll
         for (int sg = 0; sg < SG; ++sg) {
-          const int ca = (c >> 1) ? acc[sg][2] : acc[sg][0];
-          const int cb = (c >> 1) ? acc[sg][3] : acc[sg][1];
-          const float t = fmaf((float)cb, w1, (float)ca * w0);
-          const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
-          const float z = (float)((int)mz[sg * 16] >> zsh);
-          // both slices: s (16 Cm + Cl - zp X); MSB only: 16 s (Cm - (zp >> 4) X)
-          rowacc = fmaf(sc, fmaf(-z, sumw[(b * SG + sg) * 2], t), rowacc);
+          const int i0 = G == 128 ? 0 : sg, hiq = (c >> 1) ? 2 : 0;
+          ca0[sg] = (c >> 1) ? m[i0][2] : m[i0][0];
+          cb0[sg] = (c >> 1) ? m[i0][3] : m[i0][1];
+          ca1[sg] = (c >> 1) ? l[i0][2] : l[i0][0];
+          cb1[sg] = (c >> 1) ? l[i0][3] : l[i0][1];
+          if (G == 128) {
+            ca0[sg] += (c >> 1) ? m[1][2] : m[1][0];
+            cb0[sg] += (c >> 1) ? m[1][3] : m[1][1];
+            ca1[sg] += (c >> 1) ? l[1][2] : l[1][0];
+            cb1[sg] += (c >> 1) ? l[1][3] : l[1][1];
+          }
+          (void)hiq;
+          if (p8) {  // both slices: 16 Cm + Cl
+            ca0[sg] = (ca0[sg] << 4) + ca1[sg];
+            cb0[sg] = (cb0[sg] << 4) + cb1[sg];
+          }
+        }
+        // fold: scales / zero-points travel with the unit whose plane they belong to
+        const float sfix = pfix * binv[b];
+        {
+          const uint16_t* ms = reinterpret_cast<const uint16_t*>(unit0 + kPlaneUnitBytes) + (b * SG) * 16 + r;
+          const uint8_t* mz = unit0 + kPlaneUnitBytes + kScaleUnitBytes + (b * SG) * 16 + r;
+#pragma unroll
+          for (int sg = 0; sg < SG; ++sg) {
+            const float t = fmaf((float)cb0[sg], w1, (float)ca0[sg] * w0);
+            const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
+            const float z = (float)((int)mz[sg * 16] >> zsh);
+            // both slices: s (16 Cm + Cl - zp X); MSB only: 16 s (Cm - (zp >> 4) X)
+            rowacc0 = fmaf(sc, fmaf(-z, sumw[(b * SG + sg) * 2], t), rowacc0);
+          }
+        }
+        if (pair) {
+          const uint16_t* ms = reinterpret_cast<const uint16_t*>(unit1 + kPlaneUnitBytes) + (b * SG) * 16 + r;
+          const uint8_t* mz = unit1 + kPlaneUnitBytes + kScaleUnitBytes + (b * SG) * 16 + r;
+#pragma unroll
+          for (int sg = 0; sg < SG; ++sg) {
+            const float t = fmaf((float)cb1[sg], w1, (float)ca1[sg] * w0);
+            const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
+            const float z = (float)((int)mz[sg * 16] >> 4);
+            rowacc1 = fmaf(sc, fmaf(-z, sumw[(b * SG + sg) * 2], t), rowacc1);
+          }
         }
       }
     }
     __syncwarp();
     if (lane == 0) {
       mbar_arrive(empty0 + 8 * u0);
-      if (p8) mbar_arrive(empty0 + 8 * u1);
+      if (p8 || pair) mbar_arrive(empty0 + 8 * u1);
     }
-    rowacc += __shfl_xor_sync(0xffffffffu, rowacc, 1);  // digits 0,1 (even c) + digit 2 (odd c)
+    rowacc0 += __shfl_xor_sync(0xffffffffu, rowacc0, 1);  // digits 0,1 (even c) + digit 2 (odd c)
     if (flags & kFlagPhase2) {
       const Slot& sl = slots[d.x >> 24];
-      part1 = fmaf(sl.gated ? plan.gate : sl.coef, rowacc, part1);  // weighted combine over the slots
+      part1 = fmaf(sl.gated ? plan.gate : sl.coef, rowacc0, part1);  // weighted combine over the slots
+    } else if (pair) {
+      part0 += rowacc0;
+      part1 += rowacc1 + __shfl_xor_sync(0xffffffffu, rowacc1, 1);
     } else if (flags & kFlagUp) {
-      part1 += rowacc;
+      part1 += rowacc0;
     } else {
-      part0 += rowacc;
+      part0 += rowacc0;
     }
   }
 }
@@ -511,55 +540,76 @@ struct ProducerState {
   int task;  // running task number (phase-1 tasks, then phase-2 tasks)
 };
 
-// What a producer lane copies: lane 0 the MSB plane tile, lane 1 the LSB tile (8-bit slots), lane 2 the
-// scales, lane 3 the zero-points.  For all four the source of (row block rb, column block kb of 128) is
+// What a producer lane copies, for a chunk of matrix A (and, in a pair chunk, matrix B):
+//   lane 0  A's MSB tile            -> first unit, plane area
+//   lane 1  A's LSB tile (8-bit) or B's MSB tile (pair) -> second unit, plane area
+//   lane 2  A's scales, lane 3 A's zero-points          -> first unit, after the plane area
+//   lane 4  B's scales, lane 5 B's zero-points (pair)   -> second unit, after the plane area
+// For all of them the source of (row block rb, column block kb of 128) is
 // base + (rb * (K / 128) + kb) * bytes_per_block, because planes and scale / zero-point arrays are all
 // stored [row block][column][16 rows].
+constexpr int kProducerLanes = 6;
 struct ProducerLane {
   uint32_t bytes_per_block;  // bytes per (16 rows x 128 columns)
-  uint32_t dst_in_unit;      // byte offset of the destination inside the chunk's first unit
+  uint32_t dst_in_unit;      // byte offset of the destination inside its unit
+  int field;                 // which of the matrix' four pointers (pair chunk, lanes >= 4: of matrix B)
+  bool second_unit;
 };
+enum ChunkMode { kModeSingle = 0, kModeBoth = 1, kModePair = 2 };
 
-// Streams the chunks of one (slot, matrix, row block) into the ring.  Run by lanes 0..3 of the producer
-// warp together.  Returns false if a wait ran out.  act_* are the shared-memory byte offsets of the
-// activation digits / digit sums / block scales that go with the matrix' first column.
+// Streams the chunks of one (slot, row block) of matrix A - or of matrices A and B side by side - into the
+// ring.  Run by the first kProducerLanes lanes of the producer warp together.  Returns false if a wait ran
+// out.  act_* are the shared-memory byte offsets of the activation digits / digit sums / block scales that
+// go with the matrices' first column.
 template <int G>
-__device__ __forceinline__ bool produce_matrix(uint8_t* smem, ProducerState& ps, int lane, const ProducerLane& pl,
-                                               const Slot& s, int slot, int mat, int K, int rb, uint32_t base_flags,
-                                               uint32_t act_dig, uint32_t act_sum, uint32_t act_inv, volatile int* dead,
-                                               unsigned* status) {
+__device__ __forceinline__ bool produce_chunks(uint8_t* smem, ProducerState& ps, int lane, const ProducerLane& pl,
+                                               const Slot& s, int slot, int matA, int matB, int mode, int K, int rb,
+                                               uint32_t base_flags, uint32_t act_dig, uint32_t act_sum, uint32_t act_inv,
+                                               volatile int* dead, unsigned* status) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
   uint4* descs = reinterpret_cast<uint4*>(smem + SmemLayout::desc);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
   const uint32_t full0 = bars, empty0 = bars + 8 * kUnits;
   const uint32_t ring = smem_u32(smem + SmemLayout::ring);
-  const bool p8 = s.prec != 0;
-  const uint8_t* src = s.ptr[mat][lane];
-  if (lane == 1 && src == nullptr) {  // 8 bits asked of an expert without LSB planes: defined garbage, reported
-    src = s.ptr[mat][0];
-    if (p8) atomicOr(status, (unsigned)SLICEMOE_STATUS_MISSING_LSB);
+  const bool two = mode != kModeSingle;
+  bool active;
+  const uint8_t* src;
+  if (lane == 1) {
+    active = two;
+    src = mode == kModePair ? s.ptr[matB][0] : s.ptr[matA][1];
+    if (mode == kModeBoth && src == nullptr) {  // 8 bits asked of an expert without LSB planes: defined garbage, reported
+      src = s.ptr[matA][0];
+      atomicOr(status, (unsigned)SLICEMOE_STATUS_MISSING_LSB);
+    }
+  } else if (lane >= 4) {
+    active = mode == kModePair;
+    src = s.ptr[active ? matB : matA][pl.field];
+  } else {
+    active = true;
+    src = s.ptr[matA][pl.field];
   }
   src += (size_t)((unsigned)rb * (unsigned)(K >> 7)) * pl.bytes_per_block;
-  const bool active = lane != 1 || p8;
-  const uint32_t flags0 = base_flags | (p8 ? kFlagPrec8 : 0u) | ((uint32_t)(ps.task & 0xff) << 16) | ((uint32_t)slot << 24);
+  const uint32_t flags0 = base_flags | (mode == kModeBoth ? kFlagPrec8 : 0u) | (mode == kModePair ? kFlagPair : 0u) |
+                          ((uint32_t)(ps.task & 0xff) << 16) | ((uint32_t)slot << 24);
+  const uint32_t meta_per_block = (128u >> LG) * 48u;
   for (int k0 = 0; k0 < K; k0 += kChunkK) {
     const uint32_t nblk = (uint32_t)(min(kChunkK, K - k0) >> 7);
     const int u0 = ps.unit % kUnits, u1 = (ps.unit + 1) % kUnits;
     if (!mbar_wait(empty0 + 8 * u0, ((ps.unit / kUnits) & 1) ^ 1, dead, status)) return false;
-    if (p8 && !mbar_wait(empty0 + 8 * u1, (((ps.unit + 1) / kUnits) & 1) ^ 1, dead, status)) return false;
+    if (two && !mbar_wait(empty0 + 8 * u1, (((ps.unit + 1) / kUnits) & 1) ^ 1, dead, status)) return false;
     const uint32_t bar = full0 + 8 * (ps.cn % kUnits);
     if (lane == 0) {
       descs[ps.cn % kUnits] = make_uint4(flags0 | (nblk << 8) | ((uint32_t)u0 << 13), act_dig + (uint32_t)k0 * 3u,
                                          act_sum + (uint32_t)(k0 >> LG) * 8u, act_inv + (uint32_t)(k0 >> 7) * 4u);
-      mbar_arrive_expect_tx(bar, nblk * ((p8 ? 2048u : 1024u) + (128u >> LG) * 48u));
+      mbar_arrive_expect_tx(bar, nblk * ((two ? 2048u : 1024u) + (mode == kModePair ? 2u : 1u) * meta_per_block));
     }
-    __syncwarp(0xfu);
+    __syncwarp((1u << kProducerLanes) - 1u);
     if (active) {
-      // the LSB tile goes to the chunk's second unit, which wraps around the ring with the unit index
-      const uint32_t dst = ring + (lane == 1 ? (uint32_t)u1 * kUnitBytes : (uint32_t)u0 * kUnitBytes + pl.dst_in_unit);
+      // the second unit wraps around the ring with the unit index
+      const uint32_t dst = ring + (uint32_t)(pl.second_unit ? u1 : u0) * kUnitBytes + pl.dst_in_unit;
       bulk_g2s(dst, src + (size_t)(k0 >> 7) * pl.bytes_per_block, nblk * pl.bytes_per_block, bar);
     }
-    ps.unit += p8 ? 2 : 1;
+    ps.unit += two ? 2 : 1;
     ++ps.cn;
   }
   return true;
@@ -580,18 +630,25 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane) {
   ps.unit = 0;
   ps.task = 0;
   ProducerLane pl;
-  pl.bytes_per_block = lane < 2 ? 1024u : (lane == 2 ? (128u >> LG) * 32u : (128u >> LG) * 16u);
-  pl.dst_in_unit = lane < 2 ? 0u : (lane == 2 ? (uint32_t)kPlaneUnitBytes : (uint32_t)(kPlaneUnitBytes + kScaleUnitBytes));
+  pl.field = lane < 2 ? lane : 2 + (lane & 1);  // lanes 2, 4: scales; lanes 3, 5: zero-points
+  pl.bytes_per_block = lane < 2 ? 1024u : (pl.field == 2 ? (128u >> LG) * 32u : (128u >> LG) * 16u);
+  pl.dst_in_unit = lane < 2 ? 0u : (pl.field == 2 ? (uint32_t)kPlaneUnitBytes : (uint32_t)(kPlaneUnitBytes + kScaleUnitBytes));
+  pl.second_unit = lane == 1 || lane >= 4;
   bool ok = true;
   // phase 1: gate and up of (slot, row block) tasks
   {
     int slot = plan.first_slot, idx = plan.first_idx;
     for (int n = 0; n < plan.count1 && ok; ++n) {
       const Slot& s = slots[slot];
-      ok = produce_matrix<G>(smem, ps, lane, pl, s, slot, 0, p.hidden, idx, 0u, SmemLayout::xdig, SmemLayout::xsumw,
-                             SmemLayout::xinv, dead, status) &&
-           produce_matrix<G>(smem, ps, lane, pl, s, slot, 1, p.hidden, idx, kFlagUp, SmemLayout::xdig, SmemLayout::xsumw,
-                             SmemLayout::xinv, dead, status);
+      if (s.prec) {
+        ok = produce_chunks<G>(smem, ps, lane, pl, s, slot, 0, 0, kModeBoth, p.hidden, idx, 0u, SmemLayout::xdig,
+                               SmemLayout::xsumw, SmemLayout::xinv, dead, status) &&
+             produce_chunks<G>(smem, ps, lane, pl, s, slot, 1, 1, kModeBoth, p.hidden, idx, kFlagUp, SmemLayout::xdig,
+                               SmemLayout::xsumw, SmemLayout::xinv, dead, status);
+      } else {  // 4-bit slot: gate and up tiles travel together, so that every chunk carries two units
+        ok = produce_chunks<G>(smem, ps, lane, pl, s, slot, 0, 1, kModePair, p.hidden, idx, 0u, SmemLayout::xdig,
+                               SmemLayout::xsumw, SmemLayout::xinv, dead, status);
+      }
       ++ps.task;
       if (++idx >= s.inter / 16) {
         idx = 0;
@@ -604,7 +661,8 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane) {
     const int rb = blockIdx.x + n * gridDim.x;
     for (int slot = 0; slot < plan.nslots && ok; ++slot) {
       const Slot& s = slots[slot];
-      ok = produce_matrix<G>(smem, ps, lane, pl, s, slot, 2, s.inter, rb, kFlagPhase2, SmemLayout::hdig + (uint32_t)s.hoff * 3u,
+      ok = produce_chunks<G>(smem, ps, lane, pl, s, slot, 2, 2, s.prec ? kModeBoth : kModeSingle, s.inter, rb, kFlagPhase2,
+                             SmemLayout::hdig + (uint32_t)s.hoff * 3u,
                              SmemLayout::hsumw + (uint32_t)(s.hoff >> LG) * 8u,
                              SmemLayout::hinv + (uint32_t)(s.hoff >> 7) * 4u, dead, status);
     }
@@ -827,7 +885,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
     consumer_loop<G>(p, smem, warp, lane);
   } else if (warp == kEpilogueWarp) {
     epilogue_loop(p, smem, lane);
-  } else if (lane < 4) {
+  } else if (lane < kProducerLanes) {
     producer_loop<G>(p, smem, lane);
   }
   __syncthreads();
