@@ -4,9 +4,10 @@
 // The work is a pure weight stream: every plane byte is used once, so the bound is HBM bandwidth and
 // everything else is arranged so that the stream never stops.
 //   * One CTA per SM: 16 consumer warps in 4 groups, one epilogue warp, one producer warp (6 lanes, one
-//     per bulk copy of a chunk).  Chunks go to the groups round-robin and the 4 warps of a group split a
-//     chunk's 128-column blocks, so the per-chunk bookkeeping is paid by 4 warps, not 16, while 4 chunks
-//     are in work at any time.  The producer streams chunks - 16 rows x <=2048 columns: the MSB plane tile,
+//     per bulk copy of a chunk).  The 4 warps of a group split a chunk's 128-column blocks, so the
+//     per-chunk bookkeeping is paid by 4 warps, not 16, while 4 chunks are in work at any time.  The
+//     schedule is a pure function of the slot table, so every role enumerates it for itself and only
+//     data and barrier phases pass between them.  The producer streams chunks - 16 rows x <=2048 columns: the MSB plane tile,
 //     the LSB plane tile when the expert runs at 8 bits (<=16 KB each, one contiguous run thanks to the
 //     tiled layout), scales and zero-points - into a ring of eight 16 KB units with cp.async.bulk +
 //     mbarriers.  It never waits for the gate/up -> down dependency, so down-projection tiles are
@@ -36,7 +37,7 @@
 namespace slicemoe {
 
 constexpr int kConsumerWarps = 16;
-constexpr int kGroups = 4;       // consumer groups; chunk number c is handled by group c % kGroups
+constexpr int kGroups = 4;       // consumer groups: a phase-1 task belongs to one group, phase-2 chunks go round-robin
 constexpr int kGroupWarps = 4;   // warps of a group; they split the 128-column blocks of the chunk
 static_assert(kGroups * kGroupWarps == kConsumerWarps, "groups");
 constexpr int kEpilogueWarp = kConsumerWarps;
@@ -100,26 +101,23 @@ struct Slot {
   int pad_;
 };
 
-// One chunk as the consumers see it (16 bytes, written by the producer):
-//   x: flags | nblocks << 8 | first unit << 13 | task number << 16 | slot << 24   (nblocks <= 16, unit < 8)
-//   y: byte offset in shared memory of the activation digits of the chunk's first column
-//   z: byte offset in shared memory of the chunk's first (group, digit-pair) weighted digit sum
-//   w: byte offset in shared memory of the chunk's first per-128-block inverse scale
-enum : uint32_t {
-  kFlagUp = 4,            // phase 1: the chunk belongs to the up projection (else gate)
-  kFlagPair = 8,          // phase 1, 4-bit slot: two units, the gate's MSB tile and the up's, each with its scales
-  kFlagEnd = 16,          // sentinel, no data (one per group)
-  kFlagPrec8 = 32,        // two units: MSB plane, then LSB plane (sums combine as 16 Cm + Cl)
-  kFlagPhase2 = 64,
-};
-
+// The schedule of a CTA.
+//   phase 1: tasks n = 0 .. count1-1 are the (slot, 16-row block) pairs from (first_slot, first_idx) on.  A
+//     task of an 8-bit slot is 2 * nch chunks (gate then up; nch = 2048-column chunks of hidden), each two
+//     units (MSB tile, LSB tile); a task of a 4-bit slot is nch chunks, each two units (the gate's MSB tile
+//     and the up's).  Every phase-1 chunk takes two units: chunk number c sits in units 2c, 2c + 1 (mod
+//     kUnits).  Task n is consumed by group n % kGroups.
+//   phase 2: tasks m = 0 .. count2-1 are the output row blocks blockIdx.x + m * gridDim.x; each is one run of
+//     chunks over the slots in order (p2c[j] chunks and p2u[j] units come before slot j), two units per
+//     chunk for 8-bit slots and one for 4-bit slots.  Chunk number c is consumed by group c % kGroups.
 struct Plan {
-  int first_slot, first_idx, count1;  // phase 1: contiguous run of (slot, row block) tasks
-  int count2;                         // phase 2: output row blocks blockIdx.x, + gridDim.x, ...
+  int first_slot, first_idx, count1;
+  int count2;
   int nslots;
-  int htotal;  // sum of the slots' intermediate widths
-  float gate;  // sigmoid(gate_vec . x) when the shared experts are gated
-  int pad_;
+  int htotal;   // sum of the slots' intermediate widths
+  float gate;   // sigmoid(gate_vec . x) when the shared experts are gated
+  int chunks1;  // chunks of phase 1
+  short p2c[kMaxSlots + 1], p2u[kMaxSlots + 1];
 };
 
 struct SmemLayout {
@@ -131,24 +129,28 @@ struct SmemLayout {
   static constexpr int xsumw = hsumw + (kHCap / 32) * 8;     // float [kMaxHidden/32][2]
   static constexpr int hinv = xsumw + (kMaxHidden / 32) * 8;  // float [kHCap/128]: 2^-e of each 128-block of h
   static constexpr int xinv = hinv + (kHCap / 128) * 4;       // float [kMaxHidden/128]
-  static constexpr int partial = xinv + (kMaxHidden / 128) * 4;  // float [2][warps][16][2]
-  static constexpr int slots = partial + 2 * kConsumerWarps * 16 * 2 * 4;
-  static constexpr int desc = slots + kMaxSlots * (int)sizeof(Slot);  // uint4 [kUnits]
-  static constexpr int plan = desc + kUnits * 16;
+  static constexpr int partial = xinv + (kMaxHidden / 128) * 4;  // float2 [warps][16]
+  static constexpr int slots = partial + kConsumerWarps * 16 * 2 * 4;
+  static constexpr int plan = slots + kMaxSlots * (int)sizeof(Slot);
   static constexpr int bars = (plan + (int)sizeof(Plan) + 15) & ~15;  // uint64 barriers
-  static constexpr int nbars = 2 * kUnits + 6;
+  static constexpr int nbars = 2 * kUnits + 2 * kGroups + 4;
   static constexpr int dead = bars + nbars * 8;
   static constexpr int total = dead + 16;
 };
 static_assert(SmemLayout::total <= 227 * 1024, "shared memory budget");
 static_assert(sizeof(Slot) % 8 == 0, "slot alignment");
 static_assert(SmemLayout::slots % 8 == 0 && SmemLayout::hdig % 16 == 0 && SmemLayout::xdig % 16 == 0 &&
-                  SmemLayout::desc % 16 == 0 && SmemLayout::plan % 8 == 0,
+                  SmemLayout::plan % 8 == 0 && SmemLayout::partial % 8 == 0,
               "alignment");
 
-// Ring barriers: full[c % kUnits] for chunk number c (armed with the chunk's bytes), empty[u] for unit u
-// (one arrive per consumer warp).  Barrier indices after the 2 * kUnits ring barriers:
-enum { kBarPFull0 = 0, kBarPFull1, kBarPEmpty0, kBarPEmpty1, kBarHxGo, kBarHsReady };
+// Barrier indices: full[c % kUnits] for chunk number c (armed with the chunk's bytes), empty[u] for unit u
+// (an arrive from each warp of the group that consumed it), pfull1 / pempty1 per group (phase-1 partial rows
+// to the epilogue warp and back), pfull2 / pempty2 (phase-2 partial rows of all warps), hx_go (h is complete
+// in the workspace), hs_ready (h is in shared memory as digits).
+struct Bars {
+  static constexpr int full = 0, empty = kUnits, pfull1 = 2 * kUnits, pempty1 = 2 * kUnits + kGroups,
+                       pfull2 = 2 * kUnits + 2 * kGroups, pempty2 = pfull2 + 1, hx_go = pfull2 + 2, hs_ready = pfull2 + 3;
+};
 
 // ---- PTX helpers -------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -203,6 +205,9 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, 
       : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
   unsigned v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -219,8 +224,9 @@ __device__ __forceinline__ int digit_offset(int k, int t) {
 
 // One warp converts one 128-element block (lane L holds elements 4L..4L+3 of the block, whose first
 // element has index k0 in its vector): fixed point X = rint(v * 2^e) with 2^e * max|v| < 2^22, split into
-// balanced base-256 digits d0 + 256 d1 + 65536 d2 (each in int8 range), stored in B-fragment order; the
-// weighted digit sums of every group of G elements (the zero-point term of the fold) and the block's 2^-e.
+// balanced base-256 digits d0 + 256 d1 + 65536 d2 (each in int8 range; the low byte of X read as a signed
+// byte is d0, and so on up), stored in B-fragment order; the weighted digit sums of every group of G
+// elements (the zero-point term of the fold) and the block's 2^-e.
 template <int G>
 __device__ __forceinline__ void block_to_digits(const float (&v)[4], int k0, int lane, uint8_t* dig, float* sumw,
                                                 float* inv) {
@@ -234,51 +240,45 @@ __device__ __forceinline__ void block_to_digits(const float (&v)[4], int k0, int
   const int ex = (int)(mb >> 23) - 127;  // floor(log2 max) for normal numbers
   const int e = max(-100, min(100, 21 - ex));
   const float scale = __uint_as_float((unsigned)(127 + e) << 23);
-  uint32_t dw[3] = {0u, 0u, 0u};
-  int ds[3] = {0, 0, 0};
+  int X0[4], X1[4], X2[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    int X = __float2int_rn(v[j] * scale);
-    X = max(-4194304, min(4194304, X));
-    const int d0 = ((X + 128) & 255) - 128;
-    X = (X - d0) >> 8;
-    const int d1 = ((X + 128) & 255) - 128;
-    const int d2 = (X - d1) >> 8;
-    dw[0] |= (uint32_t)(d0 & 255) << (8 * j);
-    dw[1] |= (uint32_t)(d1 & 255) << (8 * j);
-    dw[2] |= (uint32_t)(d2 & 255) << (8 * j);
-    ds[0] += d0;
-    ds[1] += d1;
-    ds[2] += d2;
+    X0[j] = max(-4194304, min(4194304, __float2int_rn(v[j] * scale)));
+    X1[j] = (X0[j] + 128) >> 8;  // what is left after taking the low byte as a signed digit
+    X2[j] = (X1[j] + 128) >> 8;
   }
+  // byte 0 of each of the four values -> one word (value j in byte j)
+  const uint32_t d0 = __byte_perm(__byte_perm(X0[0], X0[1], 0x0040), __byte_perm(X0[2], X0[3], 0x0040), 0x5410);
+  const uint32_t d1 = __byte_perm(__byte_perm(X1[0], X1[1], 0x0040), __byte_perm(X1[2], X1[3], 0x0040), 0x5410);
+  const uint32_t d2 = __byte_perm(__byte_perm(X2[0], X2[1], 0x0040), __byte_perm(X2[2], X2[3], 0x0040), 0x5410);
   const int k = k0 + 4 * lane;
-#pragma unroll
-  for (int t = 0; t < 3; ++t) *reinterpret_cast<uint32_t*>(dig + digit_offset(k, t)) = dw[t];
+  *reinterpret_cast<uint32_t*>(dig + digit_offset(k, 0)) = d0;
+  *reinterpret_cast<uint32_t*>(dig + digit_offset(k, 1)) = d1;
+  *reinterpret_cast<uint32_t*>(dig + digit_offset(k, 2)) = d2;
   constexpr int lanes_per_group = G / 4;  // 8, 16 or 32 consecutive lanes cover one group
   const unsigned gmask = lanes_per_group == 32 ? 0xffffffffu
                                                : ((1u << lanes_per_group) - 1u) << (lane & ~(lanes_per_group - 1));
-  ds[0] = __reduce_add_sync(gmask, ds[0]);
-  ds[1] = __reduce_add_sync(gmask, ds[1]);
-  ds[2] = __reduce_add_sync(gmask, ds[2]);
+  const int s0 = __reduce_add_sync(gmask, __dp4a((int)d0, 0x01010101, 0));  // sums of the signed bytes
+  const int s1 = __reduce_add_sync(gmask, __dp4a((int)d1, 0x01010101, 0));
+  const int s2 = __reduce_add_sync(gmask, __dp4a((int)d2, 0x01010101, 0));
   if ((lane & (lanes_per_group - 1)) == 0) {
-    sumw[(k / G) * 2 + 0] = (float)ds[0] + 256.f * (float)ds[1];
-    sumw[(k / G) * 2 + 1] = 65536.f * (float)ds[2];
+    sumw[(k / G) * 2 + 0] = (float)s0 + 256.f * (float)s1;
+    sumw[(k / G) * 2 + 1] = 65536.f * (float)s2;
   }
   if (lane == 0) inv[k0 >> 7] = __uint_as_float((unsigned)(127 - e) << 23);
 }
 
-// ---- task enumeration (identical in every role) ---------------------------------------------------
+// ---- schedule enumeration (identical in every role) ----------------------------------------------------
 __device__ __forceinline__ int nchunks_of(int K) { return (K + kChunkK - 1) / kChunkK; }
-// ring units of one phase-1 task (gate + up of a 16-row block) of a slot
-__device__ __forceinline__ int slot_spt1(const Slot& s, int hidden) { return 2 * (s.prec ? 2 : 1) * nchunks_of(hidden); }
+enum ChunkMode { kModeSingle = 0, kModeBoth = 1, kModePair = 2 };
 
 // ---- consumers -----------------------------------------------------------------------------------
 // Phase change: wait until the epilogue warp has seen the whole grid's h in the workspace, then turn it
 // into digits (all consumer warps, one 128-block at a time).  Returns false if a wait ran out.
 template <int G>
 __device__ bool fetch_h(const DecodeParams& p, uint8_t* smem, int warp, int lane, int htotal, volatile int* dead,
-                        unsigned* status, uint32_t xbars) {
-  const uint32_t hx_go = xbars + 8 * kBarHxGo, hs_ready = xbars + 8 * kBarHsReady;
+                        unsigned* status, uint32_t bars) {
+  const uint32_t hx_go = bars + 8 * Bars::hx_go, hs_ready = bars + 8 * Bars::hs_ready;
   if (!mbar_wait(hx_go, 0, dead, status)) return false;
   if (*dead) return false;
   const int nblk = htotal >> 7;
@@ -303,169 +303,229 @@ __device__ bool fetch_h(const DecodeParams& p, uint8_t* smem, int warp, int lane
   return mbar_wait(hs_ready, 0, dead, status);
 }
 
+// Per-lane constants of the fold (see consume_chunk).
+struct LaneRole {
+  int c, r, cq, boff;
+  float w0, w1;
+};
+
+// One chunk: this warp's 128-column blocks of the 16-row tile(s) in units u0 (and u1).  The A operand is
+// the raw nibble plane, the B operand the activation digits starting at `dig`; `sumw` / `binv` are the
+// digits' weighted group sums and block scales for the same columns.
+//   kModeSingle: MSB tile only           -> *out0 += 16 s (Cm - (zp >> 4) X)
+//   kModeBoth:   MSB tile, LSB tile      -> *out0 += s (16 Cm + Cl - zp X)
+//   kModePair:   two matrices' MSB tiles -> *out0 += first, *out1 += second (each with its own scales)
+// Lane roles: lanes with c in {0, 1} take the accumulators of row g, lanes with c in {2, 3} those of row
+// g + 8 (16 times too large, because their nibbles were left in the high half of the byte); even c holds
+// digits 0 and 1, odd c digit 2 (and the unused fourth column).  The caller adds the two digit halves
+// (a shuffle with lane ^ 1) once per task.
 template <int G>
-__device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, int lane) {
+__device__ __forceinline__ void consume_chunk(const uint8_t* smem, const LaneRole& lr, int lane, int gw, int rot, int mode,
+                                              int nblocks, int u0, int u1, const uint8_t* dig, const float* sumw,
+                                              const float* binv, float* out0, float* out1) {
   constexpr int SG = 128 / G;
   constexpr int NACC = G == 32 ? 4 : 2;  // accumulators per plane pass
   constexpr int kA1 = G == 32 ? 1 : 0, kA2 = G == 32 ? 2 : 1, kA3 = G == 32 ? 3 : 1;  // accumulator of each 32-column step
-  const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
-  const uint4* descs = reinterpret_cast<const uint4*>(smem + SmemLayout::desc);
-  const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
-  float* partial = reinterpret_cast<float*>(smem + SmemLayout::partial);
-  volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
-  const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t full0 = bars, empty0 = bars + 8 * kUnits, xbars = bars + 16 * kUnits;
-  const uint32_t pfull0 = xbars + 8 * kBarPFull0, pempty0 = xbars + 8 * kBarPEmpty0;
-  unsigned* status = &p.ws->status;
-  const int group = warp / kGroupWarps, gw = warp % kGroupWarps;
-
-  // The lane folds row r of the 16-row block for the digit columns it holds: lanes with c in {0, 1} take
-  // the accumulators of row g, lanes with c in {2, 3} those of row g + 8 (which are 16 times too large
-  // because their nibbles were left in the high half of the byte); even c holds digits 0 and 1, odd c
-  // digit 2 (and the unused fourth column).
-  const int c = lane & 3, g8 = lane >> 2;
-  const int r = g8 + 8 * (c >> 1);
-  const int cq = c & 1;
-  const float rowfix = (c >> 1) ? 0.0625f : 1.f;
-  const float w0 = (cq ? 65536.f : 1.f) * rowfix, w1 = (cq ? 0.f : 256.f) * rowfix;
-  // B column n = g8 takes digit n % 4; the fourth is unused, so those lanes re-read digit 0 and are ignored
-  const int boff = ((g8 & 3) == 3 ? 0 : (g8 & 3)) * 32 + c * 8;
-  float part0 = 0.f, part1 = 0.f;  // this warp's share of the current task: (gate, up) or (-, weighted down)
-  bool fetched = false;
-  int task = 0;  // the task part0 / part1 belong to
-
-  for (int cn = group;; cn += kGroups) {  // chunk numbers of this group
-    if (!mbar_wait(full0 + 8 * (cn % kUnits), (cn / kUnits) & 1, dead, status)) return;
-    const uint4 d = descs[cn % kUnits];
-    const uint32_t flags = d.x & 0xffu;
-    const int dtask = (int)((d.x >> 16) & 0xffu);
-    // tasks this warp has finished (or never touched) go to the epilogue warp, in order
-    while ((task & 0xff) != dtask) {
-      const int buf = task & 1;
-      if (!mbar_wait(pempty0 + 8 * buf, ((task >> 1) & 1) ^ 1, dead, status)) return;
-      if (cq == 0) *reinterpret_cast<float2*>(partial + ((buf * kConsumerWarps + warp) * 16 + r) * 2) = make_float2(part0, part1);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(pfull0 + 8 * buf);
-      ++task;
-      part0 = part1 = 0.f;
-    }
-    if (plan.count2 > 0 && !fetched && (flags & (kFlagPhase2 | kFlagEnd))) {
-      if (!fetch_h<G>(p, smem, warp, lane, plan.htotal, dead, status, xbars)) return;
-      fetched = true;
-    }
-    if (flags & kFlagEnd) break;
-    const bool p8 = (flags & kFlagPrec8) != 0;
-    const int u0 = (int)((d.x >> 13) & 7u), u1 = (u0 + 1) % kUnits;
-    const int nblocks = (int)((d.x >> 8) & 31u);
-    const uint8_t* unit0 = smem + SmemLayout::ring + u0 * kUnitBytes;
-    const uint8_t* unit1 = smem + SmemLayout::ring + u1 * kUnitBytes;
-    const uint8_t* dig = smem + d.y + boff;
-    const float* sumw = reinterpret_cast<const float*>(smem + d.z) + cq;
-    const float* binv = reinterpret_cast<const float*>(smem + d.w);
-    const bool pair = (flags & kFlagPair) != 0;
-    const float pfix = p8 ? 1.f : 16.f;
-    const int zsh = p8 ? 0 : 4;
-    const int rot = (cn / kGroups) % kGroupWarps;  // rotates which warp gets the short share of a ragged chunk
-    float rowacc0 = 0.f, rowacc1 = 0.f;
+  const uint8_t* unit0 = smem + SmemLayout::ring + u0 * kUnitBytes;
+  const uint8_t* unit1 = smem + SmemLayout::ring + u1 * kUnitBytes;
+  const bool p8 = mode == kModeBoth, pair = mode == kModePair;
+  const float pfix = p8 ? 1.f : 16.f;
+  const int zsh = p8 ? 0 : 4;
+  const bool hi = (lr.c >> 1) != 0;
+  float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
-    for (int j = 0; j < kBlocksPerWarp; ++j) {
-      const int b = (gw + kGroupWarps - rot) % kGroupWarps + kGroupWarps * j;  // 128-column block of the chunk
-      if (b < nblocks) {
-        // Two plane passes with their own accumulators, two (G >= 64) or four (G = 32) per pass, so that the
-        // eight MMAs of a block form four independent chains instead of one.
-        int m[NACC][4], l[NACC][4];
+  for (int j = 0; j < kBlocksPerWarp; ++j) {
+    const int b = (gw + kGroupWarps - rot) % kGroupWarps + kGroupWarps * j;  // 128-column block of the chunk
+    if (b < nblocks) {
+      // Two plane passes with their own accumulators, two (G >= 64) or four (G = 32) per pass, so that the
+      // eight MMAs of a block form four independent chains instead of one.
+      int m[NACC][4], l[NACC][4];
 #pragma unroll
-        for (int a2 = 0; a2 < NACC; ++a2)
+      for (int a2 = 0; a2 < NACC; ++a2)
 #pragma unroll
-          for (int q = 0; q < 4; ++q) m[a2][q] = l[a2][q] = 0;
-        const uint8_t* bp = dig + b * 384;
-        const uint2 bv0 = *reinterpret_cast<const uint2*>(bp);
-        const uint2 bv1 = *reinterpret_cast<const uint2*>(bp + 96);
-        const uint2 bv2 = *reinterpret_cast<const uint2*>(bp + 192);
-        const uint2 bv3 = *reinterpret_cast<const uint2*>(bp + 288);
-        {
-          const uint8_t* ap = unit0 + b * 1024 + lane * 16;
-          const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
-          const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
-          mma_u8s8(m[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
-          mma_u8s8(m[kA1], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x, bv1.y);
-          mma_u8s8(m[kA2], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x, bv2.y);
-          mma_u8s8(m[kA3], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x, bv3.y);
+        for (int q = 0; q < 4; ++q) m[a2][q] = l[a2][q] = 0;
+      const uint8_t* bp = dig + lr.boff + b * 384;
+      const uint2 bv0 = *reinterpret_cast<const uint2*>(bp);
+      const uint2 bv1 = *reinterpret_cast<const uint2*>(bp + 96);
+      const uint2 bv2 = *reinterpret_cast<const uint2*>(bp + 192);
+      const uint2 bv3 = *reinterpret_cast<const uint2*>(bp + 288);
+      {
+        const uint8_t* ap = unit0 + b * 1024 + lane * 16;
+        const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
+        const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
+        mma_u8s8(m[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
+        mma_u8s8(m[kA1], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x, bv1.y);
+        mma_u8s8(m[kA2], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x, bv2.y);
+        mma_u8s8(m[kA3], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x, bv3.y);
+      }
+      if (mode != kModeSingle) {
+        const uint8_t* ap = unit1 + b * 1024 + lane * 16;
+        const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
+        const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
+        mma_u8s8(l[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
+        mma_u8s8(l[kA1], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x, bv1.y);
+        mma_u8s8(l[kA2], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x, bv2.y);
+        mma_u8s8(l[kA3], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x, bv3.y);
+      }
+      // this lane's row and digit columns of every group's sums
+      int ca0[SG], cb0[SG], ca1[SG], cb1[SG];
+#pragma unroll
+      for (int sg = 0; sg < SG; ++sg) {
+        const int i0 = G == 128 ? 0 : sg;
+        ca0[sg] = hi ? m[i0][2] : m[i0][0];
+        cb0[sg] = hi ? m[i0][3] : m[i0][1];
+        ca1[sg] = hi ? l[i0][2] : l[i0][0];
+        cb1[sg] = hi ? l[i0][3] : l[i0][1];
+        if (G == 128) {
+          ca0[sg] += hi ? m[1][2] : m[1][0];
+          cb0[sg] += hi ? m[1][3] : m[1][1];
+          ca1[sg] += hi ? l[1][2] : l[1][0];
+          cb1[sg] += hi ? l[1][3] : l[1][1];
         }
-        if (p8 || pair) {
-          const uint8_t* ap = unit1 + b * 1024 + lane * 16;
-          const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
-          const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
-          mma_u8s8(l[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
-          mma_u8s8(l[kA1], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x, bv1.y);
-          mma_u8s8(l[kA2], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x, bv2.y);
-          mma_u8s8(l[kA3], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x, bv3.y);
+        if (p8) {  // both slices: 16 Cm + Cl
+          ca0[sg] = (ca0[sg] << 4) + ca1[sg];
+          cb0[sg] = (cb0[sg] << 4) + cb1[sg];
         }
-        // this lane's row and digit columns of every group's sums (see above)
-        int ca0[SG], cb0[SG], ca1[SG], cb1[SG];
+      }
+      // fold: scales / zero-points travel with the unit whose plane they belong to
+      const float sfix = pfix * binv[b];
+      {
+        const uint16_t* ms = reinterpret_cast<const uint16_t*>(unit0 + kPlaneUnitBytes) + (b * SG) * 16 + lr.r;
+        const uint8_t* mz = unit0 + kPlaneUnitBytes + kScaleUnitBytes + (b * SG) * 16 + lr.r;
 #pragma unroll
         for (int sg = 0; sg < SG; ++sg) {
-          const int i0 = G == 128 ? 0 : sg, hiq = (c >> 1) ? 2 : 0;
-          ca0[sg] = (c >> 1) ? m[i0][2] : m[i0][0];
-          cb0[sg] = (c >> 1) ? m[i0][3] : m[i0][1];
-          ca1[sg] = (c >> 1) ? l[i0][2] : l[i0][0];
-          cb1[sg] = (c >> 1) ? l[i0][3] : l[i0][1];
-          if (G == 128) {
-            ca0[sg] += (c >> 1) ? m[1][2] : m[1][0];
-            cb0[sg] += (c >> 1) ? m[1][3] : m[1][1];
-            ca1[sg] += (c >> 1) ? l[1][2] : l[1][0];
-            cb1[sg] += (c >> 1) ? l[1][3] : l[1][1];
-          }
-          (void)hiq;
-          if (p8) {  // both slices: 16 Cm + Cl
-            ca0[sg] = (ca0[sg] << 4) + ca1[sg];
-            cb0[sg] = (cb0[sg] << 4) + cb1[sg];
-          }
+          const float t = fmaf((float)cb0[sg], lr.w1, (float)ca0[sg] * lr.w0);
+          const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
+          const float z = (float)((int)mz[sg * 16] >> zsh);
+          acc0 = fmaf(sc, fmaf(-z, sumw[(b * SG + sg) * 2 + lr.cq], t), acc0);
         }
-        // fold: scales / zero-points travel with the unit whose plane they belong to
-        const float sfix = pfix * binv[b];
-        {
-          const uint16_t* ms = reinterpret_cast<const uint16_t*>(unit0 + kPlaneUnitBytes) + (b * SG) * 16 + r;
-          const uint8_t* mz = unit0 + kPlaneUnitBytes + kScaleUnitBytes + (b * SG) * 16 + r;
+      }
+      if (pair) {
+        const uint16_t* ms = reinterpret_cast<const uint16_t*>(unit1 + kPlaneUnitBytes) + (b * SG) * 16 + lr.r;
+        const uint8_t* mz = unit1 + kPlaneUnitBytes + kScaleUnitBytes + (b * SG) * 16 + lr.r;
 #pragma unroll
-          for (int sg = 0; sg < SG; ++sg) {
-            const float t = fmaf((float)cb0[sg], w1, (float)ca0[sg] * w0);
-            const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
-            const float z = (float)((int)mz[sg * 16] >> zsh);
-            // both slices: s (16 Cm + Cl - zp X); MSB only: 16 s (Cm - (zp >> 4) X)
-            rowacc0 = fmaf(sc, fmaf(-z, sumw[(b * SG + sg) * 2], t), rowacc0);
-          }
-        }
-        if (pair) {
-          const uint16_t* ms = reinterpret_cast<const uint16_t*>(unit1 + kPlaneUnitBytes) + (b * SG) * 16 + r;
-          const uint8_t* mz = unit1 + kPlaneUnitBytes + kScaleUnitBytes + (b * SG) * 16 + r;
-#pragma unroll
-          for (int sg = 0; sg < SG; ++sg) {
-            const float t = fmaf((float)cb1[sg], w1, (float)ca1[sg] * w0);
-            const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
-            const float z = (float)((int)mz[sg * 16] >> 4);
-            rowacc1 = fmaf(sc, fmaf(-z, sumw[(b * SG + sg) * 2], t), rowacc1);
-          }
+        for (int sg = 0; sg < SG; ++sg) {
+          const float t = fmaf((float)cb1[sg], lr.w1, (float)ca1[sg] * lr.w0);
+          const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
+          const float z = (float)((int)mz[sg * 16] >> 4);
+          acc1 = fmaf(sc, fmaf(-z, sumw[(b * SG + sg) * 2 + lr.cq], t), acc1);
         }
       }
     }
+  }
+  *out0 += acc0;
+  *out1 += acc1;
+}
+
+template <int G>
+__device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, int lane) {
+  constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
+  const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
+  const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
+  float2* partial = reinterpret_cast<float2*>(smem + SmemLayout::partial);
+  volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
+  const uint32_t bars = smem_u32(smem + SmemLayout::bars);
+  const uint32_t full0 = bars + 8 * Bars::full, empty0 = bars + 8 * Bars::empty;
+  unsigned* status = &p.ws->status;
+  const int group = warp / kGroupWarps, gw = warp % kGroupWarps;
+  LaneRole lr;
+  lr.c = lane & 3;
+  const int g8 = lane >> 2;
+  lr.r = g8 + 8 * (lr.c >> 1);
+  lr.cq = lr.c & 1;
+  const float rowfix = (lr.c >> 1) ? 0.0625f : 1.f;
+  lr.w0 = (lr.cq ? 65536.f : 1.f) * rowfix;
+  lr.w1 = (lr.cq ? 0.f : 256.f) * rowfix;
+  // B column n = g8 takes digit n % 4; the fourth is unused, so those lanes re-read digit 0 and are ignored
+  lr.boff = ((g8 & 3) == 3 ? 0 : (g8 & 3)) * 32 + lr.c * 8;
+
+  // ---- phase 1: the tasks of this group ----
+  const int nch = nchunks_of(p.hidden);
+  {
+    int slot = plan.first_slot, idx = plan.first_idx, cn = 0;
+    for (int n = 0; n < plan.count1; ++n) {
+      const Slot& sl = slots[slot];
+      const int nchunks = sl.prec ? 2 * nch : nch;
+      if (n % kGroups == group) {
+        float part0 = 0.f, part1 = 0.f, unused = 0.f;
+        for (int q = 0; q < nchunks; ++q) {
+          const int c = cn + q;
+          const int kc = q % nch;  // which 2048-column chunk of hidden
+          if (!mbar_wait(full0 + 8 * (c % kUnits), (c / kUnits) & 1, dead, status)) return;
+          const int u0 = (2 * c) % kUnits, u1 = u0 + 1;
+          const int nblocks = min(kChunkK, p.hidden - kc * kChunkK) >> 7;
+          const uint8_t* dig = smem + SmemLayout::xdig + kc * (kChunkK * 3);
+          const float* sumw = reinterpret_cast<const float*>(smem + SmemLayout::xsumw) + kc * (kChunkK >> LG) * 2;
+          const float* binv = reinterpret_cast<const float*>(smem + SmemLayout::xinv) + kc * (kChunkK >> 7);
+          if (sl.prec) {
+            consume_chunk<G>(smem, lr, lane, gw, c % kGroupWarps, kModeBoth, nblocks, u0, u1, dig, sumw, binv,
+                             q < nch ? &part0 : &part1, &unused);
+          } else {
+            consume_chunk<G>(smem, lr, lane, gw, c % kGroupWarps, kModePair, nblocks, u0, u1, dig, sumw, binv, &part0, &part1);
+          }
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(empty0 + 8 * u0);
+            mbar_arrive(empty0 + 8 * u1);
+          }
+        }
+        // hand the four warps' shares of the K split to the epilogue warp
+        part0 += __shfl_xor_sync(0xffffffffu, part0, 1);  // digits 0,1 (even c) + digit 2 (odd c)
+        part1 += __shfl_xor_sync(0xffffffffu, part1, 1);
+        const int round = n / kGroups;
+        if (!mbar_wait(bars + 8 * (Bars::pempty1 + group), (round & 1) ^ 1, dead, status)) return;
+        if (lr.cq == 0) partial[warp * 16 + lr.r] = make_float2(part0, part1);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + 8 * (Bars::pfull1 + group));
+      }
+      cn += nchunks;
+      if (++idx >= sl.inter / 16) {
+        idx = 0;
+        ++slot;
+      }
+    }
+  }
+  if (plan.count2 == 0) return;
+
+  // ---- the grid's h ----
+  if (!fetch_h<G>(p, smem, warp, lane, plan.htotal, dead, status, bars)) return;
+
+  // ---- phase 2: chunks round-robin over the groups, all warps contribute to every task ----
+  const int chunks2 = plan.p2c[plan.nslots], units2 = plan.p2u[plan.nslots];
+  for (int m = 0; m < plan.count2; ++m) {
+    float part = 0.f, unused = 0.f;
+    for (int j = 0; j < plan.nslots; ++j) {
+      const Slot& sl = slots[j];
+      const int nchj = plan.p2c[j + 1] - plan.p2c[j];
+      float sacc = 0.f;
+      bool mine = false;
+      for (int kc = 0; kc < nchj; ++kc) {
+        const int c = plan.chunks1 + m * chunks2 + plan.p2c[j] + kc;
+        if (c % kGroups != group) continue;
+        mine = true;
+        if (!mbar_wait(full0 + 8 * (c % kUnits), (c / kUnits) & 1, dead, status)) return;
+        const int unit = 2 * plan.chunks1 + m * units2 + plan.p2u[j] + kc * (sl.prec ? 2 : 1);
+        const int u0 = unit % kUnits, u1 = (unit + 1) % kUnits;
+        const int k0 = kc * kChunkK;
+        const int nblocks = min(kChunkK, sl.inter - k0) >> 7;
+        const uint8_t* dig = smem + SmemLayout::hdig + (sl.hoff + k0) * 3;
+        const float* sumw = reinterpret_cast<const float*>(smem + SmemLayout::hsumw) + ((sl.hoff + k0) >> LG) * 2;
+        const float* binv = reinterpret_cast<const float*>(smem + SmemLayout::hinv) + ((sl.hoff + k0) >> 7);
+        consume_chunk<G>(smem, lr, lane, gw, (c / kGroups) % kGroupWarps, sl.prec ? kModeBoth : kModeSingle, nblocks, u0, u1,
+                         dig, sumw, binv, &sacc, &unused);
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(empty0 + 8 * u0);
+          if (sl.prec) mbar_arrive(empty0 + 8 * u1);
+        }
+      }
+      if (mine) part = fmaf(sl.gated ? plan.gate : sl.coef, sacc, part);  // weighted combine, in slot order
+    }
+    part += __shfl_xor_sync(0xffffffffu, part, 1);
+    if (!mbar_wait(bars + 8 * Bars::pempty2, (m & 1) ^ 1, dead, status)) return;
+    if (lr.cq == 0) partial[warp * 16 + lr.r] = make_float2(0.f, part);
     __syncwarp();
-    if (lane == 0) {
-      mbar_arrive(empty0 + 8 * u0);
-      if (p8 || pair) mbar_arrive(empty0 + 8 * u1);
-    }
-    rowacc0 += __shfl_xor_sync(0xffffffffu, rowacc0, 1);  // digits 0,1 (even c) + digit 2 (odd c)
-    if (flags & kFlagPhase2) {
-      const Slot& sl = slots[d.x >> 24];
-      part1 = fmaf(sl.gated ? plan.gate : sl.coef, rowacc0, part1);  // weighted combine over the slots
-    } else if (pair) {
-      part0 += rowacc0;
-      part1 += rowacc1 + __shfl_xor_sync(0xffffffffu, rowacc1, 1);
-    } else if (flags & kFlagUp) {
-      part1 += rowacc0;
-    } else {
-      part0 += rowacc0;
-    }
+    if (lane == 0) mbar_arrive(bars + 8 * Bars::pfull2);
   }
 }
 
@@ -473,73 +533,68 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
 __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
   const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
   const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
-  const float* partial = reinterpret_cast<const float*>(smem + SmemLayout::partial);
+  const float2* partial = reinterpret_cast<const float2*>(smem + SmemLayout::partial);
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t xbars = bars + 16 * kUnits;
-  const uint32_t pfull0 = xbars + 8 * kBarPFull0, pempty0 = xbars + 8 * kBarPEmpty0, hx_go = xbars + 8 * kBarHxGo;
   unsigned* status = &p.ws->status;
-  const int total = plan.count1 + plan.count2;
-  int slot = plan.first_slot, idx = plan.first_idx;
-  for (int tc = 0;; ++tc) {
-    if (tc == plan.count1) {
-      // ---- the single grid-wide dependency: every CTA has written its rows of h ----
-      __syncwarp();
-      if (lane == 0) {
-        __threadfence();
-        atomicAdd(&p.ws->bar_arrive, 1u);
-      }
-      __syncwarp();
-      if (plan.count2 > 0) {
-        // the whole warp polls, converged: no lane spins on something another lane must provide
-        const long long t0 = clock64();
-        while (ld_acquire_u32(&p.ws->bar_arrive) < gridDim.x) {
-          if (*dead) break;
-          if ((unsigned long long)(clock64() - t0) > kWaitCycles) {
-            *dead = 1;
-            atomicOr(status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
-            break;
-          }
-        }
-        __threadfence();
-        __syncwarp();
-        if (*dead) return;
-        if (lane == 0) mbar_arrive(hx_go);
-      }
-    }
-    if (tc == total) break;
-    const int buf = tc & 1;
-    if (!mbar_wait(pfull0 + 8 * buf, (tc >> 1) & 1, dead, status)) return;
-    float a = 0.f, b = 0.f;
-    if (lane < 16) {
+  // phase 1: one group's four partial rows per task -> SwiGLU -> h
+  {
+    int slot = plan.first_slot, idx = plan.first_idx;
+    for (int n = 0; n < plan.count1; ++n) {
+      const int group = n % kGroups, round = n / kGroups;
+      if (!mbar_wait(bars + 8 * (Bars::pfull1 + group), round & 1, dead, status)) return;
+      float a = 0.f, b = 0.f;
+      if (lane < 16) {
 #pragma unroll
-      for (int w = 0; w < kConsumerWarps; ++w) {
-        const float2 v = *reinterpret_cast<const float2*>(partial + ((buf * kConsumerWarps + w) * 16 + lane) * 2);
-        a += v.x;
-        b += v.y;
+        for (int w = 0; w < kGroupWarps; ++w) {
+          const float2 v = partial[(group * kGroupWarps + w) * 16 + lane];
+          a += v.x;
+          b += v.y;
+        }
       }
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(pempty0 + 8 * buf);
-    if (tc < plan.count1) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + 8 * (Bars::pempty1 + group));
       if (lane < 16) p.ws_h[slots[slot].hoff + idx * 16 + lane] = a / (1.f + expf(-a)) * b;  // silu(gate) * up
       if (++idx >= slots[slot].inter / 16) {
         idx = 0;
         ++slot;
       }
-    } else if (lane < 16) {
-      p.y[(blockIdx.x + (tc - plan.count1) * gridDim.x) * 16 + lane] = b;
     }
+  }
+  // ---- the single grid-wide dependency: every CTA has written its rows of h ----
+  __syncwarp();
+  if (lane == 0) red_release_add(&p.ws->bar_arrive, 1u);
+  if (plan.count2 == 0) return;
+  {
+    // the whole warp polls, converged: no lane spins on something another lane must provide
+    const long long t0 = clock64();
+    while (ld_acquire_u32(&p.ws->bar_arrive) < gridDim.x) {
+      if (*dead) break;
+      if ((unsigned long long)(clock64() - t0) > kWaitCycles) {
+        *dead = 1;
+        atomicOr(status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
+        break;
+      }
+    }
+    __syncwarp();
+    if (*dead) return;
+    if (lane == 0) mbar_arrive(bars + 8 * Bars::hx_go);
+  }
+  // phase 2: all warps' partial rows per output row block -> y
+  for (int m = 0; m < plan.count2; ++m) {
+    if (!mbar_wait(bars + 8 * Bars::pfull2, m & 1, dead, status)) return;
+    float b = 0.f;
+    if (lane < 16) {
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) b += partial[w * 16 + lane].y;
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bars + 8 * Bars::pempty2);
+    if (lane < 16) p.y[(blockIdx.x + m * gridDim.x) * 16 + lane] = b;
   }
 }
 
 // ---- producer --------------------------------------------------------------------------------------
-struct ProducerState {
-  int cn;    // chunk number: selects the full barrier, the descriptor slot and the consumer group
-  int unit;  // running unit counter: a chunk takes one unit per plane
-  int task;  // running task number (phase-1 tasks, then phase-2 tasks)
-};
-
 // What a producer lane copies, for a chunk of matrix A (and, in a pair chunk, matrix B):
 //   lane 0  A's MSB tile            -> first unit, plane area
 //   lane 1  A's LSB tile (8-bit) or B's MSB tile (pair) -> second unit, plane area
@@ -549,27 +604,26 @@ struct ProducerState {
 // base + (rb * (K / 128) + kb) * bytes_per_block, because planes and scale / zero-point arrays are all
 // stored [row block][column][16 rows].
 constexpr int kProducerLanes = 6;
+struct ProducerState {
+  int cn;    // chunk number: selects the full barrier
+  int unit;  // running unit counter: a chunk takes one unit per plane
+};
 struct ProducerLane {
   uint32_t bytes_per_block;  // bytes per (16 rows x 128 columns)
   uint32_t dst_in_unit;      // byte offset of the destination inside its unit
-  int field;                 // which of the matrix' four pointers (pair chunk, lanes >= 4: of matrix B)
+  int field;                 // which of the matrix' four pointers
   bool second_unit;
 };
-enum ChunkMode { kModeSingle = 0, kModeBoth = 1, kModePair = 2 };
 
 // Streams the chunks of one (slot, row block) of matrix A - or of matrices A and B side by side - into the
-// ring.  Run by the first kProducerLanes lanes of the producer warp together.  Returns false if a wait ran
-// out.  act_* are the shared-memory byte offsets of the activation digits / digit sums / block scales that
-// go with the matrices' first column.
+// ring.  Run by the first kProducerLanes lanes of the producer warp together.  Returns false if a wait ran out.
 template <int G>
 __device__ __forceinline__ bool produce_chunks(uint8_t* smem, ProducerState& ps, int lane, const ProducerLane& pl,
-                                               const Slot& s, int slot, int matA, int matB, int mode, int K, int rb,
-                                               uint32_t base_flags, uint32_t act_dig, uint32_t act_sum, uint32_t act_inv,
+                                               const Slot& s, int matA, int matB, int mode, int K, int rb,
                                                volatile int* dead, unsigned* status) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
-  uint4* descs = reinterpret_cast<uint4*>(smem + SmemLayout::desc);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t full0 = bars, empty0 = bars + 8 * kUnits;
+  const uint32_t full0 = bars + 8 * Bars::full, empty0 = bars + 8 * Bars::empty;
   const uint32_t ring = smem_u32(smem + SmemLayout::ring);
   const bool two = mode != kModeSingle;
   bool active;
@@ -589,20 +643,14 @@ __device__ __forceinline__ bool produce_chunks(uint8_t* smem, ProducerState& ps,
     src = s.ptr[matA][pl.field];
   }
   src += (size_t)((unsigned)rb * (unsigned)(K >> 7)) * pl.bytes_per_block;
-  const uint32_t flags0 = base_flags | (mode == kModeBoth ? kFlagPrec8 : 0u) | (mode == kModePair ? kFlagPair : 0u) |
-                          ((uint32_t)(ps.task & 0xff) << 16) | ((uint32_t)slot << 24);
-  const uint32_t meta_per_block = (128u >> LG) * 48u;
+  const uint32_t bytes_per_block = (two ? 2048u : 1024u) + (mode == kModePair ? 2u : 1u) * ((128u >> LG) * 48u);
   for (int k0 = 0; k0 < K; k0 += kChunkK) {
     const uint32_t nblk = (uint32_t)(min(kChunkK, K - k0) >> 7);
     const int u0 = ps.unit % kUnits, u1 = (ps.unit + 1) % kUnits;
     if (!mbar_wait(empty0 + 8 * u0, ((ps.unit / kUnits) & 1) ^ 1, dead, status)) return false;
     if (two && !mbar_wait(empty0 + 8 * u1, (((ps.unit + 1) / kUnits) & 1) ^ 1, dead, status)) return false;
     const uint32_t bar = full0 + 8 * (ps.cn % kUnits);
-    if (lane == 0) {
-      descs[ps.cn % kUnits] = make_uint4(flags0 | (nblk << 8) | ((uint32_t)u0 << 13), act_dig + (uint32_t)k0 * 3u,
-                                         act_sum + (uint32_t)(k0 >> LG) * 8u, act_inv + (uint32_t)(k0 >> 7) * 4u);
-      mbar_arrive_expect_tx(bar, nblk * ((two ? 2048u : 1024u) + (mode == kModePair ? 2u : 1u) * meta_per_block));
-    }
+    if (lane == 0) mbar_arrive_expect_tx(bar, nblk * bytes_per_block);
     __syncwarp((1u << kProducerLanes) - 1u);
     if (active) {
       // the second unit wraps around the ring with the unit index
@@ -619,16 +667,14 @@ template <int G>
 __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
   const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
-  uint4* descs = reinterpret_cast<uint4*>(smem + SmemLayout::desc);
   const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t full0 = bars;
+  const uint32_t full0 = bars + 8 * Bars::full;
   unsigned* status = &p.ws->status;
   ProducerState ps;
   ps.cn = 0;
   ps.unit = 0;
-  ps.task = 0;
   ProducerLane pl;
   pl.field = lane < 2 ? lane : 2 + (lane & 1);  // lanes 2, 4: scales; lanes 3, 5: zero-points
   pl.bytes_per_block = lane < 2 ? 1024u : (pl.field == 2 ? (128u >> LG) * 32u : (128u >> LG) * 16u);
@@ -641,15 +687,11 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane) {
     for (int n = 0; n < plan.count1 && ok; ++n) {
       const Slot& s = slots[slot];
       if (s.prec) {
-        ok = produce_chunks<G>(smem, ps, lane, pl, s, slot, 0, 0, kModeBoth, p.hidden, idx, 0u, SmemLayout::xdig,
-                               SmemLayout::xsumw, SmemLayout::xinv, dead, status) &&
-             produce_chunks<G>(smem, ps, lane, pl, s, slot, 1, 1, kModeBoth, p.hidden, idx, kFlagUp, SmemLayout::xdig,
-                               SmemLayout::xsumw, SmemLayout::xinv, dead, status);
+        ok = produce_chunks<G>(smem, ps, lane, pl, s, 0, 0, kModeBoth, p.hidden, idx, dead, status) &&
+             produce_chunks<G>(smem, ps, lane, pl, s, 1, 1, kModeBoth, p.hidden, idx, dead, status);
       } else {  // 4-bit slot: gate and up tiles travel together, so that every chunk carries two units
-        ok = produce_chunks<G>(smem, ps, lane, pl, s, slot, 0, 1, kModePair, p.hidden, idx, 0u, SmemLayout::xdig,
-                               SmemLayout::xsumw, SmemLayout::xinv, dead, status);
+        ok = produce_chunks<G>(smem, ps, lane, pl, s, 0, 1, kModePair, p.hidden, idx, dead, status);
       }
-      ++ps.task;
       if (++idx >= s.inter / 16) {
         idx = 0;
         ++slot;
@@ -657,27 +699,11 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane) {
     }
   }
   // phase 2: down rows of every slot for the output row blocks of this CTA
-  for (int n = 0; n < plan.count2 && ok; ++n) {
-    const int rb = blockIdx.x + n * gridDim.x;
+  for (int m = 0; m < plan.count2 && ok; ++m) {
+    const int rb = blockIdx.x + m * gridDim.x;
     for (int slot = 0; slot < plan.nslots && ok; ++slot) {
       const Slot& s = slots[slot];
-      ok = produce_chunks<G>(smem, ps, lane, pl, s, slot, 2, 2, s.prec ? kModeBoth : kModeSingle, s.inter, rb, kFlagPhase2,
-                             SmemLayout::hdig + (uint32_t)s.hoff * 3u,
-                             SmemLayout::hsumw + (uint32_t)(s.hoff >> LG) * 8u,
-                             SmemLayout::hinv + (uint32_t)(s.hoff >> 7) * 4u, dead, status);
-    }
-    ++ps.task;
-  }
-  // One sentinel per consumer group: a descriptor slot each, no unit.  Waiting for the units that real
-  // one-unit chunks would take is what guarantees that the slots' previous users have been consumed.
-  for (int i = 0; i < kGroups && ok; ++i) {
-    ok = mbar_wait(bars + 8 * kUnits + 8 * ((ps.unit + i) % kUnits), (((ps.unit + i) / kUnits) & 1) ^ 1, dead, status);
-    if (ok) {
-      if (lane == 0) {
-        descs[ps.cn % kUnits] = make_uint4(kFlagEnd | ((uint32_t)(ps.task & 0xff) << 16), 0u, 0u, 0u);
-        mbar_arrive(full0 + 8 * (ps.cn % kUnits));
-      }
-      ++ps.cn;
+      ok = produce_chunks<G>(smem, ps, lane, pl, s, 2, 2, s.prec ? kModeBoth : kModeSingle, s.inter, rb, dead, status);
     }
   }
   // Never leave the CTA with bulk copies still landing in its shared memory: wait (bounded) for the
@@ -747,6 +773,31 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
     s.gated = p.sigmoid_gate;
     s.hoff = (lane - 16) * p.shared_inter;
   }
+  const int nslots = p.n_shared + rt.nbig + rt.nsmall;
+  // phase-2 chunk and unit counts before each slot: lane j handles slot j (8-bit: shared and the first nbig routed)
+  {
+    int cj = 0, uj = 0;
+    if (lane < nslots) {
+      const int inter = lane < p.n_shared ? p.shared_inter : p.inter;
+      const bool p8 = lane < p.n_shared + rt.nbig;
+      cj = nchunks_of(inter);
+      uj = p8 ? 2 * cj : cj;
+    }
+    int ci = cj, ui = uj;  // inclusive scans
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int a = __shfl_up_sync(0xffffffffu, ci, off), b = __shfl_up_sync(0xffffffffu, ui, off);
+      if (lane >= off) {
+        ci += a;
+        ui += b;
+      }
+    }
+    if (lane < nslots) {
+      plan->p2c[lane + 1] = (short)ci;
+      plan->p2u[lane + 1] = (short)ui;
+    }
+    if (lane == 0) plan->p2c[0] = plan->p2u[0] = 0;
+  }
   if (lane == 0) {
     const unsigned nsh = (unsigned)p.n_shared, nbig = (unsigned)rt.nbig, nsmall = (unsigned)rt.nsmall;
     const unsigned nts = nsh ? (unsigned)p.shared_inter / 16u : 0u, ntr = (unsigned)p.inter / 16u;
@@ -773,10 +824,13 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
       slot = (int)(nsh + (o0 - T1) / ntr);
       idx = (int)((o0 - T1) % ntr);
     }
-    const int nslots = (int)(nsh + nbig + nsmall);
     plan->first_slot = slot;
     plan->first_idx = idx;
     plan->count1 = (int)(o1 - o0);
+    // phase-1 chunks of this CTA: 2 nch per 8-bit task, nch per 4-bit task
+    const unsigned big_end = T1 + T2;
+    const unsigned nb = (o0 < big_end ? (o1 < big_end ? o1 : big_end) - o0 : 0u);
+    plan->chunks1 = (int)(nb * 2u * nch + ((o1 - o0) - nb) * nch);
     const int nrb = p.hidden / 16;
     plan->count2 = (nslots > 0 && (int)blockIdx.x < nrb) ? (nrb - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     plan->nslots = nslots;
@@ -842,16 +896,17 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
       *reinterpret_cast<int*>(smem + SmemLayout::dead) = 0;
       const uint32_t bars = smem_u32(smem + SmemLayout::bars);
       for (int s = 0; s < kUnits; ++s) {
-        mbar_init(bars + 8 * s, 1);                           // full: lane 0's expect_tx arrive
-        mbar_init(bars + 8 * kUnits + 8 * s, kGroupWarps);  // empty: one arrive per warp of the group
+        mbar_init(bars + 8 * (Bars::full + s), 1);             // lane 0's expect_tx arrive
+        mbar_init(bars + 8 * (Bars::empty + s), kGroupWarps);  // one arrive per warp of the consuming group
       }
-      const uint32_t xbars = bars + 16 * kUnits;
-      mbar_init(xbars + 8 * kBarPFull0, kConsumerWarps);
-      mbar_init(xbars + 8 * kBarPFull1, kConsumerWarps);
-      mbar_init(xbars + 8 * kBarPEmpty0, 1);
-      mbar_init(xbars + 8 * kBarPEmpty1, 1);
-      mbar_init(xbars + 8 * kBarHxGo, 1);
-      mbar_init(xbars + 8 * kBarHsReady, kConsumerWarps);
+      for (int g = 0; g < kGroups; ++g) {
+        mbar_init(bars + 8 * (Bars::pfull1 + g), kGroupWarps);
+        mbar_init(bars + 8 * (Bars::pempty1 + g), 1);
+      }
+      mbar_init(bars + 8 * Bars::pfull2, kConsumerWarps);
+      mbar_init(bars + 8 * Bars::pempty2, 1);
+      mbar_init(bars + 8 * Bars::hx_go, 1);
+      mbar_init(bars + 8 * Bars::hs_ready, kConsumerWarps);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
