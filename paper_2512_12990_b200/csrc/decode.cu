@@ -17,8 +17,8 @@
 //     three balanced base-256 digits (int8).  The digits sit in separate columns of the B operand of
 //     mma.sync m16n8k32 (u8 x s8 -> s32); the A operand is the raw nibble plane: the layout stores
 //     the two row halves of a fragment in the low and high nibbles of each byte, so `w & 0x0f0f0f0f`
-//     and `w & 0xf0f0f0f0` are the whole unpack (the second half comes out 16 times too large, which
-//     the per-row fold divides away).  Sums are exact in int32; MSB and LSB planes combine as
+//     and `w` itself are the whole unpack (the second half then carries 16 x its rows plus the first
+//     half's, which one subtraction and the fold weight undo).  Sums are exact in int32; MSB and LSB planes combine as
 //     16 * Cm + Cl.  Scale and zero-point are applied once per (row, group):
 //        sum_k x_k s (q_k - zp) = s (sum_k q_k x_k - zp sum_{k in group} x_k).
 //     The plain ALUs could not unpack + convert + FMA two weights per byte at HBM rate; this costs
@@ -41,8 +41,10 @@ constexpr int kGroups = 4;       // consumer groups: a phase-1 task belongs to o
 constexpr int kGroupWarps = 4;   // warps of a group; they split the 128-column blocks of the chunk
 static_assert(kGroups * kGroupWarps == kConsumerWarps, "groups");
 constexpr int kEpilogueWarp = kConsumerWarps;
-constexpr int kProducerWarp = kConsumerWarps + 1;
-constexpr int kThreads = 32 * (kConsumerWarps + 2);
+constexpr int kProducerWarp = kConsumerWarps + 1;  // first of kProducers producer warps
+constexpr int kProducers = 2;                      // they take alternate tasks (phase 1) / chunks (phase 2)
+constexpr int kThreads = 32 * (kConsumerWarps + 1 + kProducers);
+constexpr int kUnits2 = 16;                        // at most this many (smaller) units in phase 2
 constexpr int kUnits = 8;                                 // ring units; a chunk takes one per plane
 constexpr int kChunkK = 2048;                             // K columns per chunk (16 blocks of 128)
 constexpr int kBlocksPerWarp = kChunkK / 128 / kGroupWarps;
@@ -110,6 +112,9 @@ struct Slot {
 //   phase 2: tasks m = 0 .. count2-1 are the output row blocks blockIdx.x + m * gridDim.x; each is one run of
 //     chunks over the slots in order (p2c[j] chunks and p2u[j] units come before slot j), two units per
 //     chunk for 8-bit slots and one for 4-bit slots.  Chunk number c is consumed by group c % kGroups.
+//     Phase 2 re-cuts the ring into nunits2 units of unit2_bytes, just large enough for the widest down
+//     chunk (plane area, then scales at scale2_off, zero-points at zp2_off), so that more - for the
+//     benchmark shapes all - of the phase's tiles are in shared memory before h arrives.
 struct Plan {
   int first_slot, first_idx, count1;
   int count2;
@@ -117,6 +122,7 @@ struct Plan {
   int htotal;   // sum of the slots' intermediate widths
   float gate;   // sigmoid(gate_vec . x) when the shared experts are gated
   int chunks1;  // chunks of phase 1
+  int unit2_bytes, nunits2, scale2_off, zp2_off;
   short p2c[kMaxSlots + 1], p2u[kMaxSlots + 1];
 };
 
@@ -133,7 +139,7 @@ struct SmemLayout {
   static constexpr int slots = partial + kConsumerWarps * 16 * 2 * 4;
   static constexpr int plan = slots + kMaxSlots * (int)sizeof(Slot);
   static constexpr int bars = (plan + (int)sizeof(Plan) + 15) & ~15;  // uint64 barriers
-  static constexpr int nbars = 2 * kUnits + 2 * kGroups + 4;
+  static constexpr int nbars = 2 * kUnits + 2 * kUnits2 + 2 * kGroups + 5;
   static constexpr int dead = bars + nbars * 8;
   static constexpr int total = dead + 16;
 };
@@ -143,13 +149,16 @@ static_assert(SmemLayout::slots % 8 == 0 && SmemLayout::hdig % 16 == 0 && SmemLa
                   SmemLayout::plan % 8 == 0 && SmemLayout::partial % 8 == 0,
               "alignment");
 
-// Barrier indices: full[c % kUnits] for chunk number c (armed with the chunk's bytes), empty[u] for unit u
-// (an arrive from each warp of the group that consumed it), pfull1 / pempty1 per group (phase-1 partial rows
+// Barrier indices: full[c % kUnits] for phase-1 chunk number c (armed with the chunk's bytes), empty[u] for
+// unit u (an arrive from each warp of the group that consumed it), full2 / empty2 likewise for phase 2
+// (chunk numbers and units counted from the start of the phase), pfull1 / pempty1 per group (phase-1 partial rows
 // to the epilogue warp and back), pfull2 / pempty2 (phase-2 partial rows of all warps), hx_go (h is complete
-// in the workspace), hs_ready (h is in shared memory as digits).
+// in the workspace), hs_ready (h is in shared memory as digits), p1_done (every consumer warp is through with
+// phase 1, so the ring may be re-cut).
 struct Bars {
-  static constexpr int full = 0, empty = kUnits, pfull1 = 2 * kUnits, pempty1 = 2 * kUnits + kGroups,
-                       pfull2 = 2 * kUnits + 2 * kGroups, pempty2 = pfull2 + 1, hx_go = pfull2 + 2, hs_ready = pfull2 + 3;
+  static constexpr int full = 0, empty = kUnits, full2 = 2 * kUnits, empty2 = full2 + kUnits2, pfull1 = empty2 + kUnits2,
+                       pempty1 = pfull1 + kGroups, pfull2 = pempty1 + kGroups, pempty2 = pfull2 + 1, hx_go = pfull2 + 2,
+                       hs_ready = pfull2 + 3, p1_done = pfull2 + 4;
 };
 
 // ---- PTX helpers -------------------------------------------------------------------------------
@@ -204,6 +213,14 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, 
   asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// d = a * b (no accumulator input: the first step of a chain)
+__device__ __forceinline__ void mma_u8s8_first(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  const int z = 0;
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(z));
 }
 __device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
   asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
@@ -309,25 +326,47 @@ struct LaneRole {
   float w0, w1;
 };
 
-// One chunk: this warp's 128-column blocks of the 16-row tile(s) in units u0 (and u1).  The A operand is
-// the raw nibble plane, the B operand the activation digits starting at `dig`; `sumw` / `binv` are the
+// One chunk: this warp's 128-column blocks of the 16-row tile(s) in unit0 (and unit1).  The A operand is
+// the nibble plane, the B operand the activation digits starting at `dig`; `sumw` / `binv` are the
 // digits' weighted group sums and block scales for the same columns.
 //   kModeSingle: MSB tile only           -> *out0 += 16 s (Cm - (zp >> 4) X)
 //   kModeBoth:   MSB tile, LSB tile      -> *out0 += s (16 Cm + Cl - zp X)
 //   kModePair:   two matrices' MSB tiles -> *out0 += first, *out1 += second (each with its own scales)
-// Lane roles: lanes with c in {0, 1} take the accumulators of row g, lanes with c in {2, 3} those of row
-// g + 8 (16 times too large, because their nibbles were left in the high half of the byte); even c holds
-// digits 0 and 1, odd c digit 2 (and the unused fourth column).  The caller adds the two digit halves
-// (a shuffle with lane ^ 1) once per task.
+// Unpacking: a plane byte holds row g's nibble (low) and row g + 8's (high).  The fragment registers of
+// row g are the bytes masked to their low nibble; those of row g + 8 are the bytes as they are, worth
+// 16 * high + low, so that accumulator rows g + 8 come out as 16 * C[g + 8] + C[g] and one subtraction per
+// folded value recovers 16 * C[g + 8] (the 16 goes into the lane's fold weight).  One AND per register pair.
+// Lane roles: lanes with c in {0, 1} fold row g, lanes with c in {2, 3} row g + 8; even c holds digits 0
+// and 1, odd c digit 2 (and the unused fourth column).  The caller adds the two digit halves (a shuffle
+// with lane ^ 1) once per task.
 template <int G>
-__device__ __forceinline__ void consume_chunk(const uint8_t* smem, const LaneRole& lr, int lane, int gw, int rot, int mode,
-                                              int nblocks, int u0, int u1, const uint8_t* dig, const float* sumw,
-                                              const float* binv, float* out0, float* out1) {
+__device__ __forceinline__ void pass_mma(int (&acc)[128 / G][4], const uint8_t* ap, const uint2& bv0, const uint2& bv1,
+                                         const uint2& bv2, const uint2& bv3) {
+  const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
+  const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
+  constexpr uint32_t kLow = 0x0f0f0f0fu;
+  mma_u8s8_first(acc[0], wlo.x & kLow, wlo.x, wlo.y & kLow, wlo.y, bv0.x, bv0.y);
+  if (G == 32) {
+    mma_u8s8_first(acc[32 / G], wlo.z & kLow, wlo.z, wlo.w & kLow, wlo.w, bv1.x, bv1.y);
+    mma_u8s8_first(acc[64 / G], whi.x & kLow, whi.x, whi.y & kLow, whi.y, bv2.x, bv2.y);
+    mma_u8s8_first(acc[96 / G], whi.z & kLow, whi.z, whi.w & kLow, whi.w, bv3.x, bv3.y);
+  } else if (G == 64) {
+    mma_u8s8_first(acc[64 / G], whi.x & kLow, whi.x, whi.y & kLow, whi.y, bv2.x, bv2.y);
+    mma_u8s8(acc[0], wlo.z & kLow, wlo.z, wlo.w & kLow, wlo.w, bv1.x, bv1.y);
+    mma_u8s8(acc[64 / G], whi.z & kLow, whi.z, whi.w & kLow, whi.w, bv3.x, bv3.y);
+  } else {
+    mma_u8s8(acc[0], wlo.z & kLow, wlo.z, wlo.w & kLow, wlo.w, bv1.x, bv1.y);
+    mma_u8s8(acc[0], whi.x & kLow, whi.x, whi.y & kLow, whi.y, bv2.x, bv2.y);
+    mma_u8s8(acc[0], whi.z & kLow, whi.z, whi.w & kLow, whi.w, bv3.x, bv3.y);
+  }
+}
+
+template <int G>
+__device__ __forceinline__ void consume_chunk(const LaneRole& lr, int lane, int gw, int rot, int mode, int nblocks,
+                                              const uint8_t* unit0, const uint8_t* unit1, int scale_off, int zp_off,
+                                              const uint8_t* dig, const float* sumw, const float* binv, float* out0,
+                                              float* out1) {
   constexpr int SG = 128 / G;
-  constexpr int NACC = G == 32 ? 4 : 2;  // accumulators per plane pass
-  constexpr int kA1 = G == 32 ? 1 : 0, kA2 = G == 32 ? 2 : 1, kA3 = G == 32 ? 3 : 1;  // accumulator of each 32-column step
-  const uint8_t* unit0 = smem + SmemLayout::ring + u0 * kUnitBytes;
-  const uint8_t* unit1 = smem + SmemLayout::ring + u1 * kUnitBytes;
   const bool p8 = mode == kModeBoth, pair = mode == kModePair;
   const float pfix = p8 ? 1.f : 16.f;
   const int zsh = p8 ? 0 : 4;
@@ -337,78 +376,46 @@ __device__ __forceinline__ void consume_chunk(const uint8_t* smem, const LaneRol
   for (int j = 0; j < kBlocksPerWarp; ++j) {
     const int b = (gw + kGroupWarps - rot) % kGroupWarps + kGroupWarps * j;  // 128-column block of the chunk
     if (b < nblocks) {
-      // Two plane passes with their own accumulators, two (G >= 64) or four (G = 32) per pass, so that the
-      // eight MMAs of a block form four independent chains instead of one.
-      int m[NACC][4], l[NACC][4];
-#pragma unroll
-      for (int a2 = 0; a2 < NACC; ++a2)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) m[a2][q] = l[a2][q] = 0;
       const uint8_t* bp = dig + lr.boff + b * 384;
       const uint2 bv0 = *reinterpret_cast<const uint2*>(bp);
       const uint2 bv1 = *reinterpret_cast<const uint2*>(bp + 96);
       const uint2 bv2 = *reinterpret_cast<const uint2*>(bp + 192);
       const uint2 bv3 = *reinterpret_cast<const uint2*>(bp + 288);
-      {
-        const uint8_t* ap = unit0 + b * 1024 + lane * 16;
-        const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
-        const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
-        mma_u8s8(m[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
-        mma_u8s8(m[kA1], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x, bv1.y);
-        mma_u8s8(m[kA2], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x, bv2.y);
-        mma_u8s8(m[kA3], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x, bv3.y);
-      }
-      if (mode != kModeSingle) {
-        const uint8_t* ap = unit1 + b * 1024 + lane * 16;
-        const uint4 wlo = *reinterpret_cast<const uint4*>(ap);
-        const uint4 whi = *reinterpret_cast<const uint4*>(ap + 512);
-        mma_u8s8(l[0], wlo.x & 0x0f0f0f0fu, wlo.x & 0xf0f0f0f0u, wlo.y & 0x0f0f0f0fu, wlo.y & 0xf0f0f0f0u, bv0.x, bv0.y);
-        mma_u8s8(l[kA1], wlo.z & 0x0f0f0f0fu, wlo.z & 0xf0f0f0f0u, wlo.w & 0x0f0f0f0fu, wlo.w & 0xf0f0f0f0u, bv1.x, bv1.y);
-        mma_u8s8(l[kA2], whi.x & 0x0f0f0f0fu, whi.x & 0xf0f0f0f0u, whi.y & 0x0f0f0f0fu, whi.y & 0xf0f0f0f0u, bv2.x, bv2.y);
-        mma_u8s8(l[kA3], whi.z & 0x0f0f0f0fu, whi.z & 0xf0f0f0f0u, whi.w & 0x0f0f0f0fu, whi.w & 0xf0f0f0f0u, bv3.x, bv3.y);
-      }
-      // this lane's row and digit columns of every group's sums
-      int ca0[SG], cb0[SG], ca1[SG], cb1[SG];
+      int m[SG][4], l[SG][4];
+      pass_mma<G>(m, unit0 + b * 1024 + lane * 16, bv0, bv1, bv2, bv3);
+      if (mode != kModeSingle) pass_mma<G>(l, unit1 + b * 1024 + lane * 16, bv0, bv1, bv2, bv3);
+      const float sfix = pfix * binv[b];
+      const uint16_t* ms = reinterpret_cast<const uint16_t*>(unit0 + scale_off) + (b * SG) * 16 + lr.r;
+      const uint8_t* mz = unit0 + zp_off + (b * SG) * 16 + lr.r;
 #pragma unroll
       for (int sg = 0; sg < SG; ++sg) {
-        const int i0 = G == 128 ? 0 : sg;
-        ca0[sg] = hi ? m[i0][2] : m[i0][0];
-        cb0[sg] = hi ? m[i0][3] : m[i0][1];
-        ca1[sg] = hi ? l[i0][2] : l[i0][0];
-        cb1[sg] = hi ? l[i0][3] : l[i0][1];
-        if (G == 128) {
-          ca0[sg] += hi ? m[1][2] : m[1][0];
-          cb0[sg] += hi ? m[1][3] : m[1][1];
-          ca1[sg] += hi ? l[1][2] : l[1][0];
-          cb1[sg] += hi ? l[1][3] : l[1][1];
+        // this lane's row (g, or 16 x row g + 8) and digit columns
+        int ca = hi ? m[sg][2] - m[sg][0] : m[sg][0];
+        int cb = hi ? m[sg][3] - m[sg][1] : m[sg][1];
+        int ca1 = 0, cb1 = 0;
+        if (mode != kModeSingle) {
+          ca1 = hi ? l[sg][2] - l[sg][0] : l[sg][0];
+          cb1 = hi ? l[sg][3] - l[sg][1] : l[sg][1];
         }
         if (p8) {  // both slices: 16 Cm + Cl
-          ca0[sg] = (ca0[sg] << 4) + ca1[sg];
-          cb0[sg] = (cb0[sg] << 4) + cb1[sg];
+          ca = (ca << 4) + ca1;
+          cb = (cb << 4) + cb1;
         }
-      }
-      // fold: scales / zero-points travel with the unit whose plane they belong to
-      const float sfix = pfix * binv[b];
-      {
-        const uint16_t* ms = reinterpret_cast<const uint16_t*>(unit0 + kPlaneUnitBytes) + (b * SG) * 16 + lr.r;
-        const uint8_t* mz = unit0 + kPlaneUnitBytes + kScaleUnitBytes + (b * SG) * 16 + lr.r;
-#pragma unroll
-        for (int sg = 0; sg < SG; ++sg) {
-          const float t = fmaf((float)cb0[sg], lr.w1, (float)ca0[sg] * lr.w0);
+        const float x0 = sumw[(b * SG + sg) * 2 + lr.cq];
+        {
+          const float t = fmaf((float)cb, lr.w1, (float)ca * lr.w0);
           const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
           const float z = (float)((int)mz[sg * 16] >> zsh);
-          acc0 = fmaf(sc, fmaf(-z, sumw[(b * SG + sg) * 2 + lr.cq], t), acc0);
+          // both slices: s (16 Cm + Cl - zp X); MSB only: 16 s (Cm - (zp >> 4) X)
+          acc0 = fmaf(sc, fmaf(-z, x0, t), acc0);
         }
-      }
-      if (pair) {
-        const uint16_t* ms = reinterpret_cast<const uint16_t*>(unit1 + kPlaneUnitBytes) + (b * SG) * 16 + lr.r;
-        const uint8_t* mz = unit1 + kPlaneUnitBytes + kScaleUnitBytes + (b * SG) * 16 + lr.r;
-#pragma unroll
-        for (int sg = 0; sg < SG; ++sg) {
-          const float t = fmaf((float)cb1[sg], lr.w1, (float)ca1[sg] * lr.w0);
-          const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
-          const float z = (float)((int)mz[sg * 16] >> 4);
-          acc1 = fmaf(sc, fmaf(-z, sumw[(b * SG + sg) * 2 + lr.cq], t), acc1);
+        if (pair) {  // the second matrix' scales / zero-points travel in the second unit
+          const uint16_t* ms1 = reinterpret_cast<const uint16_t*>(unit1 + scale_off) + (b * SG) * 16 + lr.r;
+          const uint8_t* mz1 = unit1 + zp_off + (b * SG) * 16 + lr.r;
+          const float t = fmaf((float)cb1, lr.w1, (float)ca1 * lr.w0);
+          const float sc = __half2float(__ushort_as_half(ms1[sg * 16])) * sfix;
+          const float z = (float)((int)mz1[sg * 16] >> 4);
+          acc1 = fmaf(sc, fmaf(-z, x0, t), acc1);
         }
       }
     }
@@ -457,11 +464,13 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
           const uint8_t* dig = smem + SmemLayout::xdig + kc * (kChunkK * 3);
           const float* sumw = reinterpret_cast<const float*>(smem + SmemLayout::xsumw) + kc * (kChunkK >> LG) * 2;
           const float* binv = reinterpret_cast<const float*>(smem + SmemLayout::xinv) + kc * (kChunkK >> 7);
+          const uint8_t* unit0 = smem + SmemLayout::ring + u0 * kUnitBytes;
           if (sl.prec) {
-            consume_chunk<G>(smem, lr, lane, gw, c % kGroupWarps, kModeBoth, nblocks, u0, u1, dig, sumw, binv,
-                             q < nch ? &part0 : &part1, &unused);
+            consume_chunk<G>(lr, lane, gw, c % kGroupWarps, kModeBoth, nblocks, unit0, unit0 + kUnitBytes, kPlaneUnitBytes,
+                             kPlaneUnitBytes + kScaleUnitBytes, dig, sumw, binv, q < nch ? &part0 : &part1, &unused);
           } else {
-            consume_chunk<G>(smem, lr, lane, gw, c % kGroupWarps, kModePair, nblocks, u0, u1, dig, sumw, binv, &part0, &part1);
+            consume_chunk<G>(lr, lane, gw, c % kGroupWarps, kModePair, nblocks, unit0, unit0 + kUnitBytes, kPlaneUnitBytes,
+                             kPlaneUnitBytes + kScaleUnitBytes, dig, sumw, binv, &part0, &part1);
           }
           __syncwarp();
           if (lane == 0) {
@@ -485,6 +494,8 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
       }
     }
   }
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bars + 8 * Bars::p1_done);  // this warp no longer reads phase-1 units
   if (plan.count2 == 0) return;
 
   // ---- the grid's h ----
@@ -492,6 +503,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
 
   // ---- phase 2: chunks round-robin over the groups, all warps contribute to every task ----
   const int chunks2 = plan.p2c[plan.nslots], units2 = plan.p2u[plan.nslots];
+  const uint32_t full2 = bars + 8 * Bars::full2, empty2 = bars + 8 * Bars::empty2;
   for (int m = 0; m < plan.count2; ++m) {
     float part = 0.f, unused = 0.f;
     for (int j = 0; j < plan.nslots; ++j) {
@@ -500,23 +512,24 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
       float sacc = 0.f;
       bool mine = false;
       for (int kc = 0; kc < nchj; ++kc) {
-        const int c = plan.chunks1 + m * chunks2 + plan.p2c[j] + kc;
+        const int c = m * chunks2 + plan.p2c[j] + kc;  // chunk number within the phase
         if (c % kGroups != group) continue;
         mine = true;
-        if (!mbar_wait(full0 + 8 * (c % kUnits), (c / kUnits) & 1, dead, status)) return;
-        const int unit = 2 * plan.chunks1 + m * units2 + plan.p2u[j] + kc * (sl.prec ? 2 : 1);
-        const int u0 = unit % kUnits, u1 = (unit + 1) % kUnits;
+        if (!mbar_wait(full2 + 8 * (c % kUnits2), (c / kUnits2) & 1, dead, status)) return;
+        const int unit = m * units2 + plan.p2u[j] + kc * (sl.prec ? 2 : 1);
+        const int u0 = unit % plan.nunits2, u1 = (unit + 1) % plan.nunits2;
         const int k0 = kc * kChunkK;
         const int nblocks = min(kChunkK, sl.inter - k0) >> 7;
         const uint8_t* dig = smem + SmemLayout::hdig + (sl.hoff + k0) * 3;
         const float* sumw = reinterpret_cast<const float*>(smem + SmemLayout::hsumw) + ((sl.hoff + k0) >> LG) * 2;
         const float* binv = reinterpret_cast<const float*>(smem + SmemLayout::hinv) + ((sl.hoff + k0) >> 7);
-        consume_chunk<G>(smem, lr, lane, gw, (c / kGroups) % kGroupWarps, sl.prec ? kModeBoth : kModeSingle, nblocks, u0, u1,
-                         dig, sumw, binv, &sacc, &unused);
+        consume_chunk<G>(lr, lane, gw, (c / kGroups) % kGroupWarps, sl.prec ? kModeBoth : kModeSingle, nblocks,
+                         smem + SmemLayout::ring + u0 * plan.unit2_bytes, smem + SmemLayout::ring + u1 * plan.unit2_bytes,
+                         plan.scale2_off, plan.zp2_off, dig, sumw, binv, &sacc, &unused);
         __syncwarp();
         if (lane == 0) {
-          mbar_arrive(empty0 + 8 * u0);
-          if (sl.prec) mbar_arrive(empty0 + 8 * u1);
+          mbar_arrive(empty2 + 8 * u0);
+          if (sl.prec) mbar_arrive(empty2 + 8 * u1);
         }
       }
       if (mine) part = fmaf(sl.gated ? plan.gate : sl.coef, sacc, part);  // weighted combine, in slot order
@@ -604,27 +617,26 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
 // base + (rb * (K / 128) + kb) * bytes_per_block, because planes and scale / zero-point arrays are all
 // stored [row block][column][16 rows].
 constexpr int kProducerLanes = 6;
-struct ProducerState {
-  int cn;    // chunk number: selects the full barrier
-  int unit;  // running unit counter: a chunk takes one unit per plane
-};
 struct ProducerLane {
   uint32_t bytes_per_block;  // bytes per (16 rows x 128 columns)
-  uint32_t dst_in_unit;      // byte offset of the destination inside its unit
   int field;                 // which of the matrix' four pointers
   bool second_unit;
 };
+// The ring as a phase sees it.
+struct RingView {
+  uint32_t full0, empty0;  // shared-memory addresses of the phase's full / empty barriers
+  int nfull, nunits;
+  uint32_t unit_bytes, scale_off, zp_off;
+};
 
-// Streams the chunks of one (slot, row block) of matrix A - or of matrices A and B side by side - into the
-// ring.  Run by the first kProducerLanes lanes of the producer warp together.  Returns false if a wait ran out.
+// One chunk of matrix A - or of matrices A and B side by side - of (slot, row block rb), columns from k0:
+// chunk number cn and first unit number `unit` of its phase.  Run by the first kProducerLanes lanes of a
+// producer warp together.  Returns false if a wait ran out.
 template <int G>
-__device__ __forceinline__ bool produce_chunks(uint8_t* smem, ProducerState& ps, int lane, const ProducerLane& pl,
-                                               const Slot& s, int matA, int matB, int mode, int K, int rb,
-                                               volatile int* dead, unsigned* status) {
+__device__ __forceinline__ bool produce_chunk(uint8_t* smem, const RingView& rv, int cn, int unit, int lane,
+                                              const ProducerLane& pl, const Slot& s, int matA, int matB, int mode, int K,
+                                              int rb, int k0, volatile int* dead, unsigned* status) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
-  const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t full0 = bars + 8 * Bars::full, empty0 = bars + 8 * Bars::empty;
-  const uint32_t ring = smem_u32(smem + SmemLayout::ring);
   const bool two = mode != kModeSingle;
   bool active;
   const uint8_t* src;
@@ -642,77 +654,110 @@ __device__ __forceinline__ bool produce_chunks(uint8_t* smem, ProducerState& ps,
     active = true;
     src = s.ptr[matA][pl.field];
   }
-  src += (size_t)((unsigned)rb * (unsigned)(K >> 7)) * pl.bytes_per_block;
-  const uint32_t bytes_per_block = (two ? 2048u : 1024u) + (mode == kModePair ? 2u : 1u) * ((128u >> LG) * 48u);
-  for (int k0 = 0; k0 < K; k0 += kChunkK) {
-    const uint32_t nblk = (uint32_t)(min(kChunkK, K - k0) >> 7);
-    const int u0 = ps.unit % kUnits, u1 = (ps.unit + 1) % kUnits;
-    if (!mbar_wait(empty0 + 8 * u0, ((ps.unit / kUnits) & 1) ^ 1, dead, status)) return false;
-    if (two && !mbar_wait(empty0 + 8 * u1, (((ps.unit + 1) / kUnits) & 1) ^ 1, dead, status)) return false;
-    const uint32_t bar = full0 + 8 * (ps.cn % kUnits);
-    if (lane == 0) mbar_arrive_expect_tx(bar, nblk * bytes_per_block);
-    __syncwarp((1u << kProducerLanes) - 1u);
-    if (active) {
-      // the second unit wraps around the ring with the unit index
-      const uint32_t dst = ring + (uint32_t)(pl.second_unit ? u1 : u0) * kUnitBytes + pl.dst_in_unit;
-      bulk_g2s(dst, src + (size_t)(k0 >> 7) * pl.bytes_per_block, nblk * pl.bytes_per_block, bar);
-    }
-    ps.unit += two ? 2 : 1;
-    ++ps.cn;
+  src += (size_t)((unsigned)rb * (unsigned)(K >> 7) + (unsigned)(k0 >> 7)) * pl.bytes_per_block;
+  const uint32_t nblk = (uint32_t)(min(kChunkK, K - k0) >> 7);
+  // A chunk's units are released one after the other by the same warps, so the last one's barrier covers both.
+  const int ulast = unit + (two ? 1 : 0);
+  if (!mbar_wait(rv.empty0 + 8 * (ulast % rv.nunits), ((ulast / rv.nunits) & 1) ^ 1, dead, status)) return false;
+  const uint32_t bar = rv.full0 + 8 * (cn % rv.nfull);
+  if (lane == 0)
+    mbar_arrive_expect_tx(bar, nblk * ((two ? 2048u : 1024u) + (mode == kModePair ? 2u : 1u) * ((128u >> LG) * 48u)));
+  __syncwarp((1u << kProducerLanes) - 1u);
+  if (active) {
+    const uint32_t u = (uint32_t)((pl.second_unit ? unit + 1 : unit) % rv.nunits);
+    const uint32_t dst_in_unit = pl.field < 2 ? 0u : (pl.field == 2 ? rv.scale_off : rv.zp_off);
+    bulk_g2s(smem_u32(smem + SmemLayout::ring) + u * rv.unit_bytes + dst_in_unit, src, nblk * pl.bytes_per_block, bar);
   }
   return true;
 }
 
+// Producer warp `which` of kProducers: every producer walks the whole schedule and issues its share.
 template <int G>
-__device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane) {
+__device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, int which) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
   const Slot* slots = reinterpret_cast<const Slot*>(smem + SmemLayout::slots);
   const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  const uint32_t full0 = bars + 8 * Bars::full;
   unsigned* status = &p.ws->status;
-  ProducerState ps;
-  ps.cn = 0;
-  ps.unit = 0;
   ProducerLane pl;
   pl.field = lane < 2 ? lane : 2 + (lane & 1);  // lanes 2, 4: scales; lanes 3, 5: zero-points
   pl.bytes_per_block = lane < 2 ? 1024u : (pl.field == 2 ? (128u >> LG) * 32u : (128u >> LG) * 16u);
-  pl.dst_in_unit = lane < 2 ? 0u : (pl.field == 2 ? (uint32_t)kPlaneUnitBytes : (uint32_t)(kPlaneUnitBytes + kScaleUnitBytes));
   pl.second_unit = lane == 1 || lane >= 4;
   bool ok = true;
-  // phase 1: gate and up of (slot, row block) tasks
+  // phase 1: gate and up of (slot, row block) tasks; two units per chunk
+  RingView r1;
+  r1.full0 = bars + 8 * Bars::full;
+  r1.empty0 = bars + 8 * Bars::empty;
+  r1.nfull = kUnits;
+  r1.nunits = kUnits;
+  r1.unit_bytes = kUnitBytes;
+  r1.scale_off = kPlaneUnitBytes;
+  r1.zp_off = kPlaneUnitBytes + kScaleUnitBytes;
+  const int nch = nchunks_of(p.hidden);
   {
-    int slot = plan.first_slot, idx = plan.first_idx;
+    int slot = plan.first_slot, idx = plan.first_idx, cn = 0;
     for (int n = 0; n < plan.count1 && ok; ++n) {
       const Slot& s = slots[slot];
-      if (s.prec) {
-        ok = produce_chunks<G>(smem, ps, lane, pl, s, 0, 0, kModeBoth, p.hidden, idx, dead, status) &&
-             produce_chunks<G>(smem, ps, lane, pl, s, 1, 1, kModeBoth, p.hidden, idx, dead, status);
-      } else {  // 4-bit slot: gate and up tiles travel together, so that every chunk carries two units
-        ok = produce_chunks<G>(smem, ps, lane, pl, s, 0, 1, kModePair, p.hidden, idx, dead, status);
+      const int nchunks = s.prec ? 2 * nch : nch;
+      if (n % kProducers == which) {
+        for (int q = 0; q < nchunks && ok; ++q) {
+          const int mat = s.prec ? q / nch : 0;
+          ok = produce_chunk<G>(smem, r1, cn + q, 2 * (cn + q), lane, pl, s, mat, s.prec ? mat : 1, s.prec ? kModeBoth : kModePair,
+                                p.hidden, idx, (q % nch) * kChunkK, dead, status);
+        }
       }
+      cn += nchunks;
       if (++idx >= s.inter / 16) {
         idx = 0;
         ++slot;
       }
     }
   }
-  // phase 2: down rows of every slot for the output row blocks of this CTA
+  // phase 2: down rows of every slot for the output row blocks of this CTA, in the re-cut ring
+  RingView r2;
+  r2.full0 = bars + 8 * Bars::full2;
+  r2.empty0 = bars + 8 * Bars::empty2;
+  r2.nfull = kUnits2;
+  r2.nunits = plan.nunits2;
+  r2.unit_bytes = (uint32_t)plan.unit2_bytes;
+  r2.scale_off = (uint32_t)plan.scale2_off;
+  r2.zp_off = (uint32_t)plan.zp2_off;
+  // The re-cut units lie over the phase-1 units: nothing of phase 2 lands before phase 1 has been consumed.
+  // (From then until h has crossed the grid the memory system has nothing else to do.)
+  if (ok && plan.count2 > 0) ok = mbar_wait(bars + 8 * Bars::p1_done, 0, dead, status);
+  int c2 = 0, unit2 = 0;
   for (int m = 0; m < plan.count2 && ok; ++m) {
     const int rb = blockIdx.x + m * gridDim.x;
     for (int slot = 0; slot < plan.nslots && ok; ++slot) {
       const Slot& s = slots[slot];
-      ok = produce_chunks<G>(smem, ps, lane, pl, s, 2, 2, s.prec ? kModeBoth : kModeSingle, s.inter, rb, dead, status);
+      const int w = s.prec ? 2 : 1;
+      for (int k0 = 0; k0 < s.inter && ok; k0 += kChunkK) {
+        if (c2 % kProducers == which) {
+          if (ok)
+            ok = produce_chunk<G>(smem, r2, c2, unit2, lane, pl, s, 2, 2, s.prec ? kModeBoth : kModeSingle, s.inter, rb, k0, dead,
+                                  status);
+        }
+        ++c2;
+        unit2 += w;
+      }
     }
   }
-  // Never leave the CTA with bulk copies still landing in its shared memory: wait (bounded) for the
-  // last kUnits armed barriers.  In the normal path they have all completed long ago.
-  for (int j = max(0, ps.cn - kUnits); j < ps.cn; ++j) {
-    const uint32_t bar = full0 + 8 * (j % kUnits);
-    const long long t0 = clock64();
-    while (!mbar_try(bar, (j / kUnits) & 1)) {
-      if (*dead || (unsigned long long)(clock64() - t0) > kWaitCycles) break;
+  // Never leave the CTA with bulk copies still landing in its shared memory: wait (bounded) until every
+  // barrier this warp may have armed has completed its last phase.  In the normal path they have long ago.
+  {
+    const int cn1 = plan.chunks1;
+    for (int j = max(0, cn1 - kUnits); j < cn1; ++j) {
+      const long long t0 = clock64();
+      while (!mbar_try(r1.full0 + 8 * (j % kUnits), (j / kUnits) & 1)) {
+        if (*dead || (unsigned long long)(clock64() - t0) > kWaitCycles) break;
+      }
+    }
+    for (int j = max(0, c2 - kUnits2); j < c2; ++j) {
+      const long long t0 = clock64();
+      while (!mbar_try(r2.full0 + 8 * (j % kUnits2), (j / kUnits2) & 1)) {
+        if (*dead || (unsigned long long)(clock64() - t0) > kWaitCycles) break;
+      }
     }
   }
 }
@@ -835,6 +880,15 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
     plan->count2 = (nslots > 0 && (int)blockIdx.x < nrb) ? (nrb - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     plan->nslots = nslots;
     plan->htotal = (int)(nsh * (unsigned)p.shared_inter + (nbig + nsmall) * (unsigned)p.inter);
+    // phase-2 units: as large as the widest down chunk of any slot
+    int maxblk = 1;
+    if (nsh) maxblk = max(maxblk, min(kChunkK, p.shared_inter) >> 7);
+    if (nbig + nsmall) maxblk = max(maxblk, min(kChunkK, p.inter) >> 7);
+    const int meta_blk = 16 * (128 / p.group);  // scale entries per 128 columns
+    plan->scale2_off = maxblk * 1024;
+    plan->zp2_off = maxblk * 1024 + maxblk * meta_blk * 2;
+    plan->unit2_bytes = (maxblk * (1024 + meta_blk * 3) + 127) & ~127;
+    plan->nunits2 = min(kUnits2, (kUnits * kUnitBytes) / plan->unit2_bytes);
   }
 }
 
@@ -899,6 +953,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
         mbar_init(bars + 8 * (Bars::full + s), 1);             // lane 0's expect_tx arrive
         mbar_init(bars + 8 * (Bars::empty + s), kGroupWarps);  // one arrive per warp of the consuming group
       }
+      for (int s = 0; s < kUnits2; ++s) {
+        mbar_init(bars + 8 * (Bars::full2 + s), 1);
+        mbar_init(bars + 8 * (Bars::empty2 + s), kGroupWarps);
+      }
       for (int g = 0; g < kGroups; ++g) {
         mbar_init(bars + 8 * (Bars::pfull1 + g), kGroupWarps);
         mbar_init(bars + 8 * (Bars::pempty1 + g), 1);
@@ -907,6 +965,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
       mbar_init(bars + 8 * Bars::pempty2, 1);
       mbar_init(bars + 8 * Bars::hx_go, 1);
       mbar_init(bars + 8 * Bars::hs_ready, kConsumerWarps);
+      mbar_init(bars + 8 * Bars::p1_done, kConsumerWarps);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -924,7 +983,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
       if (lane == 0) plan->gate = 1.f / (1.f + expf(-dot));
     }
   } else {
-    for (int blk = warp - 3; blk < p.hidden / 128; blk += kConsumerWarps - 2) {
+    // warps 3 .. 16 and the second producer warp
+    const int nw = kConsumerWarps - 2 + kProducers - 1;
+    for (int blk = (warp > kProducerWarp ? warp - 1 : warp) - 3; blk < p.hidden / 128; blk += nw) {
       const uint2 raw = *reinterpret_cast<const uint2*>(p.x + blk * 128 + 4 * lane);
       const float v[4] = {__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u),
                           __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u)};
@@ -941,7 +1002,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
   } else if (warp == kEpilogueWarp) {
     epilogue_loop(p, smem, lane);
   } else if (lane < kProducerLanes) {
-    producer_loop<G>(p, smem, lane);
+    producer_loop<G>(p, smem, lane, warp - kProducerWarp);
   }
   __syncthreads();
   if (tid == 0) {
