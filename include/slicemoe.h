@@ -84,6 +84,8 @@ typedef struct slicemoe_expert {
 
 const char *slicemoe_strerror(int code);
 int slicemoe_version(void);
+/* Text of the CUDA runtime error behind the most recent SLICEMOE_E_CUDA of this process ("no error" if none). */
+const char *slicemoe_last_cuda_error(void);
 
 /* ---- sizes ------------------------------------------------------------------------------- */
 size_t slicemoe_plane_bytes(int N, int K);           /* bytes of one slice plane: N*K/2 */

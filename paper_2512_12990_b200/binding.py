@@ -25,7 +25,7 @@ DBSC_STAT_NAMES = ("requests", "msb_hit", "msb_miss", "lsb_hit", "lsb_miss", "ls
 
 # every symbol include/slicemoe.h declares
 EXPORTS = (
-    "slicemoe_strerror", "slicemoe_version", "slicemoe_plane_bytes", "slicemoe_meta_count", "slicemoe_pack",
+    "slicemoe_strerror", "slicemoe_version", "slicemoe_last_cuda_error", "slicemoe_plane_bytes", "slicemoe_meta_count", "slicemoe_pack",
     "slicemoe_unpack_plane", "slicemoe_unpack_meta", "slicemoe_route_topk", "slicemoe_workspace_bytes",
     "slicemoe_workspace_init", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer",
     "slicemoe_decode_step_host", "slicemoe_layer_static", "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
@@ -36,7 +36,10 @@ EXPORTS = (
 class SliceMoEError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
-        super().__init__(f"{where}: {strerror(code)} ({code})")
+        detail = ""
+        if code == E_CUDA:
+            detail = ": " + lib().slicemoe_last_cuda_error().decode()
+        super().__init__(f"{where}: {strerror(code)} ({code}){detail}")
 
 
 class Shape(Structure):
@@ -66,6 +69,7 @@ def lib() -> ctypes.CDLL:
     L.slicemoe_strerror.restype = c_char_p
     L.slicemoe_strerror.argtypes = [c_int]
     L.slicemoe_version.restype = c_int
+    L.slicemoe_last_cuda_error.restype = c_char_p
     L.slicemoe_plane_bytes.restype = c_size_t
     L.slicemoe_plane_bytes.argtypes = [c_int, c_int]
     L.slicemoe_meta_count.restype = c_size_t

@@ -13,3 +13,9 @@ extern "C" const char* slicemoe_strerror(int code) {
 }
 
 extern "C" int slicemoe_version(void) { return 100; }
+
+int g_slicemoe_last_cuda_error = 0;
+
+extern "C" const char* slicemoe_last_cuda_error(void) {
+  return cudaGetErrorString((cudaError_t)g_slicemoe_last_cuda_error);
+}

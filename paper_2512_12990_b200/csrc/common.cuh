@@ -6,16 +6,25 @@
 
 #include "slicemoe.h"
 
-#define SM_CUDA_TRY(expr)                          \
-  do {                                             \
-    cudaError_t _e = (expr);                       \
-    if (_e != cudaSuccess) return SLICEMOE_E_CUDA; \
+// The CUDA error behind the most recent SLICEMOE_E_CUDA (see slicemoe_last_cuda_error).
+extern int g_slicemoe_last_cuda_error;
+
+#define SM_CUDA_TRY(expr)                     \
+  do {                                        \
+    cudaError_t _e = (expr);                  \
+    if (_e != cudaSuccess) {                  \
+      g_slicemoe_last_cuda_error = (int)_e;   \
+      return SLICEMOE_E_CUDA;                 \
+    }                                         \
   } while (0)
 
-#define SM_LAUNCH_CHECK()                          \
-  do {                                             \
-    cudaError_t _e = cudaGetLastError();           \
-    if (_e != cudaSuccess) return SLICEMOE_E_CUDA; \
+#define SM_LAUNCH_CHECK()                     \
+  do {                                        \
+    cudaError_t _e = cudaGetLastError();      \
+    if (_e != cudaSuccess) {                  \
+      g_slicemoe_last_cuda_error = (int)_e;   \
+      return SLICEMOE_E_CUDA;                 \
+    }                                         \
   } while (0)
 
 namespace slicemoe {
