@@ -281,6 +281,23 @@ def run_reference(args, sh):
     print(json.dumps(out), flush=True)
 
 
+# ---- ranks -------------------------------------------------------------------------------------------------
+def max_over_ranks(ms: float, dist=None, device="cpu") -> float:
+    """The slowest rank's time: what every whole-job figure is computed from."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_us_per_unit(ms_max: float, steps_per_rank: int, world: int) -> float:
+    """Replicas only: every rank runs `steps_per_rank` independent steps in the same span, so the job
+    processed steps_per_rank * world units in ms_max milliseconds."""
+    return ms_max * 1e3 / (steps_per_rank * world)
+
+
 # ---- the CUDA arm ----------------------------------------------------------------------------------------
 class DeviceLayers:
     """`n_layers` independently drawn and packed layers of the workload, resident in HBM."""
@@ -414,12 +431,6 @@ def run_cuda(args, sh):
         t1 = time.time()
         return e0.elapsed_time(e1), (t0, t1)
 
-    def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
 
     sampler = ClockSampler(local)
     sampler.start()
@@ -447,8 +458,8 @@ def run_cuda(args, sh):
             g.replay()
     ms, win = timed(plan)
     windows.append(win)
-    ms = max_over_ranks(ms)
-    us_per_layer = ms * 1e3 / (K * world)
+    ms = max_over_ranks(ms, dist, dev)
+    us_per_layer = whole_job_us_per_unit(ms, K, world)
 
     # ---- roofline: the decode kernel alone, back to back ----------------------------------------------
     kplan = [(capture(0, chunk, with_route=False), reps)]
@@ -492,8 +503,8 @@ def run_cuda(args, sh):
     e1.record(stream)
     barrier()
     windows.append((t0, time.time()))
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1))
-    e2e_us = e2e_ms * 1e3 / (Ke * world)
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+    e2e_us = whole_job_us_per_unit(e2e_ms, Ke, world)
     sampler.stop()
     if B.slicemoe_get_status(ws, stream) != 0:
         raise RuntimeError("device status word set during the timed regions")
