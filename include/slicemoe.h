@@ -220,6 +220,40 @@ int slicemoe_decode_step_host(const slicemoe_shape *shape, const slicemoe_expert
                               size_t workspace_bytes, void *stream);
 
 /*
+ * slicemoe_prefill_layer - the layer for a prompt of T tokens at once (Section 3: prefill visits
+ * every expert of a layer, so the expert FFN becomes a grouped dense contraction; Section 5.3:
+ * after prefill each expert is held, and here run, at the precision its cached slices allow).
+ * Tokens are grouped by expert on the device; per 128-token tile the weight tile is dequantised
+ * from the nibble planes to fp16 in shared memory - s*(q - zp), or 16*s*(q_msb - (zp >> 4)) for an
+ * MSB-only expert - and contracted on the tensor cores with fp32 accumulation; h is rounded to
+ * fp16 between the two projections (relative error 2^-11, inside the FFN tolerance).  Each
+ * (token, expert) pair gets its own fp32 result row and y[t] sums them in list order (routed
+ * slots 0..k-1, then the shared experts), so y is bit-reproducible run to run.
+ *   x            device bf16 [T, hidden]
+ *   ids, weights device [T, k] (int32, float32)
+ *   expert_prec  device uint8 [n_experts]: 1 = both slices, 0 = MSB slice only.  Precision is per
+ *                expert, not per (token, slot): all tokens of an expert share its weight tile.
+ *                Shared experts always use both slices.
+ *   y            device float32 [T, hidden], overwritten; 16-byte aligned
+ *   workspace    device, >= slicemoe_prefill_workspace_bytes(shape, T) bytes, 256-byte aligned; holds
+ *                the token lists, the gathered x and h (fp16) and the per-pair result rows (fp32).
+ *                Needs no initialisation; contents are scratch.
+ *   status_out_device  device int32, overwritten: OR of SLICEMOE_STATUS_BAD_EXPERT_ID (a pair whose id
+ *                is outside [0, E) is skipped) and SLICEMOE_STATUS_MISSING_LSB (expert_prec 1 for an
+ *                expert without LSB planes: it runs MSB-only).
+ * Shape limits: hidden, inter, shared_inter multiples of 128 (no upper limit on hidden here);
+ * T * (k + n_shared) <= 2^28.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.  slicemoe_prefill_workspace_bytes returns 0 for a shape or T
+ * that slicemoe_prefill_layer would refuse.
+ */
+size_t slicemoe_prefill_workspace_bytes(const slicemoe_shape *shape, int T);
+int slicemoe_prefill_layer(const slicemoe_shape *shape, const slicemoe_expert *experts,
+                           const slicemoe_expert *shared, const float *shared_gate_vec, const void *x,
+                           int T, const int32_t *ids, const float *weights, const uint8_t *expert_prec,
+                           float *y, void *workspace, size_t workspace_bytes, int *status_out_device,
+                           void *stream);
+
+/*
  * Host-side Dynamic Bit-Sliced Caching bookkeeping (Section 4.1; cache implementation of Section
  * 5.1).  Pure host code: it only turns (expert id, precision request) lists into the precision
  * list the FFN runs with, plus hit/miss accounting.  MSB slices: LRU.  LSB slices: lowest priority,

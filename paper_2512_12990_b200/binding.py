@@ -28,7 +28,8 @@ EXPORTS = (
     "slicemoe_strerror", "slicemoe_version", "slicemoe_last_cuda_error", "slicemoe_plane_bytes", "slicemoe_meta_count", "slicemoe_pack",
     "slicemoe_unpack_plane", "slicemoe_unpack_meta", "slicemoe_route_topk", "slicemoe_workspace_bytes",
     "slicemoe_workspace_init", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer",
-    "slicemoe_decode_step_host", "slicemoe_layer_static", "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
+    "slicemoe_decode_step_host", "slicemoe_layer_static", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
+    "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
     "slicemoe_dbsc_assign", "slicemoe_dbsc_stats", "slicemoe_dbsc_contains",
 )
 
@@ -93,6 +94,10 @@ def lib() -> ctypes.CDLL:
     L.slicemoe_decode_step_host.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                             c_void_p, c_int, c_float, c_int, c_void_p, c_void_p, c_size_t,
                                             c_void_p]
+    L.slicemoe_prefill_workspace_bytes.restype = c_size_t
+    L.slicemoe_prefill_workspace_bytes.argtypes = [POINTER(Shape), c_int]
+    L.slicemoe_prefill_layer.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
+                                         c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
     L.slicemoe_dbsc_create.restype = c_void_p
     L.slicemoe_dbsc_create.argtypes = [c_int64, c_int64, c_int64, c_double, c_int]
     L.slicemoe_dbsc_destroy.restype = None
@@ -288,6 +293,35 @@ def slicemoe_decode_step_host(shape: Shape, experts_tbl, shared_tbl, shared_gate
                                          _stream(stream))
     _check(rc, "slicemoe_decode_step_host")
     return y_host
+
+
+def slicemoe_prefill_workspace_bytes(shape: Shape, T: int) -> int:
+    return int(lib().slicemoe_prefill_workspace_bytes(ctypes.byref(shape), T))
+
+
+def new_prefill_workspace(shape: Shape, T: int, device="cuda"):
+    import torch
+    n = slicemoe_prefill_workspace_bytes(shape, T)
+    if n == 0:
+        raise SliceMoEError(E_INVALID_ARG, "slicemoe_prefill_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def slicemoe_prefill_layer(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x, ids, weights, expert_prec, ws,
+                           y=None, status=None, stream=None):
+    """x: CUDA bf16 [T, hidden]; ids/weights: CUDA [T, k]; expert_prec: CUDA uint8 [E].  Returns (y, status) with
+    status a CUDA int32 [1] tensor (read it after synchronising)."""
+    import torch
+    T = x.shape[0]
+    if y is None:
+        y = torch.empty((T, shape.hidden), dtype=torch.float32, device=x.device)
+    if status is None:
+        status = torch.empty(1, dtype=torch.int32, device=x.device)
+    rc = lib().slicemoe_prefill_layer(ctypes.byref(shape), _ptr(experts_tbl), _ptr(shared_tbl), _ptr(shared_gate_vec),
+                                      _ptr(x), T, _ptr(ids), _ptr(weights), _ptr(expert_prec), _ptr(y), _ptr(ws),
+                                      ws.numel(), _ptr(status), _stream(stream))
+    _check(rc, "slicemoe_prefill_layer")
+    return y, status
 
 
 # ---- host DBSC -------------------------------------------------------------------------------------

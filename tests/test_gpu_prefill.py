@@ -1,0 +1,222 @@
+"""slicemoe_prefill_layer (many tokens, grouped dense contraction on the tensor cores) against the float64
+oracle, through the C ABI.  Same tolerance as the decode path: relative L2 error <= 1e-3 and max-abs error
+<= 2e-3 x output RMS, per token."""
+import numpy as np
+import pytest
+
+from oracle import amat, moe
+from paper_2512_12990_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _dev(a):
+    return _torch().from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _prefill(L: H.Layer, xbits, ids, w, expert_prec):
+    from paper_2512_12990_b200 import binding as B
+    torch = _torch()
+    T = xbits.shape[0]
+    ws = B.new_prefill_workspace(L.cshape, T)
+    x = H.to_dev_bf16(xbits)
+    y, status = B.slicemoe_prefill_layer(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x,
+                                         _dev(ids.astype(np.int32)), _dev(w.astype(np.float32)),
+                                         _dev(expert_prec.astype(np.uint8)), ws)
+    torch.cuda.synchronize()
+    return y.cpu().numpy(), int(status.item())
+
+
+def _oracle(L: H.Layer, x64, ids, w, expert_prec):
+    prec = expert_prec[ids]
+    return moe.layer(x64, L.oracle_list(), ids, prec, w, shared=L.oracle_shared, shared_gate_vec=L.gate_vec)
+
+
+def _small_shape(group, n_shared, gated, seed):
+    return synth.Shape(f"pf_small_g{group}", 256, 128, 8, 2, group, n_shared=n_shared, shared_inter=256 if n_shared else 0,
+                       shared_sigmoid_gate=gated, n_layers=1, seed=seed)
+
+
+@pytest.mark.parametrize("group,n_shared,gated", [(64, 0, False), (128, 1, True), (32, 2, False)])
+def test_small_layers_every_token(group, n_shared, gated):
+    """300 tokens over 8 experts: several 128-row tiles with ragged tails, one expert without any token,
+    mixed per-expert precision; every token compared."""
+    sh = _small_shape(group, n_shared, gated, 4100 + group)
+    L = H.Layer(sh, range(sh.n_experts))
+    T = 300
+    logits = synth.router_logits_normal(sh.seed, ("pf-logits",), T, sh.n_experts)
+    logits[:, 5] = -30.0                       # expert 5 is never selected
+    ids, w, _ = moe.route_topk(logits, sh.top_k)
+    assert not (ids == 5).any()
+    expert_prec = (np.arange(sh.n_experts) % 2).astype(np.uint8)
+    xbits, x64 = H.x_inputs(sh, T, "pf-x")
+    y, status = _prefill(L, xbits, ids, w, expert_prec)
+    assert status == 0
+    y_ref = _oracle(L, x64, ids, w, expert_prec)
+    for t in range(T):
+        H.assert_close(y[t], y_ref[t], f"token {t}")
+    # run to run bit-identical although the row a (token, expert) pair takes may differ
+    y2, _ = _prefill(L, xbits, ids, w, expert_prec)
+    assert np.array_equal(y, y2)
+    # the precision list is honoured: flipping it changes the result by the oracle's amount
+    y_flip, _ = _prefill(L, xbits, ids, w, 1 - expert_prec)
+    y_flip_ref = _oracle(L, x64, ids, w, 1 - expert_prec)
+    H.assert_close(y_flip, y_flip_ref, "flipped precision")
+    assert np.linalg.norm(y_flip_ref - y_ref) > 50 * np.linalg.norm(y - y_ref)
+
+
+def test_single_token_and_agreement_with_decode_kernel():
+    """T = 1 (one ragged tile per expert) and T = 5: the prefill path and the batch-1 decode path agree
+    with the oracle and therefore with each other."""
+    from paper_2512_12990_b200 import binding as B
+    torch = _torch()
+    sh = synth.SHAPES["tiny"]
+    L = H.Layer(sh, range(sh.n_experts))
+    expert_prec = (np.arange(sh.n_experts) >= 4).astype(np.uint8)
+    for T in (1, 5):
+        logits = synth.router_logits_normal(sh.seed, ("pf-logits", T), T, sh.n_experts)
+        ids, w, _ = moe.route_topk(logits, sh.top_k)
+        xbits, x64 = H.x_inputs(sh, T, f"pf-x{T}")
+        y, status = _prefill(L, xbits, ids, w, expert_prec)
+        assert status == 0
+        y_ref = _oracle(L, x64, ids, w, expert_prec)
+        prec = expert_prec[ids]
+        y_dec = B.slicemoe_layer(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, H.to_dev_bf16(xbits),
+                                 _dev(ids.astype(np.int32)), _dev(prec), _dev(w.astype(np.float32)), L.ws)
+        torch.cuda.synchronize()
+        for t in range(T):
+            H.assert_close(y[t], y_ref[t], f"prefill T={T} token {t}")
+            H.assert_close(y_dec[t].cpu().numpy(), y_ref[t], f"decode T={T} token {t}")
+
+
+def test_bad_expert_id_is_reported_and_skipped():
+    from paper_2512_12990_b200 import binding as B
+    sh = synth.SHAPES["tiny"]
+    L = H.Layer(sh, range(sh.n_experts))
+    T = 4
+    logits = synth.router_logits_normal(sh.seed, ("pf-bad",), T, sh.n_experts)
+    ids, w, _ = moe.route_topk(logits, sh.top_k)
+    xbits, x64 = H.x_inputs(sh, T, "pf-bad-x")
+    expert_prec = np.ones(sh.n_experts, dtype=np.uint8)
+    bad = ids.copy()
+    bad[2, 1] = sh.n_experts + 3
+    y, status = _prefill(L, xbits, bad, w, expert_prec)
+    assert status & B.STATUS_BAD_EXPERT_ID
+    # the bad pair is skipped, the rest is computed
+    w_skip = w.copy()
+    w_skip[2, 1] = 0.0
+    y_ref = _oracle(L, x64, ids, w_skip, expert_prec)
+    for t in range(T):
+        H.assert_close(y[t], y_ref[t], f"token {t}")
+
+
+def test_argument_checks():
+    from paper_2512_12990_b200 import binding as B
+    sh = synth.SHAPES["tiny"]
+    cs = B.make_shape(sh.hidden, sh.inter, sh.n_experts, sh.top_k, sh.group)
+    assert B.slicemoe_prefill_workspace_bytes(cs, 0) == 0
+    assert B.slicemoe_prefill_workspace_bytes(cs, 16) > 0
+    odd = B.make_shape(sh.hidden, 96, sh.n_experts, sh.top_k, sh.group)
+    assert B.slicemoe_prefill_workspace_bytes(odd, 16) == 0
+    L = H.Layer(sh, [0, 1])
+    torch = _torch()
+    x = torch.zeros((4, sh.hidden), dtype=torch.bfloat16, device="cuda")
+    ids = torch.zeros((4, sh.top_k), dtype=torch.int32, device="cuda")
+    w = torch.zeros((4, sh.top_k), dtype=torch.float32, device="cuda")
+    ep = torch.zeros(sh.n_experts, dtype=torch.uint8, device="cuda")
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.SliceMoEError) as ei:
+        B.slicemoe_prefill_layer(L.cshape, L.experts_tbl, None, None, x, ids, w, ep, small)
+    assert ei.value.code == B.E_INVALID_ARG
+
+
+# ---- the full-size prefill layer ------------------------------------------------------------------------
+class _QwenPrefill:
+    """2048 tokens, 60 experts x 1408, top-4, one gated shared expert of 5632, half of the experts held at
+    both slices.  All experts are packed on the device; the oracle packs only what the sampled tokens use."""
+
+    def __init__(self):
+        torch = _torch()
+        from paper_2512_12990_b200 import binding as B
+        sh = self.sh = synth.SHAPES["qwen_prefill"]
+        self.cshape = B.make_shape(sh.hidden, sh.inter, sh.n_experts, sh.top_k, sh.group, sh.n_shared,
+                                   sh.shared_inter, sh.shared_sigmoid_gate)
+        self.packed, self._W = [], {}
+
+        def dev_pack(tag, inter):
+            W = synth.expert_weights(sh.seed, 0, tag, sh.hidden, inter)
+            return {k: B.slicemoe_pack(torch.from_numpy(W[k]).cuda(), sh.group) for k in ("gate", "up", "down")}
+
+        for e in range(sh.n_experts):
+            self.packed.append(dev_pack(e, sh.inter))
+        self.packed_shared = [dev_pack("shared0", sh.shared_inter)]
+        self.experts_tbl = B.expert_table(self.packed)
+        self.shared_tbl = B.expert_table(self.packed_shared)
+        self.gate_vec = synth.normal_f32(sh.seed, ("gate_vec", 0), (sh.hidden,), 0.02)
+        self.gate_vec_dev = torch.from_numpy(self.gate_vec).cuda()
+        self.T = 2048
+        logits, _ = synth.zipf_gumbel_logits(sh.seed, ("prefill-logits",), self.T, sh.n_experts, 0.6)
+        self.ids, self.w, _ = moe.route_topk(logits, sh.top_k, renorm=True)
+        self.expert_prec = (synth.rng(sh.seed, "prefill-prec").permutation(sh.n_experts) < sh.n_experts // 2).astype(np.uint8)
+        self.xbits, self.x64 = H.x_inputs(sh, self.T, "prefill-x")
+        self._oracle_experts = {}
+        self._oracle_shared = None
+
+    def oracle_expert(self, e):
+        sh = self.sh
+        if e not in self._oracle_experts:
+            W = synth.expert_weights(sh.seed, 0, int(e), sh.hidden, sh.inter)
+            self._oracle_experts[e] = {k: amat.pack_matrix(W[k], sh.group) for k in ("gate", "up", "down")}
+        return self._oracle_experts[e]
+
+    def oracle_token(self, t):
+        sh = self.sh
+        if self._oracle_shared is None:
+            W = synth.expert_weights(sh.seed, 0, "shared0", sh.hidden, sh.shared_inter)
+            self._oracle_shared = [{k: amat.pack_matrix(W[k], sh.group) for k in ("gate", "up", "down")}]
+        ids = self.ids[t:t + 1]
+        experts = {int(e): self.oracle_expert(int(e)) for e in ids[0]}
+        return moe.layer(self.x64[t:t + 1], experts, ids, self.expert_prec[ids], self.w[t:t + 1],
+                         shared=self._oracle_shared, shared_gate_vec=self.gate_vec)[0]
+
+
+@pytest.fixture(scope="module")
+def qwen_prefill():
+    return _QwenPrefill()
+
+
+def test_full_size_prefill_layer_sampled_tokens(qwen_prefill):
+    from paper_2512_12990_b200 import binding as B
+    torch = _torch()
+    q = qwen_prefill
+    counts = np.bincount(q.ids.ravel(), minlength=q.sh.n_experts)
+    assert counts.min() > 0 and counts.max() > 2 * counts.min(), "every expert is used, load is skewed"
+    ws = B.new_prefill_workspace(q.cshape, q.T)
+    x = H.to_dev_bf16(q.xbits)
+    args = (_dev(q.ids.astype(np.int32)), _dev(q.w.astype(np.float32)), _dev(q.expert_prec))
+    y, status = B.slicemoe_prefill_layer(q.cshape, q.experts_tbl, q.shared_tbl, q.gate_vec_dev, x, *args, ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    y = y.cpu().numpy()
+    assert np.isfinite(y).all()
+    # first and last token, tile boundaries of the shared expert, a few in between
+    for t in (0, 127, 128, 1000, 1777, 2047):
+        H.assert_close(y[t], q.oracle_token(t), f"token {t}")
+    # bit-reproducible
+    y2, _ = B.slicemoe_prefill_layer(q.cshape, q.experts_tbl, q.shared_tbl, q.gate_vec_dev, x, *args, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(y, y2.cpu().numpy())
+    # property that holds at any size: a token's result does not depend on the rest of the batch
+    sel = np.array([0, 127, 128, 1000, 1777, 2047])
+    ws_s = B.new_prefill_workspace(q.cshape, len(sel))
+    y_s, _ = B.slicemoe_prefill_layer(q.cshape, q.experts_tbl, q.shared_tbl, q.gate_vec_dev,
+                                      H.to_dev_bf16(q.xbits[sel]), _dev(q.ids[sel].astype(np.int32)),
+                                      _dev(q.w[sel].astype(np.float32)), _dev(q.expert_prec), ws_s)
+    torch.cuda.synchronize()
+    assert np.array_equal(y_s.cpu().numpy(), y[sel])

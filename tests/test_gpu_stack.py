@@ -1,0 +1,86 @@
+"""Config 4: a DeepSeek-V2-Lite-shaped decode stack - 26 MoE layers, 256 batch-1 decode steps with Zipf(1.1)
+expert popularity and temporal reuse, a unified slice cache of 30 % of the 8-bit expert bytes on the host.
+
+Checked here: routing of all 6,656 (step, layer) rows on the GPU against the oracle (bit-exact ids), the
+host cache (C++) against the oracle cache over the whole trace (identical precision lists and counters),
+and the layer output of sampled (step, layer) pairs against the float64 oracle."""
+import numpy as np
+import pytest
+
+from oracle import moe
+from oracle.dbsc import SliceCache
+from paper_2512_12990_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+TAU = 0.25            # an expert is critical (asks for both slices) when its gating probability is >= TAU
+N_STEPS = 256
+
+
+def _expert_slice_bytes(sh):
+    w = sh.hidden * sh.inter
+    msb = 3 * (w // 2 + (w // sh.group) * 3)      # three MSB planes + scales and zero-points
+    lsb = 3 * (w // 2)
+    return msb, lsb
+
+
+def test_decode_stack_routing_cache_and_sampled_layers():
+    import torch
+    from paper_2512_12990_b200 import binding as B
+    sh = synth.SHAPES["dsv2_stack"]
+    L, E, k = sh.n_layers, sh.n_experts, sh.top_k
+    logits = synth.decode_trace_logits(sh.seed, N_STEPS, L, E, s=1.1, p_repeat=0.5)
+    flat = logits.reshape(-1, E)
+
+    # ---- routing: one call for every (step, layer) row ----
+    ids_d, w_d, pr_d = B.slicemoe_route_topk(torch.from_numpy(flat).cuda(), k, tau=TAU)
+    torch.cuda.synchronize()
+    ids_g, w_g, req_g = ids_d.cpu().numpy(), w_d.cpu().numpy(), pr_d.cpu().numpy()
+    ids, w, _ = moe.route_topk(flat, k)
+    assert np.array_equal(ids_g, ids)
+    assert np.allclose(w_g, w, rtol=2e-6, atol=1e-9)
+    req = moe.precision_request(w, TAU)
+    clear = np.abs(w - TAU) > 1e-6            # the request is decided in fp32 on the GPU: compare away from the edge
+    assert np.array_equal(req_g[clear], req[clear]) and clear.mean() > 0.999
+    crit = req_g.sum(1)
+    assert 0.5 < crit.mean() < 1.0 and crit.max() <= 3        # "0-2 critical experts, below one on average"
+    # temporal reuse: about half of the (step, layer) rows repeat the previous step's expert set
+    same = (ids.reshape(N_STEPS, L, k)[1:] == ids.reshape(N_STEPS, L, k)[:-1]).all(2).mean()
+    assert 0.4 < same < 0.65
+
+    # ---- host slice cache over the whole trace: C++ against the oracle ----
+    msb_b, lsb_b = _expert_slice_bytes(sh)
+    cap = int(0.30 * L * E * (msb_b + lsb_b))
+    c_host, c_orc = B.Dbsc(cap, msb_b, lsb_b), SliceCache(cap, msb_b, lsb_b)
+    ids3, req3 = ids_g.reshape(N_STEPS, L, k), req_g.reshape(N_STEPS, L, k)
+    prec3 = np.zeros_like(req3)
+    for t in range(N_STEPS):
+        for l in range(L):
+            prec3[t, l] = c_host.assign(t, l, ids3[t, l], req3[t, l])
+            for j in range(k):
+                pr, _, _, _ = c_orc.request(t, l, int(ids3[t, l, j]), bool(req3[t, l, j]))
+                assert pr == prec3[t, l, j]
+    st = c_host.stats()
+    for key, val in c_orc.stats.items():
+        assert st[key] == val, key
+    assert st["bytes_used"] <= cap
+    miss_rate = st["bytes_fetched"] / (st["requests"] * (msb_b + lsb_b))
+    print(f"stack: miss rate {miss_rate:.3f} (bytes fetched / 8-bit bytes requested), msb hit "
+          f"{st['msb_hit'] / st['requests']:.3f}, 8-bit executions {st['high_exec'] / st['requests']:.3f}")
+    assert 0.0 < miss_rate < 0.6 and st["msb_hit"] > st["msb_miss"]
+    c_host.close()
+
+    # ---- sampled (step, layer) pairs through slicemoe_layer ----
+    samples = [(0, l) for l in (0, 13, 25)] + [(t, t % L) for t in (1, 5, 9, 16, 96, 255)]
+    for (t, l) in samples:
+        lay = H.Layer(sh, ids3[t, l], layer=l)
+        xbits, x64 = H.x_inputs(sh, 1, ("x-stack", t, l))
+        row = (t * L + l)
+        y = B.slicemoe_layer(lay.cshape, lay.experts_tbl, lay.shared_tbl, None, H.to_dev_bf16(xbits),
+                             ids_d[row:row + 1], torch.from_numpy(prec3[t, l:l + 1].copy()).cuda(), w_d[row:row + 1], lay.ws)
+        torch.cuda.synchronize()
+        assert B.slicemoe_get_status(lay.ws) == 0
+        y_ref = moe.layer(x64, lay.oracle_list(), ids3[t, l:l + 1], prec3[t, l:l + 1], w[row:row + 1], shared=lay.oracle_shared)
+        rel, mx = H.assert_close(y.cpu().numpy(), y_ref, f"stack step {t} layer {l}")
+        del lay
