@@ -13,21 +13,20 @@
 // memory - s * (q - zp) from both slices, 16 s * (q_msb - (zp >> 4)) from the MSB slice alone - and fed
 // to the tensor cores (mma.sync m16n8k16, fp16 x fp16 -> fp32).  fp16 rather than bf16: a dequantised
 // weight needs 11 significant bits to stay inside the parity tolerance, bf16 has 8.
+#include <cuda.h>  // CUtensorMap (types only; the encoder is fetched through the runtime)
 #include <cuda_fp16.h>
 
 #include "common.cuh"
 
 namespace slicemoe {
 
-constexpr int kPfThreads = 512;
 constexpr int kPfTileM = 128;  // token rows per tile
 constexpr int kPfTileB = 128;  // weight rows per tile: 64 gate + 64 up columns of h (GEMM 1), 128 columns of y (GEMM 2)
 constexpr int kPfChunkK = 64;  // contraction columns per pipeline step (one plane block)
-constexpr int kPfStride = kPfChunkK + 8;  // halves per shared-memory row: 144 bytes, conflict-free for ldmatrix
 
 // ---- workspace layout (host and device agree through this one function) --------------------------------
 struct PfLayout {
-  size_t counts, cursor, offsets, tile_expert, tile_row0, ntiles, row_token, posmap, gate, xs, h, yrow, total;
+  size_t counts, cursor, offsets, tile_expert, tile_row0, item_start, ntiles, row_token, posmap, gate, xs, h, yrow, total;
   int rmax, max_tiles, nexp_all;
 };
 __host__ __device__ inline size_t pf_align(size_t v) { return (v + 255) & ~(size_t)255; }
@@ -45,6 +44,7 @@ __host__ __device__ inline PfLayout pf_layout(int T, int E, int k, int n_shared,
   L.offsets = o;      o = pf_align(o + sizeof(int) * (L.nexp_all + 1));
   L.tile_expert = o;  o = pf_align(o + sizeof(int) * L.max_tiles);
   L.tile_row0 = o;    o = pf_align(o + sizeof(int) * L.max_tiles);
+  L.item_start = o;   o = pf_align(o + sizeof(int) * (L.max_tiles + 1));
   L.ntiles = o;       o = pf_align(o + sizeof(int) * 4);
   L.row_token = o;    o = pf_align(o + sizeof(int) * L.rmax);
   L.posmap = o;       o = pf_align(o + sizeof(int) * (size_t)T * (k + n_shared));
@@ -70,23 +70,28 @@ __global__ void pf_count_kernel(const int32_t* __restrict__ ids, int n, int E, i
 }
 
 // One CTA: padded offsets of every expert (routed, then shared with T rows each) and the tile list.
-__global__ void pf_scan_kernel(const int* __restrict__ counts, int E, int n_shared, int T, int* __restrict__ offsets,
-                               int* __restrict__ tile_expert, int* __restrict__ tile_row0, int* __restrict__ ntiles) {
+__global__ void pf_scan_kernel(const int* __restrict__ counts, int E, int n_shared, int T, int inter, int shared_inter,
+                               int* __restrict__ offsets, int* __restrict__ tile_expert, int* __restrict__ tile_row0,
+                               int* __restrict__ item_start, int* __restrict__ ntiles) {
   if (threadIdx.x != 0) return;
-  int off = 0, nt = 0;
+  int off = 0, nt = 0, items = 0;
   for (int e = 0; e < E + n_shared; ++e) {
     const int c = e < E ? counts[e] : T;
     offsets[e] = off;
     for (int r = 0; r < c; r += kPfTileM) {
       tile_expert[nt] = e;
       tile_row0[nt] = off + r;
+      item_start[nt] = items;
+      items += (e < E ? inter : shared_inter) / 64;  // first GEMM: 64 columns of h per work item
       ++nt;
     }
     off += (c + kPfTileM - 1) / kPfTileM * kPfTileM;
   }
   offsets[E + n_shared] = off;
+  item_start[nt] = items;
   ntiles[0] = nt;
   ntiles[1] = off;
+  ntiles[2] = items;
 }
 
 // Every (token, slot) pair takes a row of its expert; shared experts take row t.  Which row a pair gets
@@ -127,25 +132,28 @@ __global__ void pf_gather_kernel(const uint16_t* __restrict__ x, int hidden, con
   }
 }
 
-// ---- steps 3 and 4: the grouped GEMM ------------------------------------------------------------------------
-__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
-  const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst);
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait0() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* p) {
-  const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"(a));
-}
-__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
+// ---- steps 3 and 4: the grouped GEMM on the 5th-generation tensor cores ---------------------------------
+// One persistent CTA per SM walks work items (128 token rows x 128 weight rows).  Per 64-column step of the
+// contraction:
+//   - the load warp brings the A tile (token rows of x or h, fp16) in with one TMA tiled copy, 128-byte swizzle;
+//   - eight dequantisation warps (one per 16-row block of the weight tile) read the nibble planes and the
+//     zero-points and write the INTEGER q - zp (or q_msb - (zp >> 4)), which fp16 holds exactly, into the B tile
+//     in the same swizzled K-major layout;
+//   - one thread issues four tcgen05.mma (M 128, N 128, K 16) that accumulate in tensor memory.
+// At the end of every quantisation group the accumulator (one of two, 128 columns each) is handed to eight
+// epilogue warps, which read it with tcgen05.ld, scale column n by the group's fp16 scale of weight row n in
+// fp32 and add it to the running result in registers; meanwhile the next group accumulates in the other
+// buffer.  No weight is ever rounded.  Every wait is bounded; a wait that runs out sets
+// SLICEMOE_STATUS_WAIT_TIMEOUT and the CTA winds down (tensor memory is freed on every path).
+constexpr int kUThreads = 576;      // warps 0-7 epilogue, 8-15 dequantisation, 16 loads, 17 MMA issue
+constexpr int kUStages = 6;
+constexpr int kUTileBytes = kPfTileM * kPfChunkK * 2;  // 16,384: one operand tile of a step
+constexpr int kUStageBytes = 2 * kUTileBytes;
+constexpr int kUScaleSlots = 16;    // ring of per-group scale rows: dequantisation runs at most 15 groups ahead of the epilogue
+constexpr int kUScaleBytes = kUScaleSlots * kPfTileB * 4;
+constexpr int kUSmemBytes = kUStages * kUStageBytes + kUScaleBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int kUTmemCols = 256;     // two accumulators of 128 fp32 columns
+constexpr long long kUWaitCycles = 2000000000ll;
 
 struct PfGemmParams {
   const slicemoe_expert* experts;  // routed
@@ -153,233 +161,360 @@ struct PfGemmParams {
   const uint8_t* expert_prec;      // per routed expert: 1 = both slices, 0 = MSB slice only
   const int* tile_expert;
   const int* tile_row0;
-  const int* ntiles;
-  const __half* a;                 // phase 1: gathered x [rows, hidden]; phase 2: h [rows, ldh]
-  __half* h;                       // phase 1 output
+  const int* item_start;           // phase 1: first work item of every tile (prefix sum of its n-tiles)
+  const int* ntiles;               // [0] tiles, [1] rows, [2] phase-1 work items
+  __half* h;                       // phase 1 output, phase 2 A operand [rows, ldh]
   float* yrow;                     // phase 2 output [rows, hidden]
   unsigned* status;
   int E, hidden, inter, shared_inter, ldh;
 };
 
-// Two plane words of a thread for one pipeline step, the zero-point offsets of their two rows each,
-// and (for the threads that publish them) one row's scale per quantisation group of the step.
-struct PfBRegs {
-  uint32_t mw[2], lw[2];
-  __half2 off[2][2];  // [word][low-nibble row, high-nibble row]: 1024 + zero-point (or its top 4 bits)
-  float sc[2];        // scale of B row (tid & 127), groups of this step
-};
-
-// PHASE 1: B rows 0-63 = gate rows [64 nt, 64 nt + 64), rows 64-127 = up rows of the same range; K = hidden.
-// PHASE 2: B rows = down rows [128 nt, 128 nt + 128); K = the expert's intermediate width.
-// The tensor cores contract x (or h) with the INTEGER q - zp, which fp16 holds exactly, one quantisation
-// group at a time; at the end of each group the partial sums are scaled by the group's fp16 scale in fp32
-// and added to the running result.  No weight is ever rounded.
-template <int G, int PHASE>
-__global__ void __launch_bounds__(kPfThreads, 1) pf_gemm_kernel(const PfGemmParams p) {
-  constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
-  constexpr int kStepsPerGroup = G / 16;                    // k16 MMA steps per quantisation group
-  constexpr int kGroupsPerChunk = G >= kPfChunkK ? 1 : kPfChunkK / G;
-  const int tile = blockIdx.x;
-  if (tile >= p.ntiles[0]) return;
-  const int e = p.tile_expert[tile], row0 = p.tile_row0[tile], nt = blockIdx.y;
-  const bool is_shared = e >= p.E;
-  const slicemoe_expert& ex = is_shared ? p.shared[e - p.E] : p.experts[e];
-  const int inter = is_shared ? p.shared_inter : p.inter;
-  bool prec = is_shared ? true : (p.expert_prec[e] != 0);
-  if (prec && !(PHASE == 1 ? (ex.gate.lsb && ex.up.lsb) : ex.down.lsb != nullptr)) {
-    // both slices asked of a matrix that has only one: run the MSB slice, tell the caller
-    if (threadIdx.x == 0) atomicOr(p.status, (unsigned)SLICEMOE_STATUS_MISSING_LSB);
-    prec = false;
-  }
-  const int K = PHASE == 1 ? p.hidden : inter;
-  const int nout = PHASE == 1 ? inter / 64 : p.hidden / 128;  // n-tiles this expert has
-  if (nt >= nout) return;
-  const int lda = PHASE == 1 ? p.hidden : p.ldh;
-
-  extern __shared__ __align__(16) uint8_t pf_smem[];
-  __half(*As)[kPfTileM][kPfStride] = reinterpret_cast<__half(*)[kPfTileM][kPfStride]>(pf_smem);
-  __half(*Bs)[kPfTileB][kPfStride] =
-      reinterpret_cast<__half(*)[kPfTileB][kPfStride]>(pf_smem + 2 * sizeof(__half) * kPfTileM * kPfStride);
-  float(*Ss)[2][kPfTileB] = reinterpret_cast<float(*)[2][kPfTileB]>(
-      pf_smem + 2 * sizeof(__half) * (kPfTileM + kPfTileB) * kPfStride);  // [buffer][group of the step][B row]
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int wm = warp & 3, wn = warp >> 2;  // the warp's 32 token rows and 32 B rows (phase 1: 16 gate + 16 up)
-
-  // ---- the thread's two plane words per step: which matrix, row block, position ----
-  const uint32_t* msb[2];
-  const uint32_t* lsb[2];
-  const uint8_t* zpp[2];
-  int brow[2], bk[2];
-#pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    const int ws = tid + kPfThreads * i;
-    const int rbk = ws >> 7, idx = ws & 127, L = idx >> 2, w = idx & 3, g = L >> 2, c = L & 3;
-    const slicemoe_mat& m = PHASE == 1 ? (rbk < 4 ? ex.gate : ex.up) : ex.down;
-    const int rb = PHASE == 1 ? nt * 4 + (rbk & 3) : nt * 8 + rbk;
-    msb[i] = reinterpret_cast<const uint32_t*>(m.msb) + (size_t)rb * (K >> 6) * 128 + idx;
-    lsb[i] = prec ? reinterpret_cast<const uint32_t*>(m.lsb) + (size_t)rb * (K >> 6) * 128 + idx : msb[i];
-    zpp[i] = m.zp + (size_t)rb * (K >> LG) * 16 + g;
-    brow[i] = 16 * rbk + g;
-    bk[i] = 16 * w + 4 * c;
-  }
-  // threads 0..127 publish the scale of B row tid for the first group of a step, 128..255 for the second
-  const uint16_t* scp = nullptr;
-  const int srow = tid & 127, sgrp = tid >> 7;
-  if (sgrp < kGroupsPerChunk) {
-    const int rbk = srow >> 4;
-    const slicemoe_mat& m = PHASE == 1 ? (rbk < 4 ? ex.gate : ex.up) : ex.down;
-    const int rb = PHASE == 1 ? nt * 4 + (rbk & 3) : nt * 8 + rbk;
-    scp = m.scale + (size_t)rb * (K >> LG) * 16 + (srow & 15);
-  }
-  auto load_b = [&](PfBRegs& r, int kc) {
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      r.mw[i] = __ldg(msb[i] + (size_t)kc * 128);
-      r.lw[i] = prec ? __ldg(lsb[i] + (size_t)kc * 128) : 0u;
-      const int grp = (kc * kPfChunkK + bk[i]) >> LG;
-#pragma unroll
-      for (int hi = 0; hi < 2; ++hi) {
-        const int z = __ldg(zpp[i] + grp * 16 + 8 * hi);
-        r.off[i][hi] = __half2half2(__int2half_rn(1024 + (prec ? z : (z >> 4))));
-      }
-    }
-    if (scp) {
-      const int grp = ((kc * kPfChunkK) >> LG) + sgrp;
-      const float s = __half2float(__ushort_as_half(__ldg(scp + grp * 16)));
-      r.sc[0] = prec ? s : 16.f * s;
-    }
-  };
-  auto store_b = [&](const PfBRegs& r, int buf) {
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const uint32_t m0 = r.mw[i], l0 = r.lw[i];
-      const uint32_t qlo = prec ? (((m0 & 0x0f0f0f0fu) << 4) | (l0 & 0x0f0f0f0fu)) : (m0 & 0x0f0f0f0fu);
-      const uint32_t qhi = prec ? ((m0 & 0xf0f0f0f0u) | ((l0 >> 4) & 0x0f0f0f0fu)) : ((m0 >> 4) & 0x0f0f0f0fu);
-#pragma unroll
-      for (int hi = 0; hi < 2; ++hi) {
-        const uint32_t q = hi ? qhi : qlo;
-        // bytes -> fp16 1024 + code, minus (1024 + zero-point): the integer q - zp, exact
-        uint32_t h01 = __byte_perm(q, 0x64646464u, 0x4140), h23 = __byte_perm(q, 0x64646464u, 0x4342);
-        __half2 w01 = __hsub2(*reinterpret_cast<__half2*>(&h01), r.off[i][hi]);
-        __half2 w23 = __hsub2(*reinterpret_cast<__half2*>(&h23), r.off[i][hi]);
-        uint2 o;
-        o.x = *reinterpret_cast<uint32_t*>(&w01);
-        o.y = *reinterpret_cast<uint32_t*>(&w23);
-        *reinterpret_cast<uint2*>(&Bs[buf][brow[i] + 8 * hi][bk[i]]) = o;
-      }
-    }
-    if (scp) Ss[buf][sgrp][srow] = r.sc[0];
-  };
-  auto load_a = [&](int buf, int kc) {
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int ci = tid + kPfThreads * i, row = ci >> 3, seg = ci & 7;
-      cp_async16(&As[buf][row][seg * 8], p.a + (size_t)(row0 + row) * lda + (size_t)kc * kPfChunkK + seg * 8);
-    }
-    cp_async_commit();
-  };
-
-  // B rows of the warp's four n8 tiles (tiles 2 jp, 2 jp + 1 are adjacent)
-  int nrow[2];
-#pragma unroll
-  for (int jp = 0; jp < 2; ++jp) nrow[jp] = PHASE == 1 ? 64 * jp + 16 * wn : 32 * wn + 16 * jp;
-
-  float acc[2][4][4], tot[2][4][4];
-#pragma unroll
-  for (int i = 0; i < 2; ++i)
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) acc[i][j][q] = tot[i][j][q] = 0.f;
-
-  const int nk = K / kPfChunkK;
-  const int c2 = 2 * (lane & 3);
-  PfBRegs breg;
-  load_a(0, 0);
-  load_b(breg, 0);
-  store_b(breg, 0);
-  cp_async_wait0();
-  __syncthreads();
-  for (int kc = 0; kc < nk; ++kc) {
-    const int buf = kc & 1;
-    const bool more = kc + 1 < nk;
-    if (more) {
-      load_a(buf ^ 1, kc + 1);
-      load_b(breg, kc + 1);
-    }
-#pragma unroll
-    for (int ks = 0; ks < kPfChunkK / 16; ++ks) {
-      uint32_t af[2][4];
-#pragma unroll
-      for (int i = 0; i < 2; ++i)
-        ldmatrix_x4(af[i], &As[buf][32 * wm + 16 * i + (lane & 15)][16 * ks + (lane >> 4) * 8]);
-#pragma unroll
-      for (int jp = 0; jp < 2; ++jp) {
-        uint32_t bf[4];
-        ldmatrix_x4(bf, &Bs[buf][nrow[jp] + (lane & 7) + ((lane >> 4) << 3)][16 * ks + ((lane >> 3) & 1) * 8]);
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          mma_f16(acc[i][2 * jp], af[i], bf[0], bf[1]);
-          mma_f16(acc[i][2 * jp + 1], af[i], bf[2], bf[3]);
-        }
-      }
-      // end of a quantisation group: scale the group's sums, add them to the result, start over
-      const int step = kc * (kPfChunkK / 16) + ks;
-      if ((step + 1) % kStepsPerGroup == 0) {
-        const int gi = kGroupsPerChunk == 1 ? 0 : (ks * 16) / G;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float2 s = *reinterpret_cast<const float2*>(&Ss[buf][gi][nrow[j >> 1] + 8 * (j & 1) + c2]);
-#pragma unroll
-          for (int i = 0; i < 2; ++i) {
-            tot[i][j][0] = fmaf(s.x, acc[i][j][0], tot[i][j][0]);
-            tot[i][j][1] = fmaf(s.y, acc[i][j][1], tot[i][j][1]);
-            tot[i][j][2] = fmaf(s.x, acc[i][j][2], tot[i][j][2]);
-            tot[i][j][3] = fmaf(s.y, acc[i][j][3], tot[i][j][3]);
-            acc[i][j][0] = acc[i][j][1] = acc[i][j][2] = acc[i][j][3] = 0.f;
-          }
-        }
-      }
-    }
-    if (more) {
-      store_b(breg, buf ^ 1);
-      cp_async_wait0();
-    }
-    __syncthreads();
-  }
-
-  // ---- epilogue ----
-  const int g = lane >> 2;
-  if (PHASE == 1) {
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-#pragma unroll
-      for (int j = 0; j < 2; ++j)
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          const float g0 = tot[i][j][2 * hf], g1 = tot[i][j][2 * hf + 1];
-          const float u0 = tot[i][j + 2][2 * hf], u1 = tot[i][j + 2][2 * hf + 1];
-          const float h0 = g0 / (1.f + __expf(-g0)) * u0, h1 = g1 / (1.f + __expf(-g1)) * u1;
-          const int row = row0 + 32 * wm + 16 * i + g + 8 * hf;
-          const int col = 64 * nt + 16 * wn + 8 * j + c2;
-          *reinterpret_cast<__half2*>(p.h + (size_t)row * p.ldh + col) = __floats2half2_rn(h0, h1);
-        }
-  } else {
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          const int row = row0 + 32 * wm + 16 * i + g + 8 * hf;
-          const int col = 128 * nt + 32 * wn + 8 * j + c2;
-          *reinterpret_cast<float2*>(p.yrow + (size_t)row * p.hidden + col) =
-              make_float2(tot[i][j][2 * hf], tot[i][j][2 * hf + 1]);
-        }
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
+}
+// Bounded wait for the phase of the given parity; false when the limit ran out or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+  const long long t0 = clock64();
+  for (;;) {
+    uint32_t ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok)
+                 : "r"(smem_u32(b)), "r"(parity)
+                 : "memory");
+    if (ok) return true;
+    if (*abort_flag || clock64() - t0 > kUWaitCycles) return false;
   }
 }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// Shared-memory operand descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFF) >> 4);  // start address / 16
+  d |= (uint64_t)1 << 16;                   // leading byte offset (unused with swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;         // stride byte offset / 16
+  d |= (uint64_t)1 << 46;                   // descriptor version
+  d |= (uint64_t)2 << 61;                   // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: fp16 x fp16 -> fp32, both operands K-major, M 128, N 128.
+constexpr uint32_t kUmmaIdesc = (1u << 4) | ((uint32_t)(kPfTileB >> 3) << 17) | ((uint32_t)(kPfTileM >> 4) << 24);
+
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t acc) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+      "l"(a), "l"(b), "r"(kUmmaIdesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Byte offset of element (row, k) in a swizzled [128][64] fp16 tile (k a multiple of 4 here).
+__device__ __forceinline__ uint32_t swz128(int row, int k) {
+  return (uint32_t)(row * 128 + ((((k >> 3) ^ (row & 7)) << 4) | ((k & 7) << 1)));
+}
+
+// What a work item is: which tile of token rows, which 128 weight rows of which expert.
+struct UItem {
+  const slicemoe_expert* ex;
+  int row0, nt, K;
+  bool prec;     // both slices (else the MSB slice alone)
+  bool missing;  // both slices were asked for but the LSB planes are absent
+};
+template <int PHASE>
+__device__ __forceinline__ int u_item_count(const PfGemmParams& p) {
+  return PHASE == 1 ? p.ntiles[2] : p.ntiles[0] * (p.hidden / 128);
+}
+template <int PHASE>
+__device__ __forceinline__ UItem u_item(const PfGemmParams& p, int item) {
+  int tile, nt;
+  if (PHASE == 1) {
+    int lo = 0, hi = p.ntiles[0];  // last tile whose first item is <= item
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (p.item_start[mid] <= item) lo = mid; else hi = mid;
+    }
+    tile = lo;
+    nt = item - p.item_start[lo];
+  } else {
+    const int per = p.hidden / 128;
+    tile = item / per;
+    nt = item - tile * per;
+  }
+  UItem it;
+  const int e = p.tile_expert[tile];
+  const bool is_shared = e >= p.E;
+  it.ex = is_shared ? p.shared + (e - p.E) : p.experts + e;
+  it.row0 = p.tile_row0[tile];
+  it.nt = nt;
+  it.K = PHASE == 1 ? p.hidden : (is_shared ? p.shared_inter : p.inter);
+  it.prec = is_shared ? true : (p.expert_prec[e] != 0);
+  const bool has_lsb = PHASE == 1 ? (it.ex->gate.lsb && it.ex->up.lsb) : (it.ex->down.lsb != nullptr);
+  it.missing = it.prec && !has_lsb;
+  if (it.missing) it.prec = false;
+  return it;
+}
+// Weight row block (16 rows) that row block rbk (0..7) of an item's B tile holds.  Phase 1 interleaves gate and
+// up so that each half of the accumulator columns holds 32 gate columns of h and the matching 32 up columns:
+// B rows [0,32) gate, [32,64) up, [64,96) gate, [96,128) up.
+template <int PHASE>
+__device__ __forceinline__ const slicemoe_mat& u_block_mat(const UItem& it, int rbk, int* rb) {
+  if (PHASE == 1) {
+    const int half = rbk >> 2, sub = rbk & 3;
+    *rb = it.nt * 4 + 2 * half + (sub & 1);
+    return sub < 2 ? it.ex->gate : it.ex->up;
+  }
+  *rb = it.nt * 8 + rbk;
+  return it.ex->down;
+}
+
+template <int G, int PHASE>
+__global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParams p, const __grid_constant__ CUtensorMap tm_a) {
+  constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
+  constexpr int kStepsPerGroup = G / 16;  // k16 MMA steps per quantisation group
+  extern __shared__ uint8_t u_smem_raw[];
+  uint8_t* smem = u_smem_raw + ((1024 - (smem_u32(u_smem_raw) & 1023)) & 1023);
+  float(*sc_ring)[kPfTileB] = reinterpret_cast<float(*)[kPfTileB]>(smem + kUStages * kUStageBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kUStages * kUStageBytes + kUScaleBytes);
+  uint64_t* full = bars;                    // [stage]: A landed (TMA) and B written (8 warps)
+  uint64_t* empty = bars + kUStages;        // [stage]: the MMAs that read the stage have completed
+  uint64_t* acc_full = bars + 2 * kUStages;       // [2]: a group's sums are complete in the accumulator
+  uint64_t* acc_empty = bars + 2 * kUStages + 2;  // [2]: the epilogue warps have read it
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kUStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    for (int s = 0; s < kUStages; ++s) {
+      mbar_init(&full[s], 9);
+      mbar_init(&empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&acc_full[a], 1);
+      mbar_init(&acc_empty[a], 8);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 17) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kUTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const int n_items = u_item_count<PHASE>(p);
+  bool alive = true;
+
+  if (warp == 16) {
+    // ---- A tiles: one TMA copy per step ----
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+        const UItem w = u_item<PHASE>(p, item);
+        const int nk = w.K / kPfChunkK;
+        for (int kc = 0; kc < nk; ++kc, ++it) {
+          const int s = it % kUStages;
+          if (!mbar_wait(&empty[s], ((it / kUStages) & 1) ^ 1, abort_flag)) { alive = false; break; }
+          mbar_expect_tx(&full[s], kUTileBytes);
+          asm volatile(
+              "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+                  smem_u32(smem + s * kUStageBytes)),
+              "l"(&tm_a), "r"(smem_u32(&full[s])), "r"(kc * kPfChunkK), "r"(w.row0)
+              : "memory");
+        }
+      }
+    }
+  } else if (warp == 17) {
+    // ---- MMA issue ----
+    if (lane == 0) {
+      uint32_t it = 0, gc = 0;  // steps and quantisation groups issued so far
+      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+        const UItem w = u_item<PHASE>(p, item);
+        const int nk = w.K / kPfChunkK;
+        int step = 0;
+        for (int kc = 0; kc < nk && alive; ++kc, ++it) {
+          const int s = it % kUStages;
+          if (!mbar_wait(&full[s], (it / kUStages) & 1, abort_flag)) { alive = false; break; }
+          tc_fence_after();
+          const uint64_t ad = umma_desc(smem_u32(smem + s * kUStageBytes));
+          const uint64_t bd = umma_desc(smem_u32(smem + s * kUStageBytes + kUTileBytes));
+#pragma unroll
+          for (int ks = 0; ks < kPfChunkK / 16; ++ks, ++step) {
+            const int in_group = step % kStepsPerGroup;
+            const uint32_t ab = gc & 1;
+            if (in_group == 0) {
+              // first step of a group: the accumulator must have been read out
+              if (!mbar_wait(&acc_empty[ab], ((gc >> 1) & 1) ^ 1, abort_flag)) { alive = false; break; }
+              tc_fence_after();
+            }
+            umma_f16(tmem + ab * kPfTileB, ad + 2 * ks, bd + 2 * ks, in_group ? 1u : 0u);
+            if (in_group == kStepsPerGroup - 1) {
+              umma_commit(&acc_full[ab]);
+              ++gc;
+            }
+          }
+          umma_commit(&empty[s]);
+        }
+      }
+      // the last commit must have arrived before shared memory goes away
+      if (alive && it > 0) {
+        const uint32_t last = it - 1;
+        if (!mbar_wait(&empty[last % kUStages], (last / kUStages) & 1, abort_flag)) alive = false;
+      }
+    }
+  } else if (warp >= 8) {
+    // ---- dequantisation: warp d fills B rows [16 d, 16 d + 16) of every step ----
+    const int d = warp - 8, g = lane >> 2, c = lane & 3;
+    uint32_t it = 0, gc = 0;  // steps and quantisation groups produced so far
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+      const UItem w = u_item<PHASE>(p, item);
+      int rb;
+      const slicemoe_mat& m = u_block_mat<PHASE>(w, d, &rb);
+      if (w.missing && d == 0 && lane == 0) atomicOr(p.status, (unsigned)SLICEMOE_STATUS_MISSING_LSB);
+      const int nk = w.K / kPfChunkK;
+      const uint4* mp = reinterpret_cast<const uint4*>(m.msb) + (size_t)rb * nk * 32 + lane;
+      const uint4* lp = w.prec ? reinterpret_cast<const uint4*>(m.lsb) + (size_t)rb * nk * 32 + lane : mp;
+      const uint8_t* zp = m.zp + (size_t)rb * (w.K >> LG) * 16 + g;
+      const uint16_t* sc = m.scale + (size_t)rb * (w.K >> LG) * 16 + (lane & 15);
+      uint4 mw = __ldg(mp), lw = w.prec ? __ldg(lp) : make_uint4(0, 0, 0, 0);
+      __half2 off[2];
+      for (int kc = 0; kc < nk; ++kc, ++it) {
+        uint4 mw_n = mw, lw_n = lw;
+        if (kc + 1 < nk) {
+          mw_n = __ldg(mp + (size_t)(kc + 1) * 32);
+          if (w.prec) lw_n = __ldg(lp + (size_t)(kc + 1) * 32);
+        }
+        if (kc + 12 < nk && (lane & 7) == 0) {
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(mp + (size_t)(kc + 12) * 32));
+          if (w.prec) asm volatile("prefetch.global.L2 [%0];" ::"l"(lp + (size_t)(kc + 12) * 32));
+        }
+        const int s = it % kUStages;
+        uint8_t* bs = smem + s * kUStageBytes + kUTileBytes;
+        if (!__all_sync(0xffffffffu, mbar_wait(&empty[s], ((it / kUStages) & 1) ^ 1, abort_flag))) { alive = false; break; }
+        const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w}, lws[4] = {lw.x, lw.y, lw.z, lw.w};
+#pragma unroll
+        for (int wd = 0; wd < 4; ++wd) {
+          const int k = 16 * wd + 4 * c;
+          if (G >= 64 ? (wd == 0 && ((kc * kPfChunkK) & (G - 1)) == 0) : ((wd & 1) == 0)) {
+            // a new quantisation group starts: zero-points of rows g and g + 8
+            const int grp = (kc * kPfChunkK + 16 * wd) >> LG;
+#pragma unroll
+            for (int hi = 0; hi < 2; ++hi) {
+              const int z = __ldg(zp + grp * 16 + 8 * hi);
+              off[hi] = __half2half2(__int2half_rn(1024 + (w.prec ? z : (z & 0xf0))));
+            }
+            // the group's scales of the warp's 16 rows, for the epilogue (published by the arrive below)
+            if (lane < 16) sc_ring[gc % kUScaleSlots][16 * d + lane] = __half2float(__ushort_as_half(__ldg(sc + grp * 16)));
+            ++gc;
+          }
+          const uint32_t m0 = mws[wd], l0 = lws[wd];
+          // both slices: the 8-bit code; MSB slice alone: 16 x its 4-bit code (the factor 16 of the low-bit
+          // dequantisation, exact in fp16)
+          const uint32_t qlo = ((m0 & 0x0f0f0f0fu) << 4) | (l0 & 0x0f0f0f0fu);
+          const uint32_t qhi = (m0 & 0xf0f0f0f0u) | ((l0 >> 4) & 0x0f0f0f0fu);
+#pragma unroll
+          for (int hi = 0; hi < 2; ++hi) {
+            const uint32_t q = hi ? qhi : qlo;
+            // bytes -> fp16 1024 + code, minus (1024 + zero-point): the integer q - zp (or 16 (q_msb - (zp >> 4))), exact
+            uint32_t h01 = __byte_perm(q, 0x64646464u, 0x4140), h23 = __byte_perm(q, 0x64646464u, 0x4342);
+            const __half2 w01 = __hsub2(*reinterpret_cast<__half2*>(&h01), off[hi]);
+            const __half2 w23 = __hsub2(*reinterpret_cast<__half2*>(&h23), off[hi]);
+            uint2 o;
+            o.x = *reinterpret_cast<const uint32_t*>(&w01);
+            o.y = *reinterpret_cast<const uint32_t*>(&w23);
+            *reinterpret_cast<uint2*>(bs + swz128(16 * d + g + 8 * hi, k)) = o;
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full[s]);
+        mw = mw_n;
+        lw = lw_n;
+      }
+    }
+  } else {
+    // ---- epilogue: warp (q, hh) owns accumulator lanes [32 q, 32 q + 32) x columns [64 hh, 64 hh + 64) ----
+    const int q = warp & 3, hh = warp >> 2;
+    uint32_t gc = 0;
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+      const UItem w = u_item<PHASE>(p, item);
+      const int ngroups = w.K >> LG;
+      float tot[64];
+#pragma unroll
+      for (int j = 0; j < 64; ++j) tot[j] = 0.f;
+      for (int grp = 0; grp < ngroups; ++grp, ++gc) {
+        const uint32_t ab = gc & 1;
+        if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[ab], (gc >> 1) & 1, abort_flag))) { alive = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t r[16];
+          tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + ab * kPfTileB + 64 * hh + 16 * cc, r);
+          const float4* sp = reinterpret_cast<const float4*>(&sc_ring[gc % kUScaleSlots][64 * hh + 16 * cc]);
+          float sf[16];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) *reinterpret_cast<float4*>(&sf[4 * j]) = sp[j];
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) tot[16 * cc + j] = fmaf(sf[j], __uint_as_float(r[j]), tot[16 * cc + j]);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[ab]);
+      }
+      if (!alive) break;
+      const int row = w.row0 + 32 * q + lane;
+      if (PHASE == 1) {
+        // columns 0-31 of the warp's half are gate, 32-63 the matching up columns
+        uint32_t hv[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float g0 = tot[2 * j], g1 = tot[2 * j + 1], u0 = tot[32 + 2 * j], u1 = tot[32 + 2 * j + 1];
+          const __half2 hp = __floats2half2_rn(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1);
+          hv[j] = *reinterpret_cast<const uint32_t*>(&hp);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(p.h + (size_t)row * p.ldh + 64 * w.nt + 32 * hh);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dst[j] = make_uint4(hv[4 * j], hv[4 * j + 1], hv[4 * j + 2], hv[4 * j + 3]);
+      } else {
+        float4* dst = reinterpret_cast<float4*>(p.yrow + (size_t)row * p.hidden + 128 * w.nt + 64 * hh);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) dst[j] = make_float4(tot[4 * j], tot[4 * j + 1], tot[4 * j + 2], tot[4 * j + 3]);
+      }
+    }
+  }
+  if (!alive) {
+    *abort_flag = 1;
+    if (lane == 0) atomicOr(p.status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 17) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kUTmemCols) : "memory");
+  }
+}
 
 // ---- step 5: weighted combine in list order ---------------------------------------------------------------
 __global__ void pf_gate_kernel(const uint16_t* __restrict__ x, const float* __restrict__ gate_vec, int T, int hidden,
@@ -415,25 +550,52 @@ __global__ void pf_combine_kernel(const float* __restrict__ yrow, const int* __r
   }
 }
 
-// A and B tiles double-buffered (73,728 bytes) plus the scales of the step's groups
-constexpr int kPfSmemBytes = 2 * (int)sizeof(__half) * (kPfTileM + kPfTileB) * kPfStride + 2 * 2 * kPfTileB * (int)sizeof(float);
+typedef CUresult (*PfEncodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Tensor map of a row-major fp16 matrix [rows, cols] for 128-row x 64-column tiles with 128-byte swizzle.
+static int pf_tensor_map(CUtensorMap* tm, const __half* base, int rows, int cols) {
+  static PfEncodeTiled encode = nullptr;
+  if (!encode) {
+    cudaDriverEntryPointQueryResult q;
+    void* fn = nullptr;
+    SM_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+    if (!fn || q != cudaDriverEntryPointSuccess) return SLICEMOE_E_UNSUPPORTED;
+    encode = reinterpret_cast<PfEncodeTiled>(fn);
+  }
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * sizeof(__half)};
+  const cuuint32_t box[2] = {(cuuint32_t)kPfChunkK, (cuuint32_t)kPfTileM};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<__half*>(base), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SLICEMOE_OK : SLICEMOE_E_INVALID_ARG;
+}
 
 template <int G>
-static int pf_launch_gemms(const PfGemmParams& p, int max_tiles, int inter_max, cudaStream_t st) {
+static int pf_launch_gemms(const PfGemmParams& p, const __half* xs, int rmax, cudaStream_t st) {
   static bool attr_set[64];
+  static int sm_count[64];
   int dev = 0;
   SM_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return SLICEMOE_E_UNSUPPORTED;
   if (!attr_set[dev]) {
-    SM_CUDA_TRY(cudaFuncSetAttribute(pf_gemm_kernel<G, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes));
-    SM_CUDA_TRY(cudaFuncSetAttribute(pf_gemm_kernel<G, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes));
+    SM_CUDA_TRY(cudaFuncSetAttribute(pf_umma_kernel<G, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUSmemBytes));
+    SM_CUDA_TRY(cudaFuncSetAttribute(pf_umma_kernel<G, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUSmemBytes));
+    SM_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
     attr_set[dev] = true;
   }
-  pf_gemm_kernel<G, 1><<<dim3(max_tiles, inter_max / 64), kPfThreads, kPfSmemBytes, st>>>(p);
+  CUtensorMap tm_x, tm_h;
+  int rc = pf_tensor_map(&tm_x, xs, rmax, p.hidden);
+  if (rc != SLICEMOE_OK) return rc;
+  rc = pf_tensor_map(&tm_h, p.h, rmax, p.ldh);
+  if (rc != SLICEMOE_OK) return rc;
+  // one persistent CTA per SM (shared memory admits one); each walks its share of the work items
+  pf_umma_kernel<G, 1><<<sm_count[dev], kUThreads, kUSmemBytes, st>>>(p, tm_x);
   SM_LAUNCH_CHECK();
-  PfGemmParams p2 = p;  // the second GEMM contracts h
-  p2.a = p.h;
-  pf_gemm_kernel<G, 2><<<dim3(max_tiles, p.hidden / 128), kPfThreads, kPfSmemBytes, st>>>(p2);
+  pf_umma_kernel<G, 2><<<sm_count[dev], kUThreads, kUSmemBytes, st>>>(p, tm_h);
   SM_LAUNCH_CHECK();
   return SLICEMOE_OK;
 }
@@ -482,6 +644,7 @@ extern "C" int slicemoe_prefill_layer(const slicemoe_shape* s, const slicemoe_ex
   int* offsets = reinterpret_cast<int*>(ws + L.offsets);
   int* tile_expert = reinterpret_cast<int*>(ws + L.tile_expert);
   int* tile_row0 = reinterpret_cast<int*>(ws + L.tile_row0);
+  int* item_start = reinterpret_cast<int*>(ws + L.item_start);
   int* ntiles = reinterpret_cast<int*>(ws + L.ntiles);
   int* row_token = reinterpret_cast<int*>(ws + L.row_token);
   int* posmap = reinterpret_cast<int*>(ws + L.posmap);
@@ -497,7 +660,7 @@ extern "C" int slicemoe_prefill_layer(const slicemoe_shape* s, const slicemoe_ex
   const int npairs = T * k;
   pf_count_kernel<<<(npairs + 255) / 256, 256, 0, st>>>(ids, npairs, E, counts, reinterpret_cast<unsigned*>(status_out_device));
   SM_LAUNCH_CHECK();
-  pf_scan_kernel<<<1, 32, 0, st>>>(counts, E, nsh, T, offsets, tile_expert, tile_row0, ntiles);
+  pf_scan_kernel<<<1, 32, 0, st>>>(counts, E, nsh, T, s->inter, shared_inter, offsets, tile_expert, tile_row0, item_start, ntiles);
   SM_LAUNCH_CHECK();
   const int nslots = T * (k + nsh);
   pf_scatter_kernel<<<(nslots + 255) / 256, 256, 0, st>>>(ids, T, k, E, nsh, offsets, cursor, row_token, posmap);
@@ -515,8 +678,8 @@ extern "C" int slicemoe_prefill_layer(const slicemoe_shape* s, const slicemoe_ex
   p.expert_prec = expert_prec;
   p.tile_expert = tile_expert;
   p.tile_row0 = tile_row0;
+  p.item_start = item_start;
   p.ntiles = ntiles;
-  p.a = xs;
   p.h = h;
   p.yrow = yrow;
   p.status = reinterpret_cast<unsigned*>(status_out_device);
@@ -525,13 +688,12 @@ extern "C" int slicemoe_prefill_layer(const slicemoe_shape* s, const slicemoe_ex
   p.inter = s->inter;
   p.shared_inter = shared_inter;
   p.ldh = s->inter > shared_inter ? s->inter : shared_inter;
-  const int inter_max = p.ldh;
   if (s->group == 128) {
-    rc = pf_launch_gemms<128>(p, L.max_tiles, inter_max, st);
+    rc = pf_launch_gemms<128>(p, xs, L.rmax, st);
   } else if (s->group == 64) {
-    rc = pf_launch_gemms<64>(p, L.max_tiles, inter_max, st);
+    rc = pf_launch_gemms<64>(p, xs, L.rmax, st);
   } else {
-    rc = pf_launch_gemms<32>(p, L.max_tiles, inter_max, st);
+    rc = pf_launch_gemms<32>(p, xs, L.rmax, st);
   }
   if (rc != SLICEMOE_OK) return rc;
   pf_combine_kernel<<<T, 256, 0, st>>>(yrow, posmap, weights, gated ? gate : nullptr, T, k, nsh, s->hidden, y);
