@@ -133,26 +133,32 @@ __global__ void pf_gather_kernel(const uint16_t* __restrict__ x, int hidden, con
 }
 
 // ---- steps 3 and 4: the grouped GEMM on the 5th-generation tensor cores ---------------------------------
-// One persistent CTA per SM walks work items (128 token rows x 128 weight rows).  Per 64-column step of the
-// contraction:
-//   - the load warp brings the A tile (token rows of x or h, fp16) in with one TMA tiled copy, 128-byte swizzle;
-//   - eight dequantisation warps (one per 16-row block of the weight tile) read the nibble planes and the
-//     zero-points and write the INTEGER q - zp (or q_msb - (zp >> 4)), which fp16 holds exactly, into the B tile
-//     in the same swizzled K-major layout;
+// One persistent CTA per SM walks work items (128 weight rows x 128 token rows) and computes the transposed
+// product D[weight row, token].  Per 64-column step of the contraction:
+//   - the load warp brings the token tile (rows of x or h, fp16) into shared memory with one TMA tiled copy,
+//     128-byte swizzle: the B operand;
+//   - eight dequantisation warps turn the nibble planes and zero-points into the INTEGER q - zp (or
+//     16 (q_msb - (zp >> 4))), which fp16 holds exactly, and store it straight into tensor memory with
+//     tcgen05.st: the A operand, one weight row per lane.  Weights never pass through shared memory as fp16;
 //   - one thread issues four tcgen05.mma (M 128, N 128, K 16) that accumulate in tensor memory.
 // At the end of every quantisation group the accumulator (one of two, 128 columns each) is handed to eight
-// epilogue warps, which read it with tcgen05.ld, scale column n by the group's fp16 scale of weight row n in
-// fp32 and add it to the running result in registers; meanwhile the next group accumulates in the other
+// epilogue warps, which read it with tcgen05.ld, scale it by the group's fp16 scale of the lane's weight row
+// in fp32 and add it to the running result in registers; meanwhile the next group accumulates in the other
 // buffer.  No weight is ever rounded.  Every wait is bounded; a wait that runs out sets
 // SLICEMOE_STATUS_WAIT_TIMEOUT and the CTA winds down (tensor memory is freed on every path).
 constexpr int kUThreads = 576;      // warps 0-7 epilogue, 8-15 dequantisation, 16 loads, 17 MMA issue
 constexpr int kUStages = 6;
-constexpr int kUTileBytes = kPfTileM * kPfChunkK * 2;  // 16,384: one operand tile of a step
-constexpr int kUStageBytes = 2 * kUTileBytes;
+constexpr int kUTileBytes = kPfTileM * kPfChunkK * 2;  // 16,384: the token tile of a step
 constexpr int kUScaleSlots = 16;    // ring of per-group scale rows: dequantisation runs at most 15 groups ahead of the epilogue
 constexpr int kUScaleBytes = kUScaleSlots * kPfTileB * 4;
-constexpr int kUSmemBytes = kUStages * kUStageBytes + kUScaleBytes + 1024 /* alignment slack */ + 256 /* barriers */;
-constexpr int kUTmemCols = 256;     // two accumulators of 128 fp32 columns
+constexpr int kURawDepth = 8;       // steps of raw plane words each dequantisation warp keeps in flight (cp.async)
+constexpr int kURawBytes = 8 * kURawDepth * 1024;  // per warp and step: 2 blocks x 256 bytes MSB, the same of LSB
+constexpr int kUXchBytes = 4 * 64 * 32 * 4;        // silu(gate) on its way from the gate warps to the up warps
+constexpr int kUSmemBytes =
+    kUStages * kUTileBytes + kURawBytes + kUXchBytes + kUScaleBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int kUAccCols = 256;      // two accumulators of 128 fp32 columns (tokens)
+constexpr int kUWCols = 32;         // a step's weights: 64 fp16 per row
+constexpr int kUTmemCols = 512;     // accumulators + kUStages weight stages, rounded up to a power of two
 constexpr long long kUWaitCycles = 2000000000ll;
 
 struct PfGemmParams {
@@ -192,6 +198,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile
     if (*abort_flag || clock64() - t0 > kUWaitCycles) return false;
   }
 }
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global.L2::128B [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_but() {  // all but the N most recent groups have landed
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -214,6 +231,21 @@ __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a, uint64_t b
       "l"(a), "l"(b), "r"(kUmmaIdesc), "r"(acc)
       : "memory");
 }
+// The same with the A operand in tensor memory (lane = row, 32-bit column = two consecutive k).
+__device__ __forceinline__ void umma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t acc) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b), "r"(kUmmaIdesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -272,33 +304,35 @@ __device__ __forceinline__ UItem u_item(const PfGemmParams& p, int item) {
   if (it.missing) it.prec = false;
   return it;
 }
-// Weight row block (16 rows) that row block rbk (0..7) of an item's B tile holds.  Phase 1 interleaves gate and
-// up so that each half of the accumulator columns holds 32 gate columns of h and the matching 32 up columns:
-// B rows [0,32) gate, [32,64) up, [64,96) gate, [96,128) up.
+// Weight row block (16 rows) that row block rbk (0..7) of an item's 128 weight rows holds.  First GEMM: rows
+// [0,64) are gate rows of h columns [64 nt, 64 nt + 64), rows [64,128) the up rows of the same columns.
 template <int PHASE>
 __device__ __forceinline__ const slicemoe_mat& u_block_mat(const UItem& it, int rbk, int* rb) {
   if (PHASE == 1) {
-    const int half = rbk >> 2, sub = rbk & 3;
-    *rb = it.nt * 4 + 2 * half + (sub & 1);
-    return sub < 2 ? it.ex->gate : it.ex->up;
+    *rb = it.nt * 4 + (rbk & 3);
+    return rbk < 4 ? it.ex->gate : it.ex->up;
   }
   *rb = it.nt * 8 + rbk;
   return it.ex->down;
 }
 
 template <int G, int PHASE>
-__global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParams p, const __grid_constant__ CUtensorMap tm_a) {
+__global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParams p, const __grid_constant__ CUtensorMap tm_tok) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
   constexpr int kStepsPerGroup = G / 16;  // k16 MMA steps per quantisation group
   extern __shared__ uint8_t u_smem_raw[];
   uint8_t* smem = u_smem_raw + ((1024 - (smem_u32(u_smem_raw) & 1023)) & 1023);
-  float(*sc_ring)[kPfTileB] = reinterpret_cast<float(*)[kPfTileB]>(smem + kUStages * kUStageBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kUStages * kUStageBytes + kUScaleBytes);
-  uint64_t* full = bars;                    // [stage]: A landed (TMA) and B written (8 warps)
+  uint8_t* raw_ring = smem + kUStages * kUTileBytes;
+  float(*xch)[64][32] = reinterpret_cast<float(*)[64][32]>(raw_ring + kURawBytes);  // [pair][token][row]
+  float(*sc_ring)[kPfTileB] = reinterpret_cast<float(*)[kPfTileB]>(raw_ring + kURawBytes + kUXchBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(raw_ring + kURawBytes + kUXchBytes + kUScaleBytes);
+  uint64_t* full = bars;                    // [stage]: tokens landed (TMA) and weights stored (8 warps)
   uint64_t* empty = bars + kUStages;        // [stage]: the MMAs that read the stage have completed
   uint64_t* acc_full = bars + 2 * kUStages;       // [2]: a group's sums are complete in the accumulator
   uint64_t* acc_empty = bars + 2 * kUStages + 2;  // [2]: the epilogue warps have read it
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kUStages + 4);
+  uint64_t* xch_full = bars + 2 * kUStages + 4;   // [4]: silu(gate) of a warp pair is in shared memory
+  uint64_t* xch_empty = bars + 2 * kUStages + 8;  // [4]: it has been consumed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kUStages + 12);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -310,6 +344,10 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
     for (int a = 0; a < 2; ++a) {
       mbar_init(&acc_full[a], 1);
       mbar_init(&acc_empty[a], 8);
+    }
+    for (int a = 0; a < 4; ++a) {
+      mbar_init(&xch_full[a], 1);
+      mbar_init(&xch_empty[a], 1);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -327,7 +365,7 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
   bool alive = true;
 
   if (warp == 16) {
-    // ---- A tiles: one TMA copy per step ----
+    // ---- token tiles: one TMA copy per step ----
     if (lane == 0) {
       uint32_t it = 0;
       for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
@@ -339,14 +377,14 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
           mbar_expect_tx(&full[s], kUTileBytes);
           asm volatile(
               "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
-                  smem_u32(smem + s * kUStageBytes)),
-              "l"(&tm_a), "r"(smem_u32(&full[s])), "r"(kc * kPfChunkK), "r"(w.row0)
+                  smem_u32(smem + s * kUTileBytes)),
+              "l"(&tm_tok), "r"(smem_u32(&full[s])), "r"(kc * kPfChunkK), "r"(w.row0)
               : "memory");
         }
       }
     }
   } else if (warp == 17) {
-    // ---- MMA issue ----
+    // ---- MMA issue: D[weight row, token] += W[weight row, k] (tensor memory) x X[token, k] (shared memory) ----
     if (lane == 0) {
       uint32_t it = 0, gc = 0;  // steps and quantisation groups issued so far
       for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
@@ -357,8 +395,8 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
           const int s = it % kUStages;
           if (!mbar_wait(&full[s], (it / kUStages) & 1, abort_flag)) { alive = false; break; }
           tc_fence_after();
-          const uint64_t ad = umma_desc(smem_u32(smem + s * kUStageBytes));
-          const uint64_t bd = umma_desc(smem_u32(smem + s * kUStageBytes + kUTileBytes));
+          const uint64_t bd = umma_desc(smem_u32(smem + s * kUTileBytes));
+          const uint32_t a_tmem = tmem + kUAccCols + s * kUWCols;
 #pragma unroll
           for (int ks = 0; ks < kPfChunkK / 16; ++ks, ++step) {
             const int in_group = step % kStepsPerGroup;
@@ -368,7 +406,7 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
               if (!mbar_wait(&acc_empty[ab], ((gc >> 1) & 1) ^ 1, abort_flag)) { alive = false; break; }
               tc_fence_after();
             }
-            umma_f16(tmem + ab * kPfTileB, ad + 2 * ks, bd + 2 * ks, in_group ? 1u : 0u);
+            umma_f16_ts(tmem + ab * kPfTileM, a_tmem + 8 * ks, bd + 2 * ks, in_group ? 1u : 0u);
             if (in_group == kStepsPerGroup - 1) {
               umma_commit(&acc_full[ab]);
               ++gc;
@@ -384,80 +422,124 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
       }
     }
   } else if (warp >= 8) {
-    // ---- dequantisation: warp d fills B rows [16 d, 16 d + 16) of every step ----
-    const int d = warp - 8, g = lane >> 2, c = lane & 3;
-    uint32_t it = 0, gc = 0;  // steps and quantisation groups produced so far
+    // ---- dequantisation: thread (q, lane) owns weight row 32 q + lane; its warp stores the row's 32 values of
+    // the step's k half `kh` into the stage's tensor-memory columns ----
+    const int q = warp & 3, kh = (warp - 8) >> 2;
+    const int blk = lane >> 4, g = lane & 7, sh = ((lane >> 3) & 1) * 4;  // row = 16 (2 q + blk) + g + 8 (sh / 4)
+    // Raw plane words run kURawDepth steps ahead of their use, across work items.  Per step the warp needs the
+    // k half of two 16-row blocks: 64 pieces of 8 bytes per plane; lane l copies pieces l of both blocks with
+    // cp.async into the warp's ring, and after a warp barrier every lane reads the four pieces of its row.
+    uint8_t* raw = raw_ring + (warp - 8) * (kURawDepth * 1024);
+    int i_item = blockIdx.x, i_kc = 0, i_nk = 0;
+    const uint8_t *i_mp = nullptr, *i_lp = nullptr;
+    bool i_prec = false;
+    auto i_open = [&]() {
+      if (i_item >= n_items) return;
+      const UItem w = u_item<PHASE>(p, i_item);
+      int rb;
+      const slicemoe_mat& m = u_block_mat<PHASE>(w, 2 * q, &rb);  // blocks 2 q and 2 q + 1 are neighbours in one matrix
+      i_nk = w.K / kPfChunkK;
+      i_prec = w.prec;
+      i_mp = reinterpret_cast<const uint8_t*>(m.msb) + (size_t)rb * i_nk * 512 + lane * 16 + 8 * kh;
+      i_lp = w.prec ? reinterpret_cast<const uint8_t*>(m.lsb) + (size_t)rb * i_nk * 512 + lane * 16 + 8 * kh : i_mp;
+    };
+    auto i_issue = [&](int slot) {
+      if (i_item < n_items) {
+        uint8_t* dst = raw + slot * 1024 + lane * 8;
+        const size_t o = (size_t)i_kc * 512, o1 = o + (size_t)i_nk * 512;
+        cp_async8(dst, i_mp + o);
+        cp_async8(dst + 256, i_mp + o1);
+        if (i_prec) {
+          cp_async8(dst + 512, i_lp + o);
+          cp_async8(dst + 768, i_lp + o1);
+        }
+        if (++i_kc == i_nk) {
+          i_item += gridDim.x;
+          i_kc = 0;
+          i_open();
+        }
+      }
+      cp_async_commit();
+    };
+    i_open();
+    for (int j = 0; j < kURawDepth; ++j) i_issue(j);
+    uint32_t it = 0;  // steps produced so far
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
       const UItem w = u_item<PHASE>(p, item);
       int rb;
-      const slicemoe_mat& m = u_block_mat<PHASE>(w, d, &rb);
-      if (w.missing && d == 0 && lane == 0) atomicOr(p.status, (unsigned)SLICEMOE_STATUS_MISSING_LSB);
-      const int nk = w.K / kPfChunkK;
-      const uint4* mp = reinterpret_cast<const uint4*>(m.msb) + (size_t)rb * nk * 32 + lane;
-      const uint4* lp = w.prec ? reinterpret_cast<const uint4*>(m.lsb) + (size_t)rb * nk * 32 + lane : mp;
-      const uint8_t* zp = m.zp + (size_t)rb * (w.K >> LG) * 16 + g;
-      const uint16_t* sc = m.scale + (size_t)rb * (w.K >> LG) * 16 + (lane & 15);
-      uint4 mw = __ldg(mp), lw = w.prec ? __ldg(lp) : make_uint4(0, 0, 0, 0);
-      __half2 off[2];
+      const slicemoe_mat& m = u_block_mat<PHASE>(w, 2 * q + blk, &rb);
+      if (w.missing && warp == 8 && lane == 0) atomicOr(p.status, (unsigned)SLICEMOE_STATUS_MISSING_LSB);
+      const int nk = w.K / kPfChunkK, ngroups = w.K >> LG;
+      const size_t meta = (size_t)rb * ngroups * 16 + g + 2 * sh;  // the row's entry of group 0
+      const uint8_t* zp = m.zp + meta;
+      const uint16_t* sc = m.scale + meta;
+      __half2 off = __half2half2(__float2half_rn(0.f));
+      // zero-point and scale of the thread's next group (its first: group kh when a group is 32 columns)
+      int z_next = __ldg(zp + (G == 32 ? kh * 16 : 0));
+      uint16_t s_next = __ldg(sc + (G == 32 ? kh * 16 : 0));
       for (int kc = 0; kc < nk; ++kc, ++it) {
-        uint4 mw_n = mw, lw_n = lw;
-        if (kc + 1 < nk) {
-          mw_n = __ldg(mp + (size_t)(kc + 1) * 32);
-          if (w.prec) lw_n = __ldg(lp + (size_t)(kc + 1) * 32);
+        // The thread's 32 columns of a step lie in one quantisation group: group (item-local) `grp`, and
+        // `gidx` counted over all groups this CTA has met (K is a multiple of 128, so steps and groups align).
+        const bool new_group = G == 128 ? (kc & 1) == 0 : true;
+        const int grp = (kc * kPfChunkK + 32 * kh) >> LG;
+        const uint32_t gidx = G == 128 ? (it >> 1) : (G == 64 ? it : 2 * it + kh);
+        const int slot = it % kURawDepth;
+        cp_async_wait_but<kURawDepth - 1>();
+        __syncwarp();
+        const uint8_t* src = raw + slot * 1024 + blk * 256 + g * 32;
+        const uint4 m01 = *reinterpret_cast<const uint4*>(src), m23 = *reinterpret_cast<const uint4*>(src + 16);
+        uint4 l01 = make_uint4(0, 0, 0, 0), l23 = l01;
+        if (w.prec) {
+          l01 = *reinterpret_cast<const uint4*>(src + 512);
+          l23 = *reinterpret_cast<const uint4*>(src + 528);
         }
-        if (kc + 12 < nk && (lane & 7) == 0) {
-          asm volatile("prefetch.global.L2 [%0];" ::"l"(mp + (size_t)(kc + 12) * 32));
-          if (w.prec) asm volatile("prefetch.global.L2 [%0];" ::"l"(lp + (size_t)(kc + 12) * 32));
-        }
+        // piece c (8 bytes) = words (w = 2 kh, 2 kh + 1) of plane lane 4 g + c: k = 16 w + 4 c + j
+        const uint32_t mws[8] = {m01.x, m01.y, m01.z, m01.w, m23.x, m23.y, m23.z, m23.w};
+        const uint32_t lws[8] = {l01.x, l01.y, l01.z, l01.w, l23.x, l23.y, l23.z, l23.w};
         const int s = it % kUStages;
-        uint8_t* bs = smem + s * kUStageBytes + kUTileBytes;
         if (!__all_sync(0xffffffffu, mbar_wait(&empty[s], ((it / kUStages) & 1) ^ 1, abort_flag))) { alive = false; break; }
-        const uint32_t mws[4] = {mw.x, mw.y, mw.z, mw.w}, lws[4] = {lw.x, lw.y, lw.z, lw.w};
-#pragma unroll
-        for (int wd = 0; wd < 4; ++wd) {
-          const int k = 16 * wd + 4 * c;
-          if (G >= 64 ? (wd == 0 && ((kc * kPfChunkK) & (G - 1)) == 0) : ((wd & 1) == 0)) {
-            // a new quantisation group starts: zero-points of rows g and g + 8
-            const int grp = (kc * kPfChunkK + 16 * wd) >> LG;
-#pragma unroll
-            for (int hi = 0; hi < 2; ++hi) {
-              const int z = __ldg(zp + grp * 16 + 8 * hi);
-              off[hi] = __half2half2(__int2half_rn(1024 + (w.prec ? z : (z & 0xf0))));
-            }
-            // the group's scales of the warp's 16 rows, for the epilogue (published by the arrive below)
-            if (lane < 16) sc_ring[gc % kUScaleSlots][16 * d + lane] = __half2float(__ushort_as_half(__ldg(sc + grp * 16)));
-            ++gc;
-          }
-          const uint32_t m0 = mws[wd], l0 = lws[wd];
-          // both slices: the 8-bit code; MSB slice alone: 16 x its 4-bit code (the factor 16 of the low-bit
-          // dequantisation, exact in fp16)
-          const uint32_t qlo = ((m0 & 0x0f0f0f0fu) << 4) | (l0 & 0x0f0f0f0fu);
-          const uint32_t qhi = (m0 & 0xf0f0f0f0u) | ((l0 >> 4) & 0x0f0f0f0fu);
-#pragma unroll
-          for (int hi = 0; hi < 2; ++hi) {
-            const uint32_t q = hi ? qhi : qlo;
-            // bytes -> fp16 1024 + code, minus (1024 + zero-point): the integer q - zp (or 16 (q_msb - (zp >> 4))), exact
-            uint32_t h01 = __byte_perm(q, 0x64646464u, 0x4140), h23 = __byte_perm(q, 0x64646464u, 0x4342);
-            const __half2 w01 = __hsub2(*reinterpret_cast<__half2*>(&h01), off[hi]);
-            const __half2 w23 = __hsub2(*reinterpret_cast<__half2*>(&h23), off[hi]);
-            uint2 o;
-            o.x = *reinterpret_cast<const uint32_t*>(&w01);
-            o.y = *reinterpret_cast<const uint32_t*>(&w23);
-            *reinterpret_cast<uint2*>(bs + swz128(16 * d + g + 8 * hi, k)) = o;
+        tc_fence_after();
+        if (new_group) {
+          off = __half2half2(__int2half_rn(1024 + (w.prec ? z_next : (z_next & 0xf0))));
+          // the row's scale of the group, for the epilogue (published by the arrive below)
+          if (G == 32 || kh == 0) sc_ring[gidx % kUScaleSlots][32 * q + lane] = __half2float(__ushort_as_half(s_next));
+          const int nxt = G == 32 ? grp + 2 : grp + 1;
+          if (nxt < ngroups) {
+            z_next = __ldg(zp + nxt * 16);
+            s_next = __ldg(sc + nxt * 16);
           }
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA
+        uint32_t r[16];  // column 8 wl + 2 c + jj holds k = 32 kh + 16 wl + 4 c + 2 jj, + 1
+#pragma unroll
+        for (int wl = 0; wl < 2; ++wl) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint32_t m0 = mws[2 * c + wl] >> sh, l0 = lws[2 * c + wl] >> sh;
+            // both slices: the 8-bit code; MSB slice alone: 16 x its 4-bit code (the factor 16 of the low-bit
+            // dequantisation, exact in fp16)
+            const uint32_t qv = ((m0 & 0x0f0f0f0fu) << 4) | (l0 & 0x0f0f0f0fu);
+            // bytes -> fp16 1024 + code, minus (1024 + zero-point): the integer q - zp, exact
+            uint32_t h01 = __byte_perm(qv, 0x64646464u, 0x4140), h23 = __byte_perm(qv, 0x64646464u, 0x4342);
+            const __half2 w01 = __hsub2(*reinterpret_cast<__half2*>(&h01), off);
+            const __half2 w23 = __hsub2(*reinterpret_cast<__half2*>(&h23), off);
+            r[8 * wl + 2 * c] = *reinterpret_cast<const uint32_t*>(&w01);
+            r[8 * wl + 2 * c + 1] = *reinterpret_cast<const uint32_t*>(&w23);
+          }
+        }
+        tmem_st16(tmem + ((uint32_t)(32 * q) << 16) + kUAccCols + s * kUWCols + 16 * kh, r);
+        tmem_st_wait();
+        tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&full[s]);
-        mw = mw_n;
-        lw = lw_n;
+        i_issue(slot);  // after the step's words were consumed by every lane: the slot is free
       }
     }
+    cp_async_wait_but<0>();
   } else {
-    // ---- epilogue: warp (q, hh) owns accumulator lanes [32 q, 32 q + 32) x columns [64 hh, 64 hh + 64) ----
+    // ---- epilogue: warp (q, hh) owns weight rows [32 q, 32 q + 32) x tokens [64 hh, 64 hh + 64) ----
     const int q = warp & 3, hh = warp >> 2;
-    uint32_t gc = 0;
-    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+    uint32_t gc = 0, n_done = 0;
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++n_done) {
       const UItem w = u_item<PHASE>(p, item);
       const int ngroups = w.K >> LG;
       float tot[64];
@@ -467,40 +549,43 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
         const uint32_t ab = gc & 1;
         if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[ab], (gc >> 1) & 1, abort_flag))) { alive = false; break; }
         tc_fence_after();
+        const float sf = sc_ring[gc % kUScaleSlots][32 * q + lane];
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) {
           uint32_t r[16];
-          tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + ab * kPfTileB + 64 * hh + 16 * cc, r);
-          const float4* sp = reinterpret_cast<const float4*>(&sc_ring[gc % kUScaleSlots][64 * hh + 16 * cc]);
-          float sf[16];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) *reinterpret_cast<float4*>(&sf[4 * j]) = sp[j];
+          tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + ab * kPfTileM + 64 * hh + 16 * cc, r);
           tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 16; ++j) tot[16 * cc + j] = fmaf(sf[j], __uint_as_float(r[j]), tot[16 * cc + j]);
+          for (int j = 0; j < 16; ++j) tot[16 * cc + j] = fmaf(sf, __uint_as_float(r[j]), tot[16 * cc + j]);
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[ab]);
       }
       if (!alive) break;
-      const int row = w.row0 + 32 * q + lane;
+      const int tok0 = w.row0 + 64 * hh;
       if (PHASE == 1) {
-        // columns 0-31 of the warp's half are gate, 32-63 the matching up columns
-        uint32_t hv[16];
+        // rows [0,64) hold gate, rows [64,128) up: warp (q, hh) with q < 2 hands silu(gate) to warp (q + 2, hh)
+        // through shared memory; that warp multiplies and writes h
+        const int pair = 2 * hh + (q & 1);
+        if (q < 2) {
+          if (!__all_sync(0xffffffffu, mbar_wait(&xch_empty[pair], (n_done & 1) ^ 1, abort_flag))) { alive = false; break; }
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float g0 = tot[2 * j], g1 = tot[2 * j + 1], u0 = tot[32 + 2 * j], u1 = tot[32 + 2 * j + 1];
-          const __half2 hp = __floats2half2_rn(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1);
-          hv[j] = *reinterpret_cast<const uint32_t*>(&hp);
+          for (int j = 0; j < 64; ++j) xch[pair][j][lane] = tot[j] / (1.f + __expf(-tot[j]));
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&xch_full[pair]);
+        } else {
+          if (!__all_sync(0xffffffffu, mbar_wait(&xch_full[pair], n_done & 1, abort_flag))) { alive = false; break; }
+          __half* dst = p.h + (size_t)tok0 * p.ldh + 64 * w.nt + 32 * (q & 1) + lane;
+#pragma unroll
+          for (int j = 0; j < 64; ++j) dst[(size_t)j * p.ldh] = __float2half_rn(xch[pair][j][lane] * tot[j]);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&xch_empty[pair]);
         }
-        uint4* dst = reinterpret_cast<uint4*>(p.h + (size_t)row * p.ldh + 64 * w.nt + 32 * hh);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) dst[j] = make_uint4(hv[4 * j], hv[4 * j + 1], hv[4 * j + 2], hv[4 * j + 3]);
       } else {
-        float4* dst = reinterpret_cast<float4*>(p.yrow + (size_t)row * p.hidden + 128 * w.nt + 64 * hh);
+        float* dst = p.yrow + (size_t)tok0 * p.hidden + 128 * w.nt + 32 * q + lane;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) dst[j] = make_float4(tot[4 * j], tot[4 * j + 1], tot[4 * j + 2], tot[4 * j + 3]);
+        for (int j = 0; j < 64; ++j) dst[(size_t)j * p.hidden] = tot[j];
       }
     }
   }
