@@ -151,8 +151,8 @@ constexpr int kUStages = 6;
 constexpr int kUTileBytes = kPfTileM * kPfChunkK * 2;  // 16,384: the token tile of a step
 constexpr int kUScaleSlots = 16;    // ring of per-group scale rows: dequantisation runs at most 15 groups ahead of the epilogue
 constexpr int kUScaleBytes = kUScaleSlots * kPfTileB * 4;
-constexpr int kURawDepth = 8;       // steps of raw plane words each dequantisation warp keeps in flight (cp.async)
-constexpr int kURawBytes = 8 * kURawDepth * 1024;  // per warp and step: 2 blocks x 256 bytes MSB, the same of LSB
+constexpr int kURawDepth = 4;       // steps of raw plane words each dequantisation warp keeps in flight (cp.async)
+constexpr int kURawBytes = 8 * kURawDepth * 2048;  // per warp and step: 2 blocks x 512 bytes MSB, the same of LSB
 constexpr int kUXchBytes = 4 * 64 * 32 * 4;        // silu(gate) on its way from the gate warps to the up warps
 constexpr int kUSmemBytes =
     kUStages * kUTileBytes + kURawBytes + kUXchBytes + kUScaleBytes + 1024 /* alignment slack */ + 256 /* barriers */;
@@ -186,17 +186,24 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
 }
 // Bounded wait for the phase of the given parity; false when the limit ran out or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+               : "=r"(ok)
+               : "r"(smem_u32(b)), "r"(parity)
+               : "memory");
+  return ok != 0;
+}
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
   const long long t0 = clock64();
   for (;;) {
-    uint32_t ok;
-    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                 : "=r"(ok)
-                 : "r"(smem_u32(b)), "r"(parity)
-                 : "memory");
-    if (ok) return true;
+    if (mbar_try(b, parity)) return true;
     if (*abort_flag || clock64() - t0 > kUWaitCycles) return false;
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(b, parity)) return true;  // the common case costs one instruction
+  return mbar_wait_slow(b, parity, abort_flag);
 }
 __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global.L2::128B [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
@@ -243,6 +250,17 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
       "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
       "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(
+          taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
+      "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]),
+      "r"(r[31])
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -319,7 +337,6 @@ __device__ __forceinline__ const slicemoe_mat& u_block_mat(const UItem& it, int 
 template <int G, int PHASE>
 __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParams p, const __grid_constant__ CUtensorMap tm_tok) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
-  constexpr int kStepsPerGroup = G / 16;  // k16 MMA steps per quantisation group
   extern __shared__ uint8_t u_smem_raw[];
   uint8_t* smem = u_smem_raw + ((1024 - (smem_u32(u_smem_raw) & 1023)) & 1023);
   uint8_t* raw_ring = smem + kUStages * kUTileBytes;
@@ -338,7 +355,7 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     for (int s = 0; s < kUStages; ++s) {
-      mbar_init(&full[s], 9);
+      mbar_init(&full[s], 5);  // the set's four dequantisation warps and the load warp
       mbar_init(&empty[s], 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -367,70 +384,77 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
   if (warp == 16) {
     // ---- token tiles: one TMA copy per step ----
     if (lane == 0) {
-      uint32_t it = 0;
+      uint32_t s = 0, ph = 0;
       for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
         const UItem w = u_item<PHASE>(p, item);
         const int nk = w.K / kPfChunkK;
-        for (int kc = 0; kc < nk; ++kc, ++it) {
-          const int s = it % kUStages;
-          if (!mbar_wait(&empty[s], ((it / kUStages) & 1) ^ 1, abort_flag)) { alive = false; break; }
+        for (int kc = 0; kc < nk; ++kc) {
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { alive = false; break; }
           mbar_expect_tx(&full[s], kUTileBytes);
           asm volatile(
               "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
                   smem_u32(smem + s * kUTileBytes)),
               "l"(&tm_tok), "r"(smem_u32(&full[s])), "r"(kc * kPfChunkK), "r"(w.row0)
               : "memory");
+          if (++s == kUStages) { s = 0; ph ^= 1; }
         }
       }
     }
   } else if (warp == 17) {
     // ---- MMA issue: D[weight row, token] += W[weight row, k] (tensor memory) x X[token, k] (shared memory) ----
     if (lane == 0) {
-      uint32_t it = 0, gc = 0;  // steps and quantisation groups issued so far
+      uint32_t st = 0, ph = 0, gc = 0;  // stage, its parity, quantisation groups issued so far
+      uint64_t* last_empty = nullptr;
+      uint32_t last_ph = 0;
+      const uint64_t bd0 = umma_desc(smem_u32(smem));
       for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
         const UItem w = u_item<PHASE>(p, item);
         const int nk = w.K / kPfChunkK;
-        int step = 0;
-        for (int kc = 0; kc < nk && alive; ++kc, ++it) {
-          const int s = it % kUStages;
-          if (!mbar_wait(&full[s], (it / kUStages) & 1, abort_flag)) { alive = false; break; }
+        for (int kc = 0; kc < nk && alive; ++kc) {
+          if (!mbar_wait(&full[st], ph, abort_flag)) { alive = false; break; }
           tc_fence_after();
-          const uint64_t bd = umma_desc(smem_u32(smem + s * kUTileBytes));
-          const uint32_t a_tmem = tmem + kUAccCols + s * kUWCols;
+          const uint64_t bd = bd0 + (uint64_t)(st * (kUTileBytes >> 4));
+          const uint32_t a_tmem = tmem + kUAccCols + st * kUWCols;
 #pragma unroll
-          for (int ks = 0; ks < kPfChunkK / 16; ++ks, ++step) {
-            const int in_group = step % kStepsPerGroup;
+          for (int ks = 0; ks < kPfChunkK / 16; ++ks) {
+            // where a quantisation group starts and ends among the four k16 steps of a 64-column step
+            const bool first = G == 128 ? (ks == 0 && (kc & 1) == 0) : (G == 64 ? ks == 0 : (ks & 1) == 0);
+            const bool last = G == 128 ? (ks == 3 && (kc & 1) == 1) : (G == 64 ? ks == 3 : (ks & 1) == 1);
             const uint32_t ab = gc & 1;
-            if (in_group == 0) {
-              // first step of a group: the accumulator must have been read out
+            if (first) {
+              // the accumulator must have been read out
               if (!mbar_wait(&acc_empty[ab], ((gc >> 1) & 1) ^ 1, abort_flag)) { alive = false; break; }
               tc_fence_after();
             }
-            umma_f16_ts(tmem + ab * kPfTileM, a_tmem + 8 * ks, bd + 2 * ks, in_group ? 1u : 0u);
-            if (in_group == kStepsPerGroup - 1) {
+            umma_f16_ts(tmem + ab * kPfTileM, a_tmem + 8 * ks, bd + 2 * ks, first ? 0u : 1u);
+            if (last) {
               umma_commit(&acc_full[ab]);
               ++gc;
             }
           }
-          umma_commit(&empty[s]);
+          umma_commit(&empty[st]);
+          last_empty = &empty[st];
+          last_ph = ph;
+          if (++st == kUStages) { st = 0; ph ^= 1; }
         }
       }
       // the last commit must have arrived before shared memory goes away
-      if (alive && it > 0) {
-        const uint32_t last = it - 1;
-        if (!mbar_wait(&empty[last % kUStages], (last / kUStages) & 1, abort_flag)) alive = false;
-      }
+      if (alive && last_empty && !mbar_wait(last_empty, last_ph, abort_flag)) alive = false;
     }
   } else if (warp >= 8) {
-    // ---- dequantisation: thread (q, lane) owns weight row 32 q + lane; its warp stores the row's 32 values of
-    // the step's k half `kh` into the stage's tensor-memory columns ----
-    const int q = warp & 3, kh = (warp - 8) >> 2;
+    // ---- dequantisation: two sets of four warps take the 64-column steps in turn (set = step parity); thread
+    // (q, lane) of a set owns weight row 32 q + lane and stores the row's 64 values of the step into the
+    // stage's tensor-memory columns ----
+    const int q = warp & 3, set = (warp - 8) >> 2;
     const int blk = lane >> 4, g = lane & 7, sh = ((lane >> 3) & 1) * 4;  // row = 16 (2 q + blk) + g + 8 (sh / 4)
-    // Raw plane words run kURawDepth steps ahead of their use, across work items.  Per step the warp needs the
-    // k half of two 16-row blocks: 64 pieces of 8 bytes per plane; lane l copies pieces l of both blocks with
-    // cp.async into the warp's ring, and after a warp barrier every lane reads the four pieces of its row.
-    uint8_t* raw = raw_ring + (warp - 8) * (kURawDepth * 1024);
-    int i_item = blockIdx.x, i_kc = 0, i_nk = 0;
+    constexpr int kGpc = G == 32 ? 2 : 1;  // quantisation groups in a step
+    // Raw plane words run kURawDepth of the warp's steps ahead of their use, across work items.  Per step the
+    // warp needs two 16-row blocks of 512 bytes per plane; lane l copies the 16 bytes of plane lane l of both
+    // blocks with cp.async into the warp's ring (16-byte pieces XOR-swizzled against bank conflicts), and
+    // after a warp barrier every lane reads the four pieces of its row.
+    uint8_t* raw = raw_ring + (warp - 8) * (kURawDepth * 2048);
+    const int wr_piece = (lane ^ (lane >> 3)) * 16;  // plane lane l = 4 g' + c: low two bits XOR (g' >> 1)
+    int i_item = blockIdx.x, i_kc = set, i_nk = 0;
     const uint8_t *i_mp = nullptr, *i_lp = nullptr;
     bool i_prec = false;
     auto i_open = [&]() {
@@ -440,22 +464,23 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
       const slicemoe_mat& m = u_block_mat<PHASE>(w, 2 * q, &rb);  // blocks 2 q and 2 q + 1 are neighbours in one matrix
       i_nk = w.K / kPfChunkK;
       i_prec = w.prec;
-      i_mp = reinterpret_cast<const uint8_t*>(m.msb) + (size_t)rb * i_nk * 512 + lane * 16 + 8 * kh;
-      i_lp = w.prec ? reinterpret_cast<const uint8_t*>(m.lsb) + (size_t)rb * i_nk * 512 + lane * 16 + 8 * kh : i_mp;
+      i_mp = reinterpret_cast<const uint8_t*>(m.msb) + (size_t)rb * i_nk * 512 + lane * 16;
+      i_lp = w.prec ? reinterpret_cast<const uint8_t*>(m.lsb) + (size_t)rb * i_nk * 512 + lane * 16 : i_mp;
     };
     auto i_issue = [&](int slot) {
       if (i_item < n_items) {
-        uint8_t* dst = raw + slot * 1024 + lane * 8;
+        uint8_t* dst = raw + slot * 2048 + wr_piece;
         const size_t o = (size_t)i_kc * 512, o1 = o + (size_t)i_nk * 512;
-        cp_async8(dst, i_mp + o);
-        cp_async8(dst + 256, i_mp + o1);
+        cp_async16(dst, i_mp + o);
+        cp_async16(dst + 512, i_mp + o1);
         if (i_prec) {
-          cp_async8(dst + 512, i_lp + o);
-          cp_async8(dst + 768, i_lp + o1);
+          cp_async16(dst + 1024, i_lp + o);
+          cp_async16(dst + 1536, i_lp + o1);
         }
-        if (++i_kc == i_nk) {
+        i_kc += 2;
+        if (i_kc >= i_nk) {
           i_item += gridDim.x;
-          i_kc = 0;
+          i_kc = set;
           i_open();
         }
       }
@@ -463,7 +488,7 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
     };
     i_open();
     for (int j = 0; j < kURawDepth; ++j) i_issue(j);
-    uint32_t it = 0;  // steps produced so far
+    uint32_t st = set, ph = 0, slot = 0, it0 = 0;  // stage and parity of the warp's next step; steps before this item
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
       const UItem w = u_item<PHASE>(p, item);
       int rb;
@@ -473,66 +498,86 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
       const size_t meta = (size_t)rb * ngroups * 16 + g + 2 * sh;  // the row's entry of group 0
       const uint8_t* zp = m.zp + meta;
       const uint16_t* sc = m.scale + meta;
-      __half2 off = __half2half2(__float2half_rn(0.f));
-      // zero-point and scale of the thread's next group (its first: group kh when a group is 32 columns)
-      int z_next = __ldg(zp + (G == 32 ? kh * 16 : 0));
-      uint16_t s_next = __ldg(sc + (G == 32 ? kh * 16 : 0));
-      for (int kc = 0; kc < nk; ++kc, ++it) {
-        // The thread's 32 columns of a step lie in one quantisation group: group (item-local) `grp`, and
-        // `gidx` counted over all groups this CTA has met (K is a multiple of 128, so steps and groups align).
-        const bool new_group = G == 128 ? (kc & 1) == 0 : true;
-        const int grp = (kc * kPfChunkK + 32 * kh) >> LG;
-        const uint32_t gidx = G == 128 ? (it >> 1) : (G == 64 ? it : 2 * it + kh);
-        const int slot = it % kURawDepth;
+      // zero-points and scales of the groups of the warp's next step
+      int z_next[kGpc];
+      uint16_t s_next[kGpc];
+#pragma unroll
+      for (int i = 0; i < kGpc; ++i) {
+        const int grp = ((set * kPfChunkK) >> LG) + i;
+        z_next[i] = __ldg(zp + grp * 16);
+        s_next[i] = __ldg(sc + grp * 16);
+      }
+      for (int kc = set; kc < nk; kc += 2) {
+        // groups of this step: item-local grp0 .. grp0 + kGpc - 1; gidx0 counts all groups this CTA has met
+        // (K is a multiple of 128, so steps and groups align)
+        const uint32_t it = it0 + kc;
+        const int grp0 = (kc * kPfChunkK) >> LG;
+        const uint32_t gidx0 = G == 128 ? (it >> 1) : (G == 64 ? it : 2 * it);
         cp_async_wait_but<kURawDepth - 1>();
         __syncwarp();
-        const uint8_t* src = raw + slot * 1024 + blk * 256 + g * 32;
-        const uint4 m01 = *reinterpret_cast<const uint4*>(src), m23 = *reinterpret_cast<const uint4*>(src + 16);
-        uint4 l01 = make_uint4(0, 0, 0, 0), l23 = l01;
-        if (w.prec) {
-          l01 = *reinterpret_cast<const uint4*>(src + 512);
-          l23 = *reinterpret_cast<const uint4*>(src + 528);
+        const uint8_t* src = raw + slot * 2048 + blk * 512 + g * 64;
+        const int rsw = (g >> 1) * 16;  // piece c sits at 16 (c ^ (g >> 1))
+        uint32_t mws[16], lws[16];      // [4 c + w]: word w of plane lane 4 g + c: k = 16 w + 4 c + j
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const uint4 mv = *reinterpret_cast<const uint4*>(src + ((16 * c) ^ rsw));
+          mws[4 * c] = mv.x; mws[4 * c + 1] = mv.y; mws[4 * c + 2] = mv.z; mws[4 * c + 3] = mv.w;
+          uint4 lv = make_uint4(0, 0, 0, 0);
+          if (w.prec) lv = *reinterpret_cast<const uint4*>(src + 1024 + ((16 * c) ^ rsw));
+          lws[4 * c] = lv.x; lws[4 * c + 1] = lv.y; lws[4 * c + 2] = lv.z; lws[4 * c + 3] = lv.w;
         }
-        // piece c (8 bytes) = words (w = 2 kh, 2 kh + 1) of plane lane 4 g + c: k = 16 w + 4 c + j
-        const uint32_t mws[8] = {m01.x, m01.y, m01.z, m01.w, m23.x, m23.y, m23.z, m23.w};
-        const uint32_t lws[8] = {l01.x, l01.y, l01.z, l01.w, l23.x, l23.y, l23.z, l23.w};
-        const int s = it % kUStages;
-        if (!__all_sync(0xffffffffu, mbar_wait(&empty[s], ((it / kUStages) & 1) ^ 1, abort_flag))) { alive = false; break; }
-        tc_fence_after();
-        if (new_group) {
-          off = __half2half2(__int2half_rn(1024 + (w.prec ? z_next : (z_next & 0xf0))));
-          // the row's scale of the group, for the epilogue (published by the arrive below)
-          if (G == 32 || kh == 0) sc_ring[gidx % kUScaleSlots][32 * q + lane] = __half2float(__ushort_as_half(s_next));
-          const int nxt = G == 32 ? grp + 2 : grp + 1;
-          if (nxt < ngroups) {
-            z_next = __ldg(zp + nxt * 16);
-            s_next = __ldg(sc + nxt * 16);
+        __half2 off[kGpc];
+        float sf[kGpc];
+#pragma unroll
+        for (int i = 0; i < kGpc; ++i) {
+          off[i] = __half2half2(__int2half_rn(1024 + (w.prec ? z_next[i] : (z_next[i] & 0xf0))));
+          sf[i] = __half2float(__ushort_as_half(s_next[i]));
+        }
+        if (kc + 2 < nk) {
+#pragma unroll
+          for (int i = 0; i < kGpc; ++i) {
+            const int grp = (((kc + 2) * kPfChunkK) >> LG) + i;
+            z_next[i] = __ldg(zp + grp * 16);
+            s_next[i] = __ldg(sc + grp * 16);
           }
         }
-        uint32_t r[16];  // column 8 wl + 2 c + jj holds k = 32 kh + 16 wl + 4 c + 2 jj, + 1
+        (void)grp0;
+        uint32_t r[32];  // column 8 w + 2 c + jj holds k = 16 w + 4 c + 2 jj, + 1
 #pragma unroll
-        for (int wl = 0; wl < 2; ++wl) {
+        for (int wd = 0; wd < 4; ++wd) {
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
-            const uint32_t m0 = mws[2 * c + wl] >> sh, l0 = lws[2 * c + wl] >> sh;
+            const uint32_t m0 = mws[4 * c + wd] >> sh, l0 = lws[4 * c + wd] >> sh;
             // both slices: the 8-bit code; MSB slice alone: 16 x its 4-bit code (the factor 16 of the low-bit
             // dequantisation, exact in fp16)
             const uint32_t qv = ((m0 & 0x0f0f0f0fu) << 4) | (l0 & 0x0f0f0f0fu);
             // bytes -> fp16 1024 + code, minus (1024 + zero-point): the integer q - zp, exact
             uint32_t h01 = __byte_perm(qv, 0x64646464u, 0x4140), h23 = __byte_perm(qv, 0x64646464u, 0x4342);
-            const __half2 w01 = __hsub2(*reinterpret_cast<__half2*>(&h01), off);
-            const __half2 w23 = __hsub2(*reinterpret_cast<__half2*>(&h23), off);
-            r[8 * wl + 2 * c] = *reinterpret_cast<const uint32_t*>(&w01);
-            r[8 * wl + 2 * c + 1] = *reinterpret_cast<const uint32_t*>(&w23);
+            const __half2 o = off[kGpc == 2 ? (wd >> 1) : 0];
+            const __half2 w01 = __hsub2(*reinterpret_cast<__half2*>(&h01), o);
+            const __half2 w23 = __hsub2(*reinterpret_cast<__half2*>(&h23), o);
+            r[8 * wd + 2 * c] = *reinterpret_cast<const uint32_t*>(&w01);
+            r[8 * wd + 2 * c + 1] = *reinterpret_cast<const uint32_t*>(&w23);
           }
         }
-        tmem_st16(tmem + ((uint32_t)(32 * q) << 16) + kUAccCols + s * kUWCols + 16 * kh, r);
+        if (!__all_sync(0xffffffffu, mbar_wait(&empty[st], ph ^ 1, abort_flag))) { alive = false; break; }
+        tc_fence_after();
+        // the row's scale of each group that starts in this step, for the epilogue (published by the arrive below)
+        if (G != 128 || (kc & 1) == 0) {
+#pragma unroll
+          for (int i = 0; i < kGpc; ++i) sc_ring[(gidx0 + i) % kUScaleSlots][32 * q + lane] = sf[i];
+        }
+        tmem_st32(tmem + ((uint32_t)(32 * q) << 16) + kUAccCols + st * kUWCols, r);
         tmem_st_wait();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&full[s]);
+        if (lane == 0) mbar_arrive(&full[st]);
         i_issue(slot);  // after the step's words were consumed by every lane: the slot is free
+        if (++slot == kURawDepth) slot = 0;
+        st += 2;
+        if (st >= kUStages) { st -= kUStages; ph ^= 1; }
       }
+      it0 += nk;
     }
     cp_async_wait_but<0>();
   } else {
@@ -551,12 +596,16 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
         tc_fence_after();
         const float sf = sc_ring[gc % kUScaleSlots][32 * q + lane];
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          uint32_t r[16];
-          tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + ab * kPfTileM + 64 * hh + 16 * cc, r);
+        for (int cc = 0; cc < 4; cc += 2) {
+          uint32_t r0[16], r1[16];
+          const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + ab * kPfTileM + 64 * hh + 16 * cc;
+          tmem_ld16(ta, r0);
+          tmem_ld16(ta + 16, r1);
           tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 16; ++j) tot[16 * cc + j] = fmaf(sf, __uint_as_float(r[j]), tot[16 * cc + j]);
+          for (int j = 0; j < 16; ++j) tot[16 * cc + j] = fmaf(sf, __uint_as_float(r0[j]), tot[16 * cc + j]);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) tot[16 * cc + 16 + j] = fmaf(sf, __uint_as_float(r1[j]), tot[16 * cc + 16 + j]);
         }
         tc_fence_before();
         __syncwarp();
