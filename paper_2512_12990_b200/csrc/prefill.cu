@@ -595,21 +595,26 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
         if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[ab], (gc >> 1) & 1, abort_flag))) { alive = false; break; }
         tc_fence_after();
         const float sf = sc_ring[gc % kUScaleSlots][32 * q + lane];
+        // columns 0-31, then 32-63; the accumulator is released as soon as the last load has landed
+        const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + ab * kPfTileM + 64 * hh;
+        uint32_t r0[16], r1[16];
+        tmem_ld16(ta, r0);
+        tmem_ld16(ta + 16, r1);
+        tmem_ld_wait();
 #pragma unroll
-        for (int cc = 0; cc < 4; cc += 2) {
-          uint32_t r0[16], r1[16];
-          const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + ab * kPfTileM + 64 * hh + 16 * cc;
-          tmem_ld16(ta, r0);
-          tmem_ld16(ta + 16, r1);
-          tmem_ld_wait();
+        for (int j = 0; j < 16; ++j) tot[j] = fmaf(sf, __uint_as_float(r0[j]), tot[j]);
 #pragma unroll
-          for (int j = 0; j < 16; ++j) tot[16 * cc + j] = fmaf(sf, __uint_as_float(r0[j]), tot[16 * cc + j]);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) tot[16 * cc + 16 + j] = fmaf(sf, __uint_as_float(r1[j]), tot[16 * cc + 16 + j]);
-        }
+        for (int j = 0; j < 16; ++j) tot[16 + j] = fmaf(sf, __uint_as_float(r1[j]), tot[16 + j]);
+        tmem_ld16(ta + 32, r0);
+        tmem_ld16(ta + 48, r1);
+        tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[ab]);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) tot[32 + j] = fmaf(sf, __uint_as_float(r0[j]), tot[32 + j]);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) tot[48 + j] = fmaf(sf, __uint_as_float(r1[j]), tot[48 + j]);
       }
       if (!alive) break;
       const int tok0 = w.row0 + 64 * hh;
