@@ -544,6 +544,253 @@ def run_cuda(args, sh):
         dist.destroy_process_group()
 
 
+# ---- secondary workloads (not the default line) --------------------------------------------------------------
+def measured_tensor_peak():
+    """Dense bf16 tensor-core TFLOP/s (burst) measured on this machine, or the stated fallback.  fp16 operands
+    have the same nominal rate as bf16."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        return 1590.0, "fallback"
+
+
+def prefill_flops(sh, T: int) -> int:
+    """Useful flops of one prefill layer: every (token, expert) pair and every shared expert, three projections."""
+    return 2 * T * 3 * sh.hidden * (sh.top_k * sh.inter + sh.n_shared * sh.shared_inter)
+
+
+def run_prefill(args):
+    """The prefill layer of 2048 tokens: device-resident TFLOP/s of slicemoe_prefill_layer, the same call with
+    host buffers, and the share of the tensor-core peak."""
+    import torch
+    from paper_2512_12990_b200 import binding as B
+    from paper_2512_12990_b200 import synth
+    B.lib()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (the hot path has no CPU fallback)")
+    sh = synth.SHAPES["qwen_prefill"]
+    T = 2048
+    K, W = args.steps, max(args.warmup, 3)
+    dev = torch.device("cuda", 0)
+    L = max(2, min(args.layers, 4))      # 4 layers x 0.46 GB of planes: every step reads weights that left L2
+    layers = DeviceLayers(sh, L, dev, seed=sh.seed * 1000)
+    cs = layers.cshape
+    logits_h, _ = synth.zipf_gumbel_logits(sh.seed, ("bench-prefill-logits",), T, sh.n_experts, 1.0)
+    xbits_h = synth.activations_bf16(sh.seed, ("bench-prefill-x",), (T, sh.hidden))
+    x = torch.from_numpy(xbits_h.view(np.int16)).to(dev).view(torch.bfloat16)
+    ids, wts, _ = B.slicemoe_route_topk(torch.from_numpy(logits_h).to(dev), sh.top_k, renorm=True)
+    eprec = torch.from_numpy((synth.rng(sh.seed, "bench-prefill-prec").permutation(sh.n_experts) < sh.n_experts // 2)
+                             .astype(np.uint8)).to(dev)
+    ws = B.new_prefill_workspace(cs, T, dev)
+    y = torch.empty((T, sh.hidden), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+
+    def step(i, xin=x, yout=y):
+        l = i % L
+        B.slicemoe_prefill_layer(cs, layers.tables[l], layers.shared_tables[l], layers.gate_vecs[l], xin, ids, wts, eprec,
+                                 ws, yout, status, stream)
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    if int(status.item()) != 0:
+        raise RuntimeError("device status word set during warm-up")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record(stream)
+    for i in range(K):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    windows = [(t0, time.time())]
+    ms = e0.elapsed_time(e1) / K
+    # host buffers: x in from pinned memory, y out, every step
+    xh = torch.from_numpy(xbits_h.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    yh = torch.empty((T, sh.hidden), dtype=torch.float32).pin_memory()
+    xd = torch.empty_like(x)
+    Ke = min(K, 50)
+    t0 = time.time()
+    e0.record(stream)
+    with torch.cuda.stream(stream):
+        for i in range(Ke):
+            xd.copy_(xh, non_blocking=True)
+            step(i, xd, y)
+            yh.copy_(y, non_blocking=True)
+            stream.synchronize()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    windows.append((t0, time.time()))
+    e2e_ms = e0.elapsed_time(e1) / Ke
+    sampler.stop()
+    if int(status.item()) != 0:
+        raise RuntimeError("device status word set during the timed regions")
+    flops = prefill_flops(sh, T)
+    peak, kind = measured_tensor_peak()
+    tf = flops / (ms * 1e-3) / 1e12
+    out = {
+        "metric": "prefill TFLOP/s of one MoE layer (Qwen1.5-MoE shape, 2048 tokens); share of the tensor-core peak",
+        "value": tf, "unit": "TFLOP/s", "n_gpus": 1, "steps": K, "warmup": W, "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "fp16 x integer codes held in fp16, f32 accumulate", "data": "synthetic",
+        "config": {"workload": "qwen_prefill", "tokens": T, "hidden": sh.hidden, "inter": sh.inter, "experts": sh.n_experts,
+                   "top_k": sh.top_k, "shared_inter": sh.shared_inter, "group": sh.group,
+                   "precision_mix": "half of the experts at 8-bit, half at 4-bit; shared 8-bit",
+                   "routing": "Zipf(1.0) popularity + Gumbel noise, top-4",
+                   "resident_layers": L, "l2": f"steps cycle over {L} layers, 0.46 GB of planes each, so weights exceed L2"},
+        "flops_per_step": flops,
+        "e2e": {"value": flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": 2 * T * sh.hidden,
+                "d2h_bytes_per_step": 4 * T * sh.hidden, "steps": Ke},
+        "gpu_launches": 8 * K,
+        "roofline": {"bound": "tensor", "kernel": "pf_umma_kernel (both GEMMs) within the whole step", "achieved": tf,
+                     "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "peak_kind": f"of {kind}", "traffic": None},
+        "clocks": sampler.summary(windows),
+    }
+    print(json.dumps(out), flush=True)
+
+
+def run_stack(args):
+    """The 26-layer decode stack over a 256-step routing trace with the host slice cache at 30% capacity:
+    microseconds per token for the 26 expert FFNs with precision lists resident (value) and with the cache in the
+    loop - ids to the host, cache lookup, precision list back - for every layer (e2e)."""
+    import torch
+    from paper_2512_12990_b200 import binding as B
+    from paper_2512_12990_b200 import synth
+    B.lib()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (the hot path has no CPU fallback)")
+    sh = synth.SHAPES["dsv2_stack"]
+    NL, NS, TAU = sh.n_layers, 256, 0.25
+    dev = torch.device("cuda", 0)
+    layers = DeviceLayers(sh, NL, dev, seed=sh.seed * 1000)
+    cs, ws = layers.cshape, layers.ws
+    logits_h = synth.decode_trace_logits(sh.seed, NS, NL, sh.n_experts)
+    logits = torch.from_numpy(logits_h.reshape(NS * NL, sh.n_experts)).to(dev)
+    ids, wts, preq = B.slicemoe_route_topk(logits, sh.top_k, tau=TAU)
+    torch.cuda.synchronize()
+    ids_h, preq_h = ids.cpu().numpy(), preq.cpu().numpy()
+    w = sh.hidden * sh.inter
+    msb_b, lsb_b = 3 * (w // 2 + w // sh.group * 3), 3 * (w // 2)
+    cap = int(0.30 * NL * sh.n_experts * (msb_b + lsb_b))
+    cache = B.Dbsc(cap, msb_b, lsb_b)
+    prec_h = np.empty_like(preq_h)
+    for s in range(NS):
+        for l in range(NL):
+            r = s * NL + l
+            prec_h[r] = cache.assign(s, l, ids_h[r], preq_h[r])
+    stats = cache.stats()
+    prec = torch.from_numpy(prec_h).to(dev)
+    xbits_h = synth.activations_bf16(sh.seed, ("bench-stack-x",), (NS * NL, sh.hidden))
+    x = torch.from_numpy(xbits_h.view(np.int16)).to(dev).view(torch.bfloat16)
+    y = torch.empty((NS * NL, sh.hidden), dtype=torch.float32, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    lib = B.lib()
+    import ctypes
+    from ctypes import c_void_p
+    sptr, cs_ref, nws = c_void_p(stream.cuda_stream), ctypes.byref(cs), ws.numel()
+
+    def p(t, row=None, rowbytes=0):
+        return c_void_p(t.data_ptr() + (0 if row is None else row * rowbytes))
+
+    def layer(r, l, prec_t=prec):
+        rc = lib.slicemoe_layer(cs_ref, p(layers.tables[l]), p(layers.shared_tables[l]), None, p(x, r, 2 * sh.hidden), 1,
+                                p(ids, r, 4 * sh.top_k), p(prec_t, r, sh.top_k), p(wts, r, 4 * sh.top_k),
+                                p(y, r, 4 * sh.hidden), p(ws), nws, sptr)
+        if rc:
+            raise B.SliceMoEError(rc, "slicemoe_layer")
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    with torch.cuda.stream(stream):
+        for r in range(3 * NL):
+            layer(r, r % NL)
+    torch.cuda.synchronize()
+    graphs = []
+    for s0 in range(0, NS, 32):           # 32 tokens x 26 layers per graph
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for r in range(s0 * NL, (s0 + 32) * NL):
+                layer(r, r % NL)
+        graphs.append(g)
+    with torch.cuda.stream(stream):
+        graphs[0].replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for g in graphs:
+            g.replay()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    windows = [(t0, time.time())]
+    us_per_token = e0.elapsed_time(e1) * 1e3 / NS
+    if B.slicemoe_get_status(ws, stream) != 0:
+        raise RuntimeError("device status word set")
+    # bytes the FFNs read: per (step, layer) the selected experts at their precision plus the shared experts
+    per8, per4 = expert_bytes(sh.hidden, sh.inter, sh.group, True), expert_bytes(sh.hidden, sh.inter, sh.group, False)
+    n8 = int(prec_h.sum())
+    n4 = prec_h.size - n8
+    total_bytes = n8 * per8 + n4 * per4 + NS * NL * sh.n_shared * expert_bytes(sh.hidden, sh.shared_inter, sh.group, True)
+    # cache in the loop: route on the device, ids and requests to the host, lookup, precision list back, FFN
+    cache2 = B.Dbsc(cap, msb_b, lsb_b)
+    ids_p = torch.empty((1, sh.top_k), dtype=torch.int32).pin_memory()
+    req_p = torch.empty((1, sh.top_k), dtype=torch.uint8).pin_memory()
+    prec_p = torch.empty((1, sh.top_k), dtype=torch.uint8).pin_memory()
+    prec_d = torch.empty((NS * NL, sh.top_k), dtype=torch.uint8, device=dev)
+    NE = 64
+    t0 = time.time()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for s in range(NE):
+            for l in range(NL):
+                r = s * NL + l
+                rc = lib.slicemoe_route_topk(p(logits, r, 4 * sh.n_experts), 1, sh.n_experts, sh.top_k, None, 0, TAU, 0,
+                                             p(ids, r, 4 * sh.top_k), p(wts, r, 4 * sh.top_k), p(preq, r, sh.top_k), sptr)
+                if rc:
+                    raise B.SliceMoEError(rc, "slicemoe_route_topk")
+                ids_p.copy_(ids[r:r + 1], non_blocking=True)
+                req_p.copy_(preq[r:r + 1], non_blocking=True)
+                stream.synchronize()
+                prec_p[0] = torch.from_numpy(cache2.assign(s, l, ids_p[0].numpy(), req_p[0].numpy()))
+                prec_d[r:r + 1].copy_(prec_p, non_blocking=True)
+                layer(r, l, prec_d)
+        e1.record(stream)
+    torch.cuda.synchronize()
+    windows.append((t0, time.time()))
+    e2e_us = e0.elapsed_time(e1) * 1e3 / NE
+    sampler.stop()
+    if not torch.equal(prec_d[:NE * NL], prec[:NE * NL]):
+        raise RuntimeError("cache-in-the-loop precision lists differ from the precomputed ones")
+    peak, kind = measured_hbm_peak()
+    gbs = total_bytes / (us_per_token * NS * 1e-6) / 1e9
+    out = {
+        "metric": "µs per token of a 26-layer MoE decode stack (DSV2-Lite shape, b=1), slice cache at 30%",
+        "value": us_per_token, "unit": "µs/token", "n_gpus": 1, "steps": NS, "warmup": 3,
+        "ms_per_step": us_per_token / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 x int8/int4 codes, f32 accumulate", "data": "synthetic",
+        "config": {"workload": "dsv2_stack", "layers": NL, "steps": NS, "tau": TAU, "cache_fraction": 0.30,
+                   "trace": "Zipf(1.1) popularity per layer, p=0.5 repeat of the previous step's logits",
+                   "l2": f"{NL} layers of planes resident ({NL * sh.n_experts * (msb_b + lsb_b) / 1e9:.1f} GB); a byte is "
+                         "re-read at the earliest one token later, after ~1.3 GB of other traffic",
+                   "replay": "CUDA graphs of 32 tokens x 26 layers"},
+        "gbs": gbs, "bytes_per_token": total_bytes / NS,
+        "cache": {k: int(v) for k, v in stats.items()},
+        "e2e": {"value": e2e_us, "unit": "µs/token", "h2d_bytes_per_step": NL * sh.top_k,
+                "d2h_bytes_per_step": NL * sh.top_k * 5, "steps": NE,
+                "what": "route, ids and requests to the host, cache lookup, precision list back, FFN - per layer"},
+        "gpu_launches": NS * NL,
+        "roofline": {"bound": "hbm", "kernel": "decode_layer_kernel", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                     "frac": gbs / peak, "peak_kind": f"of {kind}", "traffic": None},
+        "clocks": sampler.summary(windows),
+    }
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -552,7 +799,19 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--layers", type=int, default=16, help="independently packed layers the steps cycle over")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "stack", "prefill"],
+                    help="the default is the headline decode layer; `stack` and `prefill` are single-GPU extras")
     args = ap.parse_args()
+    if args.workload in ("stack", "prefill") and args.impl == "cuda":
+        if int(os.environ.get("WORLD_SIZE", "1")) != 1 or args.gpus != 1:
+            raise SystemExit("--workload stack/prefill run on one GPU")
+        if args.workload == "prefill":
+            if args.steps == 20000 and args.warmup == 100:
+                args.steps, args.warmup = 200, 5
+            run_prefill(args)
+        else:
+            run_stack(args)
+        return
     from paper_2512_12990_b200 import synth
     sh = synth.SHAPES[WORKLOAD]
     if args.impl == "reference":

@@ -161,7 +161,7 @@ class _QwenPrefill:
         self.gate_vec = synth.normal_f32(sh.seed, ("gate_vec", 0), (sh.hidden,), 0.02)
         self.gate_vec_dev = torch.from_numpy(self.gate_vec).cuda()
         self.T = 2048
-        logits, _ = synth.zipf_gumbel_logits(sh.seed, ("prefill-logits",), self.T, sh.n_experts, 0.6)
+        logits, _ = synth.zipf_gumbel_logits(sh.seed, ("prefill-logits",), self.T, sh.n_experts, 1.0)
         self.ids, self.w, _ = moe.route_topk(logits, sh.top_k, renorm=True)
         self.expert_prec = (synth.rng(sh.seed, "prefill-prec").permutation(sh.n_experts) < sh.n_experts // 2).astype(np.uint8)
         self.xbits, self.x64 = H.x_inputs(sh, self.T, "prefill-x")
