@@ -935,17 +935,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
 
-  // Prologue, all roles in parallel and one barrier at the end: warp 0 reads the routing list and builds
-  // the slot table and the partition; warps 1 and 2 fetch the routed and the shared experts' plane
-  // pointers; the next 14 warps turn x into digits, one 128-element block at a time; the last warp sets
-  // up the barriers and the shared-expert gate.
-  if (warp == 0) {
-    build_plan(p, smem, lane);
-  } else if (warp == 1) {
-    load_slot_pointers(p, smem, lane, true);
-  } else if (warp == 2) {
-    if (p.n_shared > 0) load_slot_pointers(p, smem, lane, false);
-  } else if (warp == kProducerWarp) {
+  // Programmatic dependent launch: the next kernel in the stream may start launching as soon as every CTA
+  // of this grid has got here (its CTAs find room only where one of ours has exited), and this kernel sets
+  // up its barriers before it waits for the grids before it.  Nothing in global memory is touched before
+  // that wait: routing lists, x and the workspace may still be in use by the previous kernels.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (warp == kProducerWarp) {
     if (lane == 0) {
       *reinterpret_cast<int*>(smem + SmemLayout::dead) = 0;
       const uint32_t bars = smem_u32(smem + SmemLayout::bars);
@@ -969,6 +964,20 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  // Prologue, all roles in parallel and one barrier at the end: warp 0 reads the routing list and builds
+  // the slot table and the partition; warps 1 and 2 fetch the routed and the shared experts' plane
+  // pointers; the next 14 warps turn x into digits, one 128-element block at a time; the last warp sets
+  // up the barriers and the shared-expert gate.
+  if (warp == 0) {
+    build_plan(p, smem, lane);
+  } else if (warp == 1) {
+    load_slot_pointers(p, smem, lane, true);
+  } else if (warp == 2) {
+    if (p.n_shared > 0) load_slot_pointers(p, smem, lane, false);
+  } else if (warp == kProducerWarp) {
     if (p.sigmoid_gate && p.n_shared > 0) {
       // Qwen-style shared-expert gate: sigmoid(v . x)
       float dot = 0.f;
@@ -1040,8 +1049,17 @@ static int launch_decode(const DecodeParams& p, int dev, int sms, int gi, cudaSt
                                      SmemLayout::total));
     g_attr_set[dev][gi] = true;
   }
-  decode_layer_kernel<G><<<sms, kThreads, SmemLayout::total, st>>>(p);
-  SM_LAUNCH_CHECK();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(sms);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = SmemLayout::total;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see the top of the kernel
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  SM_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_layer_kernel<G>, p));
   return SLICEMOE_OK;
 }
 

@@ -15,6 +15,10 @@ __global__ void route_topk_kernel(const float* __restrict__ logits, int T, int E
                                   const float* __restrict__ bias, int renorm, float tau, int rank_high,
                                   int32_t* __restrict__ ids, float* __restrict__ weights,
                                   uint8_t* __restrict__ prec_req) {
+  // Programmatic dependent launch: the kernel after this one may start launching now; this one waits for the
+  // kernels before it (which may still be producing the logits) before it reads anything.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (warp >= T) return;
@@ -112,8 +116,16 @@ extern "C" int slicemoe_route_topk(const float* logits, int T, int E, int k, con
   if (E > 32 * slicemoe::ROUTE_MAX_VPT) return SLICEMOE_E_UNSUPPORTED;
   const int threads = 128;  // 4 tokens per block
   const int blocks = (T + 3) / 4;
-  slicemoe::route_topk_kernel<<<blocks, threads, 0, (cudaStream_t)stream>>>(
-      logits, T, E, k, bias, renorm, tau, rank_high, ids, weights, prec_req);
-  SM_LAUNCH_CHECK();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks);
+  cfg.blockDim = dim3(threads);
+  cfg.stream = (cudaStream_t)stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  SM_CUDA_TRY(cudaLaunchKernelEx(&cfg, slicemoe::route_topk_kernel, logits, T, E, k, bias, renorm, tau, rank_high, ids,
+                                 weights, prec_req));
   return SLICEMOE_OK;
 }
