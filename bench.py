@@ -400,13 +400,30 @@ def run_cuda(args, sh):
         if rc:
             raise B.SliceMoEError(rc, "slicemoe_layer")
 
-    def capture(first, count, with_route=True, with_layer=True):
+    def step(s):
+        """The whole hot path of one token in one launch: routing in the kernel's prologue, then the layer."""
+        i, l = s % P, s % L
+        st = layers.shared_tables[l]
+        gv = layers.gate_vecs[l]
+        rc = lib.slicemoe_layer_routed(cs_ref, p(layers.tables[l]), p(st) if st is not None else None,
+                                       p(gv) if gv is not None else None, p(x, i, 2 * sh.hidden), 1,
+                                       p(logits, i, 4 * sh.n_experts), None, 0, ctypes.c_float(2.0), RANK_HIGH,
+                                       p(ids, i, 4 * sh.top_k), p(prec, i, sh.top_k), p(wts, i, 4 * sh.top_k),
+                                       p(y, i, 4 * sh.hidden), p(ws), nws, sptr)
+        if rc:
+            raise B.SliceMoEError(rc, "slicemoe_layer_routed")
+
+    def capture(first, count, mode="step"):
+        """mode: "step" = the fused call; "two" = slicemoe_route_topk then slicemoe_layer; "layer" = the layer
+        kernel alone on lists already routed."""
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=stream):
             for s in range(first, first + count):
-                if with_route:
-                    route(s)
-                if with_layer:
+                if mode == "step":
+                    step(s)
+                else:
+                    if mode == "two":
+                        route(s)
                     layer(s)
         return g
 
@@ -441,6 +458,7 @@ def run_cuda(args, sh):
         for s in range(max(W, 3)):
             route(s)
             layer(s)
+            step(s)
         for s in range(P):
             route(s)
     torch.cuda.synchronize()
@@ -461,10 +479,21 @@ def run_cuda(args, sh):
     ms = max_over_ranks(ms, dist, dev)
     us_per_layer = whole_job_us_per_unit(ms, K, world)
 
-    # ---- roofline: the decode kernel alone, back to back ----------------------------------------------
-    kplan = [(capture(0, chunk, with_route=False), reps)]
+    # ---- the same through the two separate entry points (routing kernel, then layer kernel) ------------
+    tplan = [(capture(0, chunk, "two"), reps)]
     if rem:
-        kplan.append((capture(reps * chunk, rem, with_route=False), 1))
+        tplan.append((capture(reps * chunk, rem, "two"), 1))
+    for g, _ in tplan:
+        with torch.cuda.stream(stream):
+            g.replay()
+    tms, win = timed(tplan)
+    windows.append(win)
+    two_call_us = tms * 1e3 / K
+
+    # ---- roofline: the decode kernel alone, back to back ----------------------------------------------
+    kplan = [(capture(0, chunk, "layer"), reps)]
+    if rem:
+        kplan.append((capture(reps * chunk, rem, "layer"), 1))
     for g, _ in kplan:
         with torch.cuda.stream(stream):
             g.replay()
@@ -531,7 +560,9 @@ def run_cuda(args, sh):
         "gbs": bytes_per_launch * world / (us_per_layer * world * 1e-6) / 1e9,
         "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": 2 * sh.hidden + 4 * sh.n_experts,
                 "d2h_bytes_per_step": 4 * sh.hidden, "steps": Ke},
-        "gpu_launches": 2 * K,
+        "gpu_launches": K,
+        "step": "slicemoe_layer_routed: routing (softmax, top-k, precision request) in the decode kernel's prologue",
+        "two_call_us": two_call_us,
         "roofline": {"bound": "hbm", "kernel": "decode_layer_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "us_per_launch": kernel_us, "bytes_per_launch": bytes_per_launch},

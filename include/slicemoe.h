@@ -174,6 +174,23 @@ int slicemoe_layer(const slicemoe_shape *shape, const slicemoe_expert *experts,
                    void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * slicemoe_layer_routed - slicemoe_route_topk and slicemoe_layer in one kernel launch per token: the decode
+ * kernel's prologue computes the routing list from the router logits with the arithmetic of
+ * slicemoe_route_topk (same bits), takes the precision request as the precision list (Section 4.1: experts
+ * whose gating score reaches tau, or the rank_high best, run at both slices), and runs the layer.
+ *   logits   device float32 [T, E]; bias, renorm, tau, rank_high as in slicemoe_route_topk
+ *   ids_out, prec_out, weights_out   device [T, k] or NULL: the list the kernel used, for the caller's cache
+ *            bookkeeping (written by one CTA; valid when the call's work on `stream` has completed)
+ * A caller whose slice cache may override the request (a missing LSB slice) uses the two separate calls.
+ * Errors: as slicemoe_layer, plus UNSUPPORTED for E > 512.
+ */
+int slicemoe_layer_routed(const slicemoe_shape *shape, const slicemoe_expert *experts,
+                          const slicemoe_expert *shared, const float *shared_gate_vec, const void *x, int T,
+                          const float *logits, const float *bias, int renorm, float tau, int rank_high,
+                          int32_t *ids_out, uint8_t *prec_out, float *weights_out, float *y,
+                          void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * slicemoe_layer_static - slicemoe_layer for callers that cannot allocate device memory.  (The paper
  * has no counterpart; this is a convenience of the library.)
  *
@@ -207,9 +224,9 @@ int slicemoe_layer_static(const slicemoe_shape *shape, const slicemoe_expert *ex
 
 /*
  * slicemoe_decode_step_host - one batch-1 decode step of a layer with HOST inputs and outputs:
- * copies x (bf16 [hidden]) and logits (float32 [E]) to the device, runs slicemoe_route_topk
- * (bias/tau/rank_high as there; the precision request is used as the precision list) and
- * slicemoe_layer, copies y (float32 [hidden]) back and synchronises `stream`.  x_host, logits_host
+ * copies x (bf16 [hidden]) and logits (float32 [E]) to the device, runs slicemoe_layer_routed
+ * (bias/tau/rank_high as in slicemoe_route_topk; the precision request is used as the precision
+ * list), copies y (float32 [hidden]) back and synchronises `stream`.  x_host, logits_host
  * and y_host should be pinned for the copies to be asynchronous.  Weights stay resident on the
  * device.  Staging buffers live in the workspace.
  */

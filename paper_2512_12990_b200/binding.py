@@ -28,7 +28,7 @@ EXPORTS = (
     "slicemoe_strerror", "slicemoe_version", "slicemoe_last_cuda_error", "slicemoe_plane_bytes", "slicemoe_meta_count", "slicemoe_pack",
     "slicemoe_unpack_plane", "slicemoe_unpack_meta", "slicemoe_route_topk", "slicemoe_workspace_bytes",
     "slicemoe_workspace_init", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer",
-    "slicemoe_decode_step_host", "slicemoe_layer_static", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
+    "slicemoe_decode_step_host", "slicemoe_layer_static", "slicemoe_layer_routed", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
     "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
     "slicemoe_dbsc_assign", "slicemoe_dbsc_stats", "slicemoe_dbsc_contains",
 )
@@ -94,6 +94,9 @@ def lib() -> ctypes.CDLL:
     L.slicemoe_decode_step_host.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                             c_void_p, c_int, c_float, c_int, c_void_p, c_void_p, c_size_t,
                                             c_void_p]
+    L.slicemoe_layer_routed.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
+                                        c_int, c_float, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                        c_size_t, c_void_p]
     L.slicemoe_prefill_workspace_bytes.restype = c_size_t
     L.slicemoe_prefill_workspace_bytes.argtypes = [POINTER(Shape), c_int]
     L.slicemoe_prefill_layer.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
@@ -280,6 +283,25 @@ def slicemoe_layer_static(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec
                                      _stream(stream))
     _check(rc, "slicemoe_layer_static")
     return y
+
+
+def slicemoe_layer_routed(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x, logits, ws, bias=None, renorm=False,
+                          tau=2.0, rank_high=0, y=None, want_lists=True, stream=None):
+    """Routing and layer in one launch per token.  Returns (y, ids, prec, weights); the lists are None unless
+    want_lists."""
+    import torch
+    T = x.shape[0]
+    k = shape.top_k
+    if y is None:
+        y = torch.empty((T, shape.hidden), dtype=torch.float32, device=x.device)
+    ids = torch.empty((T, k), dtype=torch.int32, device=x.device) if want_lists else None
+    prec = torch.empty((T, k), dtype=torch.uint8, device=x.device) if want_lists else None
+    w = torch.empty((T, k), dtype=torch.float32, device=x.device) if want_lists else None
+    rc = lib().slicemoe_layer_routed(ctypes.byref(shape), _ptr(experts_tbl), _ptr(shared_tbl), _ptr(shared_gate_vec),
+                                     _ptr(x), T, _ptr(logits), _ptr(bias), 1 if renorm else 0, tau, rank_high, _ptr(ids),
+                                     _ptr(prec), _ptr(w), _ptr(y), _ptr(ws), ws.numel(), _stream(stream))
+    _check(rc, "slicemoe_layer_routed")
+    return y, ids, prec, w
 
 
 def slicemoe_decode_step_host(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x_host, logits_host, y_host,

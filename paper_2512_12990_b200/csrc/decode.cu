@@ -33,6 +33,7 @@
 #include <cuda_fp16.h>
 
 #include "common.cuh"
+#include "route.cuh"
 
 namespace slicemoe {
 
@@ -91,6 +92,15 @@ struct DecodeParams {
   int n_experts, n_shared, k;
   int hidden, inter, shared_inter, group;
   int sigmoid_gate;
+  // fused routing (logits != nullptr): the list is computed from the router logits in the prologue instead of
+  // read from ids / prec / weights, and written to the *_out arrays (each may be null) by one CTA
+  const float* logits;
+  const float* bias;
+  int renorm, rank_high;
+  float tau;
+  int32_t* ids_out;
+  uint8_t* prec_out;
+  float* weights_out;
 };
 
 struct Slot {
@@ -775,12 +785,25 @@ struct Routed {
   int pos;  // slot index of this lane's entry
   int nbig, nsmall;
 };
-__device__ __forceinline__ Routed read_routing(const DecodeParams& p, int lane) {
+__device__ __forceinline__ Routed read_routing(const DecodeParams& p, int lane, bool publish) {
   Routed rt;
   rt.e = -1;
   rt.pr = 0;
   rt.w = 0.f;
-  if (lane < p.k) {
+  if (p.logits) {
+    // same arithmetic as the stand-alone routing kernel; the precision request is the precision
+    const RouteSel sel = route_warp(p.logits, p.n_experts, p.k, p.bias, p.renorm, p.tau, p.rank_high, lane);
+    if (lane < p.k) {
+      rt.e = sel.id;
+      rt.pr = sel.prec_req;
+      rt.w = sel.w;
+      if (publish && blockIdx.x == 0) {
+        if (p.ids_out) p.ids_out[lane] = sel.id;
+        if (p.prec_out) p.prec_out[lane] = sel.prec_req;
+        if (p.weights_out) p.weights_out[lane] = sel.w;
+      }
+    }
+  } else if (lane < p.k) {
     rt.e = p.ids[lane];
     rt.pr = p.prec[lane];
     rt.w = p.weights[lane];
@@ -800,7 +823,7 @@ __device__ __forceinline__ Routed read_routing(const DecodeParams& p, int lane) 
 __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
   Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
   Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
-  const Routed rt = read_routing(p, lane);
+  const Routed rt = read_routing(p, lane, true);
   if (lane < p.k && !rt.valid) atomicOr(&p.ws->status, (unsigned)SLICEMOE_STATUS_BAD_EXPERT_ID);
   if (rt.valid) {
     Slot& s = slots[rt.pos];
@@ -900,7 +923,7 @@ __device__ void load_slot_pointers(const DecodeParams& p, uint8_t* smem, int lan
   const uint8_t* const* src[kRounds];
   int first = 0, count = p.n_shared;
   if (routed) {
-    const Routed rt = read_routing(p, lane);
+    const Routed rt = read_routing(p, lane, false);
     first = p.n_shared;
     count = rt.nbig + rt.nsmall;
     // lane j knows its entry's slot; every lane needs every slot's expert: pass them through the slot table
@@ -1076,13 +1099,26 @@ static int check_shape(const slicemoe_shape* s) {
   return SLICEMOE_OK;
 }
 
+// Routing computed in the kernel (run_layer's `fused` argument): logits [T, E] in, lists [T, k] out (optional).
+struct FusedRouting {
+  const float* logits;
+  const float* bias;
+  int renorm, rank_high;
+  float tau;
+  int32_t* ids_out;
+  uint8_t* prec_out;
+  float* weights_out;
+};
+
 static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts, const slicemoe_expert* shared,
                      int n_shared, const float* gate_vec, const void* x, int T, const int32_t* ids,
                      const uint8_t* prec, const float* weights, float* y, void* workspace, size_t workspace_bytes,
-                     void* stream) {
+                     void* stream, const FusedRouting* fused = nullptr) {
   int rc = check_shape(shape);
   if (rc != SLICEMOE_OK) return rc;
-  if (!experts || !x || !ids || !prec || !weights || !y || !workspace || T <= 0) return SLICEMOE_E_INVALID_ARG;
+  if (!experts || !x || !y || !workspace || T <= 0) return SLICEMOE_E_INVALID_ARG;
+  if (fused ? !fused->logits : (!ids || !prec || !weights)) return SLICEMOE_E_INVALID_ARG;
+  if (fused && shape->n_experts > 32 * ROUTE_MAX_VPT) return SLICEMOE_E_UNSUPPORTED;
   if (n_shared > 0 && !shared) return SLICEMOE_E_INVALID_ARG;
   if (n_shared > 0 && shape->shared_sigmoid_gate && !gate_vec) return SLICEMOE_E_INVALID_ARG;
   if (workspace_bytes < kWsBytes || (reinterpret_cast<uintptr_t>(workspace) & 255)) return SLICEMOE_E_INVALID_ARG;
@@ -1108,11 +1144,30 @@ static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts
   p.group = shape->group;
   p.sigmoid_gate = (n_shared > 0 && shape->shared_sigmoid_gate) ? 1 : 0;
   cudaStream_t st = (cudaStream_t)stream;
+  p.logits = nullptr;
+  p.bias = fused ? fused->bias : nullptr;
+  p.renorm = fused ? fused->renorm : 0;
+  p.rank_high = fused ? fused->rank_high : 0;
+  p.tau = fused ? fused->tau : 0.f;
+  p.ids_out = nullptr;
+  p.prec_out = nullptr;
+  p.weights_out = nullptr;
+  p.ids = nullptr;
+  p.prec = nullptr;
+  p.weights = nullptr;
   for (int t = 0; t < T; ++t) {
     p.x = reinterpret_cast<const uint16_t*>(x) + (size_t)t * shape->hidden;
-    p.ids = ids + (size_t)t * shape->top_k;
-    p.prec = prec + (size_t)t * shape->top_k;
-    p.weights = weights + (size_t)t * shape->top_k;
+    if (fused) {
+      const size_t o = (size_t)t * shape->top_k;
+      p.logits = fused->logits + (size_t)t * shape->n_experts;
+      p.ids_out = fused->ids_out ? fused->ids_out + o : nullptr;
+      p.prec_out = fused->prec_out ? fused->prec_out + o : nullptr;
+      p.weights_out = fused->weights_out ? fused->weights_out + o : nullptr;
+    } else {
+      p.ids = ids + (size_t)t * shape->top_k;
+      p.prec = prec + (size_t)t * shape->top_k;
+      p.weights = weights + (size_t)t * shape->top_k;
+    }
     p.y = y + (size_t)t * shape->hidden;
     if (shape->group == 128) rc = launch_decode<128>(p, dev, sms, 0, st);
     else if (shape->group == 64) rc = launch_decode<64>(p, dev, sms, 1, st);
@@ -1166,6 +1221,25 @@ extern "C" int slicemoe_layer(const slicemoe_shape* shape, const slicemoe_expert
                    workspace_bytes, stream);
 }
 
+extern "C" int slicemoe_layer_routed(const slicemoe_shape* shape, const slicemoe_expert* experts,
+                                     const slicemoe_expert* shared, const float* shared_gate_vec, const void* x, int T,
+                                     const float* logits, const float* bias, int renorm, float tau, int rank_high,
+                                     int32_t* ids_out, uint8_t* prec_out, float* weights_out, float* y,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
+  if (!shape) return SLICEMOE_E_INVALID_ARG;
+  FusedRouting f;
+  f.logits = logits;
+  f.bias = bias;
+  f.renorm = renorm;
+  f.rank_high = rank_high;
+  f.tau = tau;
+  f.ids_out = ids_out;
+  f.prec_out = prec_out;
+  f.weights_out = weights_out;
+  return run_layer(shape, experts, shared, shape->n_shared, shared_gate_vec, x, T, nullptr, nullptr, nullptr, y, workspace,
+                   workspace_bytes, stream, &f);
+}
+
 extern "C" int slicemoe_decode_step_host(const slicemoe_shape* shape, const slicemoe_expert* experts,
                                          const slicemoe_expert* shared, const float* shared_gate_vec,
                                          const void* x_host, const float* logits_host, const float* bias, int renorm,
@@ -1185,11 +1259,8 @@ extern "C" int slicemoe_decode_step_host(const slicemoe_shape* shape, const slic
   float* dy = reinterpret_cast<float*>(ws + kWsStY);
   SM_CUDA_TRY(cudaMemcpyAsync(dx, x_host, 2 * (size_t)shape->hidden, cudaMemcpyHostToDevice, st));
   SM_CUDA_TRY(cudaMemcpyAsync(dlogits, logits_host, 4 * (size_t)shape->n_experts, cudaMemcpyHostToDevice, st));
-  rc = slicemoe_route_topk(dlogits, 1, shape->n_experts, shape->top_k, bias, renorm, tau, rank_high, dids, dw, dprec,
-                           stream);
-  if (rc != SLICEMOE_OK) return rc;
-  rc = slicemoe_layer(shape, experts, shared, shared_gate_vec, dx, 1, dids, dprec, dw, dy, workspace, workspace_bytes,
-                      stream);
+  rc = slicemoe_layer_routed(shape, experts, shared, shared_gate_vec, dx, 1, dlogits, bias, renorm, tau, rank_high, dids,
+                             dprec, dw, dy, workspace, workspace_bytes, stream);
   if (rc != SLICEMOE_OK) return rc;
   SM_CUDA_TRY(cudaMemcpyAsync(y_host, dy, 4 * (size_t)shape->hidden, cudaMemcpyDeviceToHost, st));
   SM_CUDA_TRY(cudaStreamSynchronize(st));

@@ -167,3 +167,39 @@ def test_bad_expert_id_is_skipped_and_reported():
     assert status & B.STATUS_BAD_EXPERT_ID and np.array_equal(y, np.zeros_like(y))
     y, status = _run_layer(L, xbits, ids[:, :1].repeat(2, 1), prec, w, use_layer=False)
     assert status == 0
+
+
+@pytest.mark.parametrize("name", ["dsv2", "qwen"])
+def test_layer_routed_is_route_then_layer_in_one_launch(name):
+    """slicemoe_layer_routed: the lists it reports are those of slicemoe_route_topk, bit for bit, and y equals
+    slicemoe_layer run on them, bit for bit; and y is within tolerance of the oracle."""
+    from paper_2512_12990_b200 import binding as B
+    torch = _torch()
+    sh = synth.SHAPES[name]
+    T = 3
+    logits = synth.router_logits_normal(sh.seed, ("routed-logits",), T, sh.n_experts)
+    bias = synth.normal_f32(sh.seed, ("routed-bias",), (sh.n_experts,), 0.5)
+    ids_o, w_o, _ = moe.route_topk(logits, sh.top_k, bias=bias, renorm=True)
+    L = H.Layer(sh, set(ids_o.ravel().tolist()))
+    xbits, x64 = H.x_inputs(sh, T, "routed-x")
+    x = H.to_dev_bf16(xbits)
+    dl, db = _dev(logits), _dev(bias)
+    kw = dict(bias=db, renorm=True, tau=0.2, rank_high=1)
+    ids, w, pr = B.slicemoe_route_topk(dl, sh.top_k, **kw)
+    y_sep = B.slicemoe_layer(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, ids, pr, w, L.ws)
+    y_fused, ids_f, pr_f, w_f = B.slicemoe_layer_routed(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, dl, L.ws, **kw)
+    torch.cuda.synchronize()
+    assert B.slicemoe_get_status(L.ws) == 0
+    assert torch.equal(ids, ids_f) and torch.equal(pr, pr_f) and torch.equal(w, w_f)
+    assert torch.equal(y_sep, y_fused)
+    assert np.array_equal(ids.cpu().numpy(), ids_o)
+    prec = pr.cpu().numpy()
+    assert prec[:, 0].all() and 0 < prec.sum() < prec.size      # rank_high = 1; tau splits the rest
+    y_ref = moe.layer(x64, L.oracle_list(), ids_o, prec, w_o, shared=L.oracle_shared, shared_gate_vec=L.gate_vec)
+    for t in range(T):
+        H.assert_close(y_fused[t].cpu().numpy(), y_ref[t], f"{name} routed token {t}")
+    # without the lists
+    y2, i2, _, _ = B.slicemoe_layer_routed(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, dl, L.ws,
+                                           want_lists=False, **kw)
+    torch.cuda.synchronize()
+    assert i2 is None and torch.equal(y2, y_fused)
