@@ -785,12 +785,13 @@ struct Routed {
   int pos;  // slot index of this lane's entry
   int nbig, nsmall;
 };
+template <bool FUSED>
 __device__ __forceinline__ Routed read_routing(const DecodeParams& p, int lane, bool publish) {
   Routed rt;
   rt.e = -1;
   rt.pr = 0;
   rt.w = 0.f;
-  if (p.logits) {
+  if (FUSED) {
     // same arithmetic as the stand-alone routing kernel; the precision request is the precision
     const RouteSel sel = route_warp(p.logits, p.n_experts, p.k, p.bias, p.renorm, p.tau, p.rank_high, lane);
     if (lane < p.k) {
@@ -820,10 +821,11 @@ __device__ __forceinline__ Routed read_routing(const DecodeParams& p, int lane, 
 
 // Warp 0: slot table (all but the pointers) and the static partition, in closed form: the phase-1 unit
 // sequence is three runs of equal tasks (shared, routed 8-bit, routed 4-bit).
+template <bool FUSED>
 __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
   Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
   Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
-  const Routed rt = read_routing(p, lane, true);
+  const Routed rt = read_routing<FUSED>(p, lane, true);
   if (lane < p.k && !rt.valid) atomicOr(&p.ws->status, (unsigned)SLICEMOE_STATUS_BAD_EXPERT_ID);
   if (rt.valid) {
     Slot& s = slots[rt.pos];
@@ -917,13 +919,14 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
 
 // Warp 1: the routed slots' plane pointers.  Warp 2: the shared slots' (they do not depend on the list).
 // Each slot's twelve pointers sit in slicemoe_expert in the order the slot table keeps them.
+template <bool FUSED>
 __device__ void load_slot_pointers(const DecodeParams& p, uint8_t* smem, int lane, bool routed) {
   Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
   constexpr int kRounds = (kMaxSlots * 12 + 31) / 32;
   const uint8_t* const* src[kRounds];
   int first = 0, count = p.n_shared;
   if (routed) {
-    const Routed rt = read_routing(p, lane, false);
+    const Routed rt = read_routing<FUSED>(p, lane, false);
     first = p.n_shared;
     count = rt.nbig + rt.nsmall;
     // lane j knows its entry's slot; every lane needs every slot's expert: pass them through the slot table
@@ -952,7 +955,9 @@ __device__ void load_slot_pointers(const DecodeParams& p, uint8_t* smem, int lan
 }
 
 // ---- the kernel ------------------------------------------------------------------------------------
-template <int G>
+// FUSED: the routing list is computed from the router logits in the prologue (slicemoe_layer_routed); kept
+// apart from the plain kernel so that the latter carries none of the routing code.
+template <int G, bool FUSED>
 __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_constant__ DecodeParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -995,11 +1000,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
   // pointers; the next 14 warps turn x into digits, one 128-element block at a time; the last warp sets
   // up the barriers and the shared-expert gate.
   if (warp == 0) {
-    build_plan(p, smem, lane);
+    build_plan<FUSED>(p, smem, lane);
   } else if (warp == 1) {
-    load_slot_pointers(p, smem, lane, true);
+    load_slot_pointers<FUSED>(p, smem, lane, true);
   } else if (warp == 2) {
-    if (p.n_shared > 0) load_slot_pointers(p, smem, lane, false);
+    if (p.n_shared > 0) load_slot_pointers<FUSED>(p, smem, lane, false);
   } else if (warp == kProducerWarp) {
     if (p.sigmoid_gate && p.n_shared > 0) {
       // Qwen-style shared-expert gate: sigmoid(v . x)
@@ -1049,7 +1054,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
 
 // ---- host side --------------------------------------------------------------------------------------
 static int g_num_sms[64];
-static bool g_attr_set[64][3];
+static bool g_attr_set[64][6];
 
 static int device_setup(int* dev_out, int* sms_out) {
   int dev = 0;
@@ -1065,12 +1070,13 @@ static int device_setup(int* dev_out, int* sms_out) {
   return SLICEMOE_OK;
 }
 
-template <int G>
+template <int G, bool FUSED>
 static int launch_decode(const DecodeParams& p, int dev, int sms, int gi, cudaStream_t st) {
-  if (!g_attr_set[dev][gi]) {
-    SM_CUDA_TRY(cudaFuncSetAttribute(decode_layer_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  bool& attr_set = g_attr_set[dev][2 * gi + (FUSED ? 1 : 0)];
+  if (!attr_set) {
+    SM_CUDA_TRY(cudaFuncSetAttribute(decode_layer_kernel<G, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      SmemLayout::total));
-    g_attr_set[dev][gi] = true;
+    attr_set = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(sms);
@@ -1082,7 +1088,7 @@ static int launch_decode(const DecodeParams& p, int dev, int sms, int gi, cudaSt
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  SM_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_layer_kernel<G>, p));
+  SM_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_layer_kernel<G, FUSED>, p));
   return SLICEMOE_OK;
 }
 
@@ -1169,9 +1175,15 @@ static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts
       p.weights = weights + (size_t)t * shape->top_k;
     }
     p.y = y + (size_t)t * shape->hidden;
-    if (shape->group == 128) rc = launch_decode<128>(p, dev, sms, 0, st);
-    else if (shape->group == 64) rc = launch_decode<64>(p, dev, sms, 1, st);
-    else rc = launch_decode<32>(p, dev, sms, 2, st);
+    if (fused) {
+      if (shape->group == 128) rc = launch_decode<128, true>(p, dev, sms, 0, st);
+      else if (shape->group == 64) rc = launch_decode<64, true>(p, dev, sms, 1, st);
+      else rc = launch_decode<32, true>(p, dev, sms, 2, st);
+    } else {
+      if (shape->group == 128) rc = launch_decode<128, false>(p, dev, sms, 0, st);
+      else if (shape->group == 64) rc = launch_decode<64, false>(p, dev, sms, 1, st);
+      else rc = launch_decode<32, false>(p, dev, sms, 2, st);
+    }
     if (rc != SLICEMOE_OK) return rc;
   }
   return SLICEMOE_OK;
