@@ -49,7 +49,8 @@ extern "C" {
 /* Bits of the device status word (slicemoe_get_status). */
 #define SLICEMOE_STATUS_BAD_EXPERT_ID 1 /* an id in a device list was outside [0, n_experts): skipped */
 #define SLICEMOE_STATUS_WAIT_TIMEOUT 2  /* a bounded device-side wait ran out; the output is invalid */
-#define SLICEMOE_STATUS_MISSING_LSB 4   /* prec = 1 for an expert whose lsb planes are NULL: the output is invalid */
+#define SLICEMOE_STATUS_MISSING_LSB 4   /* both slices asked of an expert whose lsb planes are NULL: no fault; the
+                                           decode output is invalid, the prefill path runs the expert MSB-only */
 
 #define SLICEMOE_MAX_TOP_K 16
 #define SLICEMOE_MAX_SHARED 4

@@ -43,3 +43,14 @@ def test_single_rank_needs_no_process_group():
     assert bench.whole_job_us_per_unit(20.0, 1000, 1) == pytest.approx(20.0)
     sh = __import__("paper_2512_12990_b200.synth", fromlist=["SHAPES"]).SHAPES["dsv2"]
     assert bench.step_bytes(sh) == 57851904            # 3 x 8-bit + 3 x 4-bit routed + 2 shared 8-bit experts
+
+
+def test_prefill_flops_and_expert_bytes_are_the_stated_formulas():
+    import bench
+    from paper_2512_12990_b200 import synth
+    sh = synth.SHAPES["qwen_prefill"]
+    # 2 flops per multiply-add, three projections, top-4 routed experts of 1408 and one shared of 5632 per token
+    assert bench.prefill_flops(sh, 2048) == 2 * 2048 * 3 * 2048 * (4 * 1408 + 5632) == 283467841536
+    # planes used x N K / 2 + 3 bytes of (fp16 scale, u8 zero-point) per group, three matrices
+    assert bench.expert_bytes(2048, 1408, 128, True) == 3 * (2048 * 1408 + 3 * 2048 * 1408 // 128) == 8853504
+    assert bench.expert_bytes(2048, 1408, 128, False) == 3 * (2048 * 1408 // 2 + 3 * 2048 * 1408 // 128) == 4528128

@@ -203,3 +203,32 @@ def test_layer_routed_is_route_then_layer_in_one_launch(name):
                                            want_lists=False, **kw)
     torch.cuda.synchronize()
     assert i2 is None and torch.equal(y2, y_fused)
+
+
+def test_decode_reports_an_expert_without_lsb_planes_asked_for_8_bits():
+    """No fault and a status bit (the output is documented as invalid); asked for 4 bits the same table is fine."""
+    from paper_2512_12990_b200 import binding as B
+    torch = _torch()
+    sh = synth.SHAPES["tiny"]
+    L = H.Layer(sh, range(sh.n_experts))
+    stripped = []
+    for e in range(sh.n_experts):
+        mats = L.packed[e]
+        if e == 1:
+            mats = {k: B.PackedMat(m.N, m.K, m.group, m.msb, None, m.scale, m.zp) for k, m in mats.items()}
+        stripped.append(mats)
+    tbl = B.expert_table(stripped)
+    ids = np.array([[1, 6]], dtype=np.int32)
+    w = np.array([[0.6, 0.4]], dtype=np.float32)
+    xbits, x64 = H.x_inputs(sh, 1, "nolsb-x")
+    x = H.to_dev_bf16(xbits)
+    y = B.slicemoe_expert_ffn(L.cshape, tbl, x, _dev(ids), _dev(np.array([[1, 1]], dtype=np.uint8)), _dev(w), L.ws)
+    torch.cuda.synchronize()
+    assert B.slicemoe_get_status(L.ws) == B.STATUS_MISSING_LSB
+    assert torch.isfinite(y).all()
+    ws2 = B.new_workspace(L.cshape)
+    prec = np.array([[0, 1]], dtype=np.uint8)
+    y = B.slicemoe_expert_ffn(L.cshape, tbl, x, _dev(ids), _dev(prec), _dev(w), ws2)
+    torch.cuda.synchronize()
+    assert B.slicemoe_get_status(ws2) == 0
+    H.assert_close(y.cpu().numpy(), moe.expert_ffn(x64, L.oracle_list(), ids, prec, w.astype(np.float64)), "4-bit from MSB only")

@@ -220,3 +220,58 @@ def test_full_size_prefill_layer_sampled_tokens(qwen_prefill):
                                       _dev(q.w[sel].astype(np.float32)), _dev(q.expert_prec), ws_s)
     torch.cuda.synchronize()
     assert np.array_equal(y_s.cpu().numpy(), y[sel])
+
+
+def test_expert_without_lsb_planes_runs_from_the_msb_slice_and_reports_it():
+    """expert_prec = 1 for an expert whose LSB planes are absent: no fault; the expert runs MSB-only and the
+    status word says so (same contract as the decode path)."""
+    from paper_2512_12990_b200 import binding as B
+    sh = synth.SHAPES["tiny"]
+    L = H.Layer(sh, range(sh.n_experts))
+    stripped = []
+    for e in range(sh.n_experts):
+        mats = L.packed[e]
+        if e == 2:   # expert 2 keeps only its MSB planes
+            mats = {k: B.PackedMat(m.N, m.K, m.group, m.msb, None, m.scale, m.zp) for k, m in mats.items()}
+        stripped.append(mats)
+    tbl = B.expert_table(stripped)
+    T = 40
+    logits = synth.router_logits_normal(sh.seed, ("pf-nolsb",), T, sh.n_experts)
+    logits[:, 2] += 3.0                       # expert 2 is selected often
+    ids, w, _ = moe.route_topk(logits, sh.top_k)
+    assert (ids == 2).sum() > 10
+    xbits, x64 = H.x_inputs(sh, T, "pf-nolsb-x")
+    ws = B.new_prefill_workspace(L.cshape, T)
+    args = (H.to_dev_bf16(xbits), _dev(ids.astype(np.int32)), _dev(w.astype(np.float32)))
+    ones = np.ones(sh.n_experts, dtype=np.uint8)
+    y, status = B.slicemoe_prefill_layer(L.cshape, tbl, None, None, *args, _dev(ones), ws)
+    _torch().cuda.synchronize()
+    assert int(status.item()) == B.STATUS_MISSING_LSB
+    eff = ones.copy()
+    eff[2] = 0                                # what actually ran
+    y_ref = _oracle(L, x64, ids, w, eff)
+    for t in range(T):
+        H.assert_close(y[t].cpu().numpy(), y_ref[t], f"token {t}")
+    # asked correctly, nothing is reported
+    y2, status2 = B.slicemoe_prefill_layer(L.cshape, tbl, None, None, *args, _dev(eff), ws)
+    _torch().cuda.synchronize()
+    assert int(status2.item()) == 0 and np.array_equal(y2.cpu().numpy(), y.cpu().numpy())
+
+
+def test_large_batch_more_tokens_than_any_tile_count_assumption():
+    """4,100 tokens on the tiny layer (33 tiles per expert on average, ragged): sampled tokens against the oracle,
+    and the first 300 rows equal a 300-token call bit for bit."""
+    sh = synth.SHAPES["tiny"]
+    L = H.Layer(sh, range(sh.n_experts))
+    T = 4100
+    logits = synth.router_logits_normal(sh.seed, ("pf-big",), T, sh.n_experts)
+    ids, w, _ = moe.route_topk(logits, sh.top_k)
+    ep = (np.arange(sh.n_experts) < 4).astype(np.uint8)
+    xbits, x64 = H.x_inputs(sh, T, "pf-big-x")
+    y, status = _prefill(L, xbits, ids, w, ep)
+    assert status == 0
+    for t in (0, 1, 299, 300, 2048, 4095, 4099):
+        y_ref = _oracle(L, x64[t:t + 1], ids[t:t + 1], w[t:t + 1], ep)
+        H.assert_close(y[t], y_ref[0], f"token {t}")
+    y300, _ = _prefill(L, xbits[:300], ids[:300], w[:300], ep)
+    assert np.array_equal(y300, y[:300])
