@@ -46,6 +46,7 @@ constexpr int kProducerWarp = kConsumerWarps + 1;  // first of kProducers produc
 constexpr int kProducers = 2;                      // they take alternate tasks (phase 1) / chunks (phase 2)
 constexpr int kThreads = 32 * (kConsumerWarps + 1 + kProducers);
 constexpr int kUnits2 = 16;                        // at most this many (smaller) units in phase 2
+constexpr int kFull2PerGroup = 8;  // >= chunks one producer can have in flight in phase 2 (kUnits2 / 2 units)
 constexpr int kUnits = 8;                                 // ring units; a chunk takes one per plane
 constexpr int kChunkK = 2048;                             // K columns per chunk (16 blocks of 128)
 constexpr int kBlocksPerWarp = kChunkK / 128 / kGroupWarps;
@@ -117,11 +118,12 @@ struct Slot {
 //   phase 1: tasks n = 0 .. count1-1 are the (slot, 16-row block) pairs from (first_slot, first_idx) on.  A
 //     task of an 8-bit slot is 2 * nch chunks (gate then up; nch = 2048-column chunks of hidden), each two
 //     units (MSB tile, LSB tile); a task of a 4-bit slot is nch chunks, each two units (the gate's MSB tile
-//     and the up's).  Every phase-1 chunk takes two units: chunk number c sits in units 2c, 2c + 1 (mod
-//     kUnits).  Task n is consumed by group n % kGroups.
+//     and the up's).  Every phase-1 chunk takes two units.  Task n is consumed by group n % kGroups and
+//     produced by producer n % kProducers; which units and barriers a chunk uses is stated at `struct Bars`.
 //   phase 2: tasks m = 0 .. count2-1 are the output row blocks blockIdx.x + m * gridDim.x; each is one run of
 //     chunks over the slots in order (p2c[j] chunks and p2u[j] units come before slot j), two units per
-//     chunk for 8-bit slots and one for 4-bit slots.  Chunk number c is consumed by group c % kGroups.
+//     chunk for 8-bit slots and one for 4-bit slots.  Chunk number c is consumed by group c % kGroups and
+//     produced by producer c % kProducers.
 //     Phase 2 re-cuts the ring into nunits2 units of unit2_bytes, just large enough for the widest down
 //     chunk (plane area, then scales at scale2_off, zero-points at zp2_off), so that more - for the
 //     benchmark shapes all - of the phase's tiles are in shared memory before h arrives.
@@ -149,7 +151,7 @@ struct SmemLayout {
   static constexpr int slots = partial + kConsumerWarps * 16 * 2 * 4;
   static constexpr int plan = slots + kMaxSlots * (int)sizeof(Slot);
   static constexpr int bars = (plan + (int)sizeof(Plan) + 15) & ~15;  // uint64 barriers
-  static constexpr int nbars = 2 * kUnits + 2 * kUnits2 + 2 * kGroups + 5;
+  static constexpr int nbars = 2 * kUnits + kGroups * kFull2PerGroup + kUnits2 + 2 * kGroups + 5;
   static constexpr int dead = bars + nbars * 8;
   static constexpr int total = dead + 16;
 };
@@ -159,14 +161,21 @@ static_assert(SmemLayout::slots % 8 == 0 && SmemLayout::hdig % 16 == 0 && SmemLa
                   SmemLayout::plan % 8 == 0 && SmemLayout::partial % 8 == 0,
               "alignment");
 
-// Barrier indices: full[c % kUnits] for phase-1 chunk number c (armed with the chunk's bytes), empty[u] for
-// unit u (an arrive from each warp of the group that consumed it), full2 / empty2 likewise for phase 2
-// (chunk numbers and units counted from the start of the phase), pfull1 / pempty1 per group (phase-1 partial rows
-// to the epilogue warp and back), pfull2 / pempty2 (phase-2 partial rows of all warps), hx_go (h is complete
-// in the workspace), hs_ready (h is in shared memory as digits), p1_done (every consumer warp is through with
-// phase 1, so the ring may be re-cut).
+// Barriers.  Every barrier has ONE waiter that meets its phases strictly in order, so a parity wait can never
+// be a phase off (mbarrier.try_wait.parity only tells the current phase from the one before it):
+//   - a chunk's "full" barrier belongs to the consumer group that consumes it: group g's i-th chunk of a phase
+//     uses full[g][i % 2] in phase 1 and full2[g][i % kFull2PerGroup] in phase 2, armed with the chunk's bytes by
+//     the producer that serves the group (group g is served by producer g % kProducers in both phases);
+//   - an "empty" barrier belongs to the producer that refills the space: producer P owns half of the ring and
+//     walks it in order.  Phase 1: P's j-th chunk takes the unit pair (4 P + 2 (j % 2), + 1) and waits on
+//     empty[2 P + j % 2]; phase 2: P's units are [P h, P h + h), h = nunits2 / 2, taken in running order, one
+//     empty2 barrier per unit (an arrive from each warp of the group that consumed it).
+// pfull1 / pempty1 per group (phase-1 partial rows to the epilogue warp and back), pfull2 / pempty2 (phase-2
+// partial rows of all warps), hx_go (h is complete in the workspace), hs_ready (h is in shared memory as
+// digits), p1_done (every consumer warp is through with phase 1, so the ring may be re-cut).
 struct Bars {
-  static constexpr int full = 0, empty = kUnits, full2 = 2 * kUnits, empty2 = full2 + kUnits2, pfull1 = empty2 + kUnits2,
+  static constexpr int full = 0, empty = kUnits, full2 = 2 * kUnits, empty2 = full2 + kGroups * kFull2PerGroup,
+                       pfull1 = empty2 + kUnits2,
                        pempty1 = pfull1 + kGroups, pfull2 = pempty1 + kGroups, pempty2 = pfull2 + 1, hx_go = pfull2 + 2,
                        hs_ready = pfull2 + 3, p1_done = pfull2 + 4;
 };
@@ -458,18 +467,21 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
 
   // ---- phase 1: the tasks of this group ----
   const int nch = nchunks_of(p.hidden);
+  const int prod = group % kProducers;  // the producer that serves this group
   {
     int slot = plan.first_slot, idx = plan.first_idx, cn = 0;
+    int jp = 0;  // chunks of this group's producer so far (they fix the unit pair)
+    int ig = 0;  // chunks of this group so far (they fix the full barrier)
     for (int n = 0; n < plan.count1; ++n) {
       const Slot& sl = slots[slot];
       const int nchunks = sl.prec ? 2 * nch : nch;
       if (n % kGroups == group) {
         float part0 = 0.f, part1 = 0.f, unused = 0.f;
-        for (int q = 0; q < nchunks; ++q) {
+        for (int q = 0; q < nchunks; ++q, ++jp, ++ig) {
           const int c = cn + q;
           const int kc = q % nch;  // which 2048-column chunk of hidden
-          if (!mbar_wait(full0 + 8 * (c % kUnits), (c / kUnits) & 1, dead, status)) return;
-          const int u0 = (2 * c) % kUnits, u1 = u0 + 1;
+          if (!mbar_wait(full0 + 8 * (2 * group + (ig & 1)), (ig >> 1) & 1, dead, status)) return;
+          const int u0 = 4 * prod + 2 * (jp & 1);
           const int nblocks = min(kChunkK, p.hidden - kc * kChunkK) >> 7;
           const uint8_t* dig = smem + SmemLayout::xdig + kc * (kChunkK * 3);
           const float* sumw = reinterpret_cast<const float*>(smem + SmemLayout::xsumw) + kc * (kChunkK >> LG) * 2;
@@ -483,10 +495,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
                              kPlaneUnitBytes + kScaleUnitBytes, dig, sumw, binv, &part0, &part1);
           }
           __syncwarp();
-          if (lane == 0) {
-            mbar_arrive(empty0 + 8 * u0);
-            mbar_arrive(empty0 + 8 * u1);
-          }
+          if (lane == 0) mbar_arrive(empty0 + 8 * (2 * prod + (jp & 1)));
         }
         // hand the four warps' shares of the K split to the epilogue warp
         part0 += __shfl_xor_sync(0xffffffffu, part0, 1);  // digits 0,1 (even c) + digit 2 (odd c)
@@ -496,6 +505,8 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
         if (lr.cq == 0) partial[warp * 16 + lr.r] = make_float2(part0, part1);
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + 8 * (Bars::pfull1 + group));
+      } else if (n % kProducers == prod) {
+        jp += nchunks;  // the other group this producer serves
       }
       cn += nchunks;
       if (++idx >= sl.inter / 16) {
@@ -512,22 +523,29 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
   if (!fetch_h<G>(p, smem, warp, lane, plan.htotal, dead, status, bars)) return;
 
   // ---- phase 2: chunks round-robin over the groups, all warps contribute to every task ----
-  const int chunks2 = plan.p2c[plan.nslots], units2 = plan.p2u[plan.nslots];
+  const int chunks2 = plan.p2c[plan.nslots];
   const uint32_t full2 = bars + 8 * Bars::full2, empty2 = bars + 8 * Bars::empty2;
+  const int half = plan.nunits2 / kProducers;  // units of one producer
+  int xp = 0;                                   // units this group's producer has handed out so far
   for (int m = 0; m < plan.count2; ++m) {
     float part = 0.f, unused = 0.f;
     for (int j = 0; j < plan.nslots; ++j) {
       const Slot& sl = slots[j];
       const int nchj = plan.p2c[j + 1] - plan.p2c[j];
+      const int wu = sl.prec ? 2 : 1;
       float sacc = 0.f;
       bool mine = false;
       for (int kc = 0; kc < nchj; ++kc) {
         const int c = m * chunks2 + plan.p2c[j] + kc;  // chunk number within the phase
+        if (c % kProducers != prod) continue;
+        const int x0 = xp;
+        xp += wu;
         if (c % kGroups != group) continue;
         mine = true;
-        if (!mbar_wait(full2 + 8 * (c % kUnits2), (c / kUnits2) & 1, dead, status)) return;
-        const int unit = m * units2 + plan.p2u[j] + kc * (sl.prec ? 2 : 1);
-        const int u0 = unit % plan.nunits2, u1 = (unit + 1) % plan.nunits2;
+        const int ig = c / kGroups;  // this group's ordinal of the chunk
+        if (!mbar_wait(full2 + 8 * (kFull2PerGroup * group + ig % kFull2PerGroup), (ig / kFull2PerGroup) & 1, dead, status))
+          return;
+        const int u0 = prod * half + x0 % half, u1 = prod * half + (x0 + 1) % half;
         const int k0 = kc * kChunkK;
         const int nblocks = min(kChunkK, sl.inter - k0) >> 7;
         const uint8_t* dig = smem + SmemLayout::hdig + (sl.hoff + k0) * 3;
@@ -634,16 +652,20 @@ struct ProducerLane {
 };
 // The ring as a phase sees it.
 struct RingView {
-  uint32_t full0, empty0;  // shared-memory addresses of the phase's full / empty barriers
-  int nfull, nunits;
   uint32_t unit_bytes, scale_off, zp_off;
 };
+// Where one chunk goes: its two units, the barrier that says its space is free (with the parity to wait for)
+// and the barrier its bytes complete.
+struct ChunkSpace {
+  int u0, u1;
+  uint32_t empty_bar, empty_parity, full_bar;
+};
 
-// One chunk of matrix A - or of matrices A and B side by side - of (slot, row block rb), columns from k0:
-// chunk number cn and first unit number `unit` of its phase.  Run by the first kProducerLanes lanes of a
-// producer warp together.  Returns false if a wait ran out.
+// One chunk of matrix A - or of matrices A and B side by side - of (slot, row block rb), columns from k0, into
+// the space `cs`.  Run by the first kProducerLanes lanes of a producer warp together.  Returns false if a
+// wait ran out.
 template <int G>
-__device__ __forceinline__ bool produce_chunk(uint8_t* smem, const RingView& rv, int cn, int unit, int lane,
+__device__ __forceinline__ bool produce_chunk(uint8_t* smem, const RingView& rv, const ChunkSpace& cs, int lane,
                                               const ProducerLane& pl, const Slot& s, int matA, int matB, int mode, int K,
                                               int rb, int k0, volatile int* dead, unsigned* status) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
@@ -666,15 +688,13 @@ __device__ __forceinline__ bool produce_chunk(uint8_t* smem, const RingView& rv,
   }
   src += (size_t)((unsigned)rb * (unsigned)(K >> 7) + (unsigned)(k0 >> 7)) * pl.bytes_per_block;
   const uint32_t nblk = (uint32_t)(min(kChunkK, K - k0) >> 7);
-  // A chunk's units are released one after the other by the same warps, so the last one's barrier covers both.
-  const int ulast = unit + (two ? 1 : 0);
-  if (!mbar_wait(rv.empty0 + 8 * (ulast % rv.nunits), ((ulast / rv.nunits) & 1) ^ 1, dead, status)) return false;
-  const uint32_t bar = rv.full0 + 8 * (cn % rv.nfull);
+  if (!mbar_wait(cs.empty_bar, cs.empty_parity, dead, status)) return false;
+  const uint32_t bar = cs.full_bar;
   if (lane == 0)
     mbar_arrive_expect_tx(bar, nblk * ((two ? 2048u : 1024u) + (mode == kModePair ? 2u : 1u) * ((128u >> LG) * 48u)));
   __syncwarp((1u << kProducerLanes) - 1u);
   if (active) {
-    const uint32_t u = (uint32_t)((pl.second_unit ? unit + 1 : unit) % rv.nunits);
+    const uint32_t u = (uint32_t)(pl.second_unit ? cs.u1 : cs.u0);
     const uint32_t dst_in_unit = pl.field < 2 ? 0u : (pl.field == 2 ? rv.scale_off : rv.zp_off);
     bulk_g2s(smem_u32(smem + SmemLayout::ring) + u * rv.unit_bytes + dst_in_unit, src, nblk * pl.bytes_per_block, bar);
   }
@@ -697,27 +717,34 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
   bool ok = true;
   // phase 1: gate and up of (slot, row block) tasks; two units per chunk
   RingView r1;
-  r1.full0 = bars + 8 * Bars::full;
-  r1.empty0 = bars + 8 * Bars::empty;
-  r1.nfull = kUnits;
-  r1.nunits = kUnits;
   r1.unit_bytes = kUnitBytes;
   r1.scale_off = kPlaneUnitBytes;
   r1.zp_off = kPlaneUnitBytes + kScaleUnitBytes;
   const int nch = nchunks_of(p.hidden);
+  static_assert(kGroups == 2 * kProducers, "a producer serves the groups `which` and `which + kProducers`");
+  int ig_lo = 0, ig_hi = 0;  // chunks armed so far for group `which` and for group `which + kProducers`
   {
-    int slot = plan.first_slot, idx = plan.first_idx, cn = 0;
+    int slot = plan.first_slot, idx = plan.first_idx;
+    int jp = 0;  // this warp's chunks so far
     for (int n = 0; n < plan.count1 && ok; ++n) {
       const Slot& s = slots[slot];
       const int nchunks = s.prec ? 2 * nch : nch;
       if (n % kProducers == which) {
-        for (int q = 0; q < nchunks && ok; ++q) {
+        const int g = n % kGroups;
+        for (int q = 0; q < nchunks && ok; ++q, ++jp) {
           const int mat = s.prec ? q / nch : 0;
-          ok = produce_chunk<G>(smem, r1, cn + q, 2 * (cn + q), lane, pl, s, mat, s.prec ? mat : 1, s.prec ? kModeBoth : kModePair,
-                                p.hidden, idx, (q % nch) * kChunkK, dead, status);
+          ChunkSpace cs;
+          cs.u0 = 4 * which + 2 * (jp & 1);
+          cs.u1 = cs.u0 + 1;
+          cs.empty_bar = bars + 8 * (Bars::empty + 2 * which + (jp & 1));
+          cs.empty_parity = ((jp >> 1) & 1) ^ 1;
+          int& igg = g == which ? ig_lo : ig_hi;
+          cs.full_bar = bars + 8 * (Bars::full + 2 * g + (igg & 1));
+          ++igg;
+          ok = produce_chunk<G>(smem, r1, cs, lane, pl, s, mat, s.prec ? mat : 1, s.prec ? kModeBoth : kModePair, p.hidden,
+                                idx, (q % nch) * kChunkK, dead, status);
         }
       }
-      cn += nchunks;
       if (++idx >= s.inter / 16) {
         idx = 0;
         ++slot;
@@ -726,46 +753,48 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
   }
   // phase 2: down rows of every slot for the output row blocks of this CTA, in the re-cut ring
   RingView r2;
-  r2.full0 = bars + 8 * Bars::full2;
-  r2.empty0 = bars + 8 * Bars::empty2;
-  r2.nfull = kUnits2;
-  r2.nunits = plan.nunits2;
   r2.unit_bytes = (uint32_t)plan.unit2_bytes;
   r2.scale_off = (uint32_t)plan.scale2_off;
   r2.zp_off = (uint32_t)plan.zp2_off;
   // The re-cut units lie over the phase-1 units: nothing of phase 2 lands before phase 1 has been consumed.
   // (From then until h has crossed the grid the memory system has nothing else to do.)
   if (ok && plan.count2 > 0) ok = mbar_wait(bars + 8 * Bars::p1_done, 0, dead, status);
-  int c2 = 0, unit2 = 0;
+  const int half = plan.nunits2 / kProducers;  // this warp's units are [which * half, which * half + half)
+  int c2 = 0, xp = 0;                           // chunks of the phase so far, units this warp has handed out
   for (int m = 0; m < plan.count2 && ok; ++m) {
     const int rb = blockIdx.x + m * gridDim.x;
     for (int slot = 0; slot < plan.nslots && ok; ++slot) {
       const Slot& s = slots[slot];
       const int w = s.prec ? 2 : 1;
-      for (int k0 = 0; k0 < s.inter && ok; k0 += kChunkK) {
-        if (c2 % kProducers == which) {
-          if (ok)
-            ok = produce_chunk<G>(smem, r2, c2, unit2, lane, pl, s, 2, 2, s.prec ? kModeBoth : kModeSingle, s.inter, rb, k0, dead,
-                                  status);
-        }
-        ++c2;
-        unit2 += w;
+      for (int k0 = 0; k0 < s.inter && ok; k0 += kChunkK, ++c2) {
+        if (c2 % kProducers != which) continue;
+        const int g = c2 % kGroups, ig = c2 / kGroups;
+        const int xl = xp + w - 1;  // a chunk's units are released together: the last one's barrier covers both
+        ChunkSpace cs;
+        cs.u0 = which * half + xp % half;
+        cs.u1 = which * half + (xp + 1) % half;
+        cs.empty_bar = bars + 8 * (Bars::empty2 + which * half + xl % half);
+        cs.empty_parity = ((xl / half) & 1) ^ 1;
+        cs.full_bar = bars + 8 * (Bars::full2 + kFull2PerGroup * g + ig % kFull2PerGroup);
+        xp += w;
+        ok = produce_chunk<G>(smem, r2, cs, lane, pl, s, 2, 2, s.prec ? kModeBoth : kModeSingle, s.inter, rb, k0, dead, status);
       }
     }
   }
   // Never leave the CTA with bulk copies still landing in its shared memory: wait (bounded) until every
   // barrier this warp may have armed has completed its last phase.  In the normal path they have long ago.
-  {
-    const int cn1 = plan.chunks1;
-    for (int j = max(0, cn1 - kUnits); j < cn1; ++j) {
+  for (int g = which; g < kGroups; g += kProducers) {
+    const int n1 = g == which ? ig_lo : ig_hi;
+    for (int i = max(0, n1 - 2); i < n1; ++i) {
       const long long t0 = clock64();
-      while (!mbar_try(r1.full0 + 8 * (j % kUnits), (j / kUnits) & 1)) {
+      while (!mbar_try(bars + 8 * (Bars::full + 2 * g + (i & 1)), (i >> 1) & 1)) {
         if (*dead || (unsigned long long)(clock64() - t0) > kWaitCycles) break;
       }
     }
-    for (int j = max(0, c2 - kUnits2); j < c2; ++j) {
+    const int n2 = c2 > g ? (c2 - 1 - g) / kGroups + 1 : 0;  // chunks of the phase that went to group g
+    for (int i = max(0, n2 - kFull2PerGroup); i < n2; ++i) {
       const long long t0 = clock64();
-      while (!mbar_try(r2.full0 + 8 * (j % kUnits2), (j / kUnits2) & 1)) {
+      while (!mbar_try(bars + 8 * (Bars::full2 + kFull2PerGroup * g + i % kFull2PerGroup), (i / kFull2PerGroup) & 1)) {
         if (*dead || (unsigned long long)(clock64() - t0) > kWaitCycles) break;
       }
     }
@@ -976,10 +1005,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
         mbar_init(bars + 8 * (Bars::full + s), 1);             // lane 0's expect_tx arrive
         mbar_init(bars + 8 * (Bars::empty + s), kGroupWarps);  // one arrive per warp of the consuming group
       }
-      for (int s = 0; s < kUnits2; ++s) {
-        mbar_init(bars + 8 * (Bars::full2 + s), 1);
-        mbar_init(bars + 8 * (Bars::empty2 + s), kGroupWarps);
-      }
+      for (int s = 0; s < kGroups * kFull2PerGroup; ++s) mbar_init(bars + 8 * (Bars::full2 + s), 1);
+      for (int s = 0; s < kUnits2; ++s) mbar_init(bars + 8 * (Bars::empty2 + s), kGroupWarps);
       for (int g = 0; g < kGroups; ++g) {
         mbar_init(bars + 8 * (Bars::pfull1 + g), kGroupWarps);
         mbar_init(bars + 8 * (Bars::pempty1 + g), 1);

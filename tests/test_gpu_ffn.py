@@ -232,3 +232,34 @@ def test_decode_reports_an_expert_without_lsb_planes_asked_for_8_bits():
     torch.cuda.synchronize()
     assert B.slicemoe_get_status(ws2) == 0
     H.assert_close(y.cpu().numpy(), moe.expert_ffn(x64, L.oracle_list(), ids, prec, w.astype(np.float64)), "4-bit from MSB only")
+
+
+def test_maximum_sizes_of_the_decode_kernel():
+    """hidden 4096 (the limit), top-16 (the limit) of 20 experts x 640 plus 4 shared experts (the limit) x 512:
+    the intermediate widths sum to 12288, exactly the capacity of the workspace; one more column is refused."""
+    from paper_2512_12990_b200 import binding as B
+    torch = _torch()
+    sh = synth.Shape("max", 4096, 640, 20, 16, 128, n_shared=4, shared_inter=512, shared_sigmoid_gate=True, seed=2900)
+    assert sh.top_k * sh.inter + sh.n_shared * sh.shared_inter == 12288
+    logits = synth.router_logits_normal(sh.seed, ("max-logits",), 1, sh.n_experts)
+    ids, w, _ = moe.route_topk(logits, sh.top_k)
+    L = H.Layer(sh, ids.ravel().tolist())
+    prec = (np.arange(sh.top_k)[None, :] % 3 == 0).astype(np.uint8)
+    xbits, x64 = H.x_inputs(sh, 1, "max-x")
+    y, status = _run_layer(L, xbits, ids, prec, w)
+    assert status == 0
+    y_ref = moe.layer(x64, L.oracle_list(), ids, prec, w, shared=L.oracle_shared, shared_gate_vec=L.gate_vec)
+    H.assert_close(y, y_ref, "maximum sizes")
+    # beyond the limits: refused on the host, nothing launched
+    x = H.to_dev_bf16(xbits)
+    args = (_dev(ids.astype(np.int32)), _dev(prec), _dev(w.astype(np.float32)))
+    wide = B.make_shape(4096, 768, 20, 16, 128, 4, 512, True)          # 16 * 768 + 4 * 512 > 12288
+    with pytest.raises(B.SliceMoEError) as ei:
+        B.slicemoe_layer(wide, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, *args, L.ws)
+    assert ei.value.code == B.E_UNSUPPORTED
+    tall = B.make_shape(4224, 640, 20, 16, 128, 4, 512, True)          # hidden > 4096
+    with pytest.raises(B.SliceMoEError) as ei:
+        B.slicemoe_layer(tall, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, *args, L.ws)
+    assert ei.value.code == B.E_UNSUPPORTED
+    torch.cuda.synchronize()
+    assert B.slicemoe_get_status(L.ws) == 0

@@ -275,3 +275,40 @@ def test_large_batch_more_tokens_than_any_tile_count_assumption():
         H.assert_close(y[t], y_ref[0], f"token {t}")
     y300, _ = _prefill(L, xbits[:300], ids[:300], w[:300], ep)
     assert np.array_equal(y300, y[:300])
+
+
+def test_wide_layer_beyond_the_decode_limits():
+    """The prefill path has no cap on hidden or on the sum of intermediate widths: hidden 4224 (above the decode
+    kernel's 4096), top-3 of 6 experts x 256, group 64."""
+    sh = synth.Shape("pf_wide", 4224, 256, 6, 3, 64, n_shared=1, shared_inter=384, shared_sigmoid_gate=False, n_layers=1,
+                     seed=4300)
+    L = H.Layer.__new__(H.Layer)  # the decode workspace of H.Layer refuses this shape: build the parts by hand
+    import torch
+    from paper_2512_12990_b200 import binding as B
+    L.shape = sh
+    L.cshape = B.make_shape(sh.hidden, sh.inter, sh.n_experts, sh.top_k, sh.group, sh.n_shared, sh.shared_inter, False)
+    L.oracle_experts, L.packed = {}, {}
+
+    def make(tag, inter):
+        W = synth.expert_weights(sh.seed, 0, tag, sh.hidden, inter)
+        o = {k: amat.pack_matrix(W[k], sh.group) for k in ("gate", "up", "down")}
+        d = {k: B.slicemoe_pack(torch.from_numpy(W[k]).cuda(), sh.group) for k in ("gate", "up", "down")}
+        return o, d
+
+    for e in range(sh.n_experts):
+        L.oracle_experts[e], L.packed[e] = make(e, sh.inter)
+    L.experts_tbl = B.expert_table([L.packed[e] for e in range(sh.n_experts)])
+    so, sd = make("shared0", sh.shared_inter)
+    L.oracle_shared, L.packed_shared = [so], [sd]
+    L.shared_tbl = B.expert_table(L.packed_shared)
+    L.gate_vec, L.gate_vec_dev = None, None
+    T = 150
+    logits = synth.router_logits_normal(sh.seed, ("pf-wide",), T, sh.n_experts)
+    ids, w, _ = moe.route_topk(logits, sh.top_k, renorm=True)
+    ep = np.array([1, 0, 1, 1, 0, 0], dtype=np.uint8)
+    xbits, x64 = H.x_inputs(sh, T, "pf-wide-x")
+    y, status = _prefill(L, xbits, ids, w, ep)
+    assert status == 0
+    y_ref = _oracle(L, x64, ids, w, ep)
+    for t in range(T):
+        H.assert_close(y[t], y_ref[t], f"token {t}")
