@@ -148,6 +148,7 @@ __global__ void pf_gather_kernel(const uint16_t* __restrict__ x, int hidden, con
 // SLICEMOE_STATUS_WAIT_TIMEOUT and the CTA winds down (tensor memory is freed on every path).
 constexpr int kUThreads = 576;      // warps 0-7 epilogue, 8-15 dequantisation, 16 loads, 17 MMA issue
 constexpr int kUStages = 6;
+static_assert(kUStages % 2 == 0, "each dequantisation set must meet every one of its stages on every lap of the ring");
 constexpr int kUTileBytes = kPfTileM * kPfChunkK * 2;  // 16,384: the token tile of a step
 constexpr int kUScaleSlots = 16;    // ring of per-group scale rows: dequantisation runs at most 15 groups ahead of the epilogue
 constexpr int kUScaleBytes = kUScaleSlots * kPfTileB * 4;
