@@ -659,6 +659,7 @@ struct RingView {
 struct ChunkSpace {
   int u0, u1;
   uint32_t empty_bar, empty_parity, full_bar;
+  uint32_t empty_bar_first, empty_parity_first;  // phase 2, two-unit chunks: the first unit has a barrier of its own
 };
 
 // One chunk of matrix A - or of matrices A and B side by side - of (slot, row block rb), columns from k0, into
@@ -688,6 +689,8 @@ __device__ __forceinline__ bool produce_chunk(uint8_t* smem, const RingView& rv,
   }
   src += (size_t)((unsigned)rb * (unsigned)(K >> 7) + (unsigned)(k0 >> 7)) * pl.bytes_per_block;
   const uint32_t nblk = (uint32_t)(min(kChunkK, K - k0) >> 7);
+  // The two units of a phase-2 chunk may last have held chunks of different consumer groups: both must be free.
+  if (cs.empty_bar_first != 0u && !mbar_wait(cs.empty_bar_first, cs.empty_parity_first, dead, status)) return false;
   if (!mbar_wait(cs.empty_bar, cs.empty_parity, dead, status)) return false;
   const uint32_t bar = cs.full_bar;
   if (lane == 0)
@@ -738,6 +741,8 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
           cs.u1 = cs.u0 + 1;
           cs.empty_bar = bars + 8 * (Bars::empty + 2 * which + (jp & 1));
           cs.empty_parity = ((jp >> 1) & 1) ^ 1;
+          cs.empty_bar_first = 0u;  // a phase-1 unit pair always holds one chunk: one barrier
+          cs.empty_parity_first = 0u;
           int& igg = g == which ? ig_lo : ig_hi;
           cs.full_bar = bars + 8 * (Bars::full + 2 * g + (igg & 1));
           ++igg;
@@ -769,12 +774,14 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
       for (int k0 = 0; k0 < s.inter && ok; k0 += kChunkK, ++c2) {
         if (c2 % kProducers != which) continue;
         const int g = c2 % kGroups, ig = c2 / kGroups;
-        const int xl = xp + w - 1;  // a chunk's units are released together: the last one's barrier covers both
+        const int xl = xp + w - 1;  // the chunk's last unit
         ChunkSpace cs;
         cs.u0 = which * half + xp % half;
         cs.u1 = which * half + (xp + 1) % half;
         cs.empty_bar = bars + 8 * (Bars::empty2 + which * half + xl % half);
         cs.empty_parity = ((xl / half) & 1) ^ 1;
+        cs.empty_bar_first = w == 2 ? bars + 8 * (Bars::empty2 + which * half + xp % half) : 0u;
+        cs.empty_parity_first = ((xp / half) & 1) ^ 1;
         cs.full_bar = bars + 8 * (Bars::full2 + kFull2PerGroup * g + ig % kFull2PerGroup);
         xp += w;
         ok = produce_chunk<G>(smem, r2, cs, lane, pl, s, 2, 2, s.prec ? kModeBoth : kModeSingle, s.inter, rb, k0, dead, status);
