@@ -34,7 +34,35 @@ def _cases():
     return out
 
 
-@pytest.mark.parametrize("case", _cases(), ids=lambda c: f"{c[0]}-h{c[1]}-i{c[2]}-E{c[3]}-k{c[4]}-g{c[5]}-s{c[6]}x{c[7]}-T{c[9]}")
+def _heavy_cases():
+    """Shapes that wrap the decode kernel's staging rings: wide slots (several 2048-column chunks per slot), small
+    groups (large units), many slots, two output row blocks per CTA."""
+    rng = np.random.default_rng(20251213)
+    out = []
+    for i in range(60):
+        hidden = int(rng.choice([2048, 2432, 3072, 4096]))
+        group = int(rng.choice([32, 32, 64, 128]))
+        k = int(rng.choice([1, 2, 3, 4, 6, 8]))
+        E = int(k + rng.integers(0, 3))
+        n_shared = int(rng.choice([0, 1, 2, 4]))
+        inter = int(rng.choice([1024, 1408, 2176, 2560, 4096]))
+        shared_inter = int(rng.choice([1408, 2176, 5632])) if n_shared else 0
+        while k * inter + n_shared * shared_inter > 12288:
+            if n_shared > 1:
+                n_shared -= 1
+            elif inter > 1024:
+                inter -= 128
+            elif shared_inter > 128:
+                shared_inter -= 128
+            else:
+                k -= 1
+        E = max(E, k)
+        gated = bool(rng.integers(0, 2)) and n_shared > 0
+        out.append((1000 + i, hidden, inter, E, k, group, n_shared, shared_inter, gated, int(rng.choice([1, 2]))))
+    return out
+
+
+@pytest.mark.parametrize("case", _cases() + _heavy_cases(), ids=lambda c: f"{c[0]}-h{c[1]}-i{c[2]}-E{c[3]}-k{c[4]}-g{c[5]}-s{c[6]}x{c[7]}-T{c[9]}")
 def test_decode_and_prefill_paths_agree(case):
     import torch
     from paper_2512_12990_b200 import binding as B
