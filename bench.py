@@ -608,12 +608,13 @@ def run_prefill(args):
     L = max(2, min(args.layers, 4))      # 4 layers x 0.46 GB of planes: every step reads weights that left L2
     layers = DeviceLayers(sh, L, dev, seed=sh.seed * 1000)
     cs = layers.cshape
-    logits_h, _ = synth.zipf_gumbel_logits(sh.seed, ("bench-prefill-logits",), T, sh.n_experts, 1.0)
+    logits_h, perm = synth.zipf_gumbel_logits(sh.seed, ("bench-prefill-logits",), T, sh.n_experts, 1.0)
     xbits_h = synth.activations_bf16(sh.seed, ("bench-prefill-x",), (T, sh.hidden))
     x = torch.from_numpy(xbits_h.view(np.int16)).to(dev).view(torch.bfloat16)
     ids, wts, _ = B.slicemoe_route_topk(torch.from_numpy(logits_h).to(dev), sh.top_k, renorm=True)
-    eprec = torch.from_numpy((synth.rng(sh.seed, "bench-prefill-prec").permutation(sh.n_experts) < sh.n_experts // 2)
-                             .astype(np.uint8)).to(dev)
+    eprec_h = np.zeros(sh.n_experts, dtype=np.uint8)
+    eprec_h[perm[1::2]] = 1              # experts of odd popularity rank hold both slices, even rank the MSB slice
+    eprec = torch.from_numpy(eprec_h).to(dev)
     ws = B.new_prefill_workspace(cs, T, dev)
     y = torch.empty((T, sh.hidden), dtype=torch.float32, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
@@ -670,7 +671,7 @@ def run_prefill(args):
         "dtype": "fp16 x integer codes held in fp16, f32 accumulate", "data": "synthetic",
         "config": {"workload": "qwen_prefill", "tokens": T, "hidden": sh.hidden, "inter": sh.inter, "experts": sh.n_experts,
                    "top_k": sh.top_k, "shared_inter": sh.shared_inter, "group": sh.group,
-                   "precision_mix": "half of the experts at 8-bit, half at 4-bit; shared 8-bit",
+                   "precision_mix": "experts of even popularity rank at 4-bit, odd rank at 8-bit; shared 8-bit",
                    "routing": "Zipf(1.0) popularity + Gumbel noise, top-4",
                    "resident_layers": L, "l2": f"steps cycle over {L} layers, 0.46 GB of planes each, so weights exceed L2"},
         "flops_per_step": flops,

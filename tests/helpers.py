@@ -85,3 +85,32 @@ def x_inputs(shape: synth.Shape, T: int, tag="x"):
 def to_dev_bf16(bits: np.ndarray, device="cuda"):
     import torch
     return torch.from_numpy(bits.view(np.int16).copy()).to(device).view(torch.bfloat16)
+
+
+def oracle_mat_from_device(pm) -> dict:
+    """The oracle's view (canonical arrays, as oracle.amat.pack_matrix returns them) of a matrix packed on the
+    GPU, read back through slicemoe_unpack_plane / slicemoe_unpack_meta.  For the large configurations, where
+    packing every matrix a second time in numpy would take minutes; slicemoe_pack itself is compared bit for bit
+    with the oracle's quantiser in test_gpu_pack.py."""
+    from paper_2512_12990_b200 import binding as B
+    msb = B.slicemoe_unpack_plane(pm.msb, pm.N, pm.K).cpu().numpy()
+    lsb = B.slicemoe_unpack_plane(pm.lsb, pm.N, pm.K).cpu().numpy()
+    s, z = B.slicemoe_unpack_meta(pm.scale, pm.zp, pm.N, pm.K, pm.group)
+    return dict(scale=s.cpu().numpy(), zp=z.cpu().numpy(), msb=msb, lsb=lsb, group=pm.group, b_high=8, b_low=4)
+
+
+def oracle_expert_from_device(packed: dict) -> dict:
+    return {k: oracle_mat_from_device(packed[k]) for k in ("gate", "up", "down")}
+
+
+def device_expert(seed: int, tag, hidden: int, inter: int, group: int, std: float = 0.02) -> dict:
+    """One SwiGLU expert drawn on the GPU (torch generator seeded by (seed, tag)) and packed there."""
+    import hashlib
+    import torch
+    from paper_2512_12990_b200 import binding as B
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(int.from_bytes(hashlib.sha256(repr((seed, tag)).encode()).digest()[:7], "little"))
+    out = {}
+    for name, shape in (("gate", (inter, hidden)), ("up", (inter, hidden)), ("down", (hidden, inter))):
+        out[name] = B.slicemoe_pack(torch.randn(shape, device="cuda", generator=gen) * std, group)
+    return out

@@ -71,16 +71,29 @@ def test_decode_stack_routing_cache_and_sampled_layers():
     assert 0.0 < miss_rate < 0.6 and st["msb_hit"] > st["msb_miss"]
     c_host.close()
 
-    # ---- sampled (step, layer) pairs through slicemoe_layer ----
-    samples = [(0, l) for l in (0, 13, 25)] + [(t, t % L) for t in (1, 5, 9, 16, 96, 255)]
+    # ---- sampled (step, layer) pairs through slicemoe_layer: every layer at step 0, steps 1-9, every 16th step ----
+    # The experts of a sampled pair are drawn and packed on the GPU; the oracle works on the planes read back.
+    samples = [(0, l) for l in range(L)] + [(t, t % L) for t in range(1, 10)] + [(t, t % L) for t in range(16, N_STEPS, 16)]
+    cshape = B.make_shape(sh.hidden, sh.inter, E, k, sh.group, sh.n_shared, sh.shared_inter, False)
+    ws = B.new_workspace(cshape)
+    worst = 0.0
     for (t, l) in samples:
-        lay = H.Layer(sh, ids3[t, l], layer=l)
+        need = [int(e) for e in ids3[t, l]]
+        packed = {e: H.device_expert(sh.seed, ("stack", l, e), sh.hidden, sh.inter, sh.group) for e in need}
+        decoy = H.device_expert(sh.seed, ("stack", l, "decoy"), sh.hidden, sh.inter, sh.group)
+        shared = [H.device_expert(sh.seed, ("stack", l, "shared", j), sh.hidden, sh.shared_inter, sh.group)
+                  for j in range(sh.n_shared)]
+        tbl = B.expert_table([packed.get(e, decoy) for e in range(E)])
+        stbl = B.expert_table(shared)
         xbits, x64 = H.x_inputs(sh, 1, ("x-stack", t, l))
         row = (t * L + l)
-        y = B.slicemoe_layer(lay.cshape, lay.experts_tbl, lay.shared_tbl, None, H.to_dev_bf16(xbits),
-                             ids_d[row:row + 1], torch.from_numpy(prec3[t, l:l + 1].copy()).cuda(), w_d[row:row + 1], lay.ws)
+        y = B.slicemoe_layer(cshape, tbl, stbl, None, H.to_dev_bf16(xbits), ids_d[row:row + 1],
+                             torch.from_numpy(prec3[t, l:l + 1].copy()).cuda(), w_d[row:row + 1], ws)
         torch.cuda.synchronize()
-        assert B.slicemoe_get_status(lay.ws) == 0
-        y_ref = moe.layer(x64, lay.oracle_list(), ids3[t, l:l + 1], prec3[t, l:l + 1], w[row:row + 1], shared=lay.oracle_shared)
+        assert B.slicemoe_get_status(ws) == 0
+        o_experts = {e: H.oracle_expert_from_device(packed[e]) for e in need}
+        o_shared = [H.oracle_expert_from_device(sx) for sx in shared]
+        y_ref = moe.layer(x64, o_experts, ids3[t, l:l + 1], prec3[t, l:l + 1], w[row:row + 1], shared=o_shared)
         rel, mx = H.assert_close(y.cpu().numpy(), y_ref, f"stack step {t} layer {l}")
-        del lay
+        worst = max(worst, rel)
+    print(f"stack: {len(samples)} sampled (step, layer) pairs, worst rel-L2 {worst:.2e}")
