@@ -504,6 +504,44 @@ def run_cuda(args, sh):
     peak, peak_kind = measured_hbm_peak()
     achieved = bytes_per_launch / (kernel_us * 1e-6) / 1e9
 
+    # ---- beside the headline: spread over graph replays, plain-stream launches, warm L2 -----------------
+    # (a) the layer-kernel graph replay by replay: median and minimum of the per-launch average
+    per_replay = []
+    g0, n0 = kplan[0]
+    for _ in range(min(n0, 10)):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            g0.replay()
+            e1.record(stream)
+        torch.cuda.synchronize()
+        per_replay.append(e0.elapsed_time(e1) * 1e3 / chunk)
+    # (b) the step without a graph: plain launches on the stream (the host's launch rate is part of it)
+    Ks = min(K, 2000)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for s_ in range(Ks):
+            route(s_)
+            layer(s_)
+        e1.record(stream)
+    torch.cuda.synchronize()
+    stream_us = e0.elapsed_time(e1) * 1e3 / Ks
+    # (c) warm L2: the same layer and input every launch (its 58 MB stay in the 126 MB L2) - NOT the headline
+    gw = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gw, stream=stream):
+        for _ in range(min(chunk, 200)):
+            layer(0)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        gw.replay()
+        e0.record(stream)
+        gw.replay()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    warm_us = e0.elapsed_time(e1) * 1e3 / min(chunk, 200)
+
     # ---- e2e: host buffers in and out through the C ABI, every step ------------------------------------
     Ke = min(K, 2000)
     xh = torch.from_numpy(xbits_h.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
@@ -563,9 +601,12 @@ def run_cuda(args, sh):
         "gpu_launches": 2 * K,
         "step": "slicemoe_route_topk then slicemoe_layer, chained by programmatic dependent launch",
         "fused_step_us": fused_us,
+        "plain_stream_step_us": stream_us,
+        "warm_l2_us_per_launch": warm_us,
         "roofline": {"bound": "hbm", "kernel": "decode_layer_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "us_per_launch": kernel_us, "bytes_per_launch": bytes_per_launch},
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "us_per_launch": kernel_us, "bytes_per_launch": bytes_per_launch,
+                     "us_per_launch_median": float(np.median(per_replay)), "us_per_launch_min": float(np.min(per_replay))},
         "clocks": sampler.summary(windows),
     }
     if not args.no_cpu_baseline:
@@ -812,6 +853,11 @@ def run_stack(args):
                    "replay": "CUDA graphs of 32 tokens x 26 layers"},
         "gbs": gbs, "bytes_per_token": total_bytes / NS,
         "cache": {k: int(v) for k, v in stats.items()},
+        "cache_rates": {"msb_hit": stats["msb_hit"] / stats["requests"],
+                        "lsb_hit": stats["lsb_hit"] / max(stats["lsb_hit"] + stats["lsb_miss"], 1),
+                        "miss_bytes_over_8bit_bytes": stats["bytes_fetched"] / (stats["requests"] * (msb_b + lsb_b)),
+                        "exec_8bit": stats["high_exec"] / stats["requests"],
+                        "mean_critical_per_token_layer": float(preq_h.sum(1).mean())},
         "e2e": {"value": e2e_us, "unit": "µs/token", "h2d_bytes_per_step": NL * sh.top_k,
                 "d2h_bytes_per_step": NL * sh.top_k * 5, "steps": NE,
                 "what": "route, ids and requests to the host, cache lookup, precision list back, FFN - per layer"},
