@@ -167,6 +167,8 @@ def oracle_layer_inputs(sh, step: int):
     for j in range(sh.n_shared):
         W = synth.expert_weights(sh.seed, layer, f"shared{j}", sh.hidden, sh.shared_inter)
         shared.append({k: amat.pack_matrix(W[k], sh.group) for k in ("gate", "up", "down")})
+    if sh.shared_sigmoid_gate:
+        shared = (shared, synth.normal_f32(sh.seed, ("gate_vec", layer), (sh.hidden,), 0.02))
     return logits, x64, experts, shared
 
 
@@ -178,10 +180,13 @@ def oracle_step(sh, logits, x64, experts, shared, units=None):
     intermediate rows (rows a multiple of the group size).  The oracle's functions are called as they
     stand, on the smaller inputs."""
     from oracle import moe
+    gate_vec = None
+    if isinstance(shared, tuple):        # shared experts scaled by sigmoid(v . x)
+        shared, gate_vec = shared
     ids, w, _ = moe.route_topk(logits, sh.top_k)
     prec = moe.precision_request(w, 2.0, rank_high=RANK_HIGH)
     if units is None:
-        return moe.layer(x64, experts, ids, prec, w, shared=shared)
+        return moe.layer(x64, experts, ids, prec, w, shared=shared, shared_gate_vec=gate_vec)
     n_exp, rows = units
 
     def cut(ex, m):
@@ -198,7 +203,7 @@ def oracle_step(sh, logits, x64, experts, shared, units=None):
     ns = max(0, n_exp - nr)
     ex = {int(e): cut(experts[int(e)], min(rows, sh.inter)) for e in ids[0, :nr]}
     shd = [cut(s, min(rows, sh.shared_inter)) for s in shared[:ns]]
-    return moe.layer(x64, ex, ids[:, :nr], prec[:, :nr], w[:, :nr], shared=shd)
+    return moe.layer(x64, ex, ids[:, :nr], prec[:, :nr], w[:, :nr], shared=shd, shared_gate_vec=gate_vec)
 
 
 def blas_threads() -> int:
@@ -225,7 +230,7 @@ def cpu_baseline(sh, budget_s: float = 15.0):
             break
     med = float(np.median(times))
     return {"value": med * 1e6, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-            "sample": f"{len(times)} whole steps (route + 6 routed + {sh.n_shared} shared experts, float64 numpy), "
+            "sample": f"{len(times)} whole steps (route + {sh.top_k} routed + {sh.n_shared} shared experts, float64 numpy), "
                       f"median; packing excluded; host has {os.cpu_count()} logical cores",
             "gbs": step_bytes(sh) / med / 1e9}
 
@@ -870,6 +875,7 @@ def run_stack(args):
 
 
 def main():
+    global WORKLOAD, RANK_HIGH, METRIC, NCU_TRAFFIC_BYTES_PER_LAUNCH
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20000)
@@ -877,8 +883,9 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--layers", type=int, default=16, help="independently packed layers the steps cycle over")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "stack", "prefill"],
-                    help="the default is the headline decode layer; `stack` and `prefill` are single-GPU extras")
+    ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "qwen", "stack", "prefill"],
+                    help="the default is the headline decode layer; `qwen` is the same measurement on the Qwen1.5-MoE-"
+                         "shaped layer; `stack` and `prefill` are single-GPU extras")
     args = ap.parse_args()
     if args.workload in ("stack", "prefill") and args.impl == "cuda":
         if int(os.environ.get("WORLD_SIZE", "1")) != 1 or args.gpus != 1:
@@ -891,6 +898,10 @@ def main():
             run_stack(args)
         return
     from paper_2512_12990_b200 import synth
+    if args.workload == "qwen":
+        # config 3: 60 x 1408 experts, top-4 (the 2 best at 8 bits), one gated shared expert of 5632
+        WORKLOAD, RANK_HIGH, NCU_TRAFFIC_BYTES_PER_LAUNCH = "qwen", 2, None
+        METRIC = "us per MoE layer decode (Qwen1.5-MoE-A2.7B shape, b=1)"
     sh = synth.SHAPES[WORKLOAD]
     if args.impl == "reference":
         if args.steps == 20000 and args.warmup == 100:
