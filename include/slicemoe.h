@@ -228,8 +228,10 @@ int slicemoe_layer_static(const slicemoe_shape *shape, const slicemoe_expert *ex
  * copies x (bf16 [hidden]) and logits (float32 [E]) to the device, runs slicemoe_layer_routed
  * (bias/tau/rank_high as in slicemoe_route_topk; the precision request is used as the precision
  * list), copies y (float32 [hidden]) back and synchronises `stream`.  x_host, logits_host
- * and y_host should be pinned for the copies to be asynchronous.  Weights stay resident on the
- * device.  Staging buffers live in the workspace.
+ * and y_host should be pinned for the copies to be asynchronous.  When y_host is pinned,
+ * device-mapped host memory (cudaHostAlloc / cudaHostRegister, 16-byte aligned) the kernel writes y
+ * straight into it and no copy back is issued.  Weights stay resident on the device.  Staging
+ * buffers live in the workspace.
  */
 int slicemoe_decode_step_host(const slicemoe_shape *shape, const slicemoe_expert *experts,
                               const slicemoe_expert *shared, const float *shared_gate_vec,

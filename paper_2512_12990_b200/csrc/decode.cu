@@ -1303,12 +1303,25 @@ extern "C" int slicemoe_decode_step_host(const slicemoe_shape* shape, const slic
   float* dw = reinterpret_cast<float*>(ws + kWsStW);
   uint8_t* dprec = ws + kWsStPrec;
   float* dy = reinterpret_cast<float*>(ws + kWsStY);
+  // y_host in pinned (device-mapped) host memory: the kernel writes its 16 output rows per CTA straight
+  // into it and the copy back falls away; otherwise y goes through the staging area.
+  bool y_direct = false;
+  {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, y_host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer &&
+        (reinterpret_cast<uintptr_t>(attr.devicePointer) & 15) == 0) {
+      dy = reinterpret_cast<float*>(attr.devicePointer);
+      y_direct = true;
+    } else {
+      (void)cudaGetLastError();  // an unregistered pointer is not an error here
+    }
+  }
   SM_CUDA_TRY(cudaMemcpyAsync(dx, x_host, 2 * (size_t)shape->hidden, cudaMemcpyHostToDevice, st));
   SM_CUDA_TRY(cudaMemcpyAsync(dlogits, logits_host, 4 * (size_t)shape->n_experts, cudaMemcpyHostToDevice, st));
   rc = slicemoe_layer_routed(shape, experts, shared, shared_gate_vec, dx, 1, dlogits, bias, renorm, tau, rank_high, dids,
                              dprec, dw, dy, workspace, workspace_bytes, stream);
   if (rc != SLICEMOE_OK) return rc;
-  SM_CUDA_TRY(cudaMemcpyAsync(y_host, dy, 4 * (size_t)shape->hidden, cudaMemcpyDeviceToHost, st));
+  if (!y_direct) SM_CUDA_TRY(cudaMemcpyAsync(y_host, dy, 4 * (size_t)shape->hidden, cudaMemcpyDeviceToHost, st));
   SM_CUDA_TRY(cudaStreamSynchronize(st));
   return SLICEMOE_OK;
 }

@@ -148,6 +148,11 @@ def test_qwen_decode_layer_config():
                                 rank_high=0)
     y4 = moe.layer(x64, L.oracle_list(), ids, np.zeros_like(prec), w, shared=L.oracle_shared, shared_gate_vec=L.gate_vec)
     H.assert_close(yh.numpy(), y4[0], "qwen host step (all routed 4-bit)")
+    # pageable host buffers take the staged path (pinned y is written by the kernel directly): same bits
+    yp = torch.empty(sh.hidden, dtype=torch.float32)
+    B.slicemoe_decode_step_host(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, xh.clone(), lh.clone(), yp, L.ws,
+                                tau=2.0, rank_high=0)
+    assert torch.equal(yp, yh)
 
 
 def test_bad_expert_id_is_skipped_and_reported():
