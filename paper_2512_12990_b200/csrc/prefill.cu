@@ -147,10 +147,10 @@ __global__ void pf_gather_kernel(const uint16_t* __restrict__ x, int hidden, con
 // buffer.  No weight is ever rounded.  Every wait is bounded; a wait that runs out sets
 // SLICEMOE_STATUS_WAIT_TIMEOUT and the CTA winds down (tensor memory is freed on every path).
 constexpr int kUThreads = 576;      // warps 0-7 epilogue, 8-15 dequantisation, 16 loads, 17 MMA issue
-constexpr int kUStages = 6;
+constexpr int kUStages = 4;
 static_assert(kUStages % 2 == 0, "each dequantisation set must meet every one of its stages on every lap of the ring");
 constexpr int kUTileBytes = kPfTileM * kPfChunkK * 2;  // 16,384: the token tile of a step
-constexpr int kUScaleSlots = 16;    // ring of per-group scale rows: dequantisation runs at most 15 groups ahead of the epilogue
+constexpr int kUScaleSlots = 4;     // ring of per-item row scales: dequantisation is less than 4 items ahead of the epilogue
 constexpr int kUScaleBytes = kUScaleSlots * kPfTileB * 4;
 constexpr int kURawDepth = 4;       // steps of raw plane words each dequantisation warp keeps in flight (cp.async)
 constexpr int kURawBytes = 8 * kURawDepth * 2048;  // per warp and step: 2 blocks x 512 bytes MSB, the same of LSB
@@ -158,7 +158,7 @@ constexpr int kUXchBytes = 4 * 64 * 32 * 4;        // silu(gate) on its way from
 constexpr int kUSmemBytes =
     kUStages * kUTileBytes + kURawBytes + kUXchBytes + kUScaleBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr int kUAccCols = 256;      // two accumulators of 128 fp32 columns (tokens)
-constexpr int kUWCols = 32;         // a step's weights: 64 fp16 per row
+constexpr int kUWCols = 64;         // a step's weights: 64 fp16 per row, twice (leading part, remainder)
 constexpr int kUTmemCols = 512;     // accumulators + kUStages weight stages, rounded up to a power of two
 constexpr long long kUWaitCycles = 2000000000ll;
 
@@ -342,11 +342,11 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
   uint8_t* smem = u_smem_raw + ((1024 - (smem_u32(u_smem_raw) & 1023)) & 1023);
   uint8_t* raw_ring = smem + kUStages * kUTileBytes;
   float(*xch)[64][32] = reinterpret_cast<float(*)[64][32]>(raw_ring + kURawBytes);  // [pair][token][row]
-  float(*sc_ring)[kPfTileB] = reinterpret_cast<float(*)[kPfTileB]>(raw_ring + kURawBytes + kUXchBytes);
+  float(*row_scale)[kPfTileB] = reinterpret_cast<float(*)[kPfTileB]>(raw_ring + kURawBytes + kUXchBytes);  // [item % 4][row]
   uint64_t* bars = reinterpret_cast<uint64_t*>(raw_ring + kURawBytes + kUXchBytes + kUScaleBytes);
   uint64_t* full = bars;                    // [stage]: tokens landed (TMA) and weights stored (8 warps)
   uint64_t* empty = bars + kUStages;        // [stage]: the MMAs that read the stage have completed
-  uint64_t* acc_full = bars + 2 * kUStages;       // [2]: a group's sums are complete in the accumulator
+  uint64_t* acc_full = bars + 2 * kUStages;       // [2]: an item's sums are complete in the accumulator
   uint64_t* acc_empty = bars + 2 * kUStages + 2;  // [2]: the epilogue warps have read it
   uint64_t* xch_full = bars + 2 * kUStages + 4;   // [4]: silu(gate) of a warp pair is in shared memory
   uint64_t* xch_empty = bars + 2 * kUStages + 8;  // [4]: it has been consumed
@@ -404,13 +404,17 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
   } else if (warp == 17) {
     // ---- MMA issue: D[weight row, token] += W[weight row, k] (tensor memory) x X[token, k] (shared memory) ----
     if (lane == 0) {
-      uint32_t st = 0, ph = 0, gc = 0;  // stage, its parity, quantisation groups issued so far
+      uint32_t st = 0, ph = 0, ni = 0;  // stage, its parity, items issued so far
       uint64_t* last_empty = nullptr;
       uint32_t last_ph = 0;
       const uint64_t bd0 = umma_desc(smem_u32(smem));
-      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++ni) {
         const UItem w = u_item<PHASE>(p, item);
         const int nk = w.K / kPfChunkK;
+        const uint32_t ab = ni & 1;
+        // the accumulator must have been read out (the item before the previous one used it)
+        if (!mbar_wait(&acc_empty[ab], ((ni >> 1) & 1) ^ 1, abort_flag)) { alive = false; break; }
+        tc_fence_after();
         for (int kc = 0; kc < nk && alive; ++kc) {
           if (!mbar_wait(&full[st], ph, abort_flag)) { alive = false; break; }
           tc_fence_after();
@@ -418,26 +422,16 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
           const uint32_t a_tmem = tmem + kUAccCols + st * kUWCols;
 #pragma unroll
           for (int ks = 0; ks < kPfChunkK / 16; ++ks) {
-            // where a quantisation group starts and ends among the four k16 steps of a 64-column step
-            const bool first = G == 128 ? (ks == 0 && (kc & 1) == 0) : (G == 64 ? ks == 0 : (ks & 1) == 0);
-            const bool last = G == 128 ? (ks == 3 && (kc & 1) == 1) : (G == 64 ? ks == 3 : (ks & 1) == 1);
-            const uint32_t ab = gc & 1;
-            if (first) {
-              // the accumulator must have been read out
-              if (!mbar_wait(&acc_empty[ab], ((gc >> 1) & 1) ^ 1, abort_flag)) { alive = false; break; }
-              tc_fence_after();
-            }
-            umma_f16_ts(tmem + ab * kPfTileM, a_tmem + 8 * ks, bd + 2 * ks, first ? 0u : 1u);
-            if (last) {
-              umma_commit(&acc_full[ab]);
-              ++gc;
-            }
+            // leading part and remainder of the weights against the same tokens
+            umma_f16_ts(tmem + ab * kPfTileM, a_tmem + 8 * ks, bd + 2 * ks, (kc | ks) ? 1u : 0u);
+            umma_f16_ts(tmem + ab * kPfTileM, a_tmem + 32 + 8 * ks, bd + 2 * ks, 1u);
           }
           umma_commit(&empty[st]);
           last_empty = &empty[st];
           last_ph = ph;
           if (++st == kUStages) { st = 0; ph ^= 1; }
         }
+        if (alive) umma_commit(&acc_full[ab]);
       }
       // the last commit must have arrived before shared memory goes away
       if (alive && last_empty && !mbar_wait(last_empty, last_ph, abort_flag)) alive = false;
@@ -489,8 +483,8 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
     };
     i_open();
     for (int j = 0; j < kURawDepth; ++j) i_issue(j);
-    uint32_t st = set, ph = 0, slot = 0, it0 = 0;  // stage and parity of the warp's next step; steps before this item
-    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+    uint32_t st = set, ph = 0, slot = 0, ni = 0;  // stage and parity of the warp's next step; items so far
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++ni) {
       const UItem w = u_item<PHASE>(p, item);
       int rb;
       const slicemoe_mat& m = u_block_mat<PHASE>(w, 2 * q + blk, &rb);
@@ -499,6 +493,14 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
       const size_t meta = (size_t)rb * ngroups * 16 + g + 2 * sh;  // the row's entry of group 0
       const uint8_t* zp = m.zp + meta;
       const uint16_t* sc = m.scale + meta;
+      // The row's weights are normalised by a power of two, 2^(emax - 15) with emax the largest exponent field
+      // among the row's fp16 scales: every factor f = s 2^(15 - emax) is below 2, so |(q - zp) f| < 512 sits in
+      // the middle of fp16's range for the leading part and its remainder alike.  The epilogue multiplies the
+      // row's sums by 2^(emax - 15).
+      unsigned emax = 0;
+      for (int grp = 0; grp < ngroups; ++grp) emax = max(emax, ((unsigned)__ldg(sc + grp * 16) >> 10) & 31u);
+      const float rnorm = exp2f(15.f - (float)emax);
+      if (set == 0) row_scale[ni % kUScaleSlots][32 * q + lane] = exp2f((float)emax - 15.f);
       // zero-points and scales of the groups of the warp's next step
       int z_next[kGpc];
       uint16_t s_next[kGpc];
@@ -509,11 +511,6 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
         s_next[i] = __ldg(sc + grp * 16);
       }
       for (int kc = set; kc < nk; kc += 2) {
-        // groups of this step: item-local grp0 .. grp0 + kGpc - 1; gidx0 counts all groups this CTA has met
-        // (K is a multiple of 128, so steps and groups align)
-        const uint32_t it = it0 + kc;
-        const int grp0 = (kc * kPfChunkK) >> LG;
-        const uint32_t gidx0 = G == 128 ? (it >> 1) : (G == 64 ? it : 2 * it);
         cp_async_wait_but<kURawDepth - 1>();
         __syncwarp();
         const uint8_t* src = raw + slot * 2048 + blk * 512 + g * 64;
@@ -527,12 +524,11 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
           if (w.prec) lv = *reinterpret_cast<const uint4*>(src + 1024 + ((16 * c) ^ rsw));
           lws[4 * c] = lv.x; lws[4 * c + 1] = lv.y; lws[4 * c + 2] = lv.z; lws[4 * c + 3] = lv.w;
         }
-        __half2 off[kGpc];
-        float sf[kGpc];
+        __half2 off[kGpc], fac[kGpc];
 #pragma unroll
         for (int i = 0; i < kGpc; ++i) {
           off[i] = __half2half2(__int2half_rn(1024 + (w.prec ? z_next[i] : (z_next[i] & 0xf0))));
-          sf[i] = __half2float(__ushort_as_half(s_next[i]));
+          fac[i] = __half2half2(__float2half_rn(__half2float(__ushort_as_half(s_next[i])) * rnorm));  // exact: a power of two
         }
         if (kc + 2 < nk) {
 #pragma unroll
@@ -542,33 +538,39 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
             s_next[i] = __ldg(sc + grp * 16);
           }
         }
-        (void)grp0;
-        uint32_t r[32];  // column 8 w + 2 c + jj holds k = 16 w + 4 c + 2 jj, + 1
-#pragma unroll
-        for (int wd = 0; wd < 4; ++wd) {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const uint32_t m0 = mws[4 * c + wd] >> sh, l0 = lws[4 * c + wd] >> sh;
-            // both slices: the 8-bit code; MSB slice alone: 16 x its 4-bit code (the factor 16 of the low-bit
-            // dequantisation, exact in fp16)
-            const uint32_t qv = ((m0 & 0x0f0f0f0fu) << 4) | (l0 & 0x0f0f0f0fu);
-            // bytes -> fp16 1024 + code, minus (1024 + zero-point): the integer q - zp, exact
-            uint32_t h01 = __byte_perm(qv, 0x64646464u, 0x4140), h23 = __byte_perm(qv, 0x64646464u, 0x4342);
-            const __half2 o = off[kGpc == 2 ? (wd >> 1) : 0];
-            const __half2 w01 = __hsub2(*reinterpret_cast<__half2*>(&h01), o);
-            const __half2 w23 = __hsub2(*reinterpret_cast<__half2*>(&h23), o);
-            r[8 * wd + 2 * c] = *reinterpret_cast<const uint32_t*>(&w01);
-            r[8 * wd + 2 * c + 1] = *reinterpret_cast<const uint32_t*>(&w23);
-          }
-        }
         if (!__all_sync(0xffffffffu, mbar_wait(&empty[st], ph ^ 1, abort_flag))) { alive = false; break; }
         tc_fence_after();
-        // the row's scale of each group that starts in this step, for the epilogue (published by the arrive below)
-        if (G != 128 || (kc & 1) == 0) {
+        const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + kUAccCols + st * kUWCols;
 #pragma unroll
-          for (int i = 0; i < kGpc; ++i) sc_ring[(gidx0 + i) % kUScaleSlots][32 * q + lane] = sf[i];
+        for (int half = 0; half < 2; ++half) {
+          uint32_t rh[16], rl[16];  // column 8 (w & 1) + 2 c + jj holds k = 16 w + 4 c + 2 jj, + 1 for w = 2 half, 2 half + 1
+#pragma unroll
+          for (int wi = 0; wi < 2; ++wi) {
+            const int wd = 2 * half + wi;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const uint32_t m0 = mws[4 * c + wd] >> sh, l0 = lws[4 * c + wd] >> sh;
+              // both slices: the 8-bit code; MSB slice alone: 16 x its 4-bit code (the factor 16 of the low-bit
+              // dequantisation, exact in fp16)
+              const uint32_t qv = ((m0 & 0x0f0f0f0fu) << 4) | (l0 & 0x0f0f0f0fu);
+              // bytes -> fp16 1024 + code, minus (1024 + zero-point): the integer d = q - zp, exact
+              uint32_t h01 = __byte_perm(qv, 0x64646464u, 0x4140), h23 = __byte_perm(qv, 0x64646464u, 0x4342);
+              const __half2 o = off[kGpc == 2 ? (wd >> 1) : 0], f = fac[kGpc == 2 ? (wd >> 1) : 0];
+              const __half2 d01 = __hsub2(*reinterpret_cast<__half2*>(&h01), o);
+              const __half2 d23 = __hsub2(*reinterpret_cast<__half2*>(&h23), o);
+              // d f as an unevaluated sum of two fp16: the rounded product and, by one fused multiply-add, what
+              // the rounding dropped (at most 10 significant bits, so it is exact)
+              const __half2 p01 = __hmul2(d01, f), p23 = __hmul2(d23, f);
+              const __half2 e01 = __hfma2(d01, f, __hneg2(p01)), e23 = __hfma2(d23, f, __hneg2(p23));
+              rh[8 * wi + 2 * c] = *reinterpret_cast<const uint32_t*>(&p01);
+              rh[8 * wi + 2 * c + 1] = *reinterpret_cast<const uint32_t*>(&p23);
+              rl[8 * wi + 2 * c] = *reinterpret_cast<const uint32_t*>(&e01);
+              rl[8 * wi + 2 * c + 1] = *reinterpret_cast<const uint32_t*>(&e23);
+            }
+          }
+          tmem_st16(ta + 16 * half, rh);
+          tmem_st16(ta + 32 + 16 * half, rl);
         }
-        tmem_st32(tmem + ((uint32_t)(32 * q) << 16) + kUAccCols + st * kUWCols, r);
         tmem_st_wait();
         tc_fence_before();
         __syncwarp();
@@ -578,44 +580,39 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
         st += 2;
         if (st >= kUStages) { st -= kUStages; ph ^= 1; }
       }
-      it0 += nk;
     }
     cp_async_wait_but<0>();
   } else {
     // ---- epilogue: warp (q, hh) owns weight rows [32 q, 32 q + 32) x tokens [64 hh, 64 hh + 64) ----
     const int q = warp & 3, hh = warp >> 2;
-    uint32_t gc = 0, n_done = 0;
+    uint32_t n_done = 0;
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++n_done) {
       const UItem w = u_item<PHASE>(p, item);
-      const int ngroups = w.K >> LG;
+      const uint32_t ab = n_done & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[ab], (n_done >> 1) & 1, abort_flag))) { alive = false; break; }
+      tc_fence_after();
+      const float rs = row_scale[n_done % kUScaleSlots][32 * q + lane];  // 2^(emax - 15) of the lane's weight row
+      const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + ab * kPfTileM + 64 * hh;
       float tot[64];
-#pragma unroll
-      for (int j = 0; j < 64; ++j) tot[j] = 0.f;
-      for (int grp = 0; grp < ngroups; ++grp, ++gc) {
-        const uint32_t ab = gc & 1;
-        if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[ab], (gc >> 1) & 1, abort_flag))) { alive = false; break; }
-        tc_fence_after();
-        const float sf = sc_ring[gc % kUScaleSlots][32 * q + lane];
-        // columns 0-31, then 32-63; the accumulator is released as soon as the last load has landed
-        const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + ab * kPfTileM + 64 * hh;
+      {
         uint32_t r0[16], r1[16];
         tmem_ld16(ta, r0);
         tmem_ld16(ta + 16, r1);
         tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 16; ++j) tot[j] = fmaf(sf, __uint_as_float(r0[j]), tot[j]);
+        for (int j = 0; j < 16; ++j) tot[j] = rs * __uint_as_float(r0[j]);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) tot[16 + j] = fmaf(sf, __uint_as_float(r1[j]), tot[16 + j]);
+        for (int j = 0; j < 16; ++j) tot[16 + j] = rs * __uint_as_float(r1[j]);
         tmem_ld16(ta + 32, r0);
         tmem_ld16(ta + 48, r1);
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&acc_empty[ab]);
+        if (lane == 0) mbar_arrive(&acc_empty[ab]);  // the accumulator is free for the item after the next
 #pragma unroll
-        for (int j = 0; j < 16; ++j) tot[32 + j] = fmaf(sf, __uint_as_float(r0[j]), tot[32 + j]);
+        for (int j = 0; j < 16; ++j) tot[32 + j] = rs * __uint_as_float(r0[j]);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) tot[48 + j] = fmaf(sf, __uint_as_float(r1[j]), tot[48 + j]);
+        for (int j = 0; j < 16; ++j) tot[48 + j] = rs * __uint_as_float(r1[j]);
       }
       if (!alive) break;
       const int tok0 = w.row0 + 64 * hh;
