@@ -146,14 +146,15 @@ __global__ void pf_gather_kernel(const uint16_t* __restrict__ x, int hidden, con
 // in fp32 and add it to the running result in registers; meanwhile the next group accumulates in the other
 // buffer.  No weight is ever rounded.  Every wait is bounded; a wait that runs out sets
 // SLICEMOE_STATUS_WAIT_TIMEOUT and the CTA winds down (tensor memory is freed on every path).
-constexpr int kUThreads = 576;      // warps 0-7 epilogue, 8-15 dequantisation, 16 loads, 17 MMA issue
+constexpr int kUSets = 2;           // dequantisation sets of four warps; the steps go round them
+constexpr int kUWarpTma = 8 + 4 * kUSets, kUWarpMma = kUWarpTma + 1;
+constexpr int kUThreads = 32 * (kUWarpMma + 1);  // warps 0-7 epilogue, then the dequantisation sets, loads, MMA issue
 constexpr int kUStages = 4;
-static_assert(kUStages % 2 == 0, "each dequantisation set must meet every one of its stages on every lap of the ring");
 constexpr int kUTileBytes = kPfTileM * kPfChunkK * 2;  // 16,384: the token tile of a step
 constexpr int kUScaleSlots = 4;     // ring of per-item row scales: dequantisation is less than 4 items ahead of the epilogue
 constexpr int kUScaleBytes = kUScaleSlots * kPfTileB * 4;
-constexpr int kURawDepth = 4;       // steps of raw plane words each dequantisation warp keeps in flight (cp.async)
-constexpr int kURawBytes = 8 * kURawDepth * 2048;  // per warp and step: 2 blocks x 512 bytes MSB, the same of LSB
+constexpr int kURawDepth = 3;       // steps of raw plane words each dequantisation warp keeps in flight (cp.async)
+constexpr int kURawBytes = 4 * kUSets * kURawDepth * 2048;  // per warp and step: 2 blocks x 512 bytes MSB, the same of LSB
 constexpr int kUXchBytes = 4 * 64 * 32 * 4;        // silu(gate) on its way from the gate warps to the up warps
 constexpr int kUSmemBytes =
     kUStages * kUTileBytes + kURawBytes + kUXchBytes + kUScaleBytes + 1024 /* alignment slack */ + 256 /* barriers */;
@@ -353,7 +354,9 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kUStages + 12);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // the warp index by way of a shuffle: the compiler then knows that it is uniform across the warp, and keeps
+  // the role branches and what they compute (addresses, descriptors, counters) on the uniform datapath
+  const int tid = threadIdx.x, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), lane = tid & 31;
   if (tid == 0) {
     for (int s = 0; s < kUStages; ++s) {
       mbar_init(&full[s], 5);  // the set's four dequantisation warps and the load warp
@@ -370,7 +373,7 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 17) {
+  if (warp == kUWarpMma) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kUTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -382,7 +385,7 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
   const int n_items = u_item_count<PHASE>(p);
   bool alive = true;
 
-  if (warp == 16) {
+  if (warp == kUWarpTma) {
     // ---- token tiles: one TMA copy per step ----
     if (lane == 0) {
       uint32_t s = 0, ph = 0;
@@ -401,25 +404,26 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
         }
       }
     }
-  } else if (warp == 17) {
+  } else if (warp == kUWarpMma) {
     // ---- MMA issue: D[weight row, token] += W[weight row, k] (tensor memory) x X[token, k] (shared memory) ----
-    if (lane == 0) {
-      uint32_t st = 0, ph = 0, ni = 0;  // stage, its parity, items issued so far
-      uint64_t* last_empty = nullptr;
-      uint32_t last_ph = 0;
-      const uint64_t bd0 = umma_desc(smem_u32(smem));
-      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++ni) {
-        const UItem w = u_item<PHASE>(p, item);
-        const int nk = w.K / kPfChunkK;
-        const uint32_t ab = ni & 1;
-        // the accumulator must have been read out (the item before the previous one used it)
-        if (!mbar_wait(&acc_empty[ab], ((ni >> 1) & 1) ^ 1, abort_flag)) { alive = false; break; }
+    // The whole warp walks the loop (waits included) so that its bookkeeping stays uniform; lane 0 issues.
+    uint32_t st = 0, ph = 0, ni = 0;  // stage, its parity, items issued so far
+    uint64_t* last_empty = nullptr;
+    uint32_t last_ph = 0;
+    const uint64_t bd0 = umma_desc(smem_u32(smem));
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++ni) {
+      const UItem w = u_item<PHASE>(p, item);
+      const int nk = w.K / kPfChunkK;
+      const uint32_t ab = ni & 1;
+      // the accumulator must have been read out (the item before the previous one used it)
+      if (!__all_sync(0xffffffffu, mbar_wait(&acc_empty[ab], ((ni >> 1) & 1) ^ 1, abort_flag))) { alive = false; break; }
+      tc_fence_after();
+      for (int kc = 0; kc < nk; ++kc) {
+        if (!__all_sync(0xffffffffu, mbar_wait(&full[st], ph, abort_flag))) { alive = false; break; }
         tc_fence_after();
-        for (int kc = 0; kc < nk && alive; ++kc) {
-          if (!mbar_wait(&full[st], ph, abort_flag)) { alive = false; break; }
-          tc_fence_after();
-          const uint64_t bd = bd0 + (uint64_t)(st * (kUTileBytes >> 4));
-          const uint32_t a_tmem = tmem + kUAccCols + st * kUWCols;
+        const uint64_t bd = bd0 + (uint64_t)(st * (kUTileBytes >> 4));
+        const uint32_t a_tmem = tmem + kUAccCols + st * kUWCols;
+        if (lane == 0) {
 #pragma unroll
           for (int ks = 0; ks < kPfChunkK / 16; ++ks) {
             // leading part and remainder of the weights against the same tokens
@@ -427,15 +431,18 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
             umma_f16_ts(tmem + ab * kPfTileM, a_tmem + 32 + 8 * ks, bd + 2 * ks, 1u);
           }
           umma_commit(&empty[st]);
-          last_empty = &empty[st];
-          last_ph = ph;
-          if (++st == kUStages) { st = 0; ph ^= 1; }
         }
-        if (alive) umma_commit(&acc_full[ab]);
+        __syncwarp();
+        last_empty = &empty[st];
+        last_ph = ph;
+        if (++st == kUStages) { st = 0; ph ^= 1; }
       }
-      // the last commit must have arrived before shared memory goes away
-      if (alive && last_empty && !mbar_wait(last_empty, last_ph, abort_flag)) alive = false;
+      if (!alive) break;
+      if (lane == 0) umma_commit(&acc_full[ab]);
+      __syncwarp();
     }
+    // the last commit must have arrived before shared memory goes away
+    if (alive && last_empty && !__all_sync(0xffffffffu, mbar_wait(last_empty, last_ph, abort_flag))) alive = false;
   } else if (warp >= 8) {
     // ---- dequantisation: two sets of four warps take the 64-column steps in turn (set = step parity); thread
     // (q, lane) of a set owns weight row 32 q + lane and stores the row's 64 values of the step into the
@@ -449,6 +456,9 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
     // after a warp barrier every lane reads the four pieces of its row.
     uint8_t* raw = raw_ring + (warp - 8) * (kURawDepth * 2048);
     const int wr_piece = (lane ^ (lane >> 3)) * 16;  // plane lane l = 4 g' + c: low two bits XOR (g' >> 1)
+    // Step c of the CTA (counted over all its items) belongs to set c mod kUSets and to stage c mod kUStages.
+    auto first_kc = [&](uint32_t base) { return (int)((set + kUSets - base % kUSets) % kUSets); };
+    uint32_t i_base = 0;  // steps of the items before the one the copies are in
     int i_item = blockIdx.x, i_kc = set, i_nk = 0;
     const uint8_t *i_mp = nullptr, *i_lp = nullptr;
     bool i_prec = false;
@@ -472,10 +482,11 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
           cp_async16(dst + 1024, i_lp + o);
           cp_async16(dst + 1536, i_lp + o1);
         }
-        i_kc += 2;
+        i_kc += kUSets;
         if (i_kc >= i_nk) {
+          i_base += i_nk;
           i_item += gridDim.x;
-          i_kc = set;
+          i_kc = first_kc(i_base);
           i_open();
         }
       }
@@ -483,7 +494,7 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
     };
     i_open();
     for (int j = 0; j < kURawDepth; ++j) i_issue(j);
-    uint32_t st = set, ph = 0, slot = 0, ni = 0;  // stage and parity of the warp's next step; items so far
+    uint32_t base = 0, slot = 0, ni = 0;  // steps of the items so far; ring slot of the raw words; items so far
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++ni) {
       const UItem w = u_item<PHASE>(p, item);
       int rb;
@@ -502,15 +513,17 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
       const float rnorm = exp2f(15.f - (float)emax);
       if (set == 0) row_scale[ni % kUScaleSlots][32 * q + lane] = exp2f((float)emax - 15.f);
       // zero-points and scales of the groups of the warp's next step
+      const int kc0 = first_kc(base);
       int z_next[kGpc];
       uint16_t s_next[kGpc];
 #pragma unroll
       for (int i = 0; i < kGpc; ++i) {
-        const int grp = ((set * kPfChunkK) >> LG) + i;
+        const int grp = ((kc0 * kPfChunkK) >> LG) + i;
         z_next[i] = __ldg(zp + grp * 16);
         s_next[i] = __ldg(sc + grp * 16);
       }
-      for (int kc = set; kc < nk; kc += 2) {
+      for (int kc = kc0; kc < nk; kc += kUSets) {
+        const uint32_t st = (base + kc) % kUStages, ph = ((base + kc) / kUStages) & 1;
         cp_async_wait_but<kURawDepth - 1>();
         __syncwarp();
         const uint8_t* src = raw + slot * 2048 + blk * 512 + g * 64;
@@ -530,10 +543,10 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
           off[i] = __half2half2(__int2half_rn(1024 + (w.prec ? z_next[i] : (z_next[i] & 0xf0))));
           fac[i] = __half2half2(__float2half_rn(__half2float(__ushort_as_half(s_next[i])) * rnorm));  // exact: a power of two
         }
-        if (kc + 2 < nk) {
+        if (kc + kUSets < nk) {
 #pragma unroll
           for (int i = 0; i < kGpc; ++i) {
-            const int grp = (((kc + 2) * kPfChunkK) >> LG) + i;
+            const int grp = (((kc + kUSets) * kPfChunkK) >> LG) + i;
             z_next[i] = __ldg(zp + grp * 16);
             s_next[i] = __ldg(sc + grp * 16);
           }
@@ -577,9 +590,8 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
         if (lane == 0) mbar_arrive(&full[st]);
         i_issue(slot);  // after the step's words were consumed by every lane: the slot is free
         if (++slot == kURawDepth) slot = 0;
-        st += 2;
-        if (st >= kUStages) { st -= kUStages; ph ^= 1; }
       }
+      base += nk;
     }
     cp_async_wait_but<0>();
   } else {
@@ -647,7 +659,7 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 17) {
+  if (warp == kUWarpMma) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kUTmemCols) : "memory");
   }
