@@ -714,7 +714,7 @@ def run_prefill(args):
         "metric": "prefill TFLOP/s of one MoE layer (Qwen1.5-MoE shape, 2048 tokens); share of the tensor-core peak",
         "value": tf, "unit": "TFLOP/s", "n_gpus": 1, "steps": K, "warmup": W, "ms_per_step": ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "fp16 x integer codes held in fp16, f32 accumulate", "data": "synthetic",
+        "dtype": "fp16 tokens x weights as exact sums of two fp16, f32 accumulate", "data": "synthetic",
         "config": {"workload": "qwen_prefill", "tokens": T, "hidden": sh.hidden, "inter": sh.inter, "experts": sh.n_experts,
                    "top_k": sh.top_k, "shared_inter": sh.shared_inter, "group": sh.group,
                    "precision_mix": "experts of even popularity rank at 4-bit, odd rank at 8-bit; shared 8-bit",

@@ -244,9 +244,11 @@ int slicemoe_decode_step_host(const slicemoe_shape *shape, const slicemoe_expert
  * every expert of a layer, so the expert FFN becomes a grouped dense contraction; Section 5.3:
  * after prefill each expert is held, and here run, at the precision its cached slices allow).
  * Tokens are grouped by expert on the device; per 128-token tile the weight tile is dequantised
- * from the nibble planes to fp16 in shared memory - s*(q - zp), or 16*s*(q_msb - (zp >> 4)) for an
- * MSB-only expert - and contracted on the tensor cores with fp32 accumulation; h is rounded to
- * fp16 between the two projections (relative error 2^-11, inside the FFN tolerance).  Each
+ * from the nibble planes - s*(q - zp), or 16*s*(q_msb - (zp >> 4)) for an MSB-only expert - into
+ * tensor memory as the exact sum of two fp16 numbers per weight (no weight is rounded) and
+ * contracted on the tensor cores (tcgen05, fp16 x fp16 with fp32 accumulation); tokens enter as
+ * fp16 (exact for bf16 inputs in fp16's normal range) and h is rounded to fp16 between the two
+ * projections (relative error 2^-11, inside the FFN tolerance).  Each
  * (token, expert) pair gets its own fp32 result row and y[t] sums them in list order (routed
  * slots 0..k-1, then the shared experts), so y is bit-reproducible run to run.
  *   x            device bf16 [T, hidden]

@@ -9,10 +9,11 @@
 //   3. grouped GEMM 1: per tile  H = silu(X Wg^T) * (X Wu^T)  (fp16 out);
 //   4. grouped GEMM 2: per tile  Yrow = H Wd^T  (fp32 out, one row per (token, expert) pair);
 //   5. combine: y[t] = sum_j w[t,j] Yrow[pos(t,j)] + shared experts, in list order (deterministic).
-// In both GEMMs the weight tile is dequantised on the fly from the nibble planes into fp16 in shared
-// memory - s * (q - zp) from both slices, 16 s * (q_msb - (zp >> 4)) from the MSB slice alone - and fed
-// to the tensor cores (mma.sync m16n8k16, fp16 x fp16 -> fp32).  fp16 rather than bf16: a dequantised
-// weight needs 11 significant bits to stay inside the parity tolerance, bf16 has 8.
+// In both GEMMs the weight tile is dequantised on the fly from the nibble planes - s * (q - zp) from both
+// slices, 16 s * (q_msb - (zp >> 4)) from the MSB slice alone - straight into tensor memory and multiplied on
+// the 5th-generation tensor cores (tcgen05.mma, fp16 x fp16 -> fp32).  A dequantised weight needs about 20
+// significant bits, fp16 holds 11: every weight is therefore kept as the exact sum of two fp16 numbers and
+// multiplied in two MMAs.
 #include <cuda.h>  // CUtensorMap (types only; the encoder is fetched through the runtime)
 #include <cuda_fp16.h>
 
@@ -137,15 +138,18 @@ __global__ void pf_gather_kernel(const uint16_t* __restrict__ x, int hidden, con
 // product D[weight row, token].  Per 64-column step of the contraction:
 //   - the load warp brings the token tile (rows of x or h, fp16) into shared memory with one TMA tiled copy,
 //     128-byte swizzle: the B operand;
-//   - eight dequantisation warps turn the nibble planes and zero-points into the INTEGER q - zp (or
-//     16 (q_msb - (zp >> 4))), which fp16 holds exactly, and store it straight into tensor memory with
-//     tcgen05.st: the A operand, one weight row per lane.  Weights never pass through shared memory as fp16;
-//   - one thread issues four tcgen05.mma (M 128, N 128, K 16) that accumulate in tensor memory.
-// At the end of every quantisation group the accumulator (one of two, 128 columns each) is handed to eight
-// epilogue warps, which read it with tcgen05.ld, scale it by the group's fp16 scale of the lane's weight row
-// in fp32 and add it to the running result in registers; meanwhile the next group accumulates in the other
-// buffer.  No weight is ever rounded.  Every wait is bounded; a wait that runs out sets
-// SLICEMOE_STATUS_WAIT_TIMEOUT and the CTA winds down (tensor memory is freed on every path).
+//   - the dequantisation warps (sets of four, taking the steps in turn) build from the nibble planes and
+//     zero-points the integer d = q - zp (or 16 (q_msb - (zp >> 4))), exact in fp16, and multiply it by the
+//     group's scale normalised by a power of two per weight row: the product is kept as p + e with p the
+//     rounded fp16 product and e = fma(d, f, -p) the exact remainder, and both halves go straight into tensor
+//     memory with tcgen05.st: the A operands, one weight row per lane.  Weights never pass through shared
+//     memory as fp16;
+//   - the MMA warp issues eight tcgen05.mma (M 128, N 128, K 16): leading parts and remainders against the
+//     same tokens, all accumulating into one of two fp32 accumulators in tensor memory.
+// When an item's contraction is complete its accumulator is handed to eight epilogue warps, which read it with
+// tcgen05.ld and multiply each row by its power of two; meanwhile the next item accumulates in the other
+// buffer.  No weight is ever rounded: p + e equals s 2^n (q - zp) exactly.  Every wait is bounded; a wait that
+// runs out sets SLICEMOE_STATUS_WAIT_TIMEOUT and the CTA winds down (tensor memory is freed on every path).
 constexpr int kUSets = 2;           // dequantisation sets of four warps; the steps go round them
 constexpr int kUWarpTma = 8 + 4 * kUSets, kUWarpMma = kUWarpTma + 1;
 constexpr int kUThreads = 32 * (kUWarpMma + 1);  // warps 0-7 epilogue, then the dequantisation sets, loads, MMA issue
@@ -444,9 +448,9 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
     // the last commit must have arrived before shared memory goes away
     if (alive && last_empty && !__all_sync(0xffffffffu, mbar_wait(last_empty, last_ph, abort_flag))) alive = false;
   } else if (warp >= 8) {
-    // ---- dequantisation: two sets of four warps take the 64-column steps in turn (set = step parity); thread
-    // (q, lane) of a set owns weight row 32 q + lane and stores the row's 64 values of the step into the
-    // stage's tensor-memory columns ----
+    // ---- dequantisation: sets of four warps take the 64-column steps in turn; thread (q, lane) of a set owns
+    // weight row 32 q + lane and stores the row's 64 values of the step, as leading parts and remainders,
+    // into the stage's tensor-memory columns ----
     const int q = warp & 3, set = (warp - 8) >> 2;
     const int blk = lane >> 4, g = lane & 7, sh = ((lane >> 3) & 1) * 4;  // row = 16 (2 q + blk) + g + 8 (sh / 4)
     constexpr int kGpc = G == 32 ? 2 : 1;  // quantisation groups in a step
