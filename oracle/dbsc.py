@@ -118,6 +118,14 @@ class SliceCache:
             st["win_bytes_full"] += self.msb_bytes + self.lsb_bytes
         return prec, msb_hit, lsb_hit, fetched
 
+    def install(self, msb_order, lsb_order):
+        """Replaces the content: (layer, expert) lists with the next victim first (the state a cache warmup
+        leaves behind).  Statistics are untouched."""
+        self.msb = OrderedDict((tuple(k), None) for k in msb_order)
+        self.lsb = OrderedDict((tuple(k), None) for k in lsb_order)
+        self.used = len(self.msb) * self.msb_bytes + len(self.lsb) * self.lsb_bytes
+        assert self.used <= self.capacity
+
     def contains(self, layer: int, expert: int):
         key = (layer, expert)
         return key in self.msb, key in self.lsb

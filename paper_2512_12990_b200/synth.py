@@ -158,3 +158,18 @@ def decode_trace_logits(seed: int, n_steps: int, n_layers: int, E: int, s: float
             else:
                 out[t, l] = fresh[t]
     return out
+
+
+def prefill_trace_logits(seed: int, n_tokens: int, n_layers: int, E: int, s: float = 1.1) -> np.ndarray:
+    """Router logits of a prompt that precedes the decode run of decode_trace_logits: float32
+    [n_layers, n_tokens, E].  Per layer the Zipf(s) popularity sits on the SAME expert permutation as
+    the decode trace (experts that are hot in prefill stay hot in early decode), the Gumbel noise
+    is drawn from a stream of its own."""
+    out = np.empty((n_layers, n_tokens, E), dtype=np.float32)
+    for l in range(n_layers):
+        perm = rng(seed, "trace", l).permutation(E)   # the first draw of the decode trace's stream
+        logp = _zipf_logp(E, s, perm)
+        u = rng(seed, "prefill-trace", l).random(size=(n_tokens, E), dtype=np.float64)
+        u = np.clip(u, 1e-300, 1.0 - 1e-16)
+        out[l] = (logp[None, :] - np.log(-np.log(u))).astype(np.float32)
+    return out
