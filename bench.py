@@ -731,6 +731,55 @@ def run_prefill(args):
     print(json.dumps(out), flush=True)
 
 
+def warmup_comparison(B, synth, sh, NL, ids_h, preq_h, cap, msb_b, lsb_b, tau, dev, prompt_tokens=1024, steps=(4, 32)):
+    """Predictive Cache Warmup against the naive initial cache states of Section 4.3: bytes the host cache has
+    to fetch in the first decode steps after a prompt whose routing shares the decode trace's per-layer expert
+    popularity.  The prompt is routed on the device; the cache bookkeeping is host code."""
+    import torch
+    pl = synth.prefill_trace_logits(sh.seed, prompt_tokens, NL, sh.n_experts)
+    p_ids, p_w, _ = B.slicemoe_route_topk(torch.from_numpy(pl.reshape(NL * prompt_tokens, sh.n_experts)).to(dev), sh.top_k)
+    torch.cuda.synchronize()
+    p_ids = p_ids.cpu().numpy().reshape(NL, prompt_tokens, sh.top_k)
+    p_w = p_w.cpu().numpy().reshape(NL, prompt_tokens, sh.top_k)
+
+    def warm():
+        c = B.Dbsc(cap, msb_b, lsb_b)
+        for l in range(NL):
+            c.prefill_layer(l, p_ids[l], p_w[l], sh.n_experts, tau)
+        c.prefill_end()
+        return c
+
+    def last_layers():                       # prefill without a policy: plain LRU, the last layers survive
+        c = B.Dbsc(cap, msb_b, lsb_b)
+        for l in range(NL):
+            for e in np.unique(p_ids[l]):
+                c.request(0, l, int(e), True)
+        return c
+
+    def random_keep():
+        c = B.Dbsc(cap, msb_b, lsb_b)
+        used = [(l, int(e)) for l in range(NL) for e in np.unique(p_ids[l])]
+        g = synth.rng(sh.seed, "warmup-random")
+        for i in g.permutation(len(used))[: cap // (msb_b + lsb_b)]:
+            c.request(0, used[i][0], used[i][1], True)
+        return c
+
+    out = {"prompt_tokens": prompt_tokens, "unit": "MB fetched in the first decode steps (26 layers)"}
+    for name, make in [("pcw", warm), ("empty", lambda: B.Dbsc(cap, msb_b, lsb_b)), ("last_layers", last_layers),
+                       ("random", random_keep)]:
+        c = make()
+        base = c.stats()["bytes_fetched"]
+        row, done = {}, 0
+        for n in steps:
+            for s in range(done, n):
+                for l in range(NL):
+                    c.assign(s, l, ids_h[s * NL + l], preq_h[s * NL + l])
+            done = n
+            row[f"first_{n}_steps"] = round((c.stats()["bytes_fetched"] - base) / 1e6, 1)
+        out[name] = row
+    return out
+
+
 def run_stack(args):
     """The 26-layer decode stack over a 256-step routing trace with the host slice cache at 30% capacity:
     microseconds per token for the 26 expert FFNs with precision lists resident (value) and with the cache in the
@@ -863,6 +912,7 @@ def run_stack(args):
                         "miss_bytes_over_8bit_bytes": stats["bytes_fetched"] / (stats["requests"] * (msb_b + lsb_b)),
                         "exec_8bit": stats["high_exec"] / stats["requests"],
                         "mean_critical_per_token_layer": float(preq_h.sum(1).mean())},
+        "cache_warmup": warmup_comparison(B, synth, sh, NL, ids_h, preq_h, cap, msb_b, lsb_b, TAU, dev),
         "e2e": {"value": e2e_us, "unit": "µs/token", "h2d_bytes_per_step": NL * sh.top_k,
                 "d2h_bytes_per_step": NL * sh.top_k * 5, "steps": NE,
                 "what": "route, ids and requests to the host, cache lookup, precision list back, FFN - per layer"},

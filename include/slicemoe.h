@@ -304,6 +304,26 @@ int slicemoe_dbsc_stats(const slicemoe_dbsc *c, int64_t *out);
 /* 1/0 presence of the two slices of (layer, expert). */
 int slicemoe_dbsc_contains(const slicemoe_dbsc *c, int layer, int expert, int *has_msb, int *has_lsb);
 
+/*
+ * Predictive Cache Warmup (Section 4.3): the cache is reshaped while a prompt is prefilled, so that decode
+ * starts with the slices it is likely to ask for.  Call slicemoe_dbsc_prefill_layer once per layer, in the
+ * order prefill visits them, with the layer's routing result, then slicemoe_dbsc_prefill_end.
+ *   ids, scores  host [n_pairs] (= tokens x top-k, any order): selected expert and its gating score
+ *   tau          the threshold that makes an expert critical in decode
+ * Per expert the call takes the number of pairs (access frequency) and the mean score (double sum in list
+ * order / count).  Every expert with frequency > 0 gets its MSB slice into the cache, and its LSB slice if
+ * its mean score >= tau.  While the content exceeds the capacity, LSB slices are dropped in ascending
+ * (score, frequency, layer, expert) order, then MSB slices in ascending (frequency, score, layer, expert)
+ * order; slices that were cached before the prompt (no statistics) go before any of the prompt's, LSB
+ * then MSB.  prefill_end re-orders
+ * both lists by the same keys (the most frequent MSB slice becomes the most recently used) and forgets the
+ * statistics.  Hit/miss counters are not touched: prefill loads every expert it uses anyway (Section 3).
+ * Errors: INVALID_ARG (null, negative layer or count, an id outside [0, n_experts)), NOMEM.
+ */
+int slicemoe_dbsc_prefill_layer(slicemoe_dbsc *c, int layer, const int32_t *ids, const float *scores,
+                                int64_t n_pairs, int n_experts, double tau);
+int slicemoe_dbsc_prefill_end(slicemoe_dbsc *c);
+
 #ifdef __cplusplus
 }
 #endif

@@ -31,6 +31,7 @@ EXPORTS = (
     "slicemoe_decode_step_host", "slicemoe_layer_static", "slicemoe_layer_routed", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
     "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
     "slicemoe_dbsc_assign", "slicemoe_dbsc_stats", "slicemoe_dbsc_contains",
+    "slicemoe_dbsc_prefill_layer", "slicemoe_dbsc_prefill_end",
 )
 
 
@@ -110,6 +111,8 @@ def lib() -> ctypes.CDLL:
     L.slicemoe_dbsc_assign.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_void_p]
     L.slicemoe_dbsc_stats.argtypes = [c_void_p, POINTER(c_int64)]
     L.slicemoe_dbsc_contains.argtypes = [c_void_p, c_int, c_int, POINTER(c_int), POINTER(c_int)]
+    L.slicemoe_dbsc_prefill_layer.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int64, c_int, c_double]
+    L.slicemoe_dbsc_prefill_end.argtypes = [c_void_p]
     _lib = L
     return L
 
@@ -391,6 +394,20 @@ class Dbsc:
         buf = (c_int64 * DBSC_NSTATS)()
         _check(lib().slicemoe_dbsc_stats(self._h, buf), "slicemoe_dbsc_stats")
         return dict(zip(DBSC_STAT_NAMES, list(buf)))
+
+    def prefill_layer(self, layer: int, ids, scores, n_experts: int, tau: float):
+        """Predictive cache warmup, one prefilled layer: ids / scores numpy [T, k] (the layer's routing result)."""
+        import numpy as np
+        ids = np.ascontiguousarray(ids, dtype=np.int32)
+        scores = np.ascontiguousarray(scores, dtype=np.float32)
+        if ids.shape != scores.shape:
+            raise SliceMoEError(E_INVALID_ARG, "slicemoe_dbsc_prefill_layer")
+        rc = lib().slicemoe_dbsc_prefill_layer(self._h, layer, ids.ctypes.data_as(c_void_p),
+                                               scores.ctypes.data_as(c_void_p), ids.size, n_experts, float(tau))
+        _check(rc, "slicemoe_dbsc_prefill_layer")
+
+    def prefill_end(self):
+        _check(lib().slicemoe_dbsc_prefill_end(self._h), "slicemoe_dbsc_prefill_end")
 
     def contains(self, layer: int, expert: int):
         a, b = c_int(0), c_int(0)

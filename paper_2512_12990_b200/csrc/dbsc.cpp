@@ -3,10 +3,18 @@
 // Two intrusive orderings over cached slices: MSB slices in LRU order, LSB slices in insertion
 // order.  Eviction always drains the LSB queue (oldest first) before touching the MSB list (least
 // recently used first).  Keys are (layer, expert); one cache serves all layers.
+//
+// Predictive Cache Warmup (Section 4.3): while a prompt is prefilled layer by layer the cache takes the
+// slices of every expert the layer used and, whenever it overflows, drops the LSB slice with the lowest
+// gating score, or - once no LSB slice is left - the MSB slice with the lowest prefill access frequency.
+// At the end of prefill both orderings are rebuilt from the accumulated statistics.
+#include <algorithm>
 #include <cstdint>
 #include <list>
 #include <new>
+#include <tuple>
 #include <unordered_map>
+#include <vector>
 
 #include "slicemoe.h"
 
@@ -28,6 +36,11 @@ struct Queue {
   void touch(uint64_t k) {  // move to the most-recently-used end
     auto it = where.find(k);
     order.splice(order.end(), order, it->second);
+  }
+  void erase(uint64_t k) {
+    auto it = where.find(k);
+    order.erase(it->second);
+    where.erase(it);
   }
   // Removes the first entry that is not `protect`; false if there is none.
   bool evict_one(uint64_t protect) {
@@ -51,6 +64,70 @@ struct slicemoe_dbsc {
   Queue msb, lsb;
   int64_t requests, msb_hit, msb_miss, lsb_hit, lsb_miss, lsb_skipped, bytes_fetched, high_exec, low_exec,
       win_fetched, win_full;
+  struct Hotness { int64_t freq; double score; };  // prompt tokens routed to the expert; their mean gating score
+  std::unordered_map<uint64_t, Hotness> hot;       // statistics of the prefill in progress
+
+  // Eviction keys of Section 4.3; a slice without statistics (left from before the prompt) goes first.
+  std::tuple<double, int64_t, uint64_t> lsb_rank(uint64_t k) const {
+    auto it = hot.find(k);
+    return it == hot.end() ? std::make_tuple(-1.0, int64_t(-1), k) : std::make_tuple(it->second.score, it->second.freq, k);
+  }
+  std::tuple<int64_t, double, uint64_t> msb_rank(uint64_t k) const {
+    auto it = hot.find(k);
+    return it == hot.end() ? std::make_tuple(int64_t(-1), -1.0, k) : std::make_tuple(it->second.freq, it->second.score, k);
+  }
+
+  void prefill_layer(int layer, const std::vector<int64_t>& freq, const std::vector<double>& sum, double tau) {
+    for (size_t e = 0; e < freq.size(); ++e) {
+      if (freq[e] <= 0) continue;
+      const uint64_t key = make_key(layer, static_cast<int>(e));
+      const double score = sum[e] / static_cast<double>(freq[e]);
+      hot[key] = Hotness{freq[e], score};
+      if (!msb.has(key)) {
+        msb.push_back(key);
+        used += msb_bytes;
+      }
+      if (score >= tau && !lsb.has(key)) {
+        lsb.push_back(key);
+        used += lsb_bytes;
+      }
+    }
+    if (used <= capacity) return;
+    // victims in order: slices from before the prompt (LSB, then MSB), then the prompt's LSB slices by score,
+    // then its MSB slices by frequency
+    std::vector<uint64_t> lv(lsb.order.begin(), lsb.order.end()), mv(msb.order.begin(), msb.order.end());
+    std::sort(lv.begin(), lv.end(), [&](uint64_t a, uint64_t b) { return lsb_rank(a) < lsb_rank(b); });
+    std::sort(mv.begin(), mv.end(), [&](uint64_t a, uint64_t b) { return msb_rank(a) < msb_rank(b); });
+    size_t li = 0, mi = 0;
+    for (; li < lv.size() && !hot.count(lv[li]) && used > capacity; ++li) {
+      lsb.erase(lv[li]);
+      used -= lsb_bytes;
+    }
+    for (; mi < mv.size() && !hot.count(mv[mi]) && used > capacity; ++mi) {
+      msb.erase(mv[mi]);
+      used -= msb_bytes;
+    }
+    for (; li < lv.size() && used > capacity; ++li) {
+      lsb.erase(lv[li]);
+      used -= lsb_bytes;
+    }
+    for (; mi < mv.size() && used > capacity; ++mi) {
+      msb.erase(mv[mi]);
+      used -= msb_bytes;
+    }
+  }
+
+  void prefill_end() {
+    std::vector<uint64_t> lv(lsb.order.begin(), lsb.order.end()), mv(msb.order.begin(), msb.order.end());
+    std::sort(lv.begin(), lv.end(), [&](uint64_t a, uint64_t b) { return lsb_rank(a) < lsb_rank(b); });
+    std::sort(mv.begin(), mv.end(), [&](uint64_t a, uint64_t b) { return msb_rank(a) < msb_rank(b); });
+    Queue nl, nm;
+    for (uint64_t k : lv) nl.push_back(k);
+    for (uint64_t k : mv) nm.push_back(k);
+    lsb = std::move(nl);
+    msb = std::move(nm);
+    hot.clear();
+  }
 
   bool make_room(int64_t need, uint64_t protect) {
     if (need > capacity) return false;
@@ -179,5 +256,34 @@ extern "C" int slicemoe_dbsc_contains(const slicemoe_dbsc* c, int layer, int exp
   const uint64_t key = make_key(layer, expert);
   if (has_msb) *has_msb = c->msb.has(key) ? 1 : 0;
   if (has_lsb) *has_lsb = c->lsb.has(key) ? 1 : 0;
+  return SLICEMOE_OK;
+}
+
+extern "C" int slicemoe_dbsc_prefill_layer(slicemoe_dbsc* c, int layer, const int32_t* ids, const float* scores,
+                                           int64_t n_pairs, int n_experts, double tau) {
+  if (!c || !ids || !scores || layer < 0 || n_pairs < 0 || n_experts <= 0) return SLICEMOE_E_INVALID_ARG;
+  for (int64_t i = 0; i < n_pairs; ++i)
+    if (ids[i] < 0 || ids[i] >= n_experts) return SLICEMOE_E_INVALID_ARG;
+  try {
+    std::vector<int64_t> freq(n_experts, 0);
+    std::vector<double> sum(n_experts, 0.0);
+    for (int64_t i = 0; i < n_pairs; ++i) {  // in list order: the sums are reproducible
+      ++freq[ids[i]];
+      sum[ids[i]] += static_cast<double>(scores[i]);
+    }
+    c->prefill_layer(layer, freq, sum, tau);
+  } catch (...) {
+    return SLICEMOE_E_NOMEM;
+  }
+  return SLICEMOE_OK;
+}
+
+extern "C" int slicemoe_dbsc_prefill_end(slicemoe_dbsc* c) {
+  if (!c) return SLICEMOE_E_INVALID_ARG;
+  try {
+    c->prefill_end();
+  } catch (...) {
+    return SLICEMOE_E_NOMEM;
+  }
   return SLICEMOE_OK;
 }
