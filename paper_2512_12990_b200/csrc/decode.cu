@@ -57,6 +57,8 @@ constexpr int kUnitBytes = kPlaneUnitBytes + kScaleUnitBytes + kZpUnitBytes;  //
 constexpr int kMaxSlots = SLICEMOE_MAX_TOP_K + SLICEMOE_MAX_SHARED;
 constexpr int kMaxHidden = 4096;
 constexpr int kHCap = 12288;  // sum of intermediate widths over all slots of a layer
+constexpr int kMaxMine = 32;   // phase-2 chunks one consumer group can have: (slots + kHCap / kChunkK) chunks per
+                               // output row block, at most 4 row blocks per CTA, shared by 4 groups
 constexpr unsigned long long kWaitCycles = 4000000000ull;  // ~2 s: every device-side wait is bounded
 
 // ---- workspace --------------------------------------------------------------------------------
@@ -148,7 +150,8 @@ struct SmemLayout {
   static constexpr int hinv = xsumw + (kMaxHidden / 32) * 8;  // float [kHCap/128]: 2^-e of each 128-block of h
   static constexpr int xinv = hinv + (kHCap / 128) * 4;       // float [kMaxHidden/128]
   static constexpr int partial = xinv + (kMaxHidden / 128) * 4;  // float2 [warps][16]
-  static constexpr int slots = partial + kConsumerWarps * 16 * 2 * 4;
+  static constexpr int p2list = partial + kConsumerWarps * 16 * 2 * 4;  // uint2 [warps][kMaxMine]: a warp's phase-2 chunks
+  static constexpr int slots = p2list + kConsumerWarps * kMaxMine * 8;
   static constexpr int plan = slots + kMaxSlots * (int)sizeof(Slot);
   static constexpr int bars = (plan + (int)sizeof(Plan) + 15) & ~15;  // uint64 barriers
   static constexpr int nbars = 2 * kUnits + kGroups * kFull2PerGroup + kUnits2 + 2 * kGroups + 5;
@@ -519,49 +522,75 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
   if (lane == 0) mbar_arrive(bars + 8 * Bars::p1_done);  // this warp no longer reads phase-1 units
   if (plan.count2 == 0) return;
 
+  // ---- while the grid barrier is pending: list this group's phase-2 chunks (the walk over all output row
+  // blocks, slots and chunks costs more than consuming the group's own chunks, so it is done ahead of time) ----
+  uint2* mylist = reinterpret_cast<uint2*>(smem + SmemLayout::p2list) + warp * kMaxMine;
+  int nmine = 0;
+  {
+    const int chunks2 = plan.p2c[plan.nslots];
+    const int half = plan.nunits2 / kProducers;  // units of one producer
+    int xp = 0;                                   // units this group's producer has handed out so far
+    for (int m = 0; m < plan.count2; ++m) {
+      for (int j = 0; j < plan.nslots; ++j) {
+        const int nchj = plan.p2c[j + 1] - plan.p2c[j];
+        const int wu = slots[j].prec ? 2 : 1;
+        for (int kc = 0; kc < nchj; ++kc) {
+          const int c = m * chunks2 + plan.p2c[j] + kc;  // chunk number within the phase
+          if (c % kProducers != prod) continue;
+          const int x0 = xp;
+          xp += wu;
+          if (c % kGroups != group) continue;
+          const int ig = c / kGroups;  // this group's ordinal of the chunk
+          if (lane == 0 && nmine < kMaxMine) {
+            // slot, chunk of the slot, row block, rotation of the warps | the chunk's units, full barrier, parity
+            mylist[nmine] = make_uint2((unsigned)j | (unsigned)kc << 8 | (unsigned)m << 16 | (unsigned)(ig % kGroupWarps) << 24,
+                                       (unsigned)(prod * half + x0 % half) | (unsigned)(prod * half + (x0 + 1) % half) << 8 |
+                                           (unsigned)(ig % kFull2PerGroup) << 16 | (unsigned)((ig / kFull2PerGroup) & 1) << 24);
+          }
+          ++nmine;
+        }
+      }
+    }
+    nmine = min(nmine, kMaxMine);  // the host refuses launch shapes that could exceed the list
+  }
+  __syncwarp();
+
   // ---- the grid's h ----
   if (!fetch_h<G>(p, smem, warp, lane, plan.htotal, dead, status, bars)) return;
 
   // ---- phase 2: chunks round-robin over the groups, all warps contribute to every task ----
-  const int chunks2 = plan.p2c[plan.nslots];
   const uint32_t full2 = bars + 8 * Bars::full2, empty2 = bars + 8 * Bars::empty2;
-  const int half = plan.nunits2 / kProducers;  // units of one producer
-  int xp = 0;                                   // units this group's producer has handed out so far
+  int i = 0;
   for (int m = 0; m < plan.count2; ++m) {
-    float part = 0.f, unused = 0.f;
-    for (int j = 0; j < plan.nslots; ++j) {
-      const Slot& sl = slots[j];
-      const int nchj = plan.p2c[j + 1] - plan.p2c[j];
-      const int wu = sl.prec ? 2 : 1;
-      float sacc = 0.f;
-      bool mine = false;
-      for (int kc = 0; kc < nchj; ++kc) {
-        const int c = m * chunks2 + plan.p2c[j] + kc;  // chunk number within the phase
-        if (c % kProducers != prod) continue;
-        const int x0 = xp;
-        xp += wu;
-        if (c % kGroups != group) continue;
-        mine = true;
-        const int ig = c / kGroups;  // this group's ordinal of the chunk
-        if (!mbar_wait(full2 + 8 * (kFull2PerGroup * group + ig % kFull2PerGroup), (ig / kFull2PerGroup) & 1, dead, status))
-          return;
-        const int u0 = prod * half + x0 % half, u1 = prod * half + (x0 + 1) % half;
-        const int k0 = kc * kChunkK;
-        const int nblocks = min(kChunkK, sl.inter - k0) >> 7;
-        const uint8_t* dig = smem + SmemLayout::hdig + (sl.hoff + k0) * 3;
-        const float* sumw = reinterpret_cast<const float*>(smem + SmemLayout::hsumw) + ((sl.hoff + k0) >> LG) * 2;
-        const float* binv = reinterpret_cast<const float*>(smem + SmemLayout::hinv) + ((sl.hoff + k0) >> 7);
-        consume_chunk<G>(lr, lane, gw, (c / kGroups) % kGroupWarps, sl.prec ? kModeBoth : kModeSingle, nblocks,
-                         smem + SmemLayout::ring + u0 * plan.unit2_bytes, smem + SmemLayout::ring + u1 * plan.unit2_bytes,
-                         plan.scale2_off, plan.zp2_off, dig, sumw, binv, &sacc, &unused);
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(empty2 + 8 * u0);
-          if (sl.prec) mbar_arrive(empty2 + 8 * u1);
-        }
+    float part = 0.f, unused = 0.f, sacc = 0.f;
+    int jcur = -1;
+    for (; i < nmine; ++i) {
+      const uint2 d = mylist[i];
+      if ((int)((d.x >> 16) & 0xffu) != m) break;
+      const int j = d.x & 0xffu, kc = (d.x >> 8) & 0xffu, rot = d.x >> 24;
+      if (j != jcur) {  // weighted combine, in slot order
+        if (jcur >= 0) part = fmaf(slots[jcur].gated ? plan.gate : slots[jcur].coef, sacc, part);
+        jcur = j;
+        sacc = 0.f;
       }
-      if (mine) part = fmaf(sl.gated ? plan.gate : sl.coef, sacc, part);  // weighted combine, in slot order
+      const Slot& sl = slots[j];
+      const int u0 = d.y & 0xffu, u1 = (d.y >> 8) & 0xffu;
+      if (!mbar_wait(full2 + 8 * (kFull2PerGroup * group + ((d.y >> 16) & 0xffu)), d.y >> 24, dead, status)) return;
+      const int k0 = kc * kChunkK;
+      const int nblocks = min(kChunkK, sl.inter - k0) >> 7;
+      const uint8_t* dig = smem + SmemLayout::hdig + (sl.hoff + k0) * 3;
+      const float* sumw = reinterpret_cast<const float*>(smem + SmemLayout::hsumw) + ((sl.hoff + k0) >> LG) * 2;
+      const float* binv = reinterpret_cast<const float*>(smem + SmemLayout::hinv) + ((sl.hoff + k0) >> 7);
+      consume_chunk<G>(lr, lane, gw, rot, sl.prec ? kModeBoth : kModeSingle, nblocks,
+                       smem + SmemLayout::ring + u0 * plan.unit2_bytes, smem + SmemLayout::ring + u1 * plan.unit2_bytes,
+                       plan.scale2_off, plan.zp2_off, dig, sumw, binv, &sacc, &unused);
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(empty2 + 8 * u0);
+        if (sl.prec) mbar_arrive(empty2 + 8 * u1);
+      }
     }
+    if (jcur >= 0) part = fmaf(slots[jcur].gated ? plan.gate : slots[jcur].coef, sacc, part);
     part += __shfl_xor_sync(0xffffffffu, part, 1);
     if (!mbar_wait(bars + 8 * Bars::pempty2, (m & 1) ^ 1, dead, status)) return;
     if (lr.cq == 0) partial[warp * 16 + lr.r] = make_float2(0.f, part);
@@ -1168,6 +1197,8 @@ static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts
   int dev, sms;
   rc = device_setup(&dev, &sms);
   if (rc != SLICEMOE_OK) return rc;
+  // at most 4 output row blocks per CTA: what the consumer groups' phase-2 chunk lists are sized for
+  if ((shape->hidden / 16 + sms - 1) / sms > 4) return SLICEMOE_E_UNSUPPORTED;
 
   DecodeParams p;
   p.experts = experts;

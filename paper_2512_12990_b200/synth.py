@@ -23,7 +23,7 @@ import numpy as np
 __all__ = [
     "Shape", "SHAPES", "stream_id", "rng", "normal_f32", "bf16_round", "bf16_to_f32",
     "bf16_to_f64", "activations_bf16", "expert_weights", "router_logits_normal",
-    "zipf_gumbel_logits", "decode_trace_logits",
+    "zipf_gumbel_logits", "decode_trace_logits", "prefill_trace_logits",
 ]
 
 
