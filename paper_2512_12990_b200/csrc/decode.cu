@@ -607,12 +607,29 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
   unsigned* status = &p.ws->status;
+  // A CTA is done with the barrier word once it has arrived and, if it has a second phase, seen the count
+  // complete; the last CTA to say so makes the header reusable.  (The next launch touches the header only after
+  // this whole grid has completed.)  Done here rather than at the end of the kernel: the returning atomic's round
+  // trip would otherwise sit between the last store of y and the SM being free for the next launch.
+  auto depart = [&]() {
+    if (lane == 0) {
+      const unsigned old = atomicAdd(&p.ws->depart, 1u);
+      if (old == gridDim.x - 1) {
+        p.ws->bar_arrive = 0;
+        p.ws->depart = 0;
+        __threadfence();
+      }
+    }
+  };
   // phase 1: one group's four partial rows per task -> SwiGLU -> h
   {
     int slot = plan.first_slot, idx = plan.first_idx;
     for (int n = 0; n < plan.count1; ++n) {
       const int group = n % kGroups, round = n / kGroups;
-      if (!mbar_wait(bars + 8 * (Bars::pfull1 + group), round & 1, dead, status)) return;
+      if (!mbar_wait(bars + 8 * (Bars::pfull1 + group), round & 1, dead, status)) {
+        depart();  // a wait ran out: the others will time out at the barrier, the header is still handed back
+        return;
+      }
       float a = 0.f, b = 0.f;
       if (lane < 16) {
 #pragma unroll
@@ -634,7 +651,10 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
   // ---- the single grid-wide dependency: every CTA has written its rows of h ----
   __syncwarp();
   if (lane == 0) red_release_add(&p.ws->bar_arrive, 1u);
-  if (plan.count2 == 0) return;
+  if (plan.count2 == 0) {
+    depart();
+    return;
+  }
   {
     // the whole warp polls, converged: no lane spins on something another lane must provide
     const long long t0 = clock64();
@@ -647,8 +667,12 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
       }
     }
     __syncwarp();
-    if (*dead) return;
+    if (*dead) {
+      depart();
+      return;
+    }
     if (lane == 0) mbar_arrive(bars + 8 * Bars::hx_go);
+    depart();
   }
   // phase 2: all warps' partial rows per output row block -> y
   for (int m = 0; m < plan.count2; ++m) {
@@ -1103,15 +1127,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
     epilogue_loop(p, smem, lane);
   } else if (lane < kProducerLanes) {
     producer_loop<G>(p, smem, lane, warp - kProducerWarp);
-  }
-  __syncthreads();
-  if (tid == 0) {
-    const unsigned old = atomicAdd(&p.ws->depart, 1u);
-    if (old == gridDim.x - 1) {  // everyone is past the barrier: make the header reusable
-      p.ws->bar_arrive = 0;
-      p.ws->depart = 0;
-      __threadfence();
-    }
   }
 }
 
