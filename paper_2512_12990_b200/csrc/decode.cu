@@ -908,6 +908,29 @@ __device__ __forceinline__ Routed read_routing(const DecodeParams& p, int lane, 
   return rt;
 }
 
+// What of the plan depends on the shape and the grid alone; one lane computes it while the kernel still waits
+// for the grids before it.  Assumes at least one valid routed entry when k > 0 (build_plan redoes the unit
+// size in the rare case that there is none).
+__device__ __forceinline__ int phase2_unit_blocks(const DecodeParams& p, bool any_routed) {
+  int maxblk = 1;
+  if (p.n_shared) maxblk = max(maxblk, min(kChunkK, p.shared_inter) >> 7);
+  if (any_routed) maxblk = max(maxblk, min(kChunkK, p.inter) >> 7);
+  return maxblk;
+}
+__device__ __forceinline__ void plan_units2(const DecodeParams& p, Plan* plan, int maxblk) {
+  const int meta_blk = 16 * (128 / p.group);  // scale entries per 128 columns
+  plan->scale2_off = maxblk * 1024;
+  plan->zp2_off = maxblk * 1024 + maxblk * meta_blk * 2;
+  plan->unit2_bytes = (maxblk * (1024 + meta_blk * 3) + 127) & ~127;
+  plan->nunits2 = min(kUnits2, (kUnits * kUnitBytes) / plan->unit2_bytes);
+}
+__device__ void build_plan_static(const DecodeParams& p, uint8_t* smem) {
+  Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
+  const int nrb = p.hidden / 16;
+  plan->count2 = (int)blockIdx.x < nrb ? (nrb - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  plan_units2(p, plan, phase2_unit_blocks(p, p.k > 0));
+}
+
 // Warp 0: slot table (all but the pointers) and the static partition, in closed form: the phase-1 unit
 // sequence is three runs of equal tasks (shared, routed 8-bit, routed 4-bit).
 template <bool FUSED>
@@ -957,7 +980,7 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
     }
     if (lane == 0) plan->p2c[0] = plan->p2u[0] = 0;
   }
-  if (lane == 0) {
+  {
     const unsigned nsh = (unsigned)p.n_shared, nbig = (unsigned)rt.nbig, nsmall = (unsigned)rt.nsmall;
     const unsigned nts = nsh ? (unsigned)p.shared_inter / 16u : 0u, ntr = (unsigned)p.inter / 16u;
     const unsigned nch = (unsigned)nchunks_of(p.hidden);
@@ -973,8 +996,11 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
       if (bound < U1 + U2) return T1 + (bound - U1 + spb - 1) / spb;
       return T1 + T2 + (bound - U1 - U2 + sps - 1) / sps;
     };
+    // both ends of this CTA's window at once: lane 1 takes the upper one
     const unsigned lo = blockIdx.x * T;
-    const unsigned o0 = ord_of(lo), o1 = ord_of(lo + T);
+    const unsigned o = ord_of(lo + (lane & 1) * T);
+    const unsigned o0 = __shfl_sync(0xffffffffu, o, 0), o1 = __shfl_sync(0xffffffffu, o, 1);
+    if (lane != 0) return;
     int slot, idx;
     if (o0 < T1) {
       slot = (int)(o0 / nts);
@@ -990,19 +1016,11 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
     const unsigned big_end = T1 + T2;
     const unsigned nb = (o0 < big_end ? (o1 < big_end ? o1 : big_end) - o0 : 0u);
     plan->chunks1 = (int)(nb * 2u * nch + ((o1 - o0) - nb) * nch);
-    const int nrb = p.hidden / 16;
-    plan->count2 = (nslots > 0 && (int)blockIdx.x < nrb) ? (nrb - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    if (nslots == 0) plan->count2 = 0;  // otherwise as build_plan_static left it
     plan->nslots = nslots;
     plan->htotal = (int)(nsh * (unsigned)p.shared_inter + (nbig + nsmall) * (unsigned)p.inter);
-    // phase-2 units: as large as the widest down chunk of any slot
-    int maxblk = 1;
-    if (nsh) maxblk = max(maxblk, min(kChunkK, p.shared_inter) >> 7);
-    if (nbig + nsmall) maxblk = max(maxblk, min(kChunkK, p.inter) >> 7);
-    const int meta_blk = 16 * (128 / p.group);  // scale entries per 128 columns
-    plan->scale2_off = maxblk * 1024;
-    plan->zp2_off = maxblk * 1024 + maxblk * meta_blk * 2;
-    plan->unit2_bytes = (maxblk * (1024 + meta_blk * 3) + 127) & ~127;
-    plan->nunits2 = min(kUnits2, (kUnits * kUnitBytes) / plan->unit2_bytes);
+    // phase-2 units: as large as the widest down chunk of any slot (set ahead of time for the usual case)
+    if (nbig + nsmall == 0 && p.k > 0) plan_units2(p, plan, phase2_unit_blocks(p, false));
   }
 }
 
@@ -1079,6 +1097,16 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+  }
+  // Also ahead of the wait, because it reads nothing an earlier kernel writes: the shape-only part of the plan,
+  // and the routed experts' pointer table on its way into L2 (warp 1 reads k of its entries right after the wait).
+  if (warp == 0) {
+    if (lane == 0) build_plan_static(p, smem);
+  } else if (warp == 1 && p.experts != nullptr && p.k > 0) {
+    const char* tab = reinterpret_cast<const char*>(p.experts);
+    const size_t bytes = (size_t)p.n_experts * sizeof(slicemoe_expert);
+    for (size_t off = (size_t)lane * 128; off < bytes; off += 32 * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(tab + off));
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
