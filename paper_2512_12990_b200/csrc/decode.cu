@@ -3,14 +3,14 @@
 //
 // The work is a pure weight stream: every plane byte is used once, so the bound is HBM bandwidth and
 // everything else is arranged so that the stream never stops.
-//   * One CTA per SM: 16 consumer warps in 4 groups, one epilogue warp, one producer warp (6 lanes, one
-//     per bulk copy of a chunk).  The 4 warps of a group split a chunk's 128-column blocks, so the
+//   * One CTA per SM: 16 consumer warps in 4 groups, one epilogue warp, two producer warps (6 lanes each,
+//     one per bulk copy of a chunk).  The 4 warps of a group split a chunk's 128-column blocks, so the
 //     per-chunk bookkeeping is paid by 4 warps, not 16, while 4 chunks are in work at any time.  The
 //     schedule is a pure function of the slot table, so every role enumerates it for itself and only
 //     data and barrier phases pass between them.  The producer streams chunks - 16 rows x <=2048 columns: the MSB plane tile,
 //     the LSB plane tile when the expert runs at 8 bits (<=16 KB each, one contiguous run thanks to the
-//     tiled layout), scales and zero-points - into a ring of eight 16 KB units with cp.async.bulk +
-//     mbarriers.  It never waits for the gate/up -> down dependency, so down-projection tiles are
+//     tiled layout), scales and zero-points - into a ring of eight 19 KB units with cp.async.bulk +
+//     mbarriers.  They never wait for the gate/up -> down dependency, so down-projection tiles are
 //     already in flight (up to the whole ring) while the grid exchanges h.
 //   * Integer arithmetic on the tensor pipe.  The activation vector (x, later h) is converted once,
 //     per 128-element block, to fixed point relative to the block's largest magnitude and split into
@@ -64,7 +64,7 @@ constexpr unsigned long long kWaitCycles = 4000000000ull;  // ~2 s: every device
 // ---- workspace --------------------------------------------------------------------------------
 struct WsHeader {
   unsigned bar_arrive;  // grid barrier: CTAs that finished the gate/up phase
-  unsigned depart;      // CTAs that finished the kernel (the last one re-zeroes the header)
+  unsigned depart;      // CTAs that are through with the barrier word (the last one re-zeroes the header)
   unsigned status;      // SLICEMOE_STATUS_* bits
   unsigned pad;
 };
