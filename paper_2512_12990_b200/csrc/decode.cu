@@ -150,8 +150,8 @@ struct SmemLayout {
   static constexpr int hinv = xsumw + (kMaxHidden / 32) * 8;  // float [kHCap/128]: 2^-e of each 128-block of h
   static constexpr int xinv = hinv + (kHCap / 128) * 4;       // float [kMaxHidden/128]
   static constexpr int partial = xinv + (kMaxHidden / 128) * 4;  // float2 [warps][16]
-  static constexpr int p2list = partial + kConsumerWarps * 16 * 2 * 4;  // uint2 [warps][kMaxMine]: a warp's phase-2 chunks
-  static constexpr int slots = p2list + kConsumerWarps * kMaxMine * 8;
+  static constexpr int p2list = partial + kConsumerWarps * 16 * 2 * 4;  // uint4 [warps][kMaxMine]: a warp's phase-2 chunks
+  static constexpr int slots = p2list + kConsumerWarps * kMaxMine * 16;
   static constexpr int plan = slots + kMaxSlots * (int)sizeof(Slot);
   static constexpr int bars = (plan + (int)sizeof(Plan) + 15) & ~15;  // uint64 barriers
   static constexpr int nbars = 2 * kUnits + kGroups * kFull2PerGroup + kUnits2 + 2 * kGroups + 5;
@@ -161,7 +161,7 @@ struct SmemLayout {
 static_assert(SmemLayout::total <= 227 * 1024, "shared memory budget");
 static_assert(sizeof(Slot) % 8 == 0, "slot alignment");
 static_assert(SmemLayout::slots % 8 == 0 && SmemLayout::hdig % 16 == 0 && SmemLayout::xdig % 16 == 0 &&
-                  SmemLayout::plan % 8 == 0 && SmemLayout::partial % 8 == 0,
+                  SmemLayout::plan % 8 == 0 && SmemLayout::partial % 8 == 0 && SmemLayout::p2list % 16 == 0,
               "alignment");
 
 // Barriers.  Every barrier has ONE waiter that meets its phases strictly in order, so a parity wait can never
@@ -279,17 +279,19 @@ __device__ __forceinline__ void block_to_digits(const float (&v)[4], int k0, int
   const int ex = (int)(mb >> 23) - 127;  // floor(log2 max) for normal numbers
   const int e = max(-100, min(100, 21 - ex));
   const float scale = __uint_as_float((unsigned)(127 + e) << 23);
-  int X0[4], X1[4], X2[4];
+  // Z = (X + 0x808080) ^ 0x808080 holds the three digits in its bytes: adding 128 to a byte and flipping its top
+  // bit back leaves the byte read as a signed digit, and the carry into the next byte is exactly what remains
+  // after taking that digit (X1 = (X + 128) >> 8, and so on up).
+  uint32_t Z[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    X0[j] = max(-4194304, min(4194304, __float2int_rn(v[j] * scale)));
-    X1[j] = (X0[j] + 128) >> 8;  // what is left after taking the low byte as a signed digit
-    X2[j] = (X1[j] + 128) >> 8;
+    const int X = max(-4194304, min(4194304, __float2int_rn(v[j] * scale)));
+    Z[j] = (uint32_t)(X + 0x808080) ^ 0x808080u;
   }
-  // byte 0 of each of the four values -> one word (value j in byte j)
-  const uint32_t d0 = __byte_perm(__byte_perm(X0[0], X0[1], 0x0040), __byte_perm(X0[2], X0[3], 0x0040), 0x5410);
-  const uint32_t d1 = __byte_perm(__byte_perm(X1[0], X1[1], 0x0040), __byte_perm(X1[2], X1[3], 0x0040), 0x5410);
-  const uint32_t d2 = __byte_perm(__byte_perm(X2[0], X2[1], 0x0040), __byte_perm(X2[2], X2[3], 0x0040), 0x5410);
+  // byte i of each of the four values -> one word (value j in byte j)
+  const uint32_t d0 = __byte_perm(__byte_perm(Z[0], Z[1], 0x0040), __byte_perm(Z[2], Z[3], 0x0040), 0x5410);
+  const uint32_t d1 = __byte_perm(__byte_perm(Z[0], Z[1], 0x0051), __byte_perm(Z[2], Z[3], 0x0051), 0x5410);
+  const uint32_t d2 = __byte_perm(__byte_perm(Z[0], Z[1], 0x0062), __byte_perm(Z[2], Z[3], 0x0062), 0x5410);
   const int k = k0 + 4 * lane;
   *reinterpret_cast<uint32_t*>(dig + digit_offset(k, 0)) = d0;
   *reinterpret_cast<uint32_t*>(dig + digit_offset(k, 1)) = d1;
@@ -524,7 +526,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
 
   // ---- while the grid barrier is pending: list this group's phase-2 chunks (the walk over all output row
   // blocks, slots and chunks costs more than consuming the group's own chunks, so it is done ahead of time) ----
-  uint2* mylist = reinterpret_cast<uint2*>(smem + SmemLayout::p2list) + warp * kMaxMine;
+  uint4* mylist = reinterpret_cast<uint4*>(smem + SmemLayout::p2list) + warp * kMaxMine;
   int nmine = 0;
   {
     const int chunks2 = plan.p2c[plan.nslots];
@@ -533,7 +535,8 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
     for (int m = 0; m < plan.count2; ++m) {
       for (int j = 0; j < plan.nslots; ++j) {
         const int nchj = plan.p2c[j + 1] - plan.p2c[j];
-        const int wu = slots[j].prec ? 2 : 1;
+        const Slot& sl = slots[j];
+        const int wu = sl.prec ? 2 : 1;
         for (int kc = 0; kc < nchj; ++kc) {
           const int c = m * chunks2 + plan.p2c[j] + kc;  // chunk number within the phase
           if (c % kProducers != prod) continue;
@@ -542,10 +545,14 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
           if (c % kGroups != group) continue;
           const int ig = c / kGroups;  // this group's ordinal of the chunk
           if (lane == 0 && nmine < kMaxMine) {
-            // slot, chunk of the slot, row block, rotation of the warps | the chunk's units, full barrier, parity
-            mylist[nmine] = make_uint2((unsigned)j | (unsigned)kc << 8 | (unsigned)m << 16 | (unsigned)(ig % kGroupWarps) << 24,
+            // slot, row block, rotation of the warps | the chunk's units, full barrier, parity | 128-column blocks,
+            // both slices? | first column of the chunk in h
+            const int k0 = kc * kChunkK;
+            mylist[nmine] = make_uint4((unsigned)j | (unsigned)m << 16 | (unsigned)(ig % kGroupWarps) << 24,
                                        (unsigned)(prod * half + x0 % half) | (unsigned)(prod * half + (x0 + 1) % half) << 8 |
-                                           (unsigned)(ig % kFull2PerGroup) << 16 | (unsigned)((ig / kFull2PerGroup) & 1) << 24);
+                                           (unsigned)(ig % kFull2PerGroup) << 16 | (unsigned)((ig / kFull2PerGroup) & 1) << 24,
+                                       (unsigned)(min(kChunkK, sl.inter - k0) >> 7) | (sl.prec ? 256u : 0u),
+                                       (unsigned)(sl.hoff + k0));
           }
           ++nmine;
         }
@@ -565,29 +572,28 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
     float part = 0.f, unused = 0.f, sacc = 0.f;
     int jcur = -1;
     for (; i < nmine; ++i) {
-      const uint2 d = mylist[i];
+      const uint4 d = mylist[i];
       if ((int)((d.x >> 16) & 0xffu) != m) break;
-      const int j = d.x & 0xffu, kc = (d.x >> 8) & 0xffu, rot = d.x >> 24;
+      const int j = d.x & 0xffffu, rot = d.x >> 24;
       if (j != jcur) {  // weighted combine, in slot order
         if (jcur >= 0) part = fmaf(slots[jcur].gated ? plan.gate : slots[jcur].coef, sacc, part);
         jcur = j;
         sacc = 0.f;
       }
-      const Slot& sl = slots[j];
       const int u0 = d.y & 0xffu, u1 = (d.y >> 8) & 0xffu;
+      const int nblocks = d.z & 0xffu, col = (int)d.w;
+      const bool p8 = (d.z & 256u) != 0u;
       if (!mbar_wait(full2 + 8 * (kFull2PerGroup * group + ((d.y >> 16) & 0xffu)), d.y >> 24, dead, status)) return;
-      const int k0 = kc * kChunkK;
-      const int nblocks = min(kChunkK, sl.inter - k0) >> 7;
-      const uint8_t* dig = smem + SmemLayout::hdig + (sl.hoff + k0) * 3;
-      const float* sumw = reinterpret_cast<const float*>(smem + SmemLayout::hsumw) + ((sl.hoff + k0) >> LG) * 2;
-      const float* binv = reinterpret_cast<const float*>(smem + SmemLayout::hinv) + ((sl.hoff + k0) >> 7);
-      consume_chunk<G>(lr, lane, gw, rot, sl.prec ? kModeBoth : kModeSingle, nblocks,
+      const uint8_t* dig = smem + SmemLayout::hdig + col * 3;
+      const float* sumw = reinterpret_cast<const float*>(smem + SmemLayout::hsumw) + (col >> LG) * 2;
+      const float* binv = reinterpret_cast<const float*>(smem + SmemLayout::hinv) + (col >> 7);
+      consume_chunk<G>(lr, lane, gw, rot, p8 ? kModeBoth : kModeSingle, nblocks,
                        smem + SmemLayout::ring + u0 * plan.unit2_bytes, smem + SmemLayout::ring + u1 * plan.unit2_bytes,
                        plan.scale2_off, plan.zp2_off, dig, sumw, binv, &sacc, &unused);
       __syncwarp();
       if (lane == 0) {
         mbar_arrive(empty2 + 8 * u0);
-        if (sl.prec) mbar_arrive(empty2 + 8 * u1);
+        if (p8) mbar_arrive(empty2 + 8 * u1);
       }
     }
     if (jcur >= 0) part = fmaf(slots[jcur].gated ? plan.gate : slots[jcur].coef, sacc, part);
