@@ -43,7 +43,7 @@ GRAPH_CHUNK = 1000     # steps per captured CUDA graph
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode-kernel launch on this workload, from the
 # ncu capture summarised under profiles/; None once the kernel has changed since the capture.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 58730000
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 58530000
 
 
 def expert_bytes(hidden: int, inter: int, group: int, prec8: bool) -> int:
