@@ -1078,8 +1078,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
 
   // Programmatic dependent launch: the next kernel in the stream may start launching as soon as every CTA
   // of this grid has got here (its CTAs find room only where one of ours has exited), and this kernel sets
-  // up its barriers before it waits for the grids before it.  Nothing in global memory is touched before
-  // that wait: routing lists, x and the workspace may still be in use by the previous kernels.
+  // up its barriers before it waits for the grids before it.  Nothing an earlier kernel may write is touched
+  // before that wait: routing lists, x and the workspace may still be in use by the previous kernels.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (warp == kProducerWarp) {
     if (lane == 0) {
