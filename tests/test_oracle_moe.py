@@ -201,7 +201,7 @@ def test_ffn_invariants():
     assert experts[0]["down"]["msb"].shape == (hidden, inter)
 
 
-def test_algorithmic_bytes_match_survey_figures():
+def test_algorithmic_bytes_of_a_1408_wide_expert():
     """1408-wide expert at group 128: 8-bit 8,853,504 B, 4-bit 4,528,128 B (3 matrices)."""
     mat_gu = dict(msb=np.zeros((1408, 2048), np.uint8), group=128)
     mat_d = dict(msb=np.zeros((2048, 1408), np.uint8), group=128)
