@@ -75,8 +75,9 @@ __global__ void pf_scan_kernel(const int* __restrict__ counts, int E, int n_shar
                                int* __restrict__ offsets, int* __restrict__ tile_expert, int* __restrict__ tile_row0,
                                int* __restrict__ item_start, int* __restrict__ ntiles) {
   if (threadIdx.x != 0) return;
-  int off = 0, nt = 0, items = 0;
+  int off = 0, nt = 0, items = 0, nt_routed = 0;
   for (int e = 0; e < E + n_shared; ++e) {
+    if (e == E) nt_routed = nt;
     const int c = e < E ? counts[e] : T;
     offsets[e] = off;
     for (int r = 0; r < c; r += kPfTileM) {
@@ -93,6 +94,7 @@ __global__ void pf_scan_kernel(const int* __restrict__ counts, int E, int n_shar
   ntiles[0] = nt;
   ntiles[1] = off;
   ntiles[2] = items;
+  ntiles[3] = n_shared > 0 ? nt_routed : nt;  // tiles of routed experts: they come first and have inter / 64 items each
 }
 
 // Every (token, slot) pair takes a row of its expert; shared experts take row t.  Which row a pair gets
@@ -283,13 +285,16 @@ template <int PHASE>
 __device__ __forceinline__ UItem u_item(const PfGemmParams& p, int item) {
   int tile, nt;
   if (PHASE == 1) {
-    int lo = 0, hi = p.ntiles[0];  // last tile whose first item is <= item
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (p.item_start[mid] <= item) lo = mid; else hi = mid;
+    // routed tiles first, inter / 64 items each, then the shared experts' tiles with shared_inter / 64 items each
+    const int per_r = p.inter / 64, routed_items = p.ntiles[3] * per_r;
+    if (item < routed_items) {
+      tile = item / per_r;
+      nt = item - tile * per_r;
+    } else {
+      const int per_s = p.shared_inter / 64, rest = item - routed_items;
+      tile = p.ntiles[3] + rest / per_s;
+      nt = rest - (rest / per_s) * per_s;
     }
-    tile = lo;
-    nt = item - p.item_start[lo];
   } else {
     const int per = p.hidden / 128;
     tile = item / per;
@@ -373,8 +378,12 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
     // ---- token tiles: one TMA copy per step ----
     if (lane == 0) {
       uint32_t s = 0, ph = 0;
+      // the next item's description is fetched while this item's copies go out
+      UItem w{};
+      if ((int)blockIdx.x < n_items) w = u_item<PHASE>(p, blockIdx.x);
       for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
-        const UItem w = u_item<PHASE>(p, item);
+        UItem wn = w;
+        if (item + (int)gridDim.x < n_items) wn = u_item<PHASE>(p, item + gridDim.x);
         const int nk = w.K / kPfChunkK;
         for (int kc = 0; kc < nk; ++kc) {
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { alive = false; break; }
@@ -386,6 +395,7 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
               : "memory");
           if (++s == kUStages) { s = 0; ph ^= 1; }
         }
+        w = wn;
       }
     }
   } else if (warp == kUWarpMma) {
@@ -395,8 +405,11 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
     uint64_t* last_empty = nullptr;
     uint32_t last_ph = 0;
     const uint64_t bd0 = umma_desc(smem_u32(smem));
+    UItem w{};
+      if ((int)blockIdx.x < n_items) w = u_item<PHASE>(p, blockIdx.x);
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++ni) {
-      const UItem w = u_item<PHASE>(p, item);
+      UItem wn = w;
+      if (item + (int)gridDim.x < n_items) wn = u_item<PHASE>(p, item + gridDim.x);
       const int nk = w.K / kPfChunkK;
       const uint32_t ab = ni & 1;
       // the accumulator must have been read out (the item before the previous one used it)
@@ -424,6 +437,7 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
       if (!alive) break;
       if (lane == 0) umma_commit(&acc_full[ab]);
       __syncwarp();
+      w = wn;
     }
     // the last commit must have arrived before shared memory goes away
     if (alive && last_empty && !__all_sync(0xffffffffu, mbar_wait(last_empty, last_ph, abort_flag))) alive = false;
