@@ -156,7 +156,7 @@ int slicemoe_get_status(void *workspace, int *status_out, void *stream);
  * per token); accumulation is fp32, h stays fp32 between the two projections, the summation
  * order is fixed (results are bit-reproducible run to run).
  * Errors: INVALID_ARG, UNSUPPORTED (shape limits above; sum of intermediate widths over the k + n_shared
- * slots must be <= 12288), CUDA.
+ * slots must be <= 12288; hidden / 16 must not exceed 4 x the device's SM count), CUDA.
  */
 int slicemoe_expert_ffn(const slicemoe_shape *shape, const slicemoe_expert *experts, const void *x,
                         int T, const int32_t *ids, const uint8_t *prec, const float *weights,
