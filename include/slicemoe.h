@@ -93,7 +93,7 @@ size_t slicemoe_plane_bytes(int N, int K);           /* bytes of one slice plane
 size_t slicemoe_meta_count(int N, int K, int group); /* number of (scale, zp) entries: N*K/group */
 
 /*
- * slicemoe_pack - offline preparation of one weight matrix: quantise (Table 1 fn. 1, Section 5.1:
+ * slicemoe_pack - offline preparation of one weight matrix: quantise (Table 1 fn. 1, Section 6.1:
  * grouped asymmetric codes) and split into MSB / LSB slice planes (Sections 4.1, 4.2).
  *   W      device, float32 [N, K] row-major (read only)
  *   msb, lsb, scale, zp   device outputs in the physical layout; sizes from the functions above
@@ -138,11 +138,28 @@ int slicemoe_route_topk(const float *logits, int T, int E, int k, const float *b
  * slicemoe_workspace_bytes() bytes (256-byte aligned) and call slicemoe_workspace_init() once
  * before first use (it zeroes the header; the kernels leave it zeroed again when they finish).
  * One workspace serves one stream at a time.
+ *
+ * The decode kernel's CTAs (one per SM) meet once at a grid-wide barrier, so they must all be resident
+ * together.  The library refuses (UNSUPPORTED) a device on which a CTA of the kernel does not fit an SM;
+ * it cannot know what else occupies the device at launch time.  If other work holds SMs for longer than the
+ * wait limit (default: 10^8 clock cycles, about 50 ms), the barrier's wait ends by itself: the kernel returns,
+ * SLICEMOE_STATUS_WAIT_TIMEOUT is set and y is not valid.  Run the decode calls on a device (or a
+ * partition of it) that they have to themselves while they run.  After a time-out, initialise the workspace again.
  */
 size_t slicemoe_workspace_bytes(const slicemoe_shape *shape);
 int slicemoe_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
 /* Copies the status word to *status_out (host) and clears it.  Synchronises `stream`. */
 int slicemoe_get_status(void *workspace, int *status_out, void *stream);
+/*
+ * Sets the limit of the kernels' device-side waits for this workspace, in GPU clock cycles (0 = the default),
+ * and a number of extra arrivals that the grid barrier waits for beyond the grid's own.  extra_arrivals is 0
+ * in any real use; a non-zero value makes that wait run out by construction, which is how the time-out path
+ * is exercised without faulting or hanging anything: the kernel returns by itself after `wait_cycles`,
+ * SLICEMOE_STATUS_WAIT_TIMEOUT is set and y is not valid.  slicemoe_workspace_init resets both.  Enqueued
+ * on `stream`.
+ */
+int slicemoe_workspace_set_wait(void *workspace, unsigned long long wait_cycles, unsigned extra_arrivals,
+                                void *stream);
 
 /*
  * slicemoe_expert_ffn - the mixed-precision expert FFN of Section 4.1 over an expert-id/precision
@@ -209,7 +226,8 @@ int slicemoe_layer_routed(const slicemoe_shape *shape, const slicemoe_expert *ex
  *     nothing is ever allocated to make it fit.
  *   - The call allocates nothing and frees nothing, directly or through any library.
  *   - First call on a device: the library looks up the device address of its array once per device
- *     (with that device current) and remembers it.  Make this first call outside any stream capture.
+ *     (with that device current) and remembers it.  Make this first call outside any stream capture, and
+ *     from one host thread (the look-up is not guarded against a second thread doing the same at once).
  *   - The array is shared by all calls on a device and keeps the previous call's contents; each call
  *     clears the part that must start at zero (on `stream`, before its kernels).  Two calls whose work
  *     overlaps on the GPU - different streams, or different host threads without ordering - race on
@@ -228,7 +246,8 @@ int slicemoe_layer_static(const slicemoe_shape *shape, const slicemoe_expert *ex
  * copies x (bf16 [hidden]) and logits (float32 [E]) to the device, runs slicemoe_layer_routed
  * (bias/tau/rank_high as in slicemoe_route_topk; the precision request is used as the precision
  * list), copies y (float32 [hidden]) back and synchronises `stream`.  x_host, logits_host
- * and y_host should be pinned for the copies to be asynchronous.  When y_host is pinned,
+ * and y_host should be pinned for the copies to be asynchronous.  logits_host may be NULL: the logits then
+ * follow x directly in the buffer at x_host (bf16 [hidden], then float32 [E]) and one copy brings both.  When y_host is pinned,
  * device-mapped host memory (cudaHostAlloc / cudaHostRegister, 16-byte aligned) the kernel writes y
  * straight into it and no copy back is issued.  Weights stay resident on the device.  Staging
  * buffers live in the workspace.
@@ -241,14 +260,17 @@ int slicemoe_decode_step_host(const slicemoe_shape *shape, const slicemoe_expert
 
 /*
  * slicemoe_prefill_layer - the layer for a prompt of T tokens at once (Section 3: prefill visits
- * every expert of a layer, so the expert FFN becomes a grouped dense contraction; Section 5.3:
- * after prefill each expert is held, and here run, at the precision its cached slices allow).
+ * every expert of a layer, so the expert FFN becomes a grouped dense contraction).  Section 6.3 says that
+ * prefill wants high-bit computation; the per-expert precision flag is this library's generalisation (an
+ * expert may also be run from its MSB slice alone), which a mixed-precision prefill uses.
  * Tokens are grouped by expert on the device; per 128-token tile the weight tile is dequantised
  * from the nibble planes - s*(q - zp), or 16*s*(q_msb - (zp >> 4)) for an MSB-only expert - into
  * tensor memory as the exact sum of two fp16 numbers per weight (no weight is rounded) and
  * contracted on the tensor cores (tcgen05, fp16 x fp16 with fp32 accumulation); tokens enter as
  * fp16 (exact for bf16 inputs in fp16's normal range) and h is rounded to fp16 between the two
- * projections (relative error 2^-11, inside the FFN tolerance).  Each
+ * projections (relative error 2^-11, inside the FFN tolerance).  Both conversions go to fp16's range: a token
+ * value or an h beyond +-65504 becomes infinite and that row of y is not finite (nothing faults, no status
+ * bit is set); activations of that size do not occur behind a normalisation layer.  Each
  * (token, expert) pair gets its own fp32 result row and y[t] sums them in list order (routed
  * slots 0..k-1, then the shared experts), so y is bit-reproducible run to run.
  *   x            device bf16 [T, hidden]
@@ -276,8 +298,8 @@ int slicemoe_prefill_layer(const slicemoe_shape *shape, const slicemoe_expert *e
                            void *stream);
 
 /*
- * Host-side Dynamic Bit-Sliced Caching bookkeeping (Section 4.1; cache implementation of Section
- * 5.1).  Pure host code: it only turns (expert id, precision request) lists into the precision
+ * Host-side Dynamic Bit-Sliced Caching bookkeeping (Section 4.1; cache set-up of Section
+ * 6.1).  Pure host code: it only turns (expert id, precision request) lists into the precision
  * list the FFN runs with, plus hit/miss accounting.  MSB slices: LRU.  LSB slices: lowest priority,
  * evicted (oldest first) before any MSB slice.  One cache for all layers.  Optional miss budget:
  * once step >= warmup_steps, while bytes fetched / full-precision bytes of the same requests

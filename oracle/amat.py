@@ -5,7 +5,7 @@ The paper gives the truncation rule (the displayed equation of Section 4.2):
     shift = b_high - b_low,  q_low = floor(q_high / 2^shift),  zp_low = floor(zp_high / 2^shift)
 
 and says experts use grouped asymmetric integer quantisation (Table 1, footnote 1; Section
-5.1).  It does not write the quantiser out; the reading used here is the standard affine
+6.1).  It does not write the quantiser out; the reading used here is the standard affine
 quantiser, stated step by step in `quantize`.
 """
 from __future__ import annotations
@@ -16,7 +16,7 @@ F32 = np.float32
 
 
 def quantize(W: np.ndarray, group: int, b_high: int = 8):
-    """Asymmetric per-group quantiser along K (Table 1 fn. 1 / Section 5.1: grouped asymmetric INT).
+    """Asymmetric per-group quantiser along K (Table 1 fn. 1 / Section 6.1: grouped asymmetric INT).
 
     W: float32 [N, K], K % group == 0.  Per row n and K-group g, in float32 arithmetic:
       lo = min(min_k w, 0), hi = max(max_k w, 0)

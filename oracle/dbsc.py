@@ -4,7 +4,7 @@ What the paper fixes: MSB and LSB slices of an expert are cached independently a
 produces its own hit/miss; a critical expert requests both slices, a non-critical one the MSB
 slice only; full precision is used when both slices are available, MSB-only computation
 otherwise; MSB slices follow standard LRU; LSB slices have the lowest priority and are evicted
-first; one cache is shared by all layers (Section 5.1, cache implementation); the miss-rate
+first; one cache is shared by all layers (Section 6.1, cache implementation); the miss-rate
 constraint activates after the first 10 decode steps.
 
 Readings where the paper is silent (stated once, used by both this oracle and the host code):

@@ -27,7 +27,7 @@ DBSC_STAT_NAMES = ("requests", "msb_hit", "msb_miss", "lsb_hit", "lsb_miss", "ls
 EXPORTS = (
     "slicemoe_strerror", "slicemoe_version", "slicemoe_last_cuda_error", "slicemoe_plane_bytes", "slicemoe_meta_count", "slicemoe_pack",
     "slicemoe_unpack_plane", "slicemoe_unpack_meta", "slicemoe_route_topk", "slicemoe_workspace_bytes",
-    "slicemoe_workspace_init", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer",
+    "slicemoe_workspace_init", "slicemoe_workspace_set_wait", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer",
     "slicemoe_decode_step_host", "slicemoe_layer_static", "slicemoe_layer_routed", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
     "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
     "slicemoe_dbsc_assign", "slicemoe_dbsc_stats", "slicemoe_dbsc_contains",
@@ -86,6 +86,7 @@ def lib() -> ctypes.CDLL:
     L.slicemoe_workspace_bytes.argtypes = [POINTER(Shape)]
     L.slicemoe_workspace_init.argtypes = [c_void_p, c_size_t, c_void_p]
     L.slicemoe_get_status.argtypes = [c_void_p, POINTER(c_int), c_void_p]
+    L.slicemoe_workspace_set_wait.argtypes = [c_void_p, ctypes.c_ulonglong, ctypes.c_uint, c_void_p]
     L.slicemoe_expert_ffn.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p, c_size_t, c_void_p]
     L.slicemoe_layer.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
@@ -232,6 +233,11 @@ def new_workspace(shape: Shape, device="cuda", stream=None):
     return ws
 
 
+def slicemoe_workspace_set_wait(ws, wait_cycles: int, extra_arrivals: int = 0, stream=None):
+    _check(lib().slicemoe_workspace_set_wait(_ptr(ws), wait_cycles, extra_arrivals, _stream(stream)),
+           "slicemoe_workspace_set_wait")
+
+
 def slicemoe_get_status(ws, stream=None) -> int:
     out = c_int(0)
     _check(lib().slicemoe_get_status(_ptr(ws), ctypes.byref(out), _stream(stream)), "slicemoe_get_status")
@@ -309,11 +315,12 @@ def slicemoe_layer_routed(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec
 
 def slicemoe_decode_step_host(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x_host, logits_host, y_host,
                               ws, bias=None, renorm=False, tau=2.0, rank_high=0, stream=None):
-    """x_host: pinned CPU bf16 [hidden]; logits_host: pinned CPU float32 [E]; y_host: pinned CPU float32
+    """x_host: pinned CPU bf16 [hidden]; logits_host: pinned CPU float32 [E], or None when x_host is one pinned
+    byte buffer holding x (bf16 [hidden]) and then the logits (float32 [E]); y_host: pinned CPU float32
     [hidden] (written).  Synchronises the stream."""
     rc = lib().slicemoe_decode_step_host(ctypes.byref(shape), _ptr(experts_tbl), _ptr(shared_tbl),
                                          _ptr(shared_gate_vec), c_void_p(x_host.data_ptr()),
-                                         c_void_p(logits_host.data_ptr()), _ptr(bias), 1 if renorm else 0, tau,
+                                         None if logits_host is None else c_void_p(logits_host.data_ptr()), _ptr(bias), 1 if renorm else 0, tau,
                                          rank_high, c_void_p(y_host.data_ptr()), _ptr(ws), ws.numel(),
                                          _stream(stream))
     _check(rc, "slicemoe_decode_step_host")

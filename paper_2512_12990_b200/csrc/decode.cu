@@ -59,14 +59,17 @@ constexpr int kMaxHidden = 4096;
 constexpr int kHCap = 12288;  // sum of intermediate widths over all slots of a layer
 constexpr int kMaxMine = 32;   // phase-2 chunks one consumer group can have: (slots + kHCap / kChunkK) chunks per
                                // output row block, at most 4 row blocks per CTA, shared by 4 groups
-constexpr unsigned long long kWaitCycles = 4000000000ull;  // ~2 s: every device-side wait is bounded
+// Every device-side wait is bounded: by this many clock cycles (about 50 ms; a layer takes tens of microseconds)
+// unless the workspace header carries another limit.
+constexpr unsigned long long kWaitCycles = 100000000ull;
 
 // ---- workspace --------------------------------------------------------------------------------
 struct WsHeader {
   unsigned bar_arrive;  // grid barrier: CTAs that finished the gate/up phase
   unsigned depart;      // CTAs that are through with the barrier word (the last one re-zeroes the header)
   unsigned status;      // SLICEMOE_STATUS_* bits
-  unsigned pad;
+  unsigned extra_arrivals;         // added to the grid barrier's target (slicemoe_workspace_set_wait; 0 in real use)
+  unsigned long long wait_cycles;  // limit of the device-side waits, 0 = kWaitCycles
 };
 constexpr size_t kWsHOff = 2048;                              // float h[kHCap]
 constexpr size_t kWsStageOff = kWsHOff + sizeof(float) * kHCap;
@@ -79,6 +82,7 @@ constexpr size_t kWsStPrec = kWsStW + 64;
 constexpr size_t kWsStY = kWsStPrec + 64;
 constexpr size_t kWsBytes = kWsStY + 4 * kMaxHidden;
 static_assert(sizeof(WsHeader) <= kWsHOff, "workspace header");
+static_assert(kWsStLogits + 4 * 512 <= kWsStIds, "x and the logits fit the staging area back to back too");
 
 // ---- kernel parameters -------------------------------------------------------------------------
 struct DecodeParams {
@@ -155,7 +159,7 @@ struct SmemLayout {
   static constexpr int plan = slots + kMaxSlots * (int)sizeof(Slot);
   static constexpr int bars = (plan + (int)sizeof(Plan) + 15) & ~15;  // uint64 barriers
   static constexpr int nbars = 2 * kUnits + kGroups * kFull2PerGroup + kUnits2 + 2 * kGroups + 5;
-  static constexpr int dead = bars + nbars * 8;
+  static constexpr int dead = bars + nbars * 8;  // int dead flag; 8 bytes on, the wait limit in cycles
   static constexpr int total = dead + 16;
 };
 static_assert(SmemLayout::total <= 227 * 1024, "shared memory budget");
@@ -206,6 +210,10 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The CTA's wait limit sits 8 bytes behind its dead flag.
+__device__ __forceinline__ unsigned long long wait_limit(volatile int* dead) {
+  return *reinterpret_cast<volatile unsigned long long*>(dead + 2);
+}
 // Bounded wait.  Returns false (and raises the CTA's dead flag) when the limit is hit or another
 // role of this CTA already gave up.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* dead, unsigned* status) {
@@ -214,7 +222,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
     for (int i = 0; i < 256; ++i)
       if (mbar_try(bar, parity)) return true;
     if (*dead) return false;
-    if ((unsigned long long)(clock64() - t0) > kWaitCycles) {
+    if ((unsigned long long)(clock64() - t0) > wait_limit(dead)) {
       *dead = 1;
       atomicOr(status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
       return false;
@@ -664,9 +672,10 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
   {
     // the whole warp polls, converged: no lane spins on something another lane must provide
     const long long t0 = clock64();
-    while (ld_acquire_u32(&p.ws->bar_arrive) < gridDim.x) {
+    const unsigned target = gridDim.x + p.ws->extra_arrivals;
+    while (ld_acquire_u32(&p.ws->bar_arrive) < target) {
       if (*dead) break;
-      if ((unsigned long long)(clock64() - t0) > kWaitCycles) {
+      if ((unsigned long long)(clock64() - t0) > wait_limit(dead)) {
         *dead = 1;
         atomicOr(status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
         break;
@@ -854,14 +863,14 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
     for (int i = max(0, n1 - 2); i < n1; ++i) {
       const long long t0 = clock64();
       while (!mbar_try(bars + 8 * (Bars::full + 2 * g + (i & 1)), (i >> 1) & 1)) {
-        if (*dead || (unsigned long long)(clock64() - t0) > kWaitCycles) break;
+        if (*dead || (unsigned long long)(clock64() - t0) > wait_limit(dead)) break;
       }
     }
     const int n2 = c2 > g ? (c2 - 1 - g) / kGroups + 1 : 0;  // chunks of the phase that went to group g
     for (int i = max(0, n2 - kFull2PerGroup); i < n2; ++i) {
       const long long t0 = clock64();
       while (!mbar_try(bars + 8 * (Bars::full2 + kFull2PerGroup * g + i % kFull2PerGroup), (i / kFull2PerGroup) & 1)) {
-        if (*dead || (unsigned long long)(clock64() - t0) > kWaitCycles) break;
+        if (*dead || (unsigned long long)(clock64() - t0) > wait_limit(dead)) break;
       }
     }
   }
@@ -1084,6 +1093,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
   if (warp == kProducerWarp) {
     if (lane == 0) {
       *reinterpret_cast<int*>(smem + SmemLayout::dead) = 0;
+      *reinterpret_cast<unsigned long long*>(smem + SmemLayout::dead + 8) = kWaitCycles;
       const uint32_t bars = smem_u32(smem + SmemLayout::bars);
       for (int s = 0; s < kUnits; ++s) {
         mbar_init(bars + 8 * (Bars::full + s), 1);             // lane 0's expect_tx arrive
@@ -1127,6 +1137,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
   } else if (warp == 2) {
     if (p.n_shared > 0) load_slot_pointers<FUSED>(p, smem, lane, false);
   } else if (warp == kProducerWarp) {
+    if (lane == 0) {  // a wait limit set by the host for this workspace (the thread that wrote the default)
+      const unsigned long long lim = p.ws->wait_cycles;
+      if (lim != 0ull) *reinterpret_cast<unsigned long long*>(smem + SmemLayout::dead + 8) = lim;
+    }
     if (p.sigmoid_gate && p.n_shared > 0) {
       // Qwen-style shared-expert gate: sigmoid(v . x)
       float dot = 0.f;
@@ -1188,6 +1202,13 @@ static int launch_decode(const DecodeParams& p, int dev, int sms, int gi, cudaSt
   if (!attr_set) {
     SM_CUDA_TRY(cudaFuncSetAttribute(decode_layer_kernel<G, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      SmemLayout::total));
+    // The CTAs meet at a grid barrier, so all of them must be able to be resident at once: one per SM needs
+    // the kernel to fit an SM at all.  (If another kernel holds SMs at the time, the barrier's bounded wait
+    // ends the launch with SLICEMOE_STATUS_WAIT_TIMEOUT instead of a hang.)
+    int per_sm = 0;
+    SM_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_layer_kernel<G, FUSED>, kThreads,
+                                                              SmemLayout::total));
+    if (per_sm < 1) return SLICEMOE_E_UNSUPPORTED;
     attr_set = true;
   }
   cudaLaunchConfig_t cfg = {};
@@ -1319,6 +1340,17 @@ extern "C" int slicemoe_workspace_init(void* workspace, size_t workspace_bytes, 
   return SLICEMOE_OK;
 }
 
+extern "C" int slicemoe_workspace_set_wait(void* workspace, unsigned long long wait_cycles, unsigned extra_arrivals,
+                                           void* stream) {
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return SLICEMOE_E_INVALID_ARG;
+  WsHeader* h = reinterpret_cast<WsHeader*>(workspace);
+  cudaStream_t st = (cudaStream_t)stream;
+  // small host-to-device copies from pageable memory are staged by the runtime before the call returns
+  SM_CUDA_TRY(cudaMemcpyAsync(&h->wait_cycles, &wait_cycles, sizeof(wait_cycles), cudaMemcpyHostToDevice, st));
+  SM_CUDA_TRY(cudaMemcpyAsync(&h->extra_arrivals, &extra_arrivals, sizeof(extra_arrivals), cudaMemcpyHostToDevice, st));
+  return SLICEMOE_OK;
+}
+
 extern "C" int slicemoe_get_status(void* workspace, int* status_out, void* stream) {
   if (!workspace || !status_out) return SLICEMOE_E_INVALID_ARG;
   WsHeader* h = reinterpret_cast<WsHeader*>(workspace);
@@ -1373,12 +1405,14 @@ extern "C" int slicemoe_decode_step_host(const slicemoe_shape* shape, const slic
                                          size_t workspace_bytes, void* stream) {
   int rc = check_shape(shape);
   if (rc != SLICEMOE_OK) return rc;
-  if (!x_host || !logits_host || !y_host || !workspace || workspace_bytes < kWsBytes) return SLICEMOE_E_INVALID_ARG;
+  if (!x_host || !y_host || !workspace || workspace_bytes < kWsBytes) return SLICEMOE_E_INVALID_ARG;
   if (shape->n_experts > 512) return SLICEMOE_E_UNSUPPORTED;
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   cudaStream_t st = (cudaStream_t)stream;
   void* dx = ws + kWsStX;
-  float* dlogits = reinterpret_cast<float*>(ws + kWsStLogits);
+  // logits_host == NULL: the logits follow x in the caller's buffer (x_host is bf16 [hidden] then float32 [E]) and
+  // in the staging area alike, and one copy brings both
+  float* dlogits = reinterpret_cast<float*>(logits_host ? ws + kWsStLogits : ws + kWsStX + 2 * (size_t)shape->hidden);
   int32_t* dids = reinterpret_cast<int32_t*>(ws + kWsStIds);
   float* dw = reinterpret_cast<float*>(ws + kWsStW);
   uint8_t* dprec = ws + kWsStPrec;
@@ -1396,8 +1430,13 @@ extern "C" int slicemoe_decode_step_host(const slicemoe_shape* shape, const slic
       (void)cudaGetLastError();  // an unregistered pointer is not an error here
     }
   }
-  SM_CUDA_TRY(cudaMemcpyAsync(dx, x_host, 2 * (size_t)shape->hidden, cudaMemcpyHostToDevice, st));
-  SM_CUDA_TRY(cudaMemcpyAsync(dlogits, logits_host, 4 * (size_t)shape->n_experts, cudaMemcpyHostToDevice, st));
+  if (logits_host) {
+    SM_CUDA_TRY(cudaMemcpyAsync(dx, x_host, 2 * (size_t)shape->hidden, cudaMemcpyHostToDevice, st));
+    SM_CUDA_TRY(cudaMemcpyAsync(dlogits, logits_host, 4 * (size_t)shape->n_experts, cudaMemcpyHostToDevice, st));
+  } else {
+    SM_CUDA_TRY(cudaMemcpyAsync(dx, x_host, 2 * (size_t)shape->hidden + 4 * (size_t)shape->n_experts,
+                                cudaMemcpyHostToDevice, st));
+  }
   rc = slicemoe_layer_routed(shape, experts, shared, shared_gate_vec, dx, 1, dlogits, bias, renorm, tau, rank_high, dids,
                              dprec, dw, dy, workspace, workspace_bytes, stream);
   if (rc != SLICEMOE_OK) return rc;

@@ -1,6 +1,7 @@
 // Prefill of one MoE layer from bit-sliced AMAT weights: many tokens at once, so the expert FFN is a
-// genuine dense contraction (Section 3 of the paper: prefill loads every expert of a layer; Section 5.3:
-// prefill runs at the precision each expert's cached slices allow).
+// genuine dense contraction (Section 3 of the paper: prefill loads every expert of a layer).  Section 6.3 notes
+// that prefill wants high-bit computation; the per-expert precision flag here is this library's generalisation
+// (an expert can also be run from its MSB slice alone), which the mixed-precision prefill benchmark uses.
 //
 // Steps, all on the device:
 //   1. count the tokens of every routed expert, lay the experts' token rows out one after the other

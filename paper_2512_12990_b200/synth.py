@@ -8,7 +8,7 @@ identical bits, and neither side's code is involved in producing them.
 Every stream is a counter-based Philox generator keyed by (seed, stream id), so
 any array can be regenerated on its own without generating the ones before it.
 
-The two evaluated models (Section 5.1 of the paper: DeepSeek-V2-Lite and
+The two evaluated models (Section 6.1 of the paper: DeepSeek-V2-Lite and
 Qwen1.5-MoE-A2.7B) are represented by their MoE layer *shapes* only; weights are
 N(0, 0.02), activations N(0, 1) rounded to bf16, router logits as described per
 function.  No model weights and no benchmark items are used.

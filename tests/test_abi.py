@@ -73,5 +73,7 @@ def test_argument_errors_are_codes_not_faults():
     assert L.slicemoe_layer(ctypes.byref(q), one, None, one, one, 1, one, one, one, one, ws, big, None) == B.E_INVALID_ARG
     assert L.slicemoe_workspace_init(None, big, None) == B.E_INVALID_ARG
     assert L.slicemoe_get_status(None, None, None) == B.E_INVALID_ARG
+    assert L.slicemoe_workspace_set_wait(None, 1000, 0, None) == B.E_INVALID_ARG
+    assert L.slicemoe_workspace_set_wait(ctypes.c_void_p(8), 1000, 0, None) == B.E_INVALID_ARG   # not 256-byte aligned
     assert L.slicemoe_dbsc_create(-1, 1, 1, -1.0, 10) is None
     assert L.slicemoe_dbsc_request(None, 0, 0, 0, 0, None, None, None) == B.E_INVALID_ARG

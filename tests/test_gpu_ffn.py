@@ -153,6 +153,14 @@ def test_qwen_decode_layer_config():
     B.slicemoe_decode_step_host(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, xh.clone(), lh.clone(), yp, L.ws,
                                 tau=2.0, rank_high=0)
     assert torch.equal(yp, yh)
+    # x and the logits in ONE pinned buffer (logits_host = None): a single host-to-device copy, same bits
+    both = torch.empty(2 * sh.hidden + 4 * sh.n_experts, dtype=torch.uint8).pin_memory()
+    both[:2 * sh.hidden] = xh.view(torch.uint8)
+    both[2 * sh.hidden:] = lh.view(torch.uint8)
+    y1 = torch.empty(sh.hidden, dtype=torch.float32).pin_memory()
+    B.slicemoe_decode_step_host(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, both, None, y1, L.ws, tau=2.0,
+                                rank_high=0)
+    assert torch.equal(y1, yh)
 
 
 def test_bad_expert_id_is_skipped_and_reported():
