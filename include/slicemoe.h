@@ -192,6 +192,22 @@ int slicemoe_layer(const slicemoe_shape *shape, const slicemoe_expert *experts,
                    void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * slicemoe_layer_flags - slicemoe_layer with promises from the caller that let the kernel start earlier.
+ *   SLICEMOE_LISTS_RESIDENT  ids, prec and weights were complete in device memory before the work that precedes
+ *            this call on `stream` began (lists uploaded by the host after its cache decision, or prepared for
+ *            a whole run of layers ahead of time; NOT lists written by the kernel enqueued just before this call).
+ *            The kernel then reads them, and requests the routed experts' slices, while that preceding work is
+ *            still running; only x is waited for.  Results are the same bits as slicemoe_layer's.
+ * Without the flag the kernel still requests the shared experts' slices early: they follow from the shape alone.
+ * flags = 0 is slicemoe_layer.  Errors: as slicemoe_layer; INVALID_ARG for an unknown flag.
+ */
+#define SLICEMOE_LISTS_RESIDENT 1u
+int slicemoe_layer_flags(const slicemoe_shape *shape, const slicemoe_expert *experts,
+                         const slicemoe_expert *shared, const float *shared_gate_vec, const void *x, int T,
+                         const int32_t *ids, const uint8_t *prec, const float *weights, float *y,
+                         void *workspace, size_t workspace_bytes, unsigned flags, void *stream);
+
+/*
  * slicemoe_layer_routed - slicemoe_route_topk and slicemoe_layer in one kernel launch per token: the decode
  * kernel's prologue computes the routing list from the router logits with the arithmetic of
  * slicemoe_route_topk (same bits), takes the precision request as the precision list (Section 4.1: experts

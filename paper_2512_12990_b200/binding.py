@@ -27,7 +27,7 @@ DBSC_STAT_NAMES = ("requests", "msb_hit", "msb_miss", "lsb_hit", "lsb_miss", "ls
 EXPORTS = (
     "slicemoe_strerror", "slicemoe_version", "slicemoe_last_cuda_error", "slicemoe_plane_bytes", "slicemoe_meta_count", "slicemoe_pack",
     "slicemoe_unpack_plane", "slicemoe_unpack_meta", "slicemoe_route_topk", "slicemoe_workspace_bytes",
-    "slicemoe_workspace_init", "slicemoe_workspace_set_wait", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer",
+    "slicemoe_workspace_init", "slicemoe_workspace_set_wait", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer", "slicemoe_layer_flags",
     "slicemoe_decode_step_host", "slicemoe_layer_static", "slicemoe_layer_routed", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
     "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
     "slicemoe_dbsc_assign", "slicemoe_dbsc_stats", "slicemoe_dbsc_contains",
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
                                       c_void_p, c_void_p, c_size_t, c_void_p]
     L.slicemoe_layer.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                  c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.slicemoe_layer_flags.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
+                                       c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, ctypes.c_uint, c_void_p]
     L.slicemoe_layer_static.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                         c_void_p, c_void_p, c_void_p, c_void_p]
     L.slicemoe_decode_step_host.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -270,12 +272,22 @@ def slicemoe_expert_ffn(shape: Shape, experts_tbl, x, ids, prec, weights, ws, y=
     return y
 
 
+LISTS_RESIDENT = 1
+
+
 def slicemoe_layer(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x, ids, prec, weights, ws, y=None,
-                   stream=None):
+                   stream=None, flags=0):
+    """flags = 0 calls slicemoe_layer, anything else slicemoe_layer_flags."""
     import torch
     T = x.shape[0]
     if y is None:
         y = torch.empty((T, shape.hidden), dtype=torch.float32, device=x.device)
+    if flags:
+        rc = lib().slicemoe_layer_flags(ctypes.byref(shape), _ptr(experts_tbl), _ptr(shared_tbl), _ptr(shared_gate_vec),
+                                        _ptr(x), T, _ptr(ids), _ptr(prec), _ptr(weights), _ptr(y), _ptr(ws),
+                                        ws.numel(), flags, _stream(stream))
+        _check(rc, "slicemoe_layer_flags")
+        return y
     rc = lib().slicemoe_layer(ctypes.byref(shape), _ptr(experts_tbl), _ptr(shared_tbl), _ptr(shared_gate_vec),
                               _ptr(x), T, _ptr(ids), _ptr(prec), _ptr(weights), _ptr(y), _ptr(ws), ws.numel(),
                               _stream(stream))

@@ -99,6 +99,9 @@ struct DecodeParams {
   int n_experts, n_shared, k;
   int hidden, inter, shared_inter, group;
   int sigmoid_gate;
+  // the routing lists were complete before the work ahead of this kernel in the stream began: they are read, and
+  // the routed experts' tiles requested, while that work is still running
+  int lists_resident;
   // fused routing (logits != nullptr): the list is computed from the router logits in the prologue instead of
   // read from ids / prec / weights, and written to the *_out arrays (each may be null) by one CTA
   const float* logits;
@@ -121,7 +124,9 @@ struct Slot {
 };
 
 // The schedule of a CTA.
-//   phase 1: tasks n = 0 .. count1-1 are the (slot, 16-row block) pairs from (first_slot, first_idx) on.  A
+//   phase 1: tasks n = 0 .. count1-1 are (slot, 16-row block) pairs: first count_s tasks of the shared experts,
+//     from (slot_s, idx_s) on - this part follows from the shape alone, so its tiles can be requested before the
+//     routing list is known - then the routed tasks from (first_slot, first_idx) on.  A
 //     task of an 8-bit slot is 2 * nch chunks (gate then up; nch = 2048-column chunks of hidden), each two
 //     units (MSB tile, LSB tile); a task of a 4-bit slot is nch chunks, each two units (the gate's MSB tile
 //     and the up's).  Every phase-1 chunk takes two units.  Task n is consumed by group n % kGroups and
@@ -134,12 +139,12 @@ struct Slot {
 //     chunk (plane area, then scales at scale2_off, zero-points at zp2_off), so that more - for the
 //     benchmark shapes all - of the phase's tiles are in shared memory before h arrives.
 struct Plan {
+  int slot_s, idx_s, count_s;
   int first_slot, first_idx, count1;
   int count2;
   int nslots;
   int htotal;   // sum of the slots' intermediate widths
   float gate;   // sigmoid(gate_vec . x) when the shared experts are gated
-  int chunks1;  // chunks of phase 1
   int unit2_bytes, nunits2, scale2_off, zp2_off;
   short p2c[kMaxSlots + 1], p2u[kMaxSlots + 1];
 };
@@ -158,7 +163,7 @@ struct SmemLayout {
   static constexpr int slots = p2list + kConsumerWarps * kMaxMine * 16;
   static constexpr int plan = slots + kMaxSlots * (int)sizeof(Slot);
   static constexpr int bars = (plan + (int)sizeof(Plan) + 15) & ~15;  // uint64 barriers
-  static constexpr int nbars = 2 * kUnits + kGroups * kFull2PerGroup + kUnits2 + 2 * kGroups + 5;
+  static constexpr int nbars = 2 * kUnits + kGroups * kFull2PerGroup + kUnits2 + 2 * kGroups + 6;
   static constexpr int dead = bars + nbars * 8;  // int dead flag; 8 bytes on, the wait limit in cycles
   static constexpr int total = dead + 16;
 };
@@ -179,13 +184,16 @@ static_assert(SmemLayout::slots % 8 == 0 && SmemLayout::hdig % 16 == 0 && SmemLa
 //     empty2 barrier per unit (an arrive from each warp of the group that consumed it).
 // pfull1 / pempty1 per group (phase-1 partial rows to the epilogue warp and back), pfull2 / pempty2 (phase-2
 // partial rows of all warps), hx_go (h is complete in the workspace), hs_ready (h is in shared memory as
-// digits), p1_done (every consumer warp is through with phase 1, so the ring may be re-cut).
+// digits), p1_done (every consumer warp is through with phase 1, so the ring may be re-cut), plan_ready (the
+// routed part of the plan and the routed slots stand: the producers wait for it after the shared experts' tasks).
 struct Bars {
   static constexpr int full = 0, empty = kUnits, full2 = 2 * kUnits, empty2 = full2 + kGroups * kFull2PerGroup,
                        pfull1 = empty2 + kUnits2,
                        pempty1 = pfull1 + kGroups, pfull2 = pempty1 + kGroups, pempty2 = pfull2 + 1, hx_go = pfull2 + 2,
-                       hs_ready = pfull2 + 3, p1_done = pfull2 + 4;
+                       hs_ready = pfull2 + 3, p1_done = pfull2 + 4, plan_ready = pfull2 + 5, count = pfull2 + 6;
 };
+
+static_assert(Bars::count <= SmemLayout::nbars, "barrier storage");
 
 // ---- PTX helpers -------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -233,10 +241,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (mbar_try(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, dead, status);
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
+// Weights are used once per token: they go through L2 marked evict-first, so that the stream does not push out
+// what every launch uses again (the kernel's own instructions, expert tables, h).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+      : "memory");
 }
 __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
@@ -320,6 +336,27 @@ __device__ __forceinline__ void block_to_digits(const float (&v)[4], int k0, int
 // ---- schedule enumeration (identical in every role) ----------------------------------------------------
 __device__ __forceinline__ int nchunks_of(int K) { return (K + kChunkK - 1) / kChunkK; }
 enum ChunkMode { kModeSingle = 0, kModeBoth = 1, kModePair = 2 };
+
+// The phase-1 tasks of a CTA in order: `slot`, `idx` name task n once at(n) has been called for it.
+struct TaskWalk {
+  int slot, idx;
+  __device__ __forceinline__ void start(const Plan& plan) {
+    slot = plan.slot_s;
+    idx = plan.idx_s;
+  }
+  __device__ __forceinline__ void at(const Plan& plan, int n) {
+    if (n == plan.count_s) {  // the routed run begins
+      slot = plan.first_slot;
+      idx = plan.first_idx;
+    }
+  }
+  __device__ __forceinline__ void next(const Slot* slots) {
+    if (++idx >= slots[slot].inter / 16) {
+      idx = 0;
+      ++slot;
+    }
+  }
+};
 
 // ---- consumers -----------------------------------------------------------------------------------
 // Phase change: wait until the epilogue warp has seen the whole grid's h in the workspace, then turn it
@@ -482,11 +519,14 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
   const int nch = nchunks_of(p.hidden);
   const int prod = group % kProducers;  // the producer that serves this group
   {
-    int slot = plan.first_slot, idx = plan.first_idx, cn = 0;
+    TaskWalk tw;
+    tw.start(plan);
+    int cn = 0;
     int jp = 0;  // chunks of this group's producer so far (they fix the unit pair)
     int ig = 0;  // chunks of this group so far (they fix the full barrier)
     for (int n = 0; n < plan.count1; ++n) {
-      const Slot& sl = slots[slot];
+      tw.at(plan, n);
+      const Slot& sl = slots[tw.slot];
       const int nchunks = sl.prec ? 2 * nch : nch;
       if (n % kGroups == group) {
         float part0 = 0.f, part1 = 0.f, unused = 0.f;
@@ -522,10 +562,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
         jp += nchunks;  // the other group this producer serves
       }
       cn += nchunks;
-      if (++idx >= sl.inter / 16) {
-        idx = 0;
-        ++slot;
-      }
+      tw.next(slots);
     }
   }
   __syncwarp();
@@ -637,8 +674,11 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
   };
   // phase 1: one group's four partial rows per task -> SwiGLU -> h
   {
-    int slot = plan.first_slot, idx = plan.first_idx;
+    TaskWalk tw;
+    tw.start(plan);
     for (int n = 0; n < plan.count1; ++n) {
+      tw.at(plan, n);
+      const int slot = tw.slot, idx = tw.idx;
       const int group = n % kGroups, round = n / kGroups;
       if (!mbar_wait(bars + 8 * (Bars::pfull1 + group), round & 1, dead, status)) {
         depart();  // a wait ran out: the others will time out at the barrier, the header is still handed back
@@ -656,10 +696,7 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + 8 * (Bars::pempty1 + group));
       if (lane < 16) p.ws_h[slots[slot].hoff + idx * 16 + lane] = a / (1.f + expf(-a)) * b;  // silu(gate) * up
-      if (++idx >= slots[slot].inter / 16) {
-        idx = 0;
-        ++slot;
-      }
+      tw.next(slots);
     }
   }
   // ---- the single grid-wide dependency: every CTA has written its rows of h ----
@@ -730,13 +767,31 @@ struct ChunkSpace {
   uint32_t empty_bar_first, empty_parity_first;  // phase 2, two-unit chunks: the first unit has a barrier of its own
 };
 
+// What a producer needs to wait: it starts before the kernels ahead of this one in the stream have completed, so
+// a wait that does not pass at once is first the moment to wait for those (the consumers, on whom all of a
+// producer's barriers depend, do not start earlier; and a bounded wait's clock must not run while an earlier
+// kernel is still busy).
+struct ProducerWait {
+  volatile int* dead;
+  unsigned* status;
+  bool dep_waited;  // griddepcontrol.wait has been executed
+  __device__ __forceinline__ bool operator()(uint32_t bar, uint32_t parity) {
+    if (mbar_try(bar, parity)) return true;
+    if (!dep_waited) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      dep_waited = true;
+    }
+    return mbar_wait(bar, parity, dead, status);
+  }
+};
+
 // One chunk of matrix A - or of matrices A and B side by side - of (slot, row block rb), columns from k0, into
 // the space `cs`.  Run by the first kProducerLanes lanes of a producer warp together.  Returns false if a
 // wait ran out.
 template <int G>
 __device__ __forceinline__ bool produce_chunk(uint8_t* smem, const RingView& rv, const ChunkSpace& cs, int lane,
                                               const ProducerLane& pl, const Slot& s, int matA, int matB, int mode, int K,
-                                              int rb, int k0, volatile int* dead, unsigned* status) {
+                                              int rb, int k0, ProducerWait& pw, uint64_t pol) {
   constexpr int LG = G == 128 ? 7 : (G == 64 ? 6 : 5);
   const bool two = mode != kModeSingle;
   bool active;
@@ -746,7 +801,7 @@ __device__ __forceinline__ bool produce_chunk(uint8_t* smem, const RingView& rv,
     src = mode == kModePair ? s.ptr[matB][0] : s.ptr[matA][1];
     if (mode == kModeBoth && src == nullptr) {  // 8 bits asked of an expert without LSB planes: defined garbage, reported
       src = s.ptr[matA][0];
-      atomicOr(status, (unsigned)SLICEMOE_STATUS_MISSING_LSB);
+      atomicOr(pw.status, (unsigned)SLICEMOE_STATUS_MISSING_LSB);
     }
   } else if (lane >= 4) {
     active = mode == kModePair;
@@ -758,8 +813,8 @@ __device__ __forceinline__ bool produce_chunk(uint8_t* smem, const RingView& rv,
   src += (size_t)((unsigned)rb * (unsigned)(K >> 7) + (unsigned)(k0 >> 7)) * pl.bytes_per_block;
   const uint32_t nblk = (uint32_t)(min(kChunkK, K - k0) >> 7);
   // The two units of a phase-2 chunk may last have held chunks of different consumer groups: both must be free.
-  if (cs.empty_bar_first != 0u && !mbar_wait(cs.empty_bar_first, cs.empty_parity_first, dead, status)) return false;
-  if (!mbar_wait(cs.empty_bar, cs.empty_parity, dead, status)) return false;
+  if (cs.empty_bar_first != 0u && !pw(cs.empty_bar_first, cs.empty_parity_first)) return false;
+  if (!pw(cs.empty_bar, cs.empty_parity)) return false;
   const uint32_t bar = cs.full_bar;
   if (lane == 0)
     mbar_arrive_expect_tx(bar, nblk * ((two ? 2048u : 1024u) + (mode == kModePair ? 2u : 1u) * ((128u >> LG) * 48u)));
@@ -767,7 +822,7 @@ __device__ __forceinline__ bool produce_chunk(uint8_t* smem, const RingView& rv,
   if (active) {
     const uint32_t u = (uint32_t)(pl.second_unit ? cs.u1 : cs.u0);
     const uint32_t dst_in_unit = pl.field < 2 ? 0u : (pl.field == 2 ? rv.scale_off : rv.zp_off);
-    bulk_g2s(smem_u32(smem + SmemLayout::ring) + u * rv.unit_bytes + dst_in_unit, src, nblk * pl.bytes_per_block, bar);
+    bulk_g2s(smem_u32(smem + SmemLayout::ring) + u * rv.unit_bytes + dst_in_unit, src, nblk * pl.bytes_per_block, bar, pol);
   }
   return true;
 }
@@ -780,7 +835,11 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
   const Plan& plan = *reinterpret_cast<const Plan*>(smem + SmemLayout::plan);
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
-  unsigned* status = &p.ws->status;
+  ProducerWait pw;
+  pw.dead = dead;
+  pw.status = &p.ws->status;
+  pw.dep_waited = false;
+  const uint64_t pol = l2_evict_first_policy();
   ProducerLane pl;
   pl.field = lane < 2 ? lane : 2 + (lane & 1);  // lanes 2, 4: scales; lanes 3, 5: zero-points
   pl.bytes_per_block = lane < 2 ? 1024u : (pl.field == 2 ? (128u >> LG) * 32u : (128u >> LG) * 16u);
@@ -795,9 +854,21 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
   static_assert(kGroups == 2 * kProducers, "a producer serves the groups `which` and `which + kProducers`");
   int ig_lo = 0, ig_hi = 0;  // chunks armed so far for group `which` and for group `which + kProducers`
   {
-    int slot = plan.first_slot, idx = plan.first_idx;
+    TaskWalk tw;
+    tw.start(plan);
     int jp = 0;  // this warp's chunks so far
-    for (int n = 0; n < plan.count1 && ok; ++n) {
+    // The shared experts' tasks are known from the start; what follows them - and how many tasks there are - once
+    // the plan stands.
+    int n_end = plan.count_s;
+    for (int n = 0; ok; ++n) {
+      if (n == plan.count_s) {
+        ok = pw(bars + 8 * Bars::plan_ready, 0);
+        if (!ok) break;
+        n_end = plan.count1;
+      }
+      if (n >= n_end) break;
+      tw.at(plan, n);
+      const int slot = tw.slot, idx = tw.idx;
       const Slot& s = slots[slot];
       const int nchunks = s.prec ? 2 * nch : nch;
       if (n % kProducers == which) {
@@ -815,13 +886,10 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
           cs.full_bar = bars + 8 * (Bars::full + 2 * g + (igg & 1));
           ++igg;
           ok = produce_chunk<G>(smem, r1, cs, lane, pl, s, mat, s.prec ? mat : 1, s.prec ? kModeBoth : kModePair, p.hidden,
-                                idx, (q % nch) * kChunkK, dead, status);
+                                idx, (q % nch) * kChunkK, pw, pol);
         }
       }
-      if (++idx >= s.inter / 16) {
-        idx = 0;
-        ++slot;
-      }
+      tw.next(slots);
     }
   }
   // phase 2: down rows of every slot for the output row blocks of this CTA, in the re-cut ring
@@ -831,7 +899,7 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
   r2.zp_off = (uint32_t)plan.zp2_off;
   // The re-cut units lie over the phase-1 units: nothing of phase 2 lands before phase 1 has been consumed.
   // (From then until h has crossed the grid the memory system has nothing else to do.)
-  if (ok && plan.count2 > 0) ok = mbar_wait(bars + 8 * Bars::p1_done, 0, dead, status);
+  if (ok && plan.count2 > 0) ok = pw(bars + 8 * Bars::p1_done, 0);
   const int half = plan.nunits2 / kProducers;  // this warp's units are [which * half, which * half + half)
   int c2 = 0, xp = 0;                           // chunks of the phase so far, units this warp has handed out
   for (int m = 0; m < plan.count2 && ok; ++m) {
@@ -852,7 +920,7 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
         cs.empty_parity_first = ((xp / half) & 1) ^ 1;
         cs.full_bar = bars + 8 * (Bars::full2 + kFull2PerGroup * g + ig % kFull2PerGroup);
         xp += w;
-        ok = produce_chunk<G>(smem, r2, cs, lane, pl, s, 2, 2, s.prec ? kModeBoth : kModeSingle, s.inter, rb, k0, dead, status);
+        ok = produce_chunk<G>(smem, r2, cs, lane, pl, s, 2, 2, s.prec ? kModeBoth : kModeSingle, s.inter, rb, k0, pw, pol);
       }
     }
   }
@@ -939,11 +1007,32 @@ __device__ __forceinline__ void plan_units2(const DecodeParams& p, Plan* plan, i
   plan->unit2_bytes = (maxblk * (1024 + meta_blk * 3) + 127) & ~127;
   plan->nunits2 = min(kUnits2, (kUnits * kUnitBytes) / plan->unit2_bytes);
 }
-__device__ void build_plan_static(const DecodeParams& p, uint8_t* smem) {
+// Shared-expert tasks before CTA c when the grid's T1 of them are dealt out evenly.
+__device__ __forceinline__ unsigned shared_before(unsigned c, unsigned T1, unsigned P) {
+  return (unsigned)((unsigned long long)c * T1 / P);
+}
+// Run by warp 0.
+__device__ void build_plan_static(const DecodeParams& p, uint8_t* smem, int lane) {
+  Slot* slots = reinterpret_cast<Slot*>(smem + SmemLayout::slots);
   Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
+  if (lane < p.n_shared) {
+    Slot& s = slots[lane];
+    s.inter = p.shared_inter;
+    s.prec = 1;
+    s.coef = 1.f;
+    s.gated = p.sigmoid_gate;
+    s.hoff = lane * p.shared_inter;
+  }
+  if (lane != 0) return;
   const int nrb = p.hidden / 16;
   plan->count2 = (int)blockIdx.x < nrb ? (nrb - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
   plan_units2(p, plan, phase2_unit_blocks(p, p.k > 0));
+  // this CTA's share of the shared experts' phase-1 tasks
+  const unsigned nts = p.n_shared ? (unsigned)p.shared_inter / 16u : 0u, T1 = (unsigned)p.n_shared * nts;
+  const unsigned lo = shared_before(blockIdx.x, T1, gridDim.x), hi = shared_before(blockIdx.x + 1u, T1, gridDim.x);
+  plan->slot_s = nts ? (int)(lo / nts) : 0;
+  plan->idx_s = nts ? (int)(lo % nts) : 0;
+  plan->count_s = (int)(hi - lo);
 }
 
 // Warp 0: slot table (all but the pointers) and the static partition, in closed form: the phase-1 unit
@@ -961,14 +1050,6 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
     s.coef = rt.w;
     s.gated = 0;
     s.hoff = p.n_shared * p.shared_inter + (rt.pos - p.n_shared) * p.inter;
-  }
-  if (lane >= 16 && lane - 16 < p.n_shared) {
-    Slot& s = slots[lane - 16];
-    s.inter = p.shared_inter;
-    s.prec = 1;
-    s.coef = 1.f;
-    s.gated = p.sigmoid_gate;
-    s.hoff = (lane - 16) * p.shared_inter;
   }
   const int nslots = p.n_shared + rt.nbig + rt.nsmall;
   // phase-2 chunk and unit counts before each slot: lane j handles slot j (8-bit: shared and the first nbig routed)
@@ -999,38 +1080,29 @@ __device__ void build_plan(const DecodeParams& p, uint8_t* smem, int lane) {
     const unsigned nsh = (unsigned)p.n_shared, nbig = (unsigned)rt.nbig, nsmall = (unsigned)rt.nsmall;
     const unsigned nts = nsh ? (unsigned)p.shared_inter / 16u : 0u, ntr = (unsigned)p.inter / 16u;
     const unsigned nch = (unsigned)nchunks_of(p.hidden);
-    const unsigned spb = 4u * nch, sps = 2u * nch;  // units per 8-bit / 4-bit task
+    const unsigned spb = 4u * nch, sps = 2u * nch;  // units per 8-bit / 4-bit task (shared tasks are 8-bit)
     const unsigned T1 = nsh * nts, T2 = nbig * ntr, T3 = nsmall * ntr;  // tasks per run
     const unsigned U1 = T1 * spb, U2 = T2 * spb, S = U1 + U2 + T3 * sps;
     const unsigned spmax = (nsh + nbig) ? spb : sps;
+    // Every CTA gets T units of work: its shared tasks (dealt out evenly, build_plan_static) and a window of the
+    // routed unit sequence that fills the rest.  T and every shared share are multiples of the larger task size,
+    // and the larger routed tasks come first, so the windows are cut at task boundaries.
     const unsigned T = ((S + gridDim.x - 1) / gridDim.x + spmax - 1) / spmax * spmax;
-    // ordinal of the first task that starts at or after a unit offset
+    const unsigned UR = U2 + T3 * sps;  // the routed sequence
+    // ordinal of the first routed task that starts at or after a unit offset of the routed sequence
     auto ord_of = [&](unsigned bound) -> unsigned {
-      if (bound >= S) return T1 + T2 + T3;
-      if (bound < U1) return (bound + spb - 1) / spb;
-      if (bound < U1 + U2) return T1 + (bound - U1 + spb - 1) / spb;
-      return T1 + T2 + (bound - U1 - U2 + sps - 1) / sps;
+      if (bound >= UR) return T2 + T3;
+      if (bound < U2) return (bound + spb - 1) / spb;
+      return T2 + (bound - U2 + sps - 1) / sps;
     };
     // both ends of this CTA's window at once: lane 1 takes the upper one
-    const unsigned lo = blockIdx.x * T;
-    const unsigned o = ord_of(lo + (lane & 1) * T);
+    const unsigned cc = blockIdx.x + (unsigned)(lane & 1);
+    const unsigned o = ord_of(cc * T - spb * shared_before(cc, T1, gridDim.x));
     const unsigned o0 = __shfl_sync(0xffffffffu, o, 0), o1 = __shfl_sync(0xffffffffu, o, 1);
     if (lane != 0) return;
-    int slot, idx;
-    if (o0 < T1) {
-      slot = (int)(o0 / nts);
-      idx = (int)(o0 % nts);
-    } else {
-      slot = (int)(nsh + (o0 - T1) / ntr);
-      idx = (int)((o0 - T1) % ntr);
-    }
-    plan->first_slot = slot;
-    plan->first_idx = idx;
-    plan->count1 = (int)(o1 - o0);
-    // phase-1 chunks of this CTA: 2 nch per 8-bit task, nch per 4-bit task
-    const unsigned big_end = T1 + T2;
-    const unsigned nb = (o0 < big_end ? (o1 < big_end ? o1 : big_end) - o0 : 0u);
-    plan->chunks1 = (int)(nb * 2u * nch + ((o1 - o0) - nb) * nch);
+    plan->first_slot = (int)(nsh + o0 / ntr);
+    plan->first_idx = (int)(o0 % ntr);
+    plan->count1 = plan->count_s + (int)(o1 - o0);
     if (nslots == 0) plan->count2 = 0;  // otherwise as build_plan_static left it
     plan->nslots = nslots;
     plan->htotal = (int)(nsh * (unsigned)p.shared_inter + (nbig + nsmall) * (unsigned)p.inter);
@@ -1086,10 +1158,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
   Plan* plan = reinterpret_cast<Plan*>(smem + SmemLayout::plan);
 
   // Programmatic dependent launch: the next kernel in the stream may start launching as soon as every CTA
-  // of this grid has got here (its CTAs find room only where one of ours has exited), and this kernel sets
-  // up its barriers before it waits for the grids before it.  Nothing an earlier kernel may write is touched
-  // before that wait: routing lists, x and the workspace may still be in use by the previous kernels.
+  // of this grid has got here (its CTAs find room only where one of ours has exited), and this kernel does
+  // all it can before it waits for the grids before it.  Nothing an earlier kernel may write is touched
+  // before that wait: x and the workspace always, and the routing lists unless the caller has promised that
+  // they were complete earlier (lists_resident).  The weights, the expert tables and the shape are never written
+  // by a kernel in flight.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const bool early_lists = !FUSED && p.lists_resident != 0;
   if (warp == kProducerWarp) {
     if (lane == 0) {
       *reinterpret_cast<int*>(smem + SmemLayout::dead) = 0;
@@ -1110,34 +1185,52 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
       mbar_init(bars + 8 * Bars::hx_go, 1);
       mbar_init(bars + 8 * Bars::hs_ready, kConsumerWarps);
       mbar_init(bars + 8 * Bars::p1_done, kConsumerWarps);
+      mbar_init(bars + 8 * Bars::plan_ready, early_lists ? 2 : 1);  // resident lists: warps 0 and 1 each say when done
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
   }
-  // Also ahead of the wait, because it reads nothing an earlier kernel writes: the shape-only part of the plan,
-  // and the routed experts' pointer table on its way into L2 (warp 1 reads k of its entries right after the wait).
+  // Ahead of the wait: what follows from the shape alone - the shared experts' slots, pointers and this CTA's share
+  // of their tasks - and the routed experts' pointer table on its way into L2 (its entries are read right after the
+  // wait).
   if (warp == 0) {
-    if (lane == 0) build_plan_static(p, smem);
-  } else if (warp == 1 && p.experts != nullptr && p.k > 0) {
+    build_plan_static(p, smem, lane);
+  } else if (warp == 1 && p.experts != nullptr && p.k > 0 && !early_lists) {
     const char* tab = reinterpret_cast<const char*>(p.experts);
     const size_t bytes = (size_t)p.n_experts * sizeof(slicemoe_expert);
     for (size_t off = (size_t)lane * 128; off < bytes; off += 32 * 128)
       asm volatile("prefetch.global.L2 [%0];" ::"l"(tab + off));
-  }
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-
-  // Prologue, all roles in parallel and one barrier at the end: warp 0 reads the routing list and builds
-  // the slot table and the partition; warps 1 and 2 fetch the routed and the shared experts' plane
-  // pointers; the next 14 warps turn x into digits, one 128-element block at a time; the last warp sets
-  // up the barriers and the shared-expert gate.
-  if (warp == 0) {
-    build_plan<FUSED>(p, smem, lane);
-  } else if (warp == 1) {
-    load_slot_pointers<FUSED>(p, smem, lane, true);
   } else if (warp == 2) {
     if (p.n_shared > 0) load_slot_pointers<FUSED>(p, smem, lane, false);
-  } else if (warp == kProducerWarp) {
-    if (lane == 0) {  // a wait limit set by the host for this workspace (the thread that wrote the default)
+  }
+  __syncthreads();
+  const uint32_t plan_ready = smem_u32(smem + SmemLayout::bars) + 8 * Bars::plan_ready;
+  if (warp >= kProducerWarp) {
+    // The producers start on the shared experts' tiles (and, with resident lists, go on to the routed experts')
+    // while the kernels ahead are still running; see ProducerWait for where they wait for those.
+    if (lane < kProducerLanes) producer_loop<G>(p, smem, lane, warp - kProducerWarp);
+    return;
+  }
+
+  // Everyone else waits here.  Then, in parallel and with one barrier (of these 17 warps) at the end: warp 0 reads
+  // the routing list and builds the routed slots and the partition, warp 1 fetches the routed experts' plane
+  // pointers, warp 2 takes the wait limit and the shared-expert gate, the other 14 warps turn x into digits, one
+  // 128-element block at a time.
+  // (With resident lists warps 0 and 1 do their part first, while the producers are already busy with the shared
+  // experts' tiles, and tell the producers themselves.)
+  if (early_lists && warp < 2) {
+    if (warp == 0) build_plan<FUSED>(p, smem, lane);
+    else load_slot_pointers<FUSED>(p, smem, lane, true);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(plan_ready);
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (warp == 0) {
+    if (!early_lists) build_plan<FUSED>(p, smem, lane);
+  } else if (warp == 1) {
+    if (!early_lists) load_slot_pointers<FUSED>(p, smem, lane, true);
+  } else if (warp == 2) {
+    if (lane == 0) {  // a wait limit set by the host for this workspace
       const unsigned long long lim = p.ws->wait_cycles;
       if (lim != 0ull) *reinterpret_cast<unsigned long long*>(smem + SmemLayout::dead + 8) = lim;
     }
@@ -1155,9 +1248,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
       if (lane == 0) plan->gate = 1.f / (1.f + expf(-dot));
     }
   } else {
-    // warps 3 .. 16 and the second producer warp
-    const int nw = kConsumerWarps - 2 + kProducers - 1;
-    for (int blk = (warp > kProducerWarp ? warp - 1 : warp) - 3; blk < p.hidden / 128; blk += nw) {
+    // warps 3 .. 16
+    constexpr int nw = kConsumerWarps + 1 - 3;
+    for (int blk = warp - 3; blk < p.hidden / 128; blk += nw) {
       const uint2 raw = *reinterpret_cast<const uint2*>(p.x + blk * 128 + 4 * lane);
       const float v[4] = {__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u),
                           __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u)};
@@ -1165,16 +1258,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
                          reinterpret_cast<float*>(smem + SmemLayout::xinv));
     }
   }
-  __syncthreads();
+  asm volatile("bar.sync 1, %0;" ::"n"(32 * (kConsumerWarps + 1)) : "memory");
+  if (!early_lists && tid == 0) mbar_arrive(plan_ready);
   if (plan->nslots == 0 && blockIdx.x == 0)
-    for (int i = tid; i < p.hidden; i += kThreads) p.y[i] = 0.f;
+    for (int i = tid; i < p.hidden; i += 32 * (kConsumerWarps + 1)) p.y[i] = 0.f;
 
   if (warp < kConsumerWarps) {
     consumer_loop<G>(p, smem, warp, lane);
-  } else if (warp == kEpilogueWarp) {
+  } else {
     epilogue_loop(p, smem, lane);
-  } else if (lane < kProducerLanes) {
-    producer_loop<G>(p, smem, lane, warp - kProducerWarp);
   }
 }
 
@@ -1252,12 +1344,13 @@ struct FusedRouting {
 static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts, const slicemoe_expert* shared,
                      int n_shared, const float* gate_vec, const void* x, int T, const int32_t* ids,
                      const uint8_t* prec, const float* weights, float* y, void* workspace, size_t workspace_bytes,
-                     void* stream, const FusedRouting* fused = nullptr) {
+                     void* stream, const FusedRouting* fused = nullptr, unsigned flags = 0u) {
   int rc = check_shape(shape);
   if (rc != SLICEMOE_OK) return rc;
   if (!experts || !x || !y || !workspace || T <= 0) return SLICEMOE_E_INVALID_ARG;
   if (fused ? !fused->logits : (!ids || !prec || !weights)) return SLICEMOE_E_INVALID_ARG;
   if (fused && shape->n_experts > 32 * ROUTE_MAX_VPT) return SLICEMOE_E_UNSUPPORTED;
+  if ((flags & ~(unsigned)SLICEMOE_LISTS_RESIDENT) != 0u || (fused && flags != 0u)) return SLICEMOE_E_INVALID_ARG;
   if (n_shared > 0 && !shared) return SLICEMOE_E_INVALID_ARG;
   if (n_shared > 0 && shape->shared_sigmoid_gate && !gate_vec) return SLICEMOE_E_INVALID_ARG;
   if (workspace_bytes < kWsBytes || (reinterpret_cast<uintptr_t>(workspace) & 255)) return SLICEMOE_E_INVALID_ARG;
@@ -1284,6 +1377,7 @@ static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts
   p.shared_inter = n_shared > 0 ? shape->shared_inter : 0;
   p.group = shape->group;
   p.sigmoid_gate = (n_shared > 0 && shape->shared_sigmoid_gate) ? 1 : 0;
+  p.lists_resident = (flags & SLICEMOE_LISTS_RESIDENT) ? 1 : 0;
   cudaStream_t st = (cudaStream_t)stream;
   p.logits = nullptr;
   p.bias = fused ? fused->bias : nullptr;
@@ -1377,6 +1471,15 @@ extern "C" int slicemoe_layer(const slicemoe_shape* shape, const slicemoe_expert
   if (!shape) return SLICEMOE_E_INVALID_ARG;
   return run_layer(shape, experts, shared, shape->n_shared, shared_gate_vec, x, T, ids, prec, weights, y, workspace,
                    workspace_bytes, stream);
+}
+
+extern "C" int slicemoe_layer_flags(const slicemoe_shape* shape, const slicemoe_expert* experts,
+                                    const slicemoe_expert* shared, const float* shared_gate_vec, const void* x, int T,
+                                    const int32_t* ids, const uint8_t* prec, const float* weights, float* y,
+                                    void* workspace, size_t workspace_bytes, unsigned flags, void* stream) {
+  if (!shape) return SLICEMOE_E_INVALID_ARG;
+  return run_layer(shape, experts, shared, shape->n_shared, shared_gate_vec, x, T, ids, prec, weights, y, workspace,
+                   workspace_bytes, stream, nullptr, flags);
 }
 
 extern "C" int slicemoe_layer_routed(const slicemoe_shape* shape, const slicemoe_expert* experts,

@@ -276,3 +276,33 @@ def test_maximum_sizes_of_the_decode_kernel():
     assert ei.value.code == B.E_UNSUPPORTED
     torch.cuda.synchronize()
     assert B.slicemoe_get_status(L.ws) == 0
+
+
+@pytest.mark.parametrize("name", ["tiny", "dsv2", "qwen"])
+def test_resident_lists_give_the_same_bits(name):
+    """slicemoe_layer_flags(SLICEMOE_LISTS_RESIDENT): the kernel plans and requests the routed tiles before the
+    work ahead of it has finished.  A chain of launches over several tokens (each launch overlaps the one before)
+    must give, bit for bit, what slicemoe_layer gives - and what the oracle gives within the tolerance."""
+    from paper_2512_12990_b200 import binding as B
+    torch = _torch()
+    sh = synth.SHAPES[name]
+    T = 6
+    logits = synth.router_logits_normal(sh.seed, ("resident-logits",), T, sh.n_experts)
+    ids, w, _ = moe.route_topk(logits, sh.top_k)
+    prec = (np.arange(sh.top_k)[None, :] < (1 + np.arange(T)[:, None]) % (sh.top_k + 1)).astype(np.uint8)
+    L = H.Layer(sh, sorted(set(ids.ravel().tolist())))
+    xbits, x64 = H.x_inputs(sh, T, "resident-x")
+    x = H.to_dev_bf16(xbits)
+    args = (_dev(ids.astype(np.int32)), _dev(prec), _dev(w.astype(np.float32)))
+    torch.cuda.synchronize()   # the lists are complete before anything of the chain is enqueued
+    y0 = B.slicemoe_layer(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, *args, L.ws)
+    y1 = B.slicemoe_layer(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, *args, L.ws,
+                          flags=B.LISTS_RESIDENT)
+    torch.cuda.synchronize()
+    assert B.slicemoe_get_status(L.ws) == 0
+    assert torch.equal(y0, y1)
+    y_ref = moe.layer(x64, L.oracle_list(), ids, prec, w, shared=L.oracle_shared, shared_gate_vec=L.gate_vec)
+    H.assert_close(y1.cpu().numpy(), y_ref, f"{name} resident lists")
+    # an unknown flag is refused
+    with pytest.raises(B.SliceMoEError):
+        B.slicemoe_layer(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, *args, L.ws, flags=2)
