@@ -11,11 +11,17 @@ independently packed layers, so the ~58 MB a step reads were last touched hundre
 earlier: the weight stream comes from HBM, not from L2.
 
 Reported (one JSON line on rank 0):
-  value      us per MoE layer, inputs resident in HBM, K steps replayed as CUDA graphs
-  e2e        the same through slicemoe_decode_step_host: pinned host x/logits in, host y out, every step
+  value      us per MoE layer, inputs resident in HBM, K steps replayed as CUDA graphs.  Whatever K is, the
+             K-step region is repeated until the leg holds half a second of device time; the value is the
+             median over the repetitions (`timing` gives their number, the fastest and the slowest)
+  e2e        the same through slicemoe_decode_step_host: one pinned host buffer (x, logits) in, host y out, every step
   roofline   the decode kernel alone: algorithmic bytes (slice planes read + scales + zero-points)
-             per launch / its average duration, against the measured HBM copy bandwidth
+             per launch / its average duration, against the measured HBM copy bandwidth; `traffic` comes from the
+             tracked ncu record under profiles/ and is null when decode.cu has changed since the capture
+  stream_only_us   the same bytes through the same bulk copies with no arithmetic (slicemoe_stream_probe)
   cpu_baseline   the CPU oracle timed on this host on a few steps of the same workload
+  workloads  (one GPU, default workload) short legs of the Qwen-shaped decode layer, the 26-layer decode stack and
+             the prefill layer, each with its own value, roofline and clock record
 With --gpus N > 1 (under torchrun) every rank runs an independent replica of the same job (the
 path has no exchange step); the time is the max over ranks and the value counts all ranks' steps.
 """
@@ -41,9 +47,6 @@ RANK_HIGH = 3          # of the 6 selected experts the 3 with the highest gating
 POOL = 1024            # distinct step inputs (x, logits); step s uses input s % POOL
 GRAPH_CHUNK = 1000     # steps per captured CUDA graph
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode-kernel launch on this workload, from the
-# ncu capture summarised under profiles/; None once the kernel has changed since the capture.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 58530000
 
 
 def expert_bytes(hidden: int, inter: int, group: int, prec8: bool) -> int:
@@ -53,9 +56,9 @@ def expert_bytes(hidden: int, inter: int, group: int, prec8: bool) -> int:
     return 3 * ((2 if prec8 else 1) * (w // 2) + (w // group) * 3)
 
 
-def step_bytes(sh) -> int:
-    b = RANK_HIGH * expert_bytes(sh.hidden, sh.inter, sh.group, True)
-    b += (sh.top_k - RANK_HIGH) * expert_bytes(sh.hidden, sh.inter, sh.group, False)
+def step_bytes(sh, rank_high: int = RANK_HIGH) -> int:
+    b = rank_high * expert_bytes(sh.hidden, sh.inter, sh.group, True)
+    b += (sh.top_k - rank_high) * expert_bytes(sh.hidden, sh.inter, sh.group, False)
     b += sh.n_shared * expert_bytes(sh.hidden, sh.shared_inter, sh.group, True)
     return b
 
@@ -172,7 +175,7 @@ def oracle_layer_inputs(sh, step: int):
     return logits, x64, experts, shared
 
 
-def oracle_step(sh, logits, x64, experts, shared, units=None):
+def oracle_step(sh, logits, x64, experts, shared, units=None, rank_high: int = RANK_HIGH):
     """The oracle's hot path for one token: route, precision request, mixed-precision layer.
 
     `units` bounds the work for sampling (None = the whole step): a pair (n_experts, rows) evaluates only
@@ -184,7 +187,7 @@ def oracle_step(sh, logits, x64, experts, shared, units=None):
     if isinstance(shared, tuple):        # shared experts scaled by sigmoid(v . x)
         shared, gate_vec = shared
     ids, w, _ = moe.route_topk(logits, sh.top_k)
-    prec = moe.precision_request(w, 2.0, rank_high=RANK_HIGH)
+    prec = moe.precision_request(w, 2.0, rank_high=rank_high)
     if units is None:
         return moe.layer(x64, experts, ids, prec, w, shared=shared, shared_gate_vec=gate_vec)
     n_exp, rows = units
@@ -215,7 +218,7 @@ def blas_threads() -> int:
         return 1
 
 
-def cpu_baseline(sh, budget_s: float = 15.0):
+def cpu_baseline(sh, rank_high: int = RANK_HIGH, budget_s: float = 15.0):
     """The oracle as it stands on whole steps of the workload, about `budget_s` seconds of CPU work."""
     times = []
     t_all = time.perf_counter()
@@ -223,7 +226,7 @@ def cpu_baseline(sh, budget_s: float = 15.0):
     while True:
         inp = oracle_layer_inputs(sh, step)
         t0 = time.perf_counter()
-        oracle_step(sh, *inp)
+        oracle_step(sh, *inp, rank_high=rank_high)
         times.append(time.perf_counter() - t0)
         step += 1
         if step >= 2 and (time.perf_counter() - t_all > budget_s or step >= 8):
@@ -232,10 +235,10 @@ def cpu_baseline(sh, budget_s: float = 15.0):
     return {"value": med * 1e6, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
             "sample": f"{len(times)} whole steps (route + {sh.top_k} routed + {sh.n_shared} shared experts, float64 numpy), "
                       f"median; packing excluded; host has {os.cpu_count()} logical cores",
-            "gbs": step_bytes(sh) / med / 1e9}
+            "gbs": step_bytes(sh, rank_high) / med / 1e9}
 
 
-def run_reference(args, sh):
+def run_reference(args, sh, workload: str = WORKLOAD, rank_high: int = RANK_HIGH, metric: str = METRIC):
     """--impl reference: the CPU oracle timed on the host cores, same metric and workload.  Each step is
     a bounded sample of one whole step, sized so that K + W steps end within a few minutes, and scaled
     back to a whole layer by the share of (expert, row-group) units it covered."""
@@ -245,7 +248,7 @@ def run_reference(args, sh):
     K, W = args.steps, args.warmup
     inp = oracle_layer_inputs(sh, 0)
     t0 = time.perf_counter()
-    oracle_step(sh, *inp)
+    oracle_step(sh, *inp, rank_high=rank_high)
     t_full = time.perf_counter() - t0
     budget = 150.0
     n_all = sh.top_k + sh.n_shared
@@ -266,19 +269,19 @@ def run_reference(args, sh):
                 n_exp += 1
             units = (n_exp, max(widths))
     for _ in range(W):
-        oracle_step(sh, *inp, units=units)
+        oracle_step(sh, *inp, units=units, rank_high=rank_high)
     t0 = time.perf_counter()
     for _ in range(K):
-        oracle_step(sh, *inp, units=units)
+        oracle_step(sh, *inp, units=units, rank_high=rank_high)
     dt = (time.perf_counter() - t0) / max(K, 1)
     val = dt * total_units / covered * 1e6
     sample = "whole steps (route + all routed and shared experts of one token)" if units is None else (
         f"each step = route + the first {units[0]} expert(s) of one token restricted to {min(units[1], sh.inter)} "
         f"intermediate rows ({covered} of {total_units} expert x row-group units), scaled by {total_units}/{covered}")
-    out = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
+    out = {"impl": "reference", "metric": metric, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
            "warmup": W, "ms_per_step": dt * 1e3, "sample_scale": total_units / covered, "higher_is_better": False,
            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": WORKLOAD, "hidden": sh.hidden, "inter": sh.inter, "experts": sh.n_experts,
+           "config": {"workload": workload, "hidden": sh.hidden, "inter": sh.inter, "experts": sh.n_experts,
                       "top_k": sh.top_k, "n_shared": sh.n_shared, "group": sh.group, "tokens_per_step": 1},
            "cpu_baseline": {"value": val, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -345,7 +348,37 @@ class DeviceLayers:
         torch.cuda.synchronize()
 
 
-def run_cuda(args, sh):
+MIN_LEG_S = 0.5        # every timed leg holds at least this much device time ...
+MIN_REPS = 3           # ... in at least this many repetitions of the K-step region
+MAX_REPS = 4000
+
+
+def n_reps(k_steps: int, est_us_per_step: float) -> int:
+    """Repetitions of a K-step timed region so that the leg holds MIN_LEG_S of device time."""
+    need = int(np.ceil(MIN_LEG_S * 1e6 / max(k_steps * est_us_per_step, 1e-3)))
+    return int(max(MIN_REPS, min(MAX_REPS, need)))
+
+
+def decode_traffic_record(workload: str):
+    """DRAM bytes per launch of the decode kernel from the tracked ncu record under profiles/, or None when
+    there is none for this workload or decode.cu has changed since the capture (the record stores its hash)."""
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "profiles", "decode_layer_kernel_traffic.json")) as f:
+            rec = json.load(f)
+        with open(os.path.join(ROOT, "paper_2512_12990_b200", "csrc", "decode.cu"), "rb") as f:
+            digest = hashlib.sha256(f.read()).hexdigest()
+        if rec.get("decode_cu_sha256") != digest:
+            return None
+        v = rec.get("dram_bytes_per_launch", {}).get(workload)
+        return None if v is None else int(v)
+    except Exception:
+        return None
+
+
+def run_cuda(args, sh, workload: str = WORKLOAD, rank_high: int = RANK_HIGH, metric: str = METRIC, full: bool = True):
+    """The decode-layer measurement on one workload shape.  Returns the JSON object (rank 0) or None.
+    `full` adds the legs only the headline line carries (plain-stream launches, warm L2, CPU baseline)."""
     import torch
     from paper_2512_12990_b200 import binding as B
     from paper_2512_12990_b200 import synth
@@ -360,8 +393,9 @@ def run_cuda(args, sh):
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    K, W = args.steps, args.warmup
+        if not dist.is_initialized():
+            dist.init_process_group("nccl", device_id=dev)
+    K, W = args.steps, max(args.warmup, 3)
     L = args.layers
 
     layers = DeviceLayers(sh, L, dev, seed=sh.seed * 1000 + rank)
@@ -377,6 +411,7 @@ def run_cuda(args, sh):
     ids = torch.empty((P, sh.top_k), dtype=torch.int32, device=dev)
     wts = torch.empty((P, sh.top_k), dtype=torch.float32, device=dev)
     prec = torch.empty((P, sh.top_k), dtype=torch.uint8, device=dev)
+    probe_status = torch.zeros(1, dtype=torch.int32, device=dev)
     stream = torch.cuda.Stream(device=dev)
     lib = B.lib()
     import ctypes
@@ -388,49 +423,69 @@ def run_cuda(args, sh):
     def p(t, row=None, rowbytes=0):
         return c_void_p(t.data_ptr() + (0 if row is None else row * rowbytes))
 
+    def opt(t):
+        return p(t) if t is not None else None
+
     def route(s):
         i = s % P
-        rc = lib.slicemoe_route_topk(p(logits, i, 4 * sh.n_experts), 1, sh.n_experts, sh.top_k, None, 0, 2.0, RANK_HIGH,
+        rc = lib.slicemoe_route_topk(p(logits, i, 4 * sh.n_experts), 1, sh.n_experts, sh.top_k, None, 0, 2.0, rank_high,
                                      p(ids, i, 4 * sh.top_k), p(wts, i, 4 * sh.top_k), p(prec, i, sh.top_k), sptr)
         if rc:
             raise B.SliceMoEError(rc, "slicemoe_route_topk")
 
-    def layer(s):
+    def layer(s, flags=0):
         i, l = s % P, s % L
-        st = layers.shared_tables[l]
-        gv = layers.gate_vecs[l]
-        rc = lib.slicemoe_layer(cs_ref, p(layers.tables[l]), p(st) if st is not None else None,
-                                p(gv) if gv is not None else None, p(x, i, 2 * sh.hidden), 1, p(ids, i, 4 * sh.top_k),
-                                p(prec, i, sh.top_k), p(wts, i, 4 * sh.top_k), p(y, i, 4 * sh.hidden), p(ws), nws, sptr)
+        rc = lib.slicemoe_layer_flags(cs_ref, p(layers.tables[l]), opt(layers.shared_tables[l]), opt(layers.gate_vecs[l]),
+                                      p(x, i, 2 * sh.hidden), 1, p(ids, i, 4 * sh.top_k), p(prec, i, sh.top_k),
+                                      p(wts, i, 4 * sh.top_k), p(y, i, 4 * sh.hidden), p(ws), nws, flags, sptr)
         if rc:
-            raise B.SliceMoEError(rc, "slicemoe_layer")
+            raise B.SliceMoEError(rc, "slicemoe_layer_flags")
 
     def step(s):
         """The whole hot path of one token in one launch: routing in the kernel's prologue, then the layer."""
         i, l = s % P, s % L
-        st = layers.shared_tables[l]
-        gv = layers.gate_vecs[l]
-        rc = lib.slicemoe_layer_routed(cs_ref, p(layers.tables[l]), p(st) if st is not None else None,
-                                       p(gv) if gv is not None else None, p(x, i, 2 * sh.hidden), 1,
-                                       p(logits, i, 4 * sh.n_experts), None, 0, ctypes.c_float(2.0), RANK_HIGH,
-                                       p(ids, i, 4 * sh.top_k), p(prec, i, sh.top_k), p(wts, i, 4 * sh.top_k),
-                                       p(y, i, 4 * sh.hidden), p(ws), nws, sptr)
+        rc = lib.slicemoe_layer_routed(cs_ref, p(layers.tables[l]), opt(layers.shared_tables[l]), opt(layers.gate_vecs[l]),
+                                       p(x, i, 2 * sh.hidden), 1, p(logits, i, 4 * sh.n_experts), None, 0,
+                                       ctypes.c_float(2.0), rank_high, p(ids, i, 4 * sh.top_k), p(prec, i, sh.top_k),
+                                       p(wts, i, 4 * sh.top_k), p(y, i, 4 * sh.hidden), p(ws), nws, sptr)
         if rc:
             raise B.SliceMoEError(rc, "slicemoe_layer_routed")
 
-    def capture(first, count, mode="two"):
-        """mode: "two" = slicemoe_route_topk then slicemoe_layer (the step); "step" = the fused call
-        slicemoe_layer_routed; "layer" = the layer kernel alone on lists already routed."""
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g, stream=stream):
-            for s in range(first, first + count):
-                if mode == "step":
-                    step(s)
-                else:
-                    if mode == "two":
-                        route(s)
-                    layer(s)
-        return g
+    def probe(s, dependent):
+        i, l = s % P, s % L
+        rc = lib.slicemoe_stream_probe(cs_ref, p(layers.tables[l]), opt(layers.shared_tables[l]), p(ids, i, 4 * sh.top_k),
+                                       p(prec, i, sh.top_k), dependent, None, p(probe_status), sptr)
+        if rc:
+            raise B.SliceMoEError(rc, "slicemoe_stream_probe")
+
+    MODES = {
+        "two": lambda s: (route(s), layer(s)),        # the step: slicemoe_route_topk then slicemoe_layer
+        "step": step,                                  # the fused call slicemoe_layer_routed
+        "layer": layer,                                # the layer kernel alone on lists already routed
+        "layer_resident": lambda s: layer(s, B.LISTS_RESIDENT),
+        "probe": lambda s: probe(s, 1),
+        "probe_overlapped": lambda s: probe(s, 0),
+    }
+    chunk = min(K, GRAPH_CHUNK)
+    reps_k, rem = divmod(K, chunk)
+
+    def capture_k(mode):
+        """CUDA graphs that together run steps 0 .. K-1 of `mode`: [(graph, replays)]."""
+        fn = MODES[mode]
+        plan = []
+        for first, count, n in ((0, chunk, reps_k), (reps_k * chunk, rem, 1)):
+            if count == 0 or n == 0:
+                continue
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for s in range(first, first + count):
+                    fn(s)
+            plan.append((g, n))
+        for g, _ in plan:       # instantiate/upload outside the timed region
+            with torch.cuda.stream(stream):
+                g.replay()
+        torch.cuda.synchronize()
+        return plan
 
     def barrier():
         torch.cuda.synchronize()
@@ -438,21 +493,24 @@ def run_cuda(args, sh):
             dist.barrier()
             torch.cuda.synchronize()
 
-    def timed(graphs_and_reps):
-        """Replays the graphs on `stream`, bracketed by barrier + synchronize; device time in ms."""
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    def timed_leg(plan, est_us):
+        """The K-step region, repeated until the leg holds MIN_LEG_S of device time: events between repetitions on
+        the launching stream, one barrier + synchronize on each side of the whole leg.  Returns (ms per K-step
+        region for every repetition, wall-clock window)."""
+        R = n_reps(K, est_us)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(R + 1)]
         barrier()
         t0 = time.time()
         with torch.cuda.stream(stream):
-            e0.record(stream)
-            for g, reps in graphs_and_reps:
-                for _ in range(reps):
-                    g.replay()
-            e1.record(stream)
+            ev[0].record(stream)
+            for r in range(R):
+                for g, n in plan:
+                    for _ in range(n):
+                        g.replay()
+                ev[r + 1].record(stream)
         barrier()
         t1 = time.time()
-        return e0.elapsed_time(e1), (t0, t1)
-
+        return np.array([ev[r].elapsed_time(ev[r + 1]) for r in range(R)]), (t0, t1)
 
     sampler = ClockSampler(local)
     sampler.start()
@@ -460,165 +518,161 @@ def run_cuda(args, sh):
 
     # warm-up: W whole steps as plain launches (also routes every pool entry the timed graphs use)
     with torch.cuda.stream(stream):
-        for s in range(max(W, 3)):
+        for s in range(W):
             route(s)
             layer(s)
             step(s)
         for s in range(P):
             route(s)
     torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for s in range(64):
+            layer(s)
+        e1.record(stream)
+    torch.cuda.synchronize()
+    est = max(e0.elapsed_time(e1) * 1e3 / 64, 1.0)      # us per launch, only to size the legs
     if B.slicemoe_get_status(ws, stream) != 0:
         raise RuntimeError("device status word set during warm-up")
 
-    # ---- value: K whole steps (route + layer), inputs resident in HBM --------------------------------
-    chunk = min(K, GRAPH_CHUNK)
-    reps, rem = divmod(K, chunk)
-    plan = [(capture(0, chunk), reps)]
-    if rem:
-        plan.append((capture(reps * chunk, rem), 1))
-    for g, _ in plan:       # instantiate/upload outside the timed region
-        with torch.cuda.stream(stream):
-            g.replay()
-    ms, win = timed(plan)
-    windows.append(win)
-    ms = max_over_ranks(ms, dist, dev)
-    us_per_layer = whole_job_us_per_unit(ms, K, world)
+    def leg(mode):
+        ms, win = timed_leg(capture_k(mode), est)
+        windows.append(win)
+        med = max_over_ranks(float(np.median(ms)), dist, dev)
+        return {"us_median": whole_job_us_per_unit(med, K, world), "us_min": float(ms.min()) * 1e3 / K,
+                "us_max": float(ms.max()) * 1e3 / K, "reps": int(len(ms)), "ms_median_K_steps": med}
 
-    # ---- the same as one launch per step (routing in the decode kernel's prologue) ----------------------
-    tplan = [(capture(0, chunk, "step"), reps)]
-    if rem:
-        tplan.append((capture(reps * chunk, rem, "step"), 1))
-    for g, _ in tplan:
-        with torch.cuda.stream(stream):
-            g.replay()
-    tms, win = timed(tplan)
-    windows.append(win)
-    fused_us = tms * 1e3 / K
-
-    # ---- roofline: the decode kernel alone, back to back ----------------------------------------------
-    kplan = [(capture(0, chunk, "layer"), reps)]
-    if rem:
-        kplan.append((capture(reps * chunk, rem, "layer"), 1))
-    for g, _ in kplan:
-        with torch.cuda.stream(stream):
-            g.replay()
-    kms, win = timed(kplan)
-    windows.append(win)
-    kernel_us = kms * 1e3 / K
-    bytes_per_launch = step_bytes(sh)
+    two = leg("two")          # value: whole steps (route + layer), inputs resident in HBM
+    fused = leg("step")       # the same as one launch per step
+    kern = leg("layer")       # roofline: the decode kernel alone, back to back
+    kern_res = leg("layer_resident")
+    pr_dep = leg("probe")
+    pr_ovl = leg("probe_overlapped")
+    if int(probe_status.item()) != 0:
+        raise RuntimeError("a wait of the stream probe ran out")
+    us_per_layer = two["us_median"]
+    kernel_us = kern["us_median"] * world     # per launch of one rank
+    bytes_per_launch = step_bytes(sh, rank_high)
     peak, peak_kind = measured_hbm_peak()
     achieved = bytes_per_launch / (kernel_us * 1e-6) / 1e9
 
-    # ---- beside the headline: spread over graph replays, plain-stream launches, warm L2 -----------------
-    # (a) the layer-kernel graph replay by replay: median and minimum of the per-launch average
-    per_replay = []
-    g0, n0 = kplan[0]
-    for _ in range(min(n0, 10)):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stream_us = warm_us = None
+    if full:
+        # the step without a graph: plain launches on the stream (the host's launch rate is part of it)
+        Ks = min(max(K, 2000), 20000)
         with torch.cuda.stream(stream):
             e0.record(stream)
-            g0.replay()
+            for s_ in range(Ks):
+                route(s_)
+                layer(s_)
             e1.record(stream)
         torch.cuda.synchronize()
-        per_replay.append(e0.elapsed_time(e1) * 1e3 / chunk)
-    # (b) the step without a graph: plain launches on the stream (the host's launch rate is part of it)
-    Ks = min(K, 2000)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    with torch.cuda.stream(stream):
-        e0.record(stream)
-        for s_ in range(Ks):
-            route(s_)
-            layer(s_)
-        e1.record(stream)
-    torch.cuda.synchronize()
-    stream_us = e0.elapsed_time(e1) * 1e3 / Ks
-    # (c) warm L2: the same layer and input every launch (its 58 MB stay in the 126 MB L2) - NOT the headline
-    gw = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(gw, stream=stream):
-        for _ in range(min(chunk, 200)):
-            layer(0)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with torch.cuda.stream(stream):
-        gw.replay()
-        e0.record(stream)
-        gw.replay()
-        e1.record(stream)
-    torch.cuda.synchronize()
-    warm_us = e0.elapsed_time(e1) * 1e3 / min(chunk, 200)
+        stream_us = e0.elapsed_time(e1) * 1e3 / Ks
+        # warm L2: the same layer and input every launch (its bytes stay in the 126 MB L2) - NOT the headline
+        gw = torch.cuda.CUDAGraph()
+        nw_ = 200
+        with torch.cuda.graph(gw, stream=stream):
+            for _ in range(nw_):
+                layer(0)
+        with torch.cuda.stream(stream):
+            gw.replay()
+            e0.record(stream)
+            for _ in range(20):
+                gw.replay()
+            e1.record(stream)
+        torch.cuda.synchronize()
+        warm_us = e0.elapsed_time(e1) * 1e3 / (20 * nw_)
 
     # ---- e2e: host buffers in and out through the C ABI, every step ------------------------------------
-    Ke = min(K, 2000)
-    xh = torch.from_numpy(xbits_h.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
-    lh = torch.from_numpy(logits_h.copy()).pin_memory()
+    # one pinned buffer per step holds x (bf16) and then the logits (float32): one host-to-device copy
+    row = 2 * sh.hidden + 4 * sh.n_experts
+    inh = torch.empty((P, row), dtype=torch.uint8).pin_memory()
+    inh[:, :2 * sh.hidden] = torch.from_numpy(xbits_h.view(np.uint8).reshape(P, 2 * sh.hidden))
+    inh[:, 2 * sh.hidden:] = torch.from_numpy(logits_h.view(np.uint8).reshape(P, 4 * sh.n_experts))
     yh = torch.empty((P, sh.hidden), dtype=torch.float32).pin_memory()
 
     def host_step(s):
         i, l = s % P, s % L
-        st = layers.shared_tables[l]
-        gv = layers.gate_vecs[l]
-        rc = lib.slicemoe_decode_step_host(cs_ref, p(layers.tables[l]), p(st) if st is not None else None,
-                                           p(gv) if gv is not None else None, p(xh, i, 2 * sh.hidden),
-                                           p(lh, i, 4 * sh.n_experts), None, 0, 2.0, RANK_HIGH, p(yh, i, 4 * sh.hidden),
-                                           p(ws), nws, sptr)
+        rc = lib.slicemoe_decode_step_host(cs_ref, p(layers.tables[l]), opt(layers.shared_tables[l]),
+                                           opt(layers.gate_vecs[l]), p(inh, i, row), None, None, 0, 2.0, rank_high,
+                                           p(yh, i, 4 * sh.hidden), p(ws), nws, sptr)
         if rc:
             raise B.SliceMoEError(rc, "slicemoe_decode_step_host")
 
     for s in range(3):
         host_step(s)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_probe = time.perf_counter()
+    for s in range(50):
+        host_step(s)
+    est_e = (time.perf_counter() - t_probe) * 1e6 / 50
+    Re = n_reps(K, est_e)
+    e2e_ms = []
     barrier()
     t0 = time.time()
-    e0.record(stream)
-    for s in range(Ke):
-        host_step(s)
-    e1.record(stream)
+    for _ in range(Re):
+        e0.record(stream)
+        for s in range(K):
+            host_step(s)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        e2e_ms.append(e0.elapsed_time(e1))
     barrier()
     windows.append((t0, time.time()))
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
-    e2e_us = whole_job_us_per_unit(e2e_ms, Ke, world)
+    e2e_med = max_over_ranks(float(np.median(e2e_ms)), dist, dev)
+    e2e_us = whole_job_us_per_unit(e2e_med, K, world)
     sampler.stop()
     if B.slicemoe_get_status(ws, stream) != 0:
         raise RuntimeError("device status word set during the timed regions")
     # the host-buffer path must reproduce the device path bit for bit (fixed summation order)
-    n_cmp = min(Ke, chunk, P)      # steps both paths ran
+    n_cmp = min(K, P)      # steps both paths ran
     if P % L == 0 and not torch.equal(yh[:n_cmp].to(dev), y[:n_cmp]):
         raise RuntimeError("host-buffer path and device path disagree")
 
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
+        return None
     out = {
-        "metric": METRIC, "value": us_per_layer, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(W, 3),
-        "ms_per_step": ms / K, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "metric": metric, "value": us_per_layer, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": two["ms_median_K_steps"] / K, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 x int8/int4 codes, f32 accumulate", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "hidden": sh.hidden, "inter": sh.inter, "experts": sh.n_experts,
+        "config": {"workload": workload, "hidden": sh.hidden, "inter": sh.inter, "experts": sh.n_experts,
                    "top_k": sh.top_k, "n_shared": sh.n_shared, "group": sh.group, "tokens_per_step": 1,
-                   "precision_mix": f"{RANK_HIGH} of {sh.top_k} routed at 8-bit, rest 4-bit; shared 8-bit",
+                   "precision_mix": f"{rank_high} of {sh.top_k} routed at 8-bit, rest 4-bit; shared 8-bit",
                    "resident_layers": L, "l2": f"steps cycle over {L} layers ({L * bytes_per_launch / 1e6:.0f} MB "
                    "read between reuses of a byte) so inputs exceed L2",
                    "replay": f"CUDA graphs of {chunk} steps", "parallelism": f"replicas x{world}"},
+        "timing": {"region": f"{K} steps, repeated until the leg holds {MIN_LEG_S} s of device time (at least "
+                             f"{MIN_REPS} times); value = median over repetitions, max over ranks",
+                   "reps": two["reps"], "value_min": two["us_min"] / world, "value_max": two["us_max"] / world},
         "bytes_per_step": bytes_per_launch,
-        "gbs": bytes_per_launch * world / (us_per_layer * world * 1e-6) / 1e9,
-        "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": 2 * sh.hidden + 4 * sh.n_experts,
-                "d2h_bytes_per_step": 4 * sh.hidden, "steps": Ke},
+        "gbs": bytes_per_launch / (us_per_layer * 1e-6) / 1e9,
+        "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": row, "d2h_bytes_per_step": 4 * sh.hidden,
+                "steps": K, "reps": Re, "what": "slicemoe_decode_step_host: one copy of x and the logits from a pinned "
+                "host buffer, one launch, y written to pinned host memory, one stream synchronise per step"},
         "gpu_launches": 2 * K,
         "step": "slicemoe_route_topk then slicemoe_layer, chained by programmatic dependent launch",
-        "fused_step_us": fused_us,
-        "plain_stream_step_us": stream_us,
-        "warm_l2_us_per_launch": warm_us,
+        "fused_step_us": fused["us_median"] * world,
         "roofline": {"bound": "hbm", "kernel": "decode_layer_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "us_per_launch": kernel_us, "bytes_per_launch": bytes_per_launch,
-                     "us_per_launch_median": float(np.median(per_replay)), "us_per_launch_min": float(np.min(per_replay))},
+                     "traffic": decode_traffic_record(workload), "us_per_launch": kernel_us,
+                     "bytes_per_launch": bytes_per_launch, "us_per_launch_median": kernel_us,
+                     "us_per_launch_min": kern["us_min"], "reps": kern["reps"],
+                     "lists_resident_us_per_launch": kern_res["us_median"] * world,
+                     "lists_resident_frac": bytes_per_launch / (kern_res["us_median"] * world * 1e-6) / 1e9 / peak},
+        # the same bytes through the same bulk copies with no arithmetic and no exchange (slicemoe_stream_probe):
+        # what the memory system alone needs per launch, back to back, and with launches allowed to overlap
+        "stream_only_us": pr_dep["us_median"] * world,
+        "stream_only_overlapped_us": pr_ovl["us_median"] * world,
         "clocks": sampler.summary(windows),
     }
-    if not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(sh)
-    print(json.dumps(out), flush=True)
-    if dist is not None:
-        dist.destroy_process_group()
+    if full:
+        out["plain_stream_step_us"] = stream_us
+        out["warm_l2_us_per_launch"] = warm_us
+        if not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline(sh, rank_high)
+    del layers
+    torch.cuda.empty_cache()
+    return out
 
 
 # ---- secondary workloads (not the default line) --------------------------------------------------------------
@@ -638,9 +692,9 @@ def prefill_flops(sh, T: int) -> int:
     return 2 * T * 3 * sh.hidden * (sh.top_k * sh.inter + sh.n_shared * sh.shared_inter)
 
 
-def run_prefill(args):
+def run_prefill(args, K: int, W: int):
     """The prefill layer of 2048 tokens: device-resident TFLOP/s of slicemoe_prefill_layer, the same call with
-    host buffers, and the share of the tensor-core peak."""
+    host buffers, and the share of the tensor-core peak.  Returns the JSON object."""
     import torch
     from paper_2512_12990_b200 import binding as B
     from paper_2512_12990_b200 import synth
@@ -649,7 +703,7 @@ def run_prefill(args):
         raise RuntimeError("bench.py needs a CUDA device (the hot path has no CPU fallback)")
     sh = synth.SHAPES["qwen_prefill"]
     T = 2048
-    K, W = args.steps, max(args.warmup, 3)
+    W = max(W, 3)
     dev = torch.device("cuda", 0)
     L = max(2, min(args.layers, 4))      # 4 layers x 0.46 GB of planes: every step reads weights that left L2
     layers = DeviceLayers(sh, L, dev, seed=sh.seed * 1000)
@@ -679,19 +733,28 @@ def run_prefill(args):
     if int(status.item()) != 0:
         raise RuntimeError("device status word set during warm-up")
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0 = time.time()
     e0.record(stream)
-    for i in range(K):
+    for i in range(W):
         step(i)
     e1.record(stream)
     torch.cuda.synchronize()
+    R = n_reps(K, e0.elapsed_time(e1) * 1e3 / W)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(R + 1)]
+    t0 = time.time()
+    ev[0].record(stream)
+    for r in range(R):
+        for i in range(K):
+            step(i)
+        ev[r + 1].record(stream)
+    torch.cuda.synchronize()
     windows = [(t0, time.time())]
-    ms = e0.elapsed_time(e1) / K
+    reps_ms = np.array([ev[r].elapsed_time(ev[r + 1]) / K for r in range(R)])
+    ms = float(np.median(reps_ms))
     # host buffers: x in from pinned memory, y out, every step
     xh = torch.from_numpy(xbits_h.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
     yh = torch.empty((T, sh.hidden), dtype=torch.float32).pin_memory()
     xd = torch.empty_like(x)
-    Ke = min(K, 50)
+    Ke = max(min(K, 50), int(np.ceil(MIN_LEG_S * 1e3 / max(ms, 1e-3))))
     t0 = time.time()
     e0.record(stream)
     with torch.cuda.stream(stream):
@@ -720,6 +783,8 @@ def run_prefill(args):
                    "precision_mix": "experts of even popularity rank at 4-bit, odd rank at 8-bit; shared 8-bit",
                    "routing": "Zipf(1.0) popularity + Gumbel noise, top-4",
                    "resident_layers": L, "l2": f"steps cycle over {L} layers, 0.46 GB of planes each, so weights exceed L2"},
+        "timing": {"reps": int(R), "ms_per_step_min": float(reps_ms.min()), "ms_per_step_max": float(reps_ms.max()),
+                   "region": f"{K} steps per repetition, median over repetitions"},
         "flops_per_step": flops,
         "e2e": {"value": flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": 2 * T * sh.hidden,
                 "d2h_bytes_per_step": 4 * T * sh.hidden, "steps": Ke},
@@ -728,7 +793,9 @@ def run_prefill(args):
                      "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "peak_kind": f"of {kind}", "traffic": None},
         "clocks": sampler.summary(windows),
     }
-    print(json.dumps(out), flush=True)
+    del layers, ws
+    torch.cuda.empty_cache()
+    return out
 
 
 def warmup_comparison(B, synth, sh, NL, ids_h, preq_h, cap, msb_b, lsb_b, tau, dev, prompt_tokens=1024, steps=(4, 32)):
@@ -780,7 +847,7 @@ def warmup_comparison(B, synth, sh, NL, ids_h, preq_h, cap, msb_b, lsb_b, tau, d
     return out
 
 
-def run_stack(args):
+def run_stack(args, with_warmup_table: bool = True):
     """The 26-layer decode stack over a 256-step routing trace with the host slice cache at 30% capacity:
     microseconds per token for the 26 expert FFNs with precision lists resident (value) and with the cache in the
     loop - ids to the host, cache lookup, precision list back - for every layer (e2e)."""
@@ -823,12 +890,12 @@ def run_stack(args):
     def p(t, row=None, rowbytes=0):
         return c_void_p(t.data_ptr() + (0 if row is None else row * rowbytes))
 
-    def layer(r, l, prec_t=prec):
-        rc = lib.slicemoe_layer(cs_ref, p(layers.tables[l]), p(layers.shared_tables[l]), None, p(x, r, 2 * sh.hidden), 1,
-                                p(ids, r, 4 * sh.top_k), p(prec_t, r, sh.top_k), p(wts, r, 4 * sh.top_k),
-                                p(y, r, 4 * sh.hidden), p(ws), nws, sptr)
+    def layer(r, l, prec_t=prec, flags=0):
+        rc = lib.slicemoe_layer_flags(cs_ref, p(layers.tables[l]), p(layers.shared_tables[l]), None, p(x, r, 2 * sh.hidden),
+                                      1, p(ids, r, 4 * sh.top_k), p(prec_t, r, sh.top_k), p(wts, r, 4 * sh.top_k),
+                                      p(y, r, 4 * sh.hidden), p(ws), nws, flags, sptr)
         if rc:
-            raise B.SliceMoEError(rc, "slicemoe_layer")
+            raise B.SliceMoEError(rc, "slicemoe_layer_flags")
 
     sampler = ClockSampler(0)
     sampler.start()
@@ -836,26 +903,34 @@ def run_stack(args):
         for r in range(3 * NL):
             layer(r, r % NL)
     torch.cuda.synchronize()
+    # The precision lists of the whole trace are resident before the first launch (the headline mode of this
+    # workload), so the kernels are told so: SLICEMOE_LISTS_RESIDENT.
     graphs = []
     for s0 in range(0, NS, 32):           # 32 tokens x 26 layers per graph
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=stream):
             for r in range(s0 * NL, (s0 + 32) * NL):
-                layer(r, r % NL)
+                layer(r, r % NL, flags=B.LISTS_RESIDENT)
         graphs.append(g)
-    with torch.cuda.stream(stream):
-        graphs[0].replay()
-    torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0 = time.time()
     with torch.cuda.stream(stream):
         e0.record(stream)
-        for g in graphs:
-            g.replay()
+        graphs[0].replay()
         e1.record(stream)
     torch.cuda.synchronize()
+    R = n_reps(NS, e0.elapsed_time(e1) * 1e3 / 32)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(R + 1)]
+    t0 = time.time()
+    with torch.cuda.stream(stream):
+        ev[0].record(stream)
+        for r_ in range(R):
+            for g in graphs:
+                g.replay()
+            ev[r_ + 1].record(stream)
+    torch.cuda.synchronize()
     windows = [(t0, time.time())]
-    us_per_token = e0.elapsed_time(e1) * 1e3 / NS
+    reps_us = np.array([ev[r_].elapsed_time(ev[r_ + 1]) * 1e3 / NS for r_ in range(R)])
+    us_per_token = float(np.median(reps_us))
     if B.slicemoe_get_status(ws, stream) != 0:
         raise RuntimeError("device status word set")
     # bytes the FFNs read: per (step, layer) the selected experts at their precision plus the shared experts
@@ -904,7 +979,9 @@ def run_stack(args):
                    "trace": "Zipf(1.1) popularity per layer, p=0.5 repeat of the previous step's logits",
                    "l2": f"{NL} layers of planes resident ({NL * sh.n_experts * (msb_b + lsb_b) / 1e9:.1f} GB); a byte is "
                          "re-read at the earliest one token later, after ~1.3 GB of other traffic",
-                   "replay": "CUDA graphs of 32 tokens x 26 layers"},
+                   "replay": "CUDA graphs of 32 tokens x 26 layers", "lists": "resident (SLICEMOE_LISTS_RESIDENT)"},
+        "timing": {"reps": int(R), "value_min": float(reps_us.min()), "value_max": float(reps_us.max()),
+                   "region": f"{NS} tokens per repetition, median over repetitions"},
         "gbs": gbs, "bytes_per_token": total_bytes / NS,
         "cache": {k: int(v) for k, v in stats.items()},
         "cache_rates": {"msb_hit": stats["msb_hit"] / stats["requests"],
@@ -912,7 +989,8 @@ def run_stack(args):
                         "miss_bytes_over_8bit_bytes": stats["bytes_fetched"] / (stats["requests"] * (msb_b + lsb_b)),
                         "exec_8bit": stats["high_exec"] / stats["requests"],
                         "mean_critical_per_token_layer": float(preq_h.sum(1).mean())},
-        "cache_warmup": warmup_comparison(B, synth, sh, NL, ids_h, preq_h, cap, msb_b, lsb_b, TAU, dev),
+        "cache_warmup": (warmup_comparison(B, synth, sh, NL, ids_h, preq_h, cap, msb_b, lsb_b, TAU, dev)
+                         if with_warmup_table else None),
         "e2e": {"value": e2e_us, "unit": "µs/token", "h2d_bytes_per_step": NL * sh.top_k,
                 "d2h_bytes_per_step": NL * sh.top_k * 5, "steps": NE,
                 "what": "route, ids and requests to the host, cache lookup, precision list back, FFN - per layer"},
@@ -921,11 +999,20 @@ def run_stack(args):
                      "frac": gbs / peak, "peak_kind": f"of {kind}", "traffic": None},
         "clocks": sampler.summary(windows),
     }
-    print(json.dumps(out), flush=True)
+    del layers
+    torch.cuda.empty_cache()
+    return out
+
+
+DECODE_WORKLOADS = {
+    # name: (rank_high, metric)
+    "dsv2": (RANK_HIGH, METRIC),
+    # config 3: 60 x 1408 experts, top-4 (the 2 best at 8 bits), one gated shared expert of 5632
+    "qwen": (2, "us per MoE layer decode (Qwen1.5-MoE-A2.7B shape, b=1)"),
+}
 
 
 def main():
-    global WORKLOAD, RANK_HIGH, METRIC, NCU_TRAFFIC_BYTES_PER_LAUNCH
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20000)
@@ -933,35 +1020,52 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--layers", type=int, default=16, help="independently packed layers the steps cycle over")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="the default line only: skip the qwen / stack / prefill sub-objects of a one-GPU run")
     ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "qwen", "stack", "prefill"],
-                    help="the default is the headline decode layer; `qwen` is the same measurement on the Qwen1.5-MoE-"
-                         "shaped layer; `stack` and `prefill` are single-GPU extras")
+                    help="the default is the headline decode layer (with short legs of the other three attached as "
+                         "sub-objects on one GPU); `qwen` is the same measurement on the Qwen1.5-MoE-shaped layer; "
+                         "`stack` and `prefill` are single-GPU workloads of their own")
     args = ap.parse_args()
+    explicit_steps = not (args.steps == 20000 and args.warmup == 100)
+    world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.workload in ("stack", "prefill") and args.impl == "cuda":
-        if int(os.environ.get("WORLD_SIZE", "1")) != 1 or args.gpus != 1:
+        if world != 1 or args.gpus != 1:
             raise SystemExit("--workload stack/prefill run on one GPU")
         if args.workload == "prefill":
-            if args.steps == 20000 and args.warmup == 100:
-                args.steps, args.warmup = 200, 5
-            run_prefill(args)
+            out = run_prefill(args, *((args.steps, args.warmup) if explicit_steps else (100, 5)))
         else:
-            run_stack(args)
+            out = run_stack(args)
+        print(json.dumps(out), flush=True)
         return
     from paper_2512_12990_b200 import synth
-    if args.workload == "qwen":
-        # config 3: 60 x 1408 experts, top-4 (the 2 best at 8 bits), one gated shared expert of 5632
-        WORKLOAD, RANK_HIGH, NCU_TRAFFIC_BYTES_PER_LAUNCH = "qwen", 2, None
-        METRIC = "us per MoE layer decode (Qwen1.5-MoE-A2.7B shape, b=1)"
-    sh = synth.SHAPES[WORKLOAD]
+    rank_high, metric = DECODE_WORKLOADS[args.workload]
+    sh = synth.SHAPES[args.workload]
     if args.impl == "reference":
-        if args.steps == 20000 and args.warmup == 100:
+        if not explicit_steps:
             args.steps, args.warmup = 20, 3
-        run_reference(args, sh)
+        run_reference(args, sh, args.workload, rank_high, metric)
         return
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     if world != args.gpus:
         raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run for N > 1")
-    run_cuda(args, sh)
+    out = run_cuda(args, sh, args.workload, rank_high, metric, full=True)
+    if out is not None and world == 1 and args.workload == WORKLOAD and not args.no_extras:
+        # short legs of the other workloads, each with its own roofline and clock record
+        import copy
+        a2 = copy.copy(args)
+        a2.steps, a2.warmup = min(args.steps, 5000), 20
+        q_rank, q_metric = DECODE_WORKLOADS["qwen"]
+        out["workloads"] = {
+            "qwen": run_cuda(a2, synth.SHAPES["qwen"], "qwen", q_rank, q_metric, full=False),
+            "stack": run_stack(args, with_warmup_table=False),
+            "prefill": run_prefill(args, 100, 5),
+        }
+    if out is not None:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        if dist.is_initialized():
+            dist.destroy_process_group()
 
 
 if __name__ == "__main__":

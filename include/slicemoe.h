@@ -225,6 +225,25 @@ int slicemoe_layer_routed(const slicemoe_shape *shape, const slicemoe_expert *ex
                           void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * slicemoe_stream_probe - a measuring stick, not part of the method: brings exactly the bytes that one
+ * slicemoe_layer call with T = 1 reads for this list - MSB plane, LSB plane where prec = 1, scales and zero-points
+ * of gate, up and down of every listed expert, and of the shared experts at 8 bits - into shared memory with the
+ * decode kernel's bulk copies (16 KB each, one CTA per SM, twelve copies in flight per CTA) and does nothing with
+ * them.  Its time per launch is what the memory system alone needs for a decode step of the layer.
+ *   ids, prec   device [top_k]; entries outside [0, n_experts) are skipped
+ *   dependent   1: no byte is requested before the work ahead on `stream` has completed (a kernel all of whose
+ *               input depends on its predecessor); 0: the lists must be resident in the sense of
+ *               SLICEMOE_LISTS_RESIDENT, and launches overlap as far as the hardware lets them
+ *   bytes_out_device   device, or NULL: the bytes of the step are ADDED to it (one CTA does)
+ *   status_out_device  device int32, or NULL: set to 1 if a (bounded) wait for a copy ran out
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+int slicemoe_stream_probe(const slicemoe_shape *shape, const slicemoe_expert *experts,
+                          const slicemoe_expert *shared, const int32_t *ids, const uint8_t *prec,
+                          int dependent, unsigned long long *bytes_out_device, int *status_out_device,
+                          void *stream);
+
+/*
  * slicemoe_layer_static - slicemoe_layer for callers that cannot allocate device memory.  (The paper
  * has no counterpart; this is a convenience of the library.)
  *

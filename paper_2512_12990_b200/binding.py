@@ -28,7 +28,7 @@ EXPORTS = (
     "slicemoe_strerror", "slicemoe_version", "slicemoe_last_cuda_error", "slicemoe_plane_bytes", "slicemoe_meta_count", "slicemoe_pack",
     "slicemoe_unpack_plane", "slicemoe_unpack_meta", "slicemoe_route_topk", "slicemoe_workspace_bytes",
     "slicemoe_workspace_init", "slicemoe_workspace_set_wait", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer", "slicemoe_layer_flags",
-    "slicemoe_decode_step_host", "slicemoe_layer_static", "slicemoe_layer_routed", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
+    "slicemoe_decode_step_host", "slicemoe_stream_probe", "slicemoe_layer_static", "slicemoe_layer_routed", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
     "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
     "slicemoe_dbsc_assign", "slicemoe_dbsc_stats", "slicemoe_dbsc_contains",
     "slicemoe_dbsc_prefill_layer", "slicemoe_dbsc_prefill_end",
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
                                  c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.slicemoe_layer_flags.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                        c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, ctypes.c_uint, c_void_p]
+    L.slicemoe_stream_probe.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
+                                        c_void_p]
     L.slicemoe_layer_static.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                         c_void_p, c_void_p, c_void_p, c_void_p]
     L.slicemoe_decode_step_host.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -293,6 +295,15 @@ def slicemoe_layer(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x, id
                               _stream(stream))
     _check(rc, "slicemoe_layer")
     return y
+
+
+def slicemoe_stream_probe(shape: Shape, experts_tbl, shared_tbl, ids, prec, dependent=True, bytes_out=None,
+                          status_out=None, stream=None):
+    """ids, prec: CUDA int32 / uint8 [top_k].  bytes_out: CUDA int64 [1] (added to) or None; status_out: CUDA
+    int32 [1] or None."""
+    rc = lib().slicemoe_stream_probe(ctypes.byref(shape), _ptr(experts_tbl), _ptr(shared_tbl), _ptr(ids), _ptr(prec),
+                                     1 if dependent else 0, _ptr(bytes_out), _ptr(status_out), _stream(stream))
+    _check(rc, "slicemoe_stream_probe")
 
 
 def slicemoe_layer_static(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x, ids, prec, weights, y, stream=None):

@@ -306,3 +306,28 @@ def test_resident_lists_give_the_same_bits(name):
     # an unknown flag is refused
     with pytest.raises(B.SliceMoEError):
         B.slicemoe_layer(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, *args, L.ws, flags=2)
+
+
+@pytest.mark.parametrize("name", ["tiny", "dsv2", "qwen"])
+def test_stream_probe_moves_the_algorithmic_bytes(name):
+    """slicemoe_stream_probe has to request exactly the bytes the oracle's byte count gives for the list
+    (it is the ruler the decode kernel is measured against), in both launch modes, without a wait running out."""
+    from paper_2512_12990_b200 import binding as B
+    torch = _torch()
+    sh = synth.SHAPES[name]
+    logits = synth.router_logits_normal(sh.seed, ("probe-logits",), 1, sh.n_experts)
+    ids, _, _ = moe.route_topk(logits, sh.top_k)
+    prec = (np.arange(sh.top_k) < (sh.top_k + 1) // 2).astype(np.uint8)
+    L = H.Layer(sh, sorted(set(ids.ravel().tolist())))
+    olist = L.oracle_list()
+    mats = ("gate", "up", "down")
+    want = sum(moe.algorithmic_bytes(olist[int(e)][m], int(pr)) for e, pr in zip(ids[0], prec) for m in mats)
+    want += sum(moe.algorithmic_bytes(ex[m], 1) for ex in (L.oracle_shared or []) for m in mats)
+    got = torch.zeros(1, dtype=torch.int64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ids_d, prec_d = _dev(ids[0].astype(np.int32)), _dev(prec)
+    for dependent in (True, False, True):
+        B.slicemoe_stream_probe(L.cshape, L.experts_tbl, L.shared_tbl, ids_d, prec_d, dependent, got, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert int(got.item()) == 3 * want
