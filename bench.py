@@ -1013,6 +1013,7 @@ DECODE_WORKLOADS = {
 
 
 def main():
+    global MIN_LEG_S
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20000)
@@ -1020,6 +1021,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--layers", type=int, default=16, help="independently packed layers the steps cycle over")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--leg-seconds", type=float, default=MIN_LEG_S,
+                    help="device time every timed leg must hold (a profiler capture passes 0: three repetitions)")
     ap.add_argument("--no-extras", action="store_true",
                     help="the default line only: skip the qwen / stack / prefill sub-objects of a one-GPU run")
     ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "qwen", "stack", "prefill"],
@@ -1027,6 +1030,7 @@ def main():
                          "sub-objects on one GPU); `qwen` is the same measurement on the Qwen1.5-MoE-shaped layer; "
                          "`stack` and `prefill` are single-GPU workloads of their own")
     args = ap.parse_args()
+    MIN_LEG_S = max(0.0, args.leg_seconds)
     explicit_steps = not (args.steps == 20000 and args.warmup == 100)
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.workload in ("stack", "prefill") and args.impl == "cuda":
