@@ -125,7 +125,9 @@ int slicemoe_unpack_meta(const uint16_t *scale, const uint8_t *zp, int N, int K,
  *            pass tau > 1 and rank_high = 0 for "never"
  *   ids      device int32 [T, k]: experts by descending key; ties -> lower index; NaN logit = -inf
  *   weights  device float32 [T, k]: softmax(logits)[id]
- *   prec_req device uint8 [T, k] or NULL
+ *   prec_req device uint8 [T, k] or NULL: 1 iff the float32 probability - the returned weights[t, j] when
+ *            renorm = 0 - is >= tau (a float32), or j < rank_high.  The comparison is taken in float32, so the
+ *            flag is an exact function of the returned weight
  * Errors: INVALID_ARG (null, T <= 0, k < 1, k > E, k > SLICEMOE_MAX_TOP_K), UNSUPPORTED (E > 512).
  */
 int slicemoe_route_topk(const float *logits, int T, int E, int k, const float *bias, int renorm,

@@ -331,3 +331,36 @@ def test_stream_probe_moves_the_algorithmic_bytes(name):
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert int(got.item()) == 3 * want
+
+
+@pytest.mark.parametrize("name,rank_high", [("dsv2", 3), ("qwen", 2)])
+@pytest.mark.parametrize("token", [0, 1, 2])
+def test_full_size_decode_three_tokens_three_precision_mixes(name, rank_high, token):
+    """Configs 2 and 3 at full size, element by element against the oracle: three independently drawn tokens
+    (routing, activations, and so the experts that are read), each at the benchmark's mix, with every routed expert
+    at 8 bits, with every routed expert at 4 bits, and with the same expert in two slots at different precisions."""
+    sh = synth.SHAPES[name]
+    logits = synth.router_logits_normal(sh.seed, ("full-logits", token), 1, sh.n_experts)
+    ids, w, _ = moe.route_topk(logits, sh.top_k)
+    L = H.Layer(sh, ids[0], layer=token)
+    xbits, x64 = H.x_inputs(sh, 1, f"full-x{token}")
+    mixes = {"mixed": moe.precision_request(w, 2.0, rank_high=rank_high), "all 8-bit": np.ones_like(ids, dtype=np.uint8),
+             "all 4-bit": np.zeros_like(ids, dtype=np.uint8)}
+    outs = {}
+    for label, prec in mixes.items():
+        y, status = _run_layer(L, xbits, ids, prec, w)
+        y_ref = moe.layer(x64, L.oracle_list(), ids, prec, w, shared=L.oracle_shared, shared_gate_vec=L.gate_vec)
+        assert status == 0
+        H.assert_close(y, y_ref, f"{name} token {token} {label}")
+        outs[label] = y_ref
+    # the mixes are different computations: the oracle's results are further apart than the tolerance
+    assert np.linalg.norm(outs["all 8-bit"] - outs["all 4-bit"]) > 1e-2 * np.linalg.norm(outs["all 8-bit"])
+    # the same expert twice: slot 1 repeats slot 0's expert, at the other precision and with its own weight
+    ids2 = ids.copy()
+    ids2[0, 1] = ids2[0, 0]
+    prec2 = mixes["mixed"].copy()
+    prec2[0, 0], prec2[0, 1] = 1, 0
+    y, status = _run_layer(L, xbits, ids2, prec2, w)
+    y_ref = moe.layer(x64, L.oracle_list(), ids2, prec2, w, shared=L.oracle_shared, shared_gate_vec=L.gate_vec)
+    assert status == 0
+    H.assert_close(y, y_ref, f"{name} token {token} same expert twice")

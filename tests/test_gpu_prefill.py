@@ -162,21 +162,39 @@ class _QwenPrefill:
         self.perm = perm
         self.xbits, self.x64 = H.x_inputs(sh, self.T, "prefill-x")
 
-    def oracle_rows(self, rows):
-        """Float64 layer output of the token rows `rows`: every expert they use is dequantised once."""
+    def oracle_rows(self, rows, monkeypatch):
+        """Float64 layer output of the token rows `rows`: oracle.moe.layer as it stands, token by token.  It
+        dequantises an expert anew for every (token, slot); so that this ends in reasonable time the oracle's own
+        dequantiser is memoised for the duration (same function, same results, a bounded cache keyed by the matrix
+        object and the precision) - no arithmetic happens on the test's side."""
+        from collections import OrderedDict
+        from oracle import amat
+        real, cache = amat.dequant, OrderedDict()
+
+        def memoised(mat, prec):
+            key = (id(mat), int(prec))
+            if key in cache:
+                cache.move_to_end(key)
+                return cache[key]
+            cache[key] = real(mat, prec)
+            if len(cache) > 30:
+                cache.popitem(last=False)
+            return cache[key]
+
+        monkeypatch.setattr(amat, "dequant", memoised)
         rows = np.asarray(rows)
-        X = self.x64[rows].T                                   # [hidden, n]
-        y = np.zeros((self.sh.hidden, len(rows)))
-        for e in np.unique(self.ids[rows]):
-            ex = H.oracle_expert_from_device(self.packed[int(e)])
-            hit = (self.ids[rows] == e)                        # [n, k]
-            cols = np.nonzero(hit.any(1))[0]
-            out = moe.expert_ffn_one(X[:, cols], ex, int(self.expert_prec[e]))
-            y[:, cols] += out * (self.w[rows][cols] * hit[cols]).sum(1)[None, :]
-        shared = H.oracle_expert_from_device(self.packed_shared[0])
-        gate = 1.0 / (1.0 + np.exp(-(self.gate_vec.astype(np.float64) @ X)))
-        y += moe.expert_ffn_one(X, shared, 1) * gate[None, :]
-        return y.T
+        # tokens that share their first expert next to each other: more of the cache's entries are used again
+        order = np.lexsort((rows, self.ids[rows, 0]))
+        experts = {int(e): H.oracle_expert_from_device(self.packed[int(e)]) for e in np.unique(self.ids[rows])}
+        shared = [H.oracle_expert_from_device(self.packed_shared[0])]
+        prec = self.expert_prec[self.ids]
+        y = np.empty((len(rows), self.sh.hidden))
+        for i in order:
+            t = rows[i:i + 1]
+            y[i] = moe.layer(self.x64[t], experts, self.ids[t], prec[t], self.w[t], shared=shared,
+                             shared_gate_vec=self.gate_vec)[0]
+        monkeypatch.setattr(amat, "dequant", real)
+        return y
 
 
 @pytest.fixture(scope="module")
@@ -184,7 +202,7 @@ def qwen_prefill():
     return _QwenPrefill()
 
 
-def test_full_size_prefill_layer_sampled_tokens(qwen_prefill):
+def test_full_size_prefill_layer_sampled_tokens(qwen_prefill, monkeypatch):
     from paper_2512_12990_b200 import binding as B
     torch = _torch()
     q = qwen_prefill
@@ -208,7 +226,7 @@ def test_full_size_prefill_layer_sampled_tokens(qwen_prefill):
     extra = [t for t in range(5, q.T, 61) if t not in rows][:max(0, 64 - len(rows))]
     rows = sorted(rows + extra)
     assert len(rows) >= 64 and set(np.unique(q.ids[rows])) == set(range(q.sh.n_experts))
-    y_ref = q.oracle_rows(rows)
+    y_ref = q.oracle_rows(rows, monkeypatch)
     worst = 0.0
     for i, t in enumerate(rows):
         rel, _ = H.assert_close(y[t], y_ref[i], f"token {t}")

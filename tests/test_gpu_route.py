@@ -63,5 +63,9 @@ def test_precision_request_matches_oracle_away_from_threshold():
         decided = np.abs(w_o - tau) > 1e-5          # the comparison is taken in fp32 on the device
         assert np.array_equal(pr[decided], pr_o[decided])
         assert decided.mean() > 0.99
+        # the exact definition, in the kernel's precision: the flag is the oracle's rule applied to the float32
+        # weight the kernel returns and tau as a float32 (every entry, none masked)
+        assert w.dtype == np.float32
+        assert np.array_equal(pr, moe.precision_request(w, np.float32(tau), rank_high))
         if rank_high:
             assert (pr[:, :rank_high] == 1).all()

@@ -43,6 +43,8 @@ def test_decode_stack_routing_cache_and_sampled_layers():
     req = moe.precision_request(w, TAU)
     clear = np.abs(w - TAU) > 1e-6            # the request is decided in fp32 on the GPU: compare away from the edge
     assert np.array_equal(req_g[clear], req[clear]) and clear.mean() > 0.999
+    # exactly, in the kernel's precision: the oracle's rule on the float32 weights the kernel returned
+    assert np.array_equal(req_g, moe.precision_request(w_g, np.float32(TAU)))
     crit = req_g.sum(1)
     assert 0.5 < crit.mean() < 1.0 and crit.max() <= 3        # "0-2 critical experts, below one on average"
     # temporal reuse: about half of the (step, layer) rows repeat the previous step's expert set
