@@ -16,11 +16,15 @@
  *     groups run along K.
  *
  * Weight format (Section 4.2 of the paper; Table 1 footnote 1: grouped asymmetric integer codes).
- *   Every weight has an 8-bit code q; every (row, K-group) has an fp16 scale s and a u8 zero-point
- *   zp.  The code is stored as two 4-bit slice planes: MSB = q >> 4 and LSB = q & 15 (Section 4.1:
- *   MSB and LSB slices are cached separately).  With both slices the weight is s*(q - zp); from the
- *   MSB slice alone it is 16*s*((q >> 4) - (zp >> 4)), i.e. the paper's joint truncation of code
- *   and zero-point with shift = 4.
+ *   Every weight has a b_high-bit code q; every (row, K-group) has an fp16 scale s and a u8 zero-point
+ *   zp.  The code is stored as two slice planes: MSB = q >> shift (b_low bits) and LSB = q & (2^shift - 1),
+ *   shift = b_high - b_low (Section 4.1: MSB and LSB slices are cached separately).  With both slices the
+ *   weight is s*(q - zp); from the MSB slice alone it is 2^shift*s*((q >> shift) - (zp >> shift)), i.e. the
+ *   paper's joint truncation of code and zero-point.  (b_high, b_low) is one of Table 1's three: (8, 4) -
+ *   MAT84, the default everywhere - (6, 3) and (4, 2).  A plane always gives a slice value a nibble: a 3-bit
+ *   or 2-bit slice sits in the low bits of its nibble, so one layout, and one set of kernels, serves the three
+ *   formats; on the device MAT63 and MAT42 therefore take the bytes of MAT84 (the 3- and 2-bit planes a slower
+ *   memory tier would hold are a repacking that this library does not do).
  *
  *   Physical layout of a plane (N % 16 == 0, K % 128 == 0), N*K/2 bytes: rows are grouped in blocks
  *   of 16 and K in tiles of 64; block (rb, st) is 512 contiguous bytes at ((rb*(K/64) + st)*512),
@@ -62,7 +66,7 @@ typedef struct slicemoe_shape {
   int32_t n_experts;           /* routed experts E */
   int32_t top_k;               /* experts per token k <= SLICEMOE_MAX_TOP_K */
   int32_t group;               /* quantisation group along K: 32, 64 or 128 */
-  int32_t b_high, b_low;       /* slice configuration; this build implements (8, 4) */
+  int32_t b_high, b_low;       /* slice configuration: (8, 4), (6, 3) or (4, 2) */
   int32_t n_shared;            /* always-on shared experts (<= SLICEMOE_MAX_SHARED), run at 8 bits */
   int32_t shared_inter;        /* their intermediate width; multiple of 128 */
   int32_t shared_sigmoid_gate; /* 1: shared output is scaled by sigmoid(v . x) */
@@ -97,12 +101,12 @@ size_t slicemoe_meta_count(int N, int K, int group); /* number of (scale, zp) en
  * grouped asymmetric codes) and split into MSB / LSB slice planes (Sections 4.1, 4.2).
  *   W      device, float32 [N, K] row-major (read only)
  *   msb, lsb, scale, zp   device outputs in the physical layout; sizes from the functions above
- * Per (row, group), in float32: lo = min(min w, 0), hi = max(max w, 0), s = fp16((hi - lo)/255)
- * (round to nearest even; a group with hi == lo or s in {0, inf} gets s = 1, zp = 0),
- * zp = clamp(rint(-lo/s), 0, 255), q = clamp(rint(w/s) + zp, 0, 255) with IEEE division and
+ * Per (row, group), in float32, with Q = 2^b_high - 1: lo = min(min w, 0), hi = max(max w, 0),
+ * s = fp16((hi - lo)/Q) (round to nearest even; a group with hi == lo or s in {0, inf} gets s = 1, zp = 0),
+ * zp = clamp(rint(-lo/s), 0, Q), q = clamp(rint(w/s) + zp, 0, Q) with IEEE division and
  * round-half-even.  Bit-exact and deterministic.
- * Errors: INVALID_ARG (null, N % 16, K % 128, K % group), UNSUPPORTED ((b_high,b_low) != (8,4),
- * group not in {32,64,128}), CUDA.
+ * Errors: INVALID_ARG (null, N % 16, K % 128, K % group), UNSUPPORTED ((b_high, b_low) not one of (8,4), (6,3),
+ * (4,2); group not in {32,64,128}), CUDA.
  */
 int slicemoe_pack(const float *W, int N, int K, int group, int b_high, int b_low, void *msb,
                   void *lsb, uint16_t *scale, uint8_t *zp, void *stream);
@@ -321,7 +325,8 @@ int slicemoe_decode_step_host(const slicemoe_shape *shape, const slicemoe_expert
  *                Needs no initialisation; contents are scratch.
  *   status_out_device  device int32, overwritten: OR of SLICEMOE_STATUS_BAD_EXPERT_ID (a pair whose id
  *                is outside [0, E) is skipped) and SLICEMOE_STATUS_MISSING_LSB (expert_prec 1 for an
- *                expert without LSB planes: it runs MSB-only).
+ *                expert without LSB planes: it runs MSB-only) and SLICEMOE_STATUS_WAIT_TIMEOUT (a bounded wait
+ *                inside the GEMM kernel ran out: y is not valid).
  * Shape limits: hidden, inter, shared_inter multiples of 128 (no upper limit on hidden here);
  * T * (k + n_shared) <= 2^28.
  * Errors: INVALID_ARG, UNSUPPORTED, CUDA.  slicemoe_prefill_workspace_bytes returns 0 for a shape or T

@@ -55,5 +55,9 @@ __host__ __device__ inline size_t meta_index(int ngroups, int n, int g) {
 }
 
 inline bool valid_group(int g) { return g == 32 || g == 64 || g == 128; }
+// The slice widths of Table 1: MAT84, MAT63, MAT42 (b_high-bit codes, the top b_low bits form the MSB slice).
+inline bool valid_widths(int b_high, int b_low) {
+  return (b_high == 8 && b_low == 4) || (b_high == 6 && b_low == 3) || (b_high == 4 && b_low == 2);
+}
 
 }  // namespace slicemoe

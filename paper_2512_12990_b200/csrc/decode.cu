@@ -99,6 +99,7 @@ struct DecodeParams {
   int n_experts, n_shared, k;
   int hidden, inter, shared_inter, group;
   int sigmoid_gate;
+  int shift;  // b_high - b_low: the MSB slice is worth 2^shift of the LSB slice's units
   // the routing lists were complete before the work ahead of this kernel in the stream began: they are read, and
   // the routed experts' tiles requested, while that work is still running
   int lists_resident;
@@ -398,8 +399,10 @@ struct LaneRole {
 // One chunk: this warp's 128-column blocks of the 16-row tile(s) in unit0 (and unit1).  The A operand is
 // the nibble plane, the B operand the activation digits starting at `dig`; `sumw` / `binv` are the
 // digits' weighted group sums and block scales for the same columns.
-//   kModeSingle: MSB tile only           -> *out0 += 16 s (Cm - (zp >> 4) X)
-//   kModeBoth:   MSB tile, LSB tile      -> *out0 += s (16 Cm + Cl - zp X)
+//   kModeSingle: MSB tile only           -> *out0 += 2^shift s (Cm - (zp >> shift) X)
+//   kModeBoth:   MSB tile, LSB tile      -> *out0 += s (2^shift Cm + Cl - zp X)
+// with shift = b_high - b_low (4 for 8-bit codes with 4-bit slices; a narrower slice sits in the low bits of its
+// nibble, so the planes and everything below are the same for all widths)
 //   kModePair:   two matrices' MSB tiles -> *out0 += first, *out1 += second (each with its own scales)
 // Unpacking: a plane byte holds row g's nibble (low) and row g + 8's (high).  The fragment registers of
 // row g are the bytes masked to their low nibble; those of row g + 8 are the bytes as they are, worth
@@ -434,11 +437,11 @@ template <int G>
 __device__ __forceinline__ void consume_chunk(const LaneRole& lr, int lane, int gw, int rot, int mode, int nblocks,
                                               const uint8_t* unit0, const uint8_t* unit1, int scale_off, int zp_off,
                                               const uint8_t* dig, const float* sumw, const float* binv, float* out0,
-                                              float* out1) {
+                                              float* out1, int shift) {
   constexpr int SG = 128 / G;
   const bool p8 = mode == kModeBoth, pair = mode == kModePair;
-  const float pfix = p8 ? 1.f : 16.f;
-  const int zsh = p8 ? 0 : 4;
+  const float pfix = p8 ? 1.f : (float)(1 << shift);
+  const int zsh = p8 ? 0 : shift;
   const bool hi = (lr.c >> 1) != 0;
   float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
@@ -466,16 +469,16 @@ __device__ __forceinline__ void consume_chunk(const LaneRole& lr, int lane, int 
           ca1 = hi ? l[sg][2] - l[sg][0] : l[sg][0];
           cb1 = hi ? l[sg][3] - l[sg][1] : l[sg][1];
         }
-        if (p8) {  // both slices: 16 Cm + Cl
-          ca = (ca << 4) + ca1;
-          cb = (cb << 4) + cb1;
+        if (p8) {  // both slices: 2^shift Cm + Cl
+          ca = (ca << shift) + ca1;
+          cb = (cb << shift) + cb1;
         }
         const float x0 = sumw[(b * SG + sg) * 2 + lr.cq];
         {
           const float t = fmaf((float)cb, lr.w1, (float)ca * lr.w0);
           const float sc = __half2float(__ushort_as_half(ms[sg * 16])) * sfix;
           const float z = (float)((int)mz[sg * 16] >> zsh);
-          // both slices: s (16 Cm + Cl - zp X); MSB only: 16 s (Cm - (zp >> 4) X)
+          // both slices: s (2^shift Cm + Cl - zp X); MSB only: 2^shift s (Cm - (zp >> shift) X)
           acc0 = fmaf(sc, fmaf(-z, x0, t), acc0);
         }
         if (pair) {  // the second matrix' scales / zero-points travel in the second unit
@@ -483,7 +486,7 @@ __device__ __forceinline__ void consume_chunk(const LaneRole& lr, int lane, int 
           const uint8_t* mz1 = unit1 + zp_off + (b * SG) * 16 + lr.r;
           const float t = fmaf((float)cb1, lr.w1, (float)ca1 * lr.w0);
           const float sc = __half2float(__ushort_as_half(ms1[sg * 16])) * sfix;
-          const float z = (float)((int)mz1[sg * 16] >> 4);
+          const float z = (float)((int)mz1[sg * 16] >> shift);  // pair chunks are MSB-only
           acc1 = fmaf(sc, fmaf(-z, x0, t), acc1);
         }
       }
@@ -542,10 +545,10 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
           const uint8_t* unit0 = smem + SmemLayout::ring + u0 * kUnitBytes;
           if (sl.prec) {
             consume_chunk<G>(lr, lane, gw, c % kGroupWarps, kModeBoth, nblocks, unit0, unit0 + kUnitBytes, kPlaneUnitBytes,
-                             kPlaneUnitBytes + kScaleUnitBytes, dig, sumw, binv, q < nch ? &part0 : &part1, &unused);
+                             kPlaneUnitBytes + kScaleUnitBytes, dig, sumw, binv, q < nch ? &part0 : &part1, &unused, p.shift);
           } else {
             consume_chunk<G>(lr, lane, gw, c % kGroupWarps, kModePair, nblocks, unit0, unit0 + kUnitBytes, kPlaneUnitBytes,
-                             kPlaneUnitBytes + kScaleUnitBytes, dig, sumw, binv, &part0, &part1);
+                             kPlaneUnitBytes + kScaleUnitBytes, dig, sumw, binv, &part0, &part1, p.shift);
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(empty0 + 8 * (2 * prod + (jp & 1)));
@@ -634,7 +637,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
       const float* binv = reinterpret_cast<const float*>(smem + SmemLayout::hinv) + (col >> 7);
       consume_chunk<G>(lr, lane, gw, rot, p8 ? kModeBoth : kModeSingle, nblocks,
                        smem + SmemLayout::ring + u0 * plan.unit2_bytes, smem + SmemLayout::ring + u1 * plan.unit2_bytes,
-                       plan.scale2_off, plan.zp2_off, dig, sumw, binv, &sacc, &unused);
+                       plan.scale2_off, plan.zp2_off, dig, sumw, binv, &sacc, &unused, p.shift);
       __syncwarp();
       if (lane == 0) {
         mbar_arrive(empty2 + 8 * u0);
@@ -1319,7 +1322,7 @@ static int launch_decode(const DecodeParams& p, int dev, int sms, int gi, cudaSt
 
 static int check_shape(const slicemoe_shape* s) {
   if (!s) return SLICEMOE_E_INVALID_ARG;
-  if (s->b_high != 8 || s->b_low != 4) return SLICEMOE_E_UNSUPPORTED;
+  if (!valid_widths(s->b_high, s->b_low)) return SLICEMOE_E_UNSUPPORTED;
   if (!valid_group(s->group)) return SLICEMOE_E_UNSUPPORTED;
   if (s->hidden <= 0 || s->inter <= 0 || s->n_experts <= 0 || s->top_k < 1) return SLICEMOE_E_INVALID_ARG;
   if (s->top_k > s->n_experts || s->top_k > SLICEMOE_MAX_TOP_K) return SLICEMOE_E_INVALID_ARG;
@@ -1378,6 +1381,7 @@ static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts
   p.group = shape->group;
   p.sigmoid_gate = (n_shared > 0 && shape->shared_sigmoid_gate) ? 1 : 0;
   p.lists_resident = (flags & SLICEMOE_LISTS_RESIDENT) ? 1 : 0;
+  p.shift = shape->b_high - shape->b_low;
   cudaStream_t st = (cudaStream_t)stream;
   p.logits = nullptr;
   p.bias = fused ? fused->bias : nullptr;

@@ -11,7 +11,7 @@
 
 namespace slicemoe {
 
-__global__ void pack_meta_kernel(const float* __restrict__ W, int N, int K, int group,
+__global__ void pack_meta_kernel(const float* __restrict__ W, int N, int K, int group, int qmax,
                                  uint16_t* __restrict__ scale, uint8_t* __restrict__ zp) {
   const int ngroups = K / group;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -31,7 +31,7 @@ __global__ void pack_meta_kernel(const float* __restrict__ W, int N, int K, int 
     hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, off));
   }
   if (lane == 0) {
-    const float s32 = __fdiv_rn(__fsub_rn(hi, lo), 255.0f);
+    const float s32 = __fdiv_rn(__fsub_rn(hi, lo), (float)qmax);
     __half s16 = __float2half_rn(s32);
     float s = __half2float(s16);
     int z = 0;
@@ -40,7 +40,7 @@ __global__ void pack_meta_kernel(const float* __restrict__ W, int N, int K, int 
       s16 = __float2half_rn(1.0f);
     } else {
       const float zf = rintf(__fdiv_rn(-lo, s));
-      z = (int)fminf(fmaxf(zf, 0.0f), 255.0f);
+      z = (int)fminf(fmaxf(zf, 0.0f), (float)qmax);
     }
     const size_t idx = meta_index(ngroups, n, g);
     scale[idx] = __half_as_ushort(s16);
@@ -48,14 +48,14 @@ __global__ void pack_meta_kernel(const float* __restrict__ W, int N, int K, int 
   }
 }
 
-__device__ __forceinline__ int quantise_one(float w, float s, int z) {
+__device__ __forceinline__ int quantise_one(float w, float s, int z, int qmax) {
   float r = rintf(__fdiv_rn(w, s));
   r = fminf(fmaxf(r, -1.0e9f), 1.0e9f);
   int q = (int)r + z;
-  return min(max(q, 0), 255);
+  return min(max(q, 0), qmax);
 }
 
-__global__ void pack_planes_kernel(const float* __restrict__ W, int N, int K, int group,
+__global__ void pack_planes_kernel(const float* __restrict__ W, int N, int K, int group, int qmax, int shift,
                                    const uint16_t* __restrict__ scale, const uint8_t* __restrict__ zp,
                                    uint32_t* __restrict__ msb, uint32_t* __restrict__ lsb) {
   const size_t nwords = (size_t)N * K / 8;
@@ -82,10 +82,10 @@ __global__ void pack_planes_kernel(const float* __restrict__ W, int N, int K, in
     const float vals[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int q = quantise_one(vals[j], s, z);
+      const int q = quantise_one(vals[j], s, z, qmax);
       const int pos = 2 * j + hi;
-      mw |= (uint32_t)(q >> 4) << (4 * pos);
-      lw |= (uint32_t)(q & 15) << (4 * pos);
+      mw |= (uint32_t)(q >> shift) << (4 * pos);  // a slice narrower than 4 bits sits in the low bits of its nibble
+      lw |= (uint32_t)(q & ((1 << shift) - 1)) << (4 * pos);
     }
   }
   msb[widx] = mw;
@@ -138,19 +138,20 @@ extern "C" size_t slicemoe_meta_count(int N, int K, int group) {
 extern "C" int slicemoe_pack(const float* W, int N, int K, int group, int b_high, int b_low, void* msb,
                              void* lsb, uint16_t* scale, uint8_t* zp, void* stream) {
   if (!W || !msb || !lsb || !scale || !zp) return SLICEMOE_E_INVALID_ARG;
-  if (b_high != 8 || b_low != 4) return SLICEMOE_E_UNSUPPORTED;
+  if (!valid_widths(b_high, b_low)) return SLICEMOE_E_UNSUPPORTED;
+  const int qmax = (1 << b_high) - 1, shift = b_high - b_low;
   const int rc = check_dims(N, K, group);
   if (rc != SLICEMOE_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   const long long nwarps = (long long)N * (K / group);
   const int threads = 256;
   const long long blocks_meta = (nwarps * 32 + threads - 1) / threads;
-  pack_meta_kernel<<<(unsigned)blocks_meta, threads, 0, st>>>(W, N, K, group, scale, zp);
+  pack_meta_kernel<<<(unsigned)blocks_meta, threads, 0, st>>>(W, N, K, group, qmax, scale, zp);
   SM_LAUNCH_CHECK();
   const size_t nwords = (size_t)N * K / 8;
   const size_t blocks_planes = (nwords + threads - 1) / threads;
   pack_planes_kernel<<<(unsigned)blocks_planes, threads, 0, st>>>(
-      W, N, K, group, scale, zp, reinterpret_cast<uint32_t*>(msb), reinterpret_cast<uint32_t*>(lsb));
+      W, N, K, group, qmax, shift, scale, zp, reinterpret_cast<uint32_t*>(msb), reinterpret_cast<uint32_t*>(lsb));
   SM_LAUNCH_CHECK();
   return SLICEMOE_OK;
 }

@@ -182,6 +182,7 @@ struct PfGemmParams {
   float* yrow;                     // phase 2 output [rows, hidden]
   unsigned* status;
   int E, hidden, inter, shared_inter, ldh;
+  int shift;  // b_high - b_low
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -539,7 +540,7 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
         __half2 off[kGpc], fac[kGpc];
 #pragma unroll
         for (int i = 0; i < kGpc; ++i) {
-          off[i] = __half2half2(__int2half_rn(1024 + (w.prec ? z_next[i] : (z_next[i] & 0xf0))));
+          off[i] = __half2half2(__int2half_rn(1024 + (w.prec ? z_next[i] : ((z_next[i] >> p.shift) << p.shift))));
           fac[i] = __half2half2(__float2half_rn(__half2float(__ushort_as_half(s_next[i])) * rnorm));  // exact: a power of two
         }
         if (kc + kUSets < nk) {
@@ -562,9 +563,10 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
               const uint32_t m0 = mws[4 * c + wd] >> sh, l0 = lws[4 * c + wd] >> sh;
-              // both slices: the 8-bit code; MSB slice alone: 16 x its 4-bit code (the factor 16 of the low-bit
-              // dequantisation, exact in fp16)
-              const uint32_t qv = ((m0 & 0x0f0f0f0fu) << 4) | (l0 & 0x0f0f0f0fu);
+              // both slices: the whole code; MSB slice alone: 2^shift x its code (the factor of the low-bit
+              // dequantisation, exact in fp16).  shift = 4 for 8-bit codes; narrower slices sit in the low bits
+              // of their nibbles, so a code never exceeds a byte
+              const uint32_t qv = ((m0 & 0x0f0f0f0fu) << p.shift) | (l0 & 0x0f0f0f0fu);
               // bytes -> fp16 1024 + code, minus (1024 + zero-point): the integer d = q - zp, exact
               uint32_t h01 = __byte_perm(qv, 0x64646464u, 0x4140), h23 = __byte_perm(qv, 0x64646464u, 0x4342);
               const __half2 o = off[kGpc == 2 ? (wd >> 1) : 0], f = fac[kGpc == 2 ? (wd >> 1) : 0];
@@ -750,7 +752,7 @@ static int pf_launch_gemms(const PfGemmParams& p, const __half* xs, int rmax, cu
 
 static int pf_check(const slicemoe_shape* s, int T) {
   if (!s || T <= 0) return SLICEMOE_E_INVALID_ARG;
-  if (s->b_high != 8 || s->b_low != 4) return SLICEMOE_E_UNSUPPORTED;
+  if (!valid_widths(s->b_high, s->b_low)) return SLICEMOE_E_UNSUPPORTED;
   if (!valid_group(s->group)) return SLICEMOE_E_UNSUPPORTED;
   if (s->hidden <= 0 || s->inter <= 0 || s->n_experts <= 0 || s->top_k < 1) return SLICEMOE_E_INVALID_ARG;
   if (s->top_k > s->n_experts || s->top_k > SLICEMOE_MAX_TOP_K) return SLICEMOE_E_INVALID_ARG;
@@ -836,6 +838,7 @@ extern "C" int slicemoe_prefill_layer(const slicemoe_shape* s, const slicemoe_ex
   p.inter = s->inter;
   p.shared_inter = shared_inter;
   p.ldh = s->inter > shared_inter ? s->inter : shared_inter;
+  p.shift = s->b_high - s->b_low;
   if (s->group == 128) {
     rc = pf_launch_gemms<128>(p, xs, L.rmax, st);
   } else if (s->group == 64) {

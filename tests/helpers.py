@@ -31,13 +31,13 @@ class Layer:
     Only the experts in `needed` (plus two decoys) are generated; every other slot of the device expert
     table points at a decoy, so that a wrong expert id shows up as a numerical mismatch."""
 
-    def __init__(self, shape: synth.Shape, needed, layer: int = 0, device="cuda"):
+    def __init__(self, shape: synth.Shape, needed, layer: int = 0, device="cuda", b_high: int = 8, b_low: int = 4):
         import torch
         from oracle import amat
         from paper_2512_12990_b200 import binding as B
         self.shape = shape
         self.cshape = B.make_shape(shape.hidden, shape.inter, shape.n_experts, shape.top_k, shape.group,
-                                   shape.n_shared, shape.shared_inter, shape.shared_sigmoid_gate)
+                                   shape.n_shared, shape.shared_inter, shape.shared_sigmoid_gate, b_high, b_low)
         needed = sorted(set(int(e) for e in needed))
         decoys = [e for e in range(shape.n_experts) if e not in needed][:1]
         self.oracle_experts = {}
@@ -46,11 +46,11 @@ class Layer:
 
         def make(tag, inter):
             W = synth.expert_weights(shape.seed, layer, tag, shape.hidden, inter)
-            o = {k: amat.pack_matrix(W[k], shape.group) for k in ("gate", "up", "down")}
+            o = {k: amat.pack_matrix(W[k], shape.group, b_high, b_low) for k in ("gate", "up", "down")}
             d = {}
             for k in ("gate", "up", "down"):
                 Wd = torch.from_numpy(W[k]).to(device)
-                d[k] = B.slicemoe_pack(Wd, shape.group)
+                d[k] = B.slicemoe_pack(Wd, shape.group, b_high, b_low)
             return o, d
 
         for e in needed + decoys:

@@ -44,7 +44,7 @@ def test_argument_errors_are_codes_not_faults():
     L = B.lib()
     one = ctypes.c_void_p(16)     # never dereferenced: the checks come first
     assert L.slicemoe_pack(None, 16, 128, 128, 8, 4, one, one, one, one, None) == B.E_INVALID_ARG
-    assert L.slicemoe_pack(one, 16, 128, 128, 6, 3, one, one, one, one, None) == B.E_UNSUPPORTED
+    assert L.slicemoe_pack(one, 16, 128, 128, 8, 3, one, one, one, one, None) == B.E_UNSUPPORTED
     assert L.slicemoe_pack(one, 15, 128, 128, 8, 4, one, one, one, one, None) == B.E_INVALID_ARG
     assert L.slicemoe_pack(one, 16, 192, 128, 8, 4, one, one, one, one, None) == B.E_INVALID_ARG
     assert L.slicemoe_pack(one, 16, 128, 48, 8, 4, one, one, one, one, None) == B.E_UNSUPPORTED
@@ -58,7 +58,7 @@ def test_argument_errors_are_codes_not_faults():
     assert L.slicemoe_expert_ffn(ctypes.byref(sh), one, one, 1, one, one, one, one, ws, 16, None) == B.E_INVALID_ARG
     assert L.slicemoe_expert_ffn(ctypes.byref(sh), None, one, 1, one, one, one, one, ws, big, None) == B.E_INVALID_ARG
     assert L.slicemoe_expert_ffn(ctypes.byref(sh), one, one, 0, one, one, one, one, ws, big, None) == B.E_INVALID_ARG
-    bad = B.make_shape(2048, 1408, 64, 6, 128, b_high=6, b_low=3)
+    bad = B.make_shape(2048, 1408, 64, 6, 128, b_high=6, b_low=4)
     assert L.slicemoe_expert_ffn(ctypes.byref(bad), one, one, 1, one, one, one, one, ws, big, None) == B.E_UNSUPPORTED
     bad = B.make_shape(2000, 1408, 64, 6, 128)
     assert L.slicemoe_expert_ffn(ctypes.byref(bad), one, one, 1, one, one, one, one, ws, big, None) == B.E_INVALID_ARG

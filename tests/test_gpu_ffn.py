@@ -364,3 +364,25 @@ def test_full_size_decode_three_tokens_three_precision_mixes(name, rank_high, to
     y_ref = moe.layer(x64, L.oracle_list(), ids2, prec2, w, shared=L.oracle_shared, shared_gate_vec=L.gate_vec)
     assert status == 0
     H.assert_close(y, y_ref, f"{name} token {token} same expert twice")
+
+
+@pytest.mark.parametrize("b_high,b_low", [(6, 3), (4, 2)])
+@pytest.mark.parametrize("name", ["tiny", "dsv2"])
+def test_narrower_slice_formats_decode(name, b_high, b_low):
+    """MAT63 and MAT42 (Section 4.2, Table 1) through pack and the decode kernel: the layer at the mixed precision
+    list, all from both slices and all from the MSB slice alone, against the oracle run with the same widths."""
+    sh = synth.SHAPES[name]
+    logits = synth.router_logits_normal(sh.seed, ("narrow-logits", b_high), 1, sh.n_experts)
+    ids, w, _ = moe.route_topk(logits, sh.top_k)
+    L = H.Layer(sh, ids[0], b_high=b_high, b_low=b_low)
+    xbits, x64 = H.x_inputs(sh, 1, f"narrow-x{b_high}")
+    half = (np.arange(sh.top_k)[None, :] < (sh.top_k + 1) // 2).astype(np.uint8)
+    refs = {}
+    for label, prec in (("mixed", half), ("both slices", np.ones_like(half)), ("MSB only", np.zeros_like(half))):
+        y, status = _run_layer(L, xbits, ids, prec, w)
+        y_ref = moe.layer(x64, L.oracle_list(), ids, prec, w, shared=L.oracle_shared, shared_gate_vec=L.gate_vec)
+        assert status == 0
+        H.assert_close(y, y_ref, f"{name} MAT{b_high}{b_low} {label}")
+        refs[label] = y_ref
+    # the low-bit result really is a different (coarser) model
+    assert np.linalg.norm(refs["both slices"] - refs["MSB only"]) > 2e-2 * np.linalg.norm(refs["both slices"])

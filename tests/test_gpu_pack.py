@@ -9,11 +9,11 @@ from paper_2512_12990_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def _pack_both(W, group):
+def _pack_both(W, group, b_high=8, b_low=4):
     import torch
     from paper_2512_12990_b200 import binding as B
     N, K = W.shape
-    pm = B.slicemoe_pack(torch.from_numpy(W).cuda(), group)
+    pm = B.slicemoe_pack(torch.from_numpy(W).cuda(), group, b_high, b_low)
     msb = B.slicemoe_unpack_plane(pm.msb, N, K).cpu().numpy()
     lsb = B.slicemoe_unpack_plane(pm.lsb, N, K).cpu().numpy()
     s, z = B.slicemoe_unpack_meta(pm.scale, pm.zp, N, K, group)
@@ -21,14 +21,15 @@ def _pack_both(W, group):
     return pm, msb, lsb, s.cpu().numpy(), z.cpu().numpy()
 
 
-def _check(W, group):
-    o = amat.pack_matrix(W, group)
-    pm, msb, lsb, s, z = _pack_both(W, group)
+def _check(W, group, b_high=8, b_low=4):
+    o = amat.pack_matrix(W, group, b_high, b_low)
+    pm, msb, lsb, s, z = _pack_both(W, group, b_high, b_low)
     assert np.array_equal(s.view(np.uint16), o["scale"].view(np.uint16)), "scale bits"
     assert np.array_equal(z, o["zp"]), "zero-points"
     assert np.array_equal(msb, o["msb"]), "MSB plane"
     assert np.array_equal(lsb, o["lsb"]), "LSB plane"
-    assert np.array_equal(msb.astype(np.int32) * 16 + lsb, o["q"])
+    assert np.array_equal((msb.astype(np.int32) << (b_high - b_low)) + lsb, o["q"])
+    assert msb.max() < (1 << b_low) and lsb.max() < (1 << (b_high - b_low))
     return pm, o
 
 
@@ -40,6 +41,18 @@ def _check(W, group):
 def test_pack_bit_exact(N, K, group):
     W = synth.normal_f32(77, ("pack", N, K, group), (N, K), 0.02)
     _check(W, group)
+
+
+@pytest.mark.parametrize("b_high,b_low", [(6, 3), (4, 2)])
+@pytest.mark.parametrize("N,K,group", [(128, 256, 64), (1408, 2048, 128), (2048, 1408, 128), (48, 384, 32)])
+def test_pack_bit_exact_narrower_slices(N, K, group, b_high, b_low):
+    """MAT63 and MAT42 (Table 1): 6- and 4-bit codes, MSB slice = the top 3 / 2 bits, bit for bit the oracle's."""
+    W = synth.normal_f32(79, ("pack", N, K, group, b_high), (N, K), 0.02)
+    _check(W, group, b_high, b_low)
+    # values that sit on the clamps and on rounding ties as well
+    W2 = W.copy()
+    W2[0, :8] = [0.0, 1.0, -1.0, 0.5, -0.5, 1e-8, 3.0, -3.0]
+    _check(W2, group, b_high, b_low)
 
 
 def test_pack_large_shared_expert_matrix():

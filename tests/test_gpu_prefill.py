@@ -71,6 +71,25 @@ def test_small_layers_every_token(group, n_shared, gated):
     assert np.linalg.norm(y_flip_ref - y_ref) > 50 * np.linalg.norm(y - y_ref)
 
 
+@pytest.mark.parametrize("b_high,b_low", [(6, 3), (4, 2)])
+def test_narrower_slice_formats_prefill(b_high, b_low):
+    """MAT63 and MAT42 (Section 4.2, Table 1) through pack and the prefill kernel: 200 tokens, mixed per-expert
+    precision and its flip, every token against the oracle run with the same widths."""
+    sh = _small_shape(64, 1, True, 4300 + b_high)
+    L = H.Layer(sh, range(sh.n_experts), b_high=b_high, b_low=b_low)
+    T = 200
+    logits = synth.router_logits_normal(sh.seed, ("pf-narrow-logits",), T, sh.n_experts)
+    ids, w, _ = moe.route_topk(logits, sh.top_k)
+    expert_prec = (np.arange(sh.n_experts) % 2).astype(np.uint8)
+    xbits, x64 = H.x_inputs(sh, T, "pf-narrow-x")
+    for ep in (expert_prec, 1 - expert_prec):
+        y, status = _prefill(L, xbits, ids, w, ep)
+        assert status == 0
+        y_ref = _oracle(L, x64, ids, w, ep)
+        for t in range(T):
+            H.assert_close(y[t], y_ref[t], f"MAT{b_high}{b_low} token {t}")
+
+
 def test_single_token_and_agreement_with_decode_kernel():
     """T = 1 (one ragged tile per expert) and T = 5: the prefill path and the batch-1 decode path agree
     with the oracle and therefore with each other."""

@@ -36,6 +36,8 @@ def test_static_scratch_entry_point_matches_workspace_entry_point_twice():
         assert np.isfinite(a).all()
         for t in range(T):
             H.assert_close(a[t], b[t], f"call {call} token {t}: static scratch vs caller workspace")
+        # the summation order is fixed and both paths run the same kernel on the same grid: the same bits
+        assert np.array_equal(a, b)
         y_ref = moe.layer(x64, L.oracle_list(), ids, prec, w, shared=L.oracle_shared, shared_gate_vec=L.gate_vec)
         for t in range(T):
             H.assert_close(a[t], y_ref[t], f"call {call} token {t}: static scratch vs oracle")
