@@ -847,6 +847,65 @@ def warmup_comparison(B, synth, sh, NL, ids_h, preq_h, cap, msb_b, lsb_b, tau, d
     return out
 
 
+def cost_table(B, sh, NL, NS, logits_dev, ids_h, preq_h, cap, msb_b, lsb_b, tau, dev, delta=1.0):
+    """The paper's hardware cost model (Section 5: DRAM 1.5 pJ/bit at 104 Gbps, Flash 103 pJ/bit at 10 Gbps, XPU
+    16.4 TOPS at 3.18 TOPS/W) applied to the decode trace under four cache policies of the same capacity, per token:
+    bit-sliced caching with precision on demand, without and with Cache-Prior routing; a conventional cache of whole
+    8-bit experts; the same with Cache-Prior routing (cached experts' logits raised by `delta`; routed again on the device, step by step,
+    because the selection now depends on the cache state); and all experts at the low width."""
+    import torch
+    E, k = sh.n_experts, sh.top_k
+    macs_expert = 3 * sh.hidden * sh.inter
+    shared_macs = sh.n_shared * 3 * sh.hidden * sh.shared_inter
+    shared_bytes = sh.n_shared * expert_bytes(sh.hidden, sh.shared_inter, sh.group, True)   # always resident
+    full_b = msb_b + lsb_b
+
+    def run(policy):
+        sliced = policy.startswith("bit_sliced")
+        if sliced or policy == "low_bit":
+            c = B.Dbsc(cap, msb_b, lsb_b)
+        else:                                  # whole experts: one entry of msb + lsb bytes each
+            c = B.Dbsc(cap, full_b, 1)
+        energy = latency = 0.0
+        flash_total = 0
+        for s_ in range(NS):
+            flash = dram = 0
+            for l in range(NL):
+                r = s_ * NL + l
+                if policy.endswith("cache_prior"):
+                    bias = torch.from_numpy(c.bias(l, E, delta)).to(dev)
+                    sel, _, req = B.slicemoe_route_topk(logits_dev[r:r + 1], k, bias=bias, tau=tau)
+                    row, req_row = sel.cpu().numpy()[0], req.cpu().numpy()[0]
+                else:
+                    row, req_row = ids_h[r], preq_h[r]
+                for j in range(k):
+                    if sliced:
+                        prec, _, _, fb = c.request(s_, l, int(row[j]), bool(req_row[j]))
+                        dram += full_b if prec else msb_b
+                    elif policy == "low_bit":
+                        _, _, _, fb = c.request(s_, l, int(row[j]), False)
+                        dram += msb_b
+                    else:
+                        _, _, _, fb = c.request(s_, l, int(row[j]), False)
+                        dram += full_b
+                    flash += fb
+            e, t = B.slicemoe_cost_step(flash, dram + NL * shared_bytes, NL * (k * macs_expert + shared_macs))
+            energy += e
+            latency += t
+            flash_total += flash
+        return {"mJ_per_token": energy / NS * 1e3, "ms_per_token": latency / NS * 1e3,
+                "flash_MB_per_token": flash_total / NS / 1e6}
+
+    out = {p_: run(p_) for p_ in ("bit_sliced", "bit_sliced_cache_prior", "high_bit_lru", "high_bit_cache_prior",
+                                  "low_bit")}
+    base, ours = out["high_bit_cache_prior"], out["bit_sliced_cache_prior"]
+    out["bit_sliced_cache_prior_vs_high_bit_cache_prior"] = {
+        "energy_gain": base["mJ_per_token"] / ours["mJ_per_token"], "speed_up": base["ms_per_token"] / ours["ms_per_token"]}
+    out["model"] = ("energy = 8 flash_bytes (103 + 1.5) pJ + 8 dram_bytes 1.5 pJ + 2 macs / 3.18 TOPS/W; latency = "
+                    "flash time + max(DRAM time, compute time), per token; Cache-Prior delta = %g on the logit" % delta)
+    return out
+
+
 def run_stack(args, with_warmup_table: bool = True):
     """The 26-layer decode stack over a 256-step routing trace with the host slice cache at 30% capacity:
     microseconds per token for the 26 expert FFNs with precision lists resident (value) and with the cache in the
@@ -989,6 +1048,7 @@ def run_stack(args, with_warmup_table: bool = True):
                         "miss_bytes_over_8bit_bytes": stats["bytes_fetched"] / (stats["requests"] * (msb_b + lsb_b)),
                         "exec_8bit": stats["high_exec"] / stats["requests"],
                         "mean_critical_per_token_layer": float(preq_h.sum(1).mean())},
+        "cost_model": cost_table(B, sh, NL, NS, logits, ids_h, preq_h, cap, msb_b, lsb_b, TAU, dev),
         "cache_warmup": (warmup_comparison(B, synth, sh, NL, ids_h, preq_h, cap, msb_b, lsb_b, TAU, dev)
                          if with_warmup_table else None),
         "e2e": {"value": e2e_us, "unit": "µs/token", "h2d_bytes_per_step": NL * sh.top_k,

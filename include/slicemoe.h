@@ -369,6 +369,40 @@ int slicemoe_dbsc_stats(const slicemoe_dbsc *c, int64_t *out);
 int slicemoe_dbsc_contains(const slicemoe_dbsc *c, int layer, int expert, int *has_msb, int *has_lsb);
 
 /*
+ * The cache-aware routing baselines the paper compares with (Section 2.1; Section 6.1, "Baseline MoE
+ * Acceleration").  The paper names them without formulas; what is implemented:
+ * slicemoe_dbsc_bias - Cache-Prior: bias_out[e] (host float32 [n_experts]) = delta if the MSB slice of
+ *   (layer, e) is resident, else 0: the `bias` input of slicemoe_route_topk, which uses it for selection only.
+ * slicemoe_cumsum_select - Cumsum: experts ranked by descending probability (ties: lower index); the candidate
+ *   set is the shortest prefix of the ranking that holds at least k experts and a probability mass of at least p;
+ *   cached candidates (cached[e] != 0) are selected first, then the others, each in ranking order, k in all.
+ *   probs, cached: host [n_experts]; ids_out: host int32 [k].
+ * Errors: INVALID_ARG, NOMEM.
+ */
+int slicemoe_dbsc_bias(const slicemoe_dbsc *c, int layer, int n_experts, float delta, float *bias_out);
+int slicemoe_cumsum_select(const float *probs, const uint8_t *cached, int n_experts, int k, double p,
+                           int32_t *ids_out);
+
+/*
+ * The hardware cost model of Section 5 (System Implementation), as used for the energy and speed-up figures of
+ * Section 6.3.  Host arithmetic only.  The paper prints the constants, not the model; the model here:
+ *   energy  = 8 flash_bytes (flash_pj + dram_pj) + 8 dram_bytes dram_pj   [pJ]  + 2 macs / tops_per_watt
+ *             (a byte that comes from Flash is also written to DRAM once)
+ *   latency = 8 flash_bytes / flash_gbps + max(8 dram_bytes / dram_gbps, 2 macs / tops)
+ *             (a missed slice arrives before its expert runs; DRAM reads stream under the computation)
+ * slicemoe_cost_paper_hw fills in the paper's numbers: 1.5 and 103 pJ/bit, 104 and 10 Gbps, 16.4 TOPS,
+ * 3.18 TOPS/W.  energy_joule / latency_s may be NULL.  Errors: INVALID_ARG.
+ */
+typedef struct slicemoe_cost_hw {
+  double dram_pj_per_bit, flash_pj_per_bit; /* energy per bit read or written */
+  double dram_gbps, flash_gbps;             /* bandwidth in 10^9 bit/s */
+  double tops, tops_per_watt;               /* 10^12 operations per second, and per joule */
+} slicemoe_cost_hw;
+void slicemoe_cost_paper_hw(slicemoe_cost_hw *hw);
+int slicemoe_cost_step(const slicemoe_cost_hw *hw, int64_t flash_bytes, int64_t dram_bytes, int64_t macs,
+                       double *energy_joule, double *latency_s);
+
+/*
  * Predictive Cache Warmup (Section 4.3): the cache is reshaped while a prompt is prefilled, so that decode
  * starts with the slices it is likely to ask for.  Call slicemoe_dbsc_prefill_layer once per layer, in the
  * order prefill visits them, with the layer's routing result, then slicemoe_dbsc_prefill_end.

@@ -31,7 +31,8 @@ EXPORTS = (
     "slicemoe_decode_step_host", "slicemoe_stream_probe", "slicemoe_layer_static", "slicemoe_layer_routed", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
     "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
     "slicemoe_dbsc_assign", "slicemoe_dbsc_stats", "slicemoe_dbsc_contains",
-    "slicemoe_dbsc_prefill_layer", "slicemoe_dbsc_prefill_end",
+    "slicemoe_dbsc_prefill_layer", "slicemoe_dbsc_prefill_end", "slicemoe_dbsc_bias", "slicemoe_cumsum_select",
+    "slicemoe_cost_paper_hw", "slicemoe_cost_step",
 )
 
 
@@ -42,6 +43,11 @@ class SliceMoEError(RuntimeError):
         if code == E_CUDA:
             detail = ": " + lib().slicemoe_last_cuda_error().decode()
         super().__init__(f"{where}: {strerror(code)} ({code}){detail}")
+
+
+class CostHw(Structure):
+    _fields_ = [("dram_pj_per_bit", c_double), ("flash_pj_per_bit", c_double), ("dram_gbps", c_double),
+                ("flash_gbps", c_double), ("tops", c_double), ("tops_per_watt", c_double)]
 
 
 class Shape(Structure):
@@ -118,6 +124,11 @@ def lib() -> ctypes.CDLL:
     L.slicemoe_dbsc_contains.argtypes = [c_void_p, c_int, c_int, POINTER(c_int), POINTER(c_int)]
     L.slicemoe_dbsc_prefill_layer.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int64, c_int, c_double]
     L.slicemoe_dbsc_prefill_end.argtypes = [c_void_p]
+    L.slicemoe_dbsc_bias.argtypes = [c_void_p, c_int, c_int, c_float, c_void_p]
+    L.slicemoe_cumsum_select.argtypes = [c_void_p, c_void_p, c_int, c_int, c_double, c_void_p]
+    L.slicemoe_cost_paper_hw.argtypes = [POINTER(CostHw)]
+    L.slicemoe_cost_paper_hw.restype = None
+    L.slicemoe_cost_step.argtypes = [POINTER(CostHw), c_int64, c_int64, c_int64, POINTER(c_double), POINTER(c_double)]
     _lib = L
     return L
 
@@ -420,6 +431,13 @@ class Dbsc:
         _check(rc, "slicemoe_dbsc_assign")
         return out
 
+    def bias(self, layer: int, n_experts: int, delta: float):
+        """Cache-Prior bias of a layer: numpy float32 [n_experts]."""
+        import numpy as np
+        out = np.empty(n_experts, dtype=np.float32)
+        _check(lib().slicemoe_dbsc_bias(self._h, layer, n_experts, delta, out.ctypes.data_as(c_void_p)), "slicemoe_dbsc_bias")
+        return out
+
     def stats(self) -> dict:
         buf = (c_int64 * DBSC_NSTATS)()
         _check(lib().slicemoe_dbsc_stats(self._h, buf), "slicemoe_dbsc_stats")
@@ -444,3 +462,31 @@ class Dbsc:
         _check(lib().slicemoe_dbsc_contains(self._h, layer, expert, ctypes.byref(a), ctypes.byref(b)),
                "slicemoe_dbsc_contains")
         return bool(a.value), bool(b.value)
+
+
+# ---- routing baseline and cost model (host) ---------------------------------------------------------
+def slicemoe_cumsum_select(probs, cached, k: int, p: float):
+    """probs: numpy float32 [E]; cached: numpy bool/uint8 [E] -> numpy int32 [k]."""
+    import numpy as np
+    probs = np.ascontiguousarray(probs, dtype=np.float32)
+    cached = np.ascontiguousarray(cached, dtype=np.uint8)
+    out = np.empty(k, dtype=np.int32)
+    rc = lib().slicemoe_cumsum_select(probs.ctypes.data_as(c_void_p), cached.ctypes.data_as(c_void_p), probs.size, k, p,
+                                      out.ctypes.data_as(c_void_p))
+    _check(rc, "slicemoe_cumsum_select")
+    return out
+
+
+def paper_hw() -> CostHw:
+    hw = CostHw()
+    lib().slicemoe_cost_paper_hw(ctypes.byref(hw))
+    return hw
+
+
+def slicemoe_cost_step(flash_bytes: int, dram_bytes: int, macs: int, hw: CostHw | None = None):
+    """(energy in joules, latency in seconds) of one step under the cost model of Section 5."""
+    hw = hw or paper_hw()
+    e, t = c_double(0), c_double(0)
+    _check(lib().slicemoe_cost_step(ctypes.byref(hw), flash_bytes, dram_bytes, macs, ctypes.byref(e), ctypes.byref(t)),
+           "slicemoe_cost_step")
+    return e.value, t.value

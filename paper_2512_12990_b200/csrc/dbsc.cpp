@@ -287,3 +287,59 @@ extern "C" int slicemoe_dbsc_prefill_end(slicemoe_dbsc* c) {
   }
   return SLICEMOE_OK;
 }
+
+// ---- cache-aware routing baselines (Section 2.1; Section 6.1 "Baseline MoE Acceleration") -------------------
+extern "C" int slicemoe_dbsc_bias(const slicemoe_dbsc* c, int layer, int n_experts, float delta, float* bias_out) {
+  if (!c || !bias_out || layer < 0 || n_experts <= 0) return SLICEMOE_E_INVALID_ARG;
+  for (int e = 0; e < n_experts; ++e) bias_out[e] = c->msb.has(make_key(layer, e)) ? delta : 0.0f;
+  return SLICEMOE_OK;
+}
+
+extern "C" int slicemoe_cumsum_select(const float* probs, const uint8_t* cached, int n_experts, int k, double p,
+                                      int32_t* ids_out) {
+  if (!probs || !cached || !ids_out || n_experts <= 0 || k < 1 || k > n_experts) return SLICEMOE_E_INVALID_ARG;
+  try {
+    std::vector<int> order(n_experts);
+    for (int e = 0; e < n_experts; ++e) order[e] = e;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return probs[a] > probs[b]; });
+    // the shortest prefix that holds k experts and a probability mass of at least p (summed in double)
+    int n = 0;
+    double acc = 0.0;
+    while (n < n_experts && (n < k || acc < p)) acc += static_cast<double>(probs[order[n++]]);
+    int out = 0;
+    for (int pass = 0; pass < 2 && out < k; ++pass)  // cached candidates first, each class in ranking order
+      for (int i = 0; i < n && out < k; ++i)
+        if ((cached[order[i]] != 0) == (pass == 0)) ids_out[out++] = order[i];
+  } catch (...) {
+    return SLICEMOE_E_NOMEM;
+  }
+  return SLICEMOE_OK;
+}
+
+// ---- the hardware cost model (Section 5) -------------------------------------------------------------------
+extern "C" void slicemoe_cost_paper_hw(slicemoe_cost_hw* hw) {
+  if (!hw) return;
+  hw->dram_pj_per_bit = 1.5;
+  hw->flash_pj_per_bit = 103.0;
+  hw->dram_gbps = 104.0;
+  hw->flash_gbps = 10.0;
+  hw->tops = 16.4;
+  hw->tops_per_watt = 3.18;
+}
+
+extern "C" int slicemoe_cost_step(const slicemoe_cost_hw* hw, int64_t flash_bytes, int64_t dram_bytes, int64_t macs,
+                                  double* energy_joule, double* latency_s) {
+  if (!hw || flash_bytes < 0 || dram_bytes < 0 || macs < 0) return SLICEMOE_E_INVALID_ARG;
+  if (!(hw->dram_gbps > 0.0) || !(hw->flash_gbps > 0.0) || !(hw->tops > 0.0) || !(hw->tops_per_watt > 0.0))
+    return SLICEMOE_E_INVALID_ARG;
+  const double flash_bits = 8.0 * static_cast<double>(flash_bytes), dram_bits = 8.0 * static_cast<double>(dram_bytes);
+  const double ops = 2.0 * static_cast<double>(macs);
+  if (energy_joule)
+    *energy_joule = flash_bits * hw->flash_pj_per_bit * 1e-12 + (flash_bits + dram_bits) * hw->dram_pj_per_bit * 1e-12 +
+                    ops / (hw->tops_per_watt * 1e12);
+  if (latency_s) {
+    const double t_dram = dram_bits / (hw->dram_gbps * 1e9), t_compute = ops / (hw->tops * 1e12);
+    *latency_s = flash_bits / (hw->flash_gbps * 1e9) + (t_dram > t_compute ? t_dram : t_compute);
+  }
+  return SLICEMOE_OK;
+}
