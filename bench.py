@@ -1027,6 +1027,59 @@ def run_stack(args, with_warmup_table: bool = True):
     sampler.stop()
     if not torch.equal(prec_d[:NE * NL], prec[:NE * NL]):
         raise RuntimeError("cache-in-the-loop precision lists differ from the precomputed ones")
+    # ---- prefill -> decode on the device (Section 4.3): a 512-token prompt through the 26 prefill layers at both
+    # slices while the host cache is reshaped from its routing, the re-order at the end of prefill, then the first
+    # decode tokens with the warmed cache in the loop; the same decode tokens from an empty cache beside it
+    TP, ND = 512, 32
+    pl = torch.from_numpy(synth.prefill_trace_logits(sh.seed, TP, NL, sh.n_experts)).to(dev)
+    xp = torch.from_numpy(synth.activations_bf16(sh.seed, ("bench-stack-prompt",), (TP, sh.hidden)).view(np.int16)).to(dev)
+    xp = xp.view(torch.bfloat16)
+    ws_p = B.new_prefill_workspace(cs, TP, dev)
+    yp = torch.empty((TP, sh.hidden), dtype=torch.float32, device=dev)
+    st_p = torch.zeros(1, dtype=torch.int32, device=dev)
+    all8 = torch.ones(sh.n_experts, dtype=torch.uint8, device=dev)
+    warm = B.Dbsc(cap, msb_b, lsb_b)
+    with torch.cuda.stream(stream):
+        for l in range(2):      # warm-up of the prefill kernels
+            pi, pw_, _ = B.slicemoe_route_topk(pl[l], sh.top_k, stream=stream)
+            B.slicemoe_prefill_layer(cs, layers.tables[l], layers.shared_tables[l], None, xp, pi, pw_, all8, ws_p, yp, st_p, stream)
+        stream.synchronize()
+        t0 = time.time()
+        e0.record(stream)
+        for l in range(NL):
+            pi, pw_, _ = B.slicemoe_route_topk(pl[l], sh.top_k, stream=stream)
+            B.slicemoe_prefill_layer(cs, layers.tables[l], layers.shared_tables[l], None, xp, pi, pw_, all8, ws_p, yp, st_p, stream)
+            warm.prefill_layer(l, pi.cpu().numpy(), pw_.cpu().numpy(), sh.n_experts, TAU)   # synchronises: host bookkeeping
+        warm.prefill_end()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    windows.append((t0, time.time()))
+    prefill_ms = e0.elapsed_time(e1)
+    if int(st_p.item()) != 0:
+        raise RuntimeError("device status word set during the prompt")
+
+    def first_tokens(c):
+        base = c.stats()["bytes_fetched"]
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for s in range(ND):
+                for l in range(NL):
+                    r = s * NL + l
+                    prec_p[0] = torch.from_numpy(c.assign(s, l, ids_h[r], preq_h[r]))
+                    prec_d[r:r + 1].copy_(prec_p, non_blocking=True)
+                    layer(r, l, prec_d)
+            e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / ND, (c.stats()["bytes_fetched"] - base) / 1e6
+
+    warm_us, warm_mb = first_tokens(warm)
+    cold_us, cold_mb = first_tokens(B.Dbsc(cap, msb_b, lsb_b))
+    chain = {"prompt_tokens": TP, "prefill_ms_26_layers": prefill_ms,
+             "prefill_what": "per layer: slicemoe_route_topk, slicemoe_prefill_layer (all experts from both slices), "
+                             "routing result to the host, cache reshaped; then the re-order",
+             "decode_tokens": ND, "decode_us_per_token_warm_cache": warm_us,
+             "MB_fetched_warm_cache": warm_mb, "MB_fetched_empty_cache": cold_mb}
+
     peak, kind = measured_hbm_peak()
     gbs = total_bytes / (us_per_token * NS * 1e-6) / 1e9
     out = {
@@ -1048,6 +1101,7 @@ def run_stack(args, with_warmup_table: bool = True):
                         "miss_bytes_over_8bit_bytes": stats["bytes_fetched"] / (stats["requests"] * (msb_b + lsb_b)),
                         "exec_8bit": stats["high_exec"] / stats["requests"],
                         "mean_critical_per_token_layer": float(preq_h.sum(1).mean())},
+        "prefill_to_decode": chain,
         "cost_model": cost_table(B, sh, NL, NS, logits, ids_h, preq_h, cap, msb_b, lsb_b, TAU, dev),
         "cache_warmup": (warmup_comparison(B, synth, sh, NL, ids_h, preq_h, cap, msb_b, lsb_b, TAU, dev)
                          if with_warmup_table else None),
