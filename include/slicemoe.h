@@ -139,16 +139,16 @@ int slicemoe_route_topk(const float *logits, int T, int E, int k, const float *b
                         void *stream);
 
 /*
- * Workspace.  The FFN kernels need caller-owned device scratch: a header (grid barrier, tickets,
- * status word), the fp32 intermediate h and per-expert partial outputs.  Allocate
- * slicemoe_workspace_bytes() bytes (256-byte aligned) and call slicemoe_workspace_init() once
- * before first use (it zeroes the header; the kernels leave it zeroed again when they finish).
- * One workspace serves one stream at a time.
+ * Workspace.  The FFN kernels need caller-owned device scratch: a header (launch count, status word, wait
+ * limit), two buffers for the fp32 intermediate h (alternate launches use alternate buffers) and staging for the
+ * host-buffer entry point.  Allocate slicemoe_workspace_bytes() bytes (256-byte aligned) and call
+ * slicemoe_workspace_init() once before first use (it zeroes the header and marks both h buffers empty; every
+ * launch leaves the workspace ready for the next).  One workspace serves one stream at a time.
  *
- * The decode kernel's CTAs (one per SM) meet once at a grid-wide barrier, so they must all be resident
- * together.  The library refuses (UNSUPPORTED) a device on which a CTA of the kernel does not fit an SM;
+ * The decode kernel's CTAs (one per SM) wait for the h values that the other CTAs write, so they must all be
+ * resident together.  The library refuses (UNSUPPORTED) a device on which a CTA of the kernel does not fit an SM;
  * it cannot know what else occupies the device at launch time.  If other work holds SMs for longer than the
- * wait limit (default: 10^8 clock cycles, about 50 ms), the barrier's wait ends by itself: the kernel returns,
+ * wait limit (default: 10^8 clock cycles, about 50 ms), the wait for h ends by itself: the kernel returns,
  * SLICEMOE_STATUS_WAIT_TIMEOUT is set and y is not valid.  Run the decode calls on a device (or a
  * partition of it) that they have to themselves while they run.  After a time-out, initialise the workspace again.
  */
@@ -158,8 +158,8 @@ int slicemoe_workspace_init(void *workspace, size_t workspace_bytes, void *strea
 int slicemoe_get_status(void *workspace, int *status_out, void *stream);
 /*
  * Sets the limit of the kernels' device-side waits for this workspace, in GPU clock cycles (0 = the default),
- * and a number of extra arrivals that the grid barrier waits for beyond the grid's own.  extra_arrivals is 0
- * in any real use; a non-zero value makes that wait run out by construction, which is how the time-out path
+ * and a switch that makes the kernels treat h as never complete.  extra_arrivals is 0 in any real use; a
+ * non-zero value makes the wait for h run out by construction, which is how the time-out path
  * is exercised without faulting or hanging anything: the kernel returns by itself after `wait_cycles`,
  * SLICEMOE_STATUS_WAIT_TIMEOUT is set and y is not valid.  slicemoe_workspace_init resets both.  Enqueued
  * on `stream`.
@@ -257,7 +257,7 @@ int slicemoe_stream_probe(const slicemoe_shape *shape, const slicemoe_expert *ex
  * context where the CUDA runtime forbids allocation, under a memory pool that owns every byte of the
  * device, or in a plug-in that receives input and output buffers from its host application and has
  * no allocator of its own.  Such a caller cannot provide the workspace that slicemoe_layer asks for,
- * so this variant keeps the workspace inside the library: a fixed array of 78,016 bytes in device
+ * so this variant keeps the workspace inside the library: a fixed array of 127,168 bytes in device
  * memory that every GPU holds from the moment it loads the library until the process exits.
  *
  * Arguments are those of slicemoe_layer without workspace / workspace_bytes; inputs and outputs are

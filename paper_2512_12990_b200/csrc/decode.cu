@@ -25,7 +25,8 @@
 //     about seven instructions per 512 weights.
 //   * Phase 1 (gate/up + SwiGLU): tasks are (expert slot, 16-row block), split over the CTAs by
 //     bytes.  The epilogue warp adds the warps' partial rows, applies SwiGLU and writes h (fp32) to
-//     the workspace; one bounded grid barrier publishes it.
+//     the workspace.  There is no barrier between the phases: readers poll the h words themselves (two
+//     buffers used by alternate launches, each left "empty" by the launch before; every wait bounded).
 //   * Phase 2 (down + weighted combine): a task is a 16-row block of the OUTPUT over ALL slots, so
 //     the top-k combine stays inside the CTA: no atomics, no cross-CTA reduction, fixed summation
 //     order (results are bit-reproducible).
@@ -65,14 +66,20 @@ constexpr unsigned long long kWaitCycles = 100000000ull;
 
 // ---- workspace --------------------------------------------------------------------------------
 struct WsHeader {
-  unsigned bar_arrive;  // grid barrier: CTAs that finished the gate/up phase
-  unsigned depart;      // CTAs that are through with the barrier word (the last one re-zeroes the header)
+  unsigned readers;     // CTAs of the running launch that have read `epoch` (the last one moves it on)
+  unsigned epoch;       // launches so far on this workspace; its parity selects the h buffer
   unsigned status;      // SLICEMOE_STATUS_* bits
-  unsigned extra_arrivals;         // added to the grid barrier's target (slicemoe_workspace_set_wait; 0 in real use)
+  unsigned extra_arrivals;         // != 0: h never counts as complete (slicemoe_workspace_set_wait; 0 in real use)
   unsigned long long wait_cycles;  // limit of the device-side waits, 0 = kWaitCycles
 };
-constexpr size_t kWsHOff = 2048;                              // float h[kHCap]
-constexpr size_t kWsStageOff = kWsHOff + sizeof(float) * kHCap;
+// The intermediate vector h crosses the grid through the workspace without a barrier: there are two buffers,
+// used by alternate launches; a buffer's words all hold kHEmpty when its launch begins (the launch before
+// wrote that, after the launch before it had read them; slicemoe_workspace_init writes both), a CTA stores its
+// h values with plain stores, and a reader polls the words it needs until none of them is kHEmpty any more.
+// kHEmpty is a NaN pattern that no arithmetic produces (the sign bit of a generated NaN is clear).
+constexpr unsigned kHEmpty = 0xffffffffu;
+constexpr size_t kWsHOff = 2048;                              // float h[2][kHCap]
+constexpr size_t kWsStageOff = kWsHOff + 2 * sizeof(float) * kHCap;
 // host-step staging: x bf16[kMaxHidden] | logits f32[512] | ids i32[16] | w f32[16] | prec u8[16] | y f32[kMaxHidden]
 constexpr size_t kWsStX = kWsStageOff;
 constexpr size_t kWsStLogits = kWsStX + 2 * kMaxHidden;
@@ -141,6 +148,8 @@ struct Slot {
 //     benchmark shapes all - of the phase's tiles are in shared memory before h arrives.
 struct Plan {
   int slot_s, idx_s, count_s;
+  int hpar;         // which h buffer this launch uses
+  int never_ready;  // the time-out exercise: treat h as never complete
   int first_slot, first_idx, count1;
   int count2;
   int nslots;
@@ -184,7 +193,7 @@ static_assert(SmemLayout::slots % 8 == 0 && SmemLayout::hdig % 16 == 0 && SmemLa
 //     empty[2 P + j % 2]; phase 2: P's units are [P h, P h + h), h = nunits2 / 2, taken in running order, one
 //     empty2 barrier per unit (an arrive from each warp of the group that consumed it).
 // pfull1 / pempty1 per group (phase-1 partial rows to the epilogue warp and back), pfull2 / pempty2 (phase-2
-// partial rows of all warps), hx_go (h is complete in the workspace), hs_ready (h is in shared memory as
+// partial rows of all warps), hs_ready (h is in shared memory as
 // digits), p1_done (every consumer warp is through with phase 1, so the ring may be re-cut), plan_ready (the
 // routed part of the plan and the routed slots stand: the producers wait for it after the shared experts' tasks).
 struct Bars {
@@ -269,15 +278,6 @@ __device__ __forceinline__ void mma_u8s8_first(int (&d)[4], uint32_t a0, uint32_
       : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(z));
 }
-__device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
-  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
-  unsigned v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-
 // ---- fixed-point activations ---------------------------------------------------------------------
 // Byte offset, inside a digit buffer, of digit t of the four values k..k+3 (k % 4 == 0): steps of 32
 // columns, 3 digit rows of 32 bytes, and inside a row the order in which the B fragment of m16n8k32 wants
@@ -360,29 +360,45 @@ struct TaskWalk {
 };
 
 // ---- consumers -----------------------------------------------------------------------------------
-// Phase change: wait until the epilogue warp has seen the whole grid's h in the workspace, then turn it
-// into digits (all consumer warps, one 128-block at a time).  Returns false if a wait ran out.
+// Phase change: every consumer warp polls its 128-blocks of the grid's h in the workspace until all of a block's
+// values have been written (see kHEmpty), and turns the block into digits at once: blocks whose CTAs finished early
+// are done before the last CTA's values arrive.  Returns false if the (bounded) wait ran out.
 template <int G>
-__device__ bool fetch_h(const DecodeParams& p, uint8_t* smem, int warp, int lane, int htotal, volatile int* dead,
-                        unsigned* status, uint32_t bars) {
-  const uint32_t hx_go = bars + 8 * Bars::hx_go, hs_ready = bars + 8 * Bars::hs_ready;
-  if (!mbar_wait(hx_go, 0, dead, status)) return false;
-  if (*dead) return false;
+__device__ bool fetch_h(const DecodeParams& p, uint8_t* smem, int warp, int lane, int htotal, const float* hbuf,
+                        bool never_ready, volatile int* dead, unsigned* status, uint32_t bars) {
+  const uint32_t hs_ready = bars + 8 * Bars::hs_ready;
   const int nblk = htotal >> 7;
   constexpr int kMaxIt = (kHCap / 128 + kConsumerWarps - 1) / kConsumerWarps;
-  float4 v[kMaxIt];
+  unsigned pending = 0u;  // warp-uniform
 #pragma unroll
-  for (int it = 0; it < kMaxIt; ++it) {
-    const int blk = it * kConsumerWarps + warp;
-    if (blk < nblk) v[it] = __ldcg(reinterpret_cast<const float4*>(p.ws_h) + blk * 32 + lane);
-  }
+  for (int it = 0; it < kMaxIt; ++it)
+    if (it * kConsumerWarps + warp < nblk) pending |= 1u << it;
+  const long long t0 = clock64();
+  while (pending != 0u) {
+    float4 v[kMaxIt];
 #pragma unroll
-  for (int it = 0; it < kMaxIt; ++it) {
-    const int blk = it * kConsumerWarps + warp;
-    if (blk < nblk) {
-      const float q[4] = {v[it].x, v[it].y, v[it].z, v[it].w};
-      block_to_digits<G>(q, blk * 128, lane, smem + SmemLayout::hdig, reinterpret_cast<float*>(smem + SmemLayout::hsumw),
-                         reinterpret_cast<float*>(smem + SmemLayout::hinv));
+    for (int it = 0; it < kMaxIt; ++it)  // all of the warp's open blocks in flight together; L2 is the point of coherence
+      if ((pending >> it) & 1u) v[it] = __ldcg(reinterpret_cast<const float4*>(hbuf) + (it * kConsumerWarps + warp) * 32 + lane);
+#pragma unroll
+    for (int it = 0; it < kMaxIt; ++it) {
+      if ((pending >> it) & 1u) {
+        const bool mine = __float_as_uint(v[it].x) != kHEmpty && __float_as_uint(v[it].y) != kHEmpty &&
+                          __float_as_uint(v[it].z) != kHEmpty && __float_as_uint(v[it].w) != kHEmpty;
+        if (__all_sync(0xffffffffu, mine) && !never_ready) {
+          const float q[4] = {v[it].x, v[it].y, v[it].z, v[it].w};
+          block_to_digits<G>(q, (it * kConsumerWarps + warp) * 128, lane, smem + SmemLayout::hdig,
+                             reinterpret_cast<float*>(smem + SmemLayout::hsumw), reinterpret_cast<float*>(smem + SmemLayout::hinv));
+          pending &= ~(1u << it);
+        }
+      }
+    }
+    if (pending != 0u) {
+      if (*dead) return false;
+      if ((unsigned long long)(clock64() - t0) > wait_limit(dead)) {
+        *dead = 1;
+        atomicOr(status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
+        return false;
+      }
     }
   }
   __syncwarp();
@@ -572,7 +588,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
   if (lane == 0) mbar_arrive(bars + 8 * Bars::p1_done);  // this warp no longer reads phase-1 units
   if (plan.count2 == 0) return;
 
-  // ---- while the grid barrier is pending: list this group's phase-2 chunks (the walk over all output row
+  // ---- ahead of the phase change: list this group's phase-2 chunks (the walk over all output row
   // blocks, slots and chunks costs more than consuming the group's own chunks, so it is done ahead of time) ----
   uint4* mylist = reinterpret_cast<uint4*>(smem + SmemLayout::p2list) + warp * kMaxMine;
   int nmine = 0;
@@ -611,7 +627,9 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
   __syncwarp();
 
   // ---- the grid's h ----
-  if (!fetch_h<G>(p, smem, warp, lane, plan.htotal, dead, status, bars)) return;
+  if (!fetch_h<G>(p, smem, warp, lane, plan.htotal, p.ws_h + (size_t)plan.hpar * kHCap, plan.never_ready != 0, dead, status,
+                  bars))
+    return;
 
   // ---- phase 2: chunks round-robin over the groups, all warps contribute to every task ----
   const uint32_t full2 = bars + 8 * Bars::full2, empty2 = bars + 8 * Bars::empty2;
@@ -661,20 +679,16 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
   volatile int* dead = reinterpret_cast<volatile int*>(smem + SmemLayout::dead);
   const uint32_t bars = smem_u32(smem + SmemLayout::bars);
   unsigned* status = &p.ws->status;
-  // A CTA is done with the barrier word once it has arrived and, if it has a second phase, seen the count
-  // complete; the last CTA to say so makes the header reusable.  (The next launch touches the header only after
-  // this whole grid has completed.)  Done here rather than at the end of the kernel: the returning atomic's round
-  // trip would otherwise sit between the last store of y and the SM being free for the next launch.
-  auto depart = [&]() {
-    if (lane == 0) {
-      const unsigned old = atomicAdd(&p.ws->depart, 1u);
-      if (old == gridDim.x - 1) {
-        p.ws->bar_arrive = 0;
-        p.ws->depart = 0;
-        __threadfence();
-      }
-    }
-  };
+  // This CTA's share of the OTHER h buffer goes back to "empty" for the next launch: its last readers were the
+  // launch before this one.
+  {
+    uint4* other = reinterpret_cast<uint4*>(p.ws_h + (size_t)(plan.hpar ^ 1) * kHCap);
+    constexpr int n16 = kHCap / 4;
+    const int per = (n16 + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int lo = (int)blockIdx.x * per, hi = min(n16, lo + per);
+    for (int i = lo + lane; i < hi; i += 32) other[i] = make_uint4(kHEmpty, kHEmpty, kHEmpty, kHEmpty);
+  }
+  float* hbuf = p.ws_h + (size_t)plan.hpar * kHCap;
   // phase 1: one group's four partial rows per task -> SwiGLU -> h
   {
     TaskWalk tw;
@@ -683,10 +697,7 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
       tw.at(plan, n);
       const int slot = tw.slot, idx = tw.idx;
       const int group = n % kGroups, round = n / kGroups;
-      if (!mbar_wait(bars + 8 * (Bars::pfull1 + group), round & 1, dead, status)) {
-        depart();  // a wait ran out: the others will time out at the barrier, the header is still handed back
-        return;
-      }
+      if (!mbar_wait(bars + 8 * (Bars::pfull1 + group), round & 1, dead, status)) return;
       float a = 0.f, b = 0.f;
       if (lane < 16) {
 #pragma unroll
@@ -698,36 +709,9 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + 8 * (Bars::pempty1 + group));
-      if (lane < 16) p.ws_h[slots[slot].hoff + idx * 16 + lane] = a / (1.f + expf(-a)) * b;  // silu(gate) * up
+      if (lane < 16) hbuf[slots[slot].hoff + idx * 16 + lane] = a / (1.f + expf(-a)) * b;  // silu(gate) * up
       tw.next(slots);
     }
-  }
-  // ---- the single grid-wide dependency: every CTA has written its rows of h ----
-  __syncwarp();
-  if (lane == 0) red_release_add(&p.ws->bar_arrive, 1u);
-  if (plan.count2 == 0) {
-    depart();
-    return;
-  }
-  {
-    // the whole warp polls, converged: no lane spins on something another lane must provide
-    const long long t0 = clock64();
-    const unsigned target = gridDim.x + p.ws->extra_arrivals;
-    while (ld_acquire_u32(&p.ws->bar_arrive) < target) {
-      if (*dead) break;
-      if ((unsigned long long)(clock64() - t0) > wait_limit(dead)) {
-        *dead = 1;
-        atomicOr(status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
-        break;
-      }
-    }
-    __syncwarp();
-    if (*dead) {
-      depart();
-      return;
-    }
-    if (lane == 0) mbar_arrive(bars + 8 * Bars::hx_go);
-    depart();
   }
   // phase 2: all warps' partial rows per output row block -> y
   for (int m = 0; m < plan.count2; ++m) {
@@ -1185,7 +1169,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
       }
       mbar_init(bars + 8 * Bars::pfull2, kConsumerWarps);
       mbar_init(bars + 8 * Bars::pempty2, 1);
-      mbar_init(bars + 8 * Bars::hx_go, 1);
       mbar_init(bars + 8 * Bars::hs_ready, kConsumerWarps);
       mbar_init(bars + 8 * Bars::p1_done, kConsumerWarps);
       mbar_init(bars + 8 * Bars::plan_ready, early_lists ? 2 : 1);  // resident lists: warps 0 and 1 each say when done
@@ -1233,9 +1216,20 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
   } else if (warp == 1) {
     if (!early_lists) load_slot_pointers<FUSED>(p, smem, lane, true);
   } else if (warp == 2) {
-    if (lane == 0) {  // a wait limit set by the host for this workspace
+    if (lane == 0) {
+      // a wait limit set by the host for this workspace
       const unsigned long long lim = p.ws->wait_cycles;
       if (lim != 0ull) *reinterpret_cast<unsigned long long*>(smem + SmemLayout::dead + 8) = lim;
+      // Which h buffer: the parity of the launch count.  The count moves on once every CTA of this launch has
+      // read it (the last reader does it), so all of them see the same value, and the next launch the next.
+      const unsigned epoch = p.ws->epoch;
+      plan->hpar = (int)(epoch & 1u);
+      plan->never_ready = p.ws->extra_arrivals != 0u ? 1 : 0;
+      if (atomicAdd(&p.ws->readers, 1u) == gridDim.x - 1u) {
+        p.ws->readers = 0u;
+        p.ws->epoch = epoch + 1u;
+        __threadfence();
+      }
     }
     if (p.sigmoid_gate && p.n_shared > 0) {
       // Qwen-style shared-expert gate: sigmoid(v . x)
@@ -1297,9 +1291,9 @@ static int launch_decode(const DecodeParams& p, int dev, int sms, int gi, cudaSt
   if (!attr_set) {
     SM_CUDA_TRY(cudaFuncSetAttribute(decode_layer_kernel<G, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      SmemLayout::total));
-    // The CTAs meet at a grid barrier, so all of them must be able to be resident at once: one per SM needs
-    // the kernel to fit an SM at all.  (If another kernel holds SMs at the time, the barrier's bounded wait
-    // ends the launch with SLICEMOE_STATUS_WAIT_TIMEOUT instead of a hang.)
+    // Every CTA waits for h values that the other CTAs write, so all of them must be able to be resident at
+    // once: one per SM needs the kernel to fit an SM at all.  (If another kernel holds SMs at the time, the
+    // bounded wait for h ends the launch with SLICEMOE_STATUS_WAIT_TIMEOUT instead of a hang.)
     int per_sm = 0;
     SM_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_layer_kernel<G, FUSED>, kThreads,
                                                               SmemLayout::total));
@@ -1434,7 +1428,10 @@ extern "C" size_t slicemoe_workspace_bytes(const slicemoe_shape* shape) {
 extern "C" int slicemoe_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
   if (!workspace || workspace_bytes < kWsBytes || (reinterpret_cast<uintptr_t>(workspace) & 255))
     return SLICEMOE_E_INVALID_ARG;
+  // header to zero, both h buffers to "empty" (every byte 0xff: see kHEmpty)
   SM_CUDA_TRY(cudaMemsetAsync(workspace, 0, kWsHOff, (cudaStream_t)stream));
+  SM_CUDA_TRY(cudaMemsetAsync(reinterpret_cast<uint8_t*>(workspace) + kWsHOff, 0xff, 2 * sizeof(float) * kHCap,
+                              (cudaStream_t)stream));
   return SLICEMOE_OK;
 }
 
@@ -1581,8 +1578,10 @@ extern "C" int slicemoe_layer_static(const slicemoe_shape* shape, const slicemoe
     g_static_scratch_ptr[dev] = ptr;
   }
   void* ws = g_static_scratch_ptr[dev];
-  // The array keeps whatever the previous call left: the header (barrier counters, status) must start at zero.
+  // The array keeps whatever the previous call left: the header (launch count, status) must start at zero, and the
+  // h buffer the first launch then uses must be empty (the launches clear the other one for their successors).
   SM_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHOff, (cudaStream_t)stream));
+  SM_CUDA_TRY(cudaMemsetAsync(reinterpret_cast<uint8_t*>(ws) + kWsHOff, 0xff, sizeof(float) * kHCap, (cudaStream_t)stream));
   return run_layer(shape, experts, shared, shape->n_shared, shared_gate_vec, x, T, ids, prec, weights, y, ws, kWsBytes,
                    stream);
 }

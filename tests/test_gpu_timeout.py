@@ -1,5 +1,5 @@
 """The time-out path of the decode kernel, exercised without hanging or faulting anything: the workspace is
-told that the grid barrier between the two phases must wait for one arrival more than the grid can deliver,
+told to treat the intermediate vector that the CTAs exchange between the two phases as never complete,
 and that no device-side wait may last longer than about a millisecond.  The kernel has to return by itself,
 report SLICEMOE_STATUS_WAIT_TIMEOUT, and the same workspace has to work again once it is re-initialised."""
 import time
@@ -43,7 +43,7 @@ def test_wait_timeout_is_reported_and_the_workspace_recovers():
     assert time.time() - t0 < 5.0, "the kernel must return by itself"
     status = B.slicemoe_get_status(layer.ws)
     assert status & B.STATUS_WAIT_TIMEOUT
-    assert torch.all(y_bad == 7.0), "the output is not written when the barrier was never complete"
+    assert torch.all(y_bad == 7.0), "the output is not written when h was never complete"
 
     # re-initialised, the workspace works again (and the limit is back to its default)
     B.lib().slicemoe_workspace_init(layer.ws.data_ptr(), layer.ws.numel(), None)
