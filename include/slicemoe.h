@@ -369,6 +369,56 @@ int slicemoe_dbsc_stats(const slicemoe_dbsc *c, int64_t *out);
 int slicemoe_dbsc_contains(const slicemoe_dbsc *c, int layer, int expert, int *has_msb, int *has_lsb);
 
 /*
+ * For a caller that keeps the slices themselves (slicemoe_tier_* below): with logging on, every slice that a
+ * request evicts is remembered until slicemoe_dbsc_drain_evicted hands it out (layer, expert, 1 for an LSB slice;
+ * at most `max` per call, oldest first; returns how many were written, or a negative error).
+ */
+int slicemoe_dbsc_log_evictions(slicemoe_dbsc *c, int on);
+int slicemoe_dbsc_drain_evicted(slicemoe_dbsc *c, int32_t *layers, int32_t *experts, uint8_t *is_lsb, int max);
+
+/*
+ * A second memory tier under the slice cache (Section 5: the full set of weights lives in a large, slow store
+ * and is touched only when a slice misses).  The slow store is pinned host memory, the fast tier a pool of
+ * equal slots in device memory, a miss a copy of the slice's record on a side stream; the decisions are those
+ * of slicemoe_dbsc_* (MSB slices LRU, LSB slices first to go), with both slice kinds charged one slot.
+ *
+ * Records (slicemoe_tier_sizes gives their sizes for a shape, and the slot size = the larger one rounded up to
+ * 256 bytes).  MSB record: gate MSB plane, gate scales, gate zero-points, then up's, then down's.  LSB record:
+ * gate, up, down LSB planes.  The store holds for (layer l, expert e) the MSB record followed by the LSB record
+ * at offset (l * n_experts + e) * (msb_record + lsb_record); slicemoe_tier_store_expert writes one such pair from a
+ * packed expert on the device (device-to-host copies enqueued on `stream`; offline preparation).
+ *
+ * slicemoe_tier_create: store_host (pinned, read only, must outlive the tier); pool_device (256-byte aligned,
+ * pool_bytes >= (1 + 4 * top_k) slots: slot 0 is a stand-in that the table entries of non-resident slices point
+ * to, so that a list naming an expert that was never requested reads defined bytes); tables_device: device array
+ * [n_layers * n_experts] of slicemoe_expert that the tier fills and keeps up to date - pass
+ * tables_device + l * n_experts as `experts` to the layer calls.  Synchronises `stream`.  NULL on bad arguments
+ * or allocation failure.  The tier allocates no device memory.
+ *
+ * slicemoe_tier_request: serves the n selected experts of one (step, layer): decides hits, misses, evictions
+ * and the execution precision (prec_out, host), copies missing records into free slots on `copy_stream` - after
+ * everything already enqueued on `compute_stream` has finished, so that no slice still being read is
+ * overwritten - updates the device tables, and makes `compute_stream` wait for the copies.  The next layer
+ * call on compute_stream with ids / prec_out then finds every slice it reads in the pool: a slice of the list
+ * that a later entry of the same list pushed out of the cache's books again keeps its bytes until the next
+ * request (2 * top_k slots of the pool are set aside for that; the cache is given the rest less slot 0).  ids,
+ * prec_req, prec_out are host arrays.  Errors: INVALID_ARG, UNSUPPORTED (the pool cannot hold the list), NOMEM, CUDA.
+ * Cache warm-up from a prompt (slicemoe_dbsc_prefill_*) is not connected to the tier.
+ */
+typedef struct slicemoe_tier slicemoe_tier;
+int slicemoe_tier_sizes(const slicemoe_shape *shape, size_t *msb_record, size_t *lsb_record, size_t *slot_bytes);
+int slicemoe_tier_store_expert(const slicemoe_shape *shape, const slicemoe_expert *expert, void *record_host,
+                               void *stream);
+slicemoe_tier *slicemoe_tier_create(const slicemoe_shape *shape, int n_layers, const void *store_host,
+                                    void *pool_device, size_t pool_bytes, slicemoe_expert *tables_device,
+                                    double miss_budget, int warmup_steps, void *stream);
+void slicemoe_tier_destroy(slicemoe_tier *t);
+slicemoe_dbsc *slicemoe_tier_cache(slicemoe_tier *t); /* the tier's own cache, for statistics; owned by the tier */
+int slicemoe_tier_request(slicemoe_tier *t, int step, int layer, const int32_t *ids, const uint8_t *prec_req,
+                          int n, uint8_t *prec_out, void *compute_stream, void *copy_stream);
+int slicemoe_tier_stats(const slicemoe_tier *t, int64_t *bytes_copied, int64_t *copies, int64_t *free_slots);
+
+/*
  * The cache-aware routing baselines the paper compares with (Section 2.1; Section 6.1, "Baseline MoE
  * Acceleration").  The paper names them without formulas; what is implemented:
  * slicemoe_dbsc_bias - Cache-Prior: bias_out[e] (host float32 [n_experts]) = delta if the MSB slice of

@@ -32,7 +32,9 @@ EXPORTS = (
     "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
     "slicemoe_dbsc_assign", "slicemoe_dbsc_stats", "slicemoe_dbsc_contains",
     "slicemoe_dbsc_prefill_layer", "slicemoe_dbsc_prefill_end", "slicemoe_dbsc_bias", "slicemoe_cumsum_select",
-    "slicemoe_cost_paper_hw", "slicemoe_cost_step",
+    "slicemoe_cost_paper_hw", "slicemoe_cost_step", "slicemoe_dbsc_log_evictions", "slicemoe_dbsc_drain_evicted",
+    "slicemoe_tier_sizes", "slicemoe_tier_store_expert", "slicemoe_tier_create", "slicemoe_tier_destroy",
+    "slicemoe_tier_cache", "slicemoe_tier_request", "slicemoe_tier_stats",
 )
 
 
@@ -125,6 +127,18 @@ def lib() -> ctypes.CDLL:
     L.slicemoe_dbsc_prefill_layer.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int64, c_int, c_double]
     L.slicemoe_dbsc_prefill_end.argtypes = [c_void_p]
     L.slicemoe_dbsc_bias.argtypes = [c_void_p, c_int, c_int, c_float, c_void_p]
+    L.slicemoe_dbsc_log_evictions.argtypes = [c_void_p, c_int]
+    L.slicemoe_dbsc_drain_evicted.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int]
+    L.slicemoe_tier_sizes.argtypes = [POINTER(Shape), POINTER(c_size_t), POINTER(c_size_t), POINTER(c_size_t)]
+    L.slicemoe_tier_store_expert.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p]
+    L.slicemoe_tier_create.restype = c_void_p
+    L.slicemoe_tier_create.argtypes = [POINTER(Shape), c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_double, c_int, c_void_p]
+    L.slicemoe_tier_destroy.argtypes = [c_void_p]
+    L.slicemoe_tier_destroy.restype = None
+    L.slicemoe_tier_cache.restype = c_void_p
+    L.slicemoe_tier_cache.argtypes = [c_void_p]
+    L.slicemoe_tier_request.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+    L.slicemoe_tier_stats.argtypes = [c_void_p, POINTER(c_int64), POINTER(c_int64), POINTER(c_int64)]
     L.slicemoe_cumsum_select.argtypes = [c_void_p, c_void_p, c_int, c_int, c_double, c_void_p]
     L.slicemoe_cost_paper_hw.argtypes = [POINTER(CostHw)]
     L.slicemoe_cost_paper_hw.restype = None
@@ -490,3 +504,81 @@ def slicemoe_cost_step(flash_bytes: int, dram_bytes: int, macs: int, hw: CostHw 
     _check(lib().slicemoe_cost_step(ctypes.byref(hw), flash_bytes, dram_bytes, macs, ctypes.byref(e), ctypes.byref(t)),
            "slicemoe_cost_step")
     return e.value, t.value
+
+
+# ---- second memory tier --------------------------------------------------------------------------------
+def slicemoe_tier_sizes(shape: Shape):
+    """(msb_record, lsb_record, slot_bytes) of a shape."""
+    m, l, sl = c_size_t(0), c_size_t(0), c_size_t(0)
+    _check(lib().slicemoe_tier_sizes(ctypes.byref(shape), ctypes.byref(m), ctypes.byref(l), ctypes.byref(sl)),
+           "slicemoe_tier_sizes")
+    return m.value, l.value, sl.value
+
+
+class Tier:
+    """slicemoe_tier_*: a pool of slice slots in device memory over a store in pinned host memory.
+
+    `layers`: list (per layer) of lists (per expert) of dict(gate=PackedMat, up=..., down=...) on the device; their
+    records are copied into one pinned host buffer (the slow store), after which the caller may drop them.  All
+    memory is allocated here, in the binding, with torch; the library allocates none."""
+
+    def __init__(self, shape: Shape, layers, pool_slots: int, miss_budget: float | None = None, warmup_steps: int = 10,
+                 device="cuda"):
+        import torch
+        self.shape, self.n_layers, self.n_experts = shape, len(layers), len(layers[0])
+        m, l, slot = slicemoe_tier_sizes(shape)
+        self.msb_record, self.lsb_record, self.slot_bytes = m, l, slot
+        self.store = torch.empty((self.n_layers * self.n_experts, m + l), dtype=torch.uint8).pin_memory()
+        for li, experts in enumerate(layers):
+            for e, ex in enumerate(experts):
+                rec = Expert(ex["gate"].desc(), ex["up"].desc(), ex["down"].desc())
+                rc = lib().slicemoe_tier_store_expert(ctypes.byref(shape), ctypes.byref(rec),
+                                                      c_void_p(self.store[li * self.n_experts + e].data_ptr()), _stream(None))
+                _check(rc, "slicemoe_tier_store_expert")
+        torch.cuda.synchronize()
+        self.pool = torch.empty(pool_slots * slot, dtype=torch.uint8, device=device)
+        self.tables = torch.empty(self.n_layers * self.n_experts * ctypes.sizeof(Expert), dtype=torch.uint8, device=device)
+        self.copy_stream = torch.cuda.Stream(device=device)
+        self._h = lib().slicemoe_tier_create(ctypes.byref(shape), self.n_layers, c_void_p(self.store.data_ptr()),
+                                             _ptr(self.pool), self.pool.numel(), _ptr(self.tables),
+                                             -1.0 if miss_budget is None else float(miss_budget), warmup_steps,
+                                             _stream(None))
+        if not self._h:
+            raise SliceMoEError(E_INVALID_ARG, "slicemoe_tier_create")
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().slicemoe_tier_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def layer_table(self, layer: int):
+        """The device expert table of a layer (a view into the tier's table array)."""
+        n = self.n_experts * ctypes.sizeof(Expert)
+        return self.tables[layer * n:(layer + 1) * n]
+
+    def request(self, step: int, layer: int, ids, prec_req, compute_stream=None):
+        """ids int32 [n], prec_req uint8 [n] (numpy, host) -> prec uint8 [n]; enqueues the copies and the waits."""
+        import numpy as np
+        ids = np.ascontiguousarray(ids, dtype=np.int32)
+        prec_req = np.ascontiguousarray(prec_req, dtype=np.uint8)
+        out = np.empty(ids.shape, dtype=np.uint8)
+        rc = lib().slicemoe_tier_request(self._h, step, layer, ids.ctypes.data_as(c_void_p),
+                                         prec_req.ctypes.data_as(c_void_p), ids.size, out.ctypes.data_as(c_void_p),
+                                         _stream(compute_stream), c_void_p(self.copy_stream.cuda_stream))
+        _check(rc, "slicemoe_tier_request")
+        return out
+
+    def stats(self) -> dict:
+        b, c, f = c_int64(0), c_int64(0), c_int64(0)
+        _check(lib().slicemoe_tier_stats(self._h, ctypes.byref(b), ctypes.byref(c), ctypes.byref(f)), "slicemoe_tier_stats")
+        out = (c_int64 * DBSC_NSTATS)()
+        _check(lib().slicemoe_dbsc_stats(lib().slicemoe_tier_cache(self._h), out), "slicemoe_dbsc_stats")
+        d = {k: int(v) for k, v in zip(DBSC_STAT_NAMES, out)}
+        d.update(bytes_copied=b.value, copies=c.value, free_slots=f.value)
+        return d

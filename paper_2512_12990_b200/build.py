@@ -12,7 +12,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libslicemoe.so")
-SOURCES = ["api.cu", "pack.cu", "route.cu", "decode.cu", "stream.cu", "prefill.cu", "dbsc.cpp"]
+SOURCES = ["api.cu", "pack.cu", "route.cu", "decode.cu", "stream.cu", "prefill.cu", "tier.cu", "dbsc.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

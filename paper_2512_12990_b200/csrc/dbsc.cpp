@@ -42,10 +42,11 @@ struct Queue {
     order.erase(it->second);
     where.erase(it);
   }
-  // Removes the first entry that is not `protect`; false if there is none.
-  bool evict_one(uint64_t protect) {
+  // Removes the first entry that is not `protect` (and names it); false if there is none.
+  bool evict_one(uint64_t protect, uint64_t* victim) {
     for (auto it = order.begin(); it != order.end(); ++it) {
       if (*it != protect) {
+        *victim = *it;
         where.erase(*it);
         order.erase(it);
         return true;
@@ -66,6 +67,9 @@ struct slicemoe_dbsc {
       win_fetched, win_full;
   struct Hotness { int64_t freq; double score; };  // prompt tokens routed to the expert; their mean gating score
   std::unordered_map<uint64_t, Hotness> hot;       // statistics of the prefill in progress
+  // For a caller that keeps the slices themselves (slicemoe_tier): what request() evicted, until it is drained.
+  bool log_evictions = false;
+  std::vector<std::pair<uint64_t, int>> evicted;   // (key, 1 = LSB slice)
 
   // Eviction keys of Section 4.3; a slice without statistics (left from before the prompt) goes first.
   std::tuple<double, int64_t, uint64_t> lsb_rank(uint64_t k) const {
@@ -132,10 +136,13 @@ struct slicemoe_dbsc {
   bool make_room(int64_t need, uint64_t protect) {
     if (need > capacity) return false;
     while (capacity - used < need) {
-      if (lsb.evict_one(protect)) {
+      uint64_t victim = 0;
+      if (lsb.evict_one(protect, &victim)) {
         used -= lsb_bytes;
-      } else if (msb.evict_one(protect)) {
+        if (log_evictions) evicted.emplace_back(victim, 1);
+      } else if (msb.evict_one(protect, &victim)) {
         used -= msb_bytes;
+        if (log_evictions) evicted.emplace_back(victim, 0);
       } else {
         return false;
       }
@@ -286,6 +293,25 @@ extern "C" int slicemoe_dbsc_prefill_end(slicemoe_dbsc* c) {
     return SLICEMOE_E_NOMEM;
   }
   return SLICEMOE_OK;
+}
+
+extern "C" int slicemoe_dbsc_log_evictions(slicemoe_dbsc* c, int on) {
+  if (!c) return SLICEMOE_E_INVALID_ARG;
+  c->log_evictions = on != 0;
+  if (!on) c->evicted.clear();
+  return SLICEMOE_OK;
+}
+
+extern "C" int slicemoe_dbsc_drain_evicted(slicemoe_dbsc* c, int32_t* layers, int32_t* experts, uint8_t* is_lsb, int max) {
+  if (!c || !layers || !experts || !is_lsb || max < 0) return SLICEMOE_E_INVALID_ARG;
+  const int n = static_cast<int>(std::min<size_t>(c->evicted.size(), static_cast<size_t>(max)));
+  for (int i = 0; i < n; ++i) {
+    layers[i] = static_cast<int32_t>(c->evicted[i].first >> 32);
+    experts[i] = static_cast<int32_t>(c->evicted[i].first & 0xffffffffu);
+    is_lsb[i] = static_cast<uint8_t>(c->evicted[i].second);
+  }
+  c->evicted.erase(c->evicted.begin(), c->evicted.begin() + n);
+  return n;
 }
 
 // ---- cache-aware routing baselines (Section 2.1; Section 6.1 "Baseline MoE Acceleration") -------------------

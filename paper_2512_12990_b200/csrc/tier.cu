@@ -1,0 +1,291 @@
+// A second memory tier under the slice cache (Section 5: all weights live in a large, slow store and are brought
+// into the fast memory only when a slice misses).  Here the fast memory is a pool of slots in device memory, the
+// slow store pinned host memory, and a miss is a copy of the slice's record on a side stream.  The cache decisions
+// are the host bookkeeping of slicemoe_dbsc_*; this file keeps the bytes where the decisions say they are, and the
+// device expert tables pointing at them.
+//
+// A record is what one slice of one expert consists of, back to back:
+//   MSB record: gate MSB plane, gate scales, gate zero-points, then the same of up, then of down
+//   LSB record: gate LSB plane, up LSB plane, down LSB plane
+// and the store holds, for (layer l, expert e), the MSB record followed by the LSB record at
+// (l * n_experts + e) * (msb_record + lsb_record).
+// Every slot of the pool has the size of the larger record (rounded up to 256 bytes), so any slice fits any slot;
+// slot 0 is never given out: table entries of slices that are not resident point there, so that a list naming
+// an expert the caller did not request reads defined bytes, never an address outside the pool.
+#include <algorithm>
+#include <new>
+#include <unordered_map>
+#include <vector>
+
+#include "common.cuh"
+
+namespace {
+
+inline uint64_t tier_key(int layer, int expert) {
+  return (static_cast<uint64_t>(static_cast<uint32_t>(layer)) << 32) | static_cast<uint32_t>(expert);
+}
+inline size_t round256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
+
+struct MatBytes {
+  size_t plane, scale, zp;
+};
+inline MatBytes mat_bytes(int N, int K, int group) {
+  const size_t w = static_cast<size_t>(N) * static_cast<size_t>(K);
+  return MatBytes{w / 2, w / static_cast<size_t>(group) * 2, w / static_cast<size_t>(group)};
+}
+
+}  // namespace
+
+struct slicemoe_tier {
+  slicemoe_shape shape;
+  int n_layers;
+  MatBytes gu, dn;           // gate/up [inter, hidden] and down [hidden, inter]
+  size_t msb_rec, lsb_rec, slot_bytes;
+  const uint8_t* store;      // pinned host
+  uint8_t* pool;             // device
+  int n_slots;
+  slicemoe_expert* tables_dev;             // device [n_layers * n_experts]
+  std::vector<slicemoe_expert> tables;     // host mirror
+  std::vector<int> free_slots;
+  std::unordered_map<uint64_t, int> msb_slot, lsb_slot;
+  // Slices of the list being served that the cache no longer counts (a later entry of the same list pushed them
+  // out, or they never fitted): their bytes stay where they are until the next request, because the launch that
+  // follows this request reads them.  2 * top_k slots of the pool are set aside for them.
+  std::vector<std::pair<uint64_t, int>> transient;  // (key, 1 = LSB slice)
+  slicemoe_dbsc* cache;
+  cudaEvent_t ev_compute, ev_copy;
+  int64_t bytes_copied, copies;
+
+  void point_msb(slicemoe_expert& ex, const uint8_t* rec) const {
+    slicemoe_mat* m[3] = {&ex.gate, &ex.up, &ex.down};
+    for (int i = 0; i < 3; ++i) {
+      const MatBytes& b = i < 2 ? gu : dn;
+      m[i]->msb = rec;
+      m[i]->scale = reinterpret_cast<const uint16_t*>(rec + b.plane);
+      m[i]->zp = rec + b.plane + b.scale;
+      rec += b.plane + b.scale + b.zp;
+    }
+  }
+  void point_lsb(slicemoe_expert& ex, const uint8_t* rec, bool resident) const {
+    slicemoe_mat* m[3] = {&ex.gate, &ex.up, &ex.down};
+    for (int i = 0; i < 3; ++i) {
+      m[i]->lsb = resident ? rec : nullptr;  // a missing LSB plane is NULL: the kernels report it instead of reading it
+      rec += (i < 2 ? gu : dn).plane;
+    }
+  }
+};
+
+extern "C" int slicemoe_tier_sizes(const slicemoe_shape* s, size_t* msb_record, size_t* lsb_record, size_t* slot_bytes) {
+  if (!s || s->hidden <= 0 || s->inter <= 0 || (s->hidden % 128) || (s->inter % 128) || !slicemoe::valid_group(s->group))
+    return SLICEMOE_E_INVALID_ARG;
+  const MatBytes gu = mat_bytes(s->inter, s->hidden, s->group), dn = mat_bytes(s->hidden, s->inter, s->group);
+  const size_t m = 2 * (gu.plane + gu.scale + gu.zp) + dn.plane + dn.scale + dn.zp, l = 2 * gu.plane + dn.plane;
+  if (msb_record) *msb_record = m;
+  if (lsb_record) *lsb_record = l;
+  if (slot_bytes) *slot_bytes = round256(std::max(m, l));
+  return SLICEMOE_OK;
+}
+
+extern "C" int slicemoe_tier_store_expert(const slicemoe_shape* s, const slicemoe_expert* expert, void* record_host,
+                                          void* stream) {
+  if (!s || !expert || !record_host) return SLICEMOE_E_INVALID_ARG;
+  size_t m = 0, l = 0;
+  const int rc = slicemoe_tier_sizes(s, &m, &l, nullptr);
+  if (rc != SLICEMOE_OK) return rc;
+  const MatBytes gu = mat_bytes(s->inter, s->hidden, s->group), dn = mat_bytes(s->hidden, s->inter, s->group);
+  const slicemoe_mat* mats[3] = {&expert->gate, &expert->up, &expert->down};
+  uint8_t* p = static_cast<uint8_t*>(record_host);
+  cudaStream_t st = (cudaStream_t)stream;
+  for (int i = 0; i < 3; ++i) {
+    const MatBytes& b = i < 2 ? gu : dn;
+    if (!mats[i]->msb || !mats[i]->lsb || !mats[i]->scale || !mats[i]->zp) return SLICEMOE_E_INVALID_ARG;
+    SM_CUDA_TRY(cudaMemcpyAsync(p, mats[i]->msb, b.plane, cudaMemcpyDeviceToHost, st));
+    SM_CUDA_TRY(cudaMemcpyAsync(p + b.plane, mats[i]->scale, b.scale, cudaMemcpyDeviceToHost, st));
+    SM_CUDA_TRY(cudaMemcpyAsync(p + b.plane + b.scale, mats[i]->zp, b.zp, cudaMemcpyDeviceToHost, st));
+    p += b.plane + b.scale + b.zp;
+  }
+  for (int i = 0; i < 3; ++i) {
+    const MatBytes& b = i < 2 ? gu : dn;
+    SM_CUDA_TRY(cudaMemcpyAsync(p, mats[i]->lsb, b.plane, cudaMemcpyDeviceToHost, st));
+    p += b.plane;
+  }
+  return SLICEMOE_OK;
+}
+
+extern "C" slicemoe_tier* slicemoe_tier_create(const slicemoe_shape* s, int n_layers, const void* store_host,
+                                               void* pool_device, size_t pool_bytes, slicemoe_expert* tables_device,
+                                               double miss_budget, int warmup_steps, void* stream) {
+  if (!s || n_layers <= 0 || !store_host || !pool_device || !tables_device || s->n_experts <= 0) return nullptr;
+  if (reinterpret_cast<uintptr_t>(pool_device) & 255) return nullptr;
+  size_t m = 0, l = 0, slot = 0;
+  if (slicemoe_tier_sizes(s, &m, &l, &slot) != SLICEMOE_OK) return nullptr;
+  const long long n_slots = static_cast<long long>(pool_bytes / slot);
+  // slot 0 is the stand-in, 2 * top_k slots are set aside for slices in transit (see `transient`), the cache
+  // gets the rest and must be able to hold one request list
+  if (n_slots < 1 + 4LL * s->top_k || n_slots > (1 << 30)) return nullptr;
+  slicemoe_tier* t = new (std::nothrow) slicemoe_tier();
+  if (!t) return nullptr;
+  t->shape = *s;
+  t->n_layers = n_layers;
+  t->gu = mat_bytes(s->inter, s->hidden, s->group);
+  t->dn = mat_bytes(s->hidden, s->inter, s->group);
+  t->msb_rec = m;
+  t->lsb_rec = l;
+  t->slot_bytes = slot;
+  t->store = static_cast<const uint8_t*>(store_host);
+  t->pool = static_cast<uint8_t*>(pool_device);
+  t->n_slots = static_cast<int>(n_slots);
+  t->tables_dev = tables_device;
+  t->bytes_copied = t->copies = 0;
+  t->ev_compute = t->ev_copy = nullptr;
+  // the cache counts slots: both slice kinds are charged one slot's bytes, which is what they occupy here
+  t->cache = slicemoe_dbsc_create(static_cast<int64_t>(n_slots - 1 - 2 * s->top_k) * static_cast<int64_t>(slot), static_cast<int64_t>(slot),
+                                  static_cast<int64_t>(slot), miss_budget, warmup_steps);
+  bool ok = t->cache != nullptr && slicemoe_dbsc_log_evictions(t->cache, 1) == SLICEMOE_OK;
+  ok = ok && cudaEventCreateWithFlags(&t->ev_compute, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&t->ev_copy, cudaEventDisableTiming) == cudaSuccess;
+  if (ok) {
+    try {
+      for (int i = t->n_slots - 1; i >= 1; --i) t->free_slots.push_back(i);
+      slicemoe_expert blank;
+      slicemoe_mat* mm[3] = {&blank.gate, &blank.up, &blank.down};
+      for (int i = 0; i < 3; ++i) {
+        mm[i]->N = i < 2 ? s->inter : s->hidden;
+        mm[i]->K = i < 2 ? s->hidden : s->inter;
+      }
+      t->point_msb(blank, t->pool);
+      t->point_lsb(blank, t->pool, false);
+      t->tables.assign(static_cast<size_t>(n_layers) * s->n_experts, blank);
+    } catch (...) {
+      ok = false;
+    }
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  ok = ok && cudaMemsetAsync(t->pool, 0, slot, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(tables_device, t->tables.data(), t->tables.size() * sizeof(slicemoe_expert),
+                             cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(st) == cudaSuccess;  // the mirror is pageable: the copy has left it before we return
+  if (!ok) {
+    (void)cudaGetLastError();
+    if (t->ev_compute) cudaEventDestroy(t->ev_compute);
+    if (t->ev_copy) cudaEventDestroy(t->ev_copy);
+    if (t->cache) slicemoe_dbsc_destroy(t->cache);
+    delete t;
+    return nullptr;
+  }
+  return t;
+}
+
+extern "C" void slicemoe_tier_destroy(slicemoe_tier* t) {
+  if (!t) return;
+  cudaEventDestroy(t->ev_compute);
+  cudaEventDestroy(t->ev_copy);
+  slicemoe_dbsc_destroy(t->cache);
+  delete t;
+}
+
+extern "C" slicemoe_dbsc* slicemoe_tier_cache(slicemoe_tier* t) { return t ? t->cache : nullptr; }
+
+extern "C" int slicemoe_tier_request(slicemoe_tier* t, int step, int layer, const int32_t* ids, const uint8_t* prec_req,
+                                     int n, uint8_t* prec_out, void* compute_stream, void* copy_stream) {
+  if (!t || !ids || !prec_req || !prec_out || n < 0 || n > SLICEMOE_MAX_TOP_K || step < 0) return SLICEMOE_E_INVALID_ARG;
+  if (layer < 0 || layer >= t->n_layers) return SLICEMOE_E_INVALID_ARG;
+  for (int i = 0; i < n; ++i)
+    if (ids[i] < 0 || ids[i] >= t->shape.n_experts) return SLICEMOE_E_INVALID_ARG;
+  cudaStream_t cs = (cudaStream_t)compute_stream, xs = (cudaStream_t)copy_stream;
+  const size_t rec = t->msb_rec + t->lsb_rec;
+  try {
+    // Nothing that is still being read may be overwritten: the copies start when the work already enqueued on
+    // the compute stream has finished.  (A slice's bytes are needed by the very next launch, whose routing
+    // depended on the launch before: there is nothing of this token to overlap them with.)
+    SM_CUDA_TRY(cudaEventRecord(t->ev_compute, cs));
+    SM_CUDA_TRY(cudaStreamWaitEvent(xs, t->ev_compute, 0));
+    std::vector<size_t> dirty;  // table entries to send
+    auto drop = [&](uint64_t k, int is_lsb) {  // the slice's slot is free again, its table entry points at the stand-in
+      auto& map = is_lsb ? t->lsb_slot : t->msb_slot;
+      auto it = map.find(k);
+      if (it == map.end()) return;
+      t->free_slots.push_back(it->second);
+      map.erase(it);
+      const size_t idx = static_cast<size_t>(k >> 32) * t->shape.n_experts + static_cast<size_t>(k & 0xffffffffu);
+      if (is_lsb) t->point_lsb(t->tables[idx], t->pool, false);
+      else t->point_msb(t->tables[idx], t->pool);
+      dirty.push_back(idx);
+    };
+    // what the previous request kept beyond the cache's books has been read by now
+    for (auto& tr : t->transient) drop(tr.first, tr.second);
+    t->transient.clear();
+    auto in_list = [&](uint64_t k) {
+      for (int i = 0; i < n; ++i)
+        if (tier_key(layer, ids[i]) == k) return true;
+      return false;
+    };
+    auto release = [&]() -> int {
+      int32_t el[64], ee[64];
+      uint8_t il[64];
+      for (;;) {
+        const int m = slicemoe_dbsc_drain_evicted(t->cache, el, ee, il, 64);
+        if (m < 0) return m;
+        for (int i = 0; i < m; ++i) {
+          const uint64_t k = tier_key(el[i], ee[i]);
+          if (in_list(k)) t->transient.emplace_back(k, (int)il[i]);  // still needed by the coming launch
+          else drop(k, il[i]);
+        }
+        if (m < 64) return SLICEMOE_OK;
+      }
+    };
+    for (int i = 0; i < n; ++i) {
+      int mh = 0, lh = 0;
+      const int prec = slicemoe_dbsc_request(t->cache, step, layer, ids[i], prec_req[i] != 0, &mh, &lh, nullptr);
+      if (prec < 0) return prec;
+      prec_out[i] = static_cast<uint8_t>(prec);
+      int rc = release();
+      if (rc != SLICEMOE_OK) return rc;
+      const uint64_t k = tier_key(layer, ids[i]);
+      const size_t idx = static_cast<size_t>(layer) * t->shape.n_experts + ids[i];
+      const uint8_t* src = t->store + idx * rec;
+      int has_m = 0, has_l = 0;
+      slicemoe_dbsc_contains(t->cache, layer, ids[i], &has_m, &has_l);
+      for (int part = 0; part < 2; ++part) {  // 0: MSB record (always needed), 1: LSB record (when run at both slices)
+        if (part == 1 && !prec) continue;
+        auto& map = part ? t->lsb_slot : t->msb_slot;
+        const bool counted = (part ? has_l : has_m) != 0;
+        auto tr = std::find(t->transient.begin(), t->transient.end(), std::make_pair(k, part));
+        if (map.find(k) != map.end()) {  // the bytes are there
+          if (counted && tr != t->transient.end()) t->transient.erase(tr);  // (the same expert twice in the list)
+          continue;
+        }
+        if (t->free_slots.empty()) return SLICEMOE_E_UNSUPPORTED;  // cannot happen with the slots set aside
+        const int slot = t->free_slots.back();
+        t->free_slots.pop_back();
+        map[k] = slot;
+        if (!counted && tr == t->transient.end()) t->transient.emplace_back(k, part);  // used by this launch, not kept
+        uint8_t* dst = t->pool + static_cast<size_t>(slot) * t->slot_bytes;
+        const size_t bytes = part ? t->lsb_rec : t->msb_rec;
+        SM_CUDA_TRY(cudaMemcpyAsync(dst, src + (part ? t->msb_rec : 0), bytes, cudaMemcpyHostToDevice, xs));
+        t->bytes_copied += static_cast<int64_t>(bytes);
+        ++t->copies;
+        if (part) t->point_lsb(t->tables[idx], dst, true);
+        else t->point_msb(t->tables[idx], dst);
+        dirty.push_back(idx);
+      }
+    }
+    std::sort(dirty.begin(), dirty.end());
+    dirty.erase(std::unique(dirty.begin(), dirty.end()), dirty.end());
+    for (size_t idx : dirty)  // 144 bytes each, from pageable memory: staged by the runtime before the call returns
+      SM_CUDA_TRY(cudaMemcpyAsync(t->tables_dev + idx, &t->tables[idx], sizeof(slicemoe_expert), cudaMemcpyHostToDevice, xs));
+    SM_CUDA_TRY(cudaEventRecord(t->ev_copy, xs));
+    SM_CUDA_TRY(cudaStreamWaitEvent(cs, t->ev_copy, 0));
+  } catch (...) {
+    return SLICEMOE_E_NOMEM;
+  }
+  return SLICEMOE_OK;
+}
+
+extern "C" int slicemoe_tier_stats(const slicemoe_tier* t, int64_t* bytes_copied, int64_t* copies, int64_t* free_slots) {
+  if (!t) return SLICEMOE_E_INVALID_ARG;
+  if (bytes_copied) *bytes_copied = t->bytes_copied;
+  if (copies) *copies = t->copies;
+  if (free_slots) *free_slots = static_cast<int64_t>(t->free_slots.size());
+  return SLICEMOE_OK;
+}

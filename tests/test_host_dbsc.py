@@ -52,3 +52,40 @@ def test_assign_batch_equals_requests():
         ref = [b.request(step, 2, int(e), bool(r))[0] for e, r in zip(ids, req)]
         assert out.tolist() == ref
     a.close()
+
+
+def test_eviction_log_names_exactly_what_left_the_cache():
+    """slicemoe_dbsc_log_evictions / _drain_evicted: what a holder of the slices themselves has to release."""
+    import ctypes
+    from ctypes import c_void_p
+    from paper_2512_12990_b200 import binding as B
+    rng = np.random.default_rng(21)
+    msb_b, lsb_b, E, NL = 100, 60, 9, 2
+    c = B.Dbsc(4 * msb_b + 2 * lsb_b, msb_b, lsb_b)
+    assert B.lib().slicemoe_dbsc_log_evictions(c._h, 1) == 0
+    held = set()
+    lay, exp, isl = (np.zeros(8, np.int32), np.zeros(8, np.int32), np.zeros(8, np.uint8))
+    for step in range(200):
+        l, e, need = int(rng.integers(0, NL)), int(rng.integers(0, E)), bool(rng.random() < 0.5)
+        c.request(step, l, e, need)
+        while True:
+            n = B.lib().slicemoe_dbsc_drain_evicted(c._h, lay.ctypes.data_as(c_void_p), exp.ctypes.data_as(c_void_p),
+                                                    isl.ctypes.data_as(c_void_p), 8)
+            assert n >= 0
+            for i in range(n):
+                key = (int(lay[i]), int(exp[i]), int(isl[i]))
+                assert key in held, "only slices that were resident are evicted"
+                held.remove(key)
+            if n < 8:
+                break
+        has_m, has_l = c.contains(l, e)
+        if has_m:
+            held.add((l, e, 0))
+        if has_l:
+            held.add((l, e, 1))
+        # the holder's view equals the cache's
+        for ll in range(NL):
+            for ee in range(E):
+                m_, l_ = c.contains(ll, ee)
+                assert ((ll, ee, 0) in held) == m_ and ((ll, ee, 1) in held) == l_
+    assert B.lib().slicemoe_dbsc_drain_evicted(None, None, None, None, 0) == B.E_INVALID_ARG
