@@ -1080,6 +1080,41 @@ def run_stack(args, with_warmup_table: bool = True):
              "decode_tokens": ND, "decode_us_per_token_warm_cache": warm_us,
              "MB_fetched_warm_cache": warm_mb, "MB_fetched_empty_cache": cold_mb}
 
+    # ---- the second memory tier (Section 5): the first 4 layers' slices in pinned host memory, a device pool of 30 % of
+    # their bytes, misses copied in on a side stream; 64 decode tokens with cache and tier in the loop
+    NLT, NT = 4, 64
+    prec_rows = torch.empty((NT * NL, sh.top_k), dtype=torch.uint8).pin_memory()
+    tier = B.Tier(cs, [layers.keep[l][0] for l in range(NLT)], pool_slots=1 + 2 * sh.top_k + int(0.30 * NLT * sh.n_experts * 2))
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for s in range(NT):
+            for l in range(NLT):
+                r = s * NL + l
+                pr = tier.request(s, l, ids_h[r], preq_h[r], compute_stream=stream)
+                prec_rows[r] = torch.from_numpy(pr)          # a pinned row of its own: the copy runs later
+                prec_d[r:r + 1].copy_(prec_rows[r:r + 1], non_blocking=True)
+                rc = lib.slicemoe_layer(cs_ref, p(tier.layer_table(l)), p(layers.shared_tables[l]), None, p(x, r, 2 * sh.hidden),
+                                        1, p(ids, r, 4 * sh.top_k), p(prec_d, r, sh.top_k), p(wts, r, 4 * sh.top_k),
+                                        p(y, r, 4 * sh.hidden), p(ws), nws, sptr)
+                if rc:
+                    raise B.SliceMoEError(rc, "slicemoe_layer")
+        e1.record(stream)
+    torch.cuda.synchronize()
+    tier_ms = e0.elapsed_time(e1)
+    tst = tier.stats()
+    if B.slicemoe_get_status(ws, stream) != 0:
+        raise RuntimeError("device status word set with the tier in the loop")
+    tier_out = {"layers": NLT, "tokens": NT, "pool_slots": tier.pool.numel() // tier.slot_bytes,
+                "slot_MB": tier.slot_bytes / 1e6, "store_GB_pinned_host": tier.store.numel() / 1e9,
+                "us_per_layer_call": tier_ms * 1e3 / (NT * NLT), "MB_copied_per_layer_call": tst["bytes_copied"] / 1e6 / (NT * NLT),
+                "copies": tst["copies"], "msb_hit_rate": tst["msb_hit"] / max(tst["requests"], 1),
+                "what": "slicemoe_tier_request (cache decision, copies of missing records from pinned host memory on a side "
+                        "stream, table update) then slicemoe_layer, per layer; the copies wait for the compute stream and "
+                        "the launch waits for the copies"}
+    tier.close()
+    del tier
+    torch.cuda.empty_cache()
+
     peak, kind = measured_hbm_peak()
     gbs = total_bytes / (us_per_token * NS * 1e-6) / 1e9
     out = {
@@ -1102,6 +1137,7 @@ def run_stack(args, with_warmup_table: bool = True):
                         "exec_8bit": stats["high_exec"] / stats["requests"],
                         "mean_critical_per_token_layer": float(preq_h.sum(1).mean())},
         "prefill_to_decode": chain,
+        "tier": tier_out,
         "cost_model": cost_table(B, sh, NL, NS, logits, ids_h, preq_h, cap, msb_b, lsb_b, TAU, dev),
         "cache_warmup": (warmup_comparison(B, synth, sh, NL, ids_h, preq_h, cap, msb_b, lsb_b, TAU, dev)
                          if with_warmup_table else None),
