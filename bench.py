@@ -625,7 +625,7 @@ def run_cuda(args, sh, workload: str = WORKLOAD, rank_high: int = RANK_HIGH, met
     if B.slicemoe_get_status(ws, stream) != 0:
         raise RuntimeError("device status word set during the timed regions")
     # the host-buffer path must reproduce the device path bit for bit (fixed summation order)
-    n_cmp = min(K, P)      # steps both paths ran
+    n_cmp = min(K, chunk, P)      # steps both paths ran (the graphs replay steps 0 .. chunk - 1)
     if P % L == 0 and not torch.equal(yh[:n_cmp].to(dev), y[:n_cmp]):
         raise RuntimeError("host-buffer path and device path disagree")
 
