@@ -175,7 +175,8 @@ struct SmemLayout {
   static constexpr int bars = (plan + (int)sizeof(Plan) + 15) & ~15;  // uint64 barriers
   static constexpr int nbars = 2 * kUnits + kGroups * kFull2PerGroup + kUnits2 + 2 * kGroups + 6;
   static constexpr int dead = bars + nbars * 8;  // int dead flag; 8 bytes on, the wait limit in cycles
-  static constexpr int total = dead + 16;
+  static constexpr int hready = dead + 16;       // uint8 [kHCap / 128]: the 128-block of h is in shared memory as digits
+  static constexpr int total = hready + kHCap / 128;
 };
 static_assert(SmemLayout::total <= 227 * 1024, "shared memory budget");
 static_assert(sizeof(Slot) % 8 == 0, "slot alignment");
@@ -193,8 +194,7 @@ static_assert(SmemLayout::slots % 8 == 0 && SmemLayout::hdig % 16 == 0 && SmemLa
 //     empty[2 P + j % 2]; phase 2: P's units are [P h, P h + h), h = nunits2 / 2, taken in running order, one
 //     empty2 barrier per unit (an arrive from each warp of the group that consumed it).
 // pfull1 / pempty1 per group (phase-1 partial rows to the epilogue warp and back), pfull2 / pempty2 (phase-2
-// partial rows of all warps), hs_ready (h is in shared memory as
-// digits), p1_done (every consumer warp is through with phase 1, so the ring may be re-cut), plan_ready (the
+// partial rows of all warps), p1_done (every consumer warp is through with phase 1, so the ring may be re-cut), plan_ready (the
 // routed part of the plan and the routed slots stand: the producers wait for it after the shared experts' tasks).
 struct Bars {
   static constexpr int full = 0, empty = kUnits, full2 = 2 * kUnits, empty2 = full2 + kGroups * kFull2PerGroup,
@@ -362,11 +362,11 @@ struct TaskWalk {
 // ---- consumers -----------------------------------------------------------------------------------
 // Phase change: every consumer warp polls its 128-blocks of the grid's h in the workspace until all of a block's
 // values have been written (see kHEmpty), and turns the block into digits at once: blocks whose CTAs finished early
-// are done before the last CTA's values arrive.  Returns false if the (bounded) wait ran out.
+// are done before the last CTA's values arrive.  A block's flag in `hready` tells the other warps that its digits
+// stand; nobody waits for the whole of h (see wait_h_blocks).  Returns false if the (bounded) wait ran out.
 template <int G>
 __device__ bool fetch_h(const DecodeParams& p, uint8_t* smem, int warp, int lane, int htotal, const float* hbuf,
                         bool never_ready, volatile int* dead, unsigned* status, uint32_t bars) {
-  const uint32_t hs_ready = bars + 8 * Bars::hs_ready;
   const int nblk = htotal >> 7;
   constexpr int kMaxIt = (kHCap / 128 + kConsumerWarps - 1) / kConsumerWarps;
   unsigned pending = 0u;  // warp-uniform
@@ -389,6 +389,11 @@ __device__ bool fetch_h(const DecodeParams& p, uint8_t* smem, int warp, int lane
           block_to_digits<G>(q, (it * kConsumerWarps + warp) * 128, lane, smem + SmemLayout::hdig,
                              reinterpret_cast<float*>(smem + SmemLayout::hsumw), reinterpret_cast<float*>(smem + SmemLayout::hinv));
           pending &= ~(1u << it);
+          __syncwarp();  // every lane's digits of the block are written ...
+          if (lane == 0) {
+            __threadfence_block();  // ... and visible before the flag is
+            *reinterpret_cast<volatile uint8_t*>(smem + SmemLayout::hready + it * kConsumerWarps + warp) = 1;
+          }
         }
       }
     }
@@ -401,9 +406,26 @@ __device__ bool fetch_h(const DecodeParams& p, uint8_t* smem, int warp, int lane
       }
     }
   }
-  __syncwarp();
-  if (lane == 0) mbar_arrive(hs_ready);
-  return mbar_wait(hs_ready, 0, dead, status);
+  return true;
+}
+
+// Waits (bounded) until the `n` (<= 32) 128-blocks of h from block `b0` on are in shared memory as digits.
+__device__ __forceinline__ bool wait_h_blocks(const uint8_t* smem, int b0, int n, int lane, volatile int* dead,
+                                              unsigned* status) {
+  const volatile uint8_t* flag = reinterpret_cast<const volatile uint8_t*>(smem + SmemLayout::hready) + b0 + min(lane, n - 1);
+  if (!__all_sync(0xffffffffu, *flag != 0)) {
+    const long long t0 = clock64();
+    while (!__all_sync(0xffffffffu, *flag != 0)) {
+      if (*dead) return false;
+      if ((unsigned long long)(clock64() - t0) > wait_limit(dead)) {
+        *dead = 1;
+        atomicOr(status, (unsigned)SLICEMOE_STATUS_WAIT_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  __threadfence_block();
+  return true;
 }
 
 // Per-lane constants of the fold (see consume_chunk).
@@ -650,6 +672,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
       const int nblocks = d.z & 0xffu, col = (int)d.w;
       const bool p8 = (d.z & 256u) != 0u;
       if (!mbar_wait(full2 + 8 * (kFull2PerGroup * group + ((d.y >> 16) & 0xffu)), d.y >> 24, dead, status)) return;
+      if (!wait_h_blocks(smem, col >> 7, nblocks, lane, dead, status)) return;  // this chunk's part of h, no more
       const uint8_t* dig = smem + SmemLayout::hdig + col * 3;
       const float* sumw = reinterpret_cast<const float*>(smem + SmemLayout::hsumw) + (col >> LG) * 2;
       const float* binv = reinterpret_cast<const float*>(smem + SmemLayout::hinv) + (col >> 7);
@@ -1156,6 +1179,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
     if (lane == 0) {
       *reinterpret_cast<int*>(smem + SmemLayout::dead) = 0;
       *reinterpret_cast<unsigned long long*>(smem + SmemLayout::dead + 8) = kWaitCycles;
+      for (int i = 0; i < kHCap / 128; i += 8) *reinterpret_cast<unsigned long long*>(smem + SmemLayout::hready + i) = 0ull;
       const uint32_t bars = smem_u32(smem + SmemLayout::bars);
       for (int s = 0; s < kUnits; ++s) {
         mbar_init(bars + 8 * (Bars::full + s), 1);             // lane 0's expect_tx arrive
@@ -1169,7 +1193,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
       }
       mbar_init(bars + 8 * Bars::pfull2, kConsumerWarps);
       mbar_init(bars + 8 * Bars::pempty2, 1);
-      mbar_init(bars + 8 * Bars::hs_ready, kConsumerWarps);
       mbar_init(bars + 8 * Bars::p1_done, kConsumerWarps);
       mbar_init(bars + 8 * Bars::plan_ready, early_lists ? 2 : 1);  // resident lists: warps 0 and 1 each say when done
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
