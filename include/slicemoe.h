@@ -403,7 +403,13 @@ int slicemoe_dbsc_drain_evicted(slicemoe_dbsc *c, int32_t *layers, int32_t *expe
  * that a later entry of the same list pushed out of the cache's books again keeps its bytes until the next
  * request (2 * top_k slots of the pool are set aside for that; the cache is given the rest less slot 0).  ids,
  * prec_req, prec_out are host arrays.  Errors: INVALID_ARG, UNSUPPORTED (the pool cannot hold the list), NOMEM, CUDA.
- * Cache warm-up from a prompt (slicemoe_dbsc_prefill_*) is not connected to the tier.
+ *
+ * slicemoe_tier_sync: makes the pool hold exactly what the cache's books hold - for use after the books were
+ * changed behind the tier's back, which is how Predictive Cache Warmup (Section 4.3) reaches the tier: call
+ * slicemoe_dbsc_prefill_layer / _end on slicemoe_tier_cache(t) while the prompt is prefilled, then
+ * slicemoe_tier_sync once, and the decode steps that follow find the warmed slices in the pool.  Streams as in
+ * slicemoe_tier_request.  (What is not modelled is the traffic of the warm-up itself while the prompt is still
+ * running: the slices arrive in one go at the end.)
  */
 typedef struct slicemoe_tier slicemoe_tier;
 int slicemoe_tier_sizes(const slicemoe_shape *shape, size_t *msb_record, size_t *lsb_record, size_t *slot_bytes);
@@ -416,6 +422,7 @@ void slicemoe_tier_destroy(slicemoe_tier *t);
 slicemoe_dbsc *slicemoe_tier_cache(slicemoe_tier *t); /* the tier's own cache, for statistics; owned by the tier */
 int slicemoe_tier_request(slicemoe_tier *t, int step, int layer, const int32_t *ids, const uint8_t *prec_req,
                           int n, uint8_t *prec_out, void *compute_stream, void *copy_stream);
+int slicemoe_tier_sync(slicemoe_tier *t, void *compute_stream, void *copy_stream);
 int slicemoe_tier_stats(const slicemoe_tier *t, int64_t *bytes_copied, int64_t *copies, int64_t *free_slots);
 
 /*

@@ -34,7 +34,7 @@ EXPORTS = (
     "slicemoe_dbsc_prefill_layer", "slicemoe_dbsc_prefill_end", "slicemoe_dbsc_bias", "slicemoe_cumsum_select",
     "slicemoe_cost_paper_hw", "slicemoe_cost_step", "slicemoe_dbsc_log_evictions", "slicemoe_dbsc_drain_evicted",
     "slicemoe_tier_sizes", "slicemoe_tier_store_expert", "slicemoe_tier_create", "slicemoe_tier_destroy",
-    "slicemoe_tier_cache", "slicemoe_tier_request", "slicemoe_tier_stats",
+    "slicemoe_tier_cache", "slicemoe_tier_request", "slicemoe_tier_sync", "slicemoe_tier_stats",
 )
 
 
@@ -138,6 +138,7 @@ def lib() -> ctypes.CDLL:
     L.slicemoe_tier_cache.restype = c_void_p
     L.slicemoe_tier_cache.argtypes = [c_void_p]
     L.slicemoe_tier_request.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+    L.slicemoe_tier_sync.argtypes = [c_void_p, c_void_p, c_void_p]
     L.slicemoe_tier_stats.argtypes = [c_void_p, POINTER(c_int64), POINTER(c_int64), POINTER(c_int64)]
     L.slicemoe_cumsum_select.argtypes = [c_void_p, c_void_p, c_int, c_int, c_double, c_void_p]
     L.slicemoe_cost_paper_hw.argtypes = [POINTER(CostHw)]
@@ -506,6 +507,16 @@ def slicemoe_cost_step(flash_bytes: int, dram_bytes: int, macs: int, hw: CostHw 
     return e.value, t.value
 
 
+class _BorrowedDbsc(Dbsc):
+    """A Dbsc whose handle belongs to someone else: same methods, nothing is destroyed."""
+
+    def __init__(self, handle):
+        self._h = handle
+
+    def close(self):
+        self._h = None
+
+
 # ---- second memory tier --------------------------------------------------------------------------------
 def slicemoe_tier_sizes(shape: Shape):
     """(msb_record, lsb_record, slot_bytes) of a shape."""
@@ -573,6 +584,15 @@ class Tier:
                                          _stream(compute_stream), c_void_p(self.copy_stream.cuda_stream))
         _check(rc, "slicemoe_tier_request")
         return out
+
+    def cache(self):
+        """The tier's own host cache (owned by the tier; valid while the tier is)."""
+        return _BorrowedDbsc(lib().slicemoe_tier_cache(self._h))
+
+    def sync(self, compute_stream=None):
+        """Makes the pool hold what the cache's books hold (after a warm-up through self.cache())."""
+        _check(lib().slicemoe_tier_sync(self._h, _stream(compute_stream), c_void_p(self.copy_stream.cuda_stream)),
+               "slicemoe_tier_sync")
 
     def stats(self) -> dict:
         b, c, f = c_int64(0), c_int64(0), c_int64(0)

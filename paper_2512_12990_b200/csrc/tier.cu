@@ -282,6 +282,70 @@ extern "C" int slicemoe_tier_request(slicemoe_tier* t, int step, int layer, cons
   return SLICEMOE_OK;
 }
 
+extern "C" int slicemoe_tier_sync(slicemoe_tier* t, void* compute_stream, void* copy_stream) {
+  if (!t) return SLICEMOE_E_INVALID_ARG;
+  cudaStream_t cs = (cudaStream_t)compute_stream, xs = (cudaStream_t)copy_stream;
+  const size_t rec = t->msb_rec + t->lsb_rec;
+  try {
+    SM_CUDA_TRY(cudaEventRecord(t->ev_compute, cs));
+    SM_CUDA_TRY(cudaStreamWaitEvent(xs, t->ev_compute, 0));
+    // whatever the log holds is covered by the comparison below
+    {
+      int32_t el[64], ee[64];
+      uint8_t il[64];
+      while (slicemoe_dbsc_drain_evicted(t->cache, el, ee, il, 64) == 64) {
+      }
+    }
+    t->transient.clear();
+    std::vector<size_t> dirty;
+    const int E = t->shape.n_experts;
+    // first give back every slot whose slice the books no longer hold, then fetch what they hold and the pool lacks
+    for (int pass = 0; pass < 2; ++pass) {
+      for (int l = 0; l < t->n_layers; ++l) {
+        for (int e = 0; e < E; ++e) {
+          int has[2] = {0, 0};
+          slicemoe_dbsc_contains(t->cache, l, e, &has[0], &has[1]);
+          const uint64_t k = tier_key(l, e);
+          const size_t idx = static_cast<size_t>(l) * E + e;
+          for (int part = 0; part < 2; ++part) {
+            auto& map = part ? t->lsb_slot : t->msb_slot;
+            auto it = map.find(k);
+            if (pass == 0 && it != map.end() && !has[part]) {
+              t->free_slots.push_back(it->second);
+              map.erase(it);
+              if (part) t->point_lsb(t->tables[idx], t->pool, false);
+              else t->point_msb(t->tables[idx], t->pool);
+              dirty.push_back(idx);
+            } else if (pass == 1 && it == map.end() && has[part]) {
+              if (t->free_slots.empty()) return SLICEMOE_E_UNSUPPORTED;
+              const int slot = t->free_slots.back();
+              t->free_slots.pop_back();
+              map[k] = slot;
+              uint8_t* dst = t->pool + static_cast<size_t>(slot) * t->slot_bytes;
+              const size_t bytes = part ? t->lsb_rec : t->msb_rec;
+              SM_CUDA_TRY(cudaMemcpyAsync(dst, t->store + idx * rec + (part ? t->msb_rec : 0), bytes, cudaMemcpyHostToDevice, xs));
+              t->bytes_copied += static_cast<int64_t>(bytes);
+              ++t->copies;
+              if (part) t->point_lsb(t->tables[idx], dst, true);
+              else t->point_msb(t->tables[idx], dst);
+              dirty.push_back(idx);
+            }
+          }
+        }
+      }
+    }
+    std::sort(dirty.begin(), dirty.end());
+    dirty.erase(std::unique(dirty.begin(), dirty.end()), dirty.end());
+    for (size_t idx : dirty)
+      SM_CUDA_TRY(cudaMemcpyAsync(t->tables_dev + idx, &t->tables[idx], sizeof(slicemoe_expert), cudaMemcpyHostToDevice, xs));
+    SM_CUDA_TRY(cudaEventRecord(t->ev_copy, xs));
+    SM_CUDA_TRY(cudaStreamWaitEvent(cs, t->ev_copy, 0));
+  } catch (...) {
+    return SLICEMOE_E_NOMEM;
+  }
+  return SLICEMOE_OK;
+}
+
 extern "C" int slicemoe_tier_stats(const slicemoe_tier* t, int64_t* bytes_copied, int64_t* copies, int64_t* free_slots) {
   if (!t) return SLICEMOE_E_INVALID_ARG;
   if (bytes_copied) *bytes_copied = t->bytes_copied;

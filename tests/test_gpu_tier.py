@@ -84,3 +84,57 @@ def test_tier_argument_checks():
     assert L.slicemoe_tier_request(None, 0, 0, None, None, 0, None, None, None) == B.E_INVALID_ARG
     assert L.slicemoe_tier_stats(None, None, None, None) == B.E_INVALID_ARG
     L.slicemoe_tier_destroy(None)
+
+
+def test_cache_warmup_reaches_the_tier():
+    """Predictive Cache Warmup (Section 4.3) through the tier: the prompt's routing reshapes the tier's own cache,
+    slicemoe_tier_sync brings the pool in line with it, and the decode steps that follow hit what was warmed.
+    Every decode precision list and layer output is compared with the oracle chain (pcw.warm_state installed in
+    the oracle cache)."""
+    import torch
+    from oracle import pcw
+    from paper_2512_12990_b200 import binding as B
+    NL, T_PROMPT, N_DEC, tau = 3, 64, 6, 0.3
+    sh = synth.Shape("tier-pcw", 256, 128, 8, 2, 64, n_shared=0, shared_inter=0, shared_sigmoid_gate=False, n_layers=NL,
+                     seed=5151)
+    E, k = sh.n_experts, sh.top_k
+    layers = [H.Layer(sh, range(E), layer=l) for l in range(NL)]
+    _, _, slot = B.slicemoe_tier_sizes(layers[0].cshape)
+    pool_slots = 1 + 2 * k + 12                      # 12 cached slots for 48 slices
+    tier = B.Tier(layers[0].cshape, [[L.packed[e] for e in range(E)] for L in layers], pool_slots)
+    cap = 12 * slot
+    orc = SliceCache(cap, slot, slot)
+    cache = tier.cache()
+    freq, mean = [], []
+    for l in range(NL):
+        logits = synth.zipf_gumbel_logits(sh.seed, ("tier-prompt", l), T_PROMPT, E, 1.1)[0]
+        ids_o, w_o, _ = moe.route_topk(logits, k)
+        cache.prefill_layer(l, ids_o, w_o.astype(np.float32), E, tau)
+        f, m = pcw.prefill_stats(ids_o, w_o.astype(np.float32), E)
+        freq.append(f); mean.append(m)
+    cache.prefill_end()
+    orc.install(*pcw.warm_state(freq, mean, cap, slot, slot, tau))
+    tier.sync()
+    st0 = tier.stats()
+    assert st0["copies"] == len(orc.msb) + len(orc.lsb) == 12 and st0["requests"] == 0
+    dec = synth.decode_trace_logits(sh.seed, N_DEC, NL, E, s=1.1, p_repeat=0.3)
+    for s in range(N_DEC):
+        for l, L in enumerate(layers):
+            lg = np.ascontiguousarray(dec[s, l][None, :])
+            ids_o, w_o, _ = moe.route_topk(lg, k)
+            req = moe.precision_request(w_o, tau)
+            prec = tier.request(s, l, ids_o[0], req[0])
+            prec_o = [orc.request(s, l, int(ids_o[0, j]), bool(req[0, j]))[0] for j in range(k)]
+            assert prec.tolist() == prec_o
+            xbits, x64 = H.x_inputs(sh, 1, f"tier-pcw-x{s}-{l}")
+            y = B.slicemoe_layer(L.cshape, tier.layer_table(l), None, None, H.to_dev_bf16(xbits),
+                                 torch.from_numpy(ids_o.astype(np.int32)).cuda(), torch.from_numpy(prec[None, :].copy()).cuda(),
+                                 torch.from_numpy(w_o.astype(np.float32)).cuda(), L.ws)
+            torch.cuda.synchronize()
+            assert B.slicemoe_get_status(L.ws) == 0
+            H.assert_close(y.cpu().numpy(), moe.expert_ffn(x64, L.oracle_list(), ids_o, prec[None, :], w_o), f"step {s} layer {l}")
+    st = tier.stats()
+    for key in ("requests", "msb_hit", "msb_miss", "lsb_hit", "lsb_miss"):
+        assert st[key] == orc.stats[key], key
+    assert st["msb_hit"] > 0, "the warmed slices are hit"
+    tier.close()
