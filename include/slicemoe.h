@@ -67,7 +67,7 @@ typedef struct slicemoe_shape {
   int32_t top_k;               /* experts per token k <= SLICEMOE_MAX_TOP_K */
   int32_t group;               /* quantisation group along K: 32, 64 or 128 */
   int32_t b_high, b_low;       /* slice configuration: (8, 4), (6, 3) or (4, 2) */
-  int32_t n_shared;            /* always-on shared experts (<= SLICEMOE_MAX_SHARED), run at 8 bits */
+  int32_t n_shared;            /* always-on shared experts (<= SLICEMOE_MAX_SHARED), run from both slices */
   int32_t shared_inter;        /* their intermediate width; multiple of 128 */
   int32_t shared_sigmoid_gate; /* 1: shared output is scaled by sigmoid(v . x) */
 } slicemoe_shape;
@@ -187,7 +187,7 @@ int slicemoe_expert_ffn(const slicemoe_shape *shape, const slicemoe_expert *expe
 
 /*
  * slicemoe_layer - routed experts as above plus the always-on shared experts of the two evaluated
- * model architectures (not part of the paper's method): each shared expert runs at 8 bits and is
+ * model architectures (not part of the paper's method): each shared expert runs from both slices and is
  * added with weight 1, or with weight sigmoid(shared_gate_vec . x[t]) when shape->shared_sigmoid_gate.
  *   shared           device array [shape->n_shared] of slicemoe_expert (inter = shape->shared_inter)
  *   shared_gate_vec  device float32 [hidden] or NULL (required iff shared_sigmoid_gate)
