@@ -117,3 +117,30 @@ def nibble_pack_canonical(plane: np.ndarray) -> np.ndarray:
     flat = plane.reshape(-1).astype(np.uint8)
     assert flat.size % 2 == 0
     return (flat[0::2] | (flat[1::2] << 4)).astype(np.uint8)
+
+
+def compact_stream(values: np.ndarray, bits: int) -> np.ndarray:
+    """The dense storage of a slice narrower than a nibble (Table 1: MAT63 has 3-bit slices, MAT42 2-bit ones):
+    a little-endian bit stream, value i in bits [i * bits, (i + 1) * bits).  values: 1-D, each < 2^bits, count a
+    multiple of 8 (so the stream ends on a byte).  Returns uint8 [count * bits / 8]."""
+    v = np.asarray(values, dtype=np.uint8).reshape(-1)
+    assert bits in (2, 3, 4) and v.size % 8 == 0 and (v.size == 0 or int(v.max()) < (1 << bits))
+    out = np.zeros(v.size * bits // 8, dtype=np.uint8)
+    for i in range(v.size):                      # plain and slow on purpose
+        pos = i * bits
+        val = int(v[i]) << (pos & 7)
+        out[pos >> 3] |= val & 0xFF
+        if val >> 8:
+            out[(pos >> 3) + 1] |= val >> 8
+    return out
+
+
+def compact_unstream(stream: np.ndarray, bits: int, count: int) -> np.ndarray:
+    """Inverse of compact_stream: the first `count` values."""
+    s = np.asarray(stream, dtype=np.uint8).reshape(-1)
+    out = np.zeros(count, dtype=np.uint8)
+    for i in range(count):
+        pos = i * bits
+        word = int(s[pos >> 3]) | (int(s[(pos >> 3) + 1]) << 8 if (pos >> 3) + 1 < s.size else 0)
+        out[i] = (word >> (pos & 7)) & ((1 << bits) - 1)
+    return out

@@ -204,3 +204,28 @@ def test_truncation_error_statistics_closed_form():
 def test_canonical_nibble_packing():
     plane = np.array([[1, 2, 3, 4], [15, 0, 9, 7]], dtype=np.uint8)
     assert amat.nibble_pack_canonical(plane).tolist() == [0x21, 0x43, 0x0F, 0x79]
+
+
+def test_compact_stream_is_the_little_endian_bit_stream():
+    """Pins of the dense 2- / 3- / 4-bit slice storage: hand-worked bytes, the big-integer definition of a
+    little-endian bit stream, and the round trip."""
+    # 2 bits: values 1, 2, 3, 0 -> 0b00_11_10_01 = 0x39; then 3, 3, 3, 3 -> 0xff
+    assert amat.compact_stream(np.array([1, 2, 3, 0, 3, 3, 3, 3]), 2).tolist() == [0x39, 0xFF]
+    # 3 bits: 1, 2, 3, 4, 5, 6, 7, 0 -> bits 001 010 011 100 101 110 111 000 from the low end:
+    # 1 + 2*8 + 3*64 + 4*512 + 5*4096 + 6*32768 + 7*262144 = 2,054,353 = 0x1F58D1 -> bytes d1 58 1f
+    v = [1, 2, 3, 4, 5, 6, 7, 0]
+    total = sum(x << (3 * i) for i, x in enumerate(v))
+    assert total == 0x1F58D1
+    assert amat.compact_stream(np.array(v), 3).tolist() == [0xD1, 0x58, 0x1F]
+    # 4 bits is the nibble packing itself
+    assert amat.compact_stream(np.array([1, 2, 3, 4, 15, 0, 9, 7]), 4).tolist() == [0x21, 0x43, 0x0F, 0x79]
+    rng = np.random.default_rng(3)
+    for bits in (2, 3, 4):
+        vals = rng.integers(0, 1 << bits, 8 * 37).astype(np.uint8)
+        s = amat.compact_stream(vals, bits)
+        assert s.size == vals.size * bits // 8
+        big = sum(int(x) << (bits * i) for i, x in enumerate(vals))
+        assert bytes(s) == big.to_bytes(s.size, "little")
+        assert np.array_equal(amat.compact_unstream(s, bits, vals.size), vals)
+    with pytest.raises(AssertionError):
+        amat.compact_stream(np.array([4, 0, 0, 0, 0, 0, 0, 0]), 2)      # does not fit 2 bits
