@@ -1108,6 +1108,11 @@ def run_stack(args, with_warmup_table: bool = True):
                 "slot_MB": tier.slot_bytes / 1e6, "store_GB_pinned_host": tier.store.numel() / 1e9,
                 "us_per_layer_call": tier_ms * 1e3 / (NT * NLT), "MB_copied_per_layer_call": tst["bytes_copied"] / 1e6 / (NT * NLT),
                 "copies": tst["copies"], "msb_hit_rate": tst["msb_hit"] / max(tst["requests"], 1),
+                # what a miss moves per expert in the three slice formats of Table 1 (MSB record incl. scales and
+                # zero-points / LSB record), as stored: narrow slices are kept dense in the store
+                "stored_MB_per_expert": {f"MAT{bh}{bl}": [round(v / 1e6, 3) for v in B.slicemoe_tier_sizes(
+                    B.make_shape(sh.hidden, sh.inter, sh.n_experts, sh.top_k, sh.group, sh.n_shared, sh.shared_inter,
+                                 False, bh, bl))[:2]] for bh, bl in ((8, 4), (6, 3), (4, 2))},
                 "what": "slicemoe_tier_request (cache decision, copies of missing records from pinned host memory on a side "
                         "stream, table update) then slicemoe_layer, per layer; the copies wait for the compute stream and "
                         "the launch waits for the copies"}

@@ -23,8 +23,9 @@
  *   paper's joint truncation of code and zero-point.  (b_high, b_low) is one of Table 1's three: (8, 4) -
  *   MAT84, the default everywhere - (6, 3) and (4, 2).  A plane always gives a slice value a nibble: a 3-bit
  *   or 2-bit slice sits in the low bits of its nibble, so one layout, and one set of kernels, serves the three
- *   formats; on the device MAT63 and MAT42 therefore take the bytes of MAT84 (the 3- and 2-bit planes a slower
- *   memory tier would hold are a repacking that this library does not do).
+ *   formats; on the device MAT63 and MAT42 therefore take the bytes of MAT84.  For the slower memory tier a
+ *   plane can be stored dense, 3 or 2 bits per value (slicemoe_compact_plane / slicemoe_expand_plane; the tier
+ *   of slicemoe_tier_* does so).
  *
  *   Physical layout of a plane (N % 16 == 0, K % 128 == 0), N*K/2 bytes: rows are grouped in blocks
  *   of 16 and K in tiles of 64; block (rb, st) is 512 contiguous bytes at ((rb*(K/64) + st)*512),
@@ -113,6 +114,18 @@ int slicemoe_pack(const float *W, int N, int K, int group, int b_high, int b_low
 
 /* Inverse of the physical layout (test hook and dump helper): nibbles[n*K + k] in 0..15. */
 int slicemoe_unpack_plane(const void *plane, int N, int K, uint8_t *nibbles, void *stream);
+/*
+ * Dense storage of a slice plane for the slower memory tiers (Table 1: MAT63 has 3-bit slices, MAT42 2-bit ones).
+ * On the device a plane gives every slice value a nibble, whatever its width; slicemoe_compact_plane writes the
+ * plane's nibbles - in the order of its bytes, low nibble first - as a little-endian bit stream of `bits` bits
+ * each (value i in bits [i * bits, (i + 1) * bits)), slicemoe_compact_bytes(N, K, bits) = N*K*bits/8 bytes, and
+ * slicemoe_expand_plane is the inverse.  bits in {2, 3, 4} (4 is a plain copy); values must fit `bits` bits
+ * (higher bits of a nibble are dropped).  plane, compact: device.  Errors: INVALID_ARG, UNSUPPORTED (bits), CUDA.
+ */
+size_t slicemoe_compact_bytes(int N, int K, int bits);
+int slicemoe_compact_plane(const void *plane, int N, int K, int bits, void *compact, void *stream);
+int slicemoe_expand_plane(const void *compact, int N, int K, int bits, void *plane, void *stream);
+
 /* scale_rm / zp_rm: row-major [N, K/group]. */
 int slicemoe_unpack_meta(const uint16_t *scale, const uint8_t *zp, int N, int K, int group,
                          uint16_t *scale_rm, uint8_t *zp_rm, void *stream);
@@ -382,17 +395,23 @@ int slicemoe_dbsc_drain_evicted(slicemoe_dbsc *c, int32_t *layers, int32_t *expe
  * equal slots in device memory, a miss a copy of the slice's record on a side stream; the decisions are those
  * of slicemoe_dbsc_* (MSB slices LRU, LSB slices first to go), with both slice kinds charged one slot.
  *
- * Records (slicemoe_tier_sizes gives their sizes for a shape, and the slot size = the larger one rounded up to
- * 256 bytes).  MSB record: gate MSB plane, gate scales, gate zero-points, then up's, then down's.  LSB record:
- * gate, up, down LSB planes.  The store holds for (layer l, expert e) the MSB record followed by the LSB record
+ * Records.  MSB record: gate MSB plane, gate scales, gate zero-points, then up's, then down's.  LSB record:
+ * gate, up, down LSB planes.  In the store a plane of a slice narrower than four bits (MAT63: 3 + 3, MAT42:
+ * 2 + 2) is kept dense, as slicemoe_compact_plane writes it, so a miss moves 3 or 2 bits per weight instead of 4;
+ * the copy lands in a staging buffer and a small kernel on the side stream spreads it into the slot's nibble
+ * planes.  slicemoe_tier_sizes gives, for a shape: the stored sizes of the two records, the slot size (the larger
+ * record in its device form, rounded up to 256 bytes) and the staging size (0 for MAT84, whose records are
+ * stored as they are used).  The store holds for (layer l, expert e) the MSB record followed by the LSB record
  * at offset (l * n_experts + e) * (msb_record + lsb_record); slicemoe_tier_store_expert writes one such pair from a
- * packed expert on the device (device-to-host copies enqueued on `stream`; offline preparation).
+ * packed expert on the device (device-to-host copies enqueued on `stream`; scratch_device: device memory of the
+ * staging size, NULL for MAT84; offline preparation).
  *
  * slicemoe_tier_create: store_host (pinned, read only, must outlive the tier); pool_device (256-byte aligned,
  * pool_bytes >= (1 + 4 * top_k) slots: slot 0 is a stand-in that the table entries of non-resident slices point
  * to, so that a list naming an expert that was never requested reads defined bytes); tables_device: device array
  * [n_layers * n_experts] of slicemoe_expert that the tier fills and keeps up to date - pass
- * tables_device + l * n_experts as `experts` to the layer calls.  Synchronises `stream`.  NULL on bad arguments
+ * tables_device + l * n_experts as `experts` to the layer calls; staging_device: device memory of at least the
+ * staging size (16-byte aligned; NULL for MAT84).  Synchronises `stream`.  NULL on bad arguments
  * or allocation failure.  The tier allocates no device memory.
  *
  * slicemoe_tier_request: serves the n selected experts of one (step, layer): decides hits, misses, evictions
@@ -412,12 +431,14 @@ int slicemoe_dbsc_drain_evicted(slicemoe_dbsc *c, int32_t *layers, int32_t *expe
  * running: the slices arrive in one go at the end.)
  */
 typedef struct slicemoe_tier slicemoe_tier;
-int slicemoe_tier_sizes(const slicemoe_shape *shape, size_t *msb_record, size_t *lsb_record, size_t *slot_bytes);
+int slicemoe_tier_sizes(const slicemoe_shape *shape, size_t *msb_record, size_t *lsb_record, size_t *slot_bytes,
+                        size_t *staging_bytes);
 int slicemoe_tier_store_expert(const slicemoe_shape *shape, const slicemoe_expert *expert, void *record_host,
-                               void *stream);
+                               void *scratch_device, void *stream);
 slicemoe_tier *slicemoe_tier_create(const slicemoe_shape *shape, int n_layers, const void *store_host,
                                     void *pool_device, size_t pool_bytes, slicemoe_expert *tables_device,
-                                    double miss_budget, int warmup_steps, void *stream);
+                                    void *staging_device, size_t staging_bytes, double miss_budget,
+                                    int warmup_steps, void *stream);
 void slicemoe_tier_destroy(slicemoe_tier *t);
 slicemoe_dbsc *slicemoe_tier_cache(slicemoe_tier *t); /* the tier's own cache, for statistics; owned by the tier */
 int slicemoe_tier_request(slicemoe_tier *t, int step, int layer, const int32_t *ids, const uint8_t *prec_req,

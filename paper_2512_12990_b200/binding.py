@@ -26,7 +26,7 @@ DBSC_STAT_NAMES = ("requests", "msb_hit", "msb_miss", "lsb_hit", "lsb_miss", "ls
 # every symbol include/slicemoe.h declares
 EXPORTS = (
     "slicemoe_strerror", "slicemoe_version", "slicemoe_last_cuda_error", "slicemoe_plane_bytes", "slicemoe_meta_count", "slicemoe_pack",
-    "slicemoe_unpack_plane", "slicemoe_unpack_meta", "slicemoe_route_topk", "slicemoe_workspace_bytes",
+    "slicemoe_unpack_plane", "slicemoe_unpack_meta", "slicemoe_compact_bytes", "slicemoe_compact_plane", "slicemoe_expand_plane", "slicemoe_route_topk", "slicemoe_workspace_bytes",
     "slicemoe_workspace_init", "slicemoe_workspace_set_wait", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer", "slicemoe_layer_flags",
     "slicemoe_decode_step_host", "slicemoe_stream_probe", "slicemoe_layer_static", "slicemoe_layer_routed", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
     "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
@@ -86,6 +86,10 @@ def lib() -> ctypes.CDLL:
     L.slicemoe_meta_count.argtypes = [c_int, c_int, c_int]
     L.slicemoe_pack.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p,
                                 c_void_p, c_void_p]
+    L.slicemoe_compact_bytes.restype = c_size_t
+    L.slicemoe_compact_bytes.argtypes = [c_int, c_int, c_int]
+    L.slicemoe_compact_plane.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_void_p]
+    L.slicemoe_expand_plane.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_void_p]
     L.slicemoe_unpack_plane.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p]
     L.slicemoe_unpack_meta.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p]
     L.slicemoe_route_topk.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_int, c_float, c_int, c_void_p,
@@ -129,10 +133,11 @@ def lib() -> ctypes.CDLL:
     L.slicemoe_dbsc_bias.argtypes = [c_void_p, c_int, c_int, c_float, c_void_p]
     L.slicemoe_dbsc_log_evictions.argtypes = [c_void_p, c_int]
     L.slicemoe_dbsc_drain_evicted.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int]
-    L.slicemoe_tier_sizes.argtypes = [POINTER(Shape), POINTER(c_size_t), POINTER(c_size_t), POINTER(c_size_t)]
-    L.slicemoe_tier_store_expert.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p]
+    L.slicemoe_tier_sizes.argtypes = [POINTER(Shape), POINTER(c_size_t), POINTER(c_size_t), POINTER(c_size_t), POINTER(c_size_t)]
+    L.slicemoe_tier_store_expert.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p]
     L.slicemoe_tier_create.restype = c_void_p
-    L.slicemoe_tier_create.argtypes = [POINTER(Shape), c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_double, c_int, c_void_p]
+    L.slicemoe_tier_create.argtypes = [POINTER(Shape), c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p, c_size_t, c_double,
+                                       c_int, c_void_p]
     L.slicemoe_tier_destroy.argtypes = [c_void_p]
     L.slicemoe_tier_destroy.restype = None
     L.slicemoe_tier_cache.restype = c_void_p
@@ -507,6 +512,22 @@ def slicemoe_cost_step(flash_bytes: int, dram_bytes: int, macs: int, hw: CostHw 
     return e.value, t.value
 
 
+def slicemoe_compact_plane(plane, N: int, K: int, bits: int, stream=None):
+    """plane: CUDA uint8 [N*K/2] (physical layout) -> CUDA uint8 [N*K*bits/8], the dense bit stream."""
+    import torch
+    out = torch.empty(lib().slicemoe_compact_bytes(N, K, bits), dtype=torch.uint8, device=plane.device)
+    _check(lib().slicemoe_compact_plane(_ptr(plane), N, K, bits, _ptr(out), _stream(stream)), "slicemoe_compact_plane")
+    return out
+
+
+def slicemoe_expand_plane(compact, N: int, K: int, bits: int, stream=None):
+    """The inverse: CUDA uint8 [N*K*bits/8] -> CUDA uint8 [N*K/2] in the physical plane layout."""
+    import torch
+    out = torch.empty(N * K // 2, dtype=torch.uint8, device=compact.device)
+    _check(lib().slicemoe_expand_plane(_ptr(compact), N, K, bits, _ptr(out), _stream(stream)), "slicemoe_expand_plane")
+    return out
+
+
 class _BorrowedDbsc(Dbsc):
     """A Dbsc whose handle belongs to someone else: same methods, nothing is destroyed."""
 
@@ -519,11 +540,12 @@ class _BorrowedDbsc(Dbsc):
 
 # ---- second memory tier --------------------------------------------------------------------------------
 def slicemoe_tier_sizes(shape: Shape):
-    """(msb_record, lsb_record, slot_bytes) of a shape."""
-    m, l, sl = c_size_t(0), c_size_t(0), c_size_t(0)
-    _check(lib().slicemoe_tier_sizes(ctypes.byref(shape), ctypes.byref(m), ctypes.byref(l), ctypes.byref(sl)),
-           "slicemoe_tier_sizes")
-    return m.value, l.value, sl.value
+    """(msb_record, lsb_record, slot_bytes, staging_bytes) of a shape: the records as stored, the slot and the
+    staging buffer on the device."""
+    m, l, sl, sg = c_size_t(0), c_size_t(0), c_size_t(0), c_size_t(0)
+    _check(lib().slicemoe_tier_sizes(ctypes.byref(shape), ctypes.byref(m), ctypes.byref(l), ctypes.byref(sl),
+                                     ctypes.byref(sg)), "slicemoe_tier_sizes")
+    return m.value, l.value, sl.value, sg.value
 
 
 class Tier:
@@ -537,21 +559,24 @@ class Tier:
                  device="cuda"):
         import torch
         self.shape, self.n_layers, self.n_experts = shape, len(layers), len(layers[0])
-        m, l, slot = slicemoe_tier_sizes(shape)
+        m, l, slot, stg = slicemoe_tier_sizes(shape)
         self.msb_record, self.lsb_record, self.slot_bytes = m, l, slot
+        self.staging = torch.empty(stg, dtype=torch.uint8, device=device) if stg else None
         self.store = torch.empty((self.n_layers * self.n_experts, m + l), dtype=torch.uint8).pin_memory()
         for li, experts in enumerate(layers):
             for e, ex in enumerate(experts):
                 rec = Expert(ex["gate"].desc(), ex["up"].desc(), ex["down"].desc())
                 rc = lib().slicemoe_tier_store_expert(ctypes.byref(shape), ctypes.byref(rec),
-                                                      c_void_p(self.store[li * self.n_experts + e].data_ptr()), _stream(None))
+                                                      c_void_p(self.store[li * self.n_experts + e].data_ptr()),
+                                                      _ptr(self.staging), _stream(None))
                 _check(rc, "slicemoe_tier_store_expert")
         torch.cuda.synchronize()
         self.pool = torch.empty(pool_slots * slot, dtype=torch.uint8, device=device)
         self.tables = torch.empty(self.n_layers * self.n_experts * ctypes.sizeof(Expert), dtype=torch.uint8, device=device)
         self.copy_stream = torch.cuda.Stream(device=device)
         self._h = lib().slicemoe_tier_create(ctypes.byref(shape), self.n_layers, c_void_p(self.store.data_ptr()),
-                                             _ptr(self.pool), self.pool.numel(), _ptr(self.tables),
+                                             _ptr(self.pool), self.pool.numel(), _ptr(self.tables), _ptr(self.staging),
+                                             0 if self.staging is None else self.staging.numel(),
                                              -1.0 if miss_budget is None else float(miss_budget), warmup_steps,
                                              _stream(None))
         if not self._h:

@@ -114,6 +114,33 @@ __global__ void unpack_meta_kernel(const uint16_t* __restrict__ scale, const uin
   zp_rm[idx] = zp[mi];
 }
 
+// Dense storage of a slice narrower than a nibble: the plane's nibbles, in the order of its bytes (low nibble
+// first), as a little-endian bit stream of `bits` bits each.  One thread per 32-bit plane word = 8 nibbles =
+// `bits` bytes of the stream.
+__global__ void compact_plane_kernel(const uint32_t* __restrict__ plane, size_t n_words, int bits,
+                                     uint8_t* __restrict__ out) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_words) return;
+  const uint32_t w = plane[i], mask = (1u << bits) - 1u;
+  uint32_t packed = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) packed |= ((w >> (4 * j)) & mask) << (bits * j);
+  for (int b = 0; b < bits; ++b) out[i * bits + b] = (uint8_t)(packed >> (8 * b));
+}
+
+__global__ void expand_plane_kernel(const uint8_t* __restrict__ in, size_t n_words, int bits,
+                                    uint32_t* __restrict__ plane) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_words) return;
+  uint32_t packed = 0;
+  for (int b = 0; b < bits; ++b) packed |= (uint32_t)in[i * bits + b] << (8 * b);
+  const uint32_t mask = (1u << bits) - 1u;
+  uint32_t w = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) w |= ((packed >> (bits * j)) & mask) << (4 * j);
+  plane[i] = w;
+}
+
 static int check_dims(int N, int K, int group) {
   if (N <= 0 || K <= 0 || (N % 16) != 0 || (K % 128) != 0) return SLICEMOE_E_INVALID_ARG;
   if (!valid_group(group)) return SLICEMOE_E_UNSUPPORTED;
@@ -177,6 +204,40 @@ extern "C" int slicemoe_unpack_meta(const uint16_t* scale, const uint8_t* zp, in
   const int threads = 256;
   unpack_meta_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, (cudaStream_t)stream>>>(
       scale, zp, N, ngroups, scale_rm, zp_rm);
+  SM_LAUNCH_CHECK();
+  return SLICEMOE_OK;
+}
+
+extern "C" size_t slicemoe_compact_bytes(int N, int K, int bits) {
+  if (N <= 0 || K <= 0 || bits < 2 || bits > 4) return 0;
+  return (size_t)N * K / 8 * bits;
+}
+
+static int compact_args(const void* a, const void* b, int N, int K, int bits) {
+  if (!a || !b) return SLICEMOE_E_INVALID_ARG;
+  if (N <= 0 || K <= 0 || (N % 16) != 0 || (K % 128) != 0) return SLICEMOE_E_INVALID_ARG;
+  if (bits < 2 || bits > 4) return SLICEMOE_E_UNSUPPORTED;
+  return SLICEMOE_OK;
+}
+
+extern "C" int slicemoe_compact_plane(const void* plane, int N, int K, int bits, void* compact, void* stream) {
+  const int rc = compact_args(plane, compact, N, K, bits);
+  if (rc != SLICEMOE_OK) return rc;
+  const size_t n_words = (size_t)N * K / 8;
+  const int threads = 256;
+  compact_plane_kernel<<<(unsigned)((n_words + threads - 1) / threads), threads, 0, (cudaStream_t)stream>>>(
+      reinterpret_cast<const uint32_t*>(plane), n_words, bits, reinterpret_cast<uint8_t*>(compact));
+  SM_LAUNCH_CHECK();
+  return SLICEMOE_OK;
+}
+
+extern "C" int slicemoe_expand_plane(const void* compact, int N, int K, int bits, void* plane, void* stream) {
+  const int rc = compact_args(compact, plane, N, K, bits);
+  if (rc != SLICEMOE_OK) return rc;
+  const size_t n_words = (size_t)N * K / 8;
+  const int threads = 256;
+  expand_plane_kernel<<<(unsigned)((n_words + threads - 1) / threads), threads, 0, (cudaStream_t)stream>>>(
+      reinterpret_cast<const uint8_t*>(compact), n_words, bits, reinterpret_cast<uint32_t*>(plane));
   SM_LAUNCH_CHECK();
   return SLICEMOE_OK;
 }

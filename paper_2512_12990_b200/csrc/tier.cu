@@ -9,7 +9,10 @@
 //   LSB record: gate LSB plane, up LSB plane, down LSB plane
 // and the store holds, for (layer l, expert e), the MSB record followed by the LSB record at
 // (l * n_experts + e) * (msb_record + lsb_record).
-// Every slot of the pool has the size of the larger record (rounded up to 256 bytes), so any slice fits any slot;
+// In the store a plane of a slice narrower than four bits (MAT63, MAT42) is kept dense - the bit stream of
+// slicemoe_compact_plane - so a miss moves 3 or 2 bits per weight, not 4; the copy then lands in a staging buffer
+// and one small kernel on the side stream spreads it into the slot's nibble planes.
+// Every slot of the pool has the size of the larger record in its device form (rounded up to 256 bytes), so any slice fits any slot;
 // slot 0 is never given out: table entries of slices that are not resident point there, so that a list naming
 // an expert the caller did not request reads defined bytes, never an address outside the pool.
 #include <algorithm>
@@ -27,8 +30,33 @@ inline uint64_t tier_key(int layer, int expert) {
 inline size_t round256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
 
 struct MatBytes {
-  size_t plane, scale, zp;
+  size_t plane, scale, zp;  // plane: in the device (nibble) form
 };
+
+// One record from its stored form (in `src`, device staging) to its device form (in a slot): up to three planes as
+// dense bit streams of `bits` bits per value -> nibble planes, and whatever follows each plane copied as it is.
+struct ExpandJob {
+  unsigned long long src_plane[3], dst_plane[3], words[3];  // byte offsets; 32-bit plane words
+  unsigned long long src_meta[3], dst_meta[3], meta_bytes[3];
+  int bits;
+};
+__global__ void tier_expand_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, ExpandJob job) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x, tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const uint32_t mask = (1u << job.bits) - 1u;
+  for (int m = 0; m < 3; ++m) {
+    const uint8_t* in = src + job.src_plane[m];
+    uint32_t* out = reinterpret_cast<uint32_t*>(dst + job.dst_plane[m]);
+    for (size_t i = tid; i < job.words[m]; i += stride) {
+      uint32_t packed = 0;
+      for (int b = 0; b < job.bits; ++b) packed |= (uint32_t)in[i * job.bits + b] << (8 * b);
+      uint32_t w = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) w |= ((packed >> (job.bits * j)) & mask) << (4 * j);
+      out[i] = w;
+    }
+    for (size_t i = tid; i < job.meta_bytes[m]; i += stride) dst[job.dst_meta[m] + i] = src[job.src_meta[m] + i];
+  }
+}
 inline MatBytes mat_bytes(int N, int K, int group) {
   const size_t w = static_cast<size_t>(N) * static_cast<size_t>(K);
   return MatBytes{w / 2, w / static_cast<size_t>(group) * 2, w / static_cast<size_t>(group)};
@@ -36,11 +64,19 @@ inline MatBytes mat_bytes(int N, int K, int group) {
 
 }  // namespace
 
+namespace {
+inline int stored_bits(int width) { return width < 4 ? width : 4; }
+inline size_t stored_plane(size_t plane_bytes, int bits) { return plane_bytes / 4 * bits; }  // plane_bytes = N*K/2
+}  // namespace
+
 struct slicemoe_tier {
   slicemoe_shape shape;
   int n_layers;
   MatBytes gu, dn;           // gate/up [inter, hidden] and down [hidden, inter]
-  size_t msb_rec, lsb_rec, slot_bytes;
+  size_t msb_rec, lsb_rec, slot_bytes;  // records in their device form
+  int msb_bits, lsb_bits;               // stored bits per slice value (4: stored as on the device)
+  size_t msb_rec_st, lsb_rec_st;        // records as stored
+  uint8_t* staging;                     // device; only for stored forms that differ
   const uint8_t* store;      // pinned host
   uint8_t* pool;             // device
   int n_slots;
@@ -66,6 +102,40 @@ struct slicemoe_tier {
       rec += b.plane + b.scale + b.zp;
     }
   }
+  // Brings one record (part 0: MSB, 1: LSB) of store entry `idx` into the slot at `dst`, on stream `xs`.
+  int fetch(size_t idx, int part, uint8_t* dst, cudaStream_t xs) {
+    const size_t rec_st = msb_rec_st + lsb_rec_st;
+    const uint8_t* src = store + idx * rec_st + (part ? msb_rec_st : 0);
+    const size_t bytes = part ? lsb_rec_st : msb_rec_st;
+    const int bits = part ? lsb_bits : msb_bits;
+    if (bits == 4) {  // stored as on the device
+      SM_CUDA_TRY(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, xs));
+    } else {
+      // the staging buffer is free again: whatever used it last ran earlier on this same stream
+      SM_CUDA_TRY(cudaMemcpyAsync(staging, src, bytes, cudaMemcpyHostToDevice, xs));
+      ExpandJob job;
+      job.bits = bits;
+      unsigned long long so = 0, d_o = 0;
+      for (int i = 0; i < 3; ++i) {
+        const MatBytes& b = i < 2 ? gu : dn;
+        job.src_plane[i] = so;
+        job.dst_plane[i] = d_o;
+        job.words[i] = b.plane / 4;
+        so += stored_plane(b.plane, bits);
+        d_o += b.plane;
+        job.src_meta[i] = so;
+        job.dst_meta[i] = d_o;
+        job.meta_bytes[i] = part ? 0 : b.scale + b.zp;
+        so += job.meta_bytes[i];
+        d_o += job.meta_bytes[i];
+      }
+      tier_expand_kernel<<<64, 256, 0, xs>>>(staging, dst, job);
+      SM_LAUNCH_CHECK();
+    }
+    bytes_copied += static_cast<int64_t>(bytes);
+    ++copies;
+    return SLICEMOE_OK;
+  }
   void point_lsb(slicemoe_expert& ex, const uint8_t* rec, bool resident) const {
     slicemoe_mat* m[3] = {&ex.gate, &ex.up, &ex.down};
     for (int i = 0; i < 3; ++i) {
@@ -75,50 +145,69 @@ struct slicemoe_tier {
   }
 };
 
-extern "C" int slicemoe_tier_sizes(const slicemoe_shape* s, size_t* msb_record, size_t* lsb_record, size_t* slot_bytes) {
+
+extern "C" int slicemoe_tier_sizes(const slicemoe_shape* s, size_t* msb_record, size_t* lsb_record, size_t* slot_bytes,
+                                   size_t* staging_bytes) {
   if (!s || s->hidden <= 0 || s->inter <= 0 || (s->hidden % 128) || (s->inter % 128) || !slicemoe::valid_group(s->group))
     return SLICEMOE_E_INVALID_ARG;
+  if (!slicemoe::valid_widths(s->b_high, s->b_low)) return SLICEMOE_E_UNSUPPORTED;
   const MatBytes gu = mat_bytes(s->inter, s->hidden, s->group), dn = mat_bytes(s->hidden, s->inter, s->group);
+  const int mb = stored_bits(s->b_low), lb = stored_bits(s->b_high - s->b_low);
   const size_t m = 2 * (gu.plane + gu.scale + gu.zp) + dn.plane + dn.scale + dn.zp, l = 2 * gu.plane + dn.plane;
-  if (msb_record) *msb_record = m;
-  if (lsb_record) *lsb_record = l;
+  const size_t ms = 2 * (stored_plane(gu.plane, mb) + gu.scale + gu.zp) + stored_plane(dn.plane, mb) + dn.scale + dn.zp;
+  const size_t ls = 2 * stored_plane(gu.plane, lb) + stored_plane(dn.plane, lb);
+  if (msb_record) *msb_record = ms;
+  if (lsb_record) *lsb_record = ls;
   if (slot_bytes) *slot_bytes = round256(std::max(m, l));
+  if (staging_bytes) *staging_bytes = (mb < 4 || lb < 4) ? round256(std::max(ms, ls)) : 0;
   return SLICEMOE_OK;
 }
 
 extern "C" int slicemoe_tier_store_expert(const slicemoe_shape* s, const slicemoe_expert* expert, void* record_host,
-                                          void* stream) {
+                                          void* scratch_device, void* stream) {
   if (!s || !expert || !record_host) return SLICEMOE_E_INVALID_ARG;
-  size_t m = 0, l = 0;
-  const int rc = slicemoe_tier_sizes(s, &m, &l, nullptr);
+  size_t ms = 0, ls = 0, stg = 0;
+  const int rc = slicemoe_tier_sizes(s, &ms, &ls, nullptr, &stg);
   if (rc != SLICEMOE_OK) return rc;
+  if (stg != 0 && !scratch_device) return SLICEMOE_E_INVALID_ARG;
   const MatBytes gu = mat_bytes(s->inter, s->hidden, s->group), dn = mat_bytes(s->hidden, s->inter, s->group);
+  const int bits[2] = {stored_bits(s->b_low), stored_bits(s->b_high - s->b_low)};
   const slicemoe_mat* mats[3] = {&expert->gate, &expert->up, &expert->down};
   uint8_t* p = static_cast<uint8_t*>(record_host);
   cudaStream_t st = (cudaStream_t)stream;
-  for (int i = 0; i < 3; ++i) {
-    const MatBytes& b = i < 2 ? gu : dn;
-    if (!mats[i]->msb || !mats[i]->lsb || !mats[i]->scale || !mats[i]->zp) return SLICEMOE_E_INVALID_ARG;
-    SM_CUDA_TRY(cudaMemcpyAsync(p, mats[i]->msb, b.plane, cudaMemcpyDeviceToHost, st));
-    SM_CUDA_TRY(cudaMemcpyAsync(p + b.plane, mats[i]->scale, b.scale, cudaMemcpyDeviceToHost, st));
-    SM_CUDA_TRY(cudaMemcpyAsync(p + b.plane + b.scale, mats[i]->zp, b.zp, cudaMemcpyDeviceToHost, st));
-    p += b.plane + b.scale + b.zp;
-  }
-  for (int i = 0; i < 3; ++i) {
-    const MatBytes& b = i < 2 ? gu : dn;
-    SM_CUDA_TRY(cudaMemcpyAsync(p, mats[i]->lsb, b.plane, cudaMemcpyDeviceToHost, st));
-    p += b.plane;
+  for (int part = 0; part < 2; ++part) {
+    for (int i = 0; i < 3; ++i) {
+      const MatBytes& b = i < 2 ? gu : dn;
+      const void* plane = part ? mats[i]->lsb : mats[i]->msb;
+      if (!plane || !mats[i]->scale || !mats[i]->zp) return SLICEMOE_E_INVALID_ARG;
+      const size_t sp = stored_plane(b.plane, bits[part]);
+      if (bits[part] < 4) {  // dense form first, in the scratch (the copies and kernels of one stream run in order)
+        const int r2 = slicemoe_compact_plane(plane, mats[i]->N, mats[i]->K, bits[part], scratch_device, stream);
+        if (r2 != SLICEMOE_OK) return r2;
+        SM_CUDA_TRY(cudaMemcpyAsync(p, scratch_device, sp, cudaMemcpyDeviceToHost, st));
+      } else {
+        SM_CUDA_TRY(cudaMemcpyAsync(p, plane, sp, cudaMemcpyDeviceToHost, st));
+      }
+      p += sp;
+      if (part == 0) {
+        SM_CUDA_TRY(cudaMemcpyAsync(p, mats[i]->scale, b.scale, cudaMemcpyDeviceToHost, st));
+        SM_CUDA_TRY(cudaMemcpyAsync(p + b.scale, mats[i]->zp, b.zp, cudaMemcpyDeviceToHost, st));
+        p += b.scale + b.zp;
+      }
+    }
   }
   return SLICEMOE_OK;
 }
 
 extern "C" slicemoe_tier* slicemoe_tier_create(const slicemoe_shape* s, int n_layers, const void* store_host,
                                                void* pool_device, size_t pool_bytes, slicemoe_expert* tables_device,
-                                               double miss_budget, int warmup_steps, void* stream) {
+                                               void* staging_device, size_t staging_bytes, double miss_budget,
+                                               int warmup_steps, void* stream) {
   if (!s || n_layers <= 0 || !store_host || !pool_device || !tables_device || s->n_experts <= 0) return nullptr;
   if (reinterpret_cast<uintptr_t>(pool_device) & 255) return nullptr;
-  size_t m = 0, l = 0, slot = 0;
-  if (slicemoe_tier_sizes(s, &m, &l, &slot) != SLICEMOE_OK) return nullptr;
+  size_t ms = 0, ls = 0, slot = 0, stg = 0;
+  if (slicemoe_tier_sizes(s, &ms, &ls, &slot, &stg) != SLICEMOE_OK) return nullptr;
+  if (stg != 0 && (!staging_device || staging_bytes < stg || (reinterpret_cast<uintptr_t>(staging_device) & 15))) return nullptr;
   const long long n_slots = static_cast<long long>(pool_bytes / slot);
   // slot 0 is the stand-in, 2 * top_k slots are set aside for slices in transit (see `transient`), the cache
   // gets the rest and must be able to hold one request list
@@ -129,8 +218,13 @@ extern "C" slicemoe_tier* slicemoe_tier_create(const slicemoe_shape* s, int n_la
   t->n_layers = n_layers;
   t->gu = mat_bytes(s->inter, s->hidden, s->group);
   t->dn = mat_bytes(s->hidden, s->inter, s->group);
-  t->msb_rec = m;
-  t->lsb_rec = l;
+  t->msb_rec = 2 * (t->gu.plane + t->gu.scale + t->gu.zp) + t->dn.plane + t->dn.scale + t->dn.zp;
+  t->lsb_rec = 2 * t->gu.plane + t->dn.plane;
+  t->msb_bits = stored_bits(s->b_low);
+  t->lsb_bits = stored_bits(s->b_high - s->b_low);
+  t->msb_rec_st = ms;
+  t->lsb_rec_st = ls;
+  t->staging = static_cast<uint8_t*>(staging_device);
   t->slot_bytes = slot;
   t->store = static_cast<const uint8_t*>(store_host);
   t->pool = static_cast<uint8_t*>(pool_device);
@@ -193,7 +287,6 @@ extern "C" int slicemoe_tier_request(slicemoe_tier* t, int step, int layer, cons
   for (int i = 0; i < n; ++i)
     if (ids[i] < 0 || ids[i] >= t->shape.n_experts) return SLICEMOE_E_INVALID_ARG;
   cudaStream_t cs = (cudaStream_t)compute_stream, xs = (cudaStream_t)copy_stream;
-  const size_t rec = t->msb_rec + t->lsb_rec;
   try {
     // Nothing that is still being read may be overwritten: the copies start when the work already enqueued on
     // the compute stream has finished.  (A slice's bytes are needed by the very next launch, whose routing
@@ -243,7 +336,6 @@ extern "C" int slicemoe_tier_request(slicemoe_tier* t, int step, int layer, cons
       if (rc != SLICEMOE_OK) return rc;
       const uint64_t k = tier_key(layer, ids[i]);
       const size_t idx = static_cast<size_t>(layer) * t->shape.n_experts + ids[i];
-      const uint8_t* src = t->store + idx * rec;
       int has_m = 0, has_l = 0;
       slicemoe_dbsc_contains(t->cache, layer, ids[i], &has_m, &has_l);
       for (int part = 0; part < 2; ++part) {  // 0: MSB record (always needed), 1: LSB record (when run at both slices)
@@ -261,10 +353,8 @@ extern "C" int slicemoe_tier_request(slicemoe_tier* t, int step, int layer, cons
         map[k] = slot;
         if (!counted && tr == t->transient.end()) t->transient.emplace_back(k, part);  // used by this launch, not kept
         uint8_t* dst = t->pool + static_cast<size_t>(slot) * t->slot_bytes;
-        const size_t bytes = part ? t->lsb_rec : t->msb_rec;
-        SM_CUDA_TRY(cudaMemcpyAsync(dst, src + (part ? t->msb_rec : 0), bytes, cudaMemcpyHostToDevice, xs));
-        t->bytes_copied += static_cast<int64_t>(bytes);
-        ++t->copies;
+        rc = t->fetch(idx, part, dst, xs);
+        if (rc != SLICEMOE_OK) return rc;
         if (part) t->point_lsb(t->tables[idx], dst, true);
         else t->point_msb(t->tables[idx], dst);
         dirty.push_back(idx);
@@ -285,7 +375,6 @@ extern "C" int slicemoe_tier_request(slicemoe_tier* t, int step, int layer, cons
 extern "C" int slicemoe_tier_sync(slicemoe_tier* t, void* compute_stream, void* copy_stream) {
   if (!t) return SLICEMOE_E_INVALID_ARG;
   cudaStream_t cs = (cudaStream_t)compute_stream, xs = (cudaStream_t)copy_stream;
-  const size_t rec = t->msb_rec + t->lsb_rec;
   try {
     SM_CUDA_TRY(cudaEventRecord(t->ev_compute, cs));
     SM_CUDA_TRY(cudaStreamWaitEvent(xs, t->ev_compute, 0));
@@ -322,10 +411,8 @@ extern "C" int slicemoe_tier_sync(slicemoe_tier* t, void* compute_stream, void* 
               t->free_slots.pop_back();
               map[k] = slot;
               uint8_t* dst = t->pool + static_cast<size_t>(slot) * t->slot_bytes;
-              const size_t bytes = part ? t->lsb_rec : t->msb_rec;
-              SM_CUDA_TRY(cudaMemcpyAsync(dst, t->store + idx * rec + (part ? t->msb_rec : 0), bytes, cudaMemcpyHostToDevice, xs));
-              t->bytes_copied += static_cast<int64_t>(bytes);
-              ++t->copies;
+              const int rc = t->fetch(idx, part, dst, xs);
+              if (rc != SLICEMOE_OK) return rc;
               if (part) t->point_lsb(t->tables[idx], dst, true);
               else t->point_msb(t->tables[idx], dst);
               dirty.push_back(idx);

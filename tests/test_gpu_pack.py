@@ -121,3 +121,29 @@ def test_physical_layout_matches_header():
             es[((n // 16) * ng + gidx) * 16 + n % 16] = o["scale"].view(np.uint16)[n, gidx]
             ez[((n // 16) * ng + gidx) * 16 + n % 16] = o["zp"][n, gidx]
     assert np.array_equal(raw_s, es) and np.array_equal(raw_z, ez)
+
+
+@pytest.mark.parametrize("b_high,b_low", [(4, 2), (6, 3), (8, 4)])
+@pytest.mark.parametrize("N,K", [(16, 128), (48, 384), (1408, 2048)])
+def test_dense_storage_of_narrow_slices(N, K, b_high, b_low):
+    """slicemoe_compact_plane / _expand_plane: the plane's nibbles as the oracle's little-endian bit stream of
+    b_low (MSB slice) and b_high - b_low (LSB slice) bits each, byte for byte, and back."""
+    import torch
+    from paper_2512_12990_b200 import binding as B
+    W = synth.normal_f32(81, ("compact", N, K, b_high), (N, K), 0.02)
+    pm = B.slicemoe_pack(torch.from_numpy(W).cuda(), 64 if K % 64 == 0 else 32, b_high, b_low)
+    for plane, bits in ((pm.msb, b_low), (pm.lsb, b_high - b_low)):
+        raw = plane.cpu().numpy().view(np.uint8).reshape(-1)
+        nibbles = np.empty(raw.size * 2, dtype=np.uint8)
+        nibbles[0::2], nibbles[1::2] = raw & 15, raw >> 4
+        want = amat.compact_stream(nibbles[:8 * 4096], bits) if N * K > 8 * 4096 else amat.compact_stream(nibbles, bits)
+        c = B.slicemoe_compact_plane(plane.view(torch.uint8), N, K, bits)
+        got = c.cpu().numpy()
+        assert got.size == N * K * bits // 8 == B.lib().slicemoe_compact_bytes(N, K, bits)
+        assert np.array_equal(got[:want.size], want)
+        if N * K > 8 * 4096:                      # the oracle is a plain loop: the large plane's tail too, in part
+            tail = amat.compact_stream(nibbles[-8 * 1024:], bits)
+            assert np.array_equal(got[-tail.size:], tail)
+        back = B.slicemoe_expand_plane(c, N, K, bits)
+        torch.cuda.synchronize()
+        assert torch.equal(back, plane.view(torch.uint8).reshape(-1))

@@ -13,17 +13,20 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def test_decode_through_the_tier_matches_the_oracle():
+@pytest.mark.parametrize("b_high,b_low", [(8, 4), (6, 3), (4, 2)])
+def test_decode_through_the_tier_matches_the_oracle(b_high, b_low):
     import torch
     from paper_2512_12990_b200 import binding as B
     NL, N_STEPS, tau = 3, 14, 0.3
     sh = synth.Shape("tier", 256, 128, 8, 2, 64, n_shared=1, shared_inter=256, shared_sigmoid_gate=True, n_layers=NL,
                      seed=5150)
     E, k = sh.n_experts, sh.top_k
-    layers = [H.Layer(sh, range(E), layer=l) for l in range(NL)]
-    m, l_, slot = B.slicemoe_tier_sizes(layers[0].cshape)
+    layers = [H.Layer(sh, range(E), layer=l, b_high=b_high, b_low=b_low) for l in range(NL)]
+    m, l_, slot, staging = B.slicemoe_tier_sizes(layers[0].cshape)
     w = sh.hidden * sh.inter
-    assert m == 3 * (w // 2 + 3 * (w // sh.group)) and l_ == 3 * (w // 2) and slot % 256 == 0 and slot >= m
+    # in the store a slice takes its own width: b_low bits per weight (+ scales and zero-points), b_high - b_low bits
+    assert m == 3 * (w * b_low // 8 + 3 * (w // sh.group)) and l_ == 3 * (w * (b_high - b_low) // 8)
+    assert slot % 256 == 0 and slot >= 3 * (w // 2 + 3 * (w // sh.group)) and (staging == 0) == (b_low == 4)
     pool_slots = 1 + 4 * k + 3                       # 7 cached slots for 48 slices: evictions every step
     tier = B.Tier(layers[0].cshape, [[L.packed[e] for e in range(E)] for L in layers], pool_slots)
     # the originals are no longer needed - and must not be what the kernel reads
@@ -79,8 +82,8 @@ def test_tier_argument_checks():
     import ctypes
     sh = B.make_shape(256, 128, 8, 2, 64)
     L = B.lib()
-    assert L.slicemoe_tier_sizes(None, None, None, None) == B.E_INVALID_ARG
-    assert not L.slicemoe_tier_create(ctypes.byref(sh), 1, None, None, 0, None, -1.0, 10, None)
+    assert L.slicemoe_tier_sizes(None, None, None, None, None) == B.E_INVALID_ARG
+    assert not L.slicemoe_tier_create(ctypes.byref(sh), 1, None, None, 0, None, None, 0, -1.0, 10, None)
     assert L.slicemoe_tier_request(None, 0, 0, None, None, 0, None, None, None) == B.E_INVALID_ARG
     assert L.slicemoe_tier_stats(None, None, None, None) == B.E_INVALID_ARG
     L.slicemoe_tier_destroy(None)
@@ -99,7 +102,7 @@ def test_cache_warmup_reaches_the_tier():
                      seed=5151)
     E, k = sh.n_experts, sh.top_k
     layers = [H.Layer(sh, range(E), layer=l) for l in range(NL)]
-    _, _, slot = B.slicemoe_tier_sizes(layers[0].cshape)
+    _, _, slot, _ = B.slicemoe_tier_sizes(layers[0].cshape)
     pool_slots = 1 + 2 * k + 12                      # 12 cached slots for 48 slices
     tier = B.Tier(layers[0].cshape, [[L.packed[e] for e in range(E)] for L in layers], pool_slots)
     cap = 12 * slot
