@@ -163,7 +163,8 @@ int slicemoe_route_topk(const float *logits, int T, int E, int k, const float *b
  * it cannot know what else occupies the device at launch time.  If other work holds SMs for longer than the
  * wait limit (default: 10^8 clock cycles, about 50 ms), the wait for h ends by itself: the kernel returns,
  * SLICEMOE_STATUS_WAIT_TIMEOUT is set and y is not valid.  Run the decode calls on a device (or a
- * partition of it) that they have to themselves while they run.  After a time-out, initialise the workspace again.
+ * partition of it) that they have to themselves while they run, or pass SLICEMOE_COOPERATIVE to
+ * slicemoe_layer_flags.  After a time-out, initialise the workspace again.
  */
 size_t slicemoe_workspace_bytes(const slicemoe_shape *shape);
 int slicemoe_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
@@ -218,9 +219,14 @@ int slicemoe_layer(const slicemoe_shape *shape, const slicemoe_expert *experts,
  *            The kernel then reads them, and requests the routed experts' slices, while that preceding work is
  *            still running; only x is waited for.  Results are the same bits as slicemoe_layer's.
  * Without the flag the kernel still requests the shared experts' slices early: they follow from the shape alone.
+ *   SLICEMOE_COOPERATIVE  the kernel is launched as a cooperative grid: the driver guarantees that all its CTAs are
+ *            resident together, or fails the launch (SLICEMOE_E_CUDA), so a device shared with other kernels
+ *            cannot make the wait for h run out.  About 1.4 us per launch slower on a B200 (a cooperative grid
+ *            starts as a whole, without the CTA-by-CTA hand-over from the launch before).  Same bits.
  * flags = 0 is slicemoe_layer.  Errors: as slicemoe_layer; INVALID_ARG for an unknown flag.
  */
 #define SLICEMOE_LISTS_RESIDENT 1u
+#define SLICEMOE_COOPERATIVE 2u
 int slicemoe_layer_flags(const slicemoe_shape *shape, const slicemoe_expert *experts,
                          const slicemoe_expert *shared, const float *shared_gate_vec, const void *x, int T,
                          const int32_t *ids, const uint8_t *prec, const float *weights, float *y,

@@ -306,6 +306,7 @@ def slicemoe_expert_ffn(shape: Shape, experts_tbl, x, ids, prec, weights, ws, y=
 
 
 LISTS_RESIDENT = 1
+COOPERATIVE = 2
 
 
 def slicemoe_layer(shape: Shape, experts_tbl, shared_tbl, shared_gate_vec, x, ids, prec, weights, ws, y=None,

@@ -1309,7 +1309,7 @@ static int device_setup(int* dev_out, int* sms_out) {
 }
 
 template <int G, bool FUSED>
-static int launch_decode(const DecodeParams& p, int dev, int sms, int gi, cudaStream_t st) {
+static int launch_decode(const DecodeParams& p, int dev, int sms, int gi, cudaStream_t st, bool cooperative = false) {
   bool& attr_set = g_attr_set[dev][2 * gi + (FUSED ? 1 : 0)];
   if (!attr_set) {
     SM_CUDA_TRY(cudaFuncSetAttribute(decode_layer_kernel<G, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1328,11 +1328,16 @@ static int launch_decode(const DecodeParams& p, int dev, int sms, int gi, cudaSt
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = SmemLayout::total;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see the top of the kernel
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  // On request the driver is asked to guarantee that all CTAs are resident together (they wait for one another's
+  // h values): the launch then fails instead of timing out when the device cannot hold the grid, at the price of
+  // the CTA-by-CTA hand-over between consecutive launches.
+  attr[1].id = cudaLaunchAttributeCooperative;
+  attr[1].val.cooperative = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = cooperative ? 2 : 1;
   SM_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_layer_kernel<G, FUSED>, p));
   return SLICEMOE_OK;
 }
@@ -1370,7 +1375,8 @@ static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts
   if (!experts || !x || !y || !workspace || T <= 0) return SLICEMOE_E_INVALID_ARG;
   if (fused ? !fused->logits : (!ids || !prec || !weights)) return SLICEMOE_E_INVALID_ARG;
   if (fused && shape->n_experts > 32 * ROUTE_MAX_VPT) return SLICEMOE_E_UNSUPPORTED;
-  if ((flags & ~(unsigned)SLICEMOE_LISTS_RESIDENT) != 0u || (fused && flags != 0u)) return SLICEMOE_E_INVALID_ARG;
+  if ((flags & ~(unsigned)(SLICEMOE_LISTS_RESIDENT | SLICEMOE_COOPERATIVE)) != 0u || (fused && flags != 0u)) return SLICEMOE_E_INVALID_ARG;
+  const bool coop = (flags & SLICEMOE_COOPERATIVE) != 0u;
   if (n_shared > 0 && !shared) return SLICEMOE_E_INVALID_ARG;
   if (n_shared > 0 && shape->shared_sigmoid_gate && !gate_vec) return SLICEMOE_E_INVALID_ARG;
   if (workspace_bytes < kWsBytes || (reinterpret_cast<uintptr_t>(workspace) & 255)) return SLICEMOE_E_INVALID_ARG;
@@ -1430,9 +1436,9 @@ static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts
       else if (shape->group == 64) rc = launch_decode<64, true>(p, dev, sms, 1, st);
       else rc = launch_decode<32, true>(p, dev, sms, 2, st);
     } else {
-      if (shape->group == 128) rc = launch_decode<128, false>(p, dev, sms, 0, st);
-      else if (shape->group == 64) rc = launch_decode<64, false>(p, dev, sms, 1, st);
-      else rc = launch_decode<32, false>(p, dev, sms, 2, st);
+      if (shape->group == 128) rc = launch_decode<128, false>(p, dev, sms, 0, st, coop);
+      else if (shape->group == 64) rc = launch_decode<64, false>(p, dev, sms, 1, st, coop);
+      else rc = launch_decode<32, false>(p, dev, sms, 2, st, coop);
     }
     if (rc != SLICEMOE_OK) return rc;
   }

@@ -303,9 +303,16 @@ def test_resident_lists_give_the_same_bits(name):
     assert torch.equal(y0, y1)
     y_ref = moe.layer(x64, L.oracle_list(), ids, prec, w, shared=L.oracle_shared, shared_gate_vec=L.gate_vec)
     H.assert_close(y1.cpu().numpy(), y_ref, f"{name} resident lists")
+    # as a cooperative grid (the driver guarantees co-residency): the same bits again
+    y2 = B.slicemoe_layer(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, *args, L.ws, flags=B.COOPERATIVE)
+    y3 = B.slicemoe_layer(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, *args, L.ws,
+                          flags=B.COOPERATIVE | B.LISTS_RESIDENT)
+    torch.cuda.synchronize()
+    assert B.slicemoe_get_status(L.ws) == 0
+    assert torch.equal(y0, y2) and torch.equal(y0, y3)
     # an unknown flag is refused
     with pytest.raises(B.SliceMoEError):
-        B.slicemoe_layer(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, *args, L.ws, flags=2)
+        B.slicemoe_layer(L.cshape, L.experts_tbl, L.shared_tbl, L.gate_vec_dev, x, *args, L.ws, flags=4)
 
 
 @pytest.mark.parametrize("name", ["tiny", "dsv2", "qwen"])
