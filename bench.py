@@ -851,7 +851,7 @@ def cost_table(B, sh, NL, NS, logits_dev, ids_h, preq_h, cap, msb_b, lsb_b, tau,
     """The paper's hardware cost model (Section 5: DRAM 1.5 pJ/bit at 104 Gbps, Flash 103 pJ/bit at 10 Gbps, XPU
     16.4 TOPS at 3.18 TOPS/W) applied to the decode trace under four cache policies of the same capacity, per token:
     bit-sliced caching with precision on demand, without and with Cache-Prior routing; a conventional cache of whole
-    8-bit experts; the same with Cache-Prior routing (cached experts' logits raised by `delta`; routed again on the device, step by step,
+    8-bit experts; the same with Cache-Prior routing and with Cumsum routing (cached experts' logits raised by `delta`; routed again on the device, step by step,
     because the selection now depends on the cache state); and all experts at the low width."""
     import torch
     E, k = sh.n_experts, sh.top_k
@@ -859,6 +859,10 @@ def cost_table(B, sh, NL, NS, logits_dev, ids_h, preq_h, cap, msb_b, lsb_b, tau,
     shared_macs = sh.n_shared * 3 * sh.hidden * sh.shared_inter
     shared_bytes = sh.n_shared * expert_bytes(sh.hidden, sh.shared_inter, sh.group, True)   # always resident
     full_b = msb_b + lsb_b
+    cumsum_p = 0.6
+    lg = logits_dev.cpu().numpy()
+    ex = np.exp(lg - lg.max(axis=1, keepdims=True))
+    probs_h = (ex / ex.sum(axis=1, keepdims=True)).astype(np.float32)     # the softmax the Cumsum baseline ranks by
 
     def run(policy):
         sliced = policy.startswith("bit_sliced")
@@ -876,6 +880,11 @@ def cost_table(B, sh, NL, NS, logits_dev, ids_h, preq_h, cap, msb_b, lsb_b, tau,
                     bias = torch.from_numpy(c.bias(l, E, delta)).to(dev)
                     sel, _, req = B.slicemoe_route_topk(logits_dev[r:r + 1], k, bias=bias, tau=tau)
                     row, req_row = sel.cpu().numpy()[0], req.cpu().numpy()[0]
+                elif policy.endswith("cumsum"):
+                    # candidates by cumulative gating probability, cached ones first (slicemoe_cumsum_select)
+                    cached = c.bias(l, E, 1.0) > 0
+                    row = B.slicemoe_cumsum_select(probs_h[r], cached, k, cumsum_p)
+                    req_row = np.zeros(k, dtype=np.uint8)
                 else:
                     row, req_row = ids_h[r], preq_h[r]
                 for j in range(k):
@@ -897,12 +906,13 @@ def cost_table(B, sh, NL, NS, logits_dev, ids_h, preq_h, cap, msb_b, lsb_b, tau,
                 "flash_MB_per_token": flash_total / NS / 1e6}
 
     out = {p_: run(p_) for p_ in ("bit_sliced", "bit_sliced_cache_prior", "high_bit_lru", "high_bit_cache_prior",
-                                  "low_bit")}
+                                  "high_bit_cumsum", "low_bit")}
     base, ours = out["high_bit_cache_prior"], out["bit_sliced_cache_prior"]
     out["bit_sliced_cache_prior_vs_high_bit_cache_prior"] = {
         "energy_gain": base["mJ_per_token"] / ours["mJ_per_token"], "speed_up": base["ms_per_token"] / ours["ms_per_token"]}
     out["model"] = ("energy = 8 flash_bytes (103 + 1.5) pJ + 8 dram_bytes 1.5 pJ + 2 macs / 3.18 TOPS/W; latency = "
-                    "flash time + max(DRAM time, compute time), per token; Cache-Prior delta = %g on the logit" % delta)
+                    "flash time + max(DRAM time, compute time), per token; Cache-Prior delta = %g on the logit; Cumsum p = %g"
+                    % (delta, cumsum_p))
     return out
 
 
