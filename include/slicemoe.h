@@ -250,6 +250,15 @@ int slicemoe_layer_routed(const slicemoe_shape *shape, const slicemoe_expert *ex
                           void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * slicemoe_trace_read - time stamps of the decode kernel's most recent launch, for a library built with
+ * -DSLICEMOE_TRACE (python -m paper_2512_12990_b200.build --trace builds libslicemoe_trace.so beside the ordinary
+ * library; python -m paper_2512_12990_b200.trace prints the timeline).  out_host: host array
+ * [min(max_ctas, 256)][*slots_out] of int64: clock64 since the CTA's start at the points the source lists, and the
+ * global timer at three of them.  Synchronises the device.  The ordinary build returns UNSUPPORTED.
+ */
+int slicemoe_trace_read(long long *out_host, int max_ctas, int *slots_out);
+
+/*
  * slicemoe_stream_probe - a measuring stick, not part of the method: brings exactly the bytes that one
  * slicemoe_layer call with T = 1 reads for this list - MSB plane, LSB plane where prec = 1, scales and zero-points
  * of gate, up and down of every listed expert, and of the shared experts at 8 bits - into shared memory with the

@@ -28,7 +28,7 @@ EXPORTS = (
     "slicemoe_strerror", "slicemoe_version", "slicemoe_last_cuda_error", "slicemoe_plane_bytes", "slicemoe_meta_count", "slicemoe_pack",
     "slicemoe_unpack_plane", "slicemoe_unpack_meta", "slicemoe_compact_bytes", "slicemoe_compact_plane", "slicemoe_expand_plane", "slicemoe_route_topk", "slicemoe_workspace_bytes",
     "slicemoe_workspace_init", "slicemoe_workspace_set_wait", "slicemoe_get_status", "slicemoe_expert_ffn", "slicemoe_layer", "slicemoe_layer_flags",
-    "slicemoe_decode_step_host", "slicemoe_stream_probe", "slicemoe_layer_static", "slicemoe_layer_routed", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
+    "slicemoe_decode_step_host", "slicemoe_stream_probe", "slicemoe_trace_read", "slicemoe_layer_static", "slicemoe_layer_routed", "slicemoe_prefill_workspace_bytes", "slicemoe_prefill_layer",
     "slicemoe_dbsc_create", "slicemoe_dbsc_destroy", "slicemoe_dbsc_request",
     "slicemoe_dbsc_assign", "slicemoe_dbsc_stats", "slicemoe_dbsc_contains",
     "slicemoe_dbsc_prefill_layer", "slicemoe_dbsc_prefill_end", "slicemoe_dbsc_bias", "slicemoe_cumsum_select",
@@ -105,6 +105,7 @@ def lib() -> ctypes.CDLL:
                                  c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.slicemoe_layer_flags.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                        c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, ctypes.c_uint, c_void_p]
+    L.slicemoe_trace_read.argtypes = [c_void_p, c_int, POINTER(c_int)]
     L.slicemoe_stream_probe.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
                                         c_void_p]
     L.slicemoe_layer_static.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,

@@ -64,6 +64,36 @@ constexpr int kMaxMine = 32;   // phase-2 chunks one consumer group can have: (s
 // unless the workspace header carries another limit.
 constexpr unsigned long long kWaitCycles = 100000000ull;
 
+// ---- optional time stamps ------------------------------------------------------------------------
+// A build with -DSLICEMOE_TRACE records, per CTA and for the most recent launch, when its roles passed a few
+// points: clock64 relative to the CTA's start (and the global timer at three of them).  slicemoe_trace_read hands
+// the table out; `python -m paper_2512_12990_b200.trace` prints the timeline.  The ordinary build has none of it.
+#ifdef SLICEMOE_TRACE
+constexpr int kTraceSlots = 32;
+__device__ long long g_trace[256][kTraceSlots];
+__shared__ long long s_trace_t0;
+__device__ __forceinline__ long long trace_gtime() {
+  long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define SM_TRACE(i)                                                                   \
+  do {                                                                                \
+    if ((threadIdx.x & 31) == 0 && blockIdx.x < 256) g_trace[blockIdx.x][i] = clock64() - s_trace_t0; \
+  } while (0)
+#define SM_TRACE_G(i)                                                                 \
+  do {                                                                                \
+    if ((threadIdx.x & 31) == 0 && blockIdx.x < 256) g_trace[blockIdx.x][i] = trace_gtime(); \
+  } while (0)
+#else
+#define SM_TRACE(i) do { } while (0)
+#define SM_TRACE_G(i) do { } while (0)
+#endif
+// stamp numbers (clock64 unless noted): 1 dependency wait over, 2 plan built (warp 0), 3 x as digits (warp 3),
+// 4 prologue barrier passed, 5-8 gate/up phase done (consumer groups 0-3), 9 list of down chunks built (warp 0),
+// 10 own h blocks in digits (warp 0), 11 down phase done (warp 0), 12 last h value written, 13 y written;
+// global timer: 20 kernel entry, 21 dependency wait over, 22 y written
+
 // ---- workspace --------------------------------------------------------------------------------
 struct WsHeader {
   unsigned readers;     // CTAs of the running launch that have read `epoch` (the last one moves it on)
@@ -607,6 +637,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
     }
   }
   __syncwarp();
+  if (gw == 0) SM_TRACE(5 + group);
   if (lane == 0) mbar_arrive(bars + 8 * Bars::p1_done);  // this warp no longer reads phase-1 units
   if (plan.count2 == 0) return;
 
@@ -647,11 +678,13 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
     nmine = min(nmine, kMaxMine);  // the host refuses launch shapes that could exceed the list
   }
   __syncwarp();
+  if (warp == 0) SM_TRACE(9);
 
   // ---- the grid's h ----
   if (!fetch_h<G>(p, smem, warp, lane, plan.htotal, p.ws_h + (size_t)plan.hpar * kHCap, plan.never_ready != 0, dead, status,
                   bars))
     return;
+  if (warp == 0) SM_TRACE(10);
 
   // ---- phase 2: chunks round-robin over the groups, all warps contribute to every task ----
   const uint32_t full2 = bars + 8 * Bars::full2, empty2 = bars + 8 * Bars::empty2;
@@ -692,6 +725,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
     __syncwarp();
     if (lane == 0) mbar_arrive(bars + 8 * Bars::pfull2);
   }
+  if (warp == 0) SM_TRACE(11);
 }
 
 // ---- epilogue warp ---------------------------------------------------------------------------------
@@ -736,6 +770,7 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
       tw.next(slots);
     }
   }
+  SM_TRACE(12);
   // phase 2: all warps' partial rows per output row block -> y
   for (int m = 0; m < plan.count2; ++m) {
     if (!mbar_wait(bars + 8 * Bars::pfull2, m & 1, dead, status)) return;
@@ -748,6 +783,8 @@ __device__ void epilogue_loop(const DecodeParams& p, uint8_t* smem, int lane) {
     if (lane == 0) mbar_arrive(bars + 8 * Bars::pempty2);
     if (lane < 16) p.y[(blockIdx.x + m * gridDim.x) * 16 + lane] = b;
   }
+  SM_TRACE(13);
+  SM_TRACE_G(22);
 }
 
 // ---- producer --------------------------------------------------------------------------------------
@@ -1173,6 +1210,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
   // before that wait: x and the workspace always, and the routing lists unless the caller has promised that
   // they were complete earlier (lists_resident).  The weights, the expert tables and the shape are never written
   // by a kernel in flight.
+#ifdef SLICEMOE_TRACE
+  if (tid == 0) s_trace_t0 = clock64();
+  if (tid == 0 && blockIdx.x < 256) g_trace[blockIdx.x][20] = trace_gtime();
+#endif
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const bool early_lists = !FUSED && p.lists_resident != 0;
   if (warp == kProducerWarp) {
@@ -1234,8 +1275,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
     if (lane == 0) mbar_arrive(plan_ready);
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (warp == 3) {
+    SM_TRACE(1);
+    SM_TRACE_G(21);
+  }
   if (warp == 0) {
     if (!early_lists) build_plan<FUSED>(p, smem, lane);
+    SM_TRACE(2);
   } else if (warp == 1) {
     if (!early_lists) load_slot_pointers<FUSED>(p, smem, lane, true);
   } else if (warp == 2) {
@@ -1278,7 +1324,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_layer_kernel(const __grid_
                          reinterpret_cast<float*>(smem + SmemLayout::xinv));
     }
   }
+  if (warp == 3) SM_TRACE(3);
   asm volatile("bar.sync 1, %0;" ::"n"(32 * (kConsumerWarps + 1)) : "memory");
+  if (warp == 3) SM_TRACE(4);
   if (!early_lists && tid == 0) mbar_arrive(plan_ready);
   if (plan->nslots == 0 && blockIdx.x == 0)
     for (int i = tid; i < p.hidden; i += 32 * (kConsumerWarps + 1)) p.y[i] = 0.f;
@@ -1448,6 +1496,21 @@ static int run_layer(const slicemoe_shape* shape, const slicemoe_expert* experts
 }  // namespace slicemoe
 
 using namespace slicemoe;
+
+extern "C" int slicemoe_trace_read(long long* out_host, int max_ctas, int* slots_out) {
+#ifdef SLICEMOE_TRACE
+  if (!out_host || max_ctas <= 0) return SLICEMOE_E_INVALID_ARG;
+  if (slots_out) *slots_out = kTraceSlots;
+  const size_t n = (size_t)(max_ctas < 256 ? max_ctas : 256) * kTraceSlots * sizeof(long long);
+  SM_CUDA_TRY(cudaMemcpyFromSymbol(out_host, g_trace, n));
+  return SLICEMOE_OK;
+#else
+  (void)out_host;
+  (void)max_ctas;
+  (void)slots_out;
+  return SLICEMOE_E_UNSUPPORTED;  // this build carries no time stamps
+#endif
+}
 
 extern "C" size_t slicemoe_workspace_bytes(const slicemoe_shape* shape) {
   (void)shape;

@@ -74,6 +74,7 @@ def test_argument_errors_are_codes_not_faults():
     assert L.slicemoe_layer_flags(ctypes.byref(q), one, one, None, one, 1, one, one, one, one, ws, big, 1, None) == B.E_INVALID_ARG
     assert L.slicemoe_stream_probe(ctypes.byref(q), one, None, one, one, 1, None, None, None) == B.E_INVALID_ARG  # shared missing
     assert L.slicemoe_stream_probe(ctypes.byref(sh), None, None, one, one, 1, None, None, None) == B.E_INVALID_ARG
+    assert L.slicemoe_trace_read(None, 0, None) == B.E_UNSUPPORTED      # the ordinary build carries no time stamps
     assert L.slicemoe_workspace_init(None, big, None) == B.E_INVALID_ARG
     assert L.slicemoe_get_status(None, None, None) == B.E_INVALID_ARG
     assert L.slicemoe_workspace_set_wait(None, 1000, 0, None) == B.E_INVALID_ARG
