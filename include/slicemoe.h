@@ -254,7 +254,8 @@ int slicemoe_layer_routed(const slicemoe_shape *shape, const slicemoe_expert *ex
  * -DSLICEMOE_TRACE (python -m paper_2512_12990_b200.build --trace builds libslicemoe_trace.so beside the ordinary
  * library; python -m paper_2512_12990_b200.trace prints the timeline).  out_host: host array
  * [min(max_ctas, 256)][*slots_out] of int64: clock64 since the CTA's start at the points the source lists, and the
- * global timer at three of them.  Synchronises the device.  The ordinary build returns UNSUPPORTED.
+ * global timer at three of them; *slots_out is at most 256, so 256 * 256 entries always suffice.  Synchronises the
+ * device.  The ordinary build returns UNSUPPORTED.
  */
 int slicemoe_trace_read(long long *out_host, int max_ctas, int *slots_out);
 

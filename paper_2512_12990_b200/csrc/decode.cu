@@ -69,7 +69,7 @@ constexpr unsigned long long kWaitCycles = 100000000ull;
 // points: clock64 relative to the CTA's start (and the global timer at three of them).  slicemoe_trace_read hands
 // the table out; `python -m paper_2512_12990_b200.trace` prints the timeline.  The ordinary build has none of it.
 #ifdef SLICEMOE_TRACE
-constexpr int kTraceSlots = 32;
+constexpr int kTraceSlots = 48;
 __device__ long long g_trace[256][kTraceSlots];
 __shared__ long long s_trace_t0;
 __device__ __forceinline__ long long trace_gtime() {
@@ -92,7 +92,11 @@ __device__ __forceinline__ long long trace_gtime() {
 // stamp numbers (clock64 unless noted): 1 dependency wait over, 2 plan built (warp 0), 3 x as digits (warp 3),
 // 4 prologue barrier passed, 5-8 gate/up phase done (consumer groups 0-3), 9 list of down chunks built (warp 0),
 // 10 own h blocks in digits (warp 0), 11 down phase done (warp 0), 12 last h value written, 13 y written;
-// global timer: 20 kernel entry, 21 dependency wait over, 22 y written
+// 14-17 own h blocks in digits (first warp of consumer groups 0-3), 23-26 the h blocks of the group's last down chunk
+// flagged, 27-30 down phase done (first warp of groups 0-3), 31 producer 0 begins the down tiles, 18-19 producer 0 / 1
+// has requested all its down tiles, 32-39 producer 0 has requested its gate/up chunk 0-7, 40-43 / 44-47 the down
+// chunks of producer 0 / 1 have landed (in the order it waits for them); global timer: 20 kernel entry, 21 dependency
+// wait over, 22 y written
 
 // ---- workspace --------------------------------------------------------------------------------
 struct WsHeader {
@@ -685,6 +689,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
                   bars))
     return;
   if (warp == 0) SM_TRACE(10);
+  if (gw == 0) SM_TRACE(14 + group);
 
   // ---- phase 2: chunks round-robin over the groups, all warps contribute to every task ----
   const uint32_t full2 = bars + 8 * Bars::full2, empty2 = bars + 8 * Bars::empty2;
@@ -706,6 +711,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
       const bool p8 = (d.z & 256u) != 0u;
       if (!mbar_wait(full2 + 8 * (kFull2PerGroup * group + ((d.y >> 16) & 0xffu)), d.y >> 24, dead, status)) return;
       if (!wait_h_blocks(smem, col >> 7, nblocks, lane, dead, status)) return;  // this chunk's part of h, no more
+      if (gw == 0 && i == nmine - 1) SM_TRACE(23 + group);
       const uint8_t* dig = smem + SmemLayout::hdig + col * 3;
       const float* sumw = reinterpret_cast<const float*>(smem + SmemLayout::hsumw) + (col >> LG) * 2;
       const float* binv = reinterpret_cast<const float*>(smem + SmemLayout::hinv) + (col >> 7);
@@ -726,6 +732,7 @@ __device__ void consumer_loop(const DecodeParams& p, uint8_t* smem, int warp, in
     if (lane == 0) mbar_arrive(bars + 8 * Bars::pfull2);
   }
   if (warp == 0) SM_TRACE(11);
+  if (gw == 0) SM_TRACE(27 + group);
 }
 
 // ---- epilogue warp ---------------------------------------------------------------------------------
@@ -934,6 +941,7 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
           ++igg;
           ok = produce_chunk<G>(smem, r1, cs, lane, pl, s, mat, s.prec ? mat : 1, s.prec ? kModeBoth : kModePair, p.hidden,
                                 idx, (q % nch) * kChunkK, pw, pol);
+          if (which == 0 && lane == 0 && jp < 8) SM_TRACE(32 + jp);
         }
       }
       tw.next(slots);
@@ -947,6 +955,7 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
   // The re-cut units lie over the phase-1 units: nothing of phase 2 lands before phase 1 has been consumed.
   // (From then until h has crossed the grid the memory system has nothing else to do.)
   if (ok && plan.count2 > 0) ok = pw(bars + 8 * Bars::p1_done, 0);
+  if (which == 0 && lane == 0 && plan.count2 > 0) SM_TRACE(31);
   const int half = plan.nunits2 / kProducers;  // this warp's units are [which * half, which * half + half)
   int c2 = 0, xp = 0;                           // chunks of the phase so far, units this warp has handed out
   for (int m = 0; m < plan.count2 && ok; ++m) {
@@ -971,6 +980,10 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
       }
     }
   }
+  if (lane == 0 && plan.count2 > 0) SM_TRACE(18 + which);
+#ifdef SLICEMOE_TRACE
+  int landed = 0;
+#endif
   // Never leave the CTA with bulk copies still landing in its shared memory: wait (bounded) until every
   // barrier this warp may have armed has completed its last phase.  In the normal path they have long ago.
   for (int g = which; g < kGroups; g += kProducers) {
@@ -987,6 +1000,10 @@ __device__ void producer_loop(const DecodeParams& p, uint8_t* smem, int lane, in
       while (!mbar_try(bars + 8 * (Bars::full2 + kFull2PerGroup * g + i % kFull2PerGroup), (i / kFull2PerGroup) & 1)) {
         if (*dead || (unsigned long long)(clock64() - t0) > wait_limit(dead)) break;
       }
+#ifdef SLICEMOE_TRACE
+      if (lane == 0 && landed < 4) SM_TRACE(40 + 4 * which + landed);
+      ++landed;
+#endif
     }
   }
 }
