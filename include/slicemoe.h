@@ -344,6 +344,7 @@ int slicemoe_decode_step_host(const slicemoe_shape *shape, const slicemoe_expert
  * (token, expert) pair gets its own fp32 result row and y[t] sums them in list order (routed
  * slots 0..k-1, then the shared experts), so y is bit-reproducible run to run.
  *   x            device bf16 [T, hidden]
+ *   shared_gate_vec  as for slicemoe_layer; 8-byte aligned
  *   ids, weights device [T, k] (int32, float32)
  *   expert_prec  device uint8 [n_experts]: 1 = both slices, 0 = MSB slice only.  Precision is per
  *                expert, not per (token, slot): all tokens of an expert share its weight tile.

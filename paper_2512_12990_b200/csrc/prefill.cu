@@ -71,31 +71,51 @@ __global__ void pf_count_kernel(const int32_t* __restrict__ ids, int n, int E, i
   atomicAdd(&counts[e], 1);
 }
 
-// One CTA: padded offsets of every expert (routed, then shared with T rows each) and the tile list.
+// One warp: padded offsets of every expert (routed, then shared with T rows each) and the tile list.  Lane l takes
+// the experts l, l + 32, ...; warp scans turn the experts' tile and item counts into each tile's place in the lists.
 __global__ void pf_scan_kernel(const int* __restrict__ counts, int E, int n_shared, int T, int inter, int shared_inter,
                                int* __restrict__ offsets, int* __restrict__ tile_expert, int* __restrict__ tile_row0,
                                int* __restrict__ item_start, int* __restrict__ ntiles) {
-  if (threadIdx.x != 0) return;
-  int off = 0, nt = 0, items = 0, nt_routed = 0;
-  for (int e = 0; e < E + n_shared; ++e) {
-    if (e == E) nt_routed = nt;
-    const int c = e < E ? counts[e] : T;
-    offsets[e] = off;
-    for (int r = 0; r < c; r += kPfTileM) {
-      tile_expert[nt] = e;
-      tile_row0[nt] = off + r;
-      item_start[nt] = items;
-      items += (e < E ? inter : shared_inter) / 64;  // first GEMM: 64 columns of h per work item
-      ++nt;
+  const int lane = threadIdx.x & 31;
+  if (threadIdx.x >= 32) return;
+  const int n = E + n_shared;
+  int nt = 0, items = 0, nt_routed = 0;  // tiles / first-GEMM work items / routed experts' tiles so far
+  for (int e0 = 0; e0 < n; e0 += 32) {
+    const int e = e0 + lane;
+    const int c = e < n ? (e < E ? counts[e] : T) : 0;
+    const int tiles = (c + kPfTileM - 1) / kPfTileM;
+    const int per = (e < E ? inter : shared_inter) / 64;  // first GEMM: 64 columns of h per work item
+    int tin = tiles, iin = tiles * per;                    // inclusive scans
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int a = __shfl_up_sync(0xffffffffu, tin, off), b = __shfl_up_sync(0xffffffffu, iin, off);
+      if (lane >= off) {
+        tin += a;
+        iin += b;
+      }
     }
-    off += (c + kPfTileM - 1) / kPfTileM * kPfTileM;
+    const int routed = __reduce_add_sync(0xffffffffu, e < E ? tiles : 0);
+    if (e < n) {
+      const int first = nt + tin - tiles;  // the expert's first tile; rows are padded to whole tiles
+      offsets[e] = first * kPfTileM;
+      for (int r = 0; r < tiles; ++r) {
+        tile_expert[first + r] = e;
+        tile_row0[first + r] = (first + r) * kPfTileM;
+        item_start[first + r] = items + iin - tiles * per + r * per;
+      }
+    }
+    nt += __shfl_sync(0xffffffffu, tin, 31);
+    items += __shfl_sync(0xffffffffu, iin, 31);
+    nt_routed += routed;
   }
-  offsets[E + n_shared] = off;
-  item_start[nt] = items;
-  ntiles[0] = nt;
-  ntiles[1] = off;
-  ntiles[2] = items;
-  ntiles[3] = n_shared > 0 ? nt_routed : nt;  // tiles of routed experts: they come first and have inter / 64 items each
+  if (lane == 0) {
+    offsets[n] = nt * kPfTileM;
+    item_start[nt] = items;
+    ntiles[0] = nt;
+    ntiles[1] = nt * kPfTileM;
+    ntiles[2] = items;
+    ntiles[3] = n_shared > 0 ? nt_routed : nt;  // tiles of routed experts: they come first and have inter / 64 items each
+  }
 }
 
 // Every (token, slot) pair takes a row of its expert; shared experts take row t.  Which row a pair gets
@@ -119,8 +139,12 @@ __global__ void pf_scatter_kernel(const int32_t* __restrict__ ids, int T, int k,
 }
 
 // ---- step 2: gather x into expert order, bf16 -> fp16; padding rows are zero ----------------------------
+// With a gated shared expert the rows of the first shared expert - one per token - also give the token's gate
+// sigmoid(gate_vec . x): the row is being read anyway.  `shared_row0` points at the first shared expert's offset.
 __global__ void pf_gather_kernel(const uint16_t* __restrict__ x, int hidden, const int* __restrict__ row_token,
-                                 const int* __restrict__ ntiles, __half* __restrict__ xs) {
+                                 const int* __restrict__ ntiles, __half* __restrict__ xs,
+                                 const float* __restrict__ gate_vec, const int* __restrict__ shared_row0, int T,
+                                 float* __restrict__ gate) {
   const int row = blockIdx.x;
   if (row >= ntiles[1]) return;
   const int t = row_token[row];
@@ -129,10 +153,30 @@ __global__ void pf_gather_kernel(const uint16_t* __restrict__ x, int hidden, con
     for (int i = threadIdx.x; i < hidden / 2; i += blockDim.x) dst[i] = __floats2half2_rn(0.f, 0.f);
     return;
   }
+  const bool gated = gate_vec != nullptr && row >= shared_row0[0] && row < shared_row0[0] + T;
   const uint32_t* src = reinterpret_cast<const uint32_t*>(x + (size_t)t * hidden);
+  float dot = 0.f;
   for (int i = threadIdx.x; i < hidden / 2; i += blockDim.x) {
     const uint32_t raw = src[i];
-    dst[i] = __floats2half2_rn(__uint_as_float(raw << 16), __uint_as_float(raw & 0xffff0000u));
+    const float lo = __uint_as_float(raw << 16), hi = __uint_as_float(raw & 0xffff0000u);
+    dst[i] = __floats2half2_rn(lo, hi);
+    if (gated) {
+      const float2 gv = *reinterpret_cast<const float2*>(gate_vec + 2 * i);
+      dot = fmaf(gv.x, lo, dot);
+      dot = fmaf(gv.y, hi, dot);
+    }
+  }
+  if (gated) {  // block sum in a fixed order: lanes by butterfly, then the warps one after the other
+    __shared__ float part[32];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = dot;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float sum = 0.f;
+      for (int w = 0; w < (int)(blockDim.x >> 5); ++w) sum += part[w];
+      gate[t] = 1.f / (1.f + expf(-sum));
+    }
   }
 }
 
@@ -667,18 +711,6 @@ __global__ void __launch_bounds__(kUThreads, 1) pf_umma_kernel(const PfGemmParam
 }
 
 // ---- step 5: weighted combine in list order ---------------------------------------------------------------
-__global__ void pf_gate_kernel(const uint16_t* __restrict__ x, const float* __restrict__ gate_vec, int T, int hidden,
-                               float* __restrict__ gate) {
-  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  if (t >= T) return;
-  float dot = 0.f;
-  for (int i = lane; i < hidden; i += 32)
-    dot = fmaf(gate_vec[i], __uint_as_float((uint32_t)x[(size_t)t * hidden + i] << 16), dot);
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
-  if (lane == 0) gate[t] = 1.f / (1.f + expf(-dot));
-}
-
 __global__ void pf_combine_kernel(const float* __restrict__ yrow, const int* __restrict__ posmap,
                                   const float* __restrict__ weights, const float* __restrict__ gate, int T, int k,
                                   int n_shared, int hidden, float* __restrict__ y) {
@@ -787,6 +819,8 @@ extern "C" int slicemoe_prefill_layer(const slicemoe_shape* s, const slicemoe_ex
   const PfLayout L = pf_layout(T, E, k, nsh, s->hidden, s->inter, shared_inter);
   if (workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(workspace) & 255)) return SLICEMOE_E_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(x) & 3) || (reinterpret_cast<uintptr_t>(y) & 15)) return SLICEMOE_E_INVALID_ARG;
+  if (s->n_shared > 0 && s->shared_sigmoid_gate && (reinterpret_cast<uintptr_t>(shared_gate_vec) & 7))
+    return SLICEMOE_E_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   int* counts = reinterpret_cast<int*>(ws + L.counts);
@@ -815,13 +849,10 @@ extern "C" int slicemoe_prefill_layer(const slicemoe_shape* s, const slicemoe_ex
   const int nslots = T * (k + nsh);
   pf_scatter_kernel<<<(nslots + 255) / 256, 256, 0, st>>>(ids, T, k, E, nsh, offsets, cursor, row_token, posmap);
   SM_LAUNCH_CHECK();
-  pf_gather_kernel<<<L.rmax, 256, 0, st>>>(reinterpret_cast<const uint16_t*>(x), s->hidden, row_token, ntiles, xs);
-  SM_LAUNCH_CHECK();
   const bool gated = nsh > 0 && s->shared_sigmoid_gate;
-  if (gated) {
-    pf_gate_kernel<<<(T + 7) / 8, 256, 0, st>>>(reinterpret_cast<const uint16_t*>(x), shared_gate_vec, T, s->hidden, gate);
-    SM_LAUNCH_CHECK();
-  }
+  pf_gather_kernel<<<L.rmax, 256, 0, st>>>(reinterpret_cast<const uint16_t*>(x), s->hidden, row_token, ntiles, xs,
+                                           gated ? shared_gate_vec : nullptr, offsets + E, T, gate);
+  SM_LAUNCH_CHECK();
   PfGemmParams p;
   p.experts = experts;
   p.shared = shared;
